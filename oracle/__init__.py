@@ -1,0 +1,263 @@
+"""Python face of the CPU oracle (test infrastructure, never a product path).
+
+Loads ``liboracle.so`` (plain C, built from ``oracle.c`` with gcc) and strings
+its per-step functions together in the order the paper gives them: sample a hop,
+build the frontier, transpose the block; then per layer the mean aggregation
+(Sec. 3.1, Eq. 2) and the update (Eq. 3); then the adjoints in reverse order.
+All floating-point arrays are float64.  Nothing here imports the CUDA package.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SO = os.path.join(_HERE, "liboracle.so")
+_SRC = os.path.join(_HERE, "oracle.c")
+
+
+def build(force: bool = False) -> str:
+    """Compile oracle.c into liboracle.so (gcc -O2, strict IEEE arithmetic)."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-ffp-contract=off",
+                               "-o", _SO, _SRC, "-lm"])
+    return _SO
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.oracle_round_bf16.restype = C.c_double
+        _lib.oracle_round_bf16.argtypes = [C.c_double]
+        _lib.oracle_sample_hop.restype = C.c_int64
+        _lib.oracle_relabel.restype = C.c_int32
+        _lib.oracle_csr_from_coo.restype = C.c_int
+        _lib.oracle_bce_with_logits.restype = C.c_double
+    return _lib
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _f64(a):
+    return np.ascontiguousarray(a, dtype=np.float64)
+
+
+def _i32(a):
+    return np.ascontiguousarray(a, dtype=np.int32)
+
+
+def _i64(a):
+    return np.ascontiguousarray(a, dtype=np.int64)
+
+
+# ----------------------------------------------------------------------------- basics
+
+def round_bf16(a):
+    a = _f64(a).copy()
+    lib().oracle_round_bf16_array(_p(a), C.c_int64(a.size))
+    return a
+
+
+def philox4x32_10(ctr, key):
+    c = np.asarray(ctr, dtype=np.uint32)
+    k = np.asarray(key, dtype=np.uint32)
+    out = np.zeros(4, np.uint32)
+    lib().oracle_philox4x32_10(_p(c), _p(k), _p(out))
+    return out
+
+
+def csr_from_coo(n, row, col):
+    row, col = _i32(row), _i32(col)
+    m = row.size
+    indptr = np.zeros(n + 1, np.int64)
+    indices = np.zeros(m, np.int32)
+    rc = lib().oracle_csr_from_coo(C.c_int64(n), C.c_int64(m), _p(row), _p(col), _p(indptr), _p(indices))
+    if rc != 0:
+        raise ValueError("node id out of range")
+    return indptr, indices
+
+
+def csr_transpose(n_rows, n_cols, indptr, indices):
+    indptr, indices = _i64(indptr), _i32(indices)
+    m = int(indptr[n_rows])
+    csc_ptr = np.zeros(n_cols + 1, np.int64)
+    csc_row = np.zeros(m, np.int32)
+    csc_eid = np.zeros(m, np.int64)
+    lib().oracle_csr_transpose(C.c_int64(n_rows), C.c_int64(n_cols), _p(indptr), _p(indices),
+                               _p(csc_ptr), _p(csc_row), _p(csc_eid))
+    return csc_ptr, csc_row, csc_eid
+
+
+# ----------------------------------------------------------------------------- sampling
+
+def sample_khop(indptr, indices, seeds, fanouts, seed, step):
+    """k-hop sampled blocks (Sec. 4.1 subgraph construction; Sec. 3.1 multiset S_l(u)).
+
+    Hop h (1-based) samples for every node of D_h = F_{h-1} (F_0 = the seeds) with
+    fanouts[h-1]; returns one dict per hop with the block CSR (indptr, col,
+    nbr_global), the frontier src_nodes = F_h, the transposed block and 1/|S|.
+    """
+    indptr, indices = _i64(indptr), _i32(indices)
+    n = indptr.size - 1
+    dst = _i32(seeds)
+    blocks = []
+    for h, f in enumerate(fanouts, start=1):
+        n_dst = dst.size
+        cap = max(1, n_dst * int(f))
+        blk_indptr = np.zeros(n_dst + 1, np.int32)
+        nbr = np.zeros(cap, np.int32)
+        ne = lib().oracle_sample_hop(_p(indptr), _p(indices), _p(dst), C.c_int32(n_dst), C.c_int32(int(f)),
+                                     C.c_uint64(int(seed)), C.c_uint32(int(step)), C.c_int32(h),
+                                     _p(blk_indptr), _p(nbr))
+        nbr = nbr[:ne].copy()
+        src = np.zeros(n_dst + ne, np.int32)
+        col = np.zeros(max(ne, 1), np.int32)
+        n_src = lib().oracle_relabel(C.c_int64(n), _p(dst), C.c_int32(n_dst), _p(nbr), C.c_int64(ne),
+                                     _p(src), _p(col))
+        if n_src < 0:
+            raise ValueError("seed id out of range")
+        src = src[:n_src].copy()
+        col = col[:ne].copy()
+        csc_ptr = np.zeros(n_src + 1, np.int32)
+        csc_row = np.zeros(max(ne, 1), np.int32)
+        csc_eid = np.zeros(max(ne, 1), np.int32)
+        inv_cnt = np.zeros(max(n_dst, 1), np.float32)
+        lib().oracle_block_csc(C.c_int32(n_dst), C.c_int32(n_src), _p(blk_indptr), _p(col),
+                               _p(csc_ptr), _p(csc_row), _p(csc_eid), _p(inv_cnt))
+        blocks.append(dict(n_dst=n_dst, n_src=n_src, n_edges=int(ne), indptr=blk_indptr, col=col,
+                           nbr_global=nbr, src_nodes=src, csc_ptr=csc_ptr, csc_row=csc_row[:ne].copy(),
+                           csc_eid=csc_eid[:ne].copy(), inv_cnt=inv_cnt[:n_dst].copy()))
+        dst = src
+    return blocks
+
+
+# ----------------------------------------------------------------------------- GraphSAGE
+
+def mean_aggregate(indptr, col, H, bf16=False):
+    """Eq. 2 over a block (or a whole CSR): one mean row per destination."""
+    indptr, col, H = _i64(indptr), _i32(col), _f64(H)
+    n_dst, d = indptr.size - 1, H.shape[1]
+    agg = np.zeros((n_dst, d), np.float64)
+    lib().oracle_mean_aggregate(_p(indptr), _p(col), C.c_int64(n_dst), _p(H), C.c_int32(d), _p(agg),
+                                C.c_int(int(bf16)))
+    return agg
+
+
+def sage_update(Hself, agg, W, bias, act, bf16=False):
+    """Eq. 3: sigma(W [h || agg] (+ b)).  Returns (Z pre-activation, H)."""
+    Hself, agg, W = _f64(Hself), _f64(agg), _f64(W)
+    n_dst, d_in = Hself.shape
+    d_out = W.shape[0]
+    assert W.shape[1] == 2 * d_in
+    b = None if bias is None else _f64(bias)
+    Z = np.zeros((n_dst, d_out), np.float64)
+    Hout = np.zeros((n_dst, d_out), np.float64)
+    lib().oracle_sage_update(_p(Hself), _p(agg), C.c_int64(n_dst), C.c_int32(d_in), _p(W), _p(b),
+                             C.c_int32(d_out), C.c_int(int(act)), _p(Z), _p(Hout), C.c_int(int(bf16)))
+    return Z, Hout
+
+
+def sage_forward(blocks, X, Ws, biases=None, acts=None, bf16=False):
+    """L-layer forward on sampled blocks.  Layer l runs on block L-l; layer 0 reads X rows of F_L."""
+    L = len(Ws)
+    acts = [1] * L if acts is None else list(acts)
+    biases = [None] * L if biases is None else list(biases)
+    X = _f64(X)
+    ids = _i32(blocks[L - 1]["src_nodes"])
+    H = np.zeros((ids.size, X.shape[1]), np.float64)
+    lib().oracle_gather_rows(_p(X), C.c_int64(X.shape[1]), _p(ids), C.c_int64(ids.size),
+                             C.c_int32(X.shape[1]), _p(H))
+    ctx = dict(H=[H], agg=[], Z=[])
+    for l in range(L):
+        blk = blocks[L - 1 - l]
+        H = ctx["H"][l]
+        agg = mean_aggregate(blk["indptr"], blk["col"], H, bf16)
+        Z, Hn = sage_update(H[: blk["n_dst"]], agg, Ws[l], biases[l], acts[l], bf16)
+        ctx["agg"].append(agg)
+        ctx["Z"].append(Z)
+        ctx["H"].append(Hn)
+    return ctx["H"][L], ctx
+
+
+def sage_backward(blocks, ctx, Ws, dH_out, acts=None, bf16=False, with_bias=False):
+    """Adjoint of sage_forward: returns (dWs, dbs, dX_rows) with dX_rows aligned to F_L."""
+    L = len(Ws)
+    acts = [1] * L if acts is None else list(acts)
+    dH = _f64(dH_out)
+    dWs, dbs = [None] * L, [None] * L
+    for l in range(L - 1, -1, -1):
+        blk = blocks[L - 1 - l]
+        W = _f64(Ws[l])
+        d_out, d_in = W.shape[0], W.shape[1] // 2
+        n_dst, n_src = blk["n_dst"], blk["n_src"]
+        Hl = _f64(ctx["H"][l])
+        Hself = np.ascontiguousarray(Hl[:n_dst])
+        agg, Hout = _f64(ctx["agg"][l]), _f64(ctx["H"][l + 1])
+        dW = np.zeros_like(W)
+        db = np.zeros(d_out, np.float64)
+        dSelf = np.zeros((n_dst, d_in), np.float64)
+        dAgg = np.zeros((n_dst, d_in), np.float64)
+        dH = _f64(dH)
+        lib().oracle_sage_update_backward(_p(dH), _p(Hout), _p(Hself), _p(agg), _p(W), C.c_int64(n_dst),
+                                          C.c_int32(d_in), C.c_int32(d_out), C.c_int(int(acts[l])),
+                                          _p(dW), _p(db) if with_bias else None, _p(dSelf), _p(dAgg))
+        dHl = np.zeros((n_src, d_in), np.float64)
+        ip = _i64(blk["indptr"])
+        cl = _i32(blk["col"])
+        lib().oracle_mean_aggregate_backward(_p(ip), _p(cl), C.c_int64(n_dst), C.c_int64(n_src),
+                                             _p(dSelf), _p(dAgg), C.c_int32(d_in), _p(dHl), C.c_int(int(bf16)))
+        dWs[l], dbs[l] = dW, db
+        dH = dHl
+    return dWs, dbs, dH
+
+
+# ----------------------------------------------------------------------------- tower + loss
+
+def dense_forward(Xin, W, b, act, bf16=False):
+    Xin, W = _f64(Xin), _f64(W)
+    n, d_in = Xin.shape
+    d_out = W.shape[0]
+    bb = None if b is None else _f64(b)
+    Y = np.zeros((n, d_out), np.float64)
+    lib().oracle_dense_forward(_p(Xin), C.c_int64(n), C.c_int32(d_in), _p(W), _p(bb), C.c_int32(d_out),
+                               C.c_int(int(act)), _p(Y), C.c_int(int(bf16)))
+    return Y
+
+
+def dense_backward(dY, Y, Xin, W, act, bf16=False):
+    dY, Y, Xin, W = _f64(dY), _f64(Y), _f64(Xin), _f64(W)
+    n, d_in = Xin.shape
+    d_out = W.shape[0]
+    dW = np.zeros_like(W)
+    db = np.zeros(d_out, np.float64)
+    dX = np.zeros((n, d_in), np.float64)
+    lib().oracle_dense_backward(_p(dY), _p(Y), _p(Xin), _p(W), C.c_int64(n), C.c_int32(d_in), C.c_int32(d_out),
+                                C.c_int(int(act)), _p(dW), _p(db), _p(dX), C.c_int(int(bf16)))
+    return dW, db, dX
+
+
+def bce_with_logits(t, y):
+    t, y = _f64(t).ravel(), _f64(y).ravel()
+    dt = np.zeros_like(t)
+    loss = lib().oracle_bce_with_logits(_p(t), _p(y), C.c_int64(t.size), _p(dt))
+    return float(loss), dt
+
+
+# ----------------------------------------------------------------------------- full graph
+
+def full_aggregate_backward(indptr, indices, n_src, G, bf16=False):
+    indptr, indices, G = _i64(indptr), _i32(indices), _f64(G)
+    n_dst, d = indptr.size - 1, G.shape[1]
+    dX = np.zeros((n_src, d), np.float64)
+    lib().oracle_full_aggregate_backward(_p(indptr), _p(indices), C.c_int64(n_dst), C.c_int64(n_src),
+                                         _p(G), C.c_int32(d), _p(dX), C.c_int(int(bf16)))
+    return dX
