@@ -1,0 +1,187 @@
+/*
+ * e2egrec.h -- C ABI of the sampled-GNN training pass of E2E-GRec (arXiv 2511.20564)
+ * for one NVIDIA B200 (sm_100a).
+ *
+ * The library runs, per training step, what the paper's Figure 1 pipeline does for
+ * the GNN branch: build the sampled multi-hop subgraph of the batch (Sec. 4.1), run
+ * the GraphSAGE encoder on it (Sec. 3.1, Eqs. 2-3), and send the gradient that the
+ * recommendation model returns back through the encoder to its weights and to the
+ * input node features (Sec. 4.3.2, gradient of L_total w.r.t. the GNN parameters).
+ *
+ * Conventions shared by every entry point
+ * ---------------------------------------
+ *  - Every pointer marked "device" is memory of the current CUDA device, allocated
+ *    and owned by the caller; the library allocates no device memory and frees none.
+ *    Pointers marked "host" are ordinary host memory read during the call only.
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All work
+ *    is enqueued on it; no entry point synchronises with the device, so results are
+ *    valid once the stream reaches the end of the enqueued work.
+ *  - Sizes that depend on the data (how many distinct nodes a hop reaches) stay on the
+ *    device: each block carries `counts` = {n_dst, n_src, n_edges, status}; buffers are
+ *    sized for the worst case reported by the *_workspace / size-query calls.
+ *  - Return value: E2EGREC_OK (0) or a negative E2EGREC_ERR_* code for errors detected
+ *    on the host before anything is enqueued.  Errors that only the device can see (a
+ *    seed id out of range, a capacity overrun) set bits of counts[3] of the block (or of
+ *    the status word named by the call) and the offending element is skipped; nothing
+ *    traps, asserts or spins without a bound.
+ *  - Node ids are int32 (n_nodes < 2^31), graph offsets int64, block offsets int32.
+ *  - Feature matrices are row-major; dtype E2EGREC_F32 or E2EGREC_BF16; every row must
+ *    start on a 16-byte boundary (dim * element size and ld * element size multiples of 16).
+ *  - Size queries: where a call takes `void* buf, size_t* bytes`, calling it with
+ *    buf == NULL writes the required size to *bytes and returns E2EGREC_OK without
+ *    enqueuing anything; otherwise *bytes is the size provided and must be >= required.
+ */
+#ifndef E2EGREC_H
+#define E2EGREC_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define E2EGREC_OK               0
+#define E2EGREC_ERR_NULL        -1   /* a required pointer is NULL */
+#define E2EGREC_ERR_ARG         -2   /* a size or count is out of its documented range */
+#define E2EGREC_ERR_DTYPE       -3   /* unknown dtype, or operands of one call disagree */
+#define E2EGREC_ERR_ALIGN       -4   /* a row does not start on a 16-byte boundary */
+#define E2EGREC_ERR_WORKSPACE   -5   /* buffer smaller than the size query reports */
+#define E2EGREC_ERR_UNSUPPORTED -6   /* n_nodes >= 2^31, more than 4 hops, fanout > 128, dim > 1024 */
+#define E2EGREC_ERR_CUDA        -7   /* a launch failed; e2egrec_last_error() holds the CUDA text */
+
+/* bits of the device status word (counts[3]) */
+#define E2EGREC_DEV_RANGE     1u     /* a seed / node id was outside [0, n_nodes) and was skipped */
+#define E2EGREC_DEV_CAPACITY  2u     /* a buffer capacity would have been exceeded; output truncated */
+#define E2EGREC_DEV_TIMEOUT   4u     /* a bounded wait inside a kernel ran out */
+
+#define E2EGREC_F32  0
+#define E2EGREC_BF16 1
+
+/* flags of e2egrec_sage_backward */
+#define E2EGREC_ACCUMULATE_DW 1u     /* add to dW / dbias instead of overwriting them */
+
+/* Graph G=(V,E) in compressed sparse row form (Sec. 3, Notation): row u lists N(u),
+ * parallel edges kept.  indptr: device int64[n_nodes+1]; indices: device int32[n_edges].
+ * edge_weight is reserved for the weighted sampler (omega_uv of Sec. 4.1) and must be NULL. */
+typedef struct e2egrec_csr {
+    int64_t        n_nodes;
+    int64_t        n_edges;
+    const int64_t *indptr;
+    const int32_t *indices;
+    const float   *edge_weight;
+} e2egrec_csr;
+
+/* Row-major matrix on the device: `rows` x `dim`, leading dimension `ld` elements. */
+typedef struct e2egrec_mat {
+    void   *data;
+    int64_t rows;
+    int32_t dim;
+    int64_t ld;
+    int32_t dtype;
+} e2egrec_mat;
+
+/* One sampled hop ("block"): the bipartite graph from the frontier F_h (sources) to the
+ * nodes D_h = F_{h-1} that were sampled for (destinations).  All arrays are device
+ * memory of the stated capacity, provided by the caller:
+ *   counts     int32[4]            {n_dst, n_src, n_edges, status bits}
+ *   indptr     int32[cap_dst+1]    block CSR offsets, destination i owns [indptr[i], indptr[i+1])
+ *   col        int32[cap_edges]    local source id (position in src_nodes) of each entry
+ *   nbr_global int32[cap_edges]    global node id of each entry
+ *   src_nodes  int32[cap_src]      F_h: the destinations first (same order), then the newly
+ *                                  reached nodes in ascending id order
+ *   csc_ptr    int32[cap_src+1]    transposed block: source s owns [csc_ptr[s], csc_ptr[s+1])
+ *   csc_row    int32[cap_edges]    destination of each transposed entry
+ *   csc_eid    int32[cap_edges]    its position in the block CSR; ascending inside a column
+ *   inv_cnt    float[cap_dst]      1/|S(u)| per destination, 0 for an isolated node */
+typedef struct e2egrec_block {
+    int32_t  cap_dst, cap_src, cap_edges;
+    int32_t *counts;
+    int32_t *indptr, *col, *nbr_global, *src_nodes;
+    int32_t *csc_ptr, *csc_row, *csc_eid;
+    float   *inv_cnt;
+} e2egrec_block;
+
+/* Static text for a status code / the CUDA error text of the last E2EGREC_ERR_CUDA
+ * returned on this thread ("" if none). */
+const char *e2egrec_status_string(int32_t code);
+const char *e2egrec_last_error(void);
+
+/* Worst-case capacities of the blocks of a k-hop sample and the scratch size
+ * (Sec. 4.1: depth L, at most k neighbours per node).  fanouts: host int32[n_hops],
+ * fanouts[0] is the hop taken from the seeds.  cap_dst / cap_src / cap_edges: host
+ * int32[n_hops] outputs.  Limits: 1 <= n_hops <= 4, 1 <= fanout <= 128, n_nodes < 2^31. */
+int32_t e2egrec_sample_khop_workspace(int64_t n_nodes, int32_t n_seeds, int32_t n_hops,
+                                      const int32_t *fanouts, int32_t *cap_dst, int32_t *cap_src,
+                                      int32_t *cap_edges, size_t *scratch_bytes);
+
+/* Puts a sampler scratch buffer (device, scratch_bytes from the query above, 256-byte
+ * aligned) into its idle state.  Call once after allocating it; e2egrec_sample_khop
+ * leaves the buffer idle again when it finishes, so one buffer serves every step. */
+int32_t e2egrec_sampler_scratch_init(int64_t n_nodes, void *scratch, size_t scratch_bytes, void *stream);
+
+/* k-hop neighbour sampling (Sec. 3.1: multiset S_l(u) of N(u); Sec. 4.1: sampling
+ * probability with beta = 0, i.e. uniform over the stored entries of the row, at most
+ * fanout neighbours per node, depth n_hops).
+ *   seeds  device int32[n_seeds], distinct node ids (the batch's source nodes).
+ *   Hop h = 1..n_hops samples for every node of D_h = F_{h-1} (F_0 = seeds):
+ *     deg <= fanout: all stored neighbours once, in CSR order;
+ *     deg  > fanout: fanout independent uniform draws with replacement.  Draw j of node u
+ *       uses Philox4x32-10 with key = (seed low, seed high) and counter
+ *       (j/2, u, (1<<8)|h, step); output words 2(j%2), 2(j%2)+1 form a 64-bit r and the
+ *       entry picked is floor(r * deg / 2^64).  The lists are therefore a function of
+ *       (seed, step, h, u) only and reproducible bit for bit.
+ *   blocks host array[n_hops] of structs holding device pointers; blocks[h-1] receives hop h
+ *       including its transposed form.  F_h = D_h followed by the new nodes in ascending order.
+ *   scratch device buffer initialised by e2egrec_sampler_scratch_init for the same n_nodes. */
+int32_t e2egrec_sample_khop(const e2egrec_csr *graph, const int32_t *seeds, int32_t n_seeds,
+                            int32_t n_hops, const int32_t *fanouts, uint64_t seed, uint32_t step,
+                            uint32_t flags, const e2egrec_block *blocks,
+                            void *scratch, size_t scratch_bytes, void *stream);
+
+/* GraphSAGE forward over sampled blocks (Sec. 3.1): for layer l = 0..n_layers-1, on block
+ * h = n_layers - l,
+ *     agg_i = (1/|S(i)|) sum_{v in S(i)} h_v                         (Eq. 2; 0 if S(i) is empty)
+ *     h'_i  = act( W_l [h_i || agg_i] + b_l )                        (Eq. 3; act = ReLU or identity)
+ * Layer 0 reads h = X[src_nodes] of the outermost block directly (the h^(0) lookup).
+ *   X      features of all nodes, rows >= n_nodes.
+ *   W      host array[n_layers]; W[l] is device [d_out x 2*d_in] row-major, same dtype as X;
+ *          its first d_in columns multiply h_i, the rest multiply agg_i.
+ *   bias   host array[n_layers] of device float[d_out] pointers, or NULL, or NULL entries.
+ *   act    host int32[n_layers]: 1 = ReLU, 0 = identity.
+ *   ctx    device buffer that keeps [h_i || agg_i] and h' of every layer for the backward pass
+ *          (size query: ctx == NULL).  ctx_bytes in/out as described above.
+ *   H_out  device [cap_dst(block 0) x d_L]: rows [0, n_seeds) receive the final embeddings.
+ * bf16 operands are multiplied on the tensor cores with fp32 accumulation; fp32 operands use
+ * fp32 FMA.  The mean is accumulated in fp32 and stored in the feature dtype. */
+int32_t e2egrec_sage_forward(const e2egrec_block *blocks, int32_t n_layers, const e2egrec_mat *X,
+                             const e2egrec_mat *W, const float *const *bias, const int32_t *act,
+                             void *ctx, size_t *ctx_bytes, const e2egrec_mat *H_out, void *stream);
+
+/* Where e2egrec_sage_forward keeps its activations inside ctx (for callers that want the
+ * intermediate embeddings, Sec. 3.1 H^(l)): for layer l, cat_offset[l] is the byte offset of
+ * [h_i || agg_i], a row-major [rows[l] x 2*d_in] matrix, and h_offset[l] that of the layer output
+ * h', [rows[l] x d_out]; rows[l] is the destination capacity of the layer's block rounded up to a
+ * multiple of 128; only the first n_dst rows are meaningful.  All three are host arrays[n_layers]. */
+int32_t e2egrec_sage_ctx_layout(const e2egrec_block *blocks, int32_t n_layers, const e2egrec_mat *X,
+                                const e2egrec_mat *W, size_t *cat_offset, size_t *h_offset, int64_t *rows);
+
+/* Backward of e2egrec_sage_forward (Sec. 4.3.2: the GNN receives J^T times the gradient at
+ * its output; chain of Sec. 4.2).  dH_out: gradient w.r.t. H_out, same shape and dtype.
+ *   dW     host array[n_layers] of device float[d_out x 2*d_in]   (always fp32)
+ *   dbias  host array[n_layers] of device float[d_out], or NULL / NULL entries to skip
+ *   dX_rows device [cap_src(outermost block) x d_0], feature dtype: gradient w.r.t. the rows
+ *          X[src_nodes[i]]; row i belongs to node blocks[n_layers-1].src_nodes[i] (distinct ids).
+ *   scratch device buffer (size query: scratch == NULL).
+ * The transposed aggregation runs as a gather over the block's csc arrays: no floating-point
+ * atomics, results are bit-identical from run to run. */
+int32_t e2egrec_sage_backward(const e2egrec_block *blocks, int32_t n_layers, const e2egrec_mat *X,
+                              const e2egrec_mat *W, const int32_t *act, const void *ctx,
+                              const e2egrec_mat *dH_out, float *const *dW, float *const *dbias,
+                              const e2egrec_mat *dX_rows, void *scratch, size_t *scratch_bytes,
+                              uint32_t flags, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* E2EGREC_H */

@@ -188,8 +188,10 @@ def sage_forward(blocks, X, Ws, biases=None, acts=None, bf16=False):
     return ctx["H"][L], ctx
 
 
-def sage_backward(blocks, ctx, Ws, dH_out, acts=None, bf16=False, with_bias=False):
-    """Adjoint of sage_forward: returns (dWs, dbs, dX_rows) with dX_rows aligned to F_L."""
+def sage_backward(blocks, ctx, Ws, dH_out, acts=None, bf16=False, with_bias=False, trace=None):
+    """Adjoint of sage_forward: returns (dWs, dbs, dX_rows) with dX_rows aligned to F_L.
+
+    If `trace` is a list it receives, per layer l, the gradient that arrived at that layer's output."""
     L = len(Ws)
     acts = [1] * L if acts is None else list(acts)
     dH = _f64(dH_out)
@@ -207,6 +209,8 @@ def sage_backward(blocks, ctx, Ws, dH_out, acts=None, bf16=False, with_bias=Fals
         dSelf = np.zeros((n_dst, d_in), np.float64)
         dAgg = np.zeros((n_dst, d_in), np.float64)
         dH = _f64(dH)
+        if trace is not None:
+            trace.insert(0, dH.copy())
         lib().oracle_sage_update_backward(_p(dH), _p(Hout), _p(Hself), _p(agg), _p(W), C.c_int64(n_dst),
                                           C.c_int32(d_in), C.c_int32(d_out), C.c_int(int(acts[l])),
                                           _p(dW), _p(db) if with_bias else None, _p(dSelf), _p(dAgg))

@@ -1,0 +1,9 @@
+"""B200 (sm_100a) kernels for the sampled-GNN training pass of E2E-GRec, behind a C ABI.
+
+``binding`` mirrors the entry points of ``include/e2egrec.h`` one to one; it only
+marshals arguments (torch tensors supply device memory and the stream).
+"""
+from .binding import (  # noqa: F401
+    BF16, F32, Blocks, E2EGrecError, lib, sample_khop, sample_khop_workspace, sampler_scratch_init,
+    sage_backward, sage_ctx_views, sage_forward, status_string,
+)

@@ -1,0 +1,270 @@
+"""ctypes binding of libe2egrec.so: argument marshalling only.
+
+Every computation happens inside the library's CUDA kernels.  There is no CPU or
+PyTorch fallback: if the shared library is missing or a call fails, an exception
+is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SO = os.path.join(_HERE, "libe2egrec.so")
+
+F32, BF16 = 0, 1
+ACCUMULATE_DW = 1
+_DTYPES = {torch.float32: F32, torch.bfloat16: BF16}
+
+
+class E2EGrecError(RuntimeError):
+    pass
+
+
+class Csr(C.Structure):
+    _fields_ = [("n_nodes", C.c_int64), ("n_edges", C.c_int64), ("indptr", C.c_void_p),
+                ("indices", C.c_void_p), ("edge_weight", C.c_void_p)]
+
+
+class Mat(C.Structure):
+    _fields_ = [("data", C.c_void_p), ("rows", C.c_int64), ("dim", C.c_int32), ("ld", C.c_int64),
+                ("dtype", C.c_int32)]
+
+
+class Block(C.Structure):
+    _fields_ = [("cap_dst", C.c_int32), ("cap_src", C.c_int32), ("cap_edges", C.c_int32),
+                ("counts", C.c_void_p), ("indptr", C.c_void_p), ("col", C.c_void_p),
+                ("nbr_global", C.c_void_p), ("src_nodes", C.c_void_p), ("csc_ptr", C.c_void_p),
+                ("csc_row", C.c_void_p), ("csc_eid", C.c_void_p), ("inv_cnt", C.c_void_p)]
+
+
+_lib = None
+
+
+def lib():
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_SO):
+            raise E2EGrecError(f"{_SO} is missing: run `python -m paper_2511_20564_b200.build` "
+                               "(there is no fallback path)")
+        L = C.CDLL(_SO)
+        L.e2egrec_status_string.restype = C.c_char_p
+        L.e2egrec_status_string.argtypes = [C.c_int32]
+        L.e2egrec_last_error.restype = C.c_char_p
+        L.e2egrec_sample_khop_workspace.restype = C.c_int32
+        L.e2egrec_sample_khop_workspace.argtypes = [C.c_int64, C.c_int32, C.c_int32, C.c_void_p, C.c_void_p,
+                                                    C.c_void_p, C.c_void_p, C.POINTER(C.c_size_t)]
+        L.e2egrec_sampler_scratch_init.restype = C.c_int32
+        L.e2egrec_sampler_scratch_init.argtypes = [C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.e2egrec_sample_khop.restype = C.c_int32
+        L.e2egrec_sample_khop.argtypes = [C.POINTER(Csr), C.c_void_p, C.c_int32, C.c_int32, C.c_void_p,
+                                          C.c_uint64, C.c_uint32, C.c_uint32, C.POINTER(Block), C.c_void_p,
+                                          C.c_size_t, C.c_void_p]
+        L.e2egrec_sage_forward.restype = C.c_int32
+        L.e2egrec_sage_forward.argtypes = [C.POINTER(Block), C.c_int32, C.POINTER(Mat), C.POINTER(Mat),
+                                           C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_size_t),
+                                           C.POINTER(Mat), C.c_void_p]
+        L.e2egrec_sage_backward.restype = C.c_int32
+        L.e2egrec_sage_backward.argtypes = [C.POINTER(Block), C.c_int32, C.POINTER(Mat), C.POINTER(Mat),
+                                            C.c_void_p, C.c_void_p, C.POINTER(Mat), C.c_void_p, C.c_void_p,
+                                            C.POINTER(Mat), C.c_void_p, C.POINTER(C.c_size_t), C.c_uint32,
+                                            C.c_void_p]
+        L.e2egrec_sage_ctx_layout.restype = C.c_int32
+        L.e2egrec_sage_ctx_layout.argtypes = [C.POINTER(Block), C.c_int32, C.POINTER(Mat), C.POINTER(Mat),
+                                              C.c_void_p, C.c_void_p, C.c_void_p]
+        _lib = L
+    return _lib
+
+
+def status_string(code: int) -> str:
+    return lib().e2egrec_status_string(code).decode()
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        extra = lib().e2egrec_last_error().decode() if rc == -7 else ""
+        raise E2EGrecError(f"{what}: {status_string(rc)} ({rc}) {extra}".strip())
+
+
+def _stream(stream=None):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _ptr(t):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _mat(t: torch.Tensor) -> Mat:
+    assert t.dim() == 2 and t.stride(1) == 1
+    return Mat(t.data_ptr(), t.shape[0], t.shape[1], t.stride(0), _DTYPES[t.dtype])
+
+
+def _i32_host(values):
+    return (C.c_int32 * len(values))(*[int(v) for v in values])
+
+
+def _dev_bytes(n: int, device):
+    """256-byte aligned device buffer of at least n bytes (torch's allocator aligns to 512)."""
+    return torch.empty(max(int(n), 256), dtype=torch.uint8, device=device)
+
+
+# ------------------------------------------------------------------------------------------ sampling
+
+def sample_khop_workspace(n_nodes: int, n_seeds: int, fanouts):
+    """-> (cap_dst[], cap_src[], cap_edges[], scratch_bytes)"""
+    L = len(fanouts)
+    f = _i32_host(fanouts)
+    cd, cs, ce = (C.c_int32 * L)(), (C.c_int32 * L)(), (C.c_int32 * L)()
+    nbytes = C.c_size_t(0)
+    _check(lib().e2egrec_sample_khop_workspace(n_nodes, n_seeds, L, f, cd, cs, ce, C.byref(nbytes)),
+           "e2egrec_sample_khop_workspace")
+    return list(cd), list(cs), list(ce), nbytes.value
+
+
+class Blocks:
+    """Device buffers for the blocks of one k-hop sample, sized for the worst case."""
+
+    def __init__(self, n_nodes: int, n_seeds: int, fanouts, device="cuda"):
+        self.fanouts = [int(f) for f in fanouts]
+        self.n_nodes, self.n_seeds = int(n_nodes), int(n_seeds)
+        cd, cs, ce, self.scratch_bytes = sample_khop_workspace(n_nodes, n_seeds, self.fanouts)
+        self.caps = list(zip(cd, cs, ce))
+        self.t = []
+        i32 = dict(dtype=torch.int32, device=device)
+        for d, s, e in self.caps:
+            self.t.append(dict(
+                counts=torch.zeros(4, **i32), indptr=torch.zeros(d + 1, **i32), col=torch.zeros(max(e, 1), **i32),
+                nbr_global=torch.zeros(max(e, 1), **i32), src_nodes=torch.zeros(max(s, 1), **i32),
+                csc_ptr=torch.zeros(s + 1, **i32), csc_row=torch.zeros(max(e, 1), **i32),
+                csc_eid=torch.zeros(max(e, 1), **i32),
+                inv_cnt=torch.zeros(max(d, 1), dtype=torch.float32, device=device)))
+        self.c = (Block * len(self.caps))()
+        for h, ((d, s, e), t) in enumerate(zip(self.caps, self.t)):
+            self.c[h] = Block(d, s, e, *[t[k].data_ptr() for k in
+                                         ("counts", "indptr", "col", "nbr_global", "src_nodes", "csc_ptr",
+                                          "csc_row", "csc_eid", "inv_cnt")])
+        self.scratch = _dev_bytes(self.scratch_bytes, device)
+        sampler_scratch_init(n_nodes, self.scratch)
+
+    def __len__(self):
+        return len(self.caps)
+
+    def to_host(self):
+        """Copies the blocks back, trimmed to their true sizes (synchronises)."""
+        out = []
+        for t in self.t:
+            n_dst, n_src, n_edges, status = t["counts"].tolist()
+            out.append(dict(n_dst=n_dst, n_src=n_src, n_edges=n_edges, status=status,
+                            indptr=t["indptr"][: n_dst + 1].cpu().numpy(), col=t["col"][:n_edges].cpu().numpy(),
+                            nbr_global=t["nbr_global"][:n_edges].cpu().numpy(),
+                            src_nodes=t["src_nodes"][:n_src].cpu().numpy(),
+                            csc_ptr=t["csc_ptr"][: n_src + 1].cpu().numpy(),
+                            csc_row=t["csc_row"][:n_edges].cpu().numpy(),
+                            csc_eid=t["csc_eid"][:n_edges].cpu().numpy(),
+                            inv_cnt=t["inv_cnt"][:n_dst].cpu().numpy()))
+        return out
+
+
+def sampler_scratch_init(n_nodes: int, scratch: torch.Tensor, stream=None):
+    _check(lib().e2egrec_sampler_scratch_init(n_nodes, _ptr(scratch), scratch.numel(), _stream(stream)),
+           "e2egrec_sampler_scratch_init")
+
+
+def sample_khop(indptr: torch.Tensor, indices: torch.Tensor, seeds: torch.Tensor, blocks: Blocks, seed: int,
+                step: int, stream=None):
+    """Enqueues the k-hop sample of `seeds` into `blocks` (see e2egrec_sample_khop)."""
+    assert indptr.dtype == torch.int64 and indices.dtype == torch.int32 and seeds.dtype == torch.int32
+    g = Csr(indptr.numel() - 1, indices.numel(), indptr.data_ptr(), indices.data_ptr(), None)
+    f = _i32_host(blocks.fanouts)
+    _check(lib().e2egrec_sample_khop(C.byref(g), _ptr(seeds), seeds.numel(), len(blocks), f,
+                                     C.c_uint64(seed), C.c_uint32(step), 0, blocks.c, _ptr(blocks.scratch),
+                                     blocks.scratch.numel(), _stream(stream)), "e2egrec_sample_khop")
+
+
+# ------------------------------------------------------------------------------------------ GraphSAGE
+
+def _mats(ts):
+    arr = (Mat * len(ts))()
+    for i, t in enumerate(ts):
+        arr[i] = _mat(t)
+    return arr
+
+
+def _ptr_array(ts, n):
+    if ts is None:
+        return None
+    arr = (C.c_void_p * n)()
+    for i, t in enumerate(ts):
+        arr[i] = None if t is None else t.data_ptr()
+    return arr
+
+
+def sage_forward_ctx_bytes(blocks: Blocks, X, Ws) -> int:
+    n = C.c_size_t(0)
+    x, w = _mat(X), _mats(Ws)
+    _check(lib().e2egrec_sage_forward(blocks.c, len(Ws), C.byref(x), w, None, None, None, C.byref(n), None, None),
+           "e2egrec_sage_forward(size query)")
+    return n.value
+
+
+def sage_forward(blocks: Blocks, X, Ws, biases=None, acts=None, ctx=None, H_out=None, stream=None):
+    """Enqueues the forward pass; returns (H_out, ctx).  ctx / H_out are allocated when not given."""
+    L = len(Ws)
+    if ctx is None:
+        ctx = _dev_bytes(sage_forward_ctx_bytes(blocks, X, Ws), X.device)
+    if H_out is None:
+        H_out = torch.zeros(max(blocks.caps[0][0], 1), Ws[-1].shape[0], dtype=X.dtype, device=X.device)
+    x, w, ho = _mat(X), _mats(Ws), _mat(H_out)
+    n = C.c_size_t(ctx.numel())
+    a = None if acts is None else _i32_host(acts)
+    _check(lib().e2egrec_sage_forward(blocks.c, L, C.byref(x), w, _ptr_array(biases, L), a, _ptr(ctx), C.byref(n),
+                                      C.byref(ho), _stream(stream)), "e2egrec_sage_forward")
+    return H_out, ctx
+
+
+def sage_ctx_views(blocks: Blocks, X, Ws, ctx):
+    """Views into ctx: per layer (cat [rows x 2 d_in], h_out [rows x d_out]); see e2egrec_sage_ctx_layout."""
+    L = len(Ws)
+    co, ho, rows = (C.c_size_t * L)(), (C.c_size_t * L)(), (C.c_int64 * L)()
+    x, w = _mat(X), _mats(Ws)
+    _check(lib().e2egrec_sage_ctx_layout(blocks.c, L, C.byref(x), w, co, ho, rows), "e2egrec_sage_ctx_layout")
+    es = X.element_size()
+    out = []
+    for l, W in enumerate(Ws):
+        r, d_out, k = rows[l], W.shape[0], W.shape[1]
+        cat = ctx[co[l]: co[l] + r * k * es].view(X.dtype).view(r, k)
+        h = ctx[ho[l]: ho[l] + r * d_out * es].view(X.dtype).view(r, d_out)
+        out.append((cat, h))
+    return out
+
+
+def sage_backward_scratch_bytes(blocks: Blocks, X, Ws) -> int:
+    n = C.c_size_t(0)
+    x, w = _mat(X), _mats(Ws)
+    _check(lib().e2egrec_sage_backward(blocks.c, len(Ws), C.byref(x), w, None, None, None, None, None, None, None,
+                                       C.byref(n), 0, None), "e2egrec_sage_backward(size query)")
+    return n.value
+
+
+def sage_backward(blocks: Blocks, X, Ws, ctx, dH_out, acts=None, dWs=None, dbs=None, dX_rows=None, scratch=None,
+                  accumulate=False, stream=None):
+    """Enqueues the backward pass; returns (dWs, dX_rows).  Buffers are allocated when not given."""
+    L = len(Ws)
+    dev = X.device
+    if scratch is None:
+        scratch = _dev_bytes(sage_backward_scratch_bytes(blocks, X, Ws), dev)
+    if dWs is None:
+        dWs = [torch.zeros(W.shape, dtype=torch.float32, device=dev) for W in Ws]
+    if dX_rows is None:
+        dX_rows = torch.zeros(max(blocks.caps[L - 1][1], 1), X.shape[1], dtype=X.dtype, device=dev)
+    x, w, dh, dx = _mat(X), _mats(Ws), _mat(dH_out), _mat(dX_rows)
+    n = C.c_size_t(scratch.numel())
+    a = None if acts is None else _i32_host(acts)
+    _check(lib().e2egrec_sage_backward(blocks.c, L, C.byref(x), w, a, _ptr(ctx), C.byref(dh), _ptr_array(dWs, L),
+                                       _ptr_array(dbs, L), C.byref(dx), _ptr(scratch), C.byref(n),
+                                       ACCUMULATE_DW if accumulate else 0, _stream(stream)), "e2egrec_sage_backward")
+    return dWs, dX_rows

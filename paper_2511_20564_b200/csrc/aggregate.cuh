@@ -1,0 +1,333 @@
+// Row-gather reductions: the neighbourhood mean (Eq. 2) over a sampled block, and the
+// general "segment s = sum of gathered rows" kernel used by the transposed aggregation
+// (gather over the block's CSC) and by whole-graph aggregation with hub rows.
+//
+// A row of d values is d*sizeof(T)/16 chunks of 16 bytes.  LPR lanes (a power of two) own
+// one row at a time, lane c of the group holding chunks c, c+LPR, ... (CPL of them), so a
+// warp works on 32/LPR gathered rows at once and every lane issues several independent
+// 16-byte loads before it adds anything.  Sums are fp32; nothing uses floating-point atomics.
+#pragma once
+
+#include "common.cuh"
+
+namespace e2egrec {
+
+constexpr int kAggThreads = 256;
+
+// ---------------------------------------------------------------------------------------
+// Sampled-block mean aggregation, one warp per destination (|S(i)| <= 128).
+// Writes cat[i] = [ self row | mean row ] (2d values) for i < n_dst and zero rows up to
+// the next multiple of 128 (the dense transform reads whole 128-row tiles).
+// ---------------------------------------------------------------------------------------
+template <typename T, int LPR, int CPL>
+__global__ void __launch_bounds__(kAggThreads)
+sage_aggregate_kernel(const T *__restrict__ Hsrc, int64_t ld, const int32_t *__restrict__ nbr,
+                      const int32_t *__restrict__ self_ids, const int32_t *__restrict__ indptr,
+                      const int32_t *__restrict__ counts, T *__restrict__ cat, int d, int32_t cap_dst)
+{
+    constexpr int E = Chunk<T>::kElems;
+    constexpr int G = 32 / LPR;
+    constexpr int U = CPL >= 4 ? 1 : 4 / CPL;
+    const int lane = threadIdx.x & 31;
+    const int g = lane / LPR, c = lane % LPR;
+    const int n_chunks = d / E;
+    const int32_t n_dst = counts[CNT_DST];
+    int64_t pad_end = ((int64_t)n_dst + 127) / 128 * 128;
+    if (pad_end > cap_dst) pad_end = cap_dst;
+    const int64_t i = ((int64_t)blockIdx.x * kAggThreads + threadIdx.x) >> 5;
+    if (i >= pad_end) return;
+    T *out = cat + i * 2 * d;
+    if (i >= n_dst) {
+        float z[E];
+#pragma unroll
+        for (int k = 0; k < E; ++k) z[k] = 0.f;
+        for (int q = lane; q < 2 * n_chunks; q += 32) Chunk<T>::store(out + q * E, z);
+        return;
+    }
+    // self half: plain 16-byte copies
+    const int64_t self_row = self_ids ? (int64_t)self_ids[i] : i;
+    for (int q = lane; q < n_chunks; q += 32)
+        *reinterpret_cast<uint4 *>(out + q * E) = __ldg(reinterpret_cast<const uint4 *>(Hsrc + self_row * ld + q * E));
+
+    float acc[CPL][E];
+#pragma unroll
+    for (int q = 0; q < CPL; ++q)
+#pragma unroll
+        for (int k = 0; k < E; ++k) acc[q][k] = 0.f;
+
+    const int32_t beg = indptr[i], end = indptr[i + 1];
+    for (int32_t base = beg; base < end; base += 32) {
+        const int m = min(32, end - base);
+        const int32_t mine = lane < m ? nbr[base + lane] : 0;
+        for (int t = 0; t * G < m; t += U) {
+            float v[U][CPL][E];
+            bool ok[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int j = (t + u) * G + g;
+                ok[u] = j < m;
+                const int32_t id = __shfl_sync(0xffffffffu, mine, j & 31);
+                const T *row = Hsrc + (int64_t)id * ld;
+#pragma unroll
+                for (int q = 0; q < CPL; ++q) {
+                    const int ch = c + q * LPR;
+                    if (ok[u] && ch < n_chunks) Chunk<T>::load(row + ch * E, v[u][q]);
+                }
+            }
+#pragma unroll
+            for (int u = 0; u < U; ++u)
+#pragma unroll
+                for (int q = 0; q < CPL; ++q)
+                    if (ok[u] && c + q * LPR < n_chunks)
+#pragma unroll
+                        for (int k = 0; k < E; ++k) acc[q][k] += v[u][q][k];
+        }
+    }
+#pragma unroll
+    for (int off = LPR; off < 32; off <<= 1)
+#pragma unroll
+        for (int q = 0; q < CPL; ++q)
+#pragma unroll
+            for (int k = 0; k < E; ++k) acc[q][k] += __shfl_xor_sync(0xffffffffu, acc[q][k], off);
+    if (g == 0) {
+        const int32_t cnt = end - beg;
+        const float inv = cnt > 0 ? 1.0f / (float)cnt : 0.0f;
+#pragma unroll
+        for (int q = 0; q < CPL; ++q) {
+            const int ch = c + q * LPR;
+            if (ch < n_chunks) {
+#pragma unroll
+                for (int k = 0; k < E; ++k) acc[q][k] *= inv;
+                Chunk<T>::store(out + d + ch * E, acc[q]);
+            }
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------
+// General segment reduction   out[s] = fin( sum_{k in [ptr[s], ptr[s+1])} w[idx[k]] * in[idx[k]] )
+// with  fin(x) = mask_s * ( x * (mean ? 1/len : 1) + self[s] ).
+//
+// Work is cut into chunks of `chunk_len` consecutive entries, one warp each, so a hub
+// segment with millions of entries is shared by many warps.  A segment that lies inside
+// one chunk is finished there.  Otherwise the chunk in which it starts stores its part in
+// tail[chunk], every later chunk stores its part in head[chunk], and the finishing kernel
+// adds tail[first] + head[first+1] + ... + head[last] in that fixed order.
+// ---------------------------------------------------------------------------------------
+template <typename T>
+struct SegOut {
+    T *out;                 // [n_seg x d], leading dimension ld_out
+    int64_t ld_out;
+    const T *self;          // optional rows added for s < *n_self
+    int64_t ld_self;
+    const int32_t *n_self;
+    const T *mask;          // optional: result is zeroed where mask[s][k] <= 0 (ReLU derivative)
+    int64_t ld_mask;
+    int mean;               // divide the sum by the segment length
+};
+
+template <typename T>
+__device__ inline float seg_finish_value(const SegOut<T> &o, int64_t s, int64_t len, int k, float sum, bool has_self)
+{
+    float v = o.mean ? (len > 0 ? sum * (1.0f / (float)len) : 0.f) : sum;
+    if (has_self) v += to_float<T>(o.self[s * o.ld_self + k]);
+    v = to_float<T>(from_float<T>(v));                      // storage rounding before the mask
+    if (o.mask && !(to_float<T>(o.mask[s * o.ld_mask + k]) > 0.f)) v = 0.f;
+    return v;
+}
+
+template <typename PtrT>
+__device__ inline int64_t seg_containing(const PtrT *__restrict__ ptr, int64_t n_seg, int64_t k)
+{
+    // largest s in [0, n_seg) with ptr[s] <= k   (k < ptr[n_seg])
+    int64_t lo = 0, hi = n_seg;
+    while (hi - lo > 1) {
+        const int64_t mid = (lo + hi) >> 1;
+        if ((int64_t)ptr[mid] <= k) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+template <typename T, typename PtrT, int LPR, int CPL, bool kWeight>
+__global__ void __launch_bounds__(kAggThreads)
+seg_chunk_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__ ptr,
+                 const int32_t *__restrict__ idx, const int32_t *n_seg_dev, int64_t n_seg_host,
+                 const float *__restrict__ w, int chunk_len, int d, float *__restrict__ head,
+                 float *__restrict__ tail, SegOut<T> o)
+{
+    constexpr int E = Chunk<T>::kElems;
+    constexpr int G = 32 / LPR;
+    constexpr int U = CPL >= 4 ? 1 : 4 / CPL;
+    const int lane = threadIdx.x & 31;
+    const int g = lane / LPR, c = lane % LPR;
+    const int n_chunks = d / E;
+    const int64_t n_seg = n_seg_dev ? (int64_t)*n_seg_dev : n_seg_host;
+    if (n_seg <= 0) return;
+    const int64_t total = (int64_t)ptr[n_seg];
+    const int64_t chunk = ((int64_t)blockIdx.x * kAggThreads + threadIdx.x) >> 5;
+    const int64_t k0 = chunk * chunk_len;
+    if (k0 >= total) return;
+    const int64_t k1 = min(k0 + (int64_t)chunk_len, total);
+    const int64_t n_self = o.self ? (o.n_self ? (int64_t)*o.n_self : n_seg) : 0;
+
+    int64_t s = seg_containing(ptr, n_seg, k0);
+    int64_t k = k0;
+    while (k < k1) {
+        int64_t seg_beg = (int64_t)ptr[s], seg_end = (int64_t)ptr[s + 1];
+        while (seg_end <= k) { ++s; seg_beg = seg_end; seg_end = (int64_t)ptr[s + 1]; }   // empty segments
+        const int64_t e1 = min(seg_end, k1);
+
+        float acc[CPL][E];
+#pragma unroll
+        for (int q = 0; q < CPL; ++q)
+#pragma unroll
+            for (int kk = 0; kk < E; ++kk) acc[q][kk] = 0.f;
+        for (int64_t base = k; base < e1; base += 32) {
+            const int m = (int)min((int64_t)32, e1 - base);
+            const int32_t mine = lane < m ? idx[base + lane] : 0;
+            float wmine = 1.f;
+            if (kWeight) wmine = lane < m ? w[mine] : 0.f;
+            for (int t = 0; t * G < m; t += U) {
+                float v[U][CPL][E];
+                float wt[U];
+                bool ok[U];
+#pragma unroll
+                for (int u = 0; u < U; ++u) {
+                    const int j = (t + u) * G + g;
+                    ok[u] = j < m;
+                    const int32_t id = __shfl_sync(0xffffffffu, mine, j & 31);
+                    wt[u] = kWeight ? __shfl_sync(0xffffffffu, wmine, j & 31) : 1.f;
+                    const T *row = in + (int64_t)id * ld_in;
+#pragma unroll
+                    for (int q = 0; q < CPL; ++q) {
+                        const int ch = c + q * LPR;
+                        if (ok[u] && ch < n_chunks) Chunk<T>::load(row + ch * E, v[u][q]);
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < U; ++u)
+#pragma unroll
+                    for (int q = 0; q < CPL; ++q)
+                        if (ok[u] && c + q * LPR < n_chunks)
+#pragma unroll
+                            for (int kk = 0; kk < E; ++kk) {
+                                if (kWeight) acc[q][kk] = fmaf(wt[u], v[u][q][kk], acc[q][kk]);
+                                else acc[q][kk] += v[u][q][kk];
+                            }
+            }
+        }
+#pragma unroll
+        for (int off = LPR; off < 32; off <<= 1)
+#pragma unroll
+            for (int q = 0; q < CPL; ++q)
+#pragma unroll
+                for (int kk = 0; kk < E; ++kk) acc[q][kk] += __shfl_xor_sync(0xffffffffu, acc[q][kk], off);
+
+        const bool begins = seg_beg >= k0;
+        const bool ends = seg_end <= k1;
+        if (g == 0) {
+#pragma unroll
+            for (int q = 0; q < CPL; ++q) {
+                const int ch = c + q * LPR;
+                if (ch >= n_chunks) continue;
+                if (begins && ends) {
+                    float r[E];
+#pragma unroll
+                    for (int kk = 0; kk < E; ++kk)
+                        r[kk] = seg_finish_value(o, s, seg_end - seg_beg, ch * E + kk, acc[q][kk], s < n_self);
+                    Chunk<T>::store(o.out + s * o.ld_out + ch * E, r);
+                } else {
+                    float *dst = (begins ? tail : head) + chunk * d + ch * E;
+#pragma unroll
+                    for (int kk = 0; kk < E; kk += 4)
+                        *reinterpret_cast<float4 *>(dst + kk) =
+                            make_float4(acc[q][kk], acc[q][kk + 1], acc[q][kk + 2], acc[q][kk + 3]);
+                }
+            }
+        }
+        k = e1;
+        ++s;
+    }
+}
+
+// Finishing kernel.  Blocks [0, n_chunk_blocks): block b looks at chunk b; if the segment that
+// holds the chunk's first entry started in an earlier chunk and ends in this one, the block adds
+// its partial rows in order and writes the result.  Blocks beyond that: one thread group per
+// segment, writing fin(0) for segments without entries.
+template <typename T, typename PtrT>
+__global__ void __launch_bounds__(kAggThreads)
+seg_finish_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_t n_seg_host, int chunk_len, int d,
+                  const float *__restrict__ head, const float *__restrict__ tail, int64_t n_chunk_blocks,
+                  SegOut<T> o)
+{
+    constexpr int W = kAggThreads / 32;
+    __shared__ float4 red[W][32];
+    const int64_t n_seg = n_seg_dev ? (int64_t)*n_seg_dev : n_seg_host;
+    if (n_seg <= 0) return;
+    const int64_t total = (int64_t)ptr[n_seg];
+    const int64_t n_self = o.self ? (o.n_self ? (int64_t)*o.n_self : n_seg) : 0;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+
+    if ((int64_t)blockIdx.x >= n_chunk_blocks) {
+        // segments without entries: 8 lanes per segment
+        const int64_t s = ((int64_t)(blockIdx.x - n_chunk_blocks) * kAggThreads + threadIdx.x) >> 3;
+        if (s >= n_seg || ptr[s + 1] != ptr[s]) return;
+        for (int k = threadIdx.x & 7; k < d; k += 8)
+            o.out[s * o.ld_out + k] = from_float<T>(seg_finish_value(o, s, 0, k, 0.f, s < n_self));
+        return;
+    }
+
+    const int64_t chunk = blockIdx.x;
+    const int64_t k0 = chunk * chunk_len;
+    if (chunk == 0 || k0 >= total) return;
+    const int64_t k1 = min(k0 + (int64_t)chunk_len, total);
+    const int64_t s = seg_containing(ptr, n_seg, k0);
+    const int64_t seg_beg = (int64_t)ptr[s], seg_end = (int64_t)ptr[s + 1];
+    if (seg_beg >= k0 || seg_end > k1) return;          // not split, or finished by a later chunk
+    const int64_t first = seg_beg / chunk_len;          // its part there is tail[first]
+    const int64_t n_parts = chunk - first + 1;
+    const int n_vec = d / 4;
+    for (int vb = 0; vb < n_vec; vb += 32) {
+        const int q = vb + lane;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (q < n_vec) {
+            for (int64_t p = warp; p < n_parts; p += W) {
+                const float *src = (p == 0 ? tail + first * d : head + (first + p) * d) + q * 4;
+                const float4 x = *reinterpret_cast<const float4 *>(src);
+                a.x += x.x; a.y += x.y; a.z += x.z; a.w += x.w;
+            }
+        }
+        red[warp][lane] = a;
+        __syncthreads();
+        if (warp == 0 && q < n_vec) {
+            float4 t = red[0][lane];
+#pragma unroll
+            for (int w2 = 1; w2 < W; ++w2) {
+                const float4 x = red[w2][lane];
+                t.x += x.x; t.y += x.y; t.z += x.z; t.w += x.w;
+            }
+            const float r[4] = {t.x, t.y, t.z, t.w};
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+                o.out[s * o.ld_out + q * 4 + kk] =
+                    from_float<T>(seg_finish_value(o, s, seg_end - seg_beg, q * 4 + kk, r[kk], s < n_self));
+        }
+        __syncthreads();
+    }
+}
+
+// Host side --------------------------------------------------------------------------------
+
+struct RowShape { int lpr, cpl; };
+
+inline RowShape row_shape(int d, int32_t dtype)
+{
+    const int chunks = d * (int)dtype_size(dtype) / 16;
+    int lpr = 4;
+    while (lpr < 32 && lpr < chunks) lpr <<= 1;
+    int cpl = 1;
+    while (lpr * cpl < chunks) cpl <<= 1;
+    return {lpr, cpl};
+}
+
+}  // namespace e2egrec

@@ -1,0 +1,74 @@
+// Shared device/host helpers of the e2egrec kernels (sm_100a).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "../../include/e2egrec.h"
+
+namespace e2egrec {
+
+// indices into e2egrec_block::counts
+enum { CNT_DST = 0, CNT_SRC = 1, CNT_EDGES = 2, CNT_STATUS = 3 };
+
+constexpr int kMaxHops = 4;
+constexpr int kMaxFanout = 128;
+constexpr int kMaxDim = 1024;
+
+__host__ __device__ inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+__host__ __device__ inline int64_t ceil_div(int64_t a, int64_t b) { return (a + b - 1) / b; }
+
+inline size_t dtype_size(int32_t dtype) { return dtype == E2EGREC_BF16 ? 2 : 4; }
+
+// host side: remember the text of a failed launch for e2egrec_last_error()
+void set_last_error(const char *msg);
+int32_t check_launch(const char *what);
+
+// ---------------------------------------------------------------------------------------
+// 16-byte row chunks: 8 bf16 or 4 fp32 values, accumulated in fp32.
+// ---------------------------------------------------------------------------------------
+template <typename T> struct Chunk;
+
+template <> struct Chunk<float> {
+    static constexpr int kElems = 4;
+    __device__ static inline void load(const float *p, float (&v)[4]) {
+        float4 r = __ldg(reinterpret_cast<const float4 *>(p));
+        v[0] = r.x; v[1] = r.y; v[2] = r.z; v[3] = r.w;
+    }
+    __device__ static inline void store(float *p, const float (&v)[4]) {
+        *reinterpret_cast<float4 *>(p) = make_float4(v[0], v[1], v[2], v[3]);
+    }
+};
+
+template <> struct Chunk<__nv_bfloat16> {
+    static constexpr int kElems = 8;
+    __device__ static inline void load(const __nv_bfloat16 *p, float (&v)[8]) {
+        uint4 r = __ldg(reinterpret_cast<const uint4 *>(p));
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {           // bf16 -> fp32 is a 16-bit shift
+            v[2 * i] = __uint_as_float(w[i] << 16);
+            v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+    }
+    __device__ static inline void store(__nv_bfloat16 *p, const float (&v)[8]) {
+        uint32_t w[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * i], v[2 * i + 1]);   // round to nearest even
+            w[i] = *reinterpret_cast<uint32_t *>(&h);
+        }
+        *reinterpret_cast<uint4 *>(p) = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+template <typename T> __device__ inline float to_float(T v);
+template <> __device__ inline float to_float<float>(float v) { return v; }
+template <> __device__ inline float to_float<__nv_bfloat16>(__nv_bfloat16 v) { return __bfloat162float(v); }
+
+template <typename T> __device__ inline T from_float(float v);
+template <> __device__ inline float from_float<float>(float v) { return v; }
+template <> __device__ inline __nv_bfloat16 from_float<__nv_bfloat16>(float v) { return __float2bfloat16_rn(v); }
+
+}  // namespace e2egrec

@@ -1,0 +1,318 @@
+// GraphSAGE forward / backward over sampled blocks: host orchestration and kernel dispatch.
+#include <algorithm>
+
+#include "aggregate.cuh"
+#include "common.cuh"
+#include "gemm_simt.cuh"
+#include "gemm_tc.cuh"
+
+namespace e2egrec {
+
+static inline int64_t pad128(int64_t rows) { return (rows + 127) / 128 * 128; }
+
+struct LayerPlan {
+    int block;          // index into blocks[]: layer l runs on block n_layers-1-l
+    int d_in, d_out;
+    int64_t rows;       // destination rows allocated (cap_dst rounded up to 128)
+    size_t cat_off, h_off;    // offsets into ctx: [rows x 2 d_in], [rows x d_out]
+};
+
+// Layout of the saved activations; forward and backward derive it from the same arguments.
+static int32_t plan_layers(const e2egrec_block *blocks, int32_t n_layers, const e2egrec_mat *X, const e2egrec_mat *W,
+                           LayerPlan *plan, size_t *ctx_bytes)
+{
+    if (!blocks || !X || !W) return E2EGREC_ERR_NULL;
+    if (n_layers < 1 || n_layers > kMaxHops) return E2EGREC_ERR_UNSUPPORTED;
+    if (X->dtype != E2EGREC_F32 && X->dtype != E2EGREC_BF16) return E2EGREC_ERR_DTYPE;
+    const size_t es = dtype_size(X->dtype);
+    if (X->dim < 1 || X->dim > kMaxDim) return E2EGREC_ERR_UNSUPPORTED;
+    if ((X->dim * es) % 16 || (X->ld * es) % 16 || reinterpret_cast<uintptr_t>(X->data) % 16) return E2EGREC_ERR_ALIGN;
+    if (!X->data || X->ld < X->dim) return X->data ? E2EGREC_ERR_ARG : E2EGREC_ERR_NULL;
+    size_t off = 0;
+    int d_in = X->dim;
+    for (int l = 0; l < n_layers; ++l) {
+        const e2egrec_mat &w = W[l];
+        if (!w.data) return E2EGREC_ERR_NULL;
+        if (w.dtype != X->dtype) return E2EGREC_ERR_DTYPE;
+        if (w.dim != 2 * d_in || w.ld != w.dim || w.rows < 1 || w.rows > kMaxDim) return E2EGREC_ERR_ARG;
+        if ((w.rows * es) % 16 || reinterpret_cast<uintptr_t>(w.data) % 16) return E2EGREC_ERR_ALIGN;
+        LayerPlan &p = plan[l];
+        p.block = n_layers - 1 - l;
+        p.d_in = d_in;
+        p.d_out = (int)w.rows;
+        p.rows = pad128(blocks[p.block].cap_dst);
+        p.cat_off = off;
+        off += align_up((size_t)p.rows * 2 * d_in * es, 256);
+        p.h_off = off;
+        off += align_up((size_t)p.rows * p.d_out * es, 256);
+        d_in = p.d_out;
+    }
+    for (int l = 0; l + 1 < n_layers; ++l)      // the sources of a block are the destinations of the next one out
+        if (blocks[plan[l + 1].block].cap_src > blocks[plan[l].block].cap_dst) return E2EGREC_ERR_ARG;
+    *ctx_bytes = off;
+    return E2EGREC_OK;
+}
+
+// ------------------------------------------------------------------------------ launch helpers
+template <typename T, int LPR, int CPL>
+static void launch_sage_aggregate(const T *Hsrc, int64_t ld, const int32_t *nbr, const int32_t *self_ids,
+                                  const e2egrec_block &b, T *cat, int d, int64_t rows, cudaStream_t st)
+{
+    const unsigned grid = (unsigned)std::max<int64_t>(1, ceil_div(rows * 32, kAggThreads));
+    sage_aggregate_kernel<T, LPR, CPL><<<grid, kAggThreads, 0, st>>>(Hsrc, ld, nbr, self_ids, b.indptr, b.counts, cat, d,
+                                                                      (int32_t)rows);
+}
+
+template <typename T>
+static void dispatch_sage_aggregate(const T *Hsrc, int64_t ld, const int32_t *nbr, const int32_t *self_ids,
+                                    const e2egrec_block &b, T *cat, int d, int64_t rows, int32_t dtype, cudaStream_t st)
+{
+    const RowShape rs = row_shape(d, dtype);
+#define E2E_CASE(L, C) \
+    if (rs.lpr == L && rs.cpl == C) return launch_sage_aggregate<T, L, C>(Hsrc, ld, nbr, self_ids, b, cat, d, rows, st);
+    E2E_CASE(4, 1) E2E_CASE(8, 1) E2E_CASE(16, 1) E2E_CASE(32, 1) E2E_CASE(32, 2) E2E_CASE(32, 4)
+#undef E2E_CASE
+}
+
+// Segment reduction over a 32-bit offset array (the transposed block).
+template <typename T, int LPR, int CPL>
+static void launch_seg32(const T *in, int64_t ld_in, const int32_t *ptr, const int32_t *idx, const int32_t *n_seg_dev,
+                         int64_t cap_seg, int64_t cap_entries, int chunk_len, int d, float *head, float *tail,
+                         const SegOut<T> &o, cudaStream_t st)
+{
+    const int64_t n_chunks = ceil_div(cap_entries > 0 ? cap_entries : 1, chunk_len);
+    seg_chunk_kernel<T, int32_t, LPR, CPL, false><<<(unsigned)ceil_div(n_chunks * 32, kAggThreads), kAggThreads, 0, st>>>(
+        in, ld_in, ptr, idx, n_seg_dev, 0, nullptr, chunk_len, d, head, tail, o);
+    const int64_t empty_blocks = ceil_div((cap_seg > 0 ? cap_seg : 1) * 8, kAggThreads);
+    seg_finish_kernel<T, int32_t><<<(unsigned)(n_chunks + empty_blocks), kAggThreads, 0, st>>>(
+        ptr, n_seg_dev, 0, chunk_len, d, head, tail, n_chunks, o);
+}
+
+template <typename T>
+static void dispatch_seg32(const T *in, int64_t ld_in, const int32_t *ptr, const int32_t *idx, const int32_t *n_seg_dev,
+                           int64_t cap_seg, int64_t cap_entries, int chunk_len, int d, float *head, float *tail,
+                           const SegOut<T> &o, int32_t dtype, cudaStream_t st)
+{
+    const RowShape rs = row_shape(d, dtype);
+#define E2E_CASE(L, C)                                                                                              \
+    if (rs.lpr == L && rs.cpl == C)                                                                                 \
+        return launch_seg32<T, L, C>(in, ld_in, ptr, idx, n_seg_dev, cap_seg, cap_entries, chunk_len, d, head, tail, o, st);
+    E2E_CASE(4, 1) E2E_CASE(8, 1) E2E_CASE(16, 1) E2E_CASE(32, 1) E2E_CASE(32, 2) E2E_CASE(32, 4)
+#undef E2E_CASE
+}
+
+constexpr int kBlockChunk = 128;      // transposed-block entries per warp
+constexpr int kDwSplits = 148;        // split-K factor of the weight-gradient product
+
+// ------------------------------------------------------------------------------ forward
+template <typename T>
+static int32_t forward_impl(const e2egrec_block *blocks, int32_t n_layers, const e2egrec_mat *X, const e2egrec_mat *W,
+                            const float *const *bias, const int32_t *act, const LayerPlan *plan, char *ctx,
+                            const e2egrec_mat *H_out, cudaStream_t st)
+{
+    const size_t es = sizeof(T);
+    for (int l = 0; l < n_layers; ++l) {
+        const LayerPlan &p = plan[l];
+        const e2egrec_block &b = blocks[p.block];
+        T *cat = reinterpret_cast<T *>(ctx + p.cat_off);
+        T *hn = reinterpret_cast<T *>(ctx + p.h_off);
+        if (l == 0)   // h^(0) rows are read straight from the feature table through the global ids
+            dispatch_sage_aggregate<T>(static_cast<const T *>(X->data), X->ld, b.nbr_global, b.src_nodes, b, cat, p.d_in,
+                                       p.rows, X->dtype, st);
+        else
+            dispatch_sage_aggregate<T>(reinterpret_cast<const T *>(ctx + plan[l - 1].h_off), p.d_in, b.col, nullptr, b, cat,
+                                       p.d_in, p.rows, X->dtype, st);
+        const float *bl = bias ? bias[l] : nullptr;
+        const int relu = act ? act[l] : 1;
+        bool done = false;
+        if (X->dtype == E2EGREC_BF16)
+            done = tc_update_forward(reinterpret_cast<const __nv_bfloat16 *>(cat), p.rows, 2 * p.d_in,
+                                     static_cast<const __nv_bfloat16 *>(W[l].data), p.d_out, bl, relu,
+                                     reinterpret_cast<__nv_bfloat16 *>(hn), &b.counts[CNT_DST], st);
+        if (!done) {
+            EpiUpdate<T> epi{hn, p.d_out, bl, relu};
+            dim3 grid((unsigned)std::max<int64_t>(1, ceil_div(p.rows, kGemmBM)), (unsigned)ceil_div(p.d_out, kGemmBN), 1);
+            gemm_simt_kernel<T, false, false, EpiUpdate<T>><<<grid, kGemmThreads, 0, st>>>(
+                cat, 2 * p.d_in, static_cast<const T *>(W[l].data), 2 * p.d_in, p.rows, p.d_out, 2 * p.d_in,
+                &b.counts[CNT_DST], nullptr, epi);
+        }
+    }
+    const LayerPlan &top = plan[n_layers - 1];
+    const int64_t rows = blocks[0].cap_dst < H_out->rows ? blocks[0].cap_dst : H_out->rows;
+    if (rows > 0)
+        cudaMemcpy2DAsync(H_out->data, (size_t)H_out->ld * es, ctx + top.h_off, (size_t)top.d_out * es,
+                      (size_t)top.d_out * es, (size_t)rows, cudaMemcpyDeviceToDevice, st);
+    return check_launch("sage_forward");
+}
+
+// ------------------------------------------------------------------------------ backward
+struct BackwardScratch {
+    size_t dz_off[2], dcat_off, head_off, tail_off, part_off, bytes;
+};
+
+static BackwardScratch plan_backward(const e2egrec_block *blocks, int32_t n_layers, const LayerPlan *plan, size_t es)
+{
+    BackwardScratch s{};
+    size_t dz = 0, dcat = 0, part = 0, ht = 0;
+    for (int l = 0; l < n_layers; ++l) {
+        const LayerPlan &p = plan[l];
+        dz = std::max(dz, (size_t)p.rows * p.d_out * es);
+        dcat = std::max(dcat, (size_t)p.rows * 2 * p.d_in * es);
+        part = std::max(part, (size_t)kDwSplits * p.d_out * 2 * p.d_in * sizeof(float));
+        const int64_t n_chunks = ceil_div(std::max(blocks[p.block].cap_edges, 1), kBlockChunk);
+        ht = std::max(ht, (size_t)n_chunks * p.d_in * sizeof(float));
+    }
+    size_t off = 0;
+    auto take = [&](size_t b) { size_t o = off; off += align_up(b, 256); return o; };
+    s.dz_off[0] = take(dz);
+    s.dz_off[1] = take(dz);
+    s.dcat_off = take(dcat);
+    s.head_off = take(ht);
+    s.tail_off = take(ht);
+    s.part_off = take(part);
+    s.bytes = off;
+    return s;
+}
+
+template <typename T>
+static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, const e2egrec_mat *X, const e2egrec_mat *W,
+                             const int32_t *act, const LayerPlan *plan, const char *ctx, const e2egrec_mat *dH_out,
+                             float *const *dW, float *const *dbias, const e2egrec_mat *dX_rows, char *scratch,
+                             const BackwardScratch &bs, uint32_t flags, cudaStream_t st)
+{
+    const int accumulate = (flags & E2EGREC_ACCUMULATE_DW) ? 1 : 0;
+    T *dz_buf[2] = {reinterpret_cast<T *>(scratch + bs.dz_off[0]), reinterpret_cast<T *>(scratch + bs.dz_off[1])};
+    T *dcat = reinterpret_cast<T *>(scratch + bs.dcat_off);
+    float *head = reinterpret_cast<float *>(scratch + bs.head_off);
+    float *tail = reinterpret_cast<float *>(scratch + bs.tail_off);
+    float *part = reinterpret_cast<float *>(scratch + bs.part_off);
+
+    // gradient entering the top layer, masked by its activation
+    {
+        const LayerPlan &p = plan[n_layers - 1];
+        const e2egrec_block &b = blocks[p.block];
+        const int64_t total = p.rows * p.d_out;
+        relu_mask_kernel<T><<<(unsigned)std::max<int64_t>(1, ceil_div(total, 256)), 256, 0, st>>>(
+            static_cast<const T *>(dH_out->data), dH_out->ld, reinterpret_cast<const T *>(ctx + p.h_off), p.d_out,
+            &b.counts[CNT_DST], p.rows, p.d_out, act ? act[n_layers - 1] : 1, dz_buf[(n_layers - 1) & 1]);
+    }
+    for (int l = n_layers - 1; l >= 0; --l) {
+        const LayerPlan &p = plan[l];
+        const e2egrec_block &b = blocks[p.block];
+        const T *dz = dz_buf[l & 1];
+        const T *cat = reinterpret_cast<const T *>(ctx + p.cat_off);
+        const int32_t *n_dst = &b.counts[CNT_DST];
+        const int two_d = 2 * p.d_in;
+        // dW_l = dZ^T [h | agg]   (split over the rows, partial sums added in a fixed order)
+        {
+            EpiPartial epi{part, two_d, (int64_t)p.d_out * two_d};
+            dim3 grid((unsigned)ceil_div(p.d_out, kGemmBM), (unsigned)ceil_div(two_d, kGemmBN), kDwSplits);
+            gemm_simt_kernel<T, true, true, EpiPartial><<<grid, kGemmThreads, 0, st>>>(
+                dz, p.d_out, cat, two_d, p.d_out, two_d, p.rows, nullptr, n_dst, epi);
+            const int64_t n = (int64_t)p.d_out * two_d;
+            splitk_reduce_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(part, n, kDwSplits, accumulate, dW[l]);
+        }
+        if (dbias && dbias[l])
+            colsum_kernel<T><<<(unsigned)ceil_div(p.d_out, 32), 256, 0, st>>>(dz, p.d_out, n_dst, p.d_out, accumulate, dbias[l]);
+        // dCat = dZ W_l, the agg half scaled by 1/|S|
+        {
+            EpiDCat<T> epi{dcat, two_d, p.d_in, b.inv_cnt};
+            dim3 grid((unsigned)std::max<int64_t>(1, ceil_div(p.rows, kGemmBM)), (unsigned)ceil_div(two_d, kGemmBN), 1);
+            gemm_simt_kernel<T, false, true, EpiDCat<T>><<<grid, kGemmThreads, 0, st>>>(
+                dz, p.d_out, static_cast<const T *>(W[l].data), two_d, p.rows, two_d, p.d_out, n_dst, nullptr, epi);
+        }
+        // transposed aggregation: gather over the block's CSC, plus the self rows, masked by the
+        // activation of the layer below
+        SegOut<T> o{};
+        o.self = dcat;
+        o.ld_self = two_d;
+        o.n_self = n_dst;
+        o.mean = 0;
+        if (l > 0) {
+            o.out = dz_buf[(l - 1) & 1];
+            o.ld_out = p.d_in;
+            const int relu_below = act ? act[l - 1] : 1;
+            o.mask = relu_below ? reinterpret_cast<const T *>(ctx + plan[l - 1].h_off) : nullptr;
+            o.ld_mask = p.d_in;
+        } else {
+            o.out = static_cast<T *>(dX_rows->data);
+            o.ld_out = dX_rows->ld;
+            o.mask = nullptr;
+        }
+        dispatch_seg32<T>(dcat + p.d_in, two_d, b.csc_ptr, b.csc_row, &b.counts[CNT_SRC], b.cap_src, b.cap_edges,
+                          kBlockChunk, p.d_in, head, tail, o, X->dtype, st);
+    }
+    return check_launch("sage_backward");
+}
+
+}  // namespace e2egrec
+
+using namespace e2egrec;
+
+extern "C" int32_t e2egrec_sage_forward(const e2egrec_block *blocks, int32_t n_layers, const e2egrec_mat *X,
+                                        const e2egrec_mat *W, const float *const *bias, const int32_t *act,
+                                        void *ctx, size_t *ctx_bytes, const e2egrec_mat *H_out, void *stream)
+{
+    if (!ctx_bytes) return E2EGREC_ERR_NULL;
+    LayerPlan plan[kMaxHops];
+    size_t need = 0;
+    int32_t rc = plan_layers(blocks, n_layers, X, W, plan, &need);
+    if (rc != E2EGREC_OK) return rc;
+    if (!ctx) { *ctx_bytes = need; return E2EGREC_OK; }
+    if (*ctx_bytes < need) { *ctx_bytes = need; return E2EGREC_ERR_WORKSPACE; }
+    if (reinterpret_cast<uintptr_t>(ctx) % 256) return E2EGREC_ERR_ALIGN;
+    if (!H_out || !H_out->data) return E2EGREC_ERR_NULL;
+    if (H_out->dtype != X->dtype) return E2EGREC_ERR_DTYPE;
+    if (H_out->dim != plan[n_layers - 1].d_out || H_out->ld < H_out->dim) return E2EGREC_ERR_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (X->dtype == E2EGREC_BF16)
+        return forward_impl<__nv_bfloat16>(blocks, n_layers, X, W, bias, act, plan, static_cast<char *>(ctx), H_out, st);
+    return forward_impl<float>(blocks, n_layers, X, W, bias, act, plan, static_cast<char *>(ctx), H_out, st);
+}
+
+extern "C" int32_t e2egrec_sage_ctx_layout(const e2egrec_block *blocks, int32_t n_layers, const e2egrec_mat *X,
+                                           const e2egrec_mat *W, size_t *cat_offset, size_t *h_offset, int64_t *rows)
+{
+    if (!cat_offset || !h_offset || !rows) return E2EGREC_ERR_NULL;
+    LayerPlan plan[kMaxHops];
+    size_t need = 0;
+    int32_t rc = plan_layers(blocks, n_layers, X, W, plan, &need);
+    if (rc != E2EGREC_OK) return rc;
+    for (int l = 0; l < n_layers; ++l) {
+        cat_offset[l] = plan[l].cat_off;
+        h_offset[l] = plan[l].h_off;
+        rows[l] = plan[l].rows;
+    }
+    return E2EGREC_OK;
+}
+
+extern "C" int32_t e2egrec_sage_backward(const e2egrec_block *blocks, int32_t n_layers, const e2egrec_mat *X,
+                                         const e2egrec_mat *W, const int32_t *act, const void *ctx,
+                                         const e2egrec_mat *dH_out, float *const *dW, float *const *dbias,
+                                         const e2egrec_mat *dX_rows, void *scratch, size_t *scratch_bytes,
+                                         uint32_t flags, void *stream)
+{
+    if (!scratch_bytes) return E2EGREC_ERR_NULL;
+    LayerPlan plan[kMaxHops];
+    size_t ctx_need = 0;
+    int32_t rc = plan_layers(blocks, n_layers, X, W, plan, &ctx_need);
+    if (rc != E2EGREC_OK) return rc;
+    const BackwardScratch bs = plan_backward(blocks, n_layers, plan, dtype_size(X->dtype));
+    if (!scratch) { *scratch_bytes = bs.bytes; return E2EGREC_OK; }
+    if (*scratch_bytes < bs.bytes) { *scratch_bytes = bs.bytes; return E2EGREC_ERR_WORKSPACE; }
+    if (reinterpret_cast<uintptr_t>(scratch) % 256 || reinterpret_cast<uintptr_t>(ctx) % 256) return E2EGREC_ERR_ALIGN;
+    if (!ctx || !dH_out || !dH_out->data || !dW || !dX_rows || !dX_rows->data) return E2EGREC_ERR_NULL;
+    for (int l = 0; l < n_layers; ++l)
+        if (!dW[l]) return E2EGREC_ERR_NULL;
+    if (dH_out->dtype != X->dtype || dX_rows->dtype != X->dtype) return E2EGREC_ERR_DTYPE;
+    if (dH_out->dim != plan[n_layers - 1].d_out || dX_rows->dim != X->dim) return E2EGREC_ERR_ARG;
+    if (dX_rows->rows < blocks[n_layers - 1].cap_src || dH_out->rows < blocks[0].cap_dst) return E2EGREC_ERR_ARG;
+    const size_t es = dtype_size(X->dtype);
+    if ((dX_rows->ld * es) % 16 || reinterpret_cast<uintptr_t>(dX_rows->data) % 16) return E2EGREC_ERR_ALIGN;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (X->dtype == E2EGREC_BF16)
+        return backward_impl<__nv_bfloat16>(blocks, n_layers, X, W, act, plan, static_cast<const char *>(ctx), dH_out, dW,
+                                            dbias, dX_rows, static_cast<char *>(scratch), bs, flags, st);
+    return backward_impl<float>(blocks, n_layers, X, W, act, plan, static_cast<const char *>(ctx), dH_out, dW, dbias,
+                                dX_rows, static_cast<char *>(scratch), bs, flags, st);
+}

@@ -1,0 +1,150 @@
+"""GPU parity: the CUDA path through the C ABI against the CPU oracle, same seeded inputs."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth_inputs as S
+from helpers import (Case, assert_blocks_equal, assert_close, assert_close_budget, reduction_rss,
+                     relu_flip_budgets)
+
+pytestmark = pytest.mark.gpu
+
+
+def _check_float(case, gpu, ora):
+    n_seeds = case.seeds.size
+    n_src = ora["blocks"][-1]["n_src"]
+    rss = reduction_rss(case, ora)
+    assert_close("forward", gpu["out"][:n_seeds], ora["out"], case.bf16, rss["forward"])
+    if "dWs" in ora:
+        # ReLU decisions that differ between fp32 and float64 sums are accepted only within tau of the kink
+        tau = 2e-2 if case.bf16 else 1e-5
+        B_dW, B_dX = relu_flip_budgets(case, ora, gpu, tau)
+        for l, (g, o) in enumerate(zip(gpu["dWs"], ora["dWs"])):
+            assert_close_budget(f"dW[{l}]", g, o, B_dW[l], case.bf16, rss["dW"][l])
+        assert_close_budget("dX", gpu["dX"][:n_src], ora["dX"], B_dX, case.bf16, rss["dX"])
+
+
+@pytest.mark.parametrize("step", [0, 3])
+def test_tiny_fp32_sample_forward_backward(step):
+    case = Case(S.WORKLOADS["tiny"], step=step)
+    dH = case.upstream_grad(case.seeds.size, case.w.hidden)
+    ora = case.run_oracle(dH)
+    gpu = case.run_gpu(dH)
+    assert_blocks_equal(gpu["blocks"], ora["blocks"])
+    _check_float(case, gpu, ora)
+
+
+def test_medium_small_bf16_sample_forward_backward():
+    case = Case(S.WORKLOADS["medium_small"], step=1)
+    dH = case.upstream_grad(case.seeds.size, case.w.hidden)
+    ora = case.run_oracle(dH)
+    gpu = case.run_gpu(dH)
+    assert_blocks_equal(gpu["blocks"], ora["blocks"])
+    _check_float(case, gpu, ora)
+
+
+def test_medium_small_bf16_linear_backward_is_strict():
+    """Identity activations: no sign decisions, so every gradient element is held to the plain tolerance."""
+    case = Case(S.WORKLOADS["medium_small"], step=5, acts=[0, 0])
+    dH = case.upstream_grad(case.seeds.size, case.w.hidden)
+    ora = case.run_oracle(dH)
+    gpu = case.run_gpu(dH)
+    assert_blocks_equal(gpu["blocks"], ora["blocks"])
+    n_src = ora["blocks"][-1]["n_src"]
+    rss = reduction_rss(case, ora)
+    assert_close("forward", gpu["out"][: case.seeds.size], ora["out"], True, rss["forward"])
+    for l, (g, o) in enumerate(zip(gpu["dWs"], ora["dWs"])):
+        assert_close(f"dW[{l}]", g, o, True, rss["dW"][l])
+    assert_close("dX", gpu["dX"][:n_src], ora["dX"], True, rss["dX"])
+
+
+def test_run_to_run_bit_identical():
+    case = Case(S.WORKLOADS["medium_small"], step=2)
+    dH = case.upstream_grad(case.seeds.size, case.w.hidden)
+    a = case.run_gpu(dH)
+    b = case.run_gpu(dH)
+    assert np.array_equal(a["out"], b["out"]) and np.array_equal(a["dX"], b["dX"])
+    for x, y in zip(a["dWs"], b["dWs"]):
+        assert np.array_equal(x, y)
+    assert_blocks_equal(a["blocks"], b["blocks"])
+
+
+def test_scratch_is_reusable_across_steps():
+    """One Blocks object (one scratch buffer) serves consecutive steps."""
+    import paper_2511_20564_b200 as E
+    w = S.WORKLOADS["tiny"]
+    indptr, indices, _ = S.build_graph(w)
+    blocks = E.Blocks(w.n_nodes, w.batch, w.fanouts)
+    ip, ix = torch.from_numpy(indptr).cuda(), torch.from_numpy(indices).cuda()
+    for step in range(3):
+        seeds = S.seed_batch(w.n_nodes, w.batch, w.seed, step)
+        E.sample_khop(ip, ix, torch.from_numpy(seeds).cuda(), blocks, w.seed, step)
+        ora = oracle.sample_khop(indptr, indices, seeds, w.fanouts, w.seed, step)
+        assert_blocks_equal(blocks.to_host(), ora)
+
+
+def _star_graph(n_leaves):
+    row = np.concatenate([np.zeros(n_leaves, np.int32), np.arange(1, n_leaves + 1, dtype=np.int32)])
+    col = np.concatenate([np.arange(1, n_leaves + 1, dtype=np.int32), np.zeros(n_leaves, np.int32)])
+    return S.coo_to_csr(n_leaves + 3, row, col)       # nodes n_leaves+1, n_leaves+2 are isolated
+
+
+@pytest.mark.parametrize("fanouts,seeds", [((4, 3), [0, 5, 301]), ((128,), [0, 1, 2]), ((2, 2, 2), [7]),
+                                           ((5, 5), [301, 302])])
+def test_edge_cases_hub_isolated_and_take_all(fanouts, seeds):
+    n_leaves = 300
+    graph = _star_graph(n_leaves)
+    w = S.Workload("star", 1, n_leaves + 2, 0, None, None, 9, 8, 8, "f32", tuple(fanouts), len(seeds))
+    case = Case(w, step=4, seeds=seeds, graph=graph)
+    dH = case.upstream_grad(len(seeds), 8)
+    ora = case.run_oracle(dH)
+    gpu = case.run_gpu(dH)
+    assert_blocks_equal(gpu["blocks"], ora["blocks"])
+    _check_float(case, gpu, ora)
+
+
+def test_hub_column_longer_than_a_chunk():
+    """Many destinations sample the same hub, so its transposed column spans several warps' chunks."""
+    n_leaves = 3000
+    graph = _star_graph(n_leaves)
+    seeds = np.arange(1, 1201, dtype=np.int32)
+    for dtype, d in (("f32", 16), ("bf16", 64)):
+        w = S.Workload("star", 1, n_leaves + 2, 0, None, None, 9, d, d, dtype, (3, 2), seeds.size)
+        case = Case(w, step=0, seeds=seeds, graph=graph)
+        dH = case.upstream_grad(seeds.size, d)
+        ora = case.run_oracle(dH)
+        gpu = case.run_gpu(dH)
+        assert_blocks_equal(gpu["blocks"], ora["blocks"])
+        _check_float(case, gpu, ora)
+
+
+def test_empty_batch():
+    graph = _star_graph(10)
+    w = S.Workload("star", 1, 12, 0, None, None, 9, 8, 8, "f32", (3, 2), 0)
+    case = Case(w, step=0, seeds=np.zeros(0, np.int32), graph=graph)
+    gpu = case.run_gpu()
+    for b in gpu["blocks"]:
+        assert b["n_dst"] == 0 and b["n_src"] == 0 and b["n_edges"] == 0 and b["status"] == 0
+
+
+def test_out_of_range_seed_sets_status_and_does_not_fault():
+    import paper_2511_20564_b200 as E
+    indptr, indices = _star_graph(10)
+    blocks = E.Blocks(13, 2, (2,))
+    seeds = torch.tensor([1, 99], dtype=torch.int32, device="cuda")
+    E.sample_khop(torch.from_numpy(indptr).cuda(), torch.from_numpy(indices).cuda(), seeds, blocks, 0, 0)
+    assert blocks.to_host()[0]["status"] & 1
+
+
+def test_host_side_argument_errors():
+    import paper_2511_20564_b200 as E
+    with pytest.raises(E.E2EGrecError):
+        E.sample_khop_workspace(100, 4, [200])          # fanout above the limit
+    with pytest.raises(E.E2EGrecError):
+        E.sample_khop_workspace(100, 4, [3, 3, 3, 3, 3])  # too many hops
+    blocks = E.Blocks(100, 4, (3,))
+    X = torch.zeros(100, 6, device="cuda")              # 24-byte rows: not 16-byte aligned
+    W = torch.zeros(8, 12, device="cuda")
+    with pytest.raises(E.E2EGrecError):
+        E.sage_forward(blocks, X, [W])
