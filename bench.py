@@ -1,0 +1,375 @@
+#!/usr/bin/env python
+"""Benchmark of the sampled-GNN training pass (sample -> forward -> backward) on B200.
+
+One step = k-hop sampling of one seed batch, the GraphSAGE forward over the sampled blocks and the
+full backward (weight gradients and feature-row gradients), through the library's C ABI.  Prints one
+JSON line (rank 0).  `--impl reference` times the CPU oracle instead (a deliberately plain program).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import synth_inputs as S  # noqa: E402
+
+METRIC = "sampled_gnn_sample_fwd_bwd_edges_per_sec"
+UNIT = "edges/s"
+CLOCK_QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+               "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+               "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+TAP_NAMES = {1: "sage_aggregate_kernel (layer-0 mean aggregation, gathers X rows)",
+             2: "seg_chunk_kernel+seg_finish_kernel (layer-0 transposed aggregation -> dX rows)",
+             3: "layer-0 dense transform W[h|agg]",
+             4: "layer-0 weight gradient dZ^T[h|agg]",
+             5: "layer-0 input gradient dZ W",
+             6: "e2egrec_sample_khop (all sampling kernels)"}
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        d = json.load(open(p))
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+class ClockSampler:
+    def __init__(self, gpu_index):
+        self.path = f"/tmp/e2egrec_clocks_{os.getpid()}.csv"
+        self.gpu = gpu_index
+        self.p = None
+
+    def start(self):
+        try:
+            self.f = open(self.path, "w")
+            self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={CLOCK_QUERY}",
+                                       "--format=csv,noheader,nounits", "-lms", "100"], stdout=self.f,
+                                      stderr=subprocess.DEVNULL)
+        except Exception:
+            self.p = None
+
+    def mark(self):
+        """Wall-clock stamp in nvidia-smi's timestamp format resolution (seconds since epoch)."""
+        return time.time()
+
+    def stop(self, t_begin=None, t_end=None):
+        if self.p is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except Exception:
+            self.p.kill()
+        self.f.close()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in open(self.path):
+            c = [x.strip() for x in line.split(",")]
+            if len(c) < 9:
+                continue
+            try:
+                import datetime
+                ts = datetime.datetime.strptime(c[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                if t_begin is not None and not (t_begin - 0.05 <= ts <= t_end + 0.05):
+                    continue
+                sm.append(float(c[1]))
+                smax.append(float(c[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, c[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        try:
+            os.remove(self.path)
+        except OSError:
+            pass
+        return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(smax) if smax else None,
+                    reasons=sorted(reasons), samples=len(sm))
+
+
+def build_inputs(w: S.Workload):
+    indptr, indices, inter = S.build_graph(w)
+    X, Ws = S.build_model(w)
+    return indptr, indices, X, Ws, inter
+
+
+def make_batches(w, inter, recipe, first, count):
+    """Seed batches for steps first .. first+count-1: `activity` draws nodes as endpoints of random
+    interactions (the source nodes of a training stream), `uniform` draws them uniformly over all ids."""
+    if recipe == "uniform":
+        return np.stack([S.seed_batch(w.n_nodes, w.batch, w.seed, first + i) for i in range(count)])
+    return np.stack([S.seed_batch_from_interactions(inter[0], inter[1], w.batch, w.seed, first + i)
+                     for i in range(count)])
+
+
+def upstream_grad(w, rows):
+    g = np.random.default_rng(4321).standard_normal((rows, w.hidden)).astype(np.float32)
+    return S.to_bf16_values(g) if w.dtype == "bf16" else g
+
+
+# ------------------------------------------------------------------------------------------ reference arm
+def oracle_step(w, indptr, indices, X, Ws, seeds, step, dH):
+    import oracle
+    bf16 = w.dtype == "bf16"
+    blocks = oracle.sample_khop(indptr, indices, seeds, w.fanouts, w.seed, step)
+    out, ctx = oracle.sage_forward(blocks, X, Ws, bf16=bf16)
+    oracle.sage_backward(blocks, ctx, Ws, dH[: seeds.size], bf16=bf16)
+    return sum(b["n_edges"] for b in blocks)
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    indptr, indices, X, Ws, inter = build_inputs(w)
+    sample = args.ref_seeds
+    dH = upstream_grad(w, sample).astype(np.float64)
+    batches = make_batches(w, inter, args.seeds, 0, args.warmup + args.steps)[:, :sample]
+    for i in range(args.warmup):
+        oracle_step(w, indptr, indices, X, Ws, batches[i], i, dH)
+    t0 = time.perf_counter()
+    edges = 0
+    for i in range(args.warmup, args.warmup + args.steps):
+        edges += oracle_step(w, indptr, indices, X, Ws, batches[i], i, dH)
+    dt = time.perf_counter() - t0
+    val = edges / dt
+    desc = f"first {sample} of the {w.batch} seeds of each step's batch, full sample+forward+backward"
+    line = dict(impl="reference", metric=METRIC, value=val, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+                warmup=args.warmup, ms_per_step=dt / args.steps * 1e3, higher_is_better=True, scaling="weak",
+                vs_baseline=None, dtype="f64", data="synthetic",
+                config=dict(workload=w.name, nodes=w.n_nodes, csr_entries=int(indptr[-1]), dim=w.dim, hidden=w.hidden,
+                            layers=len(w.fanouts), fanouts=list(w.fanouts), batch=w.batch, seeds=args.seeds,
+                            sample=desc),
+                cpu_baseline=dict(value=val, unit=UNIT, cores=1, kind="oracle", sample=desc),
+                e2e=dict(value=val, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
+                gpu_launches=0)
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------ our arm
+def run_ours(args, w):
+    import torch
+    import torch.distributed as dist
+    import paper_2511_20564_b200 as E
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    E.lib()                                            # fails loudly if the CUDA library is missing
+
+    indptr_h, indices_h, X_h, Ws_h, inter = build_inputs(w)
+    dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    indptr, indices = torch.from_numpy(indptr_h).to(dev), torch.from_numpy(indices_h).to(dev)
+    X = torch.from_numpy(X_h).to(dev, dt)
+    Ws = [torch.from_numpy(W).to(dev, dt) for W in Ws_h]
+    K, Wm = args.steps, args.warmup
+    total = K + Wm
+    # every rank trains on its own batches (data parallel replicas; no exchange on the measured path)
+    seeds_h = make_batches(w, inter, args.seeds, rank * 1_000_000, total)
+    seeds_pin = torch.from_numpy(seeds_h).pin_memory()
+    seeds_dev = seeds_pin.to(dev)
+    dH_h = upstream_grad(w, w.batch)
+    dH_pin = torch.from_numpy(dH_h).to(dt).pin_memory()
+    dH = dH_pin.to(dev)
+
+    blocks = E.Blocks(w.n_nodes, w.batch, w.fanouts, dev)
+    L = len(Ws)
+    ctx = torch.empty(E.binding.sage_forward_ctx_bytes(blocks, X, Ws), dtype=torch.uint8, device=dev)
+    H_out = torch.zeros(blocks.caps[0][0], w.hidden, dtype=dt, device=dev)
+    scratch = torch.empty(E.binding.sage_backward_scratch_bytes(blocks, X, Ws), dtype=torch.uint8, device=dev)
+    dWs = [torch.zeros(W.shape, dtype=torch.float32, device=dev) for W in Ws]
+    dX = torch.zeros(blocks.caps[L - 1][1], w.dim, dtype=dt, device=dev)
+    count_log = torch.zeros(total, L, 4, dtype=torch.int32, device=dev)
+
+    def step(i, seeds_t, dH_t):
+        E.sample_khop(indptr, indices, seeds_t, blocks, w.seed, rank * 1_000_000 + i)
+        E.sage_forward(blocks, X, Ws, ctx=ctx, H_out=H_out)
+        E.sage_backward(blocks, X, Ws, ctx, dH_t, dWs=dWs, dX_rows=dX, scratch=scratch)
+        count_log[i].copy_(blocks.counts, non_blocking=True)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing, with a per-kernel tap pass for the roofline
+    for i in range(Wm):
+        step(i, seeds_dev[i], dH)
+    taps = {}
+    ev_pool = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+    for a, b in ev_pool:
+        a.record(); b.record()
+    torch.cuda.synchronize()
+    n_tap_steps = min(K, 10)
+    for which in TAP_NAMES:                              # untimed pass: where does a step spend its time
+        for i in range(n_tap_steps):
+            E.profile_tap(which, *ev_pool[i])
+            step(Wm + i, seeds_dev[Wm + i], dH)
+        torch.cuda.synchronize()
+        taps[which] = [ev_pool[i][0].elapsed_time(ev_pool[i][1]) for i in range(n_tap_steps)]
+    tap_ms = {k: float(np.mean(v)) for k, v in taps.items()}
+    dominant = max((k for k in tap_ms if k != 6), key=lambda k: tap_ms[k])
+
+    clocks = ClockSampler(local)
+    clocks.start()
+    time.sleep(0.6)                                    # let the sampler reach its steady 100 ms period
+    barrier()
+    t_begin = clocks.mark()
+    launches0 = E.launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(K):
+        E.profile_tap(dominant, *ev_pool[i])           # events around the dominant kernel, on its own stream
+        step(Wm + i, seeds_dev[Wm + i], dH)
+    e1.record()
+    barrier()
+    launches = E.launch_count() - launches0
+    clk = clocks.stop(t_begin, clocks.mark())
+    ms = e0.elapsed_time(e1)
+    dom_ms = [ev_pool[i][0].elapsed_time(ev_pool[i][1]) for i in range(K)]
+    counts = count_log[Wm:].cpu().numpy().astype(np.int64)      # [K, L, 4]
+    status = int(np.bitwise_or.reduce(counts[:, :, 3].ravel())) if counts.size else 0
+    if status:
+        raise RuntimeError(f"device status bits {status} set during the timed region")
+    edges_rank = int(counts[:, :, 2].sum())
+
+    # ---- end to end: host buffers in, results out, every step
+    res_pin = [torch.empty(H_out.shape, dtype=dt).pin_memory()] + [torch.empty(W.shape, dtype=torch.float32).pin_memory()
+                                                                   for W in Ws]
+    cnt_pin = torch.empty(L, 4, dtype=torch.int32).pin_memory()
+    seeds_in = torch.empty(w.batch, dtype=torch.int32, device=dev)
+    dH_in = torch.empty_like(dH)
+    h2d = seeds_pin[0].numel() * 4 + dH_pin.numel() * dH_pin.element_size()
+    d2h = sum(t.numel() * t.element_size() for t in res_pin) + cnt_pin.numel() * 4
+
+    def e2e_step(i):
+        seeds_in.copy_(seeds_pin[i], non_blocking=True)
+        dH_in.copy_(dH_pin, non_blocking=True)
+        step(i, seeds_in, dH_in)
+        res_pin[0].copy_(H_out, non_blocking=True)
+        for t, s in zip(res_pin[1:], dWs):
+            t.copy_(s, non_blocking=True)
+        cnt_pin.copy_(blocks.counts, non_blocking=True)
+        torch.cuda.current_stream().synchronize()      # the caller reads the results of this step
+        return int(cnt_pin[:, 2].sum())
+
+    for i in range(min(Wm, 3)):
+        e2e_step(i)
+    barrier()
+    t0 = time.perf_counter()
+    e2e_edges = 0
+    for i in range(K):
+        e2e_edges += e2e_step(Wm + i)
+    barrier()
+    e2e_s = time.perf_counter() - t0
+
+    # ---- reduce over ranks: slowest rank's time, all ranks' edges
+    if world > 1:
+        t = torch.tensor([ms, e2e_s], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms, e2e_s = float(t[0]), float(t[1])
+        c = torch.tensor([edges_rank, e2e_edges], dtype=torch.int64, device=dev)
+        dist.all_reduce(c, op=dist.ReduceOp.SUM)
+        edges_all, e2e_edges_all = int(c[0]), int(c[1])
+    else:
+        edges_all, e2e_edges_all = edges_rank, e2e_edges
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- roofline of the dominant kernel (algorithmic bytes or flops per launch / mean launch time)
+    peaks = measured_peaks()
+    es = 2 if w.dtype == "bf16" else 4
+    r = w.dim * es
+    outer = counts[:, L - 1, :].mean(axis=0)              # mean n_dst, n_src, n_edges of the outermost block
+    n_dst, n_src, n_edges = float(outer[0]), float(outer[1]), float(outer[2])
+    dom_mean_ms = float(np.mean(dom_ms))
+    if dominant == 1:      # per entry: id + gathered row; per destination: offsets, self id, self row, [self|mean] row out
+        alg = n_edges * (4 + r) + n_dst * (8 + 4 + r + 2 * r)
+        roof = dict(bound="hbm", achieved=alg / dom_mean_ms / 1e6, peak=peaks["hbm_gbs"], unit="GB/s")
+    elif dominant == 2:    # per entry: row id + gathered row; per source: offsets + row out; per destination: self row
+        alg = n_edges * (4 + r) + n_src * (8 + r) + n_dst * r
+        roof = dict(bound="hbm", achieved=alg / dom_mean_ms / 1e6, peak=peaks["hbm_gbs"], unit="GB/s")
+    else:                  # dense products of layer 0: 2 * rows * (2 d) * hidden flop each
+        alg = 2.0 * n_dst * 2 * w.dim * w.hidden
+        peak = peaks["bf16_tflops"] if w.dtype == "bf16" else peaks["bf16_tflops"] / 2.25 * 0.08
+        roof = dict(bound="tensor" if w.dtype == "bf16" else "alu", achieved=alg / dom_mean_ms / 1e9, peak=peak,
+                    unit="TFLOP/s")
+    roof.update(frac=roof["achieved"] / roof["peak"], traffic=None, kernel=TAP_NAMES[dominant],
+                ms_per_launch=dom_mean_ms, algorithmic_units_per_launch=alg, peak_source=peaks["source"])
+
+    line = dict(metric=METRIC, value=edges_all / (ms / 1e3), unit=UNIT, n_gpus=world, steps=K, warmup=Wm,
+                ms_per_step=ms / K, higher_is_better=True, scaling="weak", vs_baseline=None, dtype=w.dtype,
+                data="synthetic",
+                config=dict(workload=w.name, nodes=w.n_nodes, csr_entries=int(indptr_h[-1]), dim=w.dim, hidden=w.hidden,
+                            layers=L, fanouts=list(w.fanouts), batch=w.batch, seeds=args.seeds,
+                            parallelism=f"replicas x{world}",
+                            l2="inputs larger than L2: feature table + graph = %.0f MB, a new batch every step"
+                               % ((X.numel() * es + indices.numel() * 4 + indptr.numel() * 8) / 1e6),
+                            edges_per_step=edges_rank / K),
+                clocks=clk,
+                e2e=dict(value=e2e_edges_all / e2e_s, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
+                         ms_per_step=e2e_s / K * 1e3),
+                gpu_launches=int(launches),
+                roofline=roof,
+                kernel_ms={TAP_NAMES[k].split(" (")[0]: v for k, v in tap_ms.items()})
+
+    if world == 1 and not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        sample = args.ref_seeds
+        dH64 = dH_h[:sample].astype(np.float64)
+        t0 = time.perf_counter()
+        ce, n = 0, 0
+        while n < K and time.perf_counter() - t0 < 15.0:
+            ce += oracle_step(w, indptr_h, indices_h, X_h, Ws_h, seeds_h[Wm + n][:sample], Wm + n, dH64)
+            n += 1
+        cdt = time.perf_counter() - t0
+        line["cpu_baseline"] = dict(value=ce / cdt, unit=UNIT, cores=1, kind="oracle",
+                                    sample=f"{n} step(s) on the first {sample} of the {w.batch} seeds of the batch, "
+                                           f"full sample+forward+backward, {cdt:.1f} s")
+    print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="medium", choices=sorted(S.WORKLOADS))
+    ap.add_argument("--ref-seeds", type=int, default=256, help="seeds per step given to the CPU oracle")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--seeds", default="activity", choices=["activity", "uniform"],
+                    help="how seed batches are drawn (see make_batches)")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    w = S.WORKLOADS[args.workload]
+    if args.impl == "reference":
+        run_reference(args, w)
+    else:
+        run_ours(args, w)
+
+
+if __name__ == "__main__":
+    main()

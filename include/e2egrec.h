@@ -107,6 +107,17 @@ typedef struct e2egrec_block {
 const char *e2egrec_status_string(int32_t code);
 const char *e2egrec_last_error(void);
 
+/* Benchmark instrumentation (no counterpart in the paper).
+ * e2egrec_launch_count: number of kernels this library has launched in this process so far.
+ * e2egrec_profile_tap: arms a timing tap on the calling thread.  The next entry point that reaches
+ * kernel group `which` records start_event (a cudaEvent_t) on its stream just before the group and
+ * stop_event just after it, then disarms the tap.  Groups: 1 = mean aggregation of the outermost
+ * block (layer 0, gathers from X), 2 = transposed aggregation of the outermost block (writes dX_rows),
+ * 3 = dense transform of layer 0, 4 = weight gradient of layer 0, 5 = input gradient (dCat) of layer 0,
+ * 6 = the whole of e2egrec_sample_khop.  which = 0 disarms. */
+uint64_t e2egrec_launch_count(void);
+int32_t e2egrec_profile_tap(int32_t which, void *start_event, void *stop_event);
+
 /* Worst-case capacities of the blocks of a k-hop sample and the scratch size
  * (Sec. 4.1: depth L, at most k neighbours per node).  fanouts: host int32[n_hops],
  * fanouts[0] is the hop taken from the seeds.  cap_dst / cap_src / cap_edges: host

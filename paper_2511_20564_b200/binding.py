@@ -75,8 +75,23 @@ def lib():
         L.e2egrec_sage_ctx_layout.restype = C.c_int32
         L.e2egrec_sage_ctx_layout.argtypes = [C.POINTER(Block), C.c_int32, C.POINTER(Mat), C.POINTER(Mat),
                                               C.c_void_p, C.c_void_p, C.c_void_p]
+        L.e2egrec_launch_count.restype = C.c_uint64
+        L.e2egrec_profile_tap.restype = C.c_int32
+        L.e2egrec_profile_tap.argtypes = [C.c_int32, C.c_void_p, C.c_void_p]
         _lib = L
     return _lib
+
+
+def launch_count() -> int:
+    return int(lib().e2egrec_launch_count())
+
+
+def profile_tap(which: int, start_event=None, stop_event=None):
+    """Arms the timing tap `which` with two torch.cuda.Event(enable_timing=True) that have been recorded
+    at least once (so that their CUDA handles exist); see e2egrec_profile_tap."""
+    a = None if start_event is None else C.c_void_p(start_event.cuda_event)
+    b = None if stop_event is None else C.c_void_p(stop_event.cuda_event)
+    _check(lib().e2egrec_profile_tap(which, a, b), "e2egrec_profile_tap")
 
 
 def status_string(code: int) -> str:
@@ -135,9 +150,10 @@ class Blocks:
         self.caps = list(zip(cd, cs, ce))
         self.t = []
         i32 = dict(dtype=torch.int32, device=device)
-        for d, s, e in self.caps:
+        self.counts = torch.zeros(len(self.caps), 4, **i32)    # row h: {n_dst, n_src, n_edges, status} of hop h+1
+        for h, (d, s, e) in enumerate(self.caps):
             self.t.append(dict(
-                counts=torch.zeros(4, **i32), indptr=torch.zeros(d + 1, **i32), col=torch.zeros(max(e, 1), **i32),
+                counts=self.counts[h], indptr=torch.zeros(d + 1, **i32), col=torch.zeros(max(e, 1), **i32),
                 nbr_global=torch.zeros(max(e, 1), **i32), src_nodes=torch.zeros(max(s, 1), **i32),
                 csc_ptr=torch.zeros(s + 1, **i32), csc_row=torch.zeros(max(e, 1), **i32),
                 csc_eid=torch.zeros(max(e, 1), **i32),

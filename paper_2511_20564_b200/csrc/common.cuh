@@ -24,6 +24,14 @@ inline size_t dtype_size(int32_t dtype) { return dtype == E2EGREC_BF16 ? 2 : 4; 
 // host side: remember the text of a failed launch for e2egrec_last_error()
 void set_last_error(const char *msg);
 int32_t check_launch(const char *what);
+// host side: every kernel launch is counted (e2egrec_launch_count)
+void note_launch();
+// host side: timing taps (e2egrec_profile_tap).  tap_begin/tap_end record the armed events around
+// kernel group `which` and disarm the tap.
+enum { TAP_AGG_FWD_OUTER = 1, TAP_AGG_BWD_OUTER = 2, TAP_UPDATE_FWD_OUTER = 3, TAP_DW_OUTER = 4, TAP_DCAT_OUTER = 5,
+       TAP_SAMPLE = 6 };
+void tap_begin(int which, cudaStream_t st);
+void tap_end(int which, cudaStream_t st);
 
 // ---------------------------------------------------------------------------------------
 // 16-byte row chunks: 8 bf16 or 4 fp32 values, accumulated in fp32.

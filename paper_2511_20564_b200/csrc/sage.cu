@@ -59,6 +59,7 @@ static void launch_sage_aggregate(const T *Hsrc, int64_t ld, const int32_t *nbr,
                                   const e2egrec_block &b, T *cat, int d, int64_t rows, cudaStream_t st)
 {
     const unsigned grid = (unsigned)std::max<int64_t>(1, ceil_div(rows * 32, kAggThreads));
+    note_launch();
     sage_aggregate_kernel<T, LPR, CPL><<<grid, kAggThreads, 0, st>>>(Hsrc, ld, nbr, self_ids, b.indptr, b.counts, cat, d,
                                                                       (int32_t)rows);
 }
@@ -81,9 +82,11 @@ static void launch_seg32(const T *in, int64_t ld_in, const int32_t *ptr, const i
                          const SegOut<T> &o, cudaStream_t st)
 {
     const int64_t n_chunks = ceil_div(cap_entries > 0 ? cap_entries : 1, chunk_len);
+    note_launch();
     seg_chunk_kernel<T, int32_t, LPR, CPL, false><<<(unsigned)ceil_div(n_chunks * 32, kAggThreads), kAggThreads, 0, st>>>(
         in, ld_in, ptr, idx, n_seg_dev, 0, nullptr, chunk_len, d, head, tail, o);
     const int64_t empty_blocks = ceil_div((cap_seg > 0 ? cap_seg : 1) * 8, kAggThreads);
+    note_launch();
     seg_finish_kernel<T, int32_t><<<(unsigned)(n_chunks + empty_blocks), kAggThreads, 0, st>>>(
         ptr, n_seg_dev, 0, chunk_len, d, head, tail, n_chunks, o);
 }
@@ -116,15 +119,18 @@ static int32_t forward_impl(const e2egrec_block *blocks, int32_t n_layers, const
         const e2egrec_block &b = blocks[p.block];
         T *cat = reinterpret_cast<T *>(ctx + p.cat_off);
         T *hn = reinterpret_cast<T *>(ctx + p.h_off);
-        if (l == 0)   // h^(0) rows are read straight from the feature table through the global ids
+        if (l == 0) {  // h^(0) rows are read straight from the feature table through the global ids
+            tap_begin(TAP_AGG_FWD_OUTER, st);
             dispatch_sage_aggregate<T>(static_cast<const T *>(X->data), X->ld, b.nbr_global, b.src_nodes, b, cat, p.d_in,
                                        p.rows, X->dtype, st);
-        else
+            tap_end(TAP_AGG_FWD_OUTER, st);
+        } else
             dispatch_sage_aggregate<T>(reinterpret_cast<const T *>(ctx + plan[l - 1].h_off), p.d_in, b.col, nullptr, b, cat,
                                        p.d_in, p.rows, X->dtype, st);
         const float *bl = bias ? bias[l] : nullptr;
         const int relu = act ? act[l] : 1;
         bool done = false;
+        if (l == 0) tap_begin(TAP_UPDATE_FWD_OUTER, st);
         if (X->dtype == E2EGREC_BF16)
             done = tc_update_forward(reinterpret_cast<const __nv_bfloat16 *>(cat), p.rows, 2 * p.d_in,
                                      static_cast<const __nv_bfloat16 *>(W[l].data), p.d_out, bl, relu,
@@ -132,10 +138,12 @@ static int32_t forward_impl(const e2egrec_block *blocks, int32_t n_layers, const
         if (!done) {
             EpiUpdate<T> epi{hn, p.d_out, bl, relu};
             dim3 grid((unsigned)std::max<int64_t>(1, ceil_div(p.rows, kGemmBM)), (unsigned)ceil_div(p.d_out, kGemmBN), 1);
+            note_launch();
             gemm_simt_kernel<T, false, false, EpiUpdate<T>><<<grid, kGemmThreads, 0, st>>>(
                 cat, 2 * p.d_in, static_cast<const T *>(W[l].data), 2 * p.d_in, p.rows, p.d_out, 2 * p.d_in,
                 &b.counts[CNT_DST], nullptr, epi);
         }
+        if (l == 0) tap_end(TAP_UPDATE_FWD_OUTER, st);
     }
     const LayerPlan &top = plan[n_layers - 1];
     const int64_t rows = blocks[0].cap_dst < H_out->rows ? blocks[0].cap_dst : H_out->rows;
@@ -192,6 +200,7 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
         const LayerPlan &p = plan[n_layers - 1];
         const e2egrec_block &b = blocks[p.block];
         const int64_t total = p.rows * p.d_out;
+        note_launch();
         relu_mask_kernel<T><<<(unsigned)std::max<int64_t>(1, ceil_div(total, 256)), 256, 0, st>>>(
             static_cast<const T *>(dH_out->data), dH_out->ld, reinterpret_cast<const T *>(ctx + p.h_off), p.d_out,
             &b.counts[CNT_DST], p.rows, p.d_out, act ? act[n_layers - 1] : 1, dz_buf[(n_layers - 1) & 1]);
@@ -204,23 +213,33 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
         const int32_t *n_dst = &b.counts[CNT_DST];
         const int two_d = 2 * p.d_in;
         // dW_l = dZ^T [h | agg]   (split over the rows, partial sums added in a fixed order)
+        if (l == 0) tap_begin(TAP_DW_OUTER, st);
         {
             EpiPartial epi{part, two_d, (int64_t)p.d_out * two_d};
             dim3 grid((unsigned)ceil_div(p.d_out, kGemmBM), (unsigned)ceil_div(two_d, kGemmBN), kDwSplits);
+            note_launch();
             gemm_simt_kernel<T, true, true, EpiPartial><<<grid, kGemmThreads, 0, st>>>(
                 dz, p.d_out, cat, two_d, p.d_out, two_d, p.rows, nullptr, n_dst, epi);
             const int64_t n = (int64_t)p.d_out * two_d;
+            note_launch();
             splitk_reduce_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(part, n, kDwSplits, accumulate, dW[l]);
         }
-        if (dbias && dbias[l])
-            colsum_kernel<T><<<(unsigned)ceil_div(p.d_out, 32), 256, 0, st>>>(dz, p.d_out, n_dst, p.d_out, accumulate, dbias[l]);
+        if (l == 0) tap_end(TAP_DW_OUTER, st);
+        if (dbias && dbias[l]) {
+            note_launch();
+            colsum_kernel<T><<<(unsigned)ceil_div(p.d_out, 32), 256, 0, st>>>(dz, p.d_out, n_dst, p.d_out, accumulate,
+                                                                             dbias[l]);
+        }
         // dCat = dZ W_l, the agg half scaled by 1/|S|
+        if (l == 0) tap_begin(TAP_DCAT_OUTER, st);
         {
             EpiDCat<T> epi{dcat, two_d, p.d_in, b.inv_cnt};
             dim3 grid((unsigned)std::max<int64_t>(1, ceil_div(p.rows, kGemmBM)), (unsigned)ceil_div(two_d, kGemmBN), 1);
+            note_launch();
             gemm_simt_kernel<T, false, true, EpiDCat<T>><<<grid, kGemmThreads, 0, st>>>(
                 dz, p.d_out, static_cast<const T *>(W[l].data), two_d, p.rows, two_d, p.d_out, n_dst, nullptr, epi);
         }
+        if (l == 0) tap_end(TAP_DCAT_OUTER, st);
         // transposed aggregation: gather over the block's CSC, plus the self rows, masked by the
         // activation of the layer below
         SegOut<T> o{};
@@ -239,8 +258,10 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
             o.ld_out = dX_rows->ld;
             o.mask = nullptr;
         }
+        if (l == 0) tap_begin(TAP_AGG_BWD_OUTER, st);
         dispatch_seg32<T>(dcat + p.d_in, two_d, b.csc_ptr, b.csc_row, &b.counts[CNT_SRC], b.cap_src, b.cap_edges,
                           kBlockChunk, p.d_in, head, tail, o, X->dtype, st);
+        if (l == 0) tap_end(TAP_AGG_BWD_OUTER, st);
     }
     return check_launch("sage_backward");
 }

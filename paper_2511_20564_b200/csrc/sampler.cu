@@ -329,8 +329,10 @@ static void sort_pass(const int32_t *kin, const int32_t *vin, int32_t *kout, int
                       int shift, int n_tiles, SamplerScratch &s, cudaStream_t st)
 {
     constexpr int R = 1 << BITS;
+    note_launch();
     sort_hist_kernel<BITS><<<n_tiles, kSortThreads, 0, st>>>(kin, counts, shift, n_tiles, s.hist);
     exclusive_scan<int32_t>(s.hist, s.hist_off, nullptr, (int64_t)R * n_tiles, (int64_t)R * n_tiles, s.scan_tmp, st);
+    note_launch();
     sort_scatter_kernel<BITS><<<n_tiles, kSortThreads, 0, st>>>(kin, vin, counts, shift, n_tiles, s.hist_off, kout, vout);
 }
 
@@ -420,6 +422,7 @@ extern "C" int32_t e2egrec_sampler_scratch_init(int64_t n_nodes, void *scratch, 
     SamplerScratch s = carve(n_nodes, 0, 0, 0, scratch);
     if (scratch_bytes < s.bytes) return E2EGREC_ERR_WORKSPACE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    note_launch();
     fill_i32_kernel<<<(unsigned)std::min<int64_t>(ceil_div(n_nodes > 0 ? n_nodes : 1, 256), 148 * 16), 256, 0, st>>>(
         s.local_id, n_nodes, -1);
     cudaMemsetAsync(s.bitmap, 0, sizeof(uint32_t) * (size_t)s.n_words, st);
@@ -457,32 +460,42 @@ extern "C" int32_t e2egrec_sample_khop(const e2egrec_csr *graph, const int32_t *
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int T = 256;
     const int64_t n = graph->n_nodes;
+    tap_begin(TAP_SAMPLE, st);
+    note_launch();
     seed_init_kernel<<<grid_for(n_seeds, T), T, 0, st>>>(seeds, n_seeds, n, s.local_id, blocks[0].counts);
     const int32_t *dst_nodes = seeds;
     const int32_t *n_dst_ptr = &blocks[0].counts[CNT_DST];
     for (int h = 0; h < n_hops; ++h) {
         const e2egrec_block &b = blocks[h];
         const int32_t f = fanouts[h];
+        note_launch();
         hop_count_kernel<<<grid_for(b.cap_dst, T), T, 0, st>>>(graph->indptr, n, dst_nodes, n_dst_ptr, b.cap_dst, f,
                                                               b.counts, s.cnt, b.inv_cnt, b.src_nodes, h == 0);
         exclusive_scan<int32_t>(s.cnt, b.indptr, &b.counts[CNT_DST], 0, b.cap_dst, s.scan_tmp, st);
+        note_launch();
         hop_draw_kernel<<<grid_for((int64_t)b.cap_dst * f, T), T, 0, st>>>(
             graph->indptr, graph->indices, n, b.src_nodes, b.indptr, b.counts, f, h + 1,
             (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), step, b.cap_edges, b.nbr_global, s.edge_row,
             s.local_id, s.bitmap);
+        note_launch();
         bitmap_popc_kernel<<<grid_for(s.n_words, T), T, 0, st>>>(s.bitmap, s.n_words, s.word_cnt);
         exclusive_scan<int32_t>(s.word_cnt, s.word_rank, nullptr, s.n_words, s.n_words, s.scan_tmp, st);
+        note_launch();
         frontier_assign_kernel<<<grid_for(s.n_words, T), T, 0, st>>>(s.bitmap, s.word_rank, s.n_words, b.counts,
                                                                     b.cap_src, s.local_id, b.src_nodes);
         cudaMemsetAsync(s.csc_cnt, 0, sizeof(int32_t) * (size_t)(b.cap_src + 1), st);
+        note_launch();
         relabel_kernel<<<grid_for(b.cap_edges, T), T, 0, st>>>(b.nbr_global, s.local_id, b.counts, b.col, s.csc_cnt);
         exclusive_scan<int32_t>(s.csc_cnt, b.csc_ptr, &b.counts[CNT_SRC], 0, b.cap_src, s.scan_tmp, st);
         sort_by_col(b, s, st);
+        note_launch();
         csc_rows_kernel<<<grid_for(b.cap_edges, T), T, 0, st>>>(b.csc_eid, s.edge_row, b.counts, b.csc_row);
         dst_nodes = b.src_nodes;
         n_dst_ptr = &b.counts[CNT_SRC];
     }
     const e2egrec_block &last = blocks[n_hops - 1];
+    note_launch();
     frontier_release_kernel<<<grid_for(last.cap_src, T), T, 0, st>>>(last.src_nodes, last.counts, s.local_id);
+    tap_end(TAP_SAMPLE, st);
     return check_launch("sample_khop");
 }

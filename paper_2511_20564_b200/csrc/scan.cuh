@@ -120,6 +120,7 @@ inline void exclusive_scan(const int32_t *in, OutT *out, const int32_t *n_dev, i
                            OutT *scratch, cudaStream_t st)
 {
     const int nb = (int)ceil_div(cap > 0 ? cap : 1, kScanTile);
+    note_launch(); note_launch(); note_launch();
     scan_reduce_kernel<OutT><<<nb, kScanThreads, 0, st>>>(in, n_dev, n_host, cap, scratch);
     scan_partials_kernel<OutT><<<1, 1024, 0, st>>>(scratch, nb);
     scan_final_kernel<OutT><<<nb, kScanThreads, 0, st>>>(in, out, n_dev, n_host, cap, scratch, nb);

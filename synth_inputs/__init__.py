@@ -101,6 +101,24 @@ def seed_batch(n: int, batch: int, seed: int, step: int) -> np.ndarray:
     return _rng(seed, 1000 + step).choice(n, size=batch, replace=False).astype(np.int32)
 
 
+def seed_batch_from_interactions(users: np.ndarray, items: np.ndarray, batch: int, seed: int, step: int) -> np.ndarray:
+    """`batch` distinct node ids met as endpoints of uniformly drawn interactions (users and items in
+    turn), so that a node enters a batch in proportion to its activity, as the source nodes of a
+    training example stream do."""
+    rng = _rng(seed, 2000 + step)
+    m = users.size
+    got = np.zeros(0, np.int32)
+    while got.size < batch:
+        idx = rng.integers(0, m, 4 * batch)
+        cand = np.empty(2 * idx.size, np.int32)
+        cand[0::2] = users[idx]
+        cand[1::2] = items[idx]
+        cand = np.concatenate([got, cand])
+        _, first = np.unique(cand, return_index=True)
+        got = cand[np.sort(first)]
+    return np.ascontiguousarray(got[:batch])
+
+
 def bernoulli_labels(n: int, p: float, seed: int, stream: int = 30) -> np.ndarray:
     return (_rng(seed, stream).random(n) < p).astype(np.float32)
 
