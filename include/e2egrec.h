@@ -58,6 +58,9 @@ extern "C" {
 #define E2EGREC_F32  0
 #define E2EGREC_BF16 1
 
+/* flags of e2egrec_aggregate_forward */
+#define E2EGREC_AGG_SUM 1u           /* plain sum instead of the mean */
+
 /* flags of e2egrec_sage_backward */
 #define E2EGREC_ACCUMULATE_DW 1u     /* add to dW / dbias instead of overwriting them */
 
@@ -191,6 +194,25 @@ int32_t e2egrec_sage_backward(const e2egrec_block *blocks, int32_t n_layers, con
                               const e2egrec_mat *dH_out, float *const *dW, float *const *dbias,
                               const e2egrec_mat *dX_rows, void *scratch, size_t *scratch_bytes,
                               uint32_t flags, void *stream);
+
+/* Whole-graph neighbourhood aggregation without sampling (Sec. 3.1 Eq. 2 with S(u) = N(u); the
+ * "complete graph" case of Sec. 4.1):  out[i] = (1/deg i) sum_{e in row i} X[indices[e]]  (0 for an
+ * empty row; the plain sum with E2EGREC_AGG_SUM).  indptr: device int64[n_dst+1], indices: device
+ * int32[n_entries]; X has a row for every id in indices; out has n_dst rows, same dtype and dim.
+ * Rows of any degree are split over many warps; partial sums are added in a fixed order (no atomics).
+ * ws: device scratch, 256-byte aligned (size query: ws == NULL). */
+int32_t e2egrec_aggregate_forward(int64_t n_dst, int64_t n_entries, const int64_t *indptr,
+                                  const int32_t *indices, const e2egrec_mat *X, const e2egrec_mat *out,
+                                  uint32_t flags, void *ws, size_t *ws_bytes, void *stream);
+
+/* Its transpose, run as a gather over the CSC form of the same matrix (Sec. 4.3.2: J^T applied to the
+ * incoming gradient):  dX[s] = sum_{k in column s} inv_deg[csc_row[k]] * G[csc_row[k]].
+ * csc_ptr: device int64[n_src+1], csc_row: device int32[n_entries] (the destination of each entry),
+ * inv_deg: device float[n_dst] = 1/deg (pass 1.0 everywhere for the transposed sum), G: gradient
+ * w.r.t. out, dX: n_src rows. */
+int32_t e2egrec_aggregate_backward(int64_t n_src, int64_t n_entries, const int64_t *csc_ptr,
+                                   const int32_t *csc_row, const float *inv_deg, const e2egrec_mat *G,
+                                   const e2egrec_mat *dX, void *ws, size_t *ws_bytes, void *stream);
 
 #ifdef __cplusplus
 }

@@ -75,6 +75,14 @@ def lib():
         L.e2egrec_sage_ctx_layout.restype = C.c_int32
         L.e2egrec_sage_ctx_layout.argtypes = [C.POINTER(Block), C.c_int32, C.POINTER(Mat), C.POINTER(Mat),
                                               C.c_void_p, C.c_void_p, C.c_void_p]
+        L.e2egrec_aggregate_forward.restype = C.c_int32
+        L.e2egrec_aggregate_forward.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.POINTER(Mat),
+                                                C.POINTER(Mat), C.c_uint32, C.c_void_p, C.POINTER(C.c_size_t),
+                                                C.c_void_p]
+        L.e2egrec_aggregate_backward.restype = C.c_int32
+        L.e2egrec_aggregate_backward.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
+                                                 C.POINTER(Mat), C.POINTER(Mat), C.c_void_p, C.POINTER(C.c_size_t),
+                                                 C.c_void_p]
         L.e2egrec_launch_count.restype = C.c_uint64
         L.e2egrec_profile_tap.restype = C.c_int32
         L.e2egrec_profile_tap.argtypes = [C.c_int32, C.c_void_p, C.c_void_p]
@@ -284,3 +292,41 @@ def sage_backward(blocks: Blocks, X, Ws, ctx, dH_out, acts=None, dWs=None, dbs=N
                                        _ptr_array(dbs, L), C.byref(dx), _ptr(scratch), C.byref(n),
                                        ACCUMULATE_DW if accumulate else 0, _stream(stream)), "e2egrec_sage_backward")
     return dWs, dX_rows
+
+
+# ------------------------------------------------------------------------------------------ whole graph
+
+def aggregate_forward(indptr, indices, X, out=None, ws=None, sum_only=False, stream=None):
+    """Enqueues out[i] = mean (or sum) of X[indices[row i]]; returns (out, ws)."""
+    n_dst, n_entries = indptr.numel() - 1, indices.numel()
+    if out is None:
+        out = torch.empty(max(n_dst, 1), X.shape[1], dtype=X.dtype, device=X.device)
+    x, o = _mat(X), _mat(out)
+    n = C.c_size_t(0)
+    if ws is None:
+        _check(lib().e2egrec_aggregate_forward(n_dst, n_entries, None, None, C.byref(x), C.byref(o), 0, None,
+                                               C.byref(n), None), "e2egrec_aggregate_forward(size query)")
+        ws = _dev_bytes(n.value, X.device)
+    n = C.c_size_t(ws.numel())
+    _check(lib().e2egrec_aggregate_forward(n_dst, n_entries, _ptr(indptr), _ptr(indices), C.byref(x), C.byref(o),
+                                           1 if sum_only else 0, _ptr(ws), C.byref(n), _stream(stream)),
+           "e2egrec_aggregate_forward")
+    return out, ws
+
+
+def aggregate_backward(csc_ptr, csc_row, inv_deg, G, dX=None, ws=None, stream=None):
+    """Enqueues dX[s] = sum over column s of inv_deg[r] * G[r]; returns (dX, ws)."""
+    n_src, n_entries = csc_ptr.numel() - 1, csc_row.numel()
+    if dX is None:
+        dX = torch.empty(max(n_src, 1), G.shape[1], dtype=G.dtype, device=G.device)
+    g, o = _mat(G), _mat(dX)
+    n = C.c_size_t(0)
+    if ws is None:
+        _check(lib().e2egrec_aggregate_backward(n_src, n_entries, None, None, None, C.byref(g), C.byref(o), None,
+                                                C.byref(n), None), "e2egrec_aggregate_backward(size query)")
+        ws = _dev_bytes(n.value, G.device)
+    n = C.c_size_t(ws.numel())
+    _check(lib().e2egrec_aggregate_backward(n_src, n_entries, _ptr(csc_ptr), _ptr(csc_row), _ptr(inv_deg),
+                                            C.byref(g), C.byref(o), _ptr(ws), C.byref(n), _stream(stream)),
+           "e2egrec_aggregate_backward")
+    return dX, ws

@@ -28,7 +28,8 @@ BF16_STEP = 2.0 ** -8
 def tolerance(want, bf16, terms_rss=None):
     """Per-element tolerance.
 
-    fp32 path: 1e-5 * max(|b|, rms(b)).
+    fp32 path: 1e-5 * max(|b|, rms(b), root-sum-square of the terms of the element's last reduction):
+    a long fp32 sum with cancellation is accurate relative to the scale of its terms, not of its result.
     bf16 path: 1e-3 + 2e-2 |b| + 2^-8 * sqrt(sum of squared terms of the element's last reduction).
     The last part covers operands that the two sides stored one bf16 step apart (a value within fp32
     rounding of the midpoint of two bf16 neighbours rounds differently after an fp32 or a float64 sum).
@@ -37,7 +38,10 @@ def tolerance(want, bf16, terms_rss=None):
     """
     want = np.asarray(want, np.float64)
     if not bf16:
-        return 1e-5 * np.maximum(np.abs(want), np.sqrt(np.mean(want ** 2)) if want.size else 0.0)
+        scale = np.maximum(np.abs(want), np.sqrt(np.mean(want ** 2)) if want.size else 0.0)
+        if terms_rss is not None:
+            scale = np.maximum(scale, terms_rss)
+        return 1e-5 * scale
     tol = 1e-3 + 2e-2 * np.abs(want)
     if terms_rss is not None:
         tol = tol + BF16_STEP * terms_rss

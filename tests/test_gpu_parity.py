@@ -148,3 +148,39 @@ def test_host_side_argument_errors():
     W = torch.zeros(8, 12, device="cuda")
     with pytest.raises(E.E2EGrecError):
         E.sage_forward(blocks, X, [W])
+
+
+# ----------------------------------------------------------------------------- whole-graph aggregation
+
+def _powerlaw_graph(n, m, seed):
+    dst, src = S.powerlaw_directed(n, m, 1.1, seed)
+    return S.coo_to_csr(n, dst, src)
+
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 64), ("f32", 32), ("bf16", 256)])
+def test_full_graph_aggregation_forward_and_transpose(dtype, d):
+    """Rows with tens of thousands of entries (split over many warps), empty rows, and a ragged tail."""
+    import paper_2511_20564_b200 as E
+    n, m = 20_011, 600_000
+    indptr, indices = _powerlaw_graph(n, m, 2)
+    assert np.diff(indptr).max() > 20_000 and (np.diff(indptr) == 0).any()
+    bf16 = dtype == "bf16"
+    dt = torch.bfloat16 if bf16 else torch.float32
+    X = S.normal_features(n, d, 5)
+    G = S.normal_features(n, d, 6, stream=11)
+    if bf16:
+        X, G = S.to_bf16_values(X), S.to_bf16_values(G)
+    ip, ix = torch.from_numpy(indptr).cuda(), torch.from_numpy(indices).cuda()
+    out, _ = E.aggregate_forward(ip, ix, torch.from_numpy(X).cuda().to(dt))
+    want = oracle.mean_aggregate(indptr, indices, X, bf16)
+    deg = np.diff(indptr).astype(np.float64)[:, None]
+    rss_f = np.sqrt(oracle.mean_aggregate(indptr, indices, X.astype(np.float64) ** 2) / np.maximum(deg, 1))
+    assert_close("aggregate_forward", out.float().cpu().numpy()[:n], want, bf16, rss_f)
+    # transpose through the oracle-built CSC
+    cptr, crow, _ = oracle.csr_transpose(n, n, indptr, indices)
+    inv_deg = np.where(deg[:, 0] > 0, 1.0 / np.maximum(deg[:, 0], 1), 0.0).astype(np.float32)
+    dX, _ = E.aggregate_backward(torch.from_numpy(cptr).cuda(), torch.from_numpy(crow).cuda(),
+                                 torch.from_numpy(inv_deg).cuda(), torch.from_numpy(G).cuda().to(dt))
+    want = oracle.full_aggregate_backward(indptr, indices, n, G, bf16)
+    rss_b = np.sqrt(oracle.full_aggregate_backward(indptr, indices, n, G.astype(np.float64) ** 2 / np.maximum(deg, 1)))
+    assert_close("aggregate_backward", dX.float().cpu().numpy()[:n], want, bf16, rss_b)
