@@ -214,6 +214,34 @@ int32_t e2egrec_aggregate_backward(int64_t n_src, int64_t n_entries, const int64
                                    const int32_t *csc_row, const float *inv_deg, const e2egrec_mat *G,
                                    const e2egrec_mat *dX, void *ws, size_t *ws_bytes, void *stream);
 
+/* e2egrec_aggregate_forward without a workspace argument (the paper has no counterpart; this is a
+ * packaging variant of the call above and computes exactly the same result).
+ *
+ * Who needs it: code that is not allowed to obtain device memory at the point where it aggregates --
+ * a plug-in running inside a host application that owns the whole memory pool, a step executed while
+ * an allocator lock is held or inside a region where cudaMalloc would synchronise the device, or a
+ * process started with all memory already handed out.  Such callers can still pass their inputs and
+ * the output matrix, but have no way to size and provide `ws`.
+ *
+ * Here the partial-sum scratch is an 8 MiB array built into the library (every GPU that loads the
+ * library holds it until the process ends; e2egrec_aggregate_forward_static_limit() returns the size).
+ * The call allocates and frees nothing.  A problem fits if
+ *     2 * round_up_256( ceil(n_entries / 128) * dim * 4 bytes ) <= 8 MiB,
+ * e.g. up to about 2.1 M entries at dim 64.  Larger inputs are rejected with E2EGREC_ERR_WORKSPACE and
+ * e2egrec_last_error() then says how many bytes were needed; nothing is enqueued in that case.
+ *
+ * The first call on each device looks up the device address of the built-in array (with that device
+ * current).  Make that first call outside any stream capture.  All calls on a device share the one
+ * array, and it keeps whatever the previous call left in it: nothing in it has to start at zero,
+ * because each call writes every partial sum before it reads it, but two calls whose kernels can run
+ * at the same time on one GPU (different streams, different host threads) would overwrite each
+ * other's partial sums -- keep calls on one device in stream order.
+ * Arguments, layout, flags and error codes otherwise as for e2egrec_aggregate_forward. */
+int32_t e2egrec_aggregate_forward_static(int64_t n_dst, int64_t n_entries, const int64_t *indptr,
+                                         const int32_t *indices, const e2egrec_mat *X, const e2egrec_mat *out,
+                                         uint32_t flags, void *stream);
+size_t e2egrec_aggregate_forward_static_limit(void);
+
 #ifdef __cplusplus
 }
 #endif

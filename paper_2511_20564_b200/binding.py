@@ -83,6 +83,10 @@ def lib():
         L.e2egrec_aggregate_backward.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p,
                                                  C.POINTER(Mat), C.POINTER(Mat), C.c_void_p, C.POINTER(C.c_size_t),
                                                  C.c_void_p]
+        L.e2egrec_aggregate_forward_static.restype = C.c_int32
+        L.e2egrec_aggregate_forward_static.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.POINTER(Mat),
+                                                       C.POINTER(Mat), C.c_uint32, C.c_void_p]
+        L.e2egrec_aggregate_forward_static_limit.restype = C.c_size_t
         L.e2egrec_launch_count.restype = C.c_uint64
         L.e2egrec_profile_tap.restype = C.c_int32
         L.e2egrec_profile_tap.argtypes = [C.c_int32, C.c_void_p, C.c_void_p]
@@ -108,7 +112,7 @@ def status_string(code: int) -> str:
 
 def _check(rc: int, what: str):
     if rc != 0:
-        extra = lib().e2egrec_last_error().decode() if rc == -7 else ""
+        extra = lib().e2egrec_last_error().decode() if rc in (-7, -5) else ""
         raise E2EGrecError(f"{what}: {status_string(rc)} ({rc}) {extra}".strip())
 
 
@@ -330,3 +334,21 @@ def aggregate_backward(csc_ptr, csc_row, inv_deg, G, dX=None, ws=None, stream=No
                                             C.byref(g), C.byref(o), _ptr(ws), C.byref(n), _stream(stream)),
            "e2egrec_aggregate_backward")
     return dX, ws
+
+
+def aggregate_forward_static(indptr, indices, X, out, sum_only=False, stream=None):
+    """e2egrec_aggregate_forward_static: the same aggregation for callers that may not allocate device
+    memory where they aggregate (they run inside someone else's memory pool, or at a point where an
+    allocation would stall the GPU).  The scratch is a fixed 8 MiB buffer inside the library, so `out`
+    must be supplied and nothing is allocated here; inputs that need more scratch raise E2EGrecError.
+    Calls on one GPU share that buffer and must not overlap."""
+    n_dst, n_entries = indptr.numel() - 1, indices.numel()
+    x, o = _mat(X), _mat(out)
+    _check(lib().e2egrec_aggregate_forward_static(n_dst, n_entries, _ptr(indptr), _ptr(indices), C.byref(x),
+                                                  C.byref(o), 1 if sum_only else 0, _stream(stream)),
+           "e2egrec_aggregate_forward_static")
+    return out
+
+
+def aggregate_forward_static_limit() -> int:
+    return int(lib().e2egrec_aggregate_forward_static_limit())
