@@ -1,11 +1,358 @@
+// bf16 dense products on the 5th-generation tensor cores (tcgen05) of sm_100a.
+//
+//   D[m, n] = sum_k A[m, k] * B[n, k]        A: [rows x K] row-major, B: [N x K] row-major (both K-major)
+//
+// One CTA computes a 128 x NT tile (NT = min(N, 256)).  A single thread feeds TMA loads of
+// 128 x 64 (A) and NT x 64 (B) bf16 boxes into a ring of 128-byte-swizzled shared-memory stages,
+// a single thread issues tcgen05.mma (M = 128, N = NT, K = 16 per instruction) into an fp32
+// accumulator in tensor memory, and all four warps read the accumulator back with tcgen05.ld for
+// the epilogue (bias / ReLU / per-row scale, bf16 store).  No cluster launch, no multicast.
+// Every mbarrier wait is bounded; on a timeout the CTA raises E2EGREC_DEV_TIMEOUT in the status
+// word, skips its stores, releases its tensor memory and returns.
 #include "gemm_tc.cuh"
+
+#include <cuda.h>
 
 namespace e2egrec {
 
-bool tc_update_forward(const __nv_bfloat16 *, int64_t, int, const __nv_bfloat16 *, int, const float *, int,
-                       __nv_bfloat16 *, const int32_t *, cudaStream_t)
+namespace {
+
+constexpr int kTileM = 128;
+constexpr int kTileK = 64;                 // 64 bf16 = one 128-byte swizzle row
+constexpr int kUmmaK = 16;
+constexpr int kThreads = 128;
+constexpr int kMaxStages = 4;
+constexpr uint32_t kSpinLimit = 4u * 1000u * 1000u;
+
+// ------------------------------------------------------------------------- PTX wrappers
+__device__ inline uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ inline void mbar_init(uint64_t *bar, uint32_t count)
 {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+
+__device__ inline void mbar_expect_tx(uint64_t *bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+
+// Bounded wait for the phase with the given parity; false when the limit ran out or another
+// thread of the CTA has already given up.
+__device__ inline bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag)
+{
+    const uint32_t addr = smem_u32(bar);
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        uint32_t done;
+        asm volatile(
+            "{\n"
+            ".reg .pred p;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+            "selp.u32 %0, 1, 0, p;\n"
+            "}\n"
+            : "=r"(done)
+            : "r"(addr), "r"(parity)
+            : "memory");
+        if (done) return true;
+        if ((it & 1023u) == 1023u && *abort_flag) return false;
+    }
+    *abort_flag = 1;
     return false;
+}
+
+__device__ inline void tma_load_2d(void *smem_dst, const CUtensorMap *map, int x, int y, uint64_t *bar)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
+        : "memory");
+}
+
+__device__ inline void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ inline void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// Shared-memory operand descriptor: K-major tile of 128-byte rows, 128-byte swizzle.  Eight rows
+// form one 1024-byte swizzle atom, so the stride between 8-row groups is 1024 bytes; the leading
+// byte offset is not used for this layout.
+__device__ inline uint64_t make_smem_desc(uint32_t smem_addr)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);        // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                               // leading byte offset (ignored, canonical 1)
+    d |= (uint64_t)(1024 >> 4) << 32;                     // stride byte offset
+    d |= (uint64_t)1 << 46;                               // descriptor version of sm_100
+    d |= (uint64_t)2 << 61;                               // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor of kind::f16: bf16 x bf16 -> fp32, both operands K-major.
+__device__ inline uint32_t make_idesc(int m, int n)
+{
+    uint32_t d = 0;
+    d |= 1u << 4;                    // accumulator fp32
+    d |= 1u << 7;                    // A bf16
+    d |= 1u << 10;                   // B bf16
+    d |= (uint32_t)(n >> 3) << 17;
+    d |= (uint32_t)(m >> 4) << 24;
+    return d;
+}
+
+__device__ inline void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n"
+        ".reg .pred p;\n"
+        "setp.ne.b32 p, %4, 0;\n"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n"
+        "}\n" ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+
+__device__ inline void umma_commit(uint64_t *bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar))
+                 : "memory");
+}
+
+__device__ inline void tmem_load32(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+struct TcEpilogue {
+    __nv_bfloat16 *out;        // [rows x ldo]
+    int64_t ldo;
+    const float *bias;         // per output column, optional
+    int relu;
+    const float *row_scale;    // optional: columns >= scale_from are multiplied by row_scale[row]
+    int scale_from;
+    const int32_t *m_dev;      // rows at and beyond *m_dev are written as zeros
+    int32_t *status;           // device status word (E2EGREC_DEV_TIMEOUT)
+};
+
+// ------------------------------------------------------------------------- kernel
+__global__ void __launch_bounds__(kThreads)
+tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int k_blocks,
+                  int stages, int nt, uint32_t tmem_cols, TcEpilogue ep)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], accum_bar;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int64_t m0 = (int64_t)blockIdx.x * kTileM;
+    const int n0 = blockIdx.y * nt;
+    const int32_t m_valid = *ep.m_dev;
+    if (m0 >= m_valid) {                       // nothing but padding in this tile: rows stay as they are
+        return;
+    }
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    const uint32_t a_bytes = kTileM * kTileK * 2, b_bytes = (uint32_t)nt * kTileK * 2;
+    uint8_t *a_tiles = tiles;
+    uint8_t *b_tiles = tiles + (size_t)stages * a_bytes;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        mbar_init(&accum_bar, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {                            // tensor memory for the accumulator: tmem_cols fp32 columns x 128 lanes
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                     "r"(tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    int issued = 0;                             // k-blocks whose loads the producer has started
+    if (warp == 0 && lane == 0) {
+        // ---- producer: TMA loads into the stage ring
+        for (int kb = 0; kb < k_blocks; ++kb) {
+            const int s = kb % stages;
+            const uint32_t ph = (uint32_t)(kb / stages) & 1u;
+            if (!mbar_wait(&empty_bar[s], ph ^ 1u, &abort_flag)) break;
+            mbar_expect_tx(&full_bar[s], a_bytes + b_bytes);
+            tma_load_2d(a_tiles + (size_t)s * a_bytes, &map_a, kb * kTileK, (int)m0, &full_bar[s]);
+            tma_load_2d(b_tiles + (size_t)s * b_bytes, &map_b, kb * kTileK, n0, &full_bar[s]);
+            issued = kb + 1;
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---- MMA issuer
+        const uint32_t idesc = make_idesc(kTileM, nt);
+        bool ok = true;
+        for (int kb = 0; kb < k_blocks && ok; ++kb) {
+            const int s = kb % stages;
+            const uint32_t ph = (uint32_t)(kb / stages) & 1u;
+            ok = mbar_wait(&full_bar[s], ph, &abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t a_addr = smem_u32(a_tiles + (size_t)s * a_bytes);
+            const uint32_t b_addr = smem_u32(b_tiles + (size_t)s * b_bytes);
+#pragma unroll
+            for (int k = 0; k < kTileK / kUmmaK; ++k) {
+                const uint64_t ad = make_smem_desc(a_addr + k * kUmmaK * 2);
+                const uint64_t bd = make_smem_desc(b_addr + k * kUmmaK * 2);
+                umma(tmem_base, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+            }
+            umma_commit(&empty_bar[s]);         // the stage is free again once these MMAs have read it
+        }
+        if (ok) umma_commit(&accum_bar);        // accumulator complete
+    }
+    __syncwarp();
+
+    // ---- epilogue: warp w owns accumulator lanes 32w .. 32w+31 = rows m0 + 32w + lane
+    const bool ready = mbar_wait(&accum_bar, 0, &abort_flag);
+    tc_fence_after();
+    if (ready) {
+        const int64_t row = m0 + warp * 32 + lane;
+        const bool live = row < m_valid;
+        const float rs = (ep.row_scale && live) ? ep.row_scale[row] : 1.f;
+        __nv_bfloat16 *orow = ep.out + row * ep.ldo + n0;
+        for (int c = 0; c < nt; c += 32) {
+            uint32_t r[32];
+            tmem_load32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, r);
+            uint32_t packed[16];
+#pragma unroll
+            for (int j = 0; j < 32; j += 2) {
+                float v0 = __uint_as_float(r[j]), v1 = __uint_as_float(r[j + 1]);
+                const int col = n0 + c + j;
+                if (ep.bias) { v0 += ep.bias[col]; v1 += ep.bias[col + 1]; }
+                if (ep.relu) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
+                if (ep.row_scale) {
+                    if (col >= ep.scale_from) v0 *= rs;
+                    if (col + 1 >= ep.scale_from) v1 *= rs;
+                }
+                if (!live) { v0 = 0.f; v1 = 0.f; }
+                __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+                packed[j >> 1] = *reinterpret_cast<uint32_t *>(&h);
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                *reinterpret_cast<uint4 *>(orow + c + q * 8) =
+                    make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+        }
+    } else if (threadIdx.x == 0) {
+        atomicOr(reinterpret_cast<unsigned *>(ep.status), E2EGREC_DEV_TIMEOUT);
+        // giving up: let the copies that were started land before the shared memory is released
+        int never = 0;
+        for (int kb = issued > stages ? issued - stages : 0; kb < issued; ++kb)
+            mbar_wait(&full_bar[kb % stages], (uint32_t)(kb / stages) & 1u, &never);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = []() -> EncodeTiledFn {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+            q != cudaDriverEntryPointSuccess)
+            return nullptr;
+        return reinterpret_cast<EncodeTiledFn>(p);
+    }();
+    return fn;
+}
+
+// [rows x k] bf16 row-major, box = 64 x box_rows, 128-byte swizzle
+bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t k, int64_t ld, int box_rows)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)k, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kTileK, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool launch_tn(const __nv_bfloat16 *A, int64_t rows, int k, int64_t lda, const __nv_bfloat16 *B, int n, int64_t ldb,
+               const TcEpilogue &ep, cudaStream_t st)
+{
+    if (rows <= 0 || rows % kTileM || k % kTileK || k < kTileK) return false;
+    const int nt = n > 256 ? 256 : n;
+    if (n % nt || nt % 32 || nt < 32) return false;
+    if (reinterpret_cast<uintptr_t>(A) % 16 || reinterpret_cast<uintptr_t>(B) % 16 || (lda * 2) % 16 || (ldb * 2) % 16 ||
+        reinterpret_cast<uintptr_t>(ep.out) % 16 || (ep.ldo * 2) % 16)
+        return false;
+    CUtensorMap ma, mb;
+    if (!make_map(&ma, A, rows, k, lda, kTileM) || !make_map(&mb, B, n, k, ldb, nt)) return false;
+    const int k_blocks = k / kTileK;
+    const int stages = k_blocks < kMaxStages ? k_blocks : kMaxStages;
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < nt) tmem_cols <<= 1;
+    const size_t smem = (size_t)stages * (kTileM * kTileK * 2 + (size_t)nt * kTileK * 2) + 1024;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(tc_gemm_tn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
+            return false;
+        attr_set = true;
+    }
+    dim3 grid((unsigned)(rows / kTileM), (unsigned)(n / nt), 1);
+    note_launch();
+    tc_gemm_tn_kernel<<<grid, kThreads, smem, st>>>(ma, mb, k_blocks, stages, nt, tmem_cols, ep);
+    return true;
+}
+
+}  // namespace
+
+bool tc_update_forward(const __nv_bfloat16 *cat, int64_t rows, int k, const __nv_bfloat16 *W, int n, const float *bias,
+                       int relu, __nv_bfloat16 *out, const int32_t *m_dev, int32_t *status, cudaStream_t st)
+{
+    TcEpilogue ep{};
+    ep.out = out;
+    ep.ldo = n;
+    ep.bias = bias;
+    ep.relu = relu;
+    ep.row_scale = nullptr;
+    ep.scale_from = 0;
+    ep.m_dev = m_dev;
+    ep.status = status;
+    return launch_tn(cat, rows, k, k, W, n, k, ep, st);
+}
+
+bool tc_dcat_backward(const __nv_bfloat16 *dz, int64_t rows, int d_out, const __nv_bfloat16 *Wt, int two_d_in,
+                      const float *inv_cnt, __nv_bfloat16 *dcat, const int32_t *m_dev, int32_t *status, cudaStream_t st)
+{
+    TcEpilogue ep{};
+    ep.out = dcat;
+    ep.ldo = two_d_in;
+    ep.bias = nullptr;
+    ep.relu = 0;
+    ep.row_scale = inv_cnt;
+    ep.scale_from = two_d_in / 2;
+    ep.m_dev = m_dev;
+    ep.status = status;
+    return launch_tn(dz, rows, d_out, d_out, Wt, two_d_in, d_out, ep, st);
 }
 
 }  // namespace e2egrec

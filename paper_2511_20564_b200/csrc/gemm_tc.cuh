@@ -1,14 +1,20 @@
-// Tensor-core (tcgen05) dense transform for bf16 operands.
+// Tensor-core (tcgen05) dense products for bf16 operands.
 #pragma once
 
 #include "common.cuh"
 
 namespace e2egrec {
 
-// h' = act(cat W^T + b) for `rows` (a multiple of 128) rows of cat [rows x k] and W [n x k], both
-// bf16 row-major; rows at and beyond *m_dev are written as zeros.  Returns false when the shape is
-// outside what the kernel takes, in which case nothing was enqueued.
+// h' = act(cat W^T + b) for `rows` (a multiple of 128) rows of cat [rows x k] and W [n x k], both bf16
+// row-major; rows at and beyond *m_dev inside a partly used 128-row tile are written as zeros, tiles
+// wholly beyond it are left alone.  `status` receives E2EGREC_DEV_TIMEOUT if a bounded wait runs out.
+// Returns false when the shape is outside what the kernel takes, in which case nothing was enqueued.
 bool tc_update_forward(const __nv_bfloat16 *cat, int64_t rows, int k, const __nv_bfloat16 *W, int n, const float *bias,
-                       int relu, __nv_bfloat16 *out, const int32_t *m_dev, cudaStream_t st);
+                       int relu, __nv_bfloat16 *out, const int32_t *m_dev, int32_t *status, cudaStream_t st);
+
+// dCat = dZ Wt^T with Wt [2 d_in x d_out] (the transposed layer weight); columns >= d_in are scaled by
+// inv_cnt[row].  Same conventions as above.
+bool tc_dcat_backward(const __nv_bfloat16 *dz, int64_t rows, int d_out, const __nv_bfloat16 *Wt, int two_d_in,
+                      const float *inv_cnt, __nv_bfloat16 *dcat, const int32_t *m_dev, int32_t *status, cudaStream_t st);
 
 }  // namespace e2egrec

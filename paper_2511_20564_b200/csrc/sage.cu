@@ -134,7 +134,7 @@ static int32_t forward_impl(const e2egrec_block *blocks, int32_t n_layers, const
         if (X->dtype == E2EGREC_BF16)
             done = tc_update_forward(reinterpret_cast<const __nv_bfloat16 *>(cat), p.rows, 2 * p.d_in,
                                      static_cast<const __nv_bfloat16 *>(W[l].data), p.d_out, bl, relu,
-                                     reinterpret_cast<__nv_bfloat16 *>(hn), &b.counts[CNT_DST], st);
+                                     reinterpret_cast<__nv_bfloat16 *>(hn), &b.counts[CNT_DST], &b.counts[CNT_STATUS], st);
         if (!done) {
             EpiUpdate<T> epi{hn, p.d_out, bl, relu};
             dim3 grid((unsigned)std::max<int64_t>(1, ceil_div(p.rows, kGemmBM)), (unsigned)ceil_div(p.d_out, kGemmBN), 1);
@@ -155,18 +155,32 @@ static int32_t forward_impl(const e2egrec_block *blocks, int32_t n_layers, const
 
 // ------------------------------------------------------------------------------ backward
 struct BackwardScratch {
-    size_t dz_off[2], dcat_off, head_off, tail_off, part_off, bytes;
+    size_t dz_off[2], dcat_off, head_off, tail_off, part_off, wt_off, bytes;
 };
+
+// Wt[j][o] = W[o][j]: the dCat product reads the layer weight with d_out as the contraction index.
+template <typename T>
+__global__ void transpose_kernel(const T *__restrict__ W, int rows, int cols, T *__restrict__ Wt)
+{
+    __shared__ T tile[32][33];
+    const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+    for (int i = threadIdx.y; i < 32; i += blockDim.y)
+        if (r0 + i < rows && c0 + threadIdx.x < cols) tile[i][threadIdx.x] = W[(int64_t)(r0 + i) * cols + c0 + threadIdx.x];
+    __syncthreads();
+    for (int i = threadIdx.y; i < 32; i += blockDim.y)
+        if (c0 + i < cols && r0 + threadIdx.x < rows) Wt[(int64_t)(c0 + i) * rows + r0 + threadIdx.x] = tile[threadIdx.x][i];
+}
 
 static BackwardScratch plan_backward(const e2egrec_block *blocks, int32_t n_layers, const LayerPlan *plan, size_t es)
 {
     BackwardScratch s{};
-    size_t dz = 0, dcat = 0, part = 0, ht = 0;
+    size_t dz = 0, dcat = 0, part = 0, ht = 0, wt = 0;
     for (int l = 0; l < n_layers; ++l) {
         const LayerPlan &p = plan[l];
         dz = std::max(dz, (size_t)p.rows * p.d_out * es);
         dcat = std::max(dcat, (size_t)p.rows * 2 * p.d_in * es);
         part = std::max(part, (size_t)kDwSplits * p.d_out * 2 * p.d_in * sizeof(float));
+        wt = std::max(wt, (size_t)p.d_out * 2 * p.d_in * es);
         const int64_t n_chunks = ceil_div(std::max(blocks[p.block].cap_edges, 1), kBlockChunk);
         ht = std::max(ht, (size_t)n_chunks * p.d_in * sizeof(float));
     }
@@ -178,6 +192,7 @@ static BackwardScratch plan_backward(const e2egrec_block *blocks, int32_t n_laye
     s.head_off = take(ht);
     s.tail_off = take(ht);
     s.part_off = take(part);
+    s.wt_off = take(wt);
     s.bytes = off;
     return s;
 }
@@ -232,7 +247,16 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
         }
         // dCat = dZ W_l, the agg half scaled by 1/|S|
         if (l == 0) tap_begin(TAP_DCAT_OUTER, st);
-        {
+        bool dcat_done = false;
+        if (X->dtype == E2EGREC_BF16) {
+            __nv_bfloat16 *wt = reinterpret_cast<__nv_bfloat16 *>(scratch + bs.wt_off);
+            note_launch();
+            transpose_kernel<__nv_bfloat16><<<dim3((unsigned)ceil_div(two_d, 32), (unsigned)ceil_div(p.d_out, 32)), dim3(32, 8), 0, st>>>(
+                static_cast<const __nv_bfloat16 *>(W[l].data), p.d_out, two_d, wt);
+            dcat_done = tc_dcat_backward(reinterpret_cast<const __nv_bfloat16 *>(dz), p.rows, p.d_out, wt, two_d, b.inv_cnt,
+                                         reinterpret_cast<__nv_bfloat16 *>(dcat), n_dst, &b.counts[CNT_STATUS], st);
+        }
+        if (!dcat_done) {
             EpiDCat<T> epi{dcat, two_d, p.d_in, b.inv_cnt};
             dim3 grid((unsigned)std::max<int64_t>(1, ceil_div(p.rows, kGemmBM)), (unsigned)ceil_div(two_d, kGemmBN), 1);
             note_launch();
