@@ -3,45 +3,25 @@
 // shared by many warps.
 #include <algorithm>
 
-#include "aggregate.cuh"
+#include "segreduce.cuh"
 
 namespace e2egrec {
 
-static inline int full_chunk_len(int64_t n_entries) { return n_entries > (1ll << 24) ? 256 : 128; }
+static inline int full_run_len(int64_t n_entries) { return n_entries > (1ll << 24) ? 64 : 32; }
 
 static size_t full_ws_bytes(int64_t n_entries, int d)
 {
-    const int64_t n_chunks = ceil_div(n_entries > 0 ? n_entries : 1, full_chunk_len(n_entries));
-    return 2 * align_up((size_t)n_chunks * d * sizeof(float), 256);
-}
-
-template <typename T, int LPR, int CPL, bool kWeight>
-static void launch_seg64(const T *in, int64_t ld_in, const int64_t *ptr, const int32_t *idx, int64_t n_seg,
-                         int64_t n_entries, const float *w, int d, float *head, float *tail, const SegOut<T> &o,
-                         cudaStream_t st)
-{
-    const int chunk_len = full_chunk_len(n_entries);
-    const int64_t n_chunks = ceil_div(n_entries > 0 ? n_entries : 1, chunk_len);
-    note_launch();
-    seg_chunk_kernel<T, int64_t, LPR, CPL, kWeight><<<(unsigned)ceil_div(n_chunks * 32, kAggThreads), kAggThreads, 0, st>>>(
-        in, ld_in, ptr, idx, nullptr, n_seg, w, chunk_len, d, head, tail, o);
-    const int64_t empty_blocks = ceil_div((n_seg > 0 ? n_seg : 1) * 8, kAggThreads);
-    note_launch();
-    seg_finish_kernel<T, int64_t><<<(unsigned)(n_chunks + empty_blocks), kAggThreads, 0, st>>>(
-        ptr, nullptr, n_seg, chunk_len, d, head, tail, n_chunks, o);
+    return seg_scratch_carve(n_entries, full_run_len(n_entries), d, nullptr).bytes;
 }
 
 template <typename T, bool kWeight>
 static void dispatch_seg64(const T *in, int64_t ld_in, const int64_t *ptr, const int32_t *idx, int64_t n_seg,
-                           int64_t n_entries, const float *w, int d, float *head, float *tail, const SegOut<T> &o,
-                           int32_t dtype, cudaStream_t st)
+                           int64_t n_entries, const float *w, int d, void *ws, const SegOut<T> &o, int32_t dtype,
+                           cudaStream_t st)
 {
-    const RowShape rs = row_shape(d, dtype);
-#define E2E_CASE(L, C)                                                                                               \
-    if (rs.lpr == L && rs.cpl == C)                                                                                  \
-        return launch_seg64<T, L, C, kWeight>(in, ld_in, ptr, idx, n_seg, n_entries, w, d, head, tail, o, st);
-    E2E_CASE(4, 1) E2E_CASE(8, 1) E2E_CASE(16, 1) E2E_CASE(32, 1) E2E_CASE(32, 2) E2E_CASE(32, 4)
-#undef E2E_CASE
+    const int run_len = full_run_len(n_entries);
+    const SegScratch sc = seg_scratch_carve(n_entries, run_len, d, ws);
+    dispatch_seg_reduce<T, int64_t, kWeight>(in, ld_in, ptr, idx, nullptr, n_seg, n_seg, w, run_len, d, dtype, sc, o, st);
 }
 
 static int32_t check_mats(const e2egrec_mat *in, const e2egrec_mat *out, int64_t out_rows)
@@ -58,10 +38,9 @@ static int32_t check_mats(const e2egrec_mat *in, const e2egrec_mat *out, int64_t
     return E2EGREC_OK;
 }
 
-// Shared body of the two entry points (and of the variant that brings its own scratch).
-int32_t full_aggregate(int64_t n_seg, int64_t n_entries, const int64_t *ptr, const int32_t *idx, const float *w,
-                       const e2egrec_mat *in, const e2egrec_mat *out, int mean, float *head, float *tail,
-                       cudaStream_t st)
+// Shared body of the two entry points.
+static int32_t full_aggregate(int64_t n_seg, int64_t n_entries, const int64_t *ptr, const int32_t *idx, const float *w,
+                       const e2egrec_mat *in, const e2egrec_mat *out, int mean, void *ws, cudaStream_t st)
 {
     if (in->dtype == E2EGREC_BF16) {
         using T = __nv_bfloat16;
@@ -70,9 +49,9 @@ int32_t full_aggregate(int64_t n_seg, int64_t n_entries, const int64_t *ptr, con
         o.ld_out = out->ld;
         o.mean = mean;
         if (w) dispatch_seg64<T, true>(static_cast<const T *>(in->data), in->ld, ptr, idx, n_seg, n_entries, w, in->dim,
-                                       head, tail, o, in->dtype, st);
+                                       ws, o, in->dtype, st);
         else dispatch_seg64<T, false>(static_cast<const T *>(in->data), in->ld, ptr, idx, n_seg, n_entries, w, in->dim,
-                                      head, tail, o, in->dtype, st);
+                                      ws, o, in->dtype, st);
     } else {
         using T = float;
         SegOut<T> o{};
@@ -80,14 +59,13 @@ int32_t full_aggregate(int64_t n_seg, int64_t n_entries, const int64_t *ptr, con
         o.ld_out = out->ld;
         o.mean = mean;
         if (w) dispatch_seg64<T, true>(static_cast<const T *>(in->data), in->ld, ptr, idx, n_seg, n_entries, w, in->dim,
-                                       head, tail, o, in->dtype, st);
+                                       ws, o, in->dtype, st);
         else dispatch_seg64<T, false>(static_cast<const T *>(in->data), in->ld, ptr, idx, n_seg, n_entries, w, in->dim,
-                                      head, tail, o, in->dtype, st);
+                                      ws, o, in->dtype, st);
     }
     return check_launch("aggregate");
 }
 
-size_t full_aggregate_ws(int64_t n_entries, int d) { return full_ws_bytes(n_entries, d); }
 
 }  // namespace e2egrec
 
@@ -107,9 +85,7 @@ static int32_t aggregate_entry(int64_t n_seg, int64_t n_entries, const int64_t *
     if (*ws_bytes < need) { *ws_bytes = need; return E2EGREC_ERR_WORKSPACE; }
     if (reinterpret_cast<uintptr_t>(ws) % 256) return E2EGREC_ERR_ALIGN;
     if (!ptr || (n_entries > 0 && !idx)) return E2EGREC_ERR_NULL;
-    float *head = static_cast<float *>(ws);
-    float *tail = reinterpret_cast<float *>(static_cast<char *>(ws) + need / 2);
-    return full_aggregate(n_seg, n_entries, ptr, idx, w, in, out, mean, head, tail, static_cast<cudaStream_t>(stream));
+    return full_aggregate(n_seg, n_entries, ptr, idx, w, in, out, mean, ws, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int32_t e2egrec_aggregate_forward(int64_t n_dst, int64_t n_entries, const int64_t *indptr,

@@ -5,6 +5,7 @@
 #include "common.cuh"
 #include "gemm_simt.cuh"
 #include "gemm_tc.cuh"
+#include "segreduce.cuh"
 
 namespace e2egrec {
 
@@ -75,36 +76,7 @@ static void dispatch_sage_aggregate(const T *Hsrc, int64_t ld, const int32_t *nb
 #undef E2E_CASE
 }
 
-// Segment reduction over a 32-bit offset array (the transposed block).
-template <typename T, int LPR, int CPL>
-static void launch_seg32(const T *in, int64_t ld_in, const int32_t *ptr, const int32_t *idx, const int32_t *n_seg_dev,
-                         int64_t cap_seg, int64_t cap_entries, int chunk_len, int d, float *head, float *tail,
-                         const SegOut<T> &o, cudaStream_t st)
-{
-    const int64_t n_chunks = ceil_div(cap_entries > 0 ? cap_entries : 1, chunk_len);
-    note_launch();
-    seg_chunk_kernel<T, int32_t, LPR, CPL, false><<<(unsigned)ceil_div(n_chunks * 32, kAggThreads), kAggThreads, 0, st>>>(
-        in, ld_in, ptr, idx, n_seg_dev, 0, nullptr, chunk_len, d, head, tail, o);
-    const int64_t empty_blocks = ceil_div((cap_seg > 0 ? cap_seg : 1) * 8, kAggThreads);
-    note_launch();
-    seg_finish_kernel<T, int32_t><<<(unsigned)(n_chunks + empty_blocks), kAggThreads, 0, st>>>(
-        ptr, n_seg_dev, 0, chunk_len, d, head, tail, n_chunks, o);
-}
-
-template <typename T>
-static void dispatch_seg32(const T *in, int64_t ld_in, const int32_t *ptr, const int32_t *idx, const int32_t *n_seg_dev,
-                           int64_t cap_seg, int64_t cap_entries, int chunk_len, int d, float *head, float *tail,
-                           const SegOut<T> &o, int32_t dtype, cudaStream_t st)
-{
-    const RowShape rs = row_shape(d, dtype);
-#define E2E_CASE(L, C)                                                                                              \
-    if (rs.lpr == L && rs.cpl == C)                                                                                 \
-        return launch_seg32<T, L, C>(in, ld_in, ptr, idx, n_seg_dev, cap_seg, cap_entries, chunk_len, d, head, tail, o, st);
-    E2E_CASE(4, 1) E2E_CASE(8, 1) E2E_CASE(16, 1) E2E_CASE(32, 1) E2E_CASE(32, 2) E2E_CASE(32, 4)
-#undef E2E_CASE
-}
-
-constexpr int kBlockChunk = 128;      // transposed-block entries per warp
+constexpr int kBlockRun = 32;         // transposed-block entries per lane group (level-1 run)
 constexpr int kDwSplits = 148;        // split-K factor of the weight-gradient product
 
 // ------------------------------------------------------------------------------ forward
@@ -155,7 +127,7 @@ static int32_t forward_impl(const e2egrec_block *blocks, int32_t n_layers, const
 
 // ------------------------------------------------------------------------------ backward
 struct BackwardScratch {
-    size_t dz_off[2], dcat_off, head_off, tail_off, part_off, wt_off, bytes;
+    size_t dz_off[2], dcat_off, seg_off, seg_bytes, part_off, wt_off, bytes;
 };
 
 // Wt[j][o] = W[o][j]: the dCat product reads the layer weight with d_out as the contraction index.
@@ -181,16 +153,15 @@ static BackwardScratch plan_backward(const e2egrec_block *blocks, int32_t n_laye
         dcat = std::max(dcat, (size_t)p.rows * 2 * p.d_in * es);
         part = std::max(part, (size_t)kDwSplits * p.d_out * 2 * p.d_in * sizeof(float));
         wt = std::max(wt, (size_t)p.d_out * 2 * p.d_in * es);
-        const int64_t n_chunks = ceil_div(std::max(blocks[p.block].cap_edges, 1), kBlockChunk);
-        ht = std::max(ht, (size_t)n_chunks * p.d_in * sizeof(float));
+        ht = std::max(ht, seg_scratch_carve(blocks[p.block].cap_edges, kBlockRun, p.d_in, nullptr).bytes);
     }
     size_t off = 0;
     auto take = [&](size_t b) { size_t o = off; off += align_up(b, 256); return o; };
     s.dz_off[0] = take(dz);
     s.dz_off[1] = take(dz);
     s.dcat_off = take(dcat);
-    s.head_off = take(ht);
-    s.tail_off = take(ht);
+    s.seg_off = take(ht);
+    s.seg_bytes = ht;
     s.part_off = take(part);
     s.wt_off = take(wt);
     s.bytes = off;
@@ -206,8 +177,6 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
     const int accumulate = (flags & E2EGREC_ACCUMULATE_DW) ? 1 : 0;
     T *dz_buf[2] = {reinterpret_cast<T *>(scratch + bs.dz_off[0]), reinterpret_cast<T *>(scratch + bs.dz_off[1])};
     T *dcat = reinterpret_cast<T *>(scratch + bs.dcat_off);
-    float *head = reinterpret_cast<float *>(scratch + bs.head_off);
-    float *tail = reinterpret_cast<float *>(scratch + bs.tail_off);
     float *part = reinterpret_cast<float *>(scratch + bs.part_off);
 
     // gradient entering the top layer, masked by its activation
@@ -283,8 +252,9 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
             o.mask = nullptr;
         }
         if (l == 0) tap_begin(TAP_AGG_BWD_OUTER, st);
-        dispatch_seg32<T>(dcat + p.d_in, two_d, b.csc_ptr, b.csc_row, &b.counts[CNT_SRC], b.cap_src, b.cap_edges,
-                          kBlockChunk, p.d_in, head, tail, o, X->dtype, st);
+        const SegScratch sc = seg_scratch_carve(b.cap_edges, kBlockRun, p.d_in, scratch + bs.seg_off);
+        dispatch_seg_reduce<T, int32_t, false>(dcat + p.d_in, two_d, b.csc_ptr, b.csc_row, &b.counts[CNT_SRC], 0, b.cap_src,
+                                               nullptr, kBlockRun, p.d_in, X->dtype, sc, o, st);
         if (l == 0) tap_end(TAP_AGG_BWD_OUTER, st);
     }
     return check_launch("sage_backward");
