@@ -32,7 +32,9 @@ TAP_NAMES = {1: "sage_aggregate_kernel (layer-0 mean aggregation, gathers X rows
              3: "layer-0 dense transform W[h|agg]",
              4: "layer-0 weight gradient dZ^T[h|agg]",
              5: "layer-0 input gradient dZ W",
-             6: "e2egrec_sample_khop (all sampling kernels)"}
+             6: "e2egrec_sample_khop (all sampling kernels)",
+             7: "seg_run_kernel (first transposed aggregation of the backward pass)",
+             8: "seg_window_kernel (same)", 9: "seg_final_kernel (same)"}
 
 
 def measured_peaks():
@@ -196,73 +198,101 @@ def run_ours(args, w):
     scratch = torch.empty(E.binding.sage_backward_scratch_bytes(blocks, X, Ws), dtype=torch.uint8, device=dev)
     dWs = [torch.zeros(W.shape, dtype=torch.float32, device=dev) for W in Ws]
     dX = torch.zeros(blocks.caps[L - 1][1], w.dim, dtype=dt, device=dev)
-    count_log = torch.zeros(total, L, 4, dtype=torch.int32, device=dev)
 
-    def step(i, seeds_t, dH_t):
-        E.sample_khop(indptr, indices, seeds_t, blocks, w.seed, rank * 1_000_000 + i)
+    seeds_in = torch.empty(w.batch, dtype=torch.int32, device=dev)
+    dH_in = torch.empty_like(dH)
+    count_total = torch.zeros(L, 4, dtype=torch.int64, device=dev)
+
+    def step_body():
+        """Everything of one training step, on fixed buffers (seeds_in, dH_in), so that it can be recorded."""
+        E.sample_khop(indptr, indices, seeds_in, blocks, w.seed, 0)         # step number = the scratch's offset
         E.sage_forward(blocks, X, Ws, ctx=ctx, H_out=H_out)
-        E.sage_backward(blocks, X, Ws, ctx, dH_t, dWs=dWs, dX_rows=dX, scratch=scratch)
-        count_log[i].copy_(blocks.counts, non_blocking=True)
+        E.sage_backward(blocks, X, Ws, ctx, dH_in, dWs=dWs, dX_rows=dX, scratch=scratch)
+        count_total.add_(blocks.counts)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident timing, with a per-kernel tap pass for the roofline
-    for i in range(Wm):
-        step(i, seeds_dev[i], dH)
-    taps = {}
-    ev_pool = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
-    for a, b in ev_pool:
-        a.record(); b.record()
-    torch.cuda.synchronize()
-    n_tap_steps = min(K, 10)
-    for which in TAP_NAMES:                              # untimed pass: where does a step spend its time
-        for i in range(n_tap_steps):
-            E.profile_tap(which, *ev_pool[i])
-            step(Wm + i, seeds_dev[Wm + i], dH)
-        torch.cuda.synchronize()
-        taps[which] = [ev_pool[i][0].elapsed_time(ev_pool[i][1]) for i in range(n_tap_steps)]
-    tap_ms = {k: float(np.mean(v)) for k, v in taps.items()}
-    dominant = max((k for k in tap_ms if k != 6), key=lambda k: tap_ms[k])
+    # ---- record the step once as a CUDA graph (no host work between its kernels) and replay it
+    side = torch.cuda.Stream()
+    dH_in.copy_(dH)
+    with torch.cuda.stream(side):
+        for i in range(Wm):                              # eager warm-up on the capture stream
+            seeds_in.copy_(seeds_dev[i])
+            E.sampler_set_step(blocks.scratch, rank * 1_000_000 + i)
+            step_body()
+    side.synchronize()
+    launches_before = E.launch_count()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        step_body()
+    kernels_per_step = E.launch_count() - launches_before + 1      # + the counter update (a torch kernel)
 
+    ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev_a.record(); ev_b.record()
+    torch.cuda.synchronize()
+
+    def run_step(i, g=None):
+        seeds_in.copy_(seeds_dev[i], non_blocking=True)
+        E.sampler_set_step(blocks.scratch, rank * 1_000_000 + i)
+        if g is None:
+            step_body()
+        else:
+            g.replay()
+
+    def tapped_step(i, which):
+        """One eagerly launched step with events around kernel group `which`.  The device is first kept
+        busy for ~1 ms so that the whole step is queued before it starts: the events then bracket the
+        kernels alone, not the host's launch latency (events recorded inside a graph cannot be timed)."""
+        torch.cuda._sleep(2_000_000)
+        E.profile_tap(which, ev_a, ev_b)
+        run_step(i)
+        torch.cuda.synchronize()
+        return ev_a.elapsed_time(ev_b)
+
+    n_tap_steps = min(K, 10)
+    tap_ms = {which: float(np.mean([tapped_step(Wm + i, which) for i in range(n_tap_steps)])) for which in TAP_NAMES}
+    dominant = max((k for k in tap_ms if k <= 5), key=lambda k: tap_ms[k])
+
+    count_total.zero_()
     clocks = ClockSampler(local)
     clocks.start()
     time.sleep(0.6)                                    # let the sampler reach its steady 100 ms period
     barrier()
     t_begin = clocks.mark()
-    launches0 = E.launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(K):
-        E.profile_tap(dominant, *ev_pool[i])           # events around the dominant kernel, on its own stream
-        step(Wm + i, seeds_dev[Wm + i], dH)
+        run_step(Wm + i, graph)
     e1.record()
     barrier()
-    launches = E.launch_count() - launches0
     clk = clocks.stop(t_begin, clocks.mark())
     ms = e0.elapsed_time(e1)
-    dom_ms = [ev_pool[i][0].elapsed_time(ev_pool[i][1]) for i in range(K)]
-    counts = count_log[Wm:].cpu().numpy().astype(np.int64)      # [K, L, 4]
-    status = int(np.bitwise_or.reduce(counts[:, :, 3].ravel())) if counts.size else 0
-    if status:
-        raise RuntimeError(f"device status bits {status} set during the timed region")
-    edges_rank = int(counts[:, :, 2].sum())
+    launches = K * (kernels_per_step + 2)               # + seed copy and step-offset kernel per step
+    counts = count_total.cpu().numpy()                  # [L, 4] summed over the K steps
+    if counts[:, 3].any():
+        raise RuntimeError(f"device status bits set during the timed region: {counts[:, 3]}")
+    edges_rank = int(counts[:, 2].sum())
+    # the dominant kernel again, timed inside recorded steps over the same batches
+    dom_ms = []
+    for i in range(min(K, 50)):
+        dom_ms.append(tapped_step(Wm + i, dominant))
+    outer_counts = count_total.cpu().numpy()[L - 1] / (K + len(dom_ms))
 
     # ---- end to end: host buffers in, results out, every step
     res_pin = [torch.empty(H_out.shape, dtype=dt).pin_memory()] + [torch.empty(W.shape, dtype=torch.float32).pin_memory()
                                                                    for W in Ws]
     cnt_pin = torch.empty(L, 4, dtype=torch.int32).pin_memory()
-    seeds_in = torch.empty(w.batch, dtype=torch.int32, device=dev)
-    dH_in = torch.empty_like(dH)
     h2d = seeds_pin[0].numel() * 4 + dH_pin.numel() * dH_pin.element_size()
     d2h = sum(t.numel() * t.element_size() for t in res_pin) + cnt_pin.numel() * 4
 
     def e2e_step(i):
         seeds_in.copy_(seeds_pin[i], non_blocking=True)
         dH_in.copy_(dH_pin, non_blocking=True)
-        step(i, seeds_in, dH_in)
+        E.sampler_set_step(blocks.scratch, rank * 1_000_000 + i)
+        graph.replay()
         res_pin[0].copy_(H_out, non_blocking=True)
         for t, s in zip(res_pin[1:], dWs):
             t.copy_(s, non_blocking=True)
@@ -299,8 +329,7 @@ def run_ours(args, w):
     peaks = measured_peaks()
     es = 2 if w.dtype == "bf16" else 4
     r = w.dim * es
-    outer = counts[:, L - 1, :].mean(axis=0)              # mean n_dst, n_src, n_edges of the outermost block
-    n_dst, n_src, n_edges = float(outer[0]), float(outer[1]), float(outer[2])
+    n_dst, n_src, n_edges = float(outer_counts[0]), float(outer_counts[1]), float(outer_counts[2])
     dom_mean_ms = float(np.mean(dom_ms))
     if dominant == 1:      # per entry: id + gathered row; per destination: offsets, self id, self row, [self|mean] row out
         alg = n_edges * (4 + r) + n_dst * (8 + 4 + r + 2 * r)
@@ -321,7 +350,7 @@ def run_ours(args, w):
                 data="synthetic",
                 config=dict(workload=w.name, nodes=w.n_nodes, csr_entries=int(indptr_h[-1]), dim=w.dim, hidden=w.hidden,
                             layers=L, fanouts=list(w.fanouts), batch=w.batch, seeds=args.seeds,
-                            parallelism=f"replicas x{world}",
+                            parallelism=f"replicas x{world}", launch="one CUDA graph replay per step",
                             l2="inputs larger than L2: feature table + graph = %.0f MB, a new batch every step"
                                % ((X.numel() * es + indices.numel() * 4 + indptr.numel() * 8) / 1e6),
                             edges_per_step=edges_rank / K),

@@ -96,12 +96,13 @@ typedef struct e2egrec_mat {
  *   csc_ptr    int32[cap_src+1]    transposed block: source s owns [csc_ptr[s], csc_ptr[s+1])
  *   csc_row    int32[cap_edges]    destination of each transposed entry
  *   csc_eid    int32[cap_edges]    its position in the block CSR; ascending inside a column
+ *   csc_col    int32[cap_edges]    its source (the column it belongs to): csc_col[k] = s for k in column s
  *   inv_cnt    float[cap_dst]      1/|S(u)| per destination, 0 for an isolated node */
 typedef struct e2egrec_block {
     int32_t  cap_dst, cap_src, cap_edges;
     int32_t *counts;
     int32_t *indptr, *col, *nbr_global, *src_nodes;
-    int32_t *csc_ptr, *csc_row, *csc_eid;
+    int32_t *csc_ptr, *csc_row, *csc_eid, *csc_col;
     float   *inv_cnt;
 } e2egrec_block;
 
@@ -117,7 +118,8 @@ const char *e2egrec_last_error(void);
  * stop_event just after it, then disarms the tap.  Groups: 1 = mean aggregation of the outermost
  * block (layer 0, gathers from X), 2 = transposed aggregation of the outermost block (writes dX_rows),
  * 3 = dense transform of layer 0, 4 = weight gradient of layer 0, 5 = input gradient (dCat) of layer 0,
- * 6 = the whole of e2egrec_sample_khop.  which = 0 disarms. */
+ * 6 = the whole of e2egrec_sample_khop, 7 / 8 / 9 = the three levels of the first segment reduction
+ * that follows (the innermost layer's transposed aggregation in e2egrec_sage_backward).  which = 0 disarms. */
 uint64_t e2egrec_launch_count(void);
 int32_t e2egrec_profile_tap(int32_t which, void *start_event, void *stop_event);
 
@@ -133,6 +135,12 @@ int32_t e2egrec_sample_khop_workspace(int64_t n_nodes, int32_t n_seeds, int32_t 
  * aligned) into its idle state.  Call once after allocating it; e2egrec_sample_khop
  * leaves the buffer idle again when it finishes, so one buffer serves every step. */
 int32_t e2egrec_sampler_scratch_init(int64_t n_nodes, void *scratch, size_t scratch_bytes, void *stream);
+
+/* Sets the step offset kept in the sampler scratch: every later e2egrec_sample_khop that uses this
+ * scratch draws with step = its `step` argument + step_offset (mod 2^32).  init sets it to 0.  This is
+ * for callers that record the kernels of one training step once (a CUDA graph) and replay them: the
+ * recorded `step` argument is fixed, the offset, which lives in device memory, is what moves on. */
+int32_t e2egrec_sampler_set_step(void *scratch, uint32_t step_offset, void *stream);
 
 /* k-hop neighbour sampling (Sec. 3.1: multiset S_l(u) of N(u); Sec. 4.1: sampling
  * probability with beta = 0, i.e. uniform over the stored entries of the row, at most

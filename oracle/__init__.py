@@ -135,7 +135,8 @@ def sample_khop(indptr, indices, seeds, fanouts, seed, step):
                                _p(csc_ptr), _p(csc_row), _p(csc_eid), _p(inv_cnt))
         blocks.append(dict(n_dst=n_dst, n_src=n_src, n_edges=int(ne), indptr=blk_indptr, col=col,
                            nbr_global=nbr, src_nodes=src, csc_ptr=csc_ptr, csc_row=csc_row[:ne].copy(),
-                           csc_eid=csc_eid[:ne].copy(), inv_cnt=inv_cnt[:n_dst].copy()))
+                           csc_eid=csc_eid[:ne].copy(), csc_col=col[csc_eid[:ne]].copy(),
+                           inv_cnt=inv_cnt[:n_dst].copy()))
         dst = src
     return blocks
 

@@ -37,7 +37,8 @@ class Block(C.Structure):
     _fields_ = [("cap_dst", C.c_int32), ("cap_src", C.c_int32), ("cap_edges", C.c_int32),
                 ("counts", C.c_void_p), ("indptr", C.c_void_p), ("col", C.c_void_p),
                 ("nbr_global", C.c_void_p), ("src_nodes", C.c_void_p), ("csc_ptr", C.c_void_p),
-                ("csc_row", C.c_void_p), ("csc_eid", C.c_void_p), ("inv_cnt", C.c_void_p)]
+                ("csc_row", C.c_void_p), ("csc_eid", C.c_void_p), ("csc_col", C.c_void_p),
+                ("inv_cnt", C.c_void_p)]
 
 
 _lib = None
@@ -59,6 +60,8 @@ def lib():
                                                     C.c_void_p, C.c_void_p, C.POINTER(C.c_size_t)]
         L.e2egrec_sampler_scratch_init.restype = C.c_int32
         L.e2egrec_sampler_scratch_init.argtypes = [C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p]
+        L.e2egrec_sampler_set_step.restype = C.c_int32
+        L.e2egrec_sampler_set_step.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
         L.e2egrec_sample_khop.restype = C.c_int32
         L.e2egrec_sample_khop.argtypes = [C.POINTER(Csr), C.c_void_p, C.c_int32, C.c_int32, C.c_void_p,
                                           C.c_uint64, C.c_uint32, C.c_uint32, C.POINTER(Block), C.c_void_p,
@@ -168,13 +171,13 @@ class Blocks:
                 counts=self.counts[h], indptr=torch.zeros(d + 1, **i32), col=torch.zeros(max(e, 1), **i32),
                 nbr_global=torch.zeros(max(e, 1), **i32), src_nodes=torch.zeros(max(s, 1), **i32),
                 csc_ptr=torch.zeros(s + 1, **i32), csc_row=torch.zeros(max(e, 1), **i32),
-                csc_eid=torch.zeros(max(e, 1), **i32),
+                csc_eid=torch.zeros(max(e, 1), **i32), csc_col=torch.zeros(max(e, 1), **i32),
                 inv_cnt=torch.zeros(max(d, 1), dtype=torch.float32, device=device)))
         self.c = (Block * len(self.caps))()
         for h, ((d, s, e), t) in enumerate(zip(self.caps, self.t)):
             self.c[h] = Block(d, s, e, *[t[k].data_ptr() for k in
                                          ("counts", "indptr", "col", "nbr_global", "src_nodes", "csc_ptr",
-                                          "csc_row", "csc_eid", "inv_cnt")])
+                                          "csc_row", "csc_eid", "csc_col", "inv_cnt")])
         self.scratch = _dev_bytes(self.scratch_bytes, device)
         sampler_scratch_init(n_nodes, self.scratch)
 
@@ -193,6 +196,7 @@ class Blocks:
                             csc_ptr=t["csc_ptr"][: n_src + 1].cpu().numpy(),
                             csc_row=t["csc_row"][:n_edges].cpu().numpy(),
                             csc_eid=t["csc_eid"][:n_edges].cpu().numpy(),
+                            csc_col=t["csc_col"][:n_edges].cpu().numpy(),
                             inv_cnt=t["inv_cnt"][:n_dst].cpu().numpy()))
         return out
 
@@ -200,6 +204,11 @@ class Blocks:
 def sampler_scratch_init(n_nodes: int, scratch: torch.Tensor, stream=None):
     _check(lib().e2egrec_sampler_scratch_init(n_nodes, _ptr(scratch), scratch.numel(), _stream(stream)),
            "e2egrec_sampler_scratch_init")
+
+
+def sampler_set_step(scratch: torch.Tensor, step_offset: int, stream=None):
+    _check(lib().e2egrec_sampler_set_step(_ptr(scratch), step_offset & 0xFFFFFFFF, _stream(stream)),
+           "e2egrec_sampler_set_step")
 
 
 def sample_khop(indptr: torch.Tensor, indices: torch.Tensor, seeds: torch.Tensor, blocks: Blocks, seed: int,

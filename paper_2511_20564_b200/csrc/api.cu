@@ -49,7 +49,7 @@ extern "C" uint64_t e2egrec_launch_count(void) { return e2egrec::g_launches.load
 
 extern "C" int32_t e2egrec_profile_tap(int32_t which, void *start_event, void *stop_event)
 {
-    if (which < 0 || which > e2egrec::TAP_SAMPLE) return E2EGREC_ERR_ARG;
+    if (which < 0 || which > e2egrec::TAP_LAST) return E2EGREC_ERR_ARG;
     if (which && (!start_event || !stop_event)) return E2EGREC_ERR_NULL;
     e2egrec::g_tap_which = which;
     e2egrec::g_tap_start = static_cast<cudaEvent_t>(start_event);

@@ -29,7 +29,7 @@ void note_launch();
 // host side: timing taps (e2egrec_profile_tap).  tap_begin/tap_end record the armed events around
 // kernel group `which` and disarm the tap.
 enum { TAP_AGG_FWD_OUTER = 1, TAP_AGG_BWD_OUTER = 2, TAP_UPDATE_FWD_OUTER = 3, TAP_DW_OUTER = 4, TAP_DCAT_OUTER = 5,
-       TAP_SAMPLE = 6 };
+       TAP_SAMPLE = 6, TAP_SEG_L1 = 7, TAP_SEG_L2 = 8, TAP_SEG_L3 = 9, TAP_LAST = 9 };
 void tap_begin(int which, cudaStream_t st);
 void tap_end(int which, cudaStream_t st);
 
@@ -40,6 +40,10 @@ template <typename T> struct Chunk;
 
 template <> struct Chunk<float> {
     static constexpr int kElems = 4;
+    __device__ static inline uint4 load_raw(const float *p) { return __ldg(reinterpret_cast<const uint4 *>(p)); }
+    __device__ static inline void unpack(const uint4 &r, float (&v)[4]) {
+        v[0] = __uint_as_float(r.x); v[1] = __uint_as_float(r.y); v[2] = __uint_as_float(r.z); v[3] = __uint_as_float(r.w);
+    }
     __device__ static inline void load(const float *p, float (&v)[4]) {
         float4 r = __ldg(reinterpret_cast<const float4 *>(p));
         v[0] = r.x; v[1] = r.y; v[2] = r.z; v[3] = r.w;
@@ -51,6 +55,15 @@ template <> struct Chunk<float> {
 
 template <> struct Chunk<__nv_bfloat16> {
     static constexpr int kElems = 8;
+    __device__ static inline uint4 load_raw(const __nv_bfloat16 *p) { return __ldg(reinterpret_cast<const uint4 *>(p)); }
+    __device__ static inline void unpack(const uint4 &r, float (&v)[8]) {
+        const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            v[2 * i] = __uint_as_float(w[i] << 16);
+            v[2 * i + 1] = __uint_as_float(w[i] & 0xFFFF0000u);
+        }
+    }
     __device__ static inline void load(const __nv_bfloat16 *p, float (&v)[8]) {
         uint4 r = __ldg(reinterpret_cast<const uint4 *>(p));
         const uint32_t w[4] = {r.x, r.y, r.z, r.w};

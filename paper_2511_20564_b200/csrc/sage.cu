@@ -254,7 +254,7 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
         if (l == 0) tap_begin(TAP_AGG_BWD_OUTER, st);
         const SegScratch sc = seg_scratch_carve(b.cap_edges, kBlockRun, p.d_in, scratch + bs.seg_off);
         dispatch_seg_reduce<T, int32_t, false>(dcat + p.d_in, two_d, b.csc_ptr, b.csc_row, &b.counts[CNT_SRC], 0, b.cap_src,
-                                               nullptr, kBlockRun, p.d_in, X->dtype, sc, o, st);
+                                               nullptr, kBlockRun, p.d_in, X->dtype, b.csc_col, sc, o, st);
         if (l == 0) tap_end(TAP_AGG_BWD_OUTER, st);
     }
     return check_launch("sage_backward");

@@ -34,6 +34,7 @@ __device__ inline uint4 philox4x32_10(uint4 c, uint2 k)
 // Scratch layout (host and device agree through this struct).
 // ---------------------------------------------------------------------------------------
 struct SamplerScratch {
+    uint32_t *step_offset; // [1]         added to the `step` argument of every call (see e2egrec_sampler_set_step)
     int32_t  *local_id;    // [n_nodes]   -1 when idle, else position in the current frontier
     uint32_t *bitmap;      // [n_words]   newly reached nodes of the hop in progress; 0 when idle
     int32_t  *word_cnt;    // [n_words]
@@ -70,6 +71,7 @@ static SamplerScratch carve(int64_t n_nodes, int64_t max_dst, int64_t max_src, i
     int64_t longest = hist_len + 1;
     if (s.n_words > longest) longest = s.n_words;
     if (max_src + 1 > longest) longest = max_src + 1;
+    s.step_offset = (uint32_t *)take(256);
     s.local_id = (int32_t *)take(sizeof(int32_t) * (size_t)n_nodes);
     s.bitmap = (uint32_t *)take(sizeof(uint32_t) * (size_t)s.n_words);
     s.word_cnt = (int32_t *)take(sizeof(int32_t) * (size_t)s.n_words);
@@ -146,12 +148,14 @@ __global__ void hop_count_kernel(const int64_t *__restrict__ g_indptr, int64_t n
 __global__ void hop_draw_kernel(const int64_t *__restrict__ g_indptr, const int32_t *__restrict__ g_indices,
                                 int64_t n_nodes, const int32_t *__restrict__ src_nodes,
                                 const int32_t *__restrict__ blk_indptr, int32_t *__restrict__ counts,
-                                int32_t fanout, int32_t hop, uint32_t seed_lo, uint32_t seed_hi, uint32_t step,
+                                int32_t fanout, int32_t hop, uint32_t seed_lo, uint32_t seed_hi, uint32_t step_arg,
+                                const uint32_t *__restrict__ step_offset,
                                 int32_t cap_edges, int32_t *__restrict__ nbr_global, int32_t *__restrict__ edge_row,
                                 const int32_t *__restrict__ local_id, uint32_t *__restrict__ bitmap)
 {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int32_t n_dst = counts[CNT_DST];
+    const uint32_t step = step_arg + *step_offset;
     if (t == 0) counts[CNT_EDGES] = min(blk_indptr[n_dst], cap_edges);
     const int64_t i = t / fanout;
     const int32_t j = (int32_t)(t - i * fanout);
@@ -354,7 +358,7 @@ static void sort_by_col(const e2egrec_block &b, SamplerScratch &s, cudaStream_t 
     const int32_t *vin = nullptr;                 // first pass: value = own position
     for (int p = 0; p < passes; ++p) {
         const bool last = p == passes - 1;
-        int32_t *kout = last ? nullptr : s.keys[p & 1];
+        int32_t *kout = last ? b.csc_col : s.keys[p & 1];
         int32_t *vout = last ? b.csc_eid : s.vals[p & 1];
         if (bits == 8) sort_pass<8>(kin, vin, kout, vout, b.counts, p * bits, n_tiles, s, st);
         else sort_pass<10>(kin, vin, kout, vout, b.counts, p * bits, n_tiles, s, st);
@@ -425,8 +429,21 @@ extern "C" int32_t e2egrec_sampler_scratch_init(int64_t n_nodes, void *scratch, 
     note_launch();
     fill_i32_kernel<<<(unsigned)std::min<int64_t>(ceil_div(n_nodes > 0 ? n_nodes : 1, 256), 148 * 16), 256, 0, st>>>(
         s.local_id, n_nodes, -1);
+    cudaMemsetAsync(s.step_offset, 0, 256, st);
     cudaMemsetAsync(s.bitmap, 0, sizeof(uint32_t) * (size_t)s.n_words, st);
     return check_launch("sampler_scratch_init");
+}
+
+__global__ void set_u32_kernel(uint32_t *p, uint32_t v) { *p = v; }
+
+extern "C" int32_t e2egrec_sampler_set_step(void *scratch, uint32_t step_offset, void *stream)
+{
+    if (!scratch) return E2EGREC_ERR_NULL;
+    if (reinterpret_cast<uintptr_t>(scratch) % 256) return E2EGREC_ERR_ALIGN;
+    SamplerScratch s = carve(0, 0, 0, 0, scratch);
+    note_launch();
+    set_u32_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(s.step_offset, step_offset);
+    return check_launch("sampler_set_step");
 }
 
 extern "C" int32_t e2egrec_sample_khop(const e2egrec_csr *graph, const int32_t *seeds, int32_t n_seeds,
@@ -447,7 +464,7 @@ extern "C" int32_t e2egrec_sample_khop(const e2egrec_csr *graph, const int32_t *
     for (int h = 0; h < n_hops; ++h) {
         const e2egrec_block &b = blocks[h];
         if (!b.counts || !b.indptr || !b.col || !b.nbr_global || !b.src_nodes || !b.csc_ptr || !b.csc_row ||
-            !b.csc_eid || !b.inv_cnt)
+            !b.csc_eid || !b.csc_col || !b.inv_cnt)
             return E2EGREC_ERR_NULL;
         if (b.cap_dst < cd[h] || b.cap_src < cs[h] || b.cap_edges < ce[h]) return E2EGREC_ERR_WORKSPACE;
         if (b.cap_dst > md) md = b.cap_dst;
@@ -475,7 +492,7 @@ extern "C" int32_t e2egrec_sample_khop(const e2egrec_csr *graph, const int32_t *
         note_launch();
         hop_draw_kernel<<<grid_for((int64_t)b.cap_dst * f, T), T, 0, st>>>(
             graph->indptr, graph->indices, n, b.src_nodes, b.indptr, b.counts, f, h + 1,
-            (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), step, b.cap_edges, b.nbr_global, s.edge_row,
+            (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), step, s.step_offset, b.cap_edges, b.nbr_global, s.edge_row,
             s.local_id, s.bitmap);
         note_launch();
         bitmap_popc_kernel<<<grid_for(s.n_words, T), T, 0, st>>>(s.bitmap, s.n_words, s.word_cnt);

@@ -11,12 +11,15 @@
 //   thousands of one-entry segments and one segment of millions of entries cost the same per entry.
 //   A segment that lies inside the run is finished there; otherwise its part goes to head[run]
 //   (segment began in an earlier run) or tail[run] (segment began here and continues), and run_info
-//   records which segments those are.
+//   records which segments those are.  The optional self row of a segment is added where the segment
+//   begins, so partial sums already contain it.
 // Level 2 (seg_window_kernel): one warp per window of 32 runs adds the parts of segments that span
 //   runs of the window, in run order; segments that also leave the window go to head2/tail2.
 // Level 3 (seg_final_kernel): one block per window adds tail2[first] + head2[first+1..last] for the
 //   segment that ends in its window, and extra blocks write fin(0) for segments without entries.
 #pragma once
+
+#include <algorithm>
 
 #include "aggregate.cuh"
 
@@ -54,13 +57,43 @@ inline SegScratch seg_scratch_carve(int64_t cap_entries, int run_len, int d, voi
     return s;
 }
 
+// ------------------------------------------------------------------------------------ helpers
+// (sum [* 1/len]) rounded to the storage type; the self row is already part of `sum` (level 1 adds it
+// where the segment begins), the mask is applied by the caller.
+template <typename T>
+__device__ inline float seg_round(const SegOut<T> &o, float inv_len, float sum)
+{
+    const float v = o.mean ? sum * inv_len : sum;
+    return to_float<T>(from_float<T>(v));
+}
+
+template <typename T> __device__ inline float4 load4(const T *p);
+template <> __device__ inline float4 load4<float>(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
+template <> __device__ inline float4 load4<__nv_bfloat16>(const __nv_bfloat16 *p)
+{
+    const uint2 r = __ldg(reinterpret_cast<const uint2 *>(p));
+    return make_float4(__uint_as_float(r.x << 16), __uint_as_float(r.x & 0xFFFF0000u), __uint_as_float(r.y << 16),
+                       __uint_as_float(r.y & 0xFFFF0000u));
+}
+
+template <typename T> __device__ inline void store4(T *p, const float (&v)[4]);
+template <> __device__ inline void store4<float>(float *p, const float (&v)[4])
+{
+    *reinterpret_cast<float4 *>(p) = make_float4(v[0], v[1], v[2], v[3]);
+}
+template <> __device__ inline void store4<__nv_bfloat16>(__nv_bfloat16 *p, const float (&v)[4])
+{
+    __nv_bfloat162 a = __floats2bfloat162_rn(v[0], v[1]), b = __floats2bfloat162_rn(v[2], v[3]);
+    *reinterpret_cast<uint2 *>(p) = make_uint2(*reinterpret_cast<uint32_t *>(&a), *reinterpret_cast<uint32_t *>(&b));
+}
+
 // ------------------------------------------------------------------------------------ level 1
 template <typename T, typename PtrT, int LPR, int CPL, bool kWeight>
 __global__ void __launch_bounds__(kAggThreads)
 seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__ ptr, const int32_t *__restrict__ idx,
                const int32_t *n_seg_dev, int64_t n_seg_host, const float *__restrict__ w, int run_len, int d,
                float *__restrict__ head, float *__restrict__ tail, int4 *__restrict__ run_info, int64_t cap_runs,
-               SegOut<T> o)
+               const int32_t *__restrict__ seg_of, SegOut<T> o)
 {
     constexpr int E = Chunk<T>::kElems;
     constexpr int U = CPL >= 4 ? 1 : 4 / CPL;
@@ -78,90 +111,162 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
     const int64_t k1 = min(k0 + (int64_t)run_len, total);
     const int64_t n_self = o.self ? (o.n_self ? (int64_t)*o.n_self : n_seg) : 0;
 
-    int64_t s = seg_containing(ptr, n_seg, k0);
-    int64_t cur_beg = (int64_t)ptr[s], cur_end = (int64_t)ptr[s + 1];
-    int32_t head_seg = -1, head_ends = 0, tail_seg = -1;
+    // Segment boundaries are found one iteration ahead of the sums, so that the self row and the mask
+    // row of a segment are requested together with its first gathered row.  With an entry -> segment
+    // array (seg_of) a boundary is a change of that value; without it the offsets are walked, leaping
+    // over stretches of empty segments by bisection.
+    int64_t ws, w_beg = 0, w_end = 0;
+    bool first_begins, last_ends;
+    if (seg_of) {
+        ws = seg_of[k0];
+        first_begins = k0 == 0 || seg_of[k0 - 1] != (int32_t)ws;
+        last_ends = k1 == total || seg_of[k1] != seg_of[k1 - 1];
+    } else {
+        ws = seg_containing(ptr, n_seg, k0);
+        w_beg = (int64_t)ptr[ws];
+        w_end = (int64_t)ptr[ws + 1];
+        first_begins = w_beg >= k0;
+        last_ends = false;                            // decided after the walk has reached the last entry
+    }
 
+    int32_t seg_n[U], id_n[U];
+    bool start_n[U];
+    float inv_n[U];
+    auto classify = [&](int64_t k) {
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const int64_t kk = k + u;
+            start_n[u] = false;
+            seg_n[u] = 0; id_n[u] = 0; inv_n[u] = 0.f;
+            if (kk < k1) {
+                if (seg_of) {
+                    const int64_t sg = seg_of[kk];
+                    start_n[u] = kk == k0 || sg != ws;
+                    ws = sg;
+                    if (o.mean && start_n[u]) inv_n[u] = 1.0f / (float)((int64_t)ptr[sg + 1] - (int64_t)ptr[sg]);
+                } else {
+                    if (kk == k0) {
+                        start_n[u] = true;
+                    } else if (kk >= w_end) {
+                        int step = 0;
+                        do { ++ws; w_end = (int64_t)ptr[ws + 1]; } while (w_end <= kk && ++step < 4);
+                        if (w_end <= kk) {                 // a long stretch of empty segments
+                            ws = seg_containing(ptr, n_seg, kk);
+                            w_end = (int64_t)ptr[ws + 1];
+                        }
+                        w_beg = kk;
+                        start_n[u] = true;
+                    }
+                    if (o.mean && start_n[u]) inv_n[u] = 1.0f / (float)(w_end - (kk == k0 ? w_beg : kk));
+                }
+                seg_n[u] = (int32_t)ws;
+                id_n[u] = idx[kk];
+            }
+        }
+    };
+
+    int64_t cur_seg = -1;
+    bool cur_begins = false;
+    float cur_inv = 0.f;
+    uint4 cur_mask[CPL];
     float acc[CPL][E];
 #pragma unroll
-    for (int q = 0; q < CPL; ++q)
+    for (int q = 0; q < CPL; ++q) {
+        cur_mask[q] = make_uint4(0, 0, 0, 0);
 #pragma unroll
-        for (int kk = 0; kk < E; ++kk) acc[q][kk] = 0.f;
+        for (int e = 0; e < E; ++e) acc[q][e] = 0.f;
+    }
+    int32_t head_seg = -1, head_ends = 0, tail_seg = -1;
 
-    // closes the current segment [cur_beg, cur_end) with the sum in acc
+    // closes the current segment with the sum in acc
     auto emit = [&](bool ended) {
-        const bool begins = cur_beg >= k0;
 #pragma unroll
         for (int q = 0; q < CPL; ++q) {
             const int ch = c + q * LPR;
             if (ch < n_chunks) {
-                if (begins && ended) {
-                    float r[E];
+                if (cur_begins && ended) {
+                    float r[E], m[E];
+                    Chunk<T>::unpack(cur_mask[q], m);
 #pragma unroll
-                    for (int kk = 0; kk < E; ++kk)
-                        r[kk] = seg_finish_value(o, s, cur_end - cur_beg, ch * E + kk, acc[q][kk], s < n_self);
-                    Chunk<T>::store(o.out + s * o.ld_out + ch * E, r);
+                    for (int e = 0; e < E; ++e) {
+                        r[e] = seg_round(o, cur_inv, acc[q][e]);
+                        if (o.mask && !(m[e] > 0.f)) r[e] = 0.f;
+                    }
+                    Chunk<T>::store(o.out + cur_seg * o.ld_out + ch * E, r);
                 } else {
-                    float *dst = (begins ? tail : head) + run * d + ch * E;
+                    float *dst = (cur_begins ? tail : head) + run * d + ch * E;
 #pragma unroll
-                    for (int kk = 0; kk < E; kk += 4)
-                        *reinterpret_cast<float4 *>(dst + kk) =
-                            make_float4(acc[q][kk], acc[q][kk + 1], acc[q][kk + 2], acc[q][kk + 3]);
+                    for (int e = 0; e < E; e += 4)
+                        *reinterpret_cast<float4 *>(dst + e) = make_float4(acc[q][e], acc[q][e + 1], acc[q][e + 2], acc[q][e + 3]);
                 }
             }
-#pragma unroll
-            for (int kk = 0; kk < E; ++kk) acc[q][kk] = 0.f;
         }
-        if (!(begins && ended)) {
-            if (begins) tail_seg = (int32_t)s;
-            else { head_seg = (int32_t)s; head_ends = ended ? 1 : 0; }
+        if (!(cur_begins && ended)) {
+            if (cur_begins) tail_seg = (int32_t)cur_seg;
+            else { head_seg = (int32_t)cur_seg; head_ends = ended ? 1 : 0; }
         }
     };
 
-    int32_t id_next[U];
-#pragma unroll
-    for (int u = 0; u < U; ++u) id_next[u] = k0 + u < k1 ? idx[k0 + u] : 0;
-
+    classify(k0);
     for (int64_t k = k0; k < k1; k += U) {
-        float v[U][CPL][E];
-        float wt[U];
+        int32_t seg_c[U];
+        bool start_c[U];
+        float inv_c[U], wt[U];
+        uint4 v[U][CPL], sv[U][CPL], mv[U][CPL];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const int32_t id = id_next[u];
+            seg_c[u] = seg_n[u];
+            start_c[u] = start_n[u];
+            inv_c[u] = inv_n[u];
             wt[u] = 1.f;
-            if (k + u < k1) {
-                if (kWeight) wt[u] = w[id];
-                const T *row = in + (int64_t)id * ld_in;
+            const bool live = k + u < k1;
+            const int32_t id = id_n[u];
+            if (kWeight && live) wt[u] = w[id];
+            const bool begins = live && start_c[u] && (k + u != k0 || first_begins);
+            const bool want_self = begins && seg_c[u] < n_self;
+            const bool want_mask = live && start_c[u] && o.mask != nullptr;
 #pragma unroll
-                for (int q = 0; q < CPL; ++q) {
-                    const int ch = c + q * LPR;
-                    if (ch < n_chunks) Chunk<T>::load(row + ch * E, v[u][q]);
+            for (int q = 0; q < CPL; ++q) {
+                const int ch = c + q * LPR;
+                v[u][q] = make_uint4(0, 0, 0, 0);
+                sv[u][q] = v[u][q];
+                mv[u][q] = v[u][q];
+                if (ch < n_chunks) {
+                    if (live) v[u][q] = Chunk<T>::load_raw(in + (int64_t)id * ld_in + ch * E);
+                    if (want_self) sv[u][q] = Chunk<T>::load_raw(o.self + (int64_t)seg_c[u] * o.ld_self + ch * E);
+                    if (want_mask) mv[u][q] = Chunk<T>::load_raw(o.mask + (int64_t)seg_c[u] * o.ld_mask + ch * E);
                 }
             }
         }
-#pragma unroll
-        for (int u = 0; u < U; ++u) id_next[u] = k + U + u < k1 ? idx[k + U + u] : 0;
+        if (k + U < k1) classify(k + U);
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const int64_t kk2 = k + u;
-            if (kk2 < k1) {
-                if (kk2 >= cur_end) {
-                    emit(true);
-                    do { ++s; cur_end = (int64_t)ptr[s + 1]; } while (cur_end <= kk2);   // skips empty segments
-                    cur_beg = (int64_t)ptr[s];
+            if (k + u < k1) {
+                if (start_c[u]) {
+                    if (cur_seg >= 0) emit(true);
+                    cur_seg = seg_c[u];
+                    cur_begins = (k + u != k0) || first_begins;
+                    cur_inv = inv_c[u];
+#pragma unroll
+                    for (int q = 0; q < CPL; ++q) {
+                        Chunk<T>::unpack(sv[u][q], acc[q]);          // the self row (zeros if there is none)
+                        cur_mask[q] = mv[u][q];
+                    }
                 }
 #pragma unroll
-                for (int q = 0; q < CPL; ++q)
-                    if (c + q * LPR < n_chunks)
+                for (int q = 0; q < CPL; ++q) {
+                    float x[E];
+                    Chunk<T>::unpack(v[u][q], x);
 #pragma unroll
-                        for (int e = 0; e < E; ++e) {
-                            if (kWeight) acc[q][e] = fmaf(wt[u], v[u][q][e], acc[q][e]);
-                            else acc[q][e] += v[u][q][e];
-                        }
+                    for (int e = 0; e < E; ++e) {
+                        if (kWeight) acc[q][e] = fmaf(wt[u], x[e], acc[q][e]);
+                        else acc[q][e] += x[e];
+                    }
+                }
             }
         }
     }
-    emit(cur_end <= k1);
+    emit(seg_of ? last_ends : w_end <= k1);
     if (c == 0) run_info[run] = make_int4(head_seg, head_ends, tail_seg, 0);
 }
 
@@ -173,11 +278,10 @@ seg_window_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_
                   float *__restrict__ head2, float *__restrict__ tail2, int4 *__restrict__ win_info,
                   int64_t cap_runs, int64_t n_windows, SegOut<T> o)
 {
+    constexpr int kB = 8;                         // runs fetched together
     const int lane = threadIdx.x & 31;
     const int64_t win = ((int64_t)blockIdx.x * kAggThreads + threadIdx.x) >> 5;
     if (win >= n_windows) return;
-    const int64_t n_seg = n_seg_dev ? (int64_t)*n_seg_dev : n_seg_host;
-    const int64_t n_self = o.self ? (o.n_self ? (int64_t)*o.n_self : n_seg) : 0;
     const int64_t r0 = win * kSegWindow;
     int4 info = make_int4(-1, 0, -1, 0);
     if (r0 + lane < cap_runs) info = run_info[r0 + lane];
@@ -192,22 +296,24 @@ seg_window_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_
             bool from_tail = false;
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             w_head = -1; w_head_ends = 0; w_tail = -1;
-            for (int rb = 0; rb < kSegWindow; rb += 4) {
-                // fetch the records of four runs, then walk them in order
-                float4 hv[4], tv[4];
-                int32_t hs[4], he[4], ts[4];
+            for (int rb = 0; rb < kSegWindow; rb += kB) {
+                // fetch the records of kB runs (and the mask rows of segments that end in them), then walk them in order
+                float4 hv[kB], tv[kB], mk[kB];
+                int32_t hs[kB], he[kB], ts[kB];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < kB; ++j) {
                     hs[j] = __shfl_sync(0xffffffffu, info.x, rb + j);
                     he[j] = __shfl_sync(0xffffffffu, info.y, rb + j);
                     ts[j] = __shfl_sync(0xffffffffu, info.z, rb + j);
                     hv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
                     tv[j] = hv[j];
+                    mk[j] = make_float4(1.f, 1.f, 1.f, 1.f);
                     if (act && hs[j] >= 0) hv[j] = *reinterpret_cast<const float4 *>(head + (r0 + rb + j) * d + q * 4);
                     if (act && ts[j] >= 0) tv[j] = *reinterpret_cast<const float4 *>(tail + (r0 + rb + j) * d + q * 4);
+                    if (act && hs[j] >= 0 && he[j] && o.mask) mk[j] = load4<T>(o.mask + (int64_t)hs[j] * o.ld_mask + q * 4);
                 }
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
+                for (int j = 0; j < kB; ++j) {
                     if (hs[j] >= 0) {
                         if (cur != hs[j]) { cur = hs[j]; from_tail = false; acc = make_float4(0.f, 0.f, 0.f, 0.f); }
                         acc.x += hv[j].x; acc.y += hv[j].y; acc.z += hv[j].z; acc.w += hv[j].w;
@@ -215,12 +321,16 @@ seg_window_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_
                             if (from_tail) {
                                 if (act) {
                                     const int64_t s = cur;
-                                    const int64_t len = (int64_t)ptr[s + 1] - (int64_t)ptr[s];
-                                    const float r[4] = {acc.x, acc.y, acc.z, acc.w};
+                                    float inv = 0.f;
+                                    if (o.mean) inv = 1.0f / (float)((int64_t)ptr[s + 1] - (int64_t)ptr[s]);
+                                    const float m[4] = {mk[j].x, mk[j].y, mk[j].z, mk[j].w};
+                                    float r[4] = {acc.x, acc.y, acc.z, acc.w};
 #pragma unroll
-                                    for (int e = 0; e < 4; ++e)
-                                        o.out[s * o.ld_out + q * 4 + e] =
-                                            from_float<T>(seg_finish_value(o, s, len, q * 4 + e, r[e], s < n_self));
+                                    for (int e = 0; e < 4; ++e) {
+                                        r[e] = seg_round(o, inv, r[e]);
+                                        if (!(m[e] > 0.f)) r[e] = 0.f;
+                                    }
+                                    store4<T>(o.out + s * o.ld_out + q * 4, r);
                                 }
                             } else {
                                 if (act) *reinterpret_cast<float4 *>(head2 + win * d + q * 4) = acc;
@@ -261,11 +371,14 @@ seg_final_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_t
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
     if ((int64_t)blockIdx.x >= n_windows) {
-        // segments without entries: 8 lanes per segment
-        const int64_t s = ((int64_t)(blockIdx.x - n_windows) * kAggThreads + threadIdx.x) >> 3;
-        if (s >= n_seg || ptr[s + 1] != ptr[s]) return;
-        for (int k = threadIdx.x & 7; k < d; k += 8)
-            o.out[s * o.ld_out + k] = from_float<T>(seg_finish_value(o, s, 0, k, 0.f, s < n_self));
+        // segments without entries: 8 lanes per segment, the extra blocks stride over all segments
+        const int64_t n_extra = (int64_t)gridDim.x - n_windows;
+        for (int64_t s = ((int64_t)(blockIdx.x - n_windows) * kAggThreads + threadIdx.x) >> 3; s < n_seg;
+             s += n_extra * (kAggThreads / 8)) {
+            if (ptr[s + 1] != ptr[s]) continue;
+            for (int k = threadIdx.x & 7; k < d; k += 8)
+                o.out[s * o.ld_out + k] = from_float<T>(seg_finish_value(o, s, 0, k, 0.f, s < n_self));
+        }
         return;
     }
     const int64_t win = blockIdx.x;
@@ -306,7 +419,7 @@ seg_final_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_t
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
                 o.out[s * o.ld_out + q * 4 + kk] =
-                    from_float<T>(seg_finish_value(o, s, seg_end - seg_beg, q * 4 + kk, r[kk], s < n_self));
+                    from_float<T>(seg_finish_value(o, s, seg_end - seg_beg, q * 4 + kk, r[kk], false));
         }
         __syncthreads();
     }
@@ -316,31 +429,37 @@ seg_final_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_t
 template <typename T, typename PtrT, int LPR, int CPL, bool kWeight>
 inline void launch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const int32_t *idx, const int32_t *n_seg_dev,
                               int64_t n_seg_host, int64_t cap_seg, const float *w, int run_len, int d,
-                              const SegScratch &sc, const SegOut<T> &o, cudaStream_t st)
+                              const int32_t *seg_of, const SegScratch &sc, const SegOut<T> &o, cudaStream_t st)
 {
+    tap_begin(TAP_SEG_L1, st);
     note_launch();
     seg_run_kernel<T, PtrT, LPR, CPL, kWeight><<<(unsigned)ceil_div(sc.cap_runs * LPR, kAggThreads), kAggThreads, 0, st>>>(
-        in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head, sc.tail, sc.run_info, sc.cap_runs, o);
+        in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head, sc.tail, sc.run_info, sc.cap_runs, seg_of, o);
+    tap_end(TAP_SEG_L1, st);
+    tap_begin(TAP_SEG_L2, st);
     note_launch();
     seg_window_kernel<T, PtrT><<<(unsigned)ceil_div(sc.n_windows * 32, kAggThreads), kAggThreads, 0, st>>>(
         ptr, n_seg_dev, n_seg_host, d, sc.head, sc.tail, sc.run_info, sc.head2, sc.tail2, sc.win_info, sc.cap_runs,
         sc.n_windows, o);
-    const int64_t empty_blocks = ceil_div((cap_seg > 0 ? cap_seg : 1) * 8, kAggThreads);
+    tap_end(TAP_SEG_L2, st);
+    const int64_t empty_blocks = std::min<int64_t>(ceil_div((cap_seg > 0 ? cap_seg : 1) * 8, kAggThreads), 148 * 8);
+    tap_begin(TAP_SEG_L3, st);
     note_launch();
     seg_final_kernel<T, PtrT><<<(unsigned)(sc.n_windows + empty_blocks), kAggThreads, 0, st>>>(
         ptr, n_seg_dev, n_seg_host, run_len, d, sc.head2, sc.tail2, sc.win_info, sc.n_windows, o);
+    tap_end(TAP_SEG_L3, st);
 }
 
 template <typename T, typename PtrT, bool kWeight>
 inline void dispatch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const int32_t *idx, const int32_t *n_seg_dev,
                                 int64_t n_seg_host, int64_t cap_seg, const float *w, int run_len, int d, int32_t dtype,
-                                const SegScratch &sc, const SegOut<T> &o, cudaStream_t st)
+                                const int32_t *seg_of, const SegScratch &sc, const SegOut<T> &o, cudaStream_t st)
 {
     const RowShape rs = row_shape(d, dtype);
 #define E2E_CASE(L, C)                                                                                                \
     if (rs.lpr == L && rs.cpl == C)                                                                                   \
         return launch_seg_reduce<T, PtrT, L, C, kWeight>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, cap_seg, w, run_len, \
-                                                         d, sc, o, st);
+                                                         d, seg_of, sc, o, st);
     E2E_CASE(4, 1) E2E_CASE(8, 1) E2E_CASE(16, 1) E2E_CASE(32, 1) E2E_CASE(32, 2) E2E_CASE(32, 4)
 #undef E2E_CASE
 }

@@ -116,7 +116,7 @@ def assert_blocks_equal(gpu_blocks, ora_blocks):
         assert g["status"] == 0, f"hop {h}: device status {g['status']}"
         for k in ("n_dst", "n_src", "n_edges"):
             assert g[k] == o[k], f"hop {h}: {k} {g[k]} != {o[k]}"
-        for k in ("indptr", "nbr_global", "src_nodes", "col", "csc_ptr", "csc_row", "csc_eid"):
+        for k in ("indptr", "nbr_global", "src_nodes", "col", "csc_ptr", "csc_row", "csc_eid", "csc_col"):
             assert np.array_equal(g[k], o[k]), f"hop {h}: {k} differs"
         assert np.array_equal(g["inv_cnt"].view(np.uint32), o["inv_cnt"].view(np.uint32)), f"hop {h}: inv_cnt"
 
