@@ -31,33 +31,105 @@ __device__ inline uint4 philox4x32_10(uint4 c, uint2 k)
 }
 
 // ---------------------------------------------------------------------------------------
+// Single-pass prefix sums across thread blocks ("chained scan"): every tile publishes its own sum,
+// then looks back over the tiles before it until it meets one whose full prefix is known.  Tiles
+// are handed out by an atomic ticket, so a tile only ever waits for tiles that already run.  Every
+// wait is bounded; when the bound is hit the status word gets E2EGREC_DEV_TIMEOUT and the tile goes
+// on with what it has.
+// ---------------------------------------------------------------------------------------
+constexpr unsigned long long kChainAgg = 1ull << 62, kChainPrefix = 2ull << 62, kChainMask = (1ull << 62) - 1;
+constexpr int kChainSpinLimit = 1 << 22;
+
+__device__ inline unsigned long long chain_read(const unsigned long long *slot)
+{
+    return *reinterpret_cast<const volatile unsigned long long *>(slot);
+}
+
+// Called by all threads of the block.  Returns the sum of the aggregates of tiles 0 .. tile-1.
+__device__ inline long long chain_lookback(unsigned long long *state, int tile, long long aggregate, int32_t *status,
+                                           long long *bcast)
+{
+    if (threadIdx.x < 32) {
+        const int lane = threadIdx.x;
+        long long excl = 0;
+        if (lane == 0) atomicExch(&state[tile], (tile == 0 ? kChainPrefix : kChainAgg) | (unsigned long long)aggregate);
+        if (tile > 0) {
+            int p = tile - 1;
+            bool done = false;
+            while (!done) {
+                const int idx = p - lane;
+                unsigned long long v = kChainPrefix;                 // before tile 0: an empty prefix
+                bool timed_out = false;
+                for (int spin = 0;; ++spin) {
+                    if (idx >= 0) v = chain_read(&state[idx]);
+                    if (__all_sync(0xffffffffu, (v >> 62) != 0)) break;
+                    if (spin >= kChainSpinLimit) { timed_out = true; break; }
+                }
+                timed_out = __any_sync(0xffffffffu, timed_out);
+                const unsigned pref = __ballot_sync(0xffffffffu, (v >> 62) == 2);
+                const int first = pref ? __ffs(pref) - 1 : 31;
+                long long c = lane <= first ? (long long)(v & kChainMask) : 0;
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
+                excl += c;
+                if (timed_out) {
+                    if (lane == 0) atomicOr(reinterpret_cast<unsigned *>(status), E2EGREC_DEV_TIMEOUT);
+                    done = true;
+                } else if (pref) {
+                    done = true;
+                } else {
+                    p -= 32;
+                }
+            }
+            if (lane == 0) atomicExch(&state[tile], kChainPrefix | (unsigned long long)(excl + aggregate));
+        }
+        if (lane == 0) *bcast = excl;
+    }
+    __syncthreads();
+    return *bcast;
+}
+
+__device__ inline int chain_ticket(unsigned *ticket, int *bcast)
+{
+    if (threadIdx.x == 0) *bcast = (int)atomicAdd(ticket, 1u);
+    __syncthreads();
+    return *bcast;
+}
+
+// ---------------------------------------------------------------------------------------
 // Scratch layout (host and device agree through this struct).
 // ---------------------------------------------------------------------------------------
-struct SamplerScratch {
-    uint32_t *step_offset; // [1]         added to the `step` argument of every call (see e2egrec_sampler_set_step)
-    int32_t  *local_id;    // [n_nodes]   -1 when idle, else position in the current frontier
-    uint32_t *bitmap;      // [n_words]   newly reached nodes of the hop in progress; 0 when idle
-    int32_t  *word_cnt;    // [n_words]
-    int32_t  *word_rank;   // [n_words+1]
-    int32_t  *cnt;         // [max cap_dst]     |S(u)| per destination
-    int32_t  *csc_cnt;     // [max cap_src]
-    int32_t  *edge_row;    // [max cap_edges]   destination of each block entry
-    int32_t  *keys[2];     // [max cap_edges]   radix sort ping-pong
-    int32_t  *vals[2];
-    int32_t  *hist;        // [radix * sort blocks]
-    int32_t  *hist_off;    // [radix * sort blocks + 1]
-    int32_t  *scan_tmp;    // scan partials
-    size_t    bytes;
-    int64_t   n_words;
-};
-
 constexpr int kSortThreads = 256;
 constexpr int kSortItems = 16;
 constexpr int kSortTile = kSortThreads * kSortItems;
 constexpr int kMaxRadix = 1024;
+constexpr int kMaxPasses = 4;
+constexpr int kDstTile = 256;          // destinations per block of the sampling kernel
+constexpr int kWordTile = 2048;        // bitmap words per block of the frontier kernel
+
+struct SamplerScratch {
+    uint32_t *step_offset; // [1]         added to the `step` argument of every call (see e2egrec_sampler_set_step)
+    int32_t  *local_id;    // [n_nodes]   -1 when idle, else position in the current frontier
+    uint32_t *bitmap;      // [n_words]   newly reached nodes of the hop in progress; 0 when idle
+    int32_t  *edge_row;    // [max cap_edges]   destination of each block entry
+    int32_t  *keys[2];     // [max cap_edges]   radix sort ping-pong
+    int32_t  *vals[2];
+    // chain arena, zeroed at the start of every hop
+    char     *arena;
+    size_t    arena_bytes;
+    unsigned *tickets;                 // [8]
+    unsigned long long *state_dst;     // [dst tiles]
+    unsigned long long *state_words;   // [word tiles]
+    unsigned *ghist;                   // [kMaxPasses x kMaxRadix] digit counts of the whole key array
+    unsigned long long *state_sort;    // [kMaxPasses x kMaxRadix x sort tiles]
+    int64_t   sort_tiles;
+    size_t    bytes;
+    int64_t   n_words;
+};
 
 static SamplerScratch carve(int64_t n_nodes, int64_t max_dst, int64_t max_src, int64_t max_edges, void *base)
 {
+    (void)max_src;
     SamplerScratch s;
     s.n_words = ceil_div(n_nodes, 32);
     size_t off = 0;
@@ -66,24 +138,21 @@ static SamplerScratch carve(int64_t n_nodes, int64_t max_dst, int64_t max_src, i
         off += align_up(bytes, 256);
         return p;
     };
-    const int64_t sort_blocks = ceil_div(max_edges > 0 ? max_edges : 1, kSortTile);
-    const int64_t hist_len = (int64_t)kMaxRadix * sort_blocks;
-    int64_t longest = hist_len + 1;
-    if (s.n_words > longest) longest = s.n_words;
-    if (max_src + 1 > longest) longest = max_src + 1;
+    s.sort_tiles = ceil_div(max_edges > 0 ? max_edges : 1, kSortTile);
     s.step_offset = (uint32_t *)take(256);
     s.local_id = (int32_t *)take(sizeof(int32_t) * (size_t)n_nodes);
     s.bitmap = (uint32_t *)take(sizeof(uint32_t) * (size_t)s.n_words);
-    s.word_cnt = (int32_t *)take(sizeof(int32_t) * (size_t)s.n_words);
-    s.word_rank = (int32_t *)take(sizeof(int32_t) * (size_t)(s.n_words + 1));
-    s.cnt = (int32_t *)take(sizeof(int32_t) * (size_t)(max_dst + 1));
-    s.csc_cnt = (int32_t *)take(sizeof(int32_t) * (size_t)(max_src + 1));
     s.edge_row = (int32_t *)take(sizeof(int32_t) * (size_t)(max_edges + 1));
     for (int i = 0; i < 2; ++i) s.keys[i] = (int32_t *)take(sizeof(int32_t) * (size_t)(max_edges + 1));
     for (int i = 0; i < 2; ++i) s.vals[i] = (int32_t *)take(sizeof(int32_t) * (size_t)(max_edges + 1));
-    s.hist = (int32_t *)take(sizeof(int32_t) * (size_t)hist_len);
-    s.hist_off = (int32_t *)take(sizeof(int32_t) * (size_t)(hist_len + 1));
-    s.scan_tmp = (int32_t *)take(sizeof(int32_t) * scan_scratch_ints(longest));
+    const size_t arena_begin = off;
+    s.arena = base ? static_cast<char *>(base) + off : nullptr;
+    s.tickets = (unsigned *)take(256);
+    s.state_dst = (unsigned long long *)take(8 * (size_t)(ceil_div(max_dst > 0 ? max_dst : 1, kDstTile) + 1));
+    s.state_words = (unsigned long long *)take(8 * (size_t)(ceil_div(s.n_words > 0 ? s.n_words : 1, kWordTile) + 1));
+    s.ghist = (unsigned *)take(sizeof(unsigned) * kMaxPasses * kMaxRadix);
+    s.state_sort = (unsigned long long *)take(8 * (size_t)kMaxPasses * kMaxRadix * (size_t)s.sort_tiles);
+    s.arena_bytes = off - arena_begin;
     s.bytes = off;
     return s;
 }
@@ -111,126 +180,178 @@ __global__ void seed_init_kernel(const int32_t *__restrict__ seeds, int32_t n_se
     if ((uint32_t)u < (uint64_t)n_nodes) local_id[u] = i;
 }
 
-// |S(u)| = min(deg(u), fanout), 1/|S(u)|, and the destination prefix of the frontier.
-__global__ void hop_count_kernel(const int64_t *__restrict__ g_indptr, int64_t n_nodes,
-                                 const int32_t *__restrict__ dst_nodes, const int32_t *n_dst_ptr, int32_t cap_dst,
-                                 int32_t fanout, int32_t *__restrict__ counts, int32_t *__restrict__ cnt,
-                                 float *__restrict__ inv_cnt, int32_t *__restrict__ src_nodes, int first_hop)
+// One hop of sampling in one launch.  A block owns kDstTile destinations: |S(u)| = min(deg, fanout) per
+// destination, a chained scan for the block's offset into the entry arrays, then one thread per
+// (destination, slot).  Slot j of node u at hop h draws with the counter (j/2, u, (1<<8)|h, step) and
+// key (seed lo, seed hi); words 2(j%2), 2(j%2)+1 form r and the picked row position is
+// floor(r * deg / 2^64).  deg <= fanout copies the row instead.  Sampled nodes that are not yet in
+// the frontier are marked in the bitmap.
+__global__ void __launch_bounds__(kDstTile)
+hop_sample_kernel(const int64_t *__restrict__ g_indptr, const int32_t *__restrict__ g_indices, int64_t n_nodes,
+                  const int32_t *__restrict__ dst_nodes, const int32_t *n_dst_ptr, int32_t cap_dst, int32_t cap_edges,
+                  int32_t fanout, int32_t hop, uint32_t seed_lo, uint32_t seed_hi, uint32_t step_arg,
+                  const uint32_t *__restrict__ step_offset, int first_hop, int32_t *__restrict__ counts,
+                  int32_t *__restrict__ blk_indptr, float *__restrict__ inv_cnt, int32_t *__restrict__ src_nodes,
+                  int32_t *__restrict__ nbr_global, int32_t *__restrict__ edge_row,
+                  const int32_t *__restrict__ local_id, uint32_t *__restrict__ bitmap, unsigned *ticket,
+                  unsigned long long *state)
 {
+    __shared__ int32_t off[kDstTile + 1];
+    __shared__ int32_t node[kDstTile];
+    __shared__ int64_t gbeg_s[kDstTile];
+    __shared__ int64_t deg_s[kDstTile];
+    __shared__ int32_t scan_sm[kDstTile / 32 + 1];
+    __shared__ long long bcast;
+    __shared__ int tile_s;
+    const int tile = chain_ticket(ticket, &tile_s);
     int32_t n_dst = *n_dst_ptr;
-    uint32_t status = 0;
-    if (n_dst > cap_dst) { n_dst = cap_dst; status |= E2EGREC_DEV_CAPACITY; }
-    const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i == 0) {
+    const bool over = n_dst > cap_dst;
+    if (over) n_dst = cap_dst;
+    if (tile == 0 && threadIdx.x == 0) {
         counts[CNT_DST] = n_dst;
         if (!first_hop) counts[CNT_STATUS] = 0;
-        if (status) atomicOr((unsigned *)&counts[CNT_STATUS], status);
+        if (over) atomicOr((unsigned *)&counts[CNT_STATUS], E2EGREC_DEV_CAPACITY);
     }
-    if (i >= n_dst) return;
-    int32_t u = dst_nodes[i];
+    const int64_t i0 = (int64_t)tile * kDstTile;
+    if (i0 >= n_dst) {
+        if (n_dst == 0 && tile == 0 && threadIdx.x == 0) { blk_indptr[0] = 0; counts[CNT_EDGES] = 0; }
+        return;
+    }
+    const int64_t i = i0 + threadIdx.x;
     int32_t c = 0;
-    if ((uint32_t)u < (uint64_t)n_nodes) {
-        const int64_t deg = g_indptr[u + 1] - g_indptr[u];
+    if (i < n_dst) {
+        int32_t u = dst_nodes[i];
+        int64_t gb = 0, deg = 0;
+        if ((uint32_t)u < (uint64_t)n_nodes) {
+            gb = g_indptr[u];
+            deg = g_indptr[u + 1] - gb;
+        } else {
+            atomicOr((unsigned *)&counts[CNT_STATUS], E2EGREC_DEV_RANGE);
+            u = 0;
+        }
         c = deg < fanout ? (int32_t)deg : fanout;
-    } else {
-        atomicOr((unsigned *)&counts[CNT_STATUS], E2EGREC_DEV_RANGE);
-        u = 0;
-        c = 0;
+        node[threadIdx.x] = u;
+        gbeg_s[threadIdx.x] = gb;
+        deg_s[threadIdx.x] = deg;
+        inv_cnt[i] = c > 0 ? 1.0f / (float)c : 0.0f;
+        src_nodes[i] = u;
     }
-    cnt[i] = c;
-    inv_cnt[i] = c > 0 ? 1.0f / (float)c : 0.0f;
-    src_nodes[i] = u;
-}
-
-// One thread per (destination, slot).  Slot j of node u at hop h draws with the counter
-// (j/2, u, (1<<8)|h, step) and key (seed lo, seed hi); words 2(j%2), 2(j%2)+1 form r and the
-// picked row position is floor(r * deg / 2^64).  deg <= fanout copies the row instead.
-__global__ void hop_draw_kernel(const int64_t *__restrict__ g_indptr, const int32_t *__restrict__ g_indices,
-                                int64_t n_nodes, const int32_t *__restrict__ src_nodes,
-                                const int32_t *__restrict__ blk_indptr, int32_t *__restrict__ counts,
-                                int32_t fanout, int32_t hop, uint32_t seed_lo, uint32_t seed_hi, uint32_t step_arg,
-                                const uint32_t *__restrict__ step_offset,
-                                int32_t cap_edges, int32_t *__restrict__ nbr_global, int32_t *__restrict__ edge_row,
-                                const int32_t *__restrict__ local_id, uint32_t *__restrict__ bitmap)
-{
-    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int32_t n_dst = counts[CNT_DST];
+    int32_t tile_total;
+    const int32_t ex = block_exclusive_scan<kDstTile, int32_t>(c, tile_total, scan_sm);
+    off[threadIdx.x] = ex;
+    if (threadIdx.x == kDstTile - 1) off[kDstTile] = tile_total;
+    const long long base = chain_lookback(state, tile, tile_total, &counts[CNT_STATUS], &bcast);   // syncs the block
+    if (i < n_dst) blk_indptr[i] = (int32_t)(base + ex);
+    const bool last_tile = i0 + kDstTile >= n_dst;
+    if (last_tile && threadIdx.x == 0) {
+        const long long total = base + tile_total;
+        blk_indptr[n_dst] = (int32_t)total;
+        counts[CNT_EDGES] = total > cap_edges ? cap_edges : (int32_t)total;
+        if (total > cap_edges) atomicOr((unsigned *)&counts[CNT_STATUS], E2EGREC_DEV_CAPACITY);
+    }
     const uint32_t step = step_arg + *step_offset;
-    if (t == 0) counts[CNT_EDGES] = min(blk_indptr[n_dst], cap_edges);
-    const int64_t i = t / fanout;
-    const int32_t j = (int32_t)(t - i * fanout);
-    if (i >= n_dst) return;
-    const int32_t beg = blk_indptr[i];
-    const int32_t c = blk_indptr[i + 1] - beg;
-    if (j >= c) return;
-    const int32_t e = beg + j;
-    if (e >= cap_edges) { atomicOr((unsigned *)&counts[CNT_STATUS], E2EGREC_DEV_CAPACITY); return; }
-    const int32_t u = src_nodes[i];
-    const int64_t gbeg = g_indptr[u];
-    const int64_t deg = g_indptr[u + 1] - gbeg;
-    int64_t pos = j;
-    if (deg > fanout) {
-        const uint4 r4 = philox4x32_10(make_uint4((uint32_t)(j >> 1), (uint32_t)u, (1u << 8) | (uint32_t)hop, step),
-                                       make_uint2(seed_lo, seed_hi));
-        const uint64_t r = (j & 1) ? (((uint64_t)r4.w << 32) | r4.z) : (((uint64_t)r4.y << 32) | r4.x);
-        pos = (int64_t)__umul64hi(r, (uint64_t)deg);
+    for (int32_t sl = threadIdx.x; sl < tile_total; sl += kDstTile) {
+        int lo = 0, hi = kDstTile;                   // largest r with off[r] <= sl
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (off[mid] <= sl) lo = mid; else hi = mid;
+        }
+        const int r = lo;
+        const int32_t j = sl - off[r];
+        const long long e = base + sl;
+        if (e >= cap_edges) continue;
+        const int32_t u = node[r];
+        const int64_t deg = deg_s[r];
+        int64_t pos = j;
+        if (deg > fanout) {
+            const uint4 r4 = philox4x32_10(make_uint4((uint32_t)(j >> 1), (uint32_t)u, (1u << 8) | (uint32_t)hop, step),
+                                           make_uint2(seed_lo, seed_hi));
+            const uint64_t rr = (j & 1) ? (((uint64_t)r4.w << 32) | r4.z) : (((uint64_t)r4.y << 32) | r4.x);
+            pos = (int64_t)__umul64hi(rr, (uint64_t)deg);
+        }
+        int32_t v = g_indices[gbeg_s[r] + pos];
+        if ((uint32_t)v >= (uint64_t)n_nodes) {
+            atomicOr((unsigned *)&counts[CNT_STATUS], E2EGREC_DEV_RANGE);
+            v = u;
+        }
+        nbr_global[e] = v;
+        edge_row[e] = (int32_t)(i0 + r);
+        if (local_id[v] < 0) atomicOr(&bitmap[v >> 5], 1u << (v & 31));
     }
-    int32_t v = g_indices[gbeg + pos];
-    if ((uint32_t)v >= (uint64_t)n_nodes) {
-        atomicOr((unsigned *)&counts[CNT_STATUS], E2EGREC_DEV_RANGE);
-        v = u;
-    }
-    nbr_global[e] = v;
-    edge_row[e] = (int32_t)i;
-    if (local_id[v] < 0) atomicOr(&bitmap[v >> 5], 1u << (v & 31));
 }
 
-__global__ void bitmap_popc_kernel(const uint32_t *__restrict__ bitmap, int64_t n_words, int32_t *__restrict__ word_cnt)
+// New frontier nodes in one launch: a block owns kWordTile bitmap words, counts their set bits, takes
+// its rank offset from a chained scan and hands out local ids n_dst, n_dst+1, ... in ascending id order.
+// The bitmap returns to 0.
+__global__ void __launch_bounds__(256)
+frontier_kernel(uint32_t *__restrict__ bitmap, int64_t n_words, int32_t *__restrict__ counts, int32_t cap_src,
+                int32_t *__restrict__ local_id, int32_t *__restrict__ src_nodes, unsigned *ticket,
+                unsigned long long *state)
 {
-    const int64_t w = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (w < n_words) word_cnt[w] = __popc(bitmap[w]);
-}
-
-// New nodes, in ascending id order, take local ids n_dst, n_dst+1, ...; the bitmap returns to 0.
-__global__ void frontier_assign_kernel(uint32_t *__restrict__ bitmap, const int32_t *__restrict__ word_rank,
-                                       int64_t n_words, int32_t *__restrict__ counts, int32_t cap_src,
-                                       int32_t *__restrict__ local_id, int32_t *__restrict__ src_nodes)
-{
-    const int64_t w = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    constexpr int WPT = kWordTile / 256;
+    __shared__ int32_t scan_sm[256 / 32 + 1];
+    __shared__ long long bcast;
+    __shared__ int tile_s;
+    const int tile = chain_ticket(ticket, &tile_s);
+    const int64_t w0 = (int64_t)tile * kWordTile + (int64_t)threadIdx.x * WPT;
+    uint32_t bits[WPT];
+    int32_t c = 0;
+#pragma unroll
+    for (int k = 0; k < WPT; ++k) {
+        bits[k] = w0 + k < n_words ? bitmap[w0 + k] : 0u;
+        c += __popc(bits[k]);
+    }
+    int32_t tile_total;
+    const int32_t ex = block_exclusive_scan<256, int32_t>(c, tile_total, scan_sm);
+    const long long base = chain_lookback(state, tile, tile_total, &counts[CNT_STATUS], &bcast);
     const int32_t n_dst = counts[CNT_DST];
-    if (w == 0) {
-        int64_t n_src = (int64_t)n_dst + word_rank[n_words];
+    const bool last_tile = (int64_t)(tile + 1) * kWordTile >= n_words;
+    if (last_tile && threadIdx.x == 0) {
+        long long n_src = (long long)n_dst + base + tile_total;
         if (n_src > cap_src) { n_src = cap_src; atomicOr((unsigned *)&counts[CNT_STATUS], E2EGREC_DEV_CAPACITY); }
         counts[CNT_SRC] = (int32_t)n_src;
     }
-    if (w >= n_words) return;
-    uint32_t bits = bitmap[w];
-    if (!bits) return;
-    bitmap[w] = 0;
-    int32_t r = n_dst + word_rank[w];
-    while (bits) {
-        const int b = __ffs(bits) - 1;
-        bits &= bits - 1;
-        const int32_t id = (int32_t)(w * 32 + b);
-        if (r < cap_src) {
-            local_id[id] = r;
-            src_nodes[r] = id;
+    long long r = (long long)n_dst + base + ex;
+#pragma unroll
+    for (int k = 0; k < WPT; ++k) {
+        uint32_t b = bits[k];
+        if (!b) continue;
+        bitmap[w0 + k] = 0;
+        while (b) {
+            const int bit = __ffs(b) - 1;
+            b &= b - 1;
+            const int32_t id = (int32_t)((w0 + k) * 32 + bit);
+            if (r < cap_src) {
+                local_id[id] = (int32_t)r;
+                src_nodes[r] = id;
+            }
+            ++r;
         }
-        ++r;
     }
 }
 
-// col[e] = position of the sampled node in the frontier; column histogram for the transpose.
-__global__ void relabel_kernel(const int32_t *__restrict__ nbr_global, const int32_t *__restrict__ local_id,
-                               const int32_t *__restrict__ counts, int32_t *__restrict__ col,
-                               int32_t *__restrict__ csc_cnt)
+// col[e] = position of the sampled node in the frontier, and the digit counts of the whole col array
+// for every pass of the radix sort that follows.
+__global__ void __launch_bounds__(256)
+relabel_kernel(const int32_t *__restrict__ nbr_global, const int32_t *__restrict__ local_id,
+               const int32_t *__restrict__ counts, int32_t *__restrict__ col, int bits, int passes,
+               unsigned *__restrict__ ghist)
 {
-    const int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= counts[CNT_EDGES]) return;
-    int32_t c = local_id[nbr_global[e]];
-    if (c < 0 || c >= counts[CNT_SRC]) c = 0;        // only after a capacity overrun, which is flagged
-    col[e] = c;
-    atomicAdd(&csc_cnt[c], 1);
+    __shared__ unsigned h[kMaxPasses * kMaxRadix];
+    const int R = 1 << bits;
+    for (int d = threadIdx.x; d < passes * R; d += 256) h[d] = 0;
+    __syncthreads();
+    const int32_t n = counts[CNT_EDGES];
+    const int32_t n_src = counts[CNT_SRC];
+    for (int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x; e < n; e += (int64_t)gridDim.x * 256) {
+        int32_t c = local_id[nbr_global[e]];
+        if (c < 0 || c >= n_src) c = 0;              // only after a capacity overrun, which is flagged
+        col[e] = c;
+        for (int p = 0; p < passes; ++p) atomicAdd(&h[p * R + ((c >> (p * bits)) & (R - 1))], 1u);
+    }
+    __syncthreads();
+    for (int d = threadIdx.x; d < passes * R; d += 256)
+        if (h[d]) atomicAdd(&ghist[(d / R) * kMaxRadix + (d % R)], h[d]);
 }
 
 __global__ void frontier_release_kernel(const int32_t *__restrict__ src_nodes, const int32_t *__restrict__ counts,
@@ -241,45 +362,44 @@ __global__ void frontier_release_kernel(const int32_t *__restrict__ src_nodes, c
 }
 
 // ---------------------------------------------------------------------------------------
-// Stable LSD radix sort of (key = col, value = block position).  Tiles of kSortTile
-// consecutive elements; per pass: tile histograms, one scan over the digit-major
-// (digit, tile) table, then a scatter that ranks equal digits in element order.
+// Stable LSD radix sort of (key = col, value = block position), one launch per digit.  A block owns
+// a tile of kSortTile consecutive elements, ranks equal digits in element order (per warp by
+// match_any, then across warps), and finds where its elements of each digit start from the digit's
+// global start (digit counts of the whole array, known beforehand) plus a per-digit chained scan
+// over the tiles before it.
 // ---------------------------------------------------------------------------------------
 template <int BITS>
 __global__ void __launch_bounds__(kSortThreads)
-sort_hist_kernel(const int32_t *__restrict__ keys, const int32_t *__restrict__ counts, int shift, int n_tiles,
-                 int32_t *__restrict__ hist)
-{
-    constexpr int R = 1 << BITS;
-    __shared__ int32_t h[R];
-    for (int d = threadIdx.x; d < R; d += kSortThreads) h[d] = 0;
-    __syncthreads();
-    const int32_t n = counts[CNT_EDGES];
-    const int64_t base = (int64_t)blockIdx.x * kSortTile;
-#pragma unroll 4
-    for (int k = 0; k < kSortItems; ++k) {
-        const int64_t idx = base + k * kSortThreads + threadIdx.x;
-        if (idx < n) atomicAdd(&h[(keys[idx] >> shift) & (R - 1)], 1);
-    }
-    __syncthreads();
-    for (int d = threadIdx.x; d < R; d += kSortThreads) hist[(int64_t)d * n_tiles + blockIdx.x] = h[d];
-}
-
-template <int BITS>
-__global__ void __launch_bounds__(kSortThreads)
-sort_scatter_kernel(const int32_t *__restrict__ keys_in, const int32_t *__restrict__ vals_in,
-                    const int32_t *__restrict__ counts, int shift, int n_tiles,
-                    const int32_t *__restrict__ hist_off, int32_t *__restrict__ keys_out,
-                    int32_t *__restrict__ vals_out)
+sort_pass_kernel(const int32_t *__restrict__ keys_in, const int32_t *__restrict__ vals_in,
+                 int32_t *__restrict__ counts, int shift, const unsigned *__restrict__ ghist, int n_tiles,
+                 unsigned long long *__restrict__ state, unsigned *ticket, int32_t *__restrict__ keys_out,
+                 int32_t *__restrict__ vals_out)
 {
     constexpr int R = 1 << BITS;
     constexpr int W = kSortThreads / 32;
     __shared__ int32_t wc[W][R];                 // per-warp digit counts, then start offsets
-    for (int d = threadIdx.x; d < W * R; d += kSortThreads) (&wc[0][0])[d] = 0;
-    __syncthreads();
+    __shared__ int32_t bin_base[R];
+    __shared__ int32_t scan_sm[kSortThreads / 32 + 1];
+    __shared__ int tile_s;
+    const int tile = chain_ticket(ticket, &tile_s);
     const int32_t n = counts[CNT_EDGES];
+    if ((int64_t)tile * kSortTile >= n) return;
+    for (int d = threadIdx.x; d < W * R; d += kSortThreads) (&wc[0][0])[d] = 0;
+    // start of every digit's bin: exclusive scan of the global digit counts
+    {
+        int32_t carry = 0;
+        for (int d0 = 0; d0 < R; d0 += kSortThreads) {
+            const int d = d0 + threadIdx.x;
+            const int32_t v = d < R ? (int32_t)ghist[d] : 0;
+            int32_t tot;
+            const int32_t ex = block_exclusive_scan<kSortThreads, int32_t>(v, tot, scan_sm);
+            if (d < R) bin_base[d] = carry + ex;
+            carry += tot;
+        }
+    }
+    __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t wbase = (int64_t)blockIdx.x * kSortTile + (int64_t)warp * (32 * kSortItems);
+    const int64_t wbase = (int64_t)tile * kSortTile + (int64_t)warp * (32 * kSortItems);
     int32_t key[kSortItems], val[kSortItems], rank[kSortItems];
 #pragma unroll
     for (int k = 0; k < kSortItems; ++k) {
@@ -300,13 +420,47 @@ sort_scatter_kernel(const int32_t *__restrict__ keys_in, const int32_t *__restri
         __syncwarp();
     }
     __syncthreads();
-    for (int d = threadIdx.x; d < R; d += kSortThreads) {
-        int32_t run = hist_off[(int64_t)d * n_tiles + blockIdx.x];
+    // per digit: publish this tile's count, then a chained look-back over earlier tiles, then warp start offsets
+    constexpr int DPT = (R + kSortThreads - 1) / kSortThreads;
+    int32_t cnt[DPT];
+#pragma unroll
+    for (int q = 0; q < DPT; ++q) {
+        const int d = threadIdx.x + q * kSortThreads;
+        cnt[q] = 0;
+        if (d < R) {
+#pragma unroll
+            for (int w = 0; w < W; ++w) cnt[q] += wc[w][d];
+            atomicExch(&state[(size_t)d * n_tiles + tile], (tile == 0 ? kChainPrefix : kChainAgg) | (unsigned long long)cnt[q]);
+        }
+    }
+#pragma unroll
+    for (int q = 0; q < DPT; ++q) {
+        const int d = threadIdx.x + q * kSortThreads;
+        if (d >= R) continue;
+        unsigned long long *st = state + (size_t)d * n_tiles;
+        long long excl = 0;
+        if (tile > 0) {
+            bool timed_out = false;
+            for (int p = tile - 1; p >= 0; --p) {
+                unsigned long long v = 0;
+                for (int spin = 0;; ++spin) {
+                    v = chain_read(&st[p]);
+                    if ((v >> 62) != 0) break;
+                    if (spin >= kChainSpinLimit) { timed_out = true; break; }
+                }
+                if (timed_out) break;
+                excl += (long long)(v & kChainMask);
+                if ((v >> 62) == 2) break;
+            }
+            if (timed_out) atomicOr(reinterpret_cast<unsigned *>(&counts[CNT_STATUS]), E2EGREC_DEV_TIMEOUT);
+            atomicExch(&st[tile], kChainPrefix | (unsigned long long)(excl + cnt[q]));
+        }
+        int32_t run = bin_base[d] + (int32_t)excl;
 #pragma unroll
         for (int w = 0; w < W; ++w) {
-            const int32_t c = wc[w][d];
+            const int32_t c2 = wc[w][d];
             wc[w][d] = run;
-            run += c;
+            run += c2;
         }
     }
     __syncthreads();
@@ -315,53 +469,64 @@ sort_scatter_kernel(const int32_t *__restrict__ keys_in, const int32_t *__restri
         const int64_t idx = wbase + k * 32 + lane;
         if (idx < n) {
             const int32_t pos = wc[warp][(key[k] >> shift) & (R - 1)] + rank[k];
-            if (keys_out) keys_out[pos] = key[k];
+            keys_out[pos] = key[k];
             vals_out[pos] = val[k];
         }
     }
 }
 
-__global__ void csc_rows_kernel(const int32_t *__restrict__ csc_eid, const int32_t *__restrict__ edge_row,
-                                const int32_t *__restrict__ counts, int32_t *__restrict__ csc_row)
+// csc_ptr[s] = first position whose column is >= s (the columns are sorted), and the destination of
+// every transposed entry.
+__global__ void csc_finalize_kernel(const int32_t *__restrict__ csc_col, const int32_t *__restrict__ csc_eid,
+                                    const int32_t *__restrict__ edge_row, const int32_t *__restrict__ counts,
+                                    int32_t *__restrict__ csc_ptr, int32_t *__restrict__ csc_row)
 {
-    const int64_t k = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (k < counts[CNT_EDGES]) csc_row[k] = edge_row[csc_eid[k]];
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int32_t n = counts[CNT_EDGES], n_src = counts[CNT_SRC];
+    if (t < n) csc_row[t] = edge_row[csc_eid[t]];
+    if (t <= n_src) {
+        int32_t lo = 0, hi = n;                      // lower bound of t in csc_col[0..n)
+        while (lo < hi) {
+            const int32_t mid = (lo + hi) >> 1;
+            if (csc_col[mid] < (int32_t)t) lo = mid + 1; else hi = mid;
+        }
+        csc_ptr[t] = lo;
+    }
 }
 
-template <int BITS>
-static void sort_pass(const int32_t *kin, const int32_t *vin, int32_t *kout, int32_t *vout, const int32_t *counts,
-                      int shift, int n_tiles, SamplerScratch &s, cudaStream_t st)
-{
-    constexpr int R = 1 << BITS;
-    note_launch();
-    sort_hist_kernel<BITS><<<n_tiles, kSortThreads, 0, st>>>(kin, counts, shift, n_tiles, s.hist);
-    exclusive_scan<int32_t>(s.hist, s.hist_off, nullptr, (int64_t)R * n_tiles, (int64_t)R * n_tiles, s.scan_tmp, st);
-    note_launch();
-    sort_scatter_kernel<BITS><<<n_tiles, kSortThreads, 0, st>>>(kin, vin, counts, shift, n_tiles, s.hist_off, kout, vout);
-}
+struct SortPlan { int bits, passes; };
 
-// csc_eid = positions of the block entries ordered by (col, position).
-static void sort_by_col(const e2egrec_block &b, SamplerScratch &s, cudaStream_t st)
+static SortPlan sort_plan(int32_t cap_src)
 {
     int key_bits = 1;
-    while (key_bits < 31 && (1ll << key_bits) < (int64_t)b.cap_src) ++key_bits;
-    int bits, passes;
-    if (key_bits <= 8) { bits = 8; passes = 1; }
-    else if (key_bits <= 10) { bits = 10; passes = 1; }
-    else if (key_bits <= 16) { bits = 8; passes = 2; }
-    else if (key_bits <= 20) { bits = 10; passes = 2; }
-    else if (key_bits <= 24) { bits = 8; passes = 3; }
-    else if (key_bits <= 30) { bits = 10; passes = 3; }
-    else { bits = 8; passes = 4; }
+    while (key_bits < 31 && (1ll << key_bits) < (int64_t)cap_src) ++key_bits;
+    if (key_bits <= 8) return {8, 1};
+    if (key_bits <= 10) return {10, 1};
+    if (key_bits <= 16) return {8, 2};
+    if (key_bits <= 20) return {10, 2};
+    if (key_bits <= 24) return {8, 3};
+    if (key_bits <= 30) return {10, 3};
+    return {8, 4};
+}
+
+// csc_col / csc_eid = columns and positions of the block entries ordered by (col, position).
+static void sort_by_col(const e2egrec_block &b, const SortPlan &sp, SamplerScratch &s, cudaStream_t st)
+{
     const int n_tiles = (int)ceil_div(b.cap_edges > 0 ? b.cap_edges : 1, kSortTile);
     const int32_t *kin = b.col;
     const int32_t *vin = nullptr;                 // first pass: value = own position
-    for (int p = 0; p < passes; ++p) {
-        const bool last = p == passes - 1;
+    for (int p = 0; p < sp.passes; ++p) {
+        const bool last = p == sp.passes - 1;
         int32_t *kout = last ? b.csc_col : s.keys[p & 1];
         int32_t *vout = last ? b.csc_eid : s.vals[p & 1];
-        if (bits == 8) sort_pass<8>(kin, vin, kout, vout, b.counts, p * bits, n_tiles, s, st);
-        else sort_pass<10>(kin, vin, kout, vout, b.counts, p * bits, n_tiles, s, st);
+        unsigned long long *state = s.state_sort + (size_t)p * kMaxRadix * (size_t)s.sort_tiles;
+        note_launch();
+        if (sp.bits == 8)
+            sort_pass_kernel<8><<<n_tiles, kSortThreads, 0, st>>>(kin, vin, b.counts, p * sp.bits, s.ghist + p * kMaxRadix,
+                                                                 n_tiles, state, s.tickets + 2 + p, kout, vout);
+        else
+            sort_pass_kernel<10><<<n_tiles, kSortThreads, 0, st>>>(kin, vin, b.counts, p * sp.bits, s.ghist + p * kMaxRadix,
+                                                                  n_tiles, state, s.tickets + 2 + p, kout, vout);
         kin = kout;
         vin = vout;
     }
@@ -485,28 +650,24 @@ extern "C" int32_t e2egrec_sample_khop(const e2egrec_csr *graph, const int32_t *
     for (int h = 0; h < n_hops; ++h) {
         const e2egrec_block &b = blocks[h];
         const int32_t f = fanouts[h];
+        const SortPlan sp = sort_plan(b.cap_src);
+        cudaMemsetAsync(s.arena, 0, s.arena_bytes, st);
         note_launch();
-        hop_count_kernel<<<grid_for(b.cap_dst, T), T, 0, st>>>(graph->indptr, n, dst_nodes, n_dst_ptr, b.cap_dst, f,
-                                                              b.counts, s.cnt, b.inv_cnt, b.src_nodes, h == 0);
-        exclusive_scan<int32_t>(s.cnt, b.indptr, &b.counts[CNT_DST], 0, b.cap_dst, s.scan_tmp, st);
+        hop_sample_kernel<<<grid_for(b.cap_dst, kDstTile), kDstTile, 0, st>>>(
+            graph->indptr, graph->indices, n, dst_nodes, n_dst_ptr, b.cap_dst, b.cap_edges, f, h + 1,
+            (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), step, s.step_offset, h == 0, b.counts, b.indptr,
+            b.inv_cnt, b.src_nodes, b.nbr_global, s.edge_row, s.local_id, s.bitmap, s.tickets + 0, s.state_dst);
         note_launch();
-        hop_draw_kernel<<<grid_for((int64_t)b.cap_dst * f, T), T, 0, st>>>(
-            graph->indptr, graph->indices, n, b.src_nodes, b.indptr, b.counts, f, h + 1,
-            (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), step, s.step_offset, b.cap_edges, b.nbr_global, s.edge_row,
-            s.local_id, s.bitmap);
+        frontier_kernel<<<grid_for(s.n_words, kWordTile), 256, 0, st>>>(s.bitmap, s.n_words, b.counts, b.cap_src,
+                                                                        s.local_id, b.src_nodes, s.tickets + 1,
+                                                                        s.state_words);
         note_launch();
-        bitmap_popc_kernel<<<grid_for(s.n_words, T), T, 0, st>>>(s.bitmap, s.n_words, s.word_cnt);
-        exclusive_scan<int32_t>(s.word_cnt, s.word_rank, nullptr, s.n_words, s.n_words, s.scan_tmp, st);
+        relabel_kernel<<<(unsigned)std::min<int64_t>(grid_for(b.cap_edges, T), 148 * 4), T, 0, st>>>(
+            b.nbr_global, s.local_id, b.counts, b.col, sp.bits, sp.passes, s.ghist);
+        sort_by_col(b, sp, s, st);
         note_launch();
-        frontier_assign_kernel<<<grid_for(s.n_words, T), T, 0, st>>>(s.bitmap, s.word_rank, s.n_words, b.counts,
-                                                                    b.cap_src, s.local_id, b.src_nodes);
-        cudaMemsetAsync(s.csc_cnt, 0, sizeof(int32_t) * (size_t)(b.cap_src + 1), st);
-        note_launch();
-        relabel_kernel<<<grid_for(b.cap_edges, T), T, 0, st>>>(b.nbr_global, s.local_id, b.counts, b.col, s.csc_cnt);
-        exclusive_scan<int32_t>(s.csc_cnt, b.csc_ptr, &b.counts[CNT_SRC], 0, b.cap_src, s.scan_tmp, st);
-        sort_by_col(b, s, st);
-        note_launch();
-        csc_rows_kernel<<<grid_for(b.cap_edges, T), T, 0, st>>>(b.csc_eid, s.edge_row, b.counts, b.csc_row);
+        csc_finalize_kernel<<<grid_for(std::max<int64_t>(b.cap_edges, (int64_t)b.cap_src + 1), T), T, 0, st>>>(
+            b.csc_col, b.csc_eid, s.edge_row, b.counts, b.csc_ptr, b.csc_row);
         dst_nodes = b.src_nodes;
         n_dst_ptr = &b.counts[CNT_SRC];
     }
