@@ -203,6 +203,37 @@ int32_t e2egrec_sage_backward(const e2egrec_block *blocks, int32_t n_layers, con
                               const e2egrec_mat *dX_rows, void *scratch, size_t *scratch_bytes,
                               uint32_t flags, void *stream);
 
+/* One joint training step of the GNN and the ranking model (Theorem 1: z_i = [h_theta(x_i) || b_i] is the
+ * scorer's input, so the ranking loss reaches the GNN; Sec. 4.2 chain rule; binary cross-entropy as
+ * in Sec. 5.1).  For n_pairs training pairs (user u_p, item i_p, dense features b_p, label y_p):
+ *   seeds  = the distinct endpoints of the pairs in ascending id order;
+ *   blocks = k-hop sample of the seeds (as e2egrec_sample_khop);  h = GraphSAGE(X) on the seeds
+ *            (as e2egrec_sage_forward, ReLU on every layer, no bias);
+ *   z_p    = [h(u_p) || h(i_p) || b_p];  a1 = ReLU(W_t0 z + b_t0);  a2 = ReLU(W_t1 a1 + b_t1);
+ *   t_p    = W_t2 a2 + b_t2;  loss = mean_p [max(t,0) - y t + log(1 + exp(-|t|))];
+ *   then the full backward: tower weights and biases, the encoder weights, and the feature rows.
+ * Arguments (device memory unless "host"):
+ *   pair_user, pair_item int32[n_pairs] global node ids; dense float[n_pairs x dense_dim]; labels float[n_pairs];
+ *   W_gnn host array[n_hops] (as in e2egrec_sage_forward); W_tower host array[3] of matrices
+ *   [h1 x (2 d_L + dense_dim)], [h2 x h1], [1 x h2] in the dtype of X; b_tower host array[3] of device
+ *   float vectors, or NULL (entries may be NULL);
+ *   loss float[1]; logits float[n_pairs]; dW_gnn / dW_tower host arrays of device float matrices of the
+ *   weights' shapes; db_tower host array[3] of device float vectors or NULL;
+ *   dX_rows [cap_src of the outermost block x d_0] and dX_ids int32[same capacity]: gradient rows and the
+ *   node id of each row; n_dX_rows int32[2] = {number of valid rows, device status bits of the step}.
+ *   ws: workspace (size query with ws == NULL).  Its head is a sampler scratch: initialise it once with
+ *   e2egrec_sampler_scratch_init(n_nodes, ws, ws_bytes, stream).  n_pairs a multiple of 128 and all
+ *   widths multiples of 64 take the tensor-core kernels for bf16; other shapes use fp32-FMA kernels.
+ * With bf16 storage z, a1, a2 and the gradients flowing between the layers are stored as bf16; logits,
+ * loss and all weight gradients are fp32. */
+int32_t e2egrec_joint_step(const e2egrec_csr *graph, const e2egrec_mat *X, const int32_t *pair_user,
+                           const int32_t *pair_item, int32_t n_pairs, const float *dense, int32_t dense_dim,
+                           const float *labels, int32_t n_hops, const int32_t *fanouts,
+                           const e2egrec_mat *W_gnn, const e2egrec_mat *W_tower, const float *const *b_tower,
+                           uint64_t seed, uint32_t step, float *loss, float *logits, float *const *dW_gnn,
+                           float *const *dW_tower, float *const *db_tower, const e2egrec_mat *dX_rows,
+                           int32_t *dX_ids, int32_t *n_dX_rows, void *ws, size_t *ws_bytes, void *stream);
+
 /* Whole-graph neighbourhood aggregation without sampling (Sec. 3.1 Eq. 2 with S(u) = N(u); the
  * "complete graph" case of Sec. 4.1):  out[i] = (1/deg i) sum_{e in row i} X[indices[e]]  (0 for an
  * empty row; the plain sum with E2EGREC_AGG_SUM).  indptr: device int64[n_dst+1], indices: device

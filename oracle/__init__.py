@@ -266,3 +266,41 @@ def full_aggregate_backward(indptr, indices, n_src, G, bf16=False):
     lib().oracle_full_aggregate_backward(_p(indptr), _p(indices), C.c_int64(n_dst), C.c_int64(n_src),
                                          _p(G), C.c_int32(d), _p(dX), C.c_int(int(bf16)))
     return dX
+
+
+# ----------------------------------------------------------------------------- joint step
+
+def joint_step(indptr, indices, X, pair_user, pair_item, dense, labels, fanouts, W_gnn, W_tower, b_tower,
+               seed, step, bf16=False):
+    """Joint GNN + ranking-tower step (Theorem 1: z = [h_theta || b]; BCE on the tower output, Sec. 5.1).
+
+    seeds = ascending distinct endpoints of the pairs; z_p = [h(u_p) || h(i_p) || b_p]; three dense layers
+    (ReLU, ReLU, none); loss = mean BCE-with-logits; then the adjoints back to the tower parameters, the GNN
+    weights and the sampled feature rows.  Returns a dict of everything the GPU call returns.
+    """
+    pair_user, pair_item = _i32(pair_user), _i32(pair_item)
+    seeds = np.unique(np.concatenate([pair_user, pair_item])).astype(np.int32)
+    blocks = sample_khop(indptr, indices, seeds, fanouts, seed, step)
+    H, ctx = sage_forward(blocks, X, W_gnn, bf16=bf16)
+    pos_u, pos_i = np.searchsorted(seeds, pair_user), np.searchsorted(seeds, pair_item)
+    dL = H.shape[1]
+    dense = _f64(dense)
+    if bf16:
+        dense = round_bf16(dense)
+    z = np.concatenate([H[pos_u], H[pos_i], dense], axis=1)
+    b = [None, None, None] if b_tower is None else list(b_tower)
+    a1 = dense_forward(z, W_tower[0], b[0], 1, bf16)
+    a2 = dense_forward(a1, W_tower[1], b[1], 1, bf16)
+    t = dense_forward(a2, W_tower[2], b[2], 0, False)
+    loss, dt = bce_with_logits(t[:, 0], labels)
+    dW3, db3, da2 = dense_backward(dt[:, None], t, a2, W_tower[2], 0, bf16)
+    dW2, db2, da1 = dense_backward(da2, a2, a1, W_tower[1], 1, bf16)
+    dW1, db1, dz = dense_backward(da1, a1, z, W_tower[0], 1, bf16)
+    dH = np.zeros_like(H)
+    np.add.at(dH, pos_u, dz[:, :dL])
+    np.add.at(dH, pos_i, dz[:, dL:2 * dL])
+    if bf16:
+        dH = round_bf16(dH)
+    dW_gnn, _, dX = sage_backward(blocks, ctx, W_gnn, dH, bf16=bf16)
+    return dict(seeds=seeds, blocks=blocks, loss=loss, logits=t[:, 0], dW_tower=[dW1, dW2, dW3],
+                db_tower=[db1, db2, db3], dW_gnn=dW_gnn, dX=dX, dX_ids=blocks[-1]["src_nodes"], H=H, dH=dH)

@@ -90,6 +90,12 @@ def lib():
         L.e2egrec_aggregate_forward_static.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.POINTER(Mat),
                                                        C.POINTER(Mat), C.c_uint32, C.c_void_p]
         L.e2egrec_aggregate_forward_static_limit.restype = C.c_size_t
+        L.e2egrec_joint_step.restype = C.c_int32
+        L.e2egrec_joint_step.argtypes = [C.POINTER(Csr), C.POINTER(Mat), C.c_void_p, C.c_void_p, C.c_int32, C.c_void_p,
+                                         C.c_int32, C.c_void_p, C.c_int32, C.c_void_p, C.POINTER(Mat), C.POINTER(Mat),
+                                         C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                         C.c_void_p, C.c_void_p, C.POINTER(Mat), C.c_void_p, C.c_void_p, C.c_void_p,
+                                         C.POINTER(C.c_size_t), C.c_void_p]
         L.e2egrec_launch_count.restype = C.c_uint64
         L.e2egrec_profile_tap.restype = C.c_int32
         L.e2egrec_profile_tap.argtypes = [C.c_int32, C.c_void_p, C.c_void_p]
@@ -361,3 +367,49 @@ def aggregate_forward_static(indptr, indices, X, out, sum_only=False, stream=Non
 
 def aggregate_forward_static_limit() -> int:
     return int(lib().e2egrec_aggregate_forward_static_limit())
+
+
+# ------------------------------------------------------------------------------------------ joint step
+
+class JointStep:
+    """Buffers and arguments of e2egrec_joint_step for a fixed problem shape; `run` enqueues one step."""
+
+    def __init__(self, indptr, indices, X, n_pairs, dense_dim, fanouts, W_gnn, W_tower, b_tower=None):
+        dev = X.device
+        self.indptr, self.indices, self.X = indptr, indices, X
+        self.n_nodes = indptr.numel() - 1
+        self.n_pairs, self.dense_dim = int(n_pairs), int(dense_dim)
+        self.fanouts = [int(f) for f in fanouts]
+        self.W_gnn, self.W_tower, self.b_tower = list(W_gnn), list(W_tower), b_tower
+        L = len(self.fanouts)
+        _, cs, _, _ = sample_khop_workspace(self.n_nodes, 2 * self.n_pairs, self.fanouts)
+        self.cap_rows = max(cs[L - 1], 1)
+        f32 = dict(dtype=torch.float32, device=dev)
+        self.loss = torch.zeros(1, **f32)
+        self.logits = torch.zeros(self.n_pairs, **f32)
+        self.dW_gnn = [torch.zeros(W.shape, **f32) for W in self.W_gnn]
+        self.dW_tower = [torch.zeros(W.shape, **f32) for W in self.W_tower]
+        self.db_tower = [torch.zeros(W.shape[0], **f32) for W in self.W_tower]
+        self.dX_rows = torch.zeros(self.cap_rows, X.shape[1], dtype=X.dtype, device=dev)
+        self.dX_ids = torch.zeros(self.cap_rows, dtype=torch.int32, device=dev)
+        self.n_rows = torch.zeros(2, dtype=torch.int32, device=dev)
+        self._g = Csr(self.n_nodes, indices.numel(), indptr.data_ptr(), indices.data_ptr(), None)
+        self._x, self._wg, self._wt, self._dx = _mat(X), _mats(self.W_gnn), _mats(self.W_tower), _mat(self.dX_rows)
+        self._f = _i32_host(self.fanouts)
+        n = C.c_size_t(0)
+        self._call(None, None, None, None, n, None, 0, 0)
+        self.ws = _dev_bytes(n.value, dev)
+        sampler_scratch_init(self.n_nodes, self.ws)
+
+    def _call(self, user, item, dense, labels, nbytes, stream, seed, step):
+        L = len(self.fanouts)
+        _check(lib().e2egrec_joint_step(
+            C.byref(self._g), C.byref(self._x), _ptr(user), _ptr(item), self.n_pairs, _ptr(dense), self.dense_dim,
+            _ptr(labels), L, self._f, self._wg, self._wt, _ptr_array(self.b_tower, 3), C.c_uint64(seed),
+            C.c_uint32(step), _ptr(self.loss), _ptr(self.logits), _ptr_array(self.dW_gnn, L),
+            _ptr_array(self.dW_tower, 3), _ptr_array(self.db_tower, 3), C.byref(self._dx), _ptr(self.dX_ids),
+            _ptr(self.n_rows), None if user is None else _ptr(self.ws), C.byref(nbytes), stream), "e2egrec_joint_step")
+
+    def run(self, pair_user, pair_item, dense, labels, seed, step, stream=None):
+        self._call(pair_user, pair_item, dense, labels, C.c_size_t(self.ws.numel()), _stream(stream), seed, step)
+        return self

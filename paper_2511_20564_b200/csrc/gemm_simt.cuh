@@ -105,7 +105,7 @@ struct EpiPartial {
 };
 
 // out = (accumulate ? out : 0) + sum_z partial[z], z ascending
-__global__ void splitk_reduce_kernel(const float *__restrict__ partial, int64_t n, int splits, int accumulate,
+static __global__ void splitk_reduce_kernel(const float *__restrict__ partial, int64_t n, int splits, int accumulate,
                                      float *__restrict__ out)
 {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -153,5 +153,28 @@ colsum_kernel(const T *__restrict__ dZ, int64_t ld, const int32_t *n_dev, int d,
         db[col] = t;
     }
 }
+
+// Wt[j][o] = W[o][j]: the dCat product reads the layer weight with d_out as the contraction index.
+template <typename T>
+__global__ void transpose_kernel(const T *__restrict__ W, int rows, int cols, T *__restrict__ Wt)
+{
+    __shared__ T tile[32][33];
+    const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
+    for (int i = threadIdx.y; i < 32; i += blockDim.y)
+        if (r0 + i < rows && c0 + threadIdx.x < cols) tile[i][threadIdx.x] = W[(int64_t)(r0 + i) * cols + c0 + threadIdx.x];
+    __syncthreads();
+    for (int i = threadIdx.y; i < 32; i += blockDim.y)
+        if (c0 + i < cols && r0 + threadIdx.x < rows) Wt[(int64_t)(c0 + i) * rows + r0 + threadIdx.x] = tile[threadIdx.x][i];
+}
+
+// masked copy of the gradient of a dense layer input: out = acc where mask > 0 (no mask: plain store)
+template <typename T>
+struct EpiMasked {
+    T *out; int64_t ldo; const T *mask; int64_t ld_mask;
+    __device__ void operator()(int64_t m, int n, float v, int) const {
+        if (mask && !(to_float<T>(mask[m * ld_mask + n]) > 0.f)) v = 0.f;
+        out[m * ldo + n] = from_float<T>(v);
+    }
+};
 
 }  // namespace e2egrec

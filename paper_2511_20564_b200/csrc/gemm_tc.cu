@@ -2,7 +2,7 @@
 //
 //   D[m, n] = sum_k A[m, k] * B[n, k]        A: [rows x K] row-major, B: [N x K] row-major (both K-major)
 //
-// One CTA computes a 128 x NT tile (NT = min(N, 256)).  A single thread feeds TMA loads of
+// One CTA computes a 128 x NT tile (NT = the widest multiple of 32, at most 256, that divides N).  A single thread feeds TMA loads of
 // 128 x 64 (A) and NT x 64 (B) bf16 boxes into a ring of 128-byte-swizzled shared-memory stages,
 // a single thread issues tcgen05.mma (M = 128, N = NT, K = 16 per instruction) into an fp32
 // accumulator in tensor memory, and all four warps read the accumulator back with tcgen05.ld for
@@ -135,6 +135,8 @@ struct TcEpilogue {
     int relu;
     const float *row_scale;    // optional: columns >= scale_from are multiplied by row_scale[row]
     int scale_from;
+    const __nv_bfloat16 *mask; // optional [rows x ld_mask]: outputs are zeroed where mask <= 0 (ReLU derivative)
+    int64_t ld_mask;
     const int32_t *m_dev;      // rows at and beyond *m_dev are written as zeros
     int32_t *status;           // device status word (E2EGREC_DEV_TIMEOUT)
 };
@@ -226,10 +228,25 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const bool live = row < m_valid;
         const float rs = (ep.row_scale && live) ? ep.row_scale[row] : 1.f;
         __nv_bfloat16 *orow = ep.out + row * ep.ldo + n0;
+        const __nv_bfloat16 *mrow = ep.mask ? ep.mask + row * ep.ld_mask + n0 : nullptr;
         for (int c = 0; c < nt; c += 32) {
             uint32_t r[32];
             tmem_load32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, r);
             uint32_t packed[16];
+            uint32_t mbits = 0xFFFFFFFFu;                 // bit j: output column c + j keeps its value
+            if (mrow && live) {
+                mbits = 0;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const uint4 mv = *reinterpret_cast<const uint4 *>(mrow + c + q * 8);
+                    const uint32_t w[4] = {mv.x, mv.y, mv.z, mv.w};
+#pragma unroll
+                    for (int t = 0; t < 4; ++t) {
+                        if (__uint_as_float(w[t] << 16) > 0.f) mbits |= 1u << (q * 8 + 2 * t);
+                        if (__uint_as_float(w[t] & 0xFFFF0000u) > 0.f) mbits |= 1u << (q * 8 + 2 * t + 1);
+                    }
+                }
+            }
 #pragma unroll
             for (int j = 0; j < 32; j += 2) {
                 float v0 = __uint_as_float(r[j]), v1 = __uint_as_float(r[j + 1]);
@@ -240,7 +257,8 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     if (col >= ep.scale_from) v0 *= rs;
                     if (col + 1 >= ep.scale_from) v1 *= rs;
                 }
-                if (!live) { v0 = 0.f; v1 = 0.f; }
+                if (!live || !((mbits >> j) & 1u)) v0 = 0.f;
+                if (!live || !((mbits >> (j + 1)) & 1u)) v1 = 0.f;
                 __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
                 packed[j >> 1] = *reinterpret_cast<uint32_t *>(&h);
             }
@@ -299,8 +317,10 @@ bool launch_tn(const __nv_bfloat16 *A, int64_t rows, int k, int64_t lda, const _
                const TcEpilogue &ep, cudaStream_t st)
 {
     if (rows <= 0 || rows % kTileM || k % kTileK || k < kTileK) return false;
-    const int nt = n > 256 ? 256 : n;
-    if (n % nt || nt % 32 || nt < 32) return false;
+    int nt = 0;                                 // widest tile <= 256 columns that divides n (a multiple of 32)
+    for (int c = 256; c >= 32; c -= 32)
+        if (n % c == 0) { nt = c; break; }
+    if (!nt) return false;
     if (reinterpret_cast<uintptr_t>(A) % 16 || reinterpret_cast<uintptr_t>(B) % 16 || (lda * 2) % 16 || (ldb * 2) % 16 ||
         reinterpret_cast<uintptr_t>(ep.out) % 16 || (ep.ldo * 2) % 16)
         return false;
@@ -338,6 +358,22 @@ bool tc_update_forward(const __nv_bfloat16 *cat, int64_t rows, int k, const __nv
     ep.m_dev = m_dev;
     ep.status = status;
     return launch_tn(cat, rows, k, k, W, n, k, ep, st);
+}
+
+bool tc_linear(const __nv_bfloat16 *A, int64_t rows, int k, const __nv_bfloat16 *B, int n, const float *bias, int relu,
+               const __nv_bfloat16 *mask, int64_t ld_mask, __nv_bfloat16 *out, int64_t ldo, const int32_t *m_dev,
+               int32_t *status, cudaStream_t st)
+{
+    TcEpilogue ep{};
+    ep.out = out;
+    ep.ldo = ldo;
+    ep.bias = bias;
+    ep.relu = relu;
+    ep.mask = mask;
+    ep.ld_mask = ld_mask;
+    ep.m_dev = m_dev;
+    ep.status = status;
+    return launch_tn(A, rows, k, k, B, n, k, ep, st);
 }
 
 bool tc_dcat_backward(const __nv_bfloat16 *dz, int64_t rows, int d_out, const __nv_bfloat16 *Wt, int two_d_in,

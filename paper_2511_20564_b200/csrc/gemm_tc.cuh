@@ -17,4 +17,10 @@ bool tc_update_forward(const __nv_bfloat16 *cat, int64_t rows, int k, const __nv
 bool tc_dcat_backward(const __nv_bfloat16 *dz, int64_t rows, int d_out, const __nv_bfloat16 *Wt, int two_d_in,
                       const float *inv_cnt, __nv_bfloat16 *dcat, const int32_t *m_dev, int32_t *status, cudaStream_t st);
 
+// out = mask * act(A B^T + bias): A [rows x k], B [n x k], out [rows x ldo], optional mask [rows x ld_mask]
+// (outputs zeroed where mask <= 0).  Same conventions as above.
+bool tc_linear(const __nv_bfloat16 *A, int64_t rows, int k, const __nv_bfloat16 *B, int n, const float *bias, int relu,
+               const __nv_bfloat16 *mask, int64_t ld_mask, __nv_bfloat16 *out, int64_t ldo, const int32_t *m_dev,
+               int32_t *status, cudaStream_t st);
+
 }  // namespace e2egrec

@@ -130,19 +130,6 @@ struct BackwardScratch {
     size_t dz_off[2], dcat_off, seg_off, seg_bytes, part_off, wt_off, bytes;
 };
 
-// Wt[j][o] = W[o][j]: the dCat product reads the layer weight with d_out as the contraction index.
-template <typename T>
-__global__ void transpose_kernel(const T *__restrict__ W, int rows, int cols, T *__restrict__ Wt)
-{
-    __shared__ T tile[32][33];
-    const int c0 = blockIdx.x * 32, r0 = blockIdx.y * 32;
-    for (int i = threadIdx.y; i < 32; i += blockDim.y)
-        if (r0 + i < rows && c0 + threadIdx.x < cols) tile[i][threadIdx.x] = W[(int64_t)(r0 + i) * cols + c0 + threadIdx.x];
-    __syncthreads();
-    for (int i = threadIdx.y; i < 32; i += blockDim.y)
-        if (c0 + i < cols && r0 + threadIdx.x < rows) Wt[(int64_t)(c0 + i) * rows + r0 + threadIdx.x] = tile[threadIdx.x][i];
-}
-
 static BackwardScratch plan_backward(const e2egrec_block *blocks, int32_t n_layers, const LayerPlan *plan, size_t es)
 {
     BackwardScratch s{};

@@ -8,6 +8,7 @@
 // surplus threads leave at once.
 #include "common.cuh"
 #include "scan.cuh"
+#include "internal.cuh"
 
 #include <algorithm>
 
@@ -494,6 +495,50 @@ __global__ void csc_finalize_kernel(const int32_t *__restrict__ csc_col, const i
     }
 }
 
+// Joint step: the endpoints of the training pairs become the seed set.  Every endpoint is marked in the
+// bitmap (frontier_kernel then lists the marked ids in ascending order and gives them local ids).
+__global__ void pair_mark_kernel(const int32_t *__restrict__ user, const int32_t *__restrict__ item, int32_t n_pairs,
+                                 int64_t n_nodes, uint32_t *__restrict__ bitmap, int32_t *__restrict__ counts)
+{
+    const int p = blockIdx.x * blockDim.x + threadIdx.x;
+    if (p >= n_pairs) return;
+    const int32_t ids[2] = {user[p], item[p]};
+#pragma unroll
+    for (int k = 0; k < 2; ++k) {
+        if ((uint32_t)ids[k] < (uint64_t)n_nodes) atomicOr(&bitmap[ids[k] >> 5], 1u << (ids[k] & 31));
+        else atomicOr((unsigned *)&counts[CNT_STATUS], E2EGREC_DEV_RANGE);
+    }
+}
+
+// pair_local[e] = seed position of entry e (e < P: the user of pair e, else the item of pair e - P),
+// entry_unit[e] = where that entry's gradient row starts inside the tower's input-gradient matrix, in
+// 16-byte units, and the digit counts of pair_local for the sort that groups the entries by seed.
+__global__ void __launch_bounds__(256)
+pair_local_kernel(const int32_t *__restrict__ user, const int32_t *__restrict__ item, int32_t n_pairs, int64_t n_nodes,
+                  const int32_t *__restrict__ local_id, int32_t *__restrict__ pair_local,
+                  int32_t *__restrict__ entry_unit, int units_per_row, int item_unit_off, int32_t *__restrict__ pcounts,
+                  int bits, int passes, unsigned *__restrict__ ghist)
+{
+    __shared__ unsigned h[kMaxPasses * kMaxRadix];
+    const int R = 1 << bits;
+    for (int d = threadIdx.x; d < passes * R; d += 256) h[d] = 0;
+    __syncthreads();
+    if (blockIdx.x == 0 && threadIdx.x == 0) pcounts[CNT_EDGES] = 2 * n_pairs;
+    for (int64_t e = (int64_t)blockIdx.x * 256 + threadIdx.x; e < 2 * (int64_t)n_pairs; e += (int64_t)gridDim.x * 256) {
+        const bool is_item = e >= n_pairs;
+        const int32_t pr = (int32_t)(is_item ? e - n_pairs : e);
+        const int32_t id = is_item ? item[pr] : user[pr];
+        int32_t c = (uint32_t)id < (uint64_t)n_nodes ? local_id[id] : 0;
+        if (c < 0) c = 0;
+        pair_local[e] = c;
+        entry_unit[e] = pr * units_per_row + (is_item ? item_unit_off : 0);
+        for (int p = 0; p < passes; ++p) atomicAdd(&h[p * R + ((c >> (p * bits)) & (R - 1))], 1u);
+    }
+    __syncthreads();
+    for (int d = threadIdx.x; d < passes * R; d += 256)
+        if (h[d]) atomicAdd(&ghist[(d / R) * kMaxRadix + (d % R)], h[d]);
+}
+
 struct SortPlan { int bits, passes; };
 
 static SortPlan sort_plan(int32_t cap_src)
@@ -510,22 +555,23 @@ static SortPlan sort_plan(int32_t cap_src)
 }
 
 // csc_col / csc_eid = columns and positions of the block entries ordered by (col, position).
-static void sort_by_col(const e2egrec_block &b, const SortPlan &sp, SamplerScratch &s, cudaStream_t st)
+static void sort_by_col(const int32_t *col, int32_t *counts, int32_t cap_edges, int32_t *csc_col, int32_t *csc_eid,
+                        const SortPlan &sp, SamplerScratch &s, cudaStream_t st)
 {
-    const int n_tiles = (int)ceil_div(b.cap_edges > 0 ? b.cap_edges : 1, kSortTile);
-    const int32_t *kin = b.col;
+    const int n_tiles = (int)ceil_div(cap_edges > 0 ? cap_edges : 1, kSortTile);
+    const int32_t *kin = col;
     const int32_t *vin = nullptr;                 // first pass: value = own position
     for (int p = 0; p < sp.passes; ++p) {
         const bool last = p == sp.passes - 1;
-        int32_t *kout = last ? b.csc_col : s.keys[p & 1];
-        int32_t *vout = last ? b.csc_eid : s.vals[p & 1];
+        int32_t *kout = last ? csc_col : s.keys[p & 1];
+        int32_t *vout = last ? csc_eid : s.vals[p & 1];
         unsigned long long *state = s.state_sort + (size_t)p * kMaxRadix * (size_t)s.sort_tiles;
         note_launch();
         if (sp.bits == 8)
-            sort_pass_kernel<8><<<n_tiles, kSortThreads, 0, st>>>(kin, vin, b.counts, p * sp.bits, s.ghist + p * kMaxRadix,
+            sort_pass_kernel<8><<<n_tiles, kSortThreads, 0, st>>>(kin, vin, counts, p * sp.bits, s.ghist + p * kMaxRadix,
                                                                  n_tiles, state, s.tickets + 2 + p, kout, vout);
         else
-            sort_pass_kernel<10><<<n_tiles, kSortThreads, 0, st>>>(kin, vin, b.counts, p * sp.bits, s.ghist + p * kMaxRadix,
+            sort_pass_kernel<10><<<n_tiles, kSortThreads, 0, st>>>(kin, vin, counts, p * sp.bits, s.ghist + p * kMaxRadix,
                                                                   n_tiles, state, s.tickets + 2 + p, kout, vout);
         kin = kout;
         vin = vout;
@@ -534,6 +580,11 @@ static void sort_by_col(const e2egrec_block &b, const SortPlan &sp, SamplerScrat
 
 static inline unsigned grid_for(int64_t n, int threads) { return (unsigned)ceil_div(n > 0 ? n : 1, threads); }
 
+size_t sampler_scratch_bytes(int64_t n_nodes, int64_t max_dst, int64_t max_src, int64_t max_edges)
+{
+    return carve(n_nodes, max_dst, max_src, max_edges, nullptr).bytes;
+}
+
 }  // namespace e2egrec
 
 using namespace e2egrec;
@@ -541,7 +592,7 @@ using namespace e2egrec;
 // ---------------------------------------------------------------------------------------
 // C ABI
 // ---------------------------------------------------------------------------------------
-static int32_t khop_caps(int64_t n_nodes, int32_t n_seeds, int32_t n_hops, const int32_t *fanouts,
+int32_t e2egrec::khop_caps(int64_t n_nodes, int32_t n_seeds, int32_t n_hops, const int32_t *fanouts,
                          int32_t *cap_dst, int32_t *cap_src, int32_t *cap_edges)
 {
     if (!fanouts || !cap_dst || !cap_src || !cap_edges) return E2EGREC_ERR_NULL;
@@ -617,8 +668,16 @@ extern "C" int32_t e2egrec_sample_khop(const e2egrec_csr *graph, const int32_t *
                                        void *scratch, size_t scratch_bytes, void *stream)
 {
     (void)flags;
-    if (!graph || !fanouts || !blocks || !scratch || !graph->indptr) return E2EGREC_ERR_NULL;
     if (n_seeds > 0 && !seeds) return E2EGREC_ERR_NULL;
+    return sample_khop_impl(graph, seeds, n_seeds, nullptr, n_hops, fanouts, seed, step, blocks, scratch, scratch_bytes,
+                            static_cast<cudaStream_t>(stream));
+}
+
+int32_t e2egrec::sample_khop_impl(const e2egrec_csr *graph, const int32_t *seeds, int32_t n_seeds, const PairInput *pairs,
+                                  int32_t n_hops, const int32_t *fanouts, uint64_t seed, uint32_t step,
+                                  const e2egrec_block *blocks, void *scratch, size_t scratch_bytes, cudaStream_t st)
+{
+    if (!graph || !fanouts || !blocks || !scratch || !graph->indptr) return E2EGREC_ERR_NULL;
     if (graph->n_edges > 0 && !graph->indices) return E2EGREC_ERR_NULL;
     if (graph->edge_weight) return E2EGREC_ERR_UNSUPPORTED;
     if (reinterpret_cast<uintptr_t>(scratch) % 256) return E2EGREC_ERR_ALIGN;
@@ -639,14 +698,38 @@ extern "C" int32_t e2egrec_sample_khop(const e2egrec_csr *graph, const int32_t *
     SamplerScratch s = carve(graph->n_nodes, md, ms, me, scratch);
     if (scratch_bytes < s.bytes) return E2EGREC_ERR_WORKSPACE;
 
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
     const int T = 256;
     const int64_t n = graph->n_nodes;
     tap_begin(TAP_SAMPLE, st);
-    note_launch();
-    seed_init_kernel<<<grid_for(n_seeds, T), T, 0, st>>>(seeds, n_seeds, n, s.local_id, blocks[0].counts);
     const int32_t *dst_nodes = seeds;
     const int32_t *n_dst_ptr = &blocks[0].counts[CNT_DST];
+    if (!pairs) {
+        note_launch();
+        seed_init_kernel<<<grid_for(n_seeds, T), T, 0, st>>>(seeds, n_seeds, n, s.local_id, blocks[0].counts);
+    } else {
+        // seeds = ascending distinct endpoints of the pairs; entries (pair, side) grouped by seed
+        const PairInput &pi = *pairs;
+        const int32_t P2 = 2 * pi.n_pairs;
+        cudaMemsetAsync(s.arena, 0, s.arena_bytes, st);
+        cudaMemsetAsync(pi.pcounts, 0, 4 * sizeof(int32_t), st);
+        cudaMemsetAsync(blocks[0].counts, 0, 4 * sizeof(int32_t), st);
+        note_launch();
+        pair_mark_kernel<<<grid_for(pi.n_pairs, T), T, 0, st>>>(pi.user, pi.item, pi.n_pairs, n, s.bitmap, blocks[0].counts);
+        note_launch();
+        frontier_kernel<<<grid_for(s.n_words, kWordTile), 256, 0, st>>>(s.bitmap, s.n_words, pi.pcounts, P2, s.local_id,
+                                                                        pi.seeds_out, s.tickets + 1, s.state_words);
+        const SortPlan sp = sort_plan(P2 > 1 ? P2 : 2);
+        note_launch();
+        pair_local_kernel<<<(unsigned)std::min<int64_t>(grid_for(P2, T), 148 * 4), T, 0, st>>>(
+            pi.user, pi.item, pi.n_pairs, n, s.local_id, pi.pair_local, pi.entry_unit, pi.units_per_row, pi.item_unit_off,
+            pi.pcounts, sp.bits, sp.passes, s.ghist);
+        sort_by_col(pi.pair_local, pi.pcounts, P2, pi.pcsc_col, pi.pcsc_eid, sp, s, st);
+        note_launch();
+        csc_finalize_kernel<<<grid_for((int64_t)P2 + 1, T), T, 0, st>>>(pi.pcsc_col, pi.pcsc_eid, pi.entry_unit, pi.pcounts,
+                                                                       pi.pcsc_ptr, pi.pcsc_idx);
+        dst_nodes = pi.seeds_out;
+        n_dst_ptr = &pi.pcounts[CNT_SRC];
+    }
     for (int h = 0; h < n_hops; ++h) {
         const e2egrec_block &b = blocks[h];
         const int32_t f = fanouts[h];
@@ -664,7 +747,7 @@ extern "C" int32_t e2egrec_sample_khop(const e2egrec_csr *graph, const int32_t *
         note_launch();
         relabel_kernel<<<(unsigned)std::min<int64_t>(grid_for(b.cap_edges, T), 148 * 4), T, 0, st>>>(
             b.nbr_global, s.local_id, b.counts, b.col, sp.bits, sp.passes, s.ghist);
-        sort_by_col(b, sp, s, st);
+        sort_by_col(b.col, b.counts, b.cap_edges, b.csc_col, b.csc_eid, sp, s, st);
         note_launch();
         csc_finalize_kernel<<<grid_for(std::max<int64_t>(b.cap_edges, (int64_t)b.cap_src + 1), T), T, 0, st>>>(
             b.csc_col, b.csc_eid, s.edge_row, b.counts, b.csc_ptr, b.csc_row);
