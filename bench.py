@@ -310,6 +310,49 @@ def run_ours(args, w):
     barrier()
     e2e_s = time.perf_counter() - t0
 
+    # ---- joint step (sampled encoder + ranking tower + BCE, forward and backward) on the same graph
+    joint = None
+    if not args.no_joint:
+        P, dd = w.batch, 64
+        jr = np.random.default_rng(4 + rank)
+        picks = jr.integers(0, inter[0].size, (min(K, 200) + Wm, P))
+        pu_all = torch.from_numpy(inter[0][picks].astype(np.int32)).to(dev)
+        pi_all = torch.from_numpy(inter[1][picks].astype(np.int32)).to(dev)
+        dense = torch.from_numpy(jr.standard_normal((P, dd)).astype(np.float32)).to(dev)
+        labels = torch.from_numpy(S.bernoulli_labels(P, 0.1, 4)).to(dev)
+        zdim = 2 * w.hidden + dd
+        Wt_h = [S.glorot_uniform(512, zdim, 4, 40), S.glorot_uniform(256, 512, 4, 41), S.glorot_uniform(1, 256, 4, 42)]
+        Wt = [torch.from_numpy(a).to(dev, dt) for a in Wt_h]
+        bt = [torch.zeros(a.shape[0], dtype=torch.float32, device=dev) for a in Wt_h]
+        js = E.JointStep(indptr, indices, X, P, dd, w.fanouts, Ws, Wt, bt)
+        pu_in, pi_in = torch.empty_like(pu_all[0]), torch.empty_like(pi_all[0])
+        with torch.cuda.stream(side):
+            for i in range(Wm):
+                pu_in.copy_(pu_all[i]); pi_in.copy_(pi_all[i])
+                js.run(pu_in, pi_in, dense, labels, 4, i)
+        side.synchronize()
+        jgraph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(jgraph, stream=side):
+            js.run(pu_in, pi_in, dense, labels, 4, 0)
+        KJ = picks.shape[0] - Wm
+        barrier()
+        j0, j1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        j0.record()
+        for i in range(KJ):
+            pu_in.copy_(pu_all[Wm + i], non_blocking=True)
+            pi_in.copy_(pi_all[Wm + i], non_blocking=True)
+            E.sampler_set_step(js.ws, rank * 1_000_000 + i)
+            jgraph.replay()
+        j1.record()
+        barrier()
+        jms = j0.elapsed_time(j1)
+        n_rows, jstatus = js.n_rows.tolist()
+        if jstatus:
+            raise RuntimeError(f"joint step: device status bits {jstatus}")
+        joint = dict(metric="joint_step_samples_per_sec", value=KJ * P * world / (jms / 1e3), unit="pairs/s",
+                     ms_per_step=jms / KJ, steps=KJ, pairs_per_step=P, tower="320-512-256-1", dense_dim=dd,
+                     loss=float(js.loss), launch="one CUDA graph replay per step")
+
     # ---- reduce over ranks: slowest rank's time, all ranks' edges
     if world > 1:
         t = torch.tensor([ms, e2e_s], dtype=torch.float64, device=dev)
@@ -360,6 +403,8 @@ def run_ours(args, w):
                 gpu_launches=int(launches),
                 roofline=roof,
                 kernel_ms={TAP_NAMES[k].split(" (")[0]: v for k, v in tap_ms.items()})
+    if joint is not None:
+        line["joint"] = joint
 
     if world == 1 and not args.no_cpu_baseline:
         import oracle
@@ -389,6 +434,7 @@ def main():
     ap.add_argument("--workload", default="medium", choices=sorted(S.WORKLOADS))
     ap.add_argument("--ref-seeds", type=int, default=256, help="seeds per step given to the CPU oracle")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-joint", action="store_true", help="skip the joint-step measurement")
     ap.add_argument("--seeds", default="activity", choices=["activity", "uniform"],
                     help="how seed batches are drawn (see make_batches)")
     args = ap.parse_args()

@@ -124,6 +124,7 @@ struct SegOut {
     const T *mask;          // optional: result is zeroed where mask[s][k] <= 0 (ReLU derivative)
     int64_t ld_mask;
     int mean;               // divide the sum by the segment length
+    int64_t pad_rows;       // if > 0: rows n_seg .. min(next multiple of 128, pad_rows) - 1 of out are zeroed
 };
 
 template <typename T>

@@ -85,10 +85,27 @@ __device__ inline uint64_t make_smem_desc(uint32_t smem_addr)
     return d;
 }
 
-// Instruction descriptor of kind::f16: bf16 x bf16 -> fp32, both operands K-major.
-__device__ inline uint32_t make_idesc(int m, int n)
+// Shared-memory operand descriptor for an operand whose M (or N) index is the contiguous one: the tile is
+// a row of 64-element (128-byte) wide column blocks, each block holding one 128-byte line per K index,
+// 128-byte swizzled in groups of eight lines.  Leading byte offset = distance between column blocks,
+// stride byte offset = distance between groups of eight K lines.
+__device__ inline uint64_t make_smem_desc_mn(uint32_t smem_addr, uint32_t block_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((smem_addr & 0x3FFFFu) >> 4);
+    d |= (uint64_t)((block_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)(1024 >> 4) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)2 << 61;
+    return d;
+}
+
+// Instruction descriptor of kind::f16: bf16 x bf16 -> fp32; mn_major = both operands have their M / N
+// index contiguous in memory (a transposed product), else both are K-major.
+__device__ inline uint32_t make_idesc(int m, int n, bool mn_major = false)
 {
     uint32_t d = 0;
+    if (mn_major) d |= (1u << 15) | (1u << 16);
     d |= 1u << 4;                    // accumulator fp32
     d |= 1u << 7;                    // A bf16
     d |= 1u << 10;                   // B bf16
@@ -343,6 +360,139 @@ bool launch_tn(const __nv_bfloat16 *A, int64_t rows, int k, int64_t lda, const _
     return true;
 }
 
+
+// ------------------------------------------------------------------------- transposed product, split over rows
+//   part[z][m, n] = sum over the rows r of split z of  Y[r, m] * X[r, n]      (weight gradients)
+// Y [rows x M] and X [rows x N] are row-major, so both operands reach the tensor cores with their M / N
+// index contiguous.  A k-block is 64 rows; the blocks up to the first multiple of 64 at or above *m_dev
+// are shared evenly by gridDim.z CTAs per output tile (rows between *m_dev and that multiple must hold
+// zeros in both matrices).  A CTA without blocks writes zeros.
+__global__ void __launch_bounds__(kThreads)
+tc_gemm_rows_kernel(const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_x, int nt,
+                    uint32_t tmem_cols, int stages, const int32_t *m_dev, float *__restrict__ part, int64_t ldp,
+                    int64_t split_stride, int32_t *status)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], accum_bar;
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * kTileM, n0 = blockIdx.y * nt;
+    const int64_t m_valid = *m_dev;
+    const int64_t total_blocks = (m_valid + kTileK - 1) / kTileK;
+    const int64_t per = (total_blocks + gridDim.z - 1) / gridDim.z;
+    const int64_t kb0 = (int64_t)blockIdx.z * per;
+    const int64_t kb1 = kb0 + per < total_blocks ? kb0 + per : total_blocks;
+    const int k_blocks = kb1 > kb0 ? (int)(kb1 - kb0) : 0;
+    float *out = part + (int64_t)blockIdx.z * split_stride + (int64_t)(m0 + warp * 32 + lane) * ldp + n0;
+    if (k_blocks == 0) {
+        for (int c = 0; c < nt; c += 4) *reinterpret_cast<float4 *>(out + c) = make_float4(0.f, 0.f, 0.f, 0.f);
+        return;
+    }
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    constexpr uint32_t blk_bytes = kTileK * 128;            // one 64-column block: 64 K lines of 128 bytes
+    const uint32_t a_bytes = (kTileM / 64) * blk_bytes, b_bytes = (uint32_t)(nt / 64) * blk_bytes;
+    uint8_t *a_tiles = tiles;
+    uint8_t *b_tiles = tiles + (size_t)stages * a_bytes;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(&full_bar[s], 1);
+            mbar_init(&empty_bar[s], 1);
+        }
+        mbar_init(&accum_bar, 1);
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                     "r"(tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+
+    int issued = 0;
+    if (warp == 0 && lane == 0) {
+        for (int kb = 0; kb < k_blocks; ++kb) {
+            const int s = kb % stages;
+            const uint32_t ph = (uint32_t)(kb / stages) & 1u;
+            if (!mbar_wait(&empty_bar[s], ph ^ 1u, &abort_flag)) break;
+            mbar_expect_tx(&full_bar[s], a_bytes + b_bytes);
+            const int row = (int)((kb0 + kb) * kTileK);
+            for (int j = 0; j < kTileM / 64; ++j)
+                tma_load_2d(a_tiles + (size_t)s * a_bytes + j * blk_bytes, &map_y, m0 + j * 64, row, &full_bar[s]);
+            for (int j = 0; j < nt / 64; ++j)
+                tma_load_2d(b_tiles + (size_t)s * b_bytes + j * blk_bytes, &map_x, n0 + j * 64, row, &full_bar[s]);
+            issued = kb + 1;
+        }
+    } else if (warp == 1 && lane == 0) {
+        const uint32_t idesc = make_idesc(kTileM, nt, true);
+        bool ok = true;
+        for (int kb = 0; kb < k_blocks && ok; ++kb) {
+            const int s = kb % stages;
+            const uint32_t ph = (uint32_t)(kb / stages) & 1u;
+            ok = mbar_wait(&full_bar[s], ph, &abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t a_addr = smem_u32(a_tiles + (size_t)s * a_bytes);
+            const uint32_t b_addr = smem_u32(b_tiles + (size_t)s * b_bytes);
+#pragma unroll
+            for (int k = 0; k < kTileK / kUmmaK; ++k) {     // 16 K lines = 2048 bytes further into every block
+                const uint64_t ad = make_smem_desc_mn(a_addr + k * kUmmaK * 128, blk_bytes);
+                const uint64_t bd = make_smem_desc_mn(b_addr + k * kUmmaK * 128, blk_bytes);
+                umma(tmem_base, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+            }
+            umma_commit(&empty_bar[s]);
+        }
+        if (ok) umma_commit(&accum_bar);
+    }
+    __syncwarp();
+
+    const bool ready = mbar_wait(&accum_bar, 0, &abort_flag);
+    tc_fence_after();
+    if (ready) {
+        for (int c = 0; c < nt; c += 32) {
+            uint32_t r[32];
+            tmem_load32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, r);
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                *reinterpret_cast<float4 *>(out + c + q * 4) =
+                    make_float4(__uint_as_float(r[4 * q]), __uint_as_float(r[4 * q + 1]), __uint_as_float(r[4 * q + 2]),
+                                __uint_as_float(r[4 * q + 3]));
+        }
+    } else if (threadIdx.x == 0) {
+        atomicOr(reinterpret_cast<unsigned *>(status), E2EGREC_DEV_TIMEOUT);
+        int never = 0;
+        for (int kb = issued > stages ? issued - stages : 0; kb < issued; ++kb)
+            mbar_wait(&full_bar[kb % stages], (uint32_t)(kb / stages) & 1u, &never);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
+// [rows x cols] bf16 row-major seen with the column index innermost: box = 64 columns x 64 rows
+bool make_map_mn(CUtensorMap *map, const void *base, int64_t rows, int64_t cols)
+{
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kTileK};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 }  // namespace
 
 bool tc_update_forward(const __nv_bfloat16 *cat, int64_t rows, int k, const __nv_bfloat16 *W, int n, const float *bias,
@@ -389,6 +539,37 @@ bool tc_dcat_backward(const __nv_bfloat16 *dz, int64_t rows, int d_out, const __
     ep.m_dev = m_dev;
     ep.status = status;
     return launch_tn(dz, rows, d_out, d_out, Wt, two_d_in, d_out, ep, st);
+}
+
+}  // namespace e2egrec
+
+namespace e2egrec {
+
+bool tc_weight_grad(const __nv_bfloat16 *dY, int64_t rows, int m, const __nv_bfloat16 *Xin, int n, const int32_t *m_dev,
+                    float *part, int splits, int32_t *status, cudaStream_t st)
+{
+    if (rows <= 0 || rows % kTileK || m % kTileM || n % 64) return false;
+    int nt = 0;
+    for (int c = 256; c >= 64; c -= 64)
+        if (n % c == 0) { nt = c; break; }
+    if (!nt) return false;
+    if (reinterpret_cast<uintptr_t>(dY) % 16 || reinterpret_cast<uintptr_t>(Xin) % 16) return false;
+    CUtensorMap my, mx;
+    if (!make_map_mn(&my, dY, rows, m) || !make_map_mn(&mx, Xin, rows, n)) return false;
+    uint32_t tmem_cols = 32;
+    while ((int)tmem_cols < nt) tmem_cols <<= 1;
+    const int stages = kMaxStages;
+    const size_t smem = (size_t)stages * ((kTileM / 64) + (nt / 64)) * (kTileK * 128) + 1024;
+    static bool attr_set = false;
+    if (!attr_set) {
+        if (cudaFuncSetAttribute(tc_gemm_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
+            return false;
+        attr_set = true;
+    }
+    dim3 grid((unsigned)(m / kTileM), (unsigned)(n / nt), (unsigned)splits);
+    note_launch();
+    tc_gemm_rows_kernel<<<grid, kThreads, smem, st>>>(my, mx, nt, tmem_cols, stages, m_dev, part, n, (int64_t)m * n, status);
+    return true;
 }
 
 }  // namespace e2egrec

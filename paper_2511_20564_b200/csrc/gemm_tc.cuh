@@ -23,4 +23,9 @@ bool tc_linear(const __nv_bfloat16 *A, int64_t rows, int k, const __nv_bfloat16 
                const __nv_bfloat16 *mask, int64_t ld_mask, __nv_bfloat16 *out, int64_t ldo, const int32_t *m_dev,
                int32_t *status, cudaStream_t st);
 
+// part[z] = (rows of split z of dY)^T (same rows of Xin): dY [rows x m], Xin [rows x n] bf16 row-major, part
+// [splits x m x n] fp32.  Rows between *m_dev and the next multiple of 64 must be zero in both matrices.
+bool tc_weight_grad(const __nv_bfloat16 *dY, int64_t rows, int m, const __nv_bfloat16 *Xin, int n, const int32_t *m_dev,
+                    float *part, int splits, int32_t *status, cudaStream_t st);
+
 }  // namespace e2egrec

@@ -194,13 +194,16 @@ void linear_backward_input(const T *dY, int64_t rows, int n_out, const T *W, int
 // dW = dY^T X (fp32, rows split kSplits ways and added in order), db = column sums of dY
 template <typename T>
 void linear_backward_weight(const T *dY, int64_t rows, int n_out, const T *Xin, int n_in, const int32_t *m_dev,
-                            float *part, float *dW, float *db, cudaStream_t st)
+                            float *part, float *dW, float *db, int32_t *status, cudaStream_t st)
 {
-    EpiPartial epi{part, n_in, (int64_t)n_out * n_in};
-    dim3 grid((unsigned)ceil_div(n_out, kGemmBM), (unsigned)ceil_div(n_in, kGemmBN), kSplits);
-    note_launch();
-    gemm_simt_kernel<T, true, true, EpiPartial><<<grid, kGemmThreads, 0, st>>>(dY, n_out, Xin, n_in, n_out, n_in, rows, nullptr,
-                                                                              m_dev, epi);
+    if (!(use_tc<T>() && tc_weight_grad(reinterpret_cast<const __nv_bfloat16 *>(dY), rows, n_out,
+                                        reinterpret_cast<const __nv_bfloat16 *>(Xin), n_in, m_dev, part, kSplits, status, st))) {
+        EpiPartial epi{part, n_in, (int64_t)n_out * n_in};
+        dim3 grid((unsigned)ceil_div(n_out, kGemmBM), (unsigned)ceil_div(n_in, kGemmBN), kSplits);
+        note_launch();
+        gemm_simt_kernel<T, true, true, EpiPartial><<<grid, kGemmThreads, 0, st>>>(dY, n_out, Xin, n_in, n_out, n_in, rows,
+                                                                                  nullptr, m_dev, epi);
+    }
     const int64_t n = (int64_t)n_out * n_in;
     note_launch();
     splitk_reduce_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(part, n, kSplits, 0, dW);
@@ -369,9 +372,9 @@ int32_t run_joint(const JointPlan &jp, const e2egrec_csr *graph, const e2egrec_m
         note_launch();
         dz_top_kernel<T><<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(dt, W3, a2, jp.h2, jp.P, jp.rowsP, dz2);
     }
-    linear_backward_weight<T>(dz2, jp.rowsP, jp.h2, a1, jp.h1, pmeta, part, dW_tower[1], db_tower ? db_tower[1] : nullptr, st);
+    linear_backward_weight<T>(dz2, jp.rowsP, jp.h2, a1, jp.h1, pmeta, part, dW_tower[1], db_tower ? db_tower[1] : nullptr, status, st);
     linear_backward_input<T>(dz2, jp.rowsP, jp.h2, W2, jp.h1, a1, dz1, wt, pmeta, status, st);
-    linear_backward_weight<T>(dz1, jp.rowsP, jp.h1, z, jp.zdim, pmeta, part, dW_tower[0], db_tower ? db_tower[0] : nullptr, st);
+    linear_backward_weight<T>(dz1, jp.rowsP, jp.h1, z, jp.zdim, pmeta, part, dW_tower[0], db_tower ? db_tower[0] : nullptr, status, st);
     linear_backward_input<T>(dz1, jp.rowsP, jp.h1, W1, jp.zdim, nullptr, dz, wt, pmeta, status, st);
 
     // 5. gradient of every seed embedding: the rows of dz that belong to it, added in pair order

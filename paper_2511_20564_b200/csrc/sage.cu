@@ -185,12 +185,19 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
         const int two_d = 2 * p.d_in;
         // dW_l = dZ^T [h | agg]   (split over the rows, partial sums added in a fixed order)
         if (l == 0) tap_begin(TAP_DW_OUTER, st);
-        {
+        bool dw_done = false;
+        if (X->dtype == E2EGREC_BF16)
+            dw_done = tc_weight_grad(reinterpret_cast<const __nv_bfloat16 *>(dz), p.rows, p.d_out,
+                                     reinterpret_cast<const __nv_bfloat16 *>(cat), two_d, n_dst, part, kDwSplits,
+                                     &b.counts[CNT_STATUS], st);
+        if (!dw_done) {
             EpiPartial epi{part, two_d, (int64_t)p.d_out * two_d};
             dim3 grid((unsigned)ceil_div(p.d_out, kGemmBM), (unsigned)ceil_div(two_d, kGemmBN), kDwSplits);
             note_launch();
             gemm_simt_kernel<T, true, true, EpiPartial><<<grid, kGemmThreads, 0, st>>>(
                 dz, p.d_out, cat, two_d, p.d_out, two_d, p.rows, nullptr, n_dst, epi);
+        }
+        {
             const int64_t n = (int64_t)p.d_out * two_d;
             note_launch();
             splitk_reduce_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(part, n, kDwSplits, accumulate, dW[l]);
@@ -230,6 +237,7 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
         if (l > 0) {
             o.out = dz_buf[(l - 1) & 1];
             o.ld_out = p.d_in;
+            o.pad_rows = plan[l - 1].rows;
             const int relu_below = act ? act[l - 1] : 1;
             o.mask = relu_below ? reinterpret_cast<const T *>(ctx + plan[l - 1].h_off) : nullptr;
             o.ld_mask = p.d_in;

@@ -366,7 +366,7 @@ seg_final_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_t
     constexpr int W = kAggThreads / 32;
     __shared__ float4 red[W][32];
     const int64_t n_seg = n_seg_dev ? (int64_t)*n_seg_dev : n_seg_host;
-    if (n_seg <= 0) return;
+    if (n_seg < 0) return;
     const int64_t n_self = o.self ? (o.n_self ? (int64_t)*o.n_self : n_seg) : 0;
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
@@ -379,8 +379,16 @@ seg_final_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_t
             for (int k = threadIdx.x & 7; k < d; k += 8)
                 o.out[s * o.ld_out + k] = from_float<T>(seg_finish_value(o, s, 0, k, 0.f, s < n_self));
         }
+        if (o.pad_rows > 0) {                           // zero rows up to the next multiple of 128
+            const int64_t pad_end = min((n_seg + 127) / 128 * 128, o.pad_rows);
+            const int64_t cells = (pad_end - n_seg) * d;
+            for (int64_t t = (int64_t)(blockIdx.x - n_windows) * kAggThreads + threadIdx.x; t < cells;
+                 t += n_extra * kAggThreads)
+                o.out[(n_seg + t / d) * o.ld_out + t % d] = from_float<T>(0.f);
+        }
         return;
     }
+    if (n_seg == 0) return;
     const int64_t win = blockIdx.x;
     const int4 info = win_info[win];
     if (info.x < 0 || !info.y) return;                   // no segment that began earlier ends in this window
