@@ -425,13 +425,117 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------ whole-graph aggregation
+def run_fullgraph(args):
+    """Mean aggregation over the whole graph (no sampling) and its transpose: one forward (CSR gather) and one
+    backward (CSC gather) per step, on a directed power-law graph."""
+    import torch
+    import paper_2511_20564_b200 as E
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    n = int(5_000_000 * args.scale)
+    m = int(100_000_000 * args.scale)
+    d = 64
+    t0 = time.perf_counter()
+    dst, src = S.powerlaw_directed(n, m, 1.1, 2)
+    indptr_h, indices_h = S.coo_to_csr(n, dst, src)
+    order = np.argsort(indices_h, kind="stable")                    # CSC = entries by (source, CSR position)
+    rows_of_entry = np.repeat(np.arange(n, dtype=np.int32), np.diff(indptr_h))
+    csc_row_h = rows_of_entry[order]
+    csc_ptr_h = np.zeros(n + 1, np.int64)
+    np.cumsum(np.bincount(indices_h, minlength=n), out=csc_ptr_h[1:])
+    deg = np.diff(indptr_h)
+    inv_deg_h = np.where(deg > 0, 1.0 / np.maximum(deg, 1), 0.0).astype(np.float32)
+    setup_s = time.perf_counter() - t0
+    X_h = S.to_bf16_values(S.normal_features(n, d, 2))
+    G_h = S.to_bf16_values(S.normal_features(n, d, 2, stream=11))
+    cu = lambda a: torch.from_numpy(a).to(dev)
+    indptr, indices, csc_ptr, csc_row, inv_deg = cu(indptr_h), cu(indices_h), cu(csc_ptr_h), cu(csc_row_h), cu(inv_deg_h)
+    X, G = cu(X_h).to(torch.bfloat16), cu(G_h).to(torch.bfloat16)
+    out = torch.empty(n, d, dtype=torch.bfloat16, device=dev)
+    dX = torch.empty(n, d, dtype=torch.bfloat16, device=dev)
+    _, ws_f = E.aggregate_forward(indptr, indices, X, out)
+    _, ws_b = E.aggregate_backward(csc_ptr, csc_row, inv_deg, G, dX)
+    K, Wm = args.steps, max(args.warmup, 3)
+
+    def fwd():
+        E.aggregate_forward(indptr, indices, X, out, ws_f)
+
+    def bwd():
+        E.aggregate_backward(csc_ptr, csc_row, inv_deg, G, dX, ws_b)
+
+    for _ in range(Wm):
+        fwd(); bwd()
+    torch.cuda.synchronize()
+    clocks = ClockSampler(0)
+    clocks.start()
+    time.sleep(0.6)
+    t_begin = clocks.mark()
+    l0 = E.launch_count()
+    ef = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+          for _ in range(K)]
+    for a, b, c in ef:
+        a.record(); fwd(); b.record(); bwd(); c.record()
+    torch.cuda.synchronize()
+    clk = clocks.stop(t_begin, clocks.mark())
+    launches = E.launch_count() - l0
+    t_f = float(np.mean([a.elapsed_time(b) for a, b, _ in ef]))
+    t_b = float(np.mean([b.elapsed_time(c) for _, b, c in ef]))
+    ms = ef[0][0].elapsed_time(ef[-1][2])
+    # end to end: features from pinned host memory in, aggregated rows out, every step
+    X_pin, G_pin = X.cpu().pin_memory(), G.cpu().pin_memory()
+    out_pin, dX_pin = torch.empty_like(X_pin), torch.empty_like(X_pin)
+    ke = max(2, min(K, 5))
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(ke):
+        X.copy_(X_pin, non_blocking=True); G.copy_(G_pin, non_blocking=True)
+        fwd(); bwd()
+        out_pin.copy_(out, non_blocking=True); dX_pin.copy_(dX, non_blocking=True)
+        torch.cuda.synchronize()
+    e2e_s = (time.perf_counter() - t0) / ke
+    peaks = measured_peaks()
+    r = d * 2
+    alg_f = m * (4 + r) + n * (16 + r)          # per entry: id + gathered row; per row: two offsets + the output row
+    alg_b = m * (4 + 4 + r) + n * (16 + r)      # + the per-entry weight 1/deg
+    big = "fwd" if t_f >= t_b else "bwd"
+    alg, tk = (alg_f, t_f) if big == "fwd" else (alg_b, t_b)
+    roof = dict(bound="hbm", achieved=alg / tk / 1e6, peak=peaks["hbm_gbs"], unit="GB/s", traffic=None,
+                kernel=f"seg_run_kernel+seg_window_kernel+seg_final_kernel ({big})", ms_per_launch=tk,
+                algorithmic_units_per_launch=alg, peak_source=peaks["source"],
+                compulsory_bytes=n * r * 2 + m * 4 + n * 16)
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    line = dict(metric="fullgraph_mean_aggregation_fwd_bwd_edges_per_sec", value=m / ((t_f + t_b) / 1e3), unit="edges/s",
+                n_gpus=1, steps=K, warmup=Wm, ms_per_step=ms / K, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="bf16", data="synthetic",
+                config=dict(workload="fullgraph", nodes=n, csr_entries=m, dim=d, alpha=1.1, max_degree=int(deg.max()),
+                            l2="inputs larger than L2 (features %.0f MB, indices %.0f MB)" % (n * r / 1e6, m * 4 / 1e6),
+                            host_setup_s=round(setup_s, 1)),
+                fwd_ms=t_f, bwd_ms=t_b, fwd_edges_per_s=m / (t_f / 1e3), bwd_edges_per_s=m / (t_b / 1e3),
+                fwd_gbs=alg_f / t_f / 1e6, bwd_gbs=alg_b / t_b / 1e6, clocks=clk,
+                e2e=dict(value=m / e2e_s, unit="edges/s", h2d_bytes_per_step=2 * n * r, d2h_bytes_per_step=2 * n * r,
+                         ms_per_step=e2e_s * 1e3),
+                gpu_launches=int(launches), roofline=roof)
+    if not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        rows = min(n, 200_000)
+        t0 = time.perf_counter()
+        oracle.mean_aggregate(indptr_h[: rows + 1], indices_h[: int(indptr_h[rows])], X_h, True)
+        cdt = time.perf_counter() - t0
+        line["cpu_baseline"] = dict(value=int(indptr_h[rows]) / cdt, unit="edges/s", cores=1, kind="oracle",
+                                    sample=f"forward mean aggregation of the first {rows} rows ({int(indptr_h[rows])} entries), {cdt:.1f} s")
+    print(json.dumps(line), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=1000)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="medium", choices=sorted(S.WORKLOADS))
+    ap.add_argument("--workload", default="medium", choices=sorted(S.WORKLOADS) + ["fullgraph"])
+    ap.add_argument("--scale", type=float, default=1.0, help="fullgraph only: fraction of the 5 M node / 100 M entry graph")
     ap.add_argument("--ref-seeds", type=int, default=256, help="seeds per step given to the CPU oracle")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-joint", action="store_true", help="skip the joint-step measurement")
@@ -439,6 +543,10 @@ def main():
                     help="how seed batches are drawn (see make_batches)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.workload == "fullgraph":
+        if args.impl == "ours" and int(os.environ.get("RANK", "0")) == 0:
+            run_fullgraph(args)
+        return
     w = S.WORKLOADS[args.workload]
     if args.impl == "reference":
         run_reference(args, w)

@@ -88,7 +88,40 @@ template <> __device__ inline void store4<__nv_bfloat16>(__nv_bfloat16 *p, const
 }
 
 // ------------------------------------------------------------------------------------ level 1
-template <typename T, typename PtrT, int LPR, int CPL, bool kWeight>
+// Rarely taken paths of the level-1 kernel, kept out of line so that the streaming loop stays short.
+template <int CPL, int E>
+__device__ __noinline__ void seg_store_partial(float *dst, const float (&acc)[CPL][E], int c, int lpr, int n_chunks)
+{
+#pragma unroll
+    for (int q = 0; q < CPL; ++q) {
+        const int ch = c + q * lpr;
+        if (ch < n_chunks) {
+#pragma unroll
+            for (int e = 0; e < E; e += 4)
+                *reinterpret_cast<float4 *>(dst + ch * E + e) = make_float4(acc[q][e], acc[q][e + 1], acc[q][e + 2], acc[q][e + 3]);
+        }
+    }
+}
+
+// Advances the walk to the segment that holds entry k (k >= end of segment *ws): a few steps one by one,
+// then by bisection if a long stretch of empty segments is in the way.  Returns that segment's end.
+template <typename PtrT>
+__device__ __noinline__ int64_t seg_advance(const PtrT *__restrict__ ptr, int64_t n_seg, int64_t k, int64_t *ws)
+{
+    int64_t s = *ws, end;
+    int step = 0;
+    do { ++s; end = (int64_t)ptr[s + 1]; } while (end <= k && ++step < 4);
+    if (end <= k) {
+        s = seg_containing(ptr, n_seg, k);
+        end = (int64_t)ptr[s + 1];
+    }
+    *ws = s;
+    return end;
+}
+
+// kExtra: the output has a self row and/or a mask row per segment (they are fetched together with the
+// segment's first gathered row); without it those registers and branches disappear.
+template <typename T, typename PtrT, int LPR, int CPL, bool kWeight, bool kExtra>
 __global__ void __launch_bounds__(kAggThreads)
 seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__ ptr, const int32_t *__restrict__ idx,
                const int32_t *n_seg_dev, int64_t n_seg_host, const float *__restrict__ w, int run_len, int d,
@@ -97,6 +130,7 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
 {
     constexpr int E = Chunk<T>::kElems;
     constexpr int U = CPL >= 4 ? 1 : 4 / CPL;
+    constexpr int kFar = 1 << 30;
     const int c = threadIdx.x % LPR;
     const int n_chunks = d / E;
     const int64_t run = ((int64_t)blockIdx.x * kAggThreads + threadIdx.x) / LPR;
@@ -108,66 +142,59 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
         if (c == 0) run_info[run] = make_int4(-1, 0, -1, 0);
         return;
     }
-    const int64_t k1 = min(k0 + (int64_t)run_len, total);
-    const int64_t n_self = o.self ? (o.n_self ? (int64_t)*o.n_self : n_seg) : 0;
+    const int len = (int)min((int64_t)run_len, total - k0);       // entries of this run; positions below are relative to k0
+    const int32_t *__restrict__ idx0 = idx + k0;
+    const int32_t *__restrict__ seg0 = seg_of ? seg_of + k0 : nullptr;
+    const int64_t n_self = (kExtra && o.self) ? (o.n_self ? (int64_t)*o.n_self : n_seg) : 0;
 
-    // Segment boundaries are found one iteration ahead of the sums, so that the self row and the mask
-    // row of a segment are requested together with its first gathered row.  With an entry -> segment
-    // array (seg_of) a boundary is a change of that value; without it the offsets are walked, leaping
-    // over stretches of empty segments by bisection.
-    int64_t ws, w_beg = 0, w_end = 0;
-    bool first_begins, last_ends;
-    if (seg_of) {
-        ws = seg_of[k0];
-        first_begins = k0 == 0 || seg_of[k0 - 1] != (int32_t)ws;
-        last_ends = k1 == total || seg_of[k1] != seg_of[k1 - 1];
+    // Segment boundaries are found one iteration ahead of the sums.  With an entry -> segment array a
+    // boundary is a change of that value; without it the offsets are walked.
+    int64_t ws;                    // segment of the entry classified last
+    int rel_end = kFar;            // its end (walk mode)
+    int first_beg_rel = 0;         // where the run's first segment begins (<= 0)
+    bool first_begins, last_ends = false;
+    if (seg0) {
+        ws = seg0[0];
+        first_begins = k0 == 0 || seg0[-1] != (int32_t)ws;
+        last_ends = k0 + len == total || seg0[len] != seg0[len - 1];
+        if (o.mean) first_beg_rel = (int)max((int64_t)ptr[ws] - k0, (int64_t)-kFar);
     } else {
         ws = seg_containing(ptr, n_seg, k0);
-        w_beg = (int64_t)ptr[ws];
-        w_end = (int64_t)ptr[ws + 1];
-        first_begins = w_beg >= k0;
-        last_ends = false;                            // decided after the walk has reached the last entry
+        const int64_t wb = (int64_t)ptr[ws] - k0;
+        first_begins = wb >= 0;
+        first_beg_rel = (int)max(wb, (int64_t)-kFar);
+        rel_end = (int)min((int64_t)ptr[ws + 1] - k0, (int64_t)kFar);
     }
 
     int32_t seg_n[U], id_n[U];
     bool start_n[U];
-    float inv_n[U];
-    auto classify = [&](int64_t k) {
+    auto classify = [&](int r0) {
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            const int64_t kk = k + u;
+            const int r = r0 + u;
             start_n[u] = false;
-            seg_n[u] = 0; id_n[u] = 0; inv_n[u] = 0.f;
-            if (kk < k1) {
-                if (seg_of) {
-                    const int64_t sg = seg_of[kk];
-                    start_n[u] = kk == k0 || sg != ws;
+            seg_n[u] = 0;
+            id_n[u] = 0;
+            if (r < len) {
+                if (seg0) {
+                    const int32_t sg = seg0[r];
+                    start_n[u] = r == 0 || sg != (int32_t)ws;
                     ws = sg;
-                    if (o.mean && start_n[u]) inv_n[u] = 1.0f / (float)((int64_t)ptr[sg + 1] - (int64_t)ptr[sg]);
-                } else {
-                    if (kk == k0) {
-                        start_n[u] = true;
-                    } else if (kk >= w_end) {
-                        int step = 0;
-                        do { ++ws; w_end = (int64_t)ptr[ws + 1]; } while (w_end <= kk && ++step < 4);
-                        if (w_end <= kk) {                 // a long stretch of empty segments
-                            ws = seg_containing(ptr, n_seg, kk);
-                            w_end = (int64_t)ptr[ws + 1];
-                        }
-                        w_beg = kk;
-                        start_n[u] = true;
-                    }
-                    if (o.mean && start_n[u]) inv_n[u] = 1.0f / (float)(w_end - (kk == k0 ? w_beg : kk));
+                } else if (r == 0) {
+                    start_n[u] = true;
+                } else if (r >= rel_end) {
+                    rel_end = (int)min(seg_advance(ptr, n_seg, k0 + r, &ws) - k0, (int64_t)kFar);
+                    start_n[u] = true;
                 }
                 seg_n[u] = (int32_t)ws;
-                id_n[u] = idx[kk];
+                id_n[u] = idx0[r];
             }
         }
     };
 
-    int64_t cur_seg = -1;
+    int32_t cur_seg = -1;
+    int cur_beg_rel = 0;
     bool cur_begins = false;
-    float cur_inv = 0.f;
     uint4 cur_mask[CPL];
     float acc[CPL][E];
 #pragma unroll
@@ -178,79 +205,83 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
     }
     int32_t head_seg = -1, head_ends = 0, tail_seg = -1;
 
-    // closes the current segment with the sum in acc
-    auto emit = [&](bool ended) {
+    // closes the current segment, which ends at relative position end_rel, with the sum in acc
+    auto emit = [&](bool ended, int end_rel) {
+        if (cur_begins && ended) {
+            const float inv = o.mean ? 1.0f / (float)(end_rel - cur_beg_rel) : 1.0f;
 #pragma unroll
-        for (int q = 0; q < CPL; ++q) {
-            const int ch = c + q * LPR;
-            if (ch < n_chunks) {
-                if (cur_begins && ended) {
-                    float r[E], m[E];
-                    Chunk<T>::unpack(cur_mask[q], m);
+            for (int q = 0; q < CPL; ++q) {
+                const int ch = c + q * LPR;
+                if (ch < n_chunks) {
+                    float r[E];
 #pragma unroll
-                    for (int e = 0; e < E; ++e) {
-                        r[e] = seg_round(o, cur_inv, acc[q][e]);
-                        if (o.mask && !(m[e] > 0.f)) r[e] = 0.f;
+                    for (int e = 0; e < E; ++e) r[e] = to_float<T>(from_float<T>(acc[q][e] * inv));
+                    if (kExtra && o.mask) {
+                        float m[E];
+                        Chunk<T>::unpack(cur_mask[q], m);
+#pragma unroll
+                        for (int e = 0; e < E; ++e)
+                            if (!(m[e] > 0.f)) r[e] = 0.f;
                     }
-                    Chunk<T>::store(o.out + cur_seg * o.ld_out + ch * E, r);
-                } else {
-                    float *dst = (cur_begins ? tail : head) + run * d + ch * E;
-#pragma unroll
-                    for (int e = 0; e < E; e += 4)
-                        *reinterpret_cast<float4 *>(dst + e) = make_float4(acc[q][e], acc[q][e + 1], acc[q][e + 2], acc[q][e + 3]);
+                    Chunk<T>::store(o.out + (int64_t)cur_seg * o.ld_out + ch * E, r);
                 }
             }
-        }
-        if (!(cur_begins && ended)) {
-            if (cur_begins) tail_seg = (int32_t)cur_seg;
-            else { head_seg = (int32_t)cur_seg; head_ends = ended ? 1 : 0; }
+        } else {
+            seg_store_partial<CPL, E>((cur_begins ? tail : head) + run * d, acc, c, LPR, n_chunks);
+            if (cur_begins) tail_seg = cur_seg;
+            else { head_seg = cur_seg; head_ends = ended ? 1 : 0; }
         }
     };
 
-    classify(k0);
-    for (int64_t k = k0; k < k1; k += U) {
+    classify(0);
+    for (int r0 = 0; r0 < len; r0 += U) {
         int32_t seg_c[U];
         bool start_c[U];
-        float inv_c[U], wt[U];
-        uint4 v[U][CPL], sv[U][CPL], mv[U][CPL];
+        float wt[U];
+        uint4 v[U][CPL], sv[kExtra ? U : 1][CPL], mv[kExtra ? U : 1][CPL];
 #pragma unroll
         for (int u = 0; u < U; ++u) {
             seg_c[u] = seg_n[u];
             start_c[u] = start_n[u];
-            inv_c[u] = inv_n[u];
             wt[u] = 1.f;
-            const bool live = k + u < k1;
+            const bool live = r0 + u < len;
             const int32_t id = id_n[u];
             if (kWeight && live) wt[u] = w[id];
-            const bool begins = live && start_c[u] && (k + u != k0 || first_begins);
-            const bool want_self = begins && seg_c[u] < n_self;
-            const bool want_mask = live && start_c[u] && o.mask != nullptr;
 #pragma unroll
             for (int q = 0; q < CPL; ++q) {
                 const int ch = c + q * LPR;
                 v[u][q] = make_uint4(0, 0, 0, 0);
-                sv[u][q] = v[u][q];
-                mv[u][q] = v[u][q];
-                if (ch < n_chunks) {
-                    if (live) v[u][q] = Chunk<T>::load_raw(in + (int64_t)id * ld_in + ch * E);
-                    if (want_self) sv[u][q] = Chunk<T>::load_raw(o.self + (int64_t)seg_c[u] * o.ld_self + ch * E);
-                    if (want_mask) mv[u][q] = Chunk<T>::load_raw(o.mask + (int64_t)seg_c[u] * o.ld_mask + ch * E);
+                if (live && ch < n_chunks) v[u][q] = Chunk<T>::load_raw(in + (int64_t)id * ld_in + ch * E);
+                if (kExtra) {
+                    sv[u][q] = make_uint4(0, 0, 0, 0);
+                    mv[u][q] = make_uint4(0, 0, 0, 0);
+                    if (live && start_c[u] && ch < n_chunks) {
+                        const bool begins = r0 + u != 0 || first_begins;
+                        if (begins && seg_c[u] < n_self)
+                            sv[u][q] = Chunk<T>::load_raw(o.self + (int64_t)seg_c[u] * o.ld_self + ch * E);
+                        if (o.mask) mv[u][q] = Chunk<T>::load_raw(o.mask + (int64_t)seg_c[u] * o.ld_mask + ch * E);
+                    }
                 }
             }
         }
-        if (k + U < k1) classify(k + U);
+        if (r0 + U < len) classify(r0 + U);
 #pragma unroll
         for (int u = 0; u < U; ++u) {
-            if (k + u < k1) {
+            if (r0 + u < len) {
                 if (start_c[u]) {
-                    if (cur_seg >= 0) emit(true);
+                    if (cur_seg >= 0) emit(true, r0 + u);
                     cur_seg = seg_c[u];
-                    cur_begins = (k + u != k0) || first_begins;
-                    cur_inv = inv_c[u];
+                    cur_begins = r0 + u != 0 || first_begins;
+                    cur_beg_rel = r0 + u != 0 ? r0 + u : first_beg_rel;
 #pragma unroll
                     for (int q = 0; q < CPL; ++q) {
-                        Chunk<T>::unpack(sv[u][q], acc[q]);          // the self row (zeros if there is none)
-                        cur_mask[q] = mv[u][q];
+                        if (kExtra) {
+                            Chunk<T>::unpack(sv[u][q], acc[q]);          // the self row (zeros if there is none)
+                            cur_mask[q] = mv[u][q];
+                        } else {
+#pragma unroll
+                            for (int e = 0; e < E; ++e) acc[q][e] = 0.f;
+                        }
                     }
                 }
 #pragma unroll
@@ -266,7 +297,7 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
             }
         }
     }
-    emit(seg_of ? last_ends : w_end <= k1);
+    emit(seg0 ? last_ends : rel_end <= len, len);
     if (c == 0) run_info[run] = make_int4(head_seg, head_ends, tail_seg, 0);
 }
 
@@ -441,8 +472,13 @@ inline void launch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const
 {
     tap_begin(TAP_SEG_L1, st);
     note_launch();
-    seg_run_kernel<T, PtrT, LPR, CPL, kWeight><<<(unsigned)ceil_div(sc.cap_runs * LPR, kAggThreads), kAggThreads, 0, st>>>(
-        in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head, sc.tail, sc.run_info, sc.cap_runs, seg_of, o);
+    const unsigned grid1 = (unsigned)ceil_div(sc.cap_runs * LPR, kAggThreads);
+    if (o.self || o.mask)
+        seg_run_kernel<T, PtrT, LPR, CPL, kWeight, true><<<grid1, kAggThreads, 0, st>>>(
+            in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head, sc.tail, sc.run_info, sc.cap_runs, seg_of, o);
+    else
+        seg_run_kernel<T, PtrT, LPR, CPL, kWeight, false><<<grid1, kAggThreads, 0, st>>>(
+            in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head, sc.tail, sc.run_info, sc.cap_runs, seg_of, o);
     tap_end(TAP_SEG_L1, st);
     tap_begin(TAP_SEG_L2, st);
     note_launch();
