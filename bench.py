@@ -183,8 +183,9 @@ def run_ours(args, w):
     Ws = [torch.from_numpy(W).to(dev, dt) for W in Ws_h]
     K, Wm = args.steps, args.warmup
     total = K + Wm
+    first_step = rank * 1_000_000                      # = replicas.first_step_of(rank)
     # every rank trains on its own batches (data parallel replicas; no exchange on the measured path)
-    seeds_h = make_batches(w, inter, args.seeds, rank * 1_000_000, total)
+    seeds_h = make_batches(w, inter, args.seeds, first_step, total)
     seeds_pin = torch.from_numpy(seeds_h).pin_memory()
     seeds_dev = seeds_pin.to(dev)
     dH_h = upstream_grad(w, w.batch)
@@ -221,7 +222,7 @@ def run_ours(args, w):
     with torch.cuda.stream(side):
         for i in range(Wm):                              # eager warm-up on the capture stream
             seeds_in.copy_(seeds_dev[i])
-            E.sampler_set_step(blocks.scratch, rank * 1_000_000 + i)
+            E.sampler_set_step(blocks.scratch, first_step + i)
             step_body()
     side.synchronize()
     launches_before = E.launch_count()
@@ -236,7 +237,7 @@ def run_ours(args, w):
 
     def run_step(i, g=None):
         seeds_in.copy_(seeds_dev[i], non_blocking=True)
-        E.sampler_set_step(blocks.scratch, rank * 1_000_000 + i)
+        E.sampler_set_step(blocks.scratch, first_step + i)
         if g is None:
             step_body()
         else:
@@ -291,7 +292,7 @@ def run_ours(args, w):
     def e2e_step(i):
         seeds_in.copy_(seeds_pin[i], non_blocking=True)
         dH_in.copy_(dH_pin, non_blocking=True)
-        E.sampler_set_step(blocks.scratch, rank * 1_000_000 + i)
+        E.sampler_set_step(blocks.scratch, first_step + i)
         graph.replay()
         res_pin[0].copy_(H_out, non_blocking=True)
         for t, s in zip(res_pin[1:], dWs):
@@ -341,7 +342,7 @@ def run_ours(args, w):
         for i in range(KJ):
             pu_in.copy_(pu_all[Wm + i], non_blocking=True)
             pi_in.copy_(pi_all[Wm + i], non_blocking=True)
-            E.sampler_set_step(js.ws, rank * 1_000_000 + i)
+            E.sampler_set_step(js.ws, first_step + i)
             jgraph.replay()
         j1.record()
         barrier()
@@ -354,15 +355,8 @@ def run_ours(args, w):
                      loss=float(js.loss), launch="one CUDA graph replay per step")
 
     # ---- reduce over ranks: slowest rank's time, all ranks' edges
-    if world > 1:
-        t = torch.tensor([ms, e2e_s], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms, e2e_s = float(t[0]), float(t[1])
-        c = torch.tensor([edges_rank, e2e_edges], dtype=torch.int64, device=dev)
-        dist.all_reduce(c, op=dist.ReduceOp.SUM)
-        edges_all, e2e_edges_all = int(c[0]), int(c[1])
-    else:
-        edges_all, e2e_edges_all = edges_rank, e2e_edges
+    from paper_2511_20564_b200 import replicas
+    (ms, e2e_s), (edges_all, e2e_edges_all) = replicas.reduce_measurements([ms, e2e_s], [edges_rank, e2e_edges], dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()

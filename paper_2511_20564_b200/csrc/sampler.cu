@@ -251,33 +251,64 @@ hop_sample_kernel(const int64_t *__restrict__ g_indptr, const int32_t *__restric
         if (total > cap_edges) atomicOr((unsigned *)&counts[CNT_STATUS], E2EGREC_DEV_CAPACITY);
     }
     const uint32_t step = step_arg + *step_offset;
-    for (int32_t sl = threadIdx.x; sl < tile_total; sl += kDstTile) {
-        int lo = 0, hi = kDstTile;                   // largest r with off[r] <= sl
-        while (hi - lo > 1) {
-            const int mid = (lo + hi) >> 1;
-            if (off[mid] <= sl) lo = mid; else hi = mid;
+    // four slots per thread and round, so that the loads of the graph entry, of the frontier position and of
+    // the bitmap word are in flight for all four before any of them is needed
+    constexpr int S = 4;
+    for (int32_t sl0 = threadIdx.x; sl0 < tile_total; sl0 += kDstTile * S) {
+        int rr[S];
+        long long e[S];
+        int64_t src[S];
+        bool ok[S];
+#pragma unroll
+        for (int q = 0; q < S; ++q) {
+            const int32_t sl = sl0 + q * kDstTile;
+            ok[q] = sl < tile_total;
+            rr[q] = 0;
+            e[q] = 0;
+            src[q] = 0;
+            if (!ok[q]) continue;
+            int lo = 0, hi = kDstTile;               // largest r with off[r] <= sl
+            while (hi - lo > 1) {
+                const int mid = (lo + hi) >> 1;
+                if (off[mid] <= sl) lo = mid; else hi = mid;
+            }
+            rr[q] = lo;
+            const int32_t j = sl - off[lo];
+            e[q] = base + sl;
+            if (e[q] >= cap_edges) { ok[q] = false; continue; }
+            const int64_t deg = deg_s[lo];
+            int64_t pos = j;
+            if (deg > fanout) {
+                const uint4 r4 = philox4x32_10(make_uint4((uint32_t)(j >> 1), (uint32_t)node[lo], (1u << 8) | (uint32_t)hop, step),
+                                               make_uint2(seed_lo, seed_hi));
+                const uint64_t rnd = (j & 1) ? (((uint64_t)r4.w << 32) | r4.z) : (((uint64_t)r4.y << 32) | r4.x);
+                pos = (int64_t)__umul64hi(rnd, (uint64_t)deg);
+            }
+            src[q] = gbeg_s[lo] + pos;
         }
-        const int r = lo;
-        const int32_t j = sl - off[r];
-        const long long e = base + sl;
-        if (e >= cap_edges) continue;
-        const int32_t u = node[r];
-        const int64_t deg = deg_s[r];
-        int64_t pos = j;
-        if (deg > fanout) {
-            const uint4 r4 = philox4x32_10(make_uint4((uint32_t)(j >> 1), (uint32_t)u, (1u << 8) | (uint32_t)hop, step),
-                                           make_uint2(seed_lo, seed_hi));
-            const uint64_t rr = (j & 1) ? (((uint64_t)r4.w << 32) | r4.z) : (((uint64_t)r4.y << 32) | r4.x);
-            pos = (int64_t)__umul64hi(rr, (uint64_t)deg);
+        int32_t v[S];
+#pragma unroll
+        for (int q = 0; q < S; ++q) v[q] = ok[q] ? __ldg(&g_indices[src[q]]) : 0;
+        int32_t lid[S];
+#pragma unroll
+        for (int q = 0; q < S; ++q) {
+            if (ok[q] && (uint32_t)v[q] >= (uint64_t)n_nodes) {
+                atomicOr((unsigned *)&counts[CNT_STATUS], E2EGREC_DEV_RANGE);
+                v[q] = node[rr[q]];
+            }
+            lid[q] = ok[q] ? local_id[v[q]] : 0;
         }
-        int32_t v = g_indices[gbeg_s[r] + pos];
-        if ((uint32_t)v >= (uint64_t)n_nodes) {
-            atomicOr((unsigned *)&counts[CNT_STATUS], E2EGREC_DEV_RANGE);
-            v = u;
+        uint32_t word[S];
+#pragma unroll
+        for (int q = 0; q < S; ++q)   // hubs are sampled thousands of times per hop: look before the atomic
+            word[q] = (ok[q] && lid[q] < 0) ? *reinterpret_cast<volatile uint32_t *>(&bitmap[v[q] >> 5]) : 0xFFFFFFFFu;
+#pragma unroll
+        for (int q = 0; q < S; ++q) {
+            if (!ok[q]) continue;
+            nbr_global[e[q]] = v[q];
+            edge_row[e[q]] = (int32_t)(i0 + rr[q]);
+            if (lid[q] < 0 && !(word[q] & (1u << (v[q] & 31)))) atomicOr(&bitmap[v[q] >> 5], 1u << (v[q] & 31));
         }
-        nbr_global[e] = v;
-        edge_row[e] = (int32_t)(i0 + r);
-        if (local_id[v] < 0) atomicOr(&bitmap[v >> 5], 1u << (v & 31));
     }
 }
 
@@ -434,29 +465,56 @@ sort_pass_kernel(const int32_t *__restrict__ keys_in, const int32_t *__restrict_
             atomicExch(&state[(size_t)d * n_tiles + tile], (tile == 0 ? kChainPrefix : kChainAgg) | (unsigned long long)cnt[q]);
         }
     }
+    // look-back for all of this thread's digits together: a batch of earlier tiles per digit is read at
+    // once, then taken in order; an entry that is not published yet is polled (bounded) before going on
+    long long excl[DPT];
+    int next_p[DPT];
+    bool timed_out = false;
+#pragma unroll
+    for (int q = 0; q < DPT; ++q) {
+        excl[q] = 0;
+        next_p[q] = (threadIdx.x + q * kSortThreads < R && tile > 0) ? tile - 1 : -1;
+    }
+    for (;;) {
+        bool any = false;
+#pragma unroll
+        for (int q = 0; q < DPT; ++q) any = any || next_p[q] >= 0;
+        if (!any || timed_out) break;
+        constexpr int kBatch = 8;
+        unsigned long long v[DPT][kBatch];
+#pragma unroll
+        for (int q = 0; q < DPT; ++q) {
+            const unsigned long long *st = state + (size_t)(threadIdx.x + q * kSortThreads) * n_tiles;
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) v[q][j] = next_p[q] - j >= 0 ? chain_read(&st[next_p[q] - j]) : kChainPrefix;
+        }
+#pragma unroll
+        for (int q = 0; q < DPT; ++q) {
+            if (next_p[q] < 0) continue;
+            const unsigned long long *st = state + (size_t)(threadIdx.x + q * kSortThreads) * n_tiles;
+            bool found = false;
+#pragma unroll
+            for (int j = 0; j < kBatch; ++j) {
+                if (found || timed_out) continue;
+                unsigned long long x = v[q][j];
+                for (int spin = 0; (x >> 62) == 0; ++spin) {
+                    if (spin >= kChainSpinLimit) { timed_out = true; break; }
+                    x = chain_read(&st[next_p[q] - j]);
+                }
+                if (timed_out) continue;
+                excl[q] += (long long)(x & kChainMask);
+                if ((x >> 62) == 2) found = true;
+            }
+            next_p[q] = found ? -1 : next_p[q] - kBatch;
+        }
+    }
+    if (timed_out) atomicOr(reinterpret_cast<unsigned *>(&counts[CNT_STATUS]), E2EGREC_DEV_TIMEOUT);
 #pragma unroll
     for (int q = 0; q < DPT; ++q) {
         const int d = threadIdx.x + q * kSortThreads;
         if (d >= R) continue;
-        unsigned long long *st = state + (size_t)d * n_tiles;
-        long long excl = 0;
-        if (tile > 0) {
-            bool timed_out = false;
-            for (int p = tile - 1; p >= 0; --p) {
-                unsigned long long v = 0;
-                for (int spin = 0;; ++spin) {
-                    v = chain_read(&st[p]);
-                    if ((v >> 62) != 0) break;
-                    if (spin >= kChainSpinLimit) { timed_out = true; break; }
-                }
-                if (timed_out) break;
-                excl += (long long)(v & kChainMask);
-                if ((v >> 62) == 2) break;
-            }
-            if (timed_out) atomicOr(reinterpret_cast<unsigned *>(&counts[CNT_STATUS]), E2EGREC_DEV_TIMEOUT);
-            atomicExch(&st[tile], kChainPrefix | (unsigned long long)(excl + cnt[q]));
-        }
-        int32_t run = bin_base[d] + (int32_t)excl;
+        if (tile > 0) atomicExch(&state[(size_t)d * n_tiles + tile], kChainPrefix | (unsigned long long)(excl[q] + cnt[q]));
+        int32_t run = bin_base[d] + (int32_t)excl[q];
 #pragma unroll
         for (int w = 0; w < W; ++w) {
             const int32_t c2 = wc[w][d];
