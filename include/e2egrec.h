@@ -123,6 +123,20 @@ const char *e2egrec_last_error(void);
 uint64_t e2egrec_launch_count(void);
 int32_t e2egrec_profile_tap(int32_t which, void *start_event, void *stop_event);
 
+/* Graph ingest (Sec. 3, Notation: G = (V, E), N(u)); set-up work, not part of a training step.
+ * e2egrec_graph_from_coo: canonical CSR of an edge list.  row, col: device int32[n_edges]; outputs indptr
+ * device int64[n_nodes+1] and indices device int32[n_edges]: row u lists its neighbours in ascending id
+ * order, parallel edges kept.  The result depends only on the multiset of edges.
+ * e2egrec_csr_transpose: the CSC of a CSR with n_cols columns: csc_ptr device int64[n_cols+1]; for every
+ * transposed entry csc_row int32 (its row) and csc_eid int64 (its CSR position), entries of a column in
+ * CSR order.  status: optional device int32, receives E2EGREC_DEV_RANGE if an id was out of range (such
+ * ids are treated as 0).  ws: scratch (size query with ws == NULL).  Limits: n_edges < 2^31 - 1. */
+int32_t e2egrec_graph_from_coo(int64_t n_nodes, int64_t n_edges, const int32_t *row, const int32_t *col,
+                               int64_t *indptr, int32_t *indices, int32_t *status, void *ws, size_t *ws_bytes,
+                               void *stream);
+int32_t e2egrec_csr_transpose(const e2egrec_csr *csr, int64_t n_cols, int64_t *csc_ptr, int32_t *csc_row,
+                              int64_t *csc_eid, int32_t *status, void *ws, size_t *ws_bytes, void *stream);
+
 /* Worst-case capacities of the blocks of a k-hop sample and the scratch size
  * (Sec. 4.1: depth L, at most k neighbours per node).  fanouts: host int32[n_hops],
  * fanouts[0] is the hop taken from the seeds.  cap_dst / cap_src / cap_edges: host

@@ -96,6 +96,12 @@ def lib():
                                          C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
                                          C.c_void_p, C.c_void_p, C.POINTER(Mat), C.c_void_p, C.c_void_p, C.c_void_p,
                                          C.POINTER(C.c_size_t), C.c_void_p]
+        L.e2egrec_graph_from_coo.restype = C.c_int32
+        L.e2egrec_graph_from_coo.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                             C.c_void_p, C.c_void_p, C.POINTER(C.c_size_t), C.c_void_p]
+        L.e2egrec_csr_transpose.restype = C.c_int32
+        L.e2egrec_csr_transpose.argtypes = [C.POINTER(Csr), C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                            C.c_void_p, C.POINTER(C.c_size_t), C.c_void_p]
         L.e2egrec_launch_count.restype = C.c_uint64
         L.e2egrec_profile_tap.restype = C.c_int32
         L.e2egrec_profile_tap.argtypes = [C.c_int32, C.c_void_p, C.c_void_p]
@@ -413,3 +419,39 @@ class JointStep:
     def run(self, pair_user, pair_item, dense, labels, seed, step, stream=None):
         self._call(pair_user, pair_item, dense, labels, C.c_size_t(self.ws.numel()), _stream(stream), seed, step)
         return self
+
+
+# ------------------------------------------------------------------------------------------ graph ingest
+
+def graph_from_coo(n_nodes: int, row: torch.Tensor, col: torch.Tensor, stream=None):
+    """Enqueues the canonical CSR of an edge list; returns (indptr int64, indices int32, status int32[1])."""
+    m, dev = row.numel(), row.device
+    indptr = torch.empty(n_nodes + 1, dtype=torch.int64, device=dev)
+    indices = torch.empty(max(m, 1), dtype=torch.int32, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    n = C.c_size_t(0)
+    _check(lib().e2egrec_graph_from_coo(n_nodes, m, None, None, None, None, None, None, C.byref(n), None),
+           "e2egrec_graph_from_coo(size query)")
+    ws = _dev_bytes(n.value, dev)
+    n = C.c_size_t(ws.numel())
+    _check(lib().e2egrec_graph_from_coo(n_nodes, m, _ptr(row), _ptr(col), _ptr(indptr), _ptr(indices), _ptr(status),
+                                        _ptr(ws), C.byref(n), _stream(stream)), "e2egrec_graph_from_coo")
+    return indptr, indices[:m], status
+
+
+def csr_transpose(indptr: torch.Tensor, indices: torch.Tensor, n_cols: int, stream=None):
+    """Enqueues the CSC of a CSR; returns (csc_ptr int64, csc_row int32, csc_eid int64, status)."""
+    m, dev = indices.numel(), indptr.device
+    g = Csr(indptr.numel() - 1, m, indptr.data_ptr(), indices.data_ptr(), None)
+    csc_ptr = torch.empty(n_cols + 1, dtype=torch.int64, device=dev)
+    csc_row = torch.empty(max(m, 1), dtype=torch.int32, device=dev)
+    csc_eid = torch.empty(max(m, 1), dtype=torch.int64, device=dev)
+    status = torch.zeros(1, dtype=torch.int32, device=dev)
+    n = C.c_size_t(0)
+    _check(lib().e2egrec_csr_transpose(C.byref(g), n_cols, None, None, None, None, None, C.byref(n), None),
+           "e2egrec_csr_transpose(size query)")
+    ws = _dev_bytes(n.value, dev)
+    n = C.c_size_t(ws.numel())
+    _check(lib().e2egrec_csr_transpose(C.byref(g), n_cols, _ptr(csc_ptr), _ptr(csc_row), _ptr(csc_eid), _ptr(status),
+                                       _ptr(ws), C.byref(n), _stream(stream)), "e2egrec_csr_transpose")
+    return csc_ptr, csc_row[:m], csc_eid[:m], status

@@ -9,6 +9,7 @@
 #include "common.cuh"
 #include "scan.cuh"
 #include "internal.cuh"
+#include "radix.cuh"
 
 #include <algorithm>
 
@@ -32,79 +33,8 @@ __device__ inline uint4 philox4x32_10(uint4 c, uint2 k)
 }
 
 // ---------------------------------------------------------------------------------------
-// Single-pass prefix sums across thread blocks ("chained scan"): every tile publishes its own sum,
-// then looks back over the tiles before it until it meets one whose full prefix is known.  Tiles
-// are handed out by an atomic ticket, so a tile only ever waits for tiles that already run.  Every
-// wait is bounded; when the bound is hit the status word gets E2EGREC_DEV_TIMEOUT and the tile goes
-// on with what it has.
-// ---------------------------------------------------------------------------------------
-constexpr unsigned long long kChainAgg = 1ull << 62, kChainPrefix = 2ull << 62, kChainMask = (1ull << 62) - 1;
-constexpr int kChainSpinLimit = 1 << 22;
-
-__device__ inline unsigned long long chain_read(const unsigned long long *slot)
-{
-    return *reinterpret_cast<const volatile unsigned long long *>(slot);
-}
-
-// Called by all threads of the block.  Returns the sum of the aggregates of tiles 0 .. tile-1.
-__device__ inline long long chain_lookback(unsigned long long *state, int tile, long long aggregate, int32_t *status,
-                                           long long *bcast)
-{
-    if (threadIdx.x < 32) {
-        const int lane = threadIdx.x;
-        long long excl = 0;
-        if (lane == 0) atomicExch(&state[tile], (tile == 0 ? kChainPrefix : kChainAgg) | (unsigned long long)aggregate);
-        if (tile > 0) {
-            int p = tile - 1;
-            bool done = false;
-            while (!done) {
-                const int idx = p - lane;
-                unsigned long long v = kChainPrefix;                 // before tile 0: an empty prefix
-                bool timed_out = false;
-                for (int spin = 0;; ++spin) {
-                    if (idx >= 0) v = chain_read(&state[idx]);
-                    if (__all_sync(0xffffffffu, (v >> 62) != 0)) break;
-                    if (spin >= kChainSpinLimit) { timed_out = true; break; }
-                }
-                timed_out = __any_sync(0xffffffffu, timed_out);
-                const unsigned pref = __ballot_sync(0xffffffffu, (v >> 62) == 2);
-                const int first = pref ? __ffs(pref) - 1 : 31;
-                long long c = lane <= first ? (long long)(v & kChainMask) : 0;
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xffffffffu, c, o);
-                excl += c;
-                if (timed_out) {
-                    if (lane == 0) atomicOr(reinterpret_cast<unsigned *>(status), E2EGREC_DEV_TIMEOUT);
-                    done = true;
-                } else if (pref) {
-                    done = true;
-                } else {
-                    p -= 32;
-                }
-            }
-            if (lane == 0) atomicExch(&state[tile], kChainPrefix | (unsigned long long)(excl + aggregate));
-        }
-        if (lane == 0) *bcast = excl;
-    }
-    __syncthreads();
-    return *bcast;
-}
-
-__device__ inline int chain_ticket(unsigned *ticket, int *bcast)
-{
-    if (threadIdx.x == 0) *bcast = (int)atomicAdd(ticket, 1u);
-    __syncthreads();
-    return *bcast;
-}
-
-// ---------------------------------------------------------------------------------------
 // Scratch layout (host and device agree through this struct).
 // ---------------------------------------------------------------------------------------
-constexpr int kSortThreads = 256;
-constexpr int kSortItems = 16;
-constexpr int kSortTile = kSortThreads * kSortItems;
-constexpr int kMaxRadix = 1024;
-constexpr int kMaxPasses = 4;
 constexpr int kDstTile = 256;          // destinations per block of the sampling kernel
 constexpr int kWordTile = 2048;        // bitmap words per block of the frontier kernel
 
@@ -393,147 +323,6 @@ __global__ void frontier_release_kernel(const int32_t *__restrict__ src_nodes, c
     if (i < counts[CNT_SRC]) local_id[src_nodes[i]] = -1;
 }
 
-// ---------------------------------------------------------------------------------------
-// Stable LSD radix sort of (key = col, value = block position), one launch per digit.  A block owns
-// a tile of kSortTile consecutive elements, ranks equal digits in element order (per warp by
-// match_any, then across warps), and finds where its elements of each digit start from the digit's
-// global start (digit counts of the whole array, known beforehand) plus a per-digit chained scan
-// over the tiles before it.
-// ---------------------------------------------------------------------------------------
-template <int BITS>
-__global__ void __launch_bounds__(kSortThreads)
-sort_pass_kernel(const int32_t *__restrict__ keys_in, const int32_t *__restrict__ vals_in,
-                 int32_t *__restrict__ counts, int shift, const unsigned *__restrict__ ghist, int n_tiles,
-                 unsigned long long *__restrict__ state, unsigned *ticket, int32_t *__restrict__ keys_out,
-                 int32_t *__restrict__ vals_out)
-{
-    constexpr int R = 1 << BITS;
-    constexpr int W = kSortThreads / 32;
-    __shared__ int32_t wc[W][R];                 // per-warp digit counts, then start offsets
-    __shared__ int32_t bin_base[R];
-    __shared__ int32_t scan_sm[kSortThreads / 32 + 1];
-    __shared__ int tile_s;
-    const int tile = chain_ticket(ticket, &tile_s);
-    const int32_t n = counts[CNT_EDGES];
-    if ((int64_t)tile * kSortTile >= n) return;
-    for (int d = threadIdx.x; d < W * R; d += kSortThreads) (&wc[0][0])[d] = 0;
-    // start of every digit's bin: exclusive scan of the global digit counts
-    {
-        int32_t carry = 0;
-        for (int d0 = 0; d0 < R; d0 += kSortThreads) {
-            const int d = d0 + threadIdx.x;
-            const int32_t v = d < R ? (int32_t)ghist[d] : 0;
-            int32_t tot;
-            const int32_t ex = block_exclusive_scan<kSortThreads, int32_t>(v, tot, scan_sm);
-            if (d < R) bin_base[d] = carry + ex;
-            carry += tot;
-        }
-    }
-    __syncthreads();
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t wbase = (int64_t)tile * kSortTile + (int64_t)warp * (32 * kSortItems);
-    int32_t key[kSortItems], val[kSortItems], rank[kSortItems];
-#pragma unroll
-    for (int k = 0; k < kSortItems; ++k) {
-        const int64_t idx = wbase + k * 32 + lane;
-        const bool ok = idx < n;
-        key[k] = ok ? keys_in[idx] : 0;
-        val[k] = ok ? (vals_in ? vals_in[idx] : (int32_t)idx) : 0;
-        const uint32_t digit = ok ? (uint32_t)((key[k] >> shift) & (R - 1)) : 0xFFFFFFFFu;
-        const uint32_t peers = __match_any_sync(0xffffffffu, digit);
-        const int leader = __ffs(peers) - 1;
-        int32_t base = 0;
-        if (ok && lane == leader) {
-            base = wc[warp][digit];
-            wc[warp][digit] = base + __popc(peers);
-        }
-        base = __shfl_sync(0xffffffffu, base, leader);
-        rank[k] = base + __popc(peers & ((1u << lane) - 1u));
-        __syncwarp();
-    }
-    __syncthreads();
-    // per digit: publish this tile's count, then a chained look-back over earlier tiles, then warp start offsets
-    constexpr int DPT = (R + kSortThreads - 1) / kSortThreads;
-    int32_t cnt[DPT];
-#pragma unroll
-    for (int q = 0; q < DPT; ++q) {
-        const int d = threadIdx.x + q * kSortThreads;
-        cnt[q] = 0;
-        if (d < R) {
-#pragma unroll
-            for (int w = 0; w < W; ++w) cnt[q] += wc[w][d];
-            atomicExch(&state[(size_t)d * n_tiles + tile], (tile == 0 ? kChainPrefix : kChainAgg) | (unsigned long long)cnt[q]);
-        }
-    }
-    // look-back for all of this thread's digits together: a batch of earlier tiles per digit is read at
-    // once, then taken in order; an entry that is not published yet is polled (bounded) before going on
-    long long excl[DPT];
-    int next_p[DPT];
-    bool timed_out = false;
-#pragma unroll
-    for (int q = 0; q < DPT; ++q) {
-        excl[q] = 0;
-        next_p[q] = (threadIdx.x + q * kSortThreads < R && tile > 0) ? tile - 1 : -1;
-    }
-    for (;;) {
-        bool any = false;
-#pragma unroll
-        for (int q = 0; q < DPT; ++q) any = any || next_p[q] >= 0;
-        if (!any || timed_out) break;
-        constexpr int kBatch = 8;
-        unsigned long long v[DPT][kBatch];
-#pragma unroll
-        for (int q = 0; q < DPT; ++q) {
-            const unsigned long long *st = state + (size_t)(threadIdx.x + q * kSortThreads) * n_tiles;
-#pragma unroll
-            for (int j = 0; j < kBatch; ++j) v[q][j] = next_p[q] - j >= 0 ? chain_read(&st[next_p[q] - j]) : kChainPrefix;
-        }
-#pragma unroll
-        for (int q = 0; q < DPT; ++q) {
-            if (next_p[q] < 0) continue;
-            const unsigned long long *st = state + (size_t)(threadIdx.x + q * kSortThreads) * n_tiles;
-            bool found = false;
-#pragma unroll
-            for (int j = 0; j < kBatch; ++j) {
-                if (found || timed_out) continue;
-                unsigned long long x = v[q][j];
-                for (int spin = 0; (x >> 62) == 0; ++spin) {
-                    if (spin >= kChainSpinLimit) { timed_out = true; break; }
-                    x = chain_read(&st[next_p[q] - j]);
-                }
-                if (timed_out) continue;
-                excl[q] += (long long)(x & kChainMask);
-                if ((x >> 62) == 2) found = true;
-            }
-            next_p[q] = found ? -1 : next_p[q] - kBatch;
-        }
-    }
-    if (timed_out) atomicOr(reinterpret_cast<unsigned *>(&counts[CNT_STATUS]), E2EGREC_DEV_TIMEOUT);
-#pragma unroll
-    for (int q = 0; q < DPT; ++q) {
-        const int d = threadIdx.x + q * kSortThreads;
-        if (d >= R) continue;
-        if (tile > 0) atomicExch(&state[(size_t)d * n_tiles + tile], kChainPrefix | (unsigned long long)(excl[q] + cnt[q]));
-        int32_t run = bin_base[d] + (int32_t)excl[q];
-#pragma unroll
-        for (int w = 0; w < W; ++w) {
-            const int32_t c2 = wc[w][d];
-            wc[w][d] = run;
-            run += c2;
-        }
-    }
-    __syncthreads();
-#pragma unroll
-    for (int k = 0; k < kSortItems; ++k) {
-        const int64_t idx = wbase + k * 32 + lane;
-        if (idx < n) {
-            const int32_t pos = wc[warp][(key[k] >> shift) & (R - 1)] + rank[k];
-            keys_out[pos] = key[k];
-            vals_out[pos] = val[k];
-        }
-    }
-}
-
 // csc_ptr[s] = first position whose column is >= s (the columns are sorted), and the destination of
 // every transposed entry.
 __global__ void csc_finalize_kernel(const int32_t *__restrict__ csc_col, const int32_t *__restrict__ csc_eid,
@@ -597,43 +386,17 @@ pair_local_kernel(const int32_t *__restrict__ user, const int32_t *__restrict__ 
         if (h[d]) atomicAdd(&ghist[(d / R) * kMaxRadix + (d % R)], h[d]);
 }
 
-struct SortPlan { int bits, passes; };
-
-static SortPlan sort_plan(int32_t cap_src)
-{
-    int key_bits = 1;
-    while (key_bits < 31 && (1ll << key_bits) < (int64_t)cap_src) ++key_bits;
-    if (key_bits <= 8) return {8, 1};
-    if (key_bits <= 10) return {10, 1};
-    if (key_bits <= 16) return {8, 2};
-    if (key_bits <= 20) return {10, 2};
-    if (key_bits <= 24) return {8, 3};
-    if (key_bits <= 30) return {10, 3};
-    return {8, 4};
-}
-
-// csc_col / csc_eid = columns and positions of the block entries ordered by (col, position).
 static void sort_by_col(const int32_t *col, int32_t *counts, int32_t cap_edges, int32_t *csc_col, int32_t *csc_eid,
                         const SortPlan &sp, SamplerScratch &s, cudaStream_t st)
 {
-    const int n_tiles = (int)ceil_div(cap_edges > 0 ? cap_edges : 1, kSortTile);
-    const int32_t *kin = col;
-    const int32_t *vin = nullptr;                 // first pass: value = own position
-    for (int p = 0; p < sp.passes; ++p) {
-        const bool last = p == sp.passes - 1;
-        int32_t *kout = last ? csc_col : s.keys[p & 1];
-        int32_t *vout = last ? csc_eid : s.vals[p & 1];
-        unsigned long long *state = s.state_sort + (size_t)p * kMaxRadix * (size_t)s.sort_tiles;
-        note_launch();
-        if (sp.bits == 8)
-            sort_pass_kernel<8><<<n_tiles, kSortThreads, 0, st>>>(kin, vin, counts, p * sp.bits, s.ghist + p * kMaxRadix,
-                                                                 n_tiles, state, s.tickets + 2 + p, kout, vout);
-        else
-            sort_pass_kernel<10><<<n_tiles, kSortThreads, 0, st>>>(kin, vin, counts, p * sp.bits, s.ghist + p * kMaxRadix,
-                                                                  n_tiles, state, s.tickets + 2 + p, kout, vout);
-        kin = kout;
-        vin = vout;
-    }
+    RadixScratch rs{};
+    rs.keys[0] = s.keys[0]; rs.keys[1] = s.keys[1];
+    rs.vals[0] = s.vals[0]; rs.vals[1] = s.vals[1];
+    rs.tickets = s.tickets + 2;
+    rs.ghist = s.ghist;
+    rs.state = s.state_sort;
+    rs.tiles = s.sort_tiles;
+    radix_sort_pairs(col, nullptr, counts, cap_edges, csc_col, csc_eid, sp, rs, st);
 }
 
 static inline unsigned grid_for(int64_t n, int threads) { return (unsigned)ceil_div(n > 0 ? n : 1, threads); }

@@ -184,3 +184,31 @@ def test_full_graph_aggregation_forward_and_transpose(dtype, d):
     want = oracle.full_aggregate_backward(indptr, indices, n, G, bf16)
     rss_b = np.sqrt(oracle.full_aggregate_backward(indptr, indices, n, G.astype(np.float64) ** 2 / np.maximum(deg, 1)))
     assert_close("aggregate_backward", dX.float().cpu().numpy()[:n], want, bf16, rss_b)
+
+
+# ----------------------------------------------------------------------------- graph ingest
+
+@pytest.mark.parametrize("n,m", [(5_000, 80_000), (70_001, 300_007), (3, 0)])
+def test_graph_ingest_is_bit_exact(n, m):
+    """CSR from an edge list and its transpose: several sort tiles, a ragged tail, parallel edges, empty input."""
+    import paper_2511_20564_b200 as E
+    rng = np.random.default_rng(n)
+    row = S.zipf_ranks(rng, m, n, 1.1).astype(np.int32)
+    col = rng.integers(0, n, m).astype(np.int32)
+    indptr, indices, status = E.graph_from_coo(n, torch.from_numpy(row).cuda(), torch.from_numpy(col).cuda())
+    want_ptr, want_idx = oracle.csr_from_coo(n, row, col)
+    assert int(status) == 0
+    assert np.array_equal(indptr.cpu().numpy(), want_ptr) and np.array_equal(indices.cpu().numpy(), want_idx)
+    cptr, crow, ceid, status = E.csr_transpose(indptr, indices.contiguous(), n)
+    w_ptr, w_row, w_eid = oracle.csr_transpose(n, n, want_ptr, want_idx)
+    assert int(status) == 0
+    assert np.array_equal(cptr.cpu().numpy(), w_ptr) and np.array_equal(crow.cpu().numpy(), w_row)
+    assert np.array_equal(ceid.cpu().numpy(), w_eid)
+
+
+def test_graph_ingest_flags_ids_out_of_range():
+    import paper_2511_20564_b200 as E
+    row = torch.tensor([0, 1, 7], dtype=torch.int32, device="cuda")
+    col = torch.tensor([1, -2, 0], dtype=torch.int32, device="cuda")
+    _, _, status = E.graph_from_coo(4, row, col)
+    assert int(status) & 1
