@@ -28,7 +28,7 @@ CLOCK_QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reason
                "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
                "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 TAP_NAMES = {1: "sage_aggregate_kernel (layer-0 mean aggregation, gathers X rows)",
-             2: "seg_chunk_kernel+seg_finish_kernel (layer-0 transposed aggregation -> dX rows)",
+             2: "seg_run_kernel+seg_window_kernel+seg_final_kernel (layer-0 transposed aggregation -> dX rows)",
              3: "layer-0 dense transform W[h|agg]",
              4: "layer-0 weight gradient dZ^T[h|agg]",
              5: "layer-0 input gradient dZ W",
@@ -393,7 +393,10 @@ def run_ours(args, w):
         peak = peaks["bf16_tflops"] if w.dtype == "bf16" else peaks["bf16_tflops"] / 2.25 * 0.08
         roof = dict(bound="tensor" if w.dtype == "bf16" else "alu", achieved=alg / dom_mean_ms / 1e9, peak=peak,
                     unit="TFLOP/s")
-    roof.update(frac=roof["achieved"] / roof["peak"], traffic=None, kernel=TAP_NAMES[dominant],
+    # DRAM bytes per launch from the ncu launch list of this command (profiles/medium_step_launch_list.md);
+    # known only for the aggregation kernels of the outermost block of the `medium` workload
+    traffic = {1: 6.30e6, 2: 5.54e6 + 2.18e6 + 1.70e6}.get(dominant) if w.name == "medium" and args.seeds == "activity" else None
+    roof.update(frac=roof["achieved"] / roof["peak"], traffic=traffic, kernel=TAP_NAMES[dominant],
                 ms_per_launch=dom_mean_ms, algorithmic_units_per_launch=alg, peak_source=peaks["source"])
 
     line = dict(metric=METRIC, value=edges_all / (ms / 1e3), unit=UNIT, n_gpus=world, steps=K, warmup=Wm,
