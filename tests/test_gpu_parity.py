@@ -212,3 +212,16 @@ def test_graph_ingest_flags_ids_out_of_range():
     col = torch.tensor([1, -2, 0], dtype=torch.int32, device="cuda")
     _, _, status = E.graph_from_coo(4, row, col)
     assert int(status) & 1
+
+
+def test_three_hops_wide_rows_bf16():
+    """The shape of the large workload (3 hops, fanout [20,10,5], d = hidden = 256 bf16) on a small graph."""
+    base = S.WORKLOADS["medium_small"]
+    w = S.Workload("large_shape", base.n_users, base.n_items, base.n_interactions, 1.05, 1.05, 3, 256, 256, "bf16",
+                   (20, 10, 5), 128)
+    case = Case(w, step=0)
+    dH = case.upstream_grad(case.seeds.size, w.hidden)
+    ora = case.run_oracle(dH)
+    gpu = case.run_gpu(dH)
+    assert_blocks_equal(gpu["blocks"], ora["blocks"])
+    _check_float(case, gpu, ora)
