@@ -267,6 +267,24 @@ int32_t e2egrec_aggregate_backward(int64_t n_src, int64_t n_entries, const int64
                                    const int32_t *csc_row, const float *inv_deg, const e2egrec_mat *G,
                                    const e2egrec_mat *dX, void *ws, size_t *ws_bytes, void *stream);
 
+/* LightGCN propagation over the whole graph (Sec. 3.1, Eqs. 4-7): H^(l+1) = A_hat H^(l) with
+ * A_hat[u][i] = (number of stored entries (u, i)) * s[u] * s[i], s = inv_sqrt_deg (1/sqrt(|N(u)|), 0 for an
+ * isolated node; device float[n_nodes], supplied by the caller), and Y = (1/(L+1)) sum_{l=0..L} H^(l).
+ * H0 and Y are [n_nodes x dim] dense (ld = dim) matrices of one dtype; every H^(l) is stored in that dtype,
+ * Y is rounded once from the fp32 sum of the layers.  e2egrec_lightgcn_backward is the adjoint,
+ * dH0 = (1/(L+1)) sum_l (A_hat^T)^l dY, and takes the CSC arrays of the same graph (for a graph stored in
+ * both directions they equal the CSR arrays).  The products run on the segment-reduction kernels of the
+ * mean aggregation with a per-entry and a per-row weight.  ws: scratch (size query with ws == NULL);
+ * 0 <= n_layers <= 8. */
+int32_t e2egrec_lightgcn_forward(int64_t n_nodes, int64_t n_entries, const int64_t *indptr,
+                                 const int32_t *indices, const float *inv_sqrt_deg, int32_t n_layers,
+                                 const e2egrec_mat *H0, const e2egrec_mat *Y, void *ws, size_t *ws_bytes,
+                                 void *stream);
+int32_t e2egrec_lightgcn_backward(int64_t n_nodes, int64_t n_entries, const int64_t *csc_ptr,
+                                  const int32_t *csc_row, const float *inv_sqrt_deg, int32_t n_layers,
+                                  const e2egrec_mat *dY, const e2egrec_mat *dH0, void *ws, size_t *ws_bytes,
+                                  void *stream);
+
 /* e2egrec_aggregate_forward without a workspace argument (the paper has no counterpart; this is a
  * packaging variant of the call above and computes exactly the same result).
  *

@@ -304,3 +304,27 @@ def joint_step(indptr, indices, X, pair_user, pair_item, dense, labels, fanouts,
     dW_gnn, _, dX = sage_backward(blocks, ctx, W_gnn, dH, bf16=bf16)
     return dict(seeds=seeds, blocks=blocks, loss=loss, logits=t[:, 0], dW_tower=[dW1, dW2, dW3],
                 db_tower=[db1, db2, db3], dW_gnn=dW_gnn, dX=dX, dX_ids=blocks[-1]["src_nodes"], H=H, dH=dH)
+
+
+# ----------------------------------------------------------------------------- LightGCN
+
+def lightgcn_propagate(indptr, indices, H, bf16=False):
+    """Eqs. 4-6: one application of the symmetrically normalised adjacency (degrees = row lengths)."""
+    indptr, indices, H = _i64(indptr), _i32(indices), _f64(H)
+    n, d = indptr.size - 1, H.shape[1]
+    out = np.zeros((n, d), np.float64)
+    lib().oracle_lightgcn_propagate(_p(indptr), _p(indices), C.c_int64(n), _p(H), C.c_int32(d), _p(out),
+                                    C.c_int(int(bf16)))
+    return out
+
+
+def lightgcn_forward(indptr, indices, H0, n_layers, bf16=False):
+    """Eq. 7: Y = (1/(L+1)) sum_l H^(l), H^(l+1) = A_hat H^(l).  On a symmetric graph the adjoint w.r.t. H0 is
+    the same map applied to dY."""
+    H = _f64(H0)
+    acc = H.copy()
+    for _ in range(n_layers):
+        H = lightgcn_propagate(indptr, indices, H, bf16)
+        acc += H
+    Y = acc / (n_layers + 1)
+    return round_bf16(Y) if bf16 else Y

@@ -408,3 +408,27 @@ void oracle_full_aggregate_backward(const int64_t *indptr, const int32_t *indice
     }
     if (round_bf16) oracle_round_bf16_array(dX, n_src * d);
 }
+
+/* ------------------------------------------------------------------------- */
+/* LightGCN (Sec. 3.1, Eqs. 4-7)                                              */
+/* ------------------------------------------------------------------------- */
+
+/* One propagation: out_u = sum_{i in N(u)} h_i / (sqrt|N(u)| sqrt|N(i)|)  (Eqs. 4-5; H' = A_hat H, Eq. 6).
+ * N(.) are the rows of the (square) CSR; a node without neighbours gives and receives 0.
+ * With round_bf16 the result is stored as bf16. */
+void oracle_lightgcn_propagate(const int64_t *indptr, const int32_t *indices, int64_t n, const double *H, int32_t d,
+                               double *out, int round_bf16)
+{
+    for (int64_t u = 0; u < n; ++u) {
+        const int64_t du = indptr[u + 1] - indptr[u];
+        for (int32_t k = 0; k < d; ++k) {
+            double s = 0.0;
+            for (int64_t e = indptr[u]; e < indptr[u + 1]; ++e) {
+                const int64_t i = indices[e];
+                const int64_t di = indptr[i + 1] - indptr[i];
+                if (di > 0) s += H[i * d + k] / (sqrt((double)du) * sqrt((double)di));
+            }
+            out[u * d + k] = round_bf16 ? oracle_round_bf16(s) : s;
+        }
+    }
+}

@@ -102,6 +102,10 @@ def lib():
         L.e2egrec_csr_transpose.restype = C.c_int32
         L.e2egrec_csr_transpose.argtypes = [C.POINTER(Csr), C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                             C.c_void_p, C.POINTER(C.c_size_t), C.c_void_p]
+        for fn in (L.e2egrec_lightgcn_forward, L.e2egrec_lightgcn_backward):
+            fn.restype = C.c_int32
+            fn.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.POINTER(Mat),
+                           C.POINTER(Mat), C.c_void_p, C.POINTER(C.c_size_t), C.c_void_p]
         L.e2egrec_launch_count.restype = C.c_uint64
         L.e2egrec_profile_tap.restype = C.c_int32
         L.e2egrec_profile_tap.argtypes = [C.c_int32, C.c_void_p, C.c_void_p]
@@ -455,3 +459,32 @@ def csr_transpose(indptr: torch.Tensor, indices: torch.Tensor, n_cols: int, stre
     _check(lib().e2egrec_csr_transpose(C.byref(g), n_cols, _ptr(csc_ptr), _ptr(csc_row), _ptr(csc_eid), _ptr(status),
                                        _ptr(ws), C.byref(n), _stream(stream)), "e2egrec_csr_transpose")
     return csc_ptr, csc_row[:m], csc_eid[:m], status
+
+
+# ------------------------------------------------------------------------------------------ LightGCN
+
+def _lightgcn(fn, name, ptr, idx, inv_sqrt_deg, n_layers, Hin, out, ws, stream):
+    n, m = ptr.numel() - 1, idx.numel()
+    if out is None:
+        out = torch.empty_like(Hin)
+    a, b = _mat(Hin), _mat(out)
+    nbytes = C.c_size_t(0)
+    if ws is None:
+        _check(fn(n, m, None, None, None, n_layers, C.byref(a), C.byref(b), None, C.byref(nbytes), None), name + "(size query)")
+        ws = _dev_bytes(nbytes.value, Hin.device)
+    nbytes = C.c_size_t(ws.numel())
+    _check(fn(n, m, _ptr(ptr), _ptr(idx), _ptr(inv_sqrt_deg), n_layers, C.byref(a), C.byref(b), _ptr(ws), C.byref(nbytes),
+              _stream(stream)), name)
+    return out, ws
+
+
+def lightgcn_forward(indptr, indices, inv_sqrt_deg, n_layers, H0, Y=None, ws=None, stream=None):
+    """Enqueues Y = mean over layers of A_hat^l H0; returns (Y, ws)."""
+    return _lightgcn(lib().e2egrec_lightgcn_forward, "e2egrec_lightgcn_forward", indptr, indices, inv_sqrt_deg, n_layers,
+                     H0, Y, ws, stream)
+
+
+def lightgcn_backward(csc_ptr, csc_row, inv_sqrt_deg, n_layers, dY, dH0=None, ws=None, stream=None):
+    """Enqueues the adjoint of lightgcn_forward over the CSC arrays; returns (dH0, ws)."""
+    return _lightgcn(lib().e2egrec_lightgcn_backward, "e2egrec_lightgcn_backward", csc_ptr, csc_row, inv_sqrt_deg,
+                     n_layers, dY, dH0, ws, stream)

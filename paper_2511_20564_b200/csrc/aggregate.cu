@@ -102,3 +102,102 @@ extern "C" int32_t e2egrec_aggregate_backward(int64_t n_src, int64_t n_entries, 
 {
     return aggregate_entry(n_src, n_entries, csc_ptr, csc_row, inv_deg, G, dX, 0, ws, ws_bytes, stream);
 }
+
+// ------------------------------------------------------------------------------------------ LightGCN
+namespace e2egrec {
+
+struct LayerList { const void *p[9]; };
+
+// Y = (sum of n_in matrices) * scale, summed in fp32 and rounded once
+template <typename T>
+__global__ void layer_mean_kernel(LayerList list, int n_in, int64_t cells, float scale, T *__restrict__ out)
+{
+    const T *const *in = reinterpret_cast<const T *const *>(list.p);
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < cells; i += (int64_t)gridDim.x * blockDim.x) {
+        float s = 0.f;
+        for (int l = 0; l < n_in; ++l) s += to_float<T>(in[l][i]);
+        out[i] = from_float<T>(s * scale);
+    }
+}
+
+// out = A_hat in:  out[u] = s[u] * sum_{i in row u} s[i] * in[i]
+static int32_t lightgcn_propagate(int64_t n, int64_t m, const int64_t *ptr, const int32_t *idx, const float *s,
+                                  const e2egrec_mat *in, void *out_data, void *ws, cudaStream_t st)
+{
+    if (in->dtype == E2EGREC_BF16) {
+        using T = __nv_bfloat16;
+        SegOut<T> o{};
+        o.out = static_cast<T *>(out_data);
+        o.ld_out = in->dim;
+        o.seg_scale = s;
+        dispatch_seg64<T, true>(static_cast<const T *>(in->data), in->ld, ptr, idx, n, m, s, in->dim, ws, o, in->dtype, st);
+    } else {
+        using T = float;
+        SegOut<T> o{};
+        o.out = static_cast<T *>(out_data);
+        o.ld_out = in->dim;
+        o.seg_scale = s;
+        dispatch_seg64<T, true>(static_cast<const T *>(in->data), in->ld, ptr, idx, n, m, s, in->dim, ws, o, in->dtype, st);
+    }
+    return check_launch("lightgcn_propagate");
+}
+
+}  // namespace e2egrec
+
+// Shared body of e2egrec_lightgcn_forward / _backward: Y = (1/(L+1)) sum_{l=0..L} A^l H0 with A given by (ptr, idx, s).
+static int32_t lightgcn_entry(int64_t n, int64_t m, const int64_t *ptr, const int32_t *idx, const float *s, int32_t n_layers,
+                              const e2egrec_mat *H0, const e2egrec_mat *Y, void *ws, size_t *ws_bytes, void *stream)
+{
+    if (!ws_bytes) return E2EGREC_ERR_NULL;
+    if (n < 0 || m < 0 || n_layers < 0 || n_layers > 8) return E2EGREC_ERR_ARG;
+    if (n >= (1ll << 31)) return E2EGREC_ERR_UNSUPPORTED;
+    int32_t rc = check_mats(H0, Y, n);
+    if (rc != E2EGREC_OK) return rc;
+    if (H0->ld != H0->dim || Y->ld != Y->dim) return E2EGREC_ERR_ARG;
+    const size_t es = dtype_size(H0->dtype);
+    const size_t layer_bytes = align_up((size_t)(n > 0 ? n : 1) * H0->dim * es, 256);
+    const size_t seg_bytes = align_up(full_ws_bytes(m, H0->dim), 256);
+    const size_t need = seg_bytes + (size_t)n_layers * layer_bytes;
+    if (!ws) { *ws_bytes = need; return E2EGREC_OK; }
+    if (*ws_bytes < need) { *ws_bytes = need; return E2EGREC_ERR_WORKSPACE; }
+    if (reinterpret_cast<uintptr_t>(ws) % 256) return E2EGREC_ERR_ALIGN;
+    if (!ptr || !s || (m > 0 && !idx)) return E2EGREC_ERR_NULL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    char *base = static_cast<char *>(ws);
+    LayerList layers{};
+    layers.p[0] = H0->data;
+    e2egrec_mat cur = *H0;
+    for (int l = 0; l < n_layers; ++l) {
+        void *next = base + seg_bytes + (size_t)l * layer_bytes;
+        rc = lightgcn_propagate(n, m, ptr, idx, s, &cur, next, base, st);
+        if (rc != E2EGREC_OK) return rc;
+        layers.p[l + 1] = next;
+        cur.data = next;
+    }
+    const int64_t cells = n * H0->dim;
+    const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(cells > 0 ? cells : 1, 256), 148 * 16);
+    note_launch();
+    if (H0->dtype == E2EGREC_BF16)
+        layer_mean_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(layers, n_layers + 1, cells, 1.0f / (float)(n_layers + 1),
+                                                             static_cast<__nv_bfloat16 *>(Y->data));
+    else
+        layer_mean_kernel<float><<<grid, 256, 0, st>>>(layers, n_layers + 1, cells,
+                                                       1.0f / (float)(n_layers + 1), static_cast<float *>(Y->data));
+    return check_launch("lightgcn");
+}
+
+extern "C" int32_t e2egrec_lightgcn_forward(int64_t n_nodes, int64_t n_entries, const int64_t *indptr,
+                                            const int32_t *indices, const float *inv_sqrt_deg, int32_t n_layers,
+                                            const e2egrec_mat *H0, const e2egrec_mat *Y, void *ws, size_t *ws_bytes,
+                                            void *stream)
+{
+    return lightgcn_entry(n_nodes, n_entries, indptr, indices, inv_sqrt_deg, n_layers, H0, Y, ws, ws_bytes, stream);
+}
+
+extern "C" int32_t e2egrec_lightgcn_backward(int64_t n_nodes, int64_t n_entries, const int64_t *csc_ptr,
+                                             const int32_t *csc_row, const float *inv_sqrt_deg, int32_t n_layers,
+                                             const e2egrec_mat *dY, const e2egrec_mat *dH0, void *ws, size_t *ws_bytes,
+                                             void *stream)
+{
+    return lightgcn_entry(n_nodes, n_entries, csc_ptr, csc_row, inv_sqrt_deg, n_layers, dY, dH0, ws, ws_bytes, stream);
+}

@@ -124,13 +124,14 @@ struct SegOut {
     const T *mask;          // optional: result is zeroed where mask[s][k] <= 0 (ReLU derivative)
     int64_t ld_mask;
     int mean;               // divide the sum by the segment length
+    const float *seg_scale; // optional: multiply the sum of segment s by seg_scale[s] (not together with mean)
     int64_t pad_rows;       // if > 0: rows n_seg .. min(next multiple of 128, pad_rows) - 1 of out are zeroed
 };
 
 template <typename T>
 __device__ inline float seg_finish_value(const SegOut<T> &o, int64_t s, int64_t len, int k, float sum, bool has_self)
 {
-    float v = o.mean ? (len > 0 ? sum * (1.0f / (float)len) : 0.f) : sum;
+    float v = o.mean ? (len > 0 ? sum * (1.0f / (float)len) : 0.f) : (o.seg_scale ? sum * o.seg_scale[s] : sum);
     if (has_self) v += to_float<T>(o.self[s * o.ld_self + k]);
     v = to_float<T>(from_float<T>(v));                      // storage rounding before the mask
     if (o.mask && !(to_float<T>(o.mask[s * o.ld_mask + k]) > 0.f)) v = 0.f;

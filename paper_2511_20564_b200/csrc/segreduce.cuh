@@ -63,7 +63,7 @@ inline SegScratch seg_scratch_carve(int64_t cap_entries, int run_len, int d, voi
 template <typename T>
 __device__ inline float seg_round(const SegOut<T> &o, float inv_len, float sum)
 {
-    const float v = o.mean ? sum * inv_len : sum;
+    const float v = (o.mean || o.seg_scale) ? sum * inv_len : sum;
     return to_float<T>(from_float<T>(v));
 }
 
@@ -208,14 +208,14 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
     // closes the current segment, which ends at relative position end_rel, with the sum in acc
     auto emit = [&](bool ended, int end_rel) {
         if (cur_begins && ended) {
-            const float inv = o.mean ? 1.0f / (float)(end_rel - cur_beg_rel) : 1.0f;
+            const float inv = o.mean ? 1.0f / (float)(end_rel - cur_beg_rel) : (o.seg_scale ? o.seg_scale[cur_seg] : 1.0f);
 #pragma unroll
             for (int q = 0; q < CPL; ++q) {
                 const int ch = c + q * LPR;
                 if (ch < n_chunks) {
                     float r[E];
 #pragma unroll
-                    for (int e = 0; e < E; ++e) r[e] = to_float<T>(from_float<T>(acc[q][e] * inv));
+                    for (int e = 0; e < E; ++e) r[e] = to_float<T>(from_float<T>(acc[q][e] * inv));   // inv = 1 without mean / scale
                     if (kExtra && o.mask) {
                         float m[E];
                         Chunk<T>::unpack(cur_mask[q], m);
@@ -354,6 +354,7 @@ seg_window_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_
                                     const int64_t s = cur;
                                     float inv = 0.f;
                                     if (o.mean) inv = 1.0f / (float)((int64_t)ptr[s + 1] - (int64_t)ptr[s]);
+                                    else if (o.seg_scale) inv = o.seg_scale[s];
                                     const float m[4] = {mk[j].x, mk[j].y, mk[j].z, mk[j].w};
                                     float r[4] = {acc.x, acc.y, acc.z, acc.w};
 #pragma unroll

@@ -225,3 +225,34 @@ def test_three_hops_wide_rows_bf16():
     gpu = case.run_gpu(dH)
     assert_blocks_equal(gpu["blocks"], ora["blocks"])
     _check_float(case, gpu, ora)
+
+
+# ----------------------------------------------------------------------------- LightGCN
+
+@pytest.mark.parametrize("dtype,d", [("bf16", 64), ("f32", 32)])
+def test_lightgcn_forward_and_adjoint(dtype, d):
+    """Three propagation layers and the layer mean on a symmetric power-law graph with hubs and isolated nodes."""
+    import paper_2511_20564_b200 as E
+    n, m, L = 20_011, 300_000, 3
+    a, b = S.powerlaw_directed(n, m, 1.1, 7)
+    indptr, indices = S.coo_to_csr(n, np.concatenate([a, b]), np.concatenate([b, a]))
+    deg = np.diff(indptr)
+    assert deg.max() > 10_000 and (deg == 0).any()
+    bf16 = dtype == "bf16"
+    dt = torch.bfloat16 if bf16 else torch.float32
+    H0 = S.normal_features(n, d, 8)
+    G = S.normal_features(n, d, 8, stream=12)
+    if bf16:
+        H0, G = S.to_bf16_values(H0), S.to_bf16_values(G)
+    s = np.where(deg > 0, 1.0 / np.sqrt(np.maximum(deg, 1)), 0.0).astype(np.float32)
+    ip, ix, sd = torch.from_numpy(indptr).cuda(), torch.from_numpy(indices).cuda(), torch.from_numpy(s).cuda()
+    Y, ws = E.lightgcn_forward(ip, ix, sd, L, torch.from_numpy(H0).cuda().to(dt))
+    want = oracle.lightgcn_forward(indptr, indices, H0, L, bf16)
+    # scale of the terms of one output: s_u * sqrt(sum_i s_i^2 h_i^2) per layer, bounded by the row norm of |H|
+    rss = np.sqrt(oracle.lightgcn_propagate(indptr, indices, H0.astype(np.float64) ** 2)) if bf16 else None
+    assert_close("lightgcn_forward", Y.float().cpu().numpy(), want, bf16, rss)
+    # the graph is stored in both directions, so its CSC arrays are its CSR arrays
+    dH0, _ = E.lightgcn_backward(ip, ix, sd, L, torch.from_numpy(G).cuda().to(dt), ws=ws)
+    want = oracle.lightgcn_forward(indptr, indices, G, L, bf16)
+    rss = np.sqrt(oracle.lightgcn_propagate(indptr, indices, G.astype(np.float64) ** 2)) if bf16 else None
+    assert_close("lightgcn_backward", dH0.float().cpu().numpy(), want, bf16, rss)

@@ -215,3 +215,28 @@ def test_dense_layer_forward_backward():
     dW, db, dX = oracle.dense_backward(R, Y, X, W, act=1)
     dZ = R * (Y > 0)
     assert np.allclose(dW, dZ.T @ X) and np.allclose(db, dZ.sum(0)) and np.allclose(dX, dZ @ W)
+
+
+# ----------------------------------------------------------------------------- LightGCN
+
+def test_lightgcn_matches_dense_normalised_adjacency_and_is_self_adjoint():
+    rng = np.random.default_rng(12)
+    n, d, L = 40, 3, 3
+    row = rng.integers(0, n - 2, 150).astype(np.int32)         # the last two nodes stay isolated
+    col = rng.integers(0, n - 2, 150).astype(np.int32)
+    indptr, indices = oracle.csr_from_coo(n, np.concatenate([row, col]), np.concatenate([col, row]))   # symmetric
+    A = np.zeros((n, n))
+    for u in range(n):
+        for e in range(indptr[u], indptr[u + 1]):
+            A[u, indices[e]] += 1
+    deg = np.diff(indptr).astype(np.float64)
+    s = np.where(deg > 0, 1 / np.sqrt(np.maximum(deg, 1)), 0.0)
+    Ahat = s[:, None] * A * s[None, :]                             # D^-1/2 A D^-1/2
+    H0, G = rng.standard_normal((n, d)), rng.standard_normal((n, d))
+    assert np.allclose(oracle.lightgcn_propagate(indptr, indices, H0), Ahat @ H0, atol=1e-13)
+    want = sum(np.linalg.matrix_power(Ahat, l) @ H0 for l in range(L + 1)) / (L + 1)
+    Y = oracle.lightgcn_forward(indptr, indices, H0, L)
+    assert np.allclose(Y, want, atol=1e-13)
+    assert np.all(Y[-2:] == H0[-2:] / (L + 1))                     # isolated nodes keep only their own layer-0 term
+    # symmetric graph: <Y(H0), G> = <H0, Y(G)>
+    assert np.isclose((Y * G).sum(), (H0 * oracle.lightgcn_forward(indptr, indices, G, L)).sum(), rtol=1e-12)
