@@ -104,14 +104,22 @@ struct EpiPartial {
     __device__ void operator()(int64_t m, int n, float v, int z) const { out[z * split_stride + m * ldo + n] = v; }
 };
 
-// out = (accumulate ? out : 0) + sum_z partial[z], z ascending
+// out = (accumulate ? out : 0) + sum_z partial[z], z ascending.  With rows_dev the partials come from the
+// tensor-core weight-gradient kernel, which only fills the first ceil(total / per) splits
+// (total = ceil(rows / 64) k-blocks, per = max(8, ceil(total / splits))); without it all splits are added.
 static __global__ void splitk_reduce_kernel(const float *__restrict__ partial, int64_t n, int splits, int accumulate,
-                                     float *__restrict__ out)
+                                            float *__restrict__ out, const int32_t *rows_dev)
 {
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
+    int active = splits;
+    if (rows_dev) {
+        const int64_t total = ((int64_t)*rows_dev + 63) / 64;
+        const int64_t per = max((int64_t)8, (total + splits - 1) / splits);
+        active = (int)max((int64_t)1, (total + per - 1) / per);
+    }
     float s = accumulate ? out[i] : 0.f;
-    for (int z = 0; z < splits; ++z) s += partial[(int64_t)z * n + i];
+    for (int z = 0; z < active; ++z) s += partial[(int64_t)z * n + i];
     out[i] = s;
 }
 

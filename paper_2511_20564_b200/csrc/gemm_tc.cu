@@ -22,6 +22,7 @@ constexpr int kTileK = 64;                 // 64 bf16 = one 128-byte swizzle row
 constexpr int kUmmaK = 16;
 constexpr int kThreads = 128;
 constexpr int kMaxStages = 4;
+constexpr int kMinSplitBlocks = 8;          // k-blocks of 64 rows per split of the weight-gradient product
 constexpr uint32_t kSpinLimit = 4u * 1000u * 1000u;
 
 // ------------------------------------------------------------------------- PTX wrappers
@@ -381,7 +382,11 @@ tc_gemm_rows_kernel(const __grid_constant__ CUtensorMap map_y, const __grid_cons
     const int m0 = blockIdx.x * kTileM, n0 = blockIdx.y * nt;
     const int64_t m_valid = *m_dev;
     const int64_t total_blocks = (m_valid + kTileK - 1) / kTileK;
-    const int64_t per = (total_blocks + gridDim.z - 1) / gridDim.z;
+    // at least kMinSplitBlocks k-blocks per split: only the first ceil(total / per) splits do work and
+    // write a partial (split 0 writes zeros when there are no rows); splitk_reduce_kernel uses the same rule
+    const int64_t per = max((int64_t)kMinSplitBlocks, (total_blocks + gridDim.z - 1) / gridDim.z);
+    const int64_t active = max((int64_t)1, (total_blocks + per - 1) / per);
+    if ((int64_t)blockIdx.z >= active) return;
     const int64_t kb0 = (int64_t)blockIdx.z * per;
     const int64_t kb1 = kb0 + per < total_blocks ? kb0 + per : total_blocks;
     const int k_blocks = kb1 > kb0 ? (int)(kb1 - kb0) : 0;

@@ -196,8 +196,10 @@ template <typename T>
 void linear_backward_weight(const T *dY, int64_t rows, int n_out, const T *Xin, int n_in, const int32_t *m_dev,
                             float *part, float *dW, float *db, int32_t *status, cudaStream_t st)
 {
-    if (!(use_tc<T>() && tc_weight_grad(reinterpret_cast<const __nv_bfloat16 *>(dY), rows, n_out,
-                                        reinterpret_cast<const __nv_bfloat16 *>(Xin), n_in, m_dev, part, kSplits, status, st))) {
+    const bool on_tc = use_tc<T>() && tc_weight_grad(reinterpret_cast<const __nv_bfloat16 *>(dY), rows, n_out,
+                                                     reinterpret_cast<const __nv_bfloat16 *>(Xin), n_in, m_dev, part, kSplits,
+                                                     status, st);
+    if (!on_tc) {
         EpiPartial epi{part, n_in, (int64_t)n_out * n_in};
         dim3 grid((unsigned)ceil_div(n_out, kGemmBM), (unsigned)ceil_div(n_in, kGemmBN), kSplits);
         note_launch();
@@ -206,7 +208,7 @@ void linear_backward_weight(const T *dY, int64_t rows, int n_out, const T *Xin, 
     }
     const int64_t n = (int64_t)n_out * n_in;
     note_launch();
-    splitk_reduce_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(part, n, kSplits, 0, dW);
+    splitk_reduce_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(part, n, kSplits, 0, dW, on_tc ? m_dev : nullptr);
     if (db) {
         note_launch();
         colsum_kernel<T><<<(unsigned)ceil_div(n_out, 32), 256, 0, st>>>(dY, n_out, m_dev, n_out, 0, db);

@@ -200,7 +200,8 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
         {
             const int64_t n = (int64_t)p.d_out * two_d;
             note_launch();
-            splitk_reduce_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(part, n, kDwSplits, accumulate, dW[l]);
+            splitk_reduce_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(part, n, kDwSplits, accumulate, dW[l],
+                                                                             dw_done ? n_dst : nullptr);
         }
         if (l == 0) tap_end(TAP_DW_OUTER, st);
         if (dbias && dbias[l]) {
