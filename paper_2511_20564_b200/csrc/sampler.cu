@@ -35,7 +35,8 @@ __device__ inline uint4 philox4x32_10(uint4 c, uint2 k)
 // ---------------------------------------------------------------------------------------
 // Scratch layout (host and device agree through this struct).
 // ---------------------------------------------------------------------------------------
-constexpr int kDstTile = 256;          // destinations per block of the sampling kernel
+constexpr int kDstTile = 64;           // destinations per block of the sampling kernel
+constexpr int kDstThreads = 256;       // its threads: one per destination for the counts, then all of them draw
 constexpr int kWordTile = 2048;        // bitmap words per block of the frontier kernel
 
 struct SamplerScratch {
@@ -117,7 +118,7 @@ __global__ void seed_init_kernel(const int32_t *__restrict__ seeds, int32_t n_se
 // key (seed lo, seed hi); words 2(j%2), 2(j%2)+1 form r and the picked row position is
 // floor(r * deg / 2^64).  deg <= fanout copies the row instead.  Sampled nodes that are not yet in
 // the frontier are marked in the bitmap.
-__global__ void __launch_bounds__(kDstTile)
+__global__ void __launch_bounds__(kDstThreads)
 hop_sample_kernel(const int64_t *__restrict__ g_indptr, const int32_t *__restrict__ g_indices, int64_t n_nodes,
                   const int32_t *__restrict__ dst_nodes, const int32_t *n_dst_ptr, int32_t cap_dst, int32_t cap_edges,
                   int32_t fanout, int32_t hop, uint32_t seed_lo, uint32_t seed_hi, uint32_t step_arg,
@@ -131,7 +132,7 @@ hop_sample_kernel(const int64_t *__restrict__ g_indptr, const int32_t *__restric
     __shared__ int32_t node[kDstTile];
     __shared__ int64_t gbeg_s[kDstTile];
     __shared__ int64_t deg_s[kDstTile];
-    __shared__ int32_t scan_sm[kDstTile / 32 + 1];
+    __shared__ int32_t scan_sm[kDstThreads / 32 + 1];
     __shared__ long long bcast;
     __shared__ int tile_s;
     const int tile = chain_ticket(ticket, &tile_s);
@@ -150,7 +151,7 @@ hop_sample_kernel(const int64_t *__restrict__ g_indptr, const int32_t *__restric
     }
     const int64_t i = i0 + threadIdx.x;
     int32_t c = 0;
-    if (i < n_dst) {
+    if (threadIdx.x < kDstTile && i < n_dst) {
         int32_t u = dst_nodes[i];
         int64_t gb = 0, deg = 0;
         if ((uint32_t)u < (uint64_t)n_nodes) {
@@ -168,11 +169,10 @@ hop_sample_kernel(const int64_t *__restrict__ g_indptr, const int32_t *__restric
         src_nodes[i] = u;
     }
     int32_t tile_total;
-    const int32_t ex = block_exclusive_scan<kDstTile, int32_t>(c, tile_total, scan_sm);
-    off[threadIdx.x] = ex;
-    if (threadIdx.x == kDstTile - 1) off[kDstTile] = tile_total;
+    const int32_t ex = block_exclusive_scan<kDstThreads, int32_t>(c, tile_total, scan_sm);
+    if (threadIdx.x <= kDstTile) off[threadIdx.x] = ex;          // off[kDstTile] = the tile's total
     const long long base = chain_lookback(state, tile, tile_total, &counts[CNT_STATUS], &bcast);   // syncs the block
-    if (i < n_dst) blk_indptr[i] = (int32_t)(base + ex);
+    if (threadIdx.x < kDstTile && i < n_dst) blk_indptr[i] = (int32_t)(base + ex);
     const bool last_tile = i0 + kDstTile >= n_dst;
     if (last_tile && threadIdx.x == 0) {
         const long long total = base + tile_total;
@@ -184,14 +184,14 @@ hop_sample_kernel(const int64_t *__restrict__ g_indptr, const int32_t *__restric
     // four slots per thread and round, so that the loads of the graph entry, of the frontier position and of
     // the bitmap word are in flight for all four before any of them is needed
     constexpr int S = 4;
-    for (int32_t sl0 = threadIdx.x; sl0 < tile_total; sl0 += kDstTile * S) {
+    for (int32_t sl0 = threadIdx.x; sl0 < tile_total; sl0 += kDstThreads * S) {
         int rr[S];
         long long e[S];
         int64_t src[S];
         bool ok[S];
 #pragma unroll
         for (int q = 0; q < S; ++q) {
-            const int32_t sl = sl0 + q * kDstTile;
+            const int32_t sl = sl0 + q * kDstThreads;
             ok[q] = sl < tile_total;
             rr[q] = 0;
             e[q] = 0;
@@ -557,7 +557,7 @@ int32_t e2egrec::sample_khop_impl(const e2egrec_csr *graph, const int32_t *seeds
         const SortPlan sp = sort_plan(b.cap_src);
         cudaMemsetAsync(s.arena, 0, s.arena_bytes, st);
         note_launch();
-        hop_sample_kernel<<<grid_for(b.cap_dst, kDstTile), kDstTile, 0, st>>>(
+        hop_sample_kernel<<<grid_for(b.cap_dst, kDstTile), kDstThreads, 0, st>>>(
             graph->indptr, graph->indices, n, dst_nodes, n_dst_ptr, b.cap_dst, b.cap_edges, f, h + 1,
             (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), step, s.step_offset, h == 0, b.counts, b.indptr,
             b.inv_cnt, b.src_nodes, b.nbr_global, s.edge_row, s.local_id, s.bitmap, s.tickets + 0, s.state_dst);
