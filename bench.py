@@ -220,7 +220,7 @@ def run_ours(args, w):
 
     def step_body():
         """Everything of one training step, on fixed buffers (seeds_in, dH_in), so that it can be recorded."""
-        E.sample_khop(indptr, indices, seeds_in, blocks, w.seed, 0)         # step number = the scratch's offset
+        E.sample_khop(indptr, indices, seeds_in, blocks, w.seed, 0, defer_transpose=True)   # step = the scratch's offset
         E.sage_forward(blocks, X, Ws, ctx=ctx, H_out=H_out)
         E.sage_backward(blocks, X, Ws, ctx, dH_in, dWs=dWs, dX_rows=dX, scratch=scratch)
         count_total.add_(blocks.counts)

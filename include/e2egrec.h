@@ -61,6 +61,9 @@ extern "C" {
 /* flags of e2egrec_aggregate_forward */
 #define E2EGREC_AGG_SUM 1u           /* plain sum instead of the mean */
 
+/* flags of e2egrec_sample_khop */
+#define E2EGREC_SAMPLE_DEFER_TRANSPOSE 1u   /* csc_* arrays become valid only after e2egrec_sage_backward / e2egrec_sample_join */
+
 /* flags of e2egrec_sage_backward */
 #define E2EGREC_ACCUMULATE_DW 1u     /* add to dW / dbias instead of overwriting them */
 
@@ -169,11 +172,23 @@ int32_t e2egrec_sampler_set_step(void *scratch, uint32_t step_offset, void *stre
  *       (seed, step, h, u) only and reproducible bit for bit.
  *   blocks host array[n_hops] of structs holding device pointers; blocks[h-1] receives hop h
  *       including its transposed form.  F_h = D_h followed by the new nodes in ascending order.
- *   scratch device buffer initialised by e2egrec_sampler_scratch_init for the same n_nodes. */
+ *   scratch device buffer initialised by e2egrec_sampler_scratch_init for the same n_nodes.
+ *   flags 0 or E2EGREC_SAMPLE_DEFER_TRANSPOSE.
+ * The transposed form of a hop is built on a helper stream of the library (one per device, created on
+ * the first call) beside the sampling of the next hop.  By default the call joins that work back into
+ * `stream` before it returns.  With E2EGREC_SAMPLE_DEFER_TRANSPOSE it does not: indptr / col / nbr_global /
+ * src_nodes / inv_cnt / counts are valid in stream order as always, but the csc_* arrays are only complete
+ * after the next e2egrec_sage_backward or e2egrec_sample_join issued from the same device on this or any
+ * later-ordered stream (e2egrec_sage_forward does not need them, so the forward pass overlaps the
+ * transposition).  The next e2egrec_sample_khop joins by itself.  Do not interleave deferred calls from
+ * several host threads on one device. */
 int32_t e2egrec_sample_khop(const e2egrec_csr *graph, const int32_t *seeds, int32_t n_seeds,
                             int32_t n_hops, const int32_t *fanouts, uint64_t seed, uint32_t step,
                             uint32_t flags, const e2egrec_block *blocks,
                             void *scratch, size_t scratch_bytes, void *stream);
+
+/* Makes `stream` wait for a block transposition that e2egrec_sample_khop deferred (no-op if there is none). */
+int32_t e2egrec_sample_join(void *stream);
 
 /* GraphSAGE forward over sampled blocks (Sec. 3.1): for layer l = 0..n_layers-1, on block
  * h = n_layers - l,

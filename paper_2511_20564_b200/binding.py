@@ -62,6 +62,8 @@ def lib():
         L.e2egrec_sampler_scratch_init.argtypes = [C.c_int64, C.c_void_p, C.c_size_t, C.c_void_p]
         L.e2egrec_sampler_set_step.restype = C.c_int32
         L.e2egrec_sampler_set_step.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
+        L.e2egrec_sample_join.restype = C.c_int32
+        L.e2egrec_sample_join.argtypes = [C.c_void_p]
         L.e2egrec_sample_khop.restype = C.c_int32
         L.e2egrec_sample_khop.argtypes = [C.POINTER(Csr), C.c_void_p, C.c_int32, C.c_int32, C.c_void_p,
                                           C.c_uint64, C.c_uint32, C.c_uint32, C.POINTER(Block), C.c_void_p,
@@ -227,14 +229,22 @@ def sampler_set_step(scratch: torch.Tensor, step_offset: int, stream=None):
            "e2egrec_sampler_set_step")
 
 
+DEFER_TRANSPOSE = 1
+
+
+def sample_join(stream=None):
+    _check(lib().e2egrec_sample_join(_stream(stream)), "e2egrec_sample_join")
+
+
 def sample_khop(indptr: torch.Tensor, indices: torch.Tensor, seeds: torch.Tensor, blocks: Blocks, seed: int,
-                step: int, stream=None):
+                step: int, stream=None, defer_transpose=False):
     """Enqueues the k-hop sample of `seeds` into `blocks` (see e2egrec_sample_khop)."""
     assert indptr.dtype == torch.int64 and indices.dtype == torch.int32 and seeds.dtype == torch.int32
     g = Csr(indptr.numel() - 1, indices.numel(), indptr.data_ptr(), indices.data_ptr(), None)
     f = _i32_host(blocks.fanouts)
     _check(lib().e2egrec_sample_khop(C.byref(g), _ptr(seeds), seeds.numel(), len(blocks), f,
-                                     C.c_uint64(seed), C.c_uint32(step), 0, blocks.c, _ptr(blocks.scratch),
+                                     C.c_uint64(seed), C.c_uint32(step), DEFER_TRANSPOSE if defer_transpose else 0, blocks.c,
+                                     _ptr(blocks.scratch),
                                      blocks.scratch.numel(), _stream(stream)), "e2egrec_sample_khop")
 
 

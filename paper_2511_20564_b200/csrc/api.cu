@@ -1,5 +1,6 @@
 // Status strings and error bookkeeping of the C ABI.
 #include <atomic>
+#include <mutex>
 #include <stdio.h>
 #include <string.h>
 
@@ -25,6 +26,56 @@ int32_t check_launch(const char *what)
     return E2EGREC_ERR_CUDA;
 }
 
+static std::mutex g_side_mutex;
+static SideStream *g_side[64] = {};
+
+SideStream *SideStream::get()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_side_mutex);
+    if (!g_side[dev]) {
+        SideStream *s = new SideStream();
+        s->next = 0;
+        if (cudaStreamCreateWithFlags(&s->stream, cudaStreamNonBlocking) != cudaSuccess) { delete s; cudaGetLastError(); return nullptr; }
+        for (int i = 0; i < 32; ++i)
+            if (cudaEventCreateWithFlags(&s->ev[i], cudaEventDisableTiming) != cudaSuccess) { delete s; cudaGetLastError(); return nullptr; }
+        if (cudaEventCreateWithFlags(&s->pending, cudaEventDisableTiming) != cudaSuccess) { delete s; cudaGetLastError(); return nullptr; }
+        s->has_pending = false;
+        g_side[dev] = s;
+    }
+    return g_side[dev];
+}
+
+cudaEvent_t SideStream::event() { return ev[(next++) & 31u]; }
+
+void SideStream::fork(cudaStream_t from)
+{
+    cudaEvent_t e = event();
+    cudaEventRecord(e, from);
+    cudaStreamWaitEvent(stream, e, 0);
+}
+
+void SideStream::join(cudaStream_t into)
+{
+    cudaEvent_t e = event();
+    cudaEventRecord(e, stream);
+    cudaStreamWaitEvent(into, e, 0);
+}
+
+void SideStream::defer()
+{
+    cudaEventRecord(pending, stream);
+    has_pending = true;
+}
+
+void SideStream::join_pending(cudaStream_t into)
+{
+    if (!has_pending) return;
+    cudaStreamWaitEvent(into, pending, 0);
+    has_pending = false;
+}
+
 static std::atomic<uint64_t> g_launches{0};
 void note_launch() { g_launches.fetch_add(1, std::memory_order_relaxed); }
 
@@ -44,6 +95,13 @@ void tap_end(int which, cudaStream_t st)
 }
 
 }  // namespace e2egrec
+
+extern "C" int32_t e2egrec_sample_join(void *stream)
+{
+    e2egrec::SideStream *side = e2egrec::SideStream::get();
+    if (side) side->join_pending(static_cast<cudaStream_t>(stream));
+    return e2egrec::check_launch("sample_join");
+}
 
 extern "C" uint64_t e2egrec_launch_count(void) { return e2egrec::g_launches.load(std::memory_order_relaxed); }
 

@@ -25,7 +25,7 @@ int32_t khop_caps(int64_t n_nodes, int32_t n_seeds, int32_t n_hops, const int32_
                   int32_t *cap_src, int32_t *cap_edges);
 size_t sampler_scratch_bytes(int64_t n_nodes, int64_t max_dst, int64_t max_src, int64_t max_edges);
 int32_t sample_khop_impl(const e2egrec_csr *graph, const int32_t *seeds, int32_t n_seeds, const PairInput *pairs,
-                         int32_t n_hops, const int32_t *fanouts, uint64_t seed, uint32_t step,
+                         int32_t n_hops, const int32_t *fanouts, uint64_t seed, uint32_t step, uint32_t flags,
                          const e2egrec_block *blocks, void *scratch, size_t scratch_bytes, cudaStream_t st);
 
 }  // namespace e2egrec

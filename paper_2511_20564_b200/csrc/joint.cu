@@ -333,7 +333,8 @@ int32_t run_joint(const JointPlan &jp, const e2egrec_csr *graph, const e2egrec_m
     pi.pcsc_col = i32(jp.pcsc_col_off);
     pi.units_per_row = jp.zdim / jp.unit;
     pi.item_unit_off = jp.dL / jp.unit;
-    int32_t rc = sample_khop_impl(graph, nullptr, jp.P2, &pi, jp.n_hops, fanouts, seed, step, blocks, ws, jp.sampler_bytes, st);
+    int32_t rc = sample_khop_impl(graph, nullptr, jp.P2, &pi, jp.n_hops, fanouts, seed, step, E2EGREC_SAMPLE_DEFER_TRANSPOSE, blocks, ws,
+                                  jp.sampler_bytes, st);
     if (rc != E2EGREC_OK) return rc;
     note_launch();
     joint_meta_kernel<<<1, 1, 0, st>>>(pmeta, jp.P);

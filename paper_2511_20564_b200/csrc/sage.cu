@@ -321,6 +321,7 @@ extern "C" int32_t e2egrec_sage_backward(const e2egrec_block *blocks, int32_t n_
     const size_t es = dtype_size(X->dtype);
     if ((dX_rows->ld * es) % 16 || reinterpret_cast<uintptr_t>(dX_rows->data) % 16) return E2EGREC_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (SideStream *side = SideStream::get()) side->join_pending(st);     // a deferred block transposition
     if (X->dtype == E2EGREC_BF16)
         return backward_impl<__nv_bfloat16>(blocks, n_layers, X, W, act, plan, static_cast<const char *>(ctx), dH_out, dW,
                                             dbias, dX_rows, static_cast<char *>(scratch), bs, flags, st);

@@ -39,21 +39,30 @@ constexpr int kDstTile = 64;           // destinations per block of the sampling
 constexpr int kDstThreads = 256;       // its threads: one per destination for the counts, then all of them draw
 constexpr int kWordTile = 2048;        // bitmap words per block of the frontier kernel
 
+// Everything one block transposition (radix sort by column + offsets) needs; one lane per hop, so that the
+// transposition of hop h can run beside the sampling of hop h+1.
+struct SortLane {
+    int32_t  *edge_row;    // [max cap_edges]   destination of each block entry
+    int32_t  *keys[2];     // [max cap_edges]   radix sort ping-pong
+    int32_t  *vals[2];
+    unsigned *ghist;                   // [kMaxPasses x kMaxRadix] digit counts of the whole key array (zeroed before relabel)
+    char     *arena;                   // tickets + tile states, zeroed before the sort
+    size_t    arena_bytes;
+    unsigned *tickets;                 // [kMaxPasses]
+    unsigned long long *state;         // [kMaxPasses x kMaxRadix x sort tiles]
+};
+
 struct SamplerScratch {
     uint32_t *step_offset; // [1]         added to the `step` argument of every call (see e2egrec_sampler_set_step)
     int32_t  *local_id;    // [n_nodes]   -1 when idle, else position in the current frontier
     uint32_t *bitmap;      // [n_words]   newly reached nodes of the hop in progress; 0 when idle
-    int32_t  *edge_row;    // [max cap_edges]   destination of each block entry
-    int32_t  *keys[2];     // [max cap_edges]   radix sort ping-pong
-    int32_t  *vals[2];
-    // chain arena, zeroed at the start of every hop
+    // chain arena of the sampling / frontier kernels, zeroed at the start of every hop
     char     *arena;
     size_t    arena_bytes;
-    unsigned *tickets;                 // [8]
+    unsigned *tickets;                 // [2]
     unsigned long long *state_dst;     // [dst tiles]
     unsigned long long *state_words;   // [word tiles]
-    unsigned *ghist;                   // [kMaxPasses x kMaxRadix] digit counts of the whole key array
-    unsigned long long *state_sort;    // [kMaxPasses x kMaxRadix x sort tiles]
+    SortLane  lane[kMaxHops];
     int64_t   sort_tiles;
     size_t    bytes;
     int64_t   n_words;
@@ -74,17 +83,24 @@ static SamplerScratch carve(int64_t n_nodes, int64_t max_dst, int64_t max_src, i
     s.step_offset = (uint32_t *)take(256);
     s.local_id = (int32_t *)take(sizeof(int32_t) * (size_t)n_nodes);
     s.bitmap = (uint32_t *)take(sizeof(uint32_t) * (size_t)s.n_words);
-    s.edge_row = (int32_t *)take(sizeof(int32_t) * (size_t)(max_edges + 1));
-    for (int i = 0; i < 2; ++i) s.keys[i] = (int32_t *)take(sizeof(int32_t) * (size_t)(max_edges + 1));
-    for (int i = 0; i < 2; ++i) s.vals[i] = (int32_t *)take(sizeof(int32_t) * (size_t)(max_edges + 1));
-    const size_t arena_begin = off;
+    size_t begin = off;
     s.arena = base ? static_cast<char *>(base) + off : nullptr;
     s.tickets = (unsigned *)take(256);
     s.state_dst = (unsigned long long *)take(8 * (size_t)(ceil_div(max_dst > 0 ? max_dst : 1, kDstTile) + 1));
     s.state_words = (unsigned long long *)take(8 * (size_t)(ceil_div(s.n_words > 0 ? s.n_words : 1, kWordTile) + 1));
-    s.ghist = (unsigned *)take(sizeof(unsigned) * kMaxPasses * kMaxRadix);
-    s.state_sort = (unsigned long long *)take(8 * (size_t)kMaxPasses * kMaxRadix * (size_t)s.sort_tiles);
-    s.arena_bytes = off - arena_begin;
+    s.arena_bytes = off - begin;
+    for (int h = 0; h < kMaxHops; ++h) {
+        SortLane &l = s.lane[h];
+        l.edge_row = (int32_t *)take(sizeof(int32_t) * (size_t)(max_edges + 1));
+        for (int i = 0; i < 2; ++i) l.keys[i] = (int32_t *)take(sizeof(int32_t) * (size_t)(max_edges + 1));
+        for (int i = 0; i < 2; ++i) l.vals[i] = (int32_t *)take(sizeof(int32_t) * (size_t)(max_edges + 1));
+        l.ghist = (unsigned *)take(sizeof(unsigned) * kMaxPasses * kMaxRadix);
+        begin = off;
+        l.arena = base ? static_cast<char *>(base) + off : nullptr;
+        l.tickets = (unsigned *)take(256);
+        l.state = (unsigned long long *)take(8 * (size_t)kMaxPasses * kMaxRadix * (size_t)s.sort_tiles);
+        l.arena_bytes = off - begin;
+    }
     s.bytes = off;
     return s;
 }
@@ -387,15 +403,15 @@ pair_local_kernel(const int32_t *__restrict__ user, const int32_t *__restrict__ 
 }
 
 static void sort_by_col(const int32_t *col, int32_t *counts, int32_t cap_edges, int32_t *csc_col, int32_t *csc_eid,
-                        const SortPlan &sp, SamplerScratch &s, cudaStream_t st)
+                        const SortPlan &sp, const SortLane &l, int64_t sort_tiles, cudaStream_t st)
 {
     RadixScratch rs{};
-    rs.keys[0] = s.keys[0]; rs.keys[1] = s.keys[1];
-    rs.vals[0] = s.vals[0]; rs.vals[1] = s.vals[1];
-    rs.tickets = s.tickets + 2;
-    rs.ghist = s.ghist;
-    rs.state = s.state_sort;
-    rs.tiles = s.sort_tiles;
+    rs.keys[0] = l.keys[0]; rs.keys[1] = l.keys[1];
+    rs.vals[0] = l.vals[0]; rs.vals[1] = l.vals[1];
+    rs.tickets = l.tickets;
+    rs.ghist = l.ghist;
+    rs.state = l.state;
+    rs.tiles = sort_tiles;
     radix_sort_pairs(col, nullptr, counts, cap_edges, csc_col, csc_eid, sp, rs, st);
 }
 
@@ -488,14 +504,13 @@ extern "C" int32_t e2egrec_sample_khop(const e2egrec_csr *graph, const int32_t *
                                        uint32_t flags, const e2egrec_block *blocks,
                                        void *scratch, size_t scratch_bytes, void *stream)
 {
-    (void)flags;
     if (n_seeds > 0 && !seeds) return E2EGREC_ERR_NULL;
-    return sample_khop_impl(graph, seeds, n_seeds, nullptr, n_hops, fanouts, seed, step, blocks, scratch, scratch_bytes,
+    return sample_khop_impl(graph, seeds, n_seeds, nullptr, n_hops, fanouts, seed, step, flags, blocks, scratch, scratch_bytes,
                             static_cast<cudaStream_t>(stream));
 }
 
 int32_t e2egrec::sample_khop_impl(const e2egrec_csr *graph, const int32_t *seeds, int32_t n_seeds, const PairInput *pairs,
-                                  int32_t n_hops, const int32_t *fanouts, uint64_t seed, uint32_t step,
+                                  int32_t n_hops, const int32_t *fanouts, uint64_t seed, uint32_t step, uint32_t flags,
                                   const e2egrec_block *blocks, void *scratch, size_t scratch_bytes, cudaStream_t st)
 {
     if (!graph || !fanouts || !blocks || !scratch || !graph->indptr) return E2EGREC_ERR_NULL;
@@ -540,40 +555,59 @@ int32_t e2egrec::sample_khop_impl(const e2egrec_csr *graph, const int32_t *seeds
         frontier_kernel<<<grid_for(s.n_words, kWordTile), 256, 0, st>>>(s.bitmap, s.n_words, pi.pcounts, P2, s.local_id,
                                                                         pi.seeds_out, s.tickets + 1, s.state_words);
         const SortPlan sp = sort_plan(P2 > 1 ? P2 : 2);
+        const SortLane &l = s.lane[0];
+        cudaMemsetAsync(l.ghist, 0, sizeof(unsigned) * kMaxPasses * kMaxRadix, st);
+        cudaMemsetAsync(l.arena, 0, l.arena_bytes, st);
         note_launch();
         pair_local_kernel<<<(unsigned)std::min<int64_t>(grid_for(P2, T), 148 * 4), T, 0, st>>>(
             pi.user, pi.item, pi.n_pairs, n, s.local_id, pi.pair_local, pi.entry_unit, pi.units_per_row, pi.item_unit_off,
-            pi.pcounts, sp.bits, sp.passes, s.ghist);
-        sort_by_col(pi.pair_local, pi.pcounts, P2, pi.pcsc_col, pi.pcsc_eid, sp, s, st);
+            pi.pcounts, sp.bits, sp.passes, l.ghist);
+        sort_by_col(pi.pair_local, pi.pcounts, P2, pi.pcsc_col, pi.pcsc_eid, sp, l, s.sort_tiles, st);
         note_launch();
         csc_finalize_kernel<<<grid_for((int64_t)P2 + 1, T), T, 0, st>>>(pi.pcsc_col, pi.pcsc_eid, pi.entry_unit, pi.pcounts,
                                                                        pi.pcsc_ptr, pi.pcsc_idx);
         dst_nodes = pi.seeds_out;
         n_dst_ptr = &pi.pcounts[CNT_SRC];
     }
+    // The transposition of a hop (sort + offsets) is only needed by the backward pass, so it runs on the
+    // helper stream beside the sampling of the next hop; everything is joined before this call returns.
+    SideStream *side = SideStream::get();
+    if (side) side->join_pending(st);               // a transposition deferred by an earlier call still uses the lanes
     for (int h = 0; h < n_hops; ++h) {
         const e2egrec_block &b = blocks[h];
         const int32_t f = fanouts[h];
         const SortPlan sp = sort_plan(b.cap_src);
+        const SortLane &l = s.lane[h];
         cudaMemsetAsync(s.arena, 0, s.arena_bytes, st);
         note_launch();
         hop_sample_kernel<<<grid_for(b.cap_dst, kDstTile), kDstThreads, 0, st>>>(
             graph->indptr, graph->indices, n, dst_nodes, n_dst_ptr, b.cap_dst, b.cap_edges, f, h + 1,
             (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), step, s.step_offset, h == 0, b.counts, b.indptr,
-            b.inv_cnt, b.src_nodes, b.nbr_global, s.edge_row, s.local_id, s.bitmap, s.tickets + 0, s.state_dst);
+            b.inv_cnt, b.src_nodes, b.nbr_global, l.edge_row, s.local_id, s.bitmap, s.tickets + 0, s.state_dst);
         note_launch();
         frontier_kernel<<<grid_for(s.n_words, kWordTile), 256, 0, st>>>(s.bitmap, s.n_words, b.counts, b.cap_src,
                                                                         s.local_id, b.src_nodes, s.tickets + 1,
                                                                         s.state_words);
+        cudaMemsetAsync(l.ghist, 0, sizeof(unsigned) * kMaxPasses * kMaxRadix, st);
         note_launch();
         relabel_kernel<<<(unsigned)std::min<int64_t>(grid_for(b.cap_edges, T), 148 * 4), T, 0, st>>>(
-            b.nbr_global, s.local_id, b.counts, b.col, sp.bits, sp.passes, s.ghist);
-        sort_by_col(b.col, b.counts, b.cap_edges, b.csc_col, b.csc_eid, sp, s, st);
+            b.nbr_global, s.local_id, b.counts, b.col, sp.bits, sp.passes, l.ghist);
+        cudaStream_t ts = st;                        // stream of the transposition
+        if (side) {
+            side->fork(st);
+            ts = side->stream;
+        }
+        cudaMemsetAsync(l.arena, 0, l.arena_bytes, ts);
+        sort_by_col(b.col, b.counts, b.cap_edges, b.csc_col, b.csc_eid, sp, l, s.sort_tiles, ts);
         note_launch();
-        csc_finalize_kernel<<<grid_for(std::max<int64_t>(b.cap_edges, (int64_t)b.cap_src + 1), T), T, 0, st>>>(
-            b.csc_col, b.csc_eid, s.edge_row, b.counts, b.csc_ptr, b.csc_row);
+        csc_finalize_kernel<<<grid_for(std::max<int64_t>(b.cap_edges, (int64_t)b.cap_src + 1), T), T, 0, ts>>>(
+            b.csc_col, b.csc_eid, l.edge_row, b.counts, b.csc_ptr, b.csc_row);
         dst_nodes = b.src_nodes;
         n_dst_ptr = &b.counts[CNT_SRC];
+    }
+    if (side) {
+        if (flags & E2EGREC_SAMPLE_DEFER_TRANSPOSE) side->defer();
+        else side->join(st);
     }
     const e2egrec_block &last = blocks[n_hops - 1];
     note_launch();

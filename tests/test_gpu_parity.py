@@ -256,3 +256,34 @@ def test_lightgcn_forward_and_adjoint(dtype, d):
     want = oracle.lightgcn_forward(indptr, indices, G, L, bf16)
     rss = np.sqrt(oracle.lightgcn_propagate(indptr, indices, G.astype(np.float64) ** 2)) if bf16 else None
     assert_close("lightgcn_backward", dH0.float().cpu().numpy(), want, bf16, rss)
+
+
+def test_deferred_transposition_joins_before_use():
+    """With the defer flag the csc arrays are complete after e2egrec_sample_join, and the backward pass joins by itself."""
+    import paper_2511_20564_b200 as E
+    w = S.WORKLOADS["medium_small"]
+    case = Case(w, step=6)
+    ora = case.run_oracle(case.upstream_grad(case.seeds.size, w.hidden))
+    ip, ix = torch.from_numpy(case.indptr).cuda(), torch.from_numpy(case.indices).cuda()
+    X = torch.from_numpy(case.X).cuda().to(torch.bfloat16)
+    Ws = [torch.from_numpy(W).cuda().to(torch.bfloat16) for W in case.Ws]
+    seeds = torch.from_numpy(case.seeds).cuda()
+    blocks = E.Blocks(w.n_nodes, case.seeds.size, w.fanouts)
+    g = torch.zeros(max(blocks.caps[0][0], 1), w.hidden, dtype=torch.bfloat16, device="cuda")
+    g[: case.seeds.size] = torch.from_numpy(case.upstream_grad(case.seeds.size, w.hidden)).cuda().to(torch.bfloat16)
+    for _ in range(2):                                       # the second round starts while nothing is pending
+        E.sample_khop(ip, ix, seeds, blocks, w.seed, 6, defer_transpose=True)
+        H, ctx = E.sage_forward(blocks, X, Ws)
+        dWs, dX = E.sage_backward(blocks, X, Ws, ctx, g)     # joins the deferred work itself
+        torch.cuda.synchronize()
+        assert_blocks_equal(blocks.to_host(), ora["blocks"])
+        n_src = ora["blocks"][-1]["n_src"]
+        rss = reduction_rss(case, ora)
+        for l, (a, b) in enumerate(zip(dWs, ora["dWs"])):
+            assert_close(f"dW[{l}]", a.cpu().numpy(), b, True, rss["dW"][l] + 0 * b,
+                         budget=relu_flip_budgets(case, ora, dict(layer_out=[h.float().cpu().numpy() for _, h in
+                                                                             E.sage_ctx_views(blocks, X, Ws, ctx)]), 2e-2)[0][l])
+    E.sample_khop(ip, ix, seeds, blocks, w.seed, 6, defer_transpose=True)
+    E.sample_join()
+    torch.cuda.synchronize()
+    assert_blocks_equal(blocks.to_host(), ora["blocks"])
