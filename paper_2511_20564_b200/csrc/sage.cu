@@ -176,6 +176,8 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
             static_cast<const T *>(dH_out->data), dH_out->ld, reinterpret_cast<const T *>(ctx + p.h_off), p.d_out,
             &b.counts[CNT_DST], p.rows, p.d_out, act ? act[n_layers - 1] : 1, dz_buf[(n_layers - 1) & 1]);
     }
+    SideStream *side = SideStream::get();
+    cudaEvent_t dz_free[2] = {nullptr, nullptr};
     for (int l = n_layers - 1; l >= 0; --l) {
         const LayerPlan &p = plan[l];
         const e2egrec_block &b = blocks[p.block];
@@ -183,31 +185,42 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
         const T *cat = reinterpret_cast<const T *>(ctx + p.cat_off);
         const int32_t *n_dst = &b.counts[CNT_DST];
         const int two_d = 2 * p.d_in;
-        // dW_l = dZ^T [h | agg]   (split over the rows, partial sums added in a fixed order)
-        if (l == 0) tap_begin(TAP_DW_OUTER, st);
+        // dW_l = dZ^T [h | agg]   (split over the rows, partial sums added in a fixed order).  Nothing later in
+        // this call reads dW, so it runs on the helper stream beside the dCat product and the transposed
+        // aggregation; `dz_free` holds the event after which the helper stream no longer reads a dZ buffer.
+        cudaStream_t ws = st;
+        if (side) {
+            side->fork(st);
+            ws = side->stream;
+        }
+        if (l == 0) tap_begin(TAP_DW_OUTER, ws);
         bool dw_done = false;
         if (X->dtype == E2EGREC_BF16)
             dw_done = tc_weight_grad(reinterpret_cast<const __nv_bfloat16 *>(dz), p.rows, p.d_out,
                                      reinterpret_cast<const __nv_bfloat16 *>(cat), two_d, n_dst, part, kDwSplits,
-                                     &b.counts[CNT_STATUS], st);
+                                     &b.counts[CNT_STATUS], ws);
         if (!dw_done) {
             EpiPartial epi{part, two_d, (int64_t)p.d_out * two_d};
             dim3 grid((unsigned)ceil_div(p.d_out, kGemmBM), (unsigned)ceil_div(two_d, kGemmBN), kDwSplits);
             note_launch();
-            gemm_simt_kernel<T, true, true, EpiPartial><<<grid, kGemmThreads, 0, st>>>(
+            gemm_simt_kernel<T, true, true, EpiPartial><<<grid, kGemmThreads, 0, ws>>>(
                 dz, p.d_out, cat, two_d, p.d_out, two_d, p.rows, nullptr, n_dst, epi);
         }
         {
             const int64_t n = (int64_t)p.d_out * two_d;
             note_launch();
-            splitk_reduce_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(part, n, kDwSplits, accumulate, dW[l],
+            splitk_reduce_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, ws>>>(part, n, kDwSplits, accumulate, dW[l],
                                                                              dw_done ? n_dst : nullptr);
         }
-        if (l == 0) tap_end(TAP_DW_OUTER, st);
+        if (l == 0) tap_end(TAP_DW_OUTER, ws);
         if (dbias && dbias[l]) {
             note_launch();
-            colsum_kernel<T><<<(unsigned)ceil_div(p.d_out, 32), 256, 0, st>>>(dz, p.d_out, n_dst, p.d_out, accumulate,
+            colsum_kernel<T><<<(unsigned)ceil_div(p.d_out, 32), 256, 0, ws>>>(dz, p.d_out, n_dst, p.d_out, accumulate,
                                                                              dbias[l]);
+        }
+        if (side) {
+            dz_free[l & 1] = side->event();
+            cudaEventRecord(dz_free[l & 1], side->stream);
         }
         // dCat = dZ W_l, the agg half scaled by 1/|S|
         if (l == 0) tap_begin(TAP_DCAT_OUTER, st);
@@ -236,6 +249,11 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
         o.n_self = n_dst;
         o.mean = 0;
         if (l > 0) {
+            // the buffer that receives dZ of the layer below may still be read by the helper stream (layer l+1)
+            if (side && dz_free[(l - 1) & 1]) {
+                cudaStreamWaitEvent(st, dz_free[(l - 1) & 1], 0);
+                dz_free[(l - 1) & 1] = nullptr;
+            }
             o.out = dz_buf[(l - 1) & 1];
             o.ld_out = p.d_in;
             o.pad_rows = plan[l - 1].rows;
@@ -253,6 +271,7 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
                                                nullptr, kBlockRun, p.d_in, X->dtype, b.csc_col, sc, o, st);
         if (l == 0) tap_end(TAP_AGG_BWD_OUTER, st);
     }
+    if (side) side->join(st);
     return check_launch("sage_backward");
 }
 
