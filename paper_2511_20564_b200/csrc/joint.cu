@@ -375,9 +375,19 @@ int32_t run_joint(const JointPlan &jp, const e2egrec_csr *graph, const e2egrec_m
         note_launch();
         dz_top_kernel<T><<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(dt, W3, a2, jp.h2, jp.P, jp.rowsP, dz2);
     }
-    linear_backward_weight<T>(dz2, jp.rowsP, jp.h2, a1, jp.h1, pmeta, part, dW_tower[1], db_tower ? db_tower[1] : nullptr, status, st);
+    // the weight gradients feed nothing later in the step: they go to the helper stream (behind the block
+    // transposition that the sampler left there); the encoder backward waits for that stream before its first launch
+    SideStream *side = SideStream::get();
+    cudaStream_t ws_st = st;
+    if (side) {
+        side->fork(st);
+        ws_st = side->stream;
+    }
+    linear_backward_weight<T>(dz2, jp.rowsP, jp.h2, a1, jp.h1, pmeta, part, dW_tower[1], db_tower ? db_tower[1] : nullptr, status, ws_st);
     linear_backward_input<T>(dz2, jp.rowsP, jp.h2, W2, jp.h1, a1, dz1, wt, pmeta, status, st);
-    linear_backward_weight<T>(dz1, jp.rowsP, jp.h1, z, jp.zdim, pmeta, part, dW_tower[0], db_tower ? db_tower[0] : nullptr, status, st);
+    if (side) side->fork(st);
+    linear_backward_weight<T>(dz1, jp.rowsP, jp.h1, z, jp.zdim, pmeta, part, dW_tower[0], db_tower ? db_tower[0] : nullptr, status, ws_st);
+    if (side) side->defer();
     linear_backward_input<T>(dz1, jp.rowsP, jp.h1, W1, jp.zdim, nullptr, dz, wt, pmeta, status, st);
 
     // 5. gradient of every seed embedding: the rows of dz that belong to it, added in pair order
