@@ -88,9 +88,10 @@ template <> __device__ inline void store4<__nv_bfloat16>(__nv_bfloat16 *p, const
 }
 
 // ------------------------------------------------------------------------------------ level 1
-// Rarely taken paths of the level-1 kernel, kept out of line so that the streaming loop stays short.
+// Partial sums of a run go out as float4 stores.  Inlined on purpose: a call that receives the accumulators by
+// reference would pin them in local memory, and every add of the streaming loop would then store to it.
 template <int CPL, int E>
-__device__ __noinline__ void seg_store_partial(float *dst, const float (&acc)[CPL][E], int c, int lpr, int n_chunks)
+__device__ __forceinline__ void seg_store_partial(float *dst, const float (&acc)[CPL][E], int c, int lpr, int n_chunks)
 {
 #pragma unroll
     for (int q = 0; q < CPL; ++q) {
@@ -103,20 +104,21 @@ __device__ __noinline__ void seg_store_partial(float *dst, const float (&acc)[CP
     }
 }
 
-// Advances the walk to the segment that holds entry k (k >= end of segment *ws): a few steps one by one,
-// then by bisection if a long stretch of empty segments is in the way.  Returns that segment's end.
+// Advances the walk from segment s to the segment that holds entry k (k >= end of segment s): a few steps one
+// by one, then by bisection if a long stretch of empty segments is in the way.  Returns {segment, its end}; kept
+// out of line (the streaming loop stays short) and by value (nothing of the caller is forced into memory).
+struct SegStep { int64_t seg, end; };
 template <typename PtrT>
-__device__ __noinline__ int64_t seg_advance(const PtrT *__restrict__ ptr, int64_t n_seg, int64_t k, int64_t *ws)
+__device__ __noinline__ SegStep seg_advance(const PtrT *__restrict__ ptr, int64_t n_seg, int64_t k, int64_t s)
 {
-    int64_t s = *ws, end;
+    int64_t end;
     int step = 0;
     do { ++s; end = (int64_t)ptr[s + 1]; } while (end <= k && ++step < 4);
     if (end <= k) {
         s = seg_containing(ptr, n_seg, k);
         end = (int64_t)ptr[s + 1];
     }
-    *ws = s;
-    return end;
+    return SegStep{s, end};
 }
 
 // kExtra: the output has a self row and/or a mask row per segment (they are fetched together with the
@@ -183,7 +185,9 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
                 } else if (r == 0) {
                     start_n[u] = true;
                 } else if (r >= rel_end) {
-                    rel_end = (int)min(seg_advance(ptr, n_seg, k0 + r, &ws) - k0, (int64_t)kFar);
+                    const SegStep nx = seg_advance(ptr, n_seg, k0 + r, ws);
+                    ws = nx.seg;
+                    rel_end = (int)min(nx.end - k0, (int64_t)kFar);
                     start_n[u] = true;
                 }
                 seg_n[u] = (int32_t)ws;
