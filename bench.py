@@ -28,13 +28,13 @@ CLOCK_QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reason
                "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
                "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 TAP_NAMES = {1: "sage_aggregate_kernel (layer-0 mean aggregation, gathers X rows)",
-             2: "seg_run_kernel+seg_window_kernel+seg_final_kernel (layer-0 transposed aggregation -> dX rows)",
+             2: "seg_run_kernel+seg_final_kernel (layer-0 transposed aggregation -> dX rows)",
              3: "layer-0 dense transform W[h|agg]",
              4: "layer-0 weight gradient dZ^T[h|agg]",
              5: "layer-0 input gradient dZ W",
              6: "e2egrec_sample_khop (all sampling kernels)",
              7: "seg_run_kernel (first transposed aggregation of the backward pass)",
-             8: "seg_window_kernel (same)", 9: "seg_final_kernel (same)"}
+             9: "seg_final_kernel (same)"}
 
 
 def measured_peaks():
@@ -395,7 +395,7 @@ def run_ours(args, w):
                     unit="TFLOP/s")
     # DRAM bytes per launch from the ncu launch list of this command (profiles/medium_step_launch_list.md);
     # known only for the aggregation kernels of the outermost block of the `medium` workload
-    traffic = {1: 6.30e6, 2: 5.54e6 + 2.18e6 + 1.70e6}.get(dominant) if w.name == "medium" and args.seeds == "activity" else None
+    traffic = {1: 6.30e6}.get(dominant) if w.name == "medium" and args.seeds == "activity" else None
     roof.update(frac=roof["achieved"] / roof["peak"], traffic=traffic, kernel=TAP_NAMES[dominant],
                 ms_per_launch=dom_mean_ms, algorithmic_units_per_launch=alg, peak_source=peaks["source"])
 
@@ -513,7 +513,7 @@ def run_fullgraph(args):
     big = "fwd" if t_f >= t_b else "bwd"
     alg, tk = (alg_f, t_f) if big == "fwd" else (alg_b, t_b)
     roof = dict(bound="hbm", achieved=alg / tk / 1e6, peak=peaks["hbm_gbs"], unit="GB/s", traffic=None,
-                kernel=f"seg_run_kernel+seg_window_kernel+seg_final_kernel ({big})", ms_per_launch=tk,
+                kernel=f"seg_run_kernel+seg_final_kernel ({big})", ms_per_launch=tk,
                 algorithmic_units_per_launch=alg, peak_source=peaks["source"],
                 compulsory_bytes=n * r * 2 + m * 4 + n * 16)
     roof["frac"] = roof["achieved"] / roof["peak"]

@@ -7,11 +7,16 @@
 
 namespace e2egrec {
 
-static inline int full_run_len(int64_t n_entries) { return n_entries > (1ll << 24) ? 64 : 32; }
-
-static size_t full_ws_bytes(int64_t n_entries, int d)
+// Entries per run of the segment reduction: long runs on large inputs (fewer window records, fewer cut segments),
+// short ones where the input would not fill the machine otherwise.
+static inline int full_run_len(int64_t n_entries)
 {
-    return seg_scratch_carve(n_entries, full_run_len(n_entries), d, nullptr).bytes;
+    return n_entries >= (1ll << 24) ? 256 : n_entries >= (1ll << 22) ? 128 : n_entries >= (1ll << 20) ? 64 : 32;
+}
+
+static size_t full_ws_bytes(int64_t n_entries, int d, int32_t dtype)
+{
+    return seg_scratch_carve(n_entries, full_run_len(n_entries), d, dtype_size(dtype), nullptr).bytes;
 }
 
 template <typename T, bool kWeight>
@@ -20,7 +25,7 @@ static void dispatch_seg64(const T *in, int64_t ld_in, const int64_t *ptr, const
                            cudaStream_t st)
 {
     const int run_len = full_run_len(n_entries);
-    const SegScratch sc = seg_scratch_carve(n_entries, run_len, d, ws);
+    const SegScratch sc = seg_scratch_carve(n_entries, run_len, d, dtype_size(dtype), ws);
     dispatch_seg_reduce<T, int64_t, kWeight>(in, ld_in, ptr, idx, nullptr, n_seg, n_seg, w, run_len, d, dtype, nullptr, sc, o, st);
 }
 
@@ -80,7 +85,7 @@ static int32_t aggregate_entry(int64_t n_seg, int64_t n_entries, const int64_t *
     if (n_seg >= (1ll << 31)) return E2EGREC_ERR_UNSUPPORTED;
     int32_t rc = check_mats(in, out, n_seg);
     if (rc != E2EGREC_OK) return rc;
-    const size_t need = full_ws_bytes(n_entries, in->dim);
+    const size_t need = full_ws_bytes(n_entries, in->dim, in->dtype);
     if (!ws) { *ws_bytes = need; return E2EGREC_OK; }
     if (*ws_bytes < need) { *ws_bytes = need; return E2EGREC_ERR_WORKSPACE; }
     if (reinterpret_cast<uintptr_t>(ws) % 256) return E2EGREC_ERR_ALIGN;
@@ -156,7 +161,7 @@ static int32_t lightgcn_entry(int64_t n, int64_t m, const int64_t *ptr, const in
     if (H0->ld != H0->dim || Y->ld != Y->dim) return E2EGREC_ERR_ARG;
     const size_t es = dtype_size(H0->dtype);
     const size_t layer_bytes = align_up((size_t)(n > 0 ? n : 1) * H0->dim * es, 256);
-    const size_t seg_bytes = align_up(full_ws_bytes(m, H0->dim), 256);
+    const size_t seg_bytes = align_up(full_ws_bytes(m, H0->dim, H0->dtype), 256);
     const size_t need = seg_bytes + (size_t)n_layers * layer_bytes;
     if (!ws) { *ws_bytes = need; return E2EGREC_OK; }
     if (*ws_bytes < need) { *ws_bytes = need; return E2EGREC_ERR_WORKSPACE; }

@@ -322,14 +322,16 @@ seg_finish_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_
 
 struct RowShape { int lpr, cpl; };
 
-inline RowShape row_shape(int d, int32_t dtype)
+inline RowShape row_shape_bytes(int64_t row_bytes)
 {
-    const int chunks = d * (int)dtype_size(dtype) / 16;
+    const int chunks = (int)(row_bytes / 16);
     int lpr = 4;
     while (lpr < 32 && lpr < chunks) lpr <<= 1;
     int cpl = 1;
     while (lpr * cpl < chunks) cpl <<= 1;
     return {lpr, cpl};
 }
+
+inline RowShape row_shape(int d, int32_t dtype) { return row_shape_bytes((int64_t)d * (int64_t)dtype_size(dtype)); }
 
 }  // namespace e2egrec

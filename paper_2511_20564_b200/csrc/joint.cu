@@ -274,7 +274,7 @@ int32_t make_plan(const e2egrec_csr *graph, const e2egrec_mat *X, int32_t n_pair
     if (rc != E2EGREC_OK) return rc;
     jp.bwd_bytes = need;
     jp.bwd_off = take(need);
-    jp.seg_bytes = seg_scratch_carve(jp.P2, kPairRun, jp.dL, nullptr).bytes;
+    jp.seg_bytes = seg_scratch_carve(jp.P2, kPairRun, jp.dL, dtype_size(X->dtype), nullptr).bytes;
     jp.seg_off = take(jp.seg_bytes);
     const size_t p2 = (size_t)jp.P2;
     jp.seeds_off = take(p2 * 4);
@@ -395,7 +395,7 @@ int32_t run_joint(const JointPlan &jp, const e2egrec_csr *graph, const e2egrec_m
         SegOut<T> o{};
         o.out = tp(jp.dhseed_off);
         o.ld_out = jp.dL;
-        const SegScratch sc = seg_scratch_carve(jp.P2, kPairRun, jp.dL, ws + jp.seg_off);
+        const SegScratch sc = seg_scratch_carve(jp.P2, kPairRun, jp.dL, dtype_size(X->dtype), ws + jp.seg_off);
         dispatch_seg_reduce<T, int32_t, false>(dz, jp.unit, pi.pcsc_ptr, pi.pcsc_idx, &pcounts[CNT_SRC], 0, jp.P2, nullptr,
                                                kPairRun, jp.dL, X->dtype, pi.pcsc_col, sc, o, st);
     }

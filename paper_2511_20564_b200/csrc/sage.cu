@@ -140,7 +140,7 @@ static BackwardScratch plan_backward(const e2egrec_block *blocks, int32_t n_laye
         dcat = std::max(dcat, (size_t)p.rows * 2 * p.d_in * es);
         part = std::max(part, (size_t)kDwSplits * p.d_out * 2 * p.d_in * sizeof(float));
         wt = std::max(wt, (size_t)p.d_out * 2 * p.d_in * es);
-        ht = std::max(ht, seg_scratch_carve(blocks[p.block].cap_edges, kBlockRun, p.d_in, nullptr).bytes);
+        ht = std::max(ht, seg_scratch_carve(blocks[p.block].cap_edges, kBlockRun, p.d_in, es, nullptr).bytes);
     }
     size_t off = 0;
     auto take = [&](size_t b) { size_t o = off; off += align_up(b, 256); return o; };
@@ -266,7 +266,7 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
             o.mask = nullptr;
         }
         if (l == 0) tap_begin(TAP_AGG_BWD_OUTER, st);
-        const SegScratch sc = seg_scratch_carve(b.cap_edges, kBlockRun, p.d_in, scratch + bs.seg_off);
+        const SegScratch sc = seg_scratch_carve(b.cap_edges, kBlockRun, p.d_in, dtype_size(X->dtype), scratch + bs.seg_off);
         dispatch_seg_reduce<T, int32_t, false>(dcat + p.d_in, two_d, b.csc_ptr, b.csc_row, &b.counts[CNT_SRC], 0, b.cap_src,
                                                nullptr, kBlockRun, p.d_in, X->dtype, b.csc_col, sc, o, st);
         if (l == 0) tap_end(TAP_AGG_BWD_OUTER, st);

@@ -1,22 +1,22 @@
-// Segment reduction by gathered rows, three levels, no atomics, fixed summation order:
+// Segment reduction by gathered rows, two kernels, no atomics, fixed summation order:
 //
 //     out[s] = fin( sum_{k in [ptr[s], ptr[s+1])} w[idx[k]] * in[idx[k]] ),   fin as in SegOut.
 //
 // This is the transposed aggregation of the backward pass (segments = columns of the block CSC)
 // and the whole-graph aggregation in either direction (segments = CSR rows or CSC columns).
 //
-// Level 1 (seg_run_kernel): the entry stream is cut into runs of `run_len` consecutive entries and
-//   every group of LPR lanes owns one run.  The group streams through its run with several row loads
-//   in flight and closes a segment whenever the running entry index reaches the segment's end, so
-//   thousands of one-entry segments and one segment of millions of entries cost the same per entry.
-//   A segment that lies inside the run is finished there; otherwise its part goes to head[run]
-//   (segment began in an earlier run) or tail[run] (segment began here and continues), and run_info
-//   records which segments those are.  The optional self row of a segment is added where the segment
-//   begins, so partial sums already contain it.
-// Level 2 (seg_window_kernel): one warp per window of 32 runs adds the parts of segments that span
-//   runs of the window, in run order; segments that also leave the window go to head2/tail2.
-// Level 3 (seg_final_kernel): one block per window adds tail2[first] + head2[first+1..last] for the
-//   segment that ends in its window, and extra blocks write fin(0) for segments without entries.
+// seg_run_kernel.  The entry stream is cut into runs of `run_len` consecutive entries and every group of
+//   LPR lanes owns one run.  The group streams through its run with several row loads in flight and closes
+//   a segment whenever the running entry index reaches the segment's end, so thousands of one-entry
+//   segments and one segment of millions of entries cost the same per entry.  A segment that lies inside
+//   the run is finished there.  Otherwise its part stays in shared memory: head[run] (segment began in an
+//   earlier run) or tail[run] (segment began here and continues).  The optional self row of a segment is
+//   added where the segment begins, so partial sums already contain it.
+//   After a block barrier the runs of the block (its "window") are joined: the group whose run holds the
+//   end of a cut segment adds tail[first] + head[first+1] + ... + head[last] in run order and writes the
+//   result; a segment that also leaves the window leaves one row in head2[window] or tail2[window].
+// seg_final_kernel.  Adds tail2[first] + head2[first+1..last] for every segment cut by window boundaries
+//   (all threads of a block share one such sum), and extra blocks write fin(0) for segments without entries.
 #pragma once
 
 #include <algorithm>
@@ -25,31 +25,30 @@
 
 namespace e2egrec {
 
-constexpr int kSegWindow = 32;     // runs per level-2 window
+// runs per window = lane groups per block of seg_run_kernel
+inline int seg_runs_per_window(int d, size_t elem_size) { return kAggThreads / row_shape_bytes((int64_t)d * elem_size).lpr; }
 
 struct SegScratch {
-    float *head, *tail;            // [cap_runs x d]
-    int4 *run_info;                // {head segment or -1, head ends in this run, tail segment or -1, 0}
     float *head2, *tail2;          // [n_windows x d]
-    int4 *win_info;
+    int4 *win_info;                // {segment whose sum continues from an earlier window or -1, it ends here, segment
+                                   //  that continues into the next window or -1, 0}
     int64_t cap_runs, n_windows;
+    int runs_per_window;
     size_t bytes;
 };
 
-inline SegScratch seg_scratch_carve(int64_t cap_entries, int run_len, int d, void *base)
+inline SegScratch seg_scratch_carve(int64_t cap_entries, int run_len, int d, size_t elem_size, void *base)
 {
     SegScratch s{};
+    s.runs_per_window = seg_runs_per_window(d, elem_size);
     s.cap_runs = ceil_div(cap_entries > 0 ? cap_entries : 1, run_len);
-    s.n_windows = ceil_div(s.cap_runs, kSegWindow);
+    s.n_windows = ceil_div(s.cap_runs, s.runs_per_window);
     size_t off = 0;
     auto take = [&](size_t bytes) {
         char *p = base ? static_cast<char *>(base) + off : nullptr;
         off += align_up(bytes, 256);
         return p;
     };
-    s.head = (float *)take((size_t)s.cap_runs * d * sizeof(float));
-    s.tail = (float *)take((size_t)s.cap_runs * d * sizeof(float));
-    s.run_info = (int4 *)take((size_t)s.n_windows * kSegWindow * sizeof(int4));
     s.head2 = (float *)take((size_t)s.n_windows * d * sizeof(float));
     s.tail2 = (float *)take((size_t)s.n_windows * d * sizeof(float));
     s.win_info = (int4 *)take((size_t)s.n_windows * sizeof(int4));
@@ -87,23 +86,7 @@ template <> __device__ inline void store4<__nv_bfloat16>(__nv_bfloat16 *p, const
     *reinterpret_cast<uint2 *>(p) = make_uint2(*reinterpret_cast<uint32_t *>(&a), *reinterpret_cast<uint32_t *>(&b));
 }
 
-// ------------------------------------------------------------------------------------ level 1
-// Partial sums of a run go out as float4 stores.  Inlined on purpose: a call that receives the accumulators by
-// reference would pin them in local memory, and every add of the streaming loop would then store to it.
-template <int CPL, int E>
-__device__ __forceinline__ void seg_store_partial(float *dst, const float (&acc)[CPL][E], int c, int lpr, int n_chunks)
-{
-#pragma unroll
-    for (int q = 0; q < CPL; ++q) {
-        const int ch = c + q * lpr;
-        if (ch < n_chunks) {
-#pragma unroll
-            for (int e = 0; e < E; e += 4)
-                *reinterpret_cast<float4 *>(dst + ch * E + e) = make_float4(acc[q][e], acc[q][e + 1], acc[q][e + 2], acc[q][e + 3]);
-        }
-    }
-}
-
+// ------------------------------------------------------------------------------------ runs and windows
 // Advances the walk from segment s to the segment that holds entry k (k >= end of segment s): a few steps one
 // by one, then by bisection if a long stretch of empty segments is in the way.  Returns {segment, its end}; kept
 // out of line (the streaming loop stays short) and by value (nothing of the caller is forced into memory).
@@ -121,349 +104,426 @@ __device__ __noinline__ SegStep seg_advance(const PtrT *__restrict__ ptr, int64_
     return SegStep{s, end};
 }
 
+// Shared memory of seg_run_kernel (dynamic): head and tail rows of the block's runs, fp32, one row of
+// LPR*CPL*E floats per run, then one record per run.
+template <int LPR, int CPL, int E>
+constexpr size_t seg_run_smem_bytes()
+{
+    return (size_t)2 * (kAggThreads / LPR) * (LPR * CPL * E) * sizeof(float) + (size_t)(kAggThreads / LPR) * sizeof(int4);
+}
+
 // kExtra: the output has a self row and/or a mask row per segment (they are fetched together with the
 // segment's first gathered row); without it those registers and branches disappear.
 template <typename T, typename PtrT, int LPR, int CPL, bool kWeight, bool kExtra>
 __global__ void __launch_bounds__(kAggThreads)
 seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__ ptr, const int32_t *__restrict__ idx,
                const int32_t *n_seg_dev, int64_t n_seg_host, const float *__restrict__ w, int run_len, int d,
-               float *__restrict__ head, float *__restrict__ tail, int4 *__restrict__ run_info, int64_t cap_runs,
+               float *__restrict__ head2, float *__restrict__ tail2, int4 *__restrict__ win_info, int64_t cap_runs,
                const int32_t *__restrict__ seg_of, SegOut<T> o)
 {
     constexpr int E = Chunk<T>::kElems;
     constexpr int U = CPL >= 4 ? 1 : 4 / CPL;
+    constexpr int RB = kAggThreads / LPR;          // runs of this block = one window
+    constexpr int ROW = LPR * CPL * E;             // floats per shared row (>= d)
     constexpr int kFar = 1 << 30;
+    extern __shared__ float4 seg_smem[];
+    float *sh_head = reinterpret_cast<float *>(seg_smem);
+    float *sh_tail = sh_head + RB * ROW;
+    int4 *sh_info = reinterpret_cast<int4 *>(sh_tail + RB * ROW);
+    __shared__ int32_t sh_win[4];
+
     const int c = threadIdx.x % LPR;
+    const int rl = threadIdx.x / LPR;              // run within the block
     const int n_chunks = d / E;
-    const int64_t run = ((int64_t)blockIdx.x * kAggThreads + threadIdx.x) / LPR;
-    if (run >= cap_runs) return;
+    const int64_t run = (int64_t)blockIdx.x * RB + rl;
     const int64_t n_seg = n_seg_dev ? (int64_t)*n_seg_dev : n_seg_host;
     const int64_t total = n_seg > 0 ? (int64_t)ptr[n_seg] : 0;
     const int64_t k0 = run * run_len;
-    if (k0 >= total) {
-        if (c == 0) run_info[run] = make_int4(-1, 0, -1, 0);
-        return;
-    }
-    const int len = (int)min((int64_t)run_len, total - k0);       // entries of this run; positions below are relative to k0
-    const int32_t *__restrict__ idx0 = idx + k0;
-    const int32_t *__restrict__ seg0 = seg_of ? seg_of + k0 : nullptr;
-    const int64_t n_self = (kExtra && o.self) ? (o.n_self ? (int64_t)*o.n_self : n_seg) : 0;
+    int32_t head_seg = -1, head_ends = 0, tail_seg = -1;
 
-    // Segment boundaries are found one iteration ahead of the sums.  With an entry -> segment array a
-    // boundary is a change of that value; without it the offsets are walked.
-    int64_t ws;                    // segment of the entry classified last
-    int rel_end = kFar;            // its end (walk mode)
-    int first_beg_rel = 0;         // where the run's first segment begins (<= 0)
-    bool first_begins, last_ends = false;
-    if (seg0) {
-        ws = seg0[0];
-        first_begins = k0 == 0 || seg0[-1] != (int32_t)ws;
-        last_ends = k0 + len == total || seg0[len] != seg0[len - 1];
-        if (o.mean) first_beg_rel = (int)max((int64_t)ptr[ws] - k0, (int64_t)-kFar);
-    } else {
-        ws = seg_containing(ptr, n_seg, k0);
-        const int64_t wb = (int64_t)ptr[ws] - k0;
-        first_begins = wb >= 0;
-        first_beg_rel = (int)max(wb, (int64_t)-kFar);
-        rel_end = (int)min((int64_t)ptr[ws + 1] - k0, (int64_t)kFar);
-    }
-
-    int32_t seg_n[U], id_n[U];
-    bool start_n[U];
-    auto classify = [&](int r0) {
+    // finishes segment `seg` whose entries sum to acc: scale, round to the storage type, mask, store
+    auto finish = [&](int32_t seg, float inv, const float (&acc)[CPL][E], const uint4 (&mrow)[CPL]) {
 #pragma unroll
-        for (int u = 0; u < U; ++u) {
-            const int r = r0 + u;
-            start_n[u] = false;
-            seg_n[u] = 0;
-            id_n[u] = 0;
-            if (r < len) {
-                if (seg0) {
-                    const int32_t sg = seg0[r];
-                    start_n[u] = r == 0 || sg != (int32_t)ws;
-                    ws = sg;
-                } else if (r == 0) {
-                    start_n[u] = true;
-                } else if (r >= rel_end) {
-                    const SegStep nx = seg_advance(ptr, n_seg, k0 + r, ws);
-                    ws = nx.seg;
-                    rel_end = (int)min(nx.end - k0, (int64_t)kFar);
-                    start_n[u] = true;
+        for (int q = 0; q < CPL; ++q) {
+            const int ch = c + q * LPR;
+            if (ch < n_chunks) {
+                float r[E];
+#pragma unroll
+                for (int e = 0; e < E; ++e) r[e] = to_float<T>(from_float<T>(acc[q][e] * inv));   // inv = 1 without mean / scale
+                if (kExtra && o.mask) {
+                    float m[E];
+                    Chunk<T>::unpack(mrow[q], m);
+#pragma unroll
+                    for (int e = 0; e < E; ++e)
+                        if (!(m[e] > 0.f)) r[e] = 0.f;
                 }
-                seg_n[u] = (int32_t)ws;
-                id_n[u] = idx0[r];
+                Chunk<T>::store(o.out + (int64_t)seg * o.ld_out + ch * E, r);
             }
         }
     };
 
-    int32_t cur_seg = -1;
-    int cur_beg_rel = 0;
-    bool cur_begins = false;
-    uint4 cur_mask[CPL];
-    float acc[CPL][E];
-#pragma unroll
-    for (int q = 0; q < CPL; ++q) {
-        cur_mask[q] = make_uint4(0, 0, 0, 0);
-#pragma unroll
-        for (int e = 0; e < E; ++e) acc[q][e] = 0.f;
-    }
-    int32_t head_seg = -1, head_ends = 0, tail_seg = -1;
+    if (run < cap_runs && k0 < total) {
+        const int len = (int)min((int64_t)run_len, total - k0);   // entries of this run; positions below are relative to k0
+        const int32_t *__restrict__ idx0 = idx + k0;
+        const int32_t *__restrict__ seg0 = seg_of ? seg_of + k0 : nullptr;
+        const int64_t n_self = (kExtra && o.self) ? (o.n_self ? (int64_t)*o.n_self : n_seg) : 0;
 
-    // closes the current segment, which ends at relative position end_rel, with the sum in acc
-    auto emit = [&](bool ended, int end_rel) {
-        if (cur_begins && ended) {
-            const float inv = o.mean ? 1.0f / (float)(end_rel - cur_beg_rel) : (o.seg_scale ? o.seg_scale[cur_seg] : 1.0f);
+        // Segment boundaries are found one iteration ahead of the sums.  With an entry -> segment array a
+        // boundary is a change of that value; without it the offsets are walked.
+        int64_t ws;                    // segment of the entry classified last
+        int rel_end = kFar;            // its end (walk mode)
+        int first_beg_rel = 0;         // where the run's first segment begins (<= 0)
+        bool first_begins, last_ends = false;
+        if (seg0) {
+            ws = seg0[0];
+            first_begins = k0 == 0 || seg0[-1] != (int32_t)ws;
+            last_ends = k0 + len == total || seg0[len] != seg0[len - 1];
+            if (o.mean) first_beg_rel = (int)max((int64_t)ptr[ws] - k0, (int64_t)-kFar);
+        } else {
+            ws = seg_containing(ptr, n_seg, k0);
+            const int64_t wb = (int64_t)ptr[ws] - k0;
+            first_begins = wb >= 0;
+            first_beg_rel = (int)max(wb, (int64_t)-kFar);
+            rel_end = (int)min((int64_t)ptr[ws + 1] - k0, (int64_t)kFar);
+        }
+
+        int32_t seg_n[U], id_n[U];
+        bool start_n[U];
+        auto classify = [&](int r0) {
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                const int r = r0 + u;
+                start_n[u] = false;
+                seg_n[u] = 0;
+                id_n[u] = 0;
+                if (r < len) {
+                    if (seg0) {
+                        const int32_t sg = seg0[r];
+                        start_n[u] = r == 0 || sg != (int32_t)ws;
+                        ws = sg;
+                    } else if (r == 0) {
+                        start_n[u] = true;
+                    } else if (r >= rel_end) {
+                        const SegStep nx = seg_advance(ptr, n_seg, k0 + r, ws);
+                        ws = nx.seg;
+                        rel_end = (int)min(nx.end - k0, (int64_t)kFar);
+                        start_n[u] = true;
+                    }
+                    seg_n[u] = (int32_t)ws;
+                    id_n[u] = idx0[r];
+                }
+            }
+        };
+
+        int32_t cur_seg = -1;
+        int cur_beg_rel = 0;
+        bool cur_begins = false;
+        uint4 cur_mask[CPL];
+        float acc[CPL][E];
+#pragma unroll
+        for (int q = 0; q < CPL; ++q) {
+            cur_mask[q] = make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int e = 0; e < E; ++e) acc[q][e] = 0.f;
+        }
+
+        // closes the current segment, which ends at relative position end_rel, with the sum in acc
+        auto emit = [&](bool ended, int end_rel) {
+            if (cur_begins && ended) {
+                const float inv = o.mean ? 1.0f / (float)(end_rel - cur_beg_rel) : (o.seg_scale ? o.seg_scale[cur_seg] : 1.0f);
+                finish(cur_seg, inv, acc, cur_mask);
+            } else {
+                float *dst = (cur_begins ? sh_tail : sh_head) + rl * ROW;
+#pragma unroll
+                for (int q = 0; q < CPL; ++q) {
+                    const int ch = c + q * LPR;
+#pragma unroll
+                    for (int e = 0; e < E; e += 4)
+                        *reinterpret_cast<float4 *>(dst + ch * E + e) = make_float4(acc[q][e], acc[q][e + 1], acc[q][e + 2], acc[q][e + 3]);
+                }
+                if (cur_begins) tail_seg = cur_seg;
+                else { head_seg = cur_seg; head_ends = ended ? 1 : 0; }
+            }
+        };
+
+        classify(0);
+        for (int r0 = 0; r0 < len; r0 += U) {
+            int32_t seg_c[U];
+            bool start_c[U];
+            float wt[U];
+            uint4 v[U][CPL], sv[kExtra ? U : 1][CPL], mv[kExtra ? U : 1][CPL];
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                seg_c[u] = seg_n[u];
+                start_c[u] = start_n[u];
+                wt[u] = 1.f;
+                const bool live = r0 + u < len;
+                const int32_t id = id_n[u];
+                if (kWeight && live) wt[u] = w[id];
+#pragma unroll
+                for (int q = 0; q < CPL; ++q) {
+                    const int ch = c + q * LPR;
+                    v[u][q] = make_uint4(0, 0, 0, 0);
+                    if (live && ch < n_chunks) v[u][q] = Chunk<T>::load_raw(in + (int64_t)id * ld_in + ch * E);
+                    if (kExtra) {
+                        sv[u][q] = make_uint4(0, 0, 0, 0);
+                        mv[u][q] = make_uint4(0, 0, 0, 0);
+                        if (live && start_c[u] && ch < n_chunks) {
+                            const bool begins = r0 + u != 0 || first_begins;
+                            if (begins && seg_c[u] < n_self)
+                                sv[u][q] = Chunk<T>::load_raw(o.self + (int64_t)seg_c[u] * o.ld_self + ch * E);
+                            if (o.mask) mv[u][q] = Chunk<T>::load_raw(o.mask + (int64_t)seg_c[u] * o.ld_mask + ch * E);
+                        }
+                    }
+                }
+            }
+            if (r0 + U < len) classify(r0 + U);
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                if (r0 + u < len) {
+                    if (start_c[u]) {
+                        if (cur_seg >= 0) emit(true, r0 + u);
+                        cur_seg = seg_c[u];
+                        cur_begins = r0 + u != 0 || first_begins;
+                        cur_beg_rel = r0 + u != 0 ? r0 + u : first_beg_rel;
+#pragma unroll
+                        for (int q = 0; q < CPL; ++q) {
+                            if (kExtra) {
+                                Chunk<T>::unpack(sv[u][q], acc[q]);          // the self row (zeros if there is none)
+                                cur_mask[q] = mv[u][q];
+                            } else {
+#pragma unroll
+                                for (int e = 0; e < E; ++e) acc[q][e] = 0.f;
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int q = 0; q < CPL; ++q) {
+                        float x[E];
+                        Chunk<T>::unpack(v[u][q], x);
+#pragma unroll
+                        for (int e = 0; e < E; ++e) {
+                            if (kWeight) acc[q][e] = fmaf(wt[u], x[e], acc[q][e]);
+                            else acc[q][e] += x[e];
+                        }
+                    }
+                }
+            }
+        }
+        emit(seg0 ? last_ends : rel_end <= len, len);
+    }
+    if (c == 0) sh_info[rl] = make_int4(head_seg, head_ends, tail_seg, 0);
+    if (threadIdx.x < 4) sh_win[threadIdx.x] = threadIdx.x == 1 || threadIdx.x == 3 ? 0 : -1;
+    __syncthreads();
+
+    // ---- join the runs of the window.  The group of run rl acts where a chain of parts of one cut segment
+    // ends: at the run that holds the segment's end, or at the window's last run.  It walks back to the run in
+    // which the segment began (if that run is in the window) and adds the parts forward, in run order.
+    {
+        const bool last_run = rl == RB - 1;
+        if (head_seg >= 0 && (head_ends || last_run)) {
+            int first = rl - 1;                    // the run whose tail begins the chain, or -1: began before the window
+            while (first >= 0 && sh_info[first].z != head_seg) --first;
+            float acc[CPL][E];
+            uint4 mrow[CPL];
+#pragma unroll
+            for (int q = 0; q < CPL; ++q) {
+                const int ch = c + q * LPR;
+                mrow[q] = make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int e = 0; e < E; ++e) acc[q][e] = 0.f;
+                if (first >= 0) {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) acc[q][e] = sh_tail[first * ROW + ch * E + e];
+                }
+                for (int j = first + 1; j <= rl; ++j) {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) acc[q][e] += sh_head[j * ROW + ch * E + e];
+                }
+            }
+            if (first >= 0 && head_ends) {
+                const int64_t sg = head_seg;
+                float inv = 1.0f;
+                if (o.mean) inv = 1.0f / (float)((int64_t)ptr[sg + 1] - (int64_t)ptr[sg]);
+                else if (o.seg_scale) inv = o.seg_scale[sg];
+                if (kExtra && o.mask) {
+#pragma unroll
+                    for (int q = 0; q < CPL; ++q) {
+                        const int ch = c + q * LPR;
+                        if (ch < n_chunks) mrow[q] = Chunk<T>::load_raw(o.mask + sg * o.ld_mask + ch * E);
+                    }
+                }
+                finish(head_seg, inv, acc, mrow);
+            } else {
+                // leaves the window: towards earlier windows (head2) or, begun here and still open, later ones (tail2)
+                float *dst = (first >= 0 ? tail2 : head2) + (int64_t)blockIdx.x * d;
+#pragma unroll
+                for (int q = 0; q < CPL; ++q) {
+                    const int ch = c + q * LPR;
+                    if (ch < n_chunks) {
+#pragma unroll
+                        for (int e = 0; e < E; e += 4)
+                            *reinterpret_cast<float4 *>(dst + ch * E + e) = make_float4(acc[q][e], acc[q][e + 1], acc[q][e + 2], acc[q][e + 3]);
+                    }
+                }
+                if (c == 0) {
+                    if (first >= 0) sh_win[2] = head_seg;
+                    else { sh_win[0] = head_seg; sh_win[1] = head_ends; }
+                }
+            }
+        }
+        if (last_run && tail_seg >= 0) {           // a segment that begins in the window's last run and continues
+            float *dst = tail2 + (int64_t)blockIdx.x * d;
 #pragma unroll
             for (int q = 0; q < CPL; ++q) {
                 const int ch = c + q * LPR;
                 if (ch < n_chunks) {
-                    float r[E];
 #pragma unroll
-                    for (int e = 0; e < E; ++e) r[e] = to_float<T>(from_float<T>(acc[q][e] * inv));   // inv = 1 without mean / scale
-                    if (kExtra && o.mask) {
-                        float m[E];
-                        Chunk<T>::unpack(cur_mask[q], m);
-#pragma unroll
-                        for (int e = 0; e < E; ++e)
-                            if (!(m[e] > 0.f)) r[e] = 0.f;
-                    }
-                    Chunk<T>::store(o.out + (int64_t)cur_seg * o.ld_out + ch * E, r);
+                    for (int e = 0; e < E; e += 4)
+                        *reinterpret_cast<float4 *>(dst + ch * E + e) = *reinterpret_cast<const float4 *>(sh_tail + rl * ROW + ch * E + e);
                 }
             }
-        } else {
-            seg_store_partial<CPL, E>((cur_begins ? tail : head) + run * d, acc, c, LPR, n_chunks);
-            if (cur_begins) tail_seg = cur_seg;
-            else { head_seg = cur_seg; head_ends = ended ? 1 : 0; }
-        }
-    };
-
-    classify(0);
-    for (int r0 = 0; r0 < len; r0 += U) {
-        int32_t seg_c[U];
-        bool start_c[U];
-        float wt[U];
-        uint4 v[U][CPL], sv[kExtra ? U : 1][CPL], mv[kExtra ? U : 1][CPL];
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            seg_c[u] = seg_n[u];
-            start_c[u] = start_n[u];
-            wt[u] = 1.f;
-            const bool live = r0 + u < len;
-            const int32_t id = id_n[u];
-            if (kWeight && live) wt[u] = w[id];
-#pragma unroll
-            for (int q = 0; q < CPL; ++q) {
-                const int ch = c + q * LPR;
-                v[u][q] = make_uint4(0, 0, 0, 0);
-                if (live && ch < n_chunks) v[u][q] = Chunk<T>::load_raw(in + (int64_t)id * ld_in + ch * E);
-                if (kExtra) {
-                    sv[u][q] = make_uint4(0, 0, 0, 0);
-                    mv[u][q] = make_uint4(0, 0, 0, 0);
-                    if (live && start_c[u] && ch < n_chunks) {
-                        const bool begins = r0 + u != 0 || first_begins;
-                        if (begins && seg_c[u] < n_self)
-                            sv[u][q] = Chunk<T>::load_raw(o.self + (int64_t)seg_c[u] * o.ld_self + ch * E);
-                        if (o.mask) mv[u][q] = Chunk<T>::load_raw(o.mask + (int64_t)seg_c[u] * o.ld_mask + ch * E);
-                    }
-                }
-            }
-        }
-        if (r0 + U < len) classify(r0 + U);
-#pragma unroll
-        for (int u = 0; u < U; ++u) {
-            if (r0 + u < len) {
-                if (start_c[u]) {
-                    if (cur_seg >= 0) emit(true, r0 + u);
-                    cur_seg = seg_c[u];
-                    cur_begins = r0 + u != 0 || first_begins;
-                    cur_beg_rel = r0 + u != 0 ? r0 + u : first_beg_rel;
-#pragma unroll
-                    for (int q = 0; q < CPL; ++q) {
-                        if (kExtra) {
-                            Chunk<T>::unpack(sv[u][q], acc[q]);          // the self row (zeros if there is none)
-                            cur_mask[q] = mv[u][q];
-                        } else {
-#pragma unroll
-                            for (int e = 0; e < E; ++e) acc[q][e] = 0.f;
-                        }
-                    }
-                }
-#pragma unroll
-                for (int q = 0; q < CPL; ++q) {
-                    float x[E];
-                    Chunk<T>::unpack(v[u][q], x);
-#pragma unroll
-                    for (int e = 0; e < E; ++e) {
-                        if (kWeight) acc[q][e] = fmaf(wt[u], x[e], acc[q][e]);
-                        else acc[q][e] += x[e];
-                    }
-                }
-            }
+            if (c == 0) sh_win[2] = tail_seg;
         }
     }
-    emit(seg0 ? last_ends : rel_end <= len, len);
-    if (c == 0) run_info[run] = make_int4(head_seg, head_ends, tail_seg, 0);
+    __syncthreads();
+    if (threadIdx.x == 0) win_info[blockIdx.x] = make_int4(sh_win[0], sh_win[1], sh_win[2], 0);
 }
 
-// ------------------------------------------------------------------------------------ level 2
+// ------------------------------------------------------------------------------------ across windows
+constexpr int kFinalWindows = 64;       // windows per block of seg_final_kernel
+constexpr int kFinalWarpParts = 64;     // longest chain of window parts that one warp adds by itself
 template <typename T, typename PtrT>
 __global__ void __launch_bounds__(kAggThreads)
-seg_window_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_t n_seg_host, int d,
-                  const float *__restrict__ head, const float *__restrict__ tail, const int4 *__restrict__ run_info,
-                  float *__restrict__ head2, float *__restrict__ tail2, int4 *__restrict__ win_info,
-                  int64_t cap_runs, int64_t n_windows, SegOut<T> o)
+seg_final_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_t n_seg_host, int run_len, int runs_per_window,
+                 int d, const float *__restrict__ head2, const float *__restrict__ tail2, const int4 *__restrict__ win_info,
+                 int64_t n_windows, int64_t n_window_blocks, SegOut<T> o)
 {
-    constexpr int kB = 8;                         // runs fetched together
-    const int lane = threadIdx.x & 31;
-    const int64_t win = ((int64_t)blockIdx.x * kAggThreads + threadIdx.x) >> 5;
-    if (win >= n_windows) return;
-    const int64_t r0 = win * kSegWindow;
-    int4 info = make_int4(-1, 0, -1, 0);
-    if (r0 + lane < cap_runs) info = run_info[r0 + lane];
-    const unsigned any = __ballot_sync(0xffffffffu, info.x >= 0 || info.z >= 0);
-    int32_t w_head = -1, w_head_ends = 0, w_tail = -1;
-    if (any) {
-        const int n_vec = d / 4;
-        for (int vb = 0; vb < n_vec; vb += 32) {
-            const int q = vb + lane;
-            const bool act = q < n_vec;
-            int32_t cur = -1;
-            bool from_tail = false;
-            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            w_head = -1; w_head_ends = 0; w_tail = -1;
-            for (int rb = 0; rb < kSegWindow; rb += kB) {
-                // fetch the records of kB runs (and the mask rows of segments that end in them), then walk them in order
-                float4 hv[kB], tv[kB], mk[kB];
-                int32_t hs[kB], he[kB], ts[kB];
-#pragma unroll
-                for (int j = 0; j < kB; ++j) {
-                    hs[j] = __shfl_sync(0xffffffffu, info.x, rb + j);
-                    he[j] = __shfl_sync(0xffffffffu, info.y, rb + j);
-                    ts[j] = __shfl_sync(0xffffffffu, info.z, rb + j);
-                    hv[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    tv[j] = hv[j];
-                    mk[j] = make_float4(1.f, 1.f, 1.f, 1.f);
-                    if (act && hs[j] >= 0) hv[j] = *reinterpret_cast<const float4 *>(head + (r0 + rb + j) * d + q * 4);
-                    if (act && ts[j] >= 0) tv[j] = *reinterpret_cast<const float4 *>(tail + (r0 + rb + j) * d + q * 4);
-                    if (act && hs[j] >= 0 && he[j] && o.mask) mk[j] = load4<T>(o.mask + (int64_t)hs[j] * o.ld_mask + q * 4);
-                }
-#pragma unroll
-                for (int j = 0; j < kB; ++j) {
-                    if (hs[j] >= 0) {
-                        if (cur != hs[j]) { cur = hs[j]; from_tail = false; acc = make_float4(0.f, 0.f, 0.f, 0.f); }
-                        acc.x += hv[j].x; acc.y += hv[j].y; acc.z += hv[j].z; acc.w += hv[j].w;
-                        if (he[j]) {
-                            if (from_tail) {
-                                if (act) {
-                                    const int64_t s = cur;
-                                    float inv = 0.f;
-                                    if (o.mean) inv = 1.0f / (float)((int64_t)ptr[s + 1] - (int64_t)ptr[s]);
-                                    else if (o.seg_scale) inv = o.seg_scale[s];
-                                    const float m[4] = {mk[j].x, mk[j].y, mk[j].z, mk[j].w};
-                                    float r[4] = {acc.x, acc.y, acc.z, acc.w};
-#pragma unroll
-                                    for (int e = 0; e < 4; ++e) {
-                                        r[e] = seg_round(o, inv, r[e]);
-                                        if (!(m[e] > 0.f)) r[e] = 0.f;
-                                    }
-                                    store4<T>(o.out + s * o.ld_out + q * 4, r);
-                                }
-                            } else {
-                                if (act) *reinterpret_cast<float4 *>(head2 + win * d + q * 4) = acc;
-                                w_head = cur; w_head_ends = 1;
-                            }
-                            cur = -1;
-                        }
-                    }
-                    if (ts[j] >= 0) { cur = ts[j]; from_tail = true; acc = tv[j]; }
-                }
-            }
-            if (cur >= 0) {
-                if (from_tail) {
-                    if (act) *reinterpret_cast<float4 *>(tail2 + win * d + q * 4) = acc;
-                    w_tail = cur;
-                } else {
-                    if (act) *reinterpret_cast<float4 *>(head2 + win * d + q * 4) = acc;
-                    w_head = cur; w_head_ends = 0;
-                }
-            }
-        }
-    }
-    if (lane == 0) win_info[win] = make_int4(w_head, w_head_ends, w_tail, 0);
-}
-
-// ------------------------------------------------------------------------------------ level 3
-template <typename T, typename PtrT>
-__global__ void __launch_bounds__(kAggThreads)
-seg_final_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_t n_seg_host, int run_len, int d,
-                 const float *__restrict__ head2, const float *__restrict__ tail2, const int4 *__restrict__ win_info,
-                 int64_t n_windows, SegOut<T> o)
-{
-    constexpr int W = kAggThreads / 32;
-    __shared__ float4 red[W][32];
+    __shared__ float4 red[kAggThreads];
+    __shared__ int32_t sh_seg[kFinalWindows];
+    __shared__ int sh_long[kFinalWindows];
+    __shared__ int sh_n_long;
     const int64_t n_seg = n_seg_dev ? (int64_t)*n_seg_dev : n_seg_host;
     if (n_seg < 0) return;
     const int64_t n_self = o.self ? (o.n_self ? (int64_t)*o.n_self : n_seg) : 0;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 
-    if ((int64_t)blockIdx.x >= n_windows) {
-        // segments without entries: 8 lanes per segment, the extra blocks stride over all segments
-        const int64_t n_extra = (int64_t)gridDim.x - n_windows;
-        for (int64_t s = ((int64_t)(blockIdx.x - n_windows) * kAggThreads + threadIdx.x) >> 3; s < n_seg;
-             s += n_extra * (kAggThreads / 8)) {
-            if (ptr[s + 1] != ptr[s]) continue;
-            for (int k = threadIdx.x & 7; k < d; k += 8)
-                o.out[s * o.ld_out + k] = from_float<T>(seg_finish_value(o, s, 0, k, 0.f, s < n_self));
+    if ((int64_t)blockIdx.x >= n_window_blocks) {
+        // segments without entries, the extra blocks stride over all segments
+        const int64_t n_extra = (int64_t)gridDim.x - n_window_blocks;
+        const int64_t b = (int64_t)blockIdx.x - n_window_blocks;
+        if (!o.self && (d * (int)sizeof(T)) % 16 == 0 && o.ld_out * (int64_t)sizeof(T) % 16 == 0 &&
+            reinterpret_cast<uintptr_t>(o.out) % 16 == 0) {
+            // fin(0) = 0: one thread per segment, whole row in 16-byte stores
+            const int n16 = d * (int)sizeof(T) / 16;
+            for (int64_t s = b * kAggThreads + threadIdx.x; s < n_seg; s += n_extra * kAggThreads) {
+                if (ptr[s + 1] != ptr[s]) continue;
+                uint4 *row = reinterpret_cast<uint4 *>(o.out + s * o.ld_out);
+                for (int q = 0; q < n16; ++q) row[q] = make_uint4(0, 0, 0, 0);
+            }
+        } else {
+            for (int64_t s = (b * kAggThreads + threadIdx.x) >> 3; s < n_seg; s += n_extra * (kAggThreads / 8)) {
+                if (ptr[s + 1] != ptr[s]) continue;
+                for (int k = threadIdx.x & 7; k < d; k += 8)
+                    o.out[s * o.ld_out + k] = from_float<T>(seg_finish_value(o, s, 0, k, 0.f, s < n_self));
+            }
         }
         if (o.pad_rows > 0) {                           // zero rows up to the next multiple of 128
             const int64_t pad_end = min((n_seg + 127) / 128 * 128, o.pad_rows);
             const int64_t cells = (pad_end - n_seg) * d;
-            for (int64_t t = (int64_t)(blockIdx.x - n_windows) * kAggThreads + threadIdx.x; t < cells;
-                 t += n_extra * kAggThreads)
+            for (int64_t t = b * kAggThreads + threadIdx.x; t < cells; t += n_extra * kAggThreads)
                 o.out[(n_seg + t / d) * o.ld_out + t % d] = from_float<T>(0.f);
         }
         return;
     }
     if (n_seg == 0) return;
-    const int64_t win = blockIdx.x;
-    const int4 info = win_info[win];
-    if (info.x < 0 || !info.y) return;                   // no segment that began earlier ends in this window
-    const int64_t s = info.x;
-    const int64_t seg_beg = (int64_t)ptr[s], seg_end = (int64_t)ptr[s + 1];
-    const int64_t first = (seg_beg / run_len) / kSegWindow;      // its first part is tail2[first]
-    const int64_t n_parts = win - first + 1;
-    const int n_vec = d / 4;
-    for (int vb = 0; vb < n_vec; vb += 32) {
-        const int q = vb + lane;
-        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (q < n_vec) {
-            for (int64_t p0 = warp * 4; p0 < n_parts; p0 += W * 4) {
+
+    // kFinalWindows windows per block.  A chain of up to kFinalWarpParts parts is added by one warp (the warps of
+    // the block work on different windows at the same time); a longer one is left to the whole block.
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t win0 = (int64_t)blockIdx.x * kFinalWindows;
+    if (threadIdx.x < kFinalWindows) {
+        int32_t sg = -1;
+        const int64_t wi = win0 + threadIdx.x;
+        if (wi < n_windows) {
+            const int4 info = win_info[wi];
+            if (info.x >= 0 && info.y) sg = info.x;         // a segment that began in an earlier window ends here
+        }
+        sh_seg[threadIdx.x] = sg;
+    }
+    if (threadIdx.x == 0) sh_n_long = 0;
+    __syncthreads();
+    const int n_vec = d / 4;                                // float4 columns (<= kAggThreads since d <= 1024)
+    for (int j = warp; j < kFinalWindows; j += kAggThreads / 32) {
+        const int32_t sg = sh_seg[j];
+        if (sg < 0) continue;                               // uniform over the warp
+        const int64_t win = win0 + j;
+        const int64_t seg_beg = (int64_t)ptr[sg], seg_end = (int64_t)ptr[sg + 1];
+        const int64_t first = (seg_beg / run_len) / runs_per_window;     // its first part is tail2[first]
+        const int64_t n_parts = win - first + 1;
+        if (n_parts > kFinalWarpParts) {
+            if (lane == 0) sh_long[atomicAdd(&sh_n_long, 1)] = j;
+            continue;
+        }
+        for (int vb = 0; vb < n_vec; vb += 32) {
+            const int q = vb + lane;
+            if (q >= n_vec) continue;
+            float4 a = *reinterpret_cast<const float4 *>(tail2 + first * d + q * 4);
+            for (int64_t p0 = 1; p0 < n_parts; p0 += 4) {
                 float4 x[4];
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const int64_t p = p0 + j;
-                    x[j] = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (p < n_parts)
-                        x[j] = *reinterpret_cast<const float4 *>((p == 0 ? tail2 + first * d : head2 + (first + p) * d) + q * 4);
+                for (int t = 0; t < 4; ++t) {
+                    x[t] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (p0 + t < n_parts) x[t] = *reinterpret_cast<const float4 *>(head2 + (first + p0 + t) * d + q * 4);
                 }
 #pragma unroll
-                for (int j = 0; j < 4; ++j) { a.x += x[j].x; a.y += x[j].y; a.z += x[j].z; a.w += x[j].w; }
+                for (int t = 0; t < 4; ++t) { a.x += x[t].x; a.y += x[t].y; a.z += x[t].z; a.w += x[t].w; }
+            }
+            const float r[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+            for (int kk = 0; kk < 4; ++kk)
+                o.out[(int64_t)sg * o.ld_out + q * 4 + kk] =
+                    from_float<T>(seg_finish_value(o, sg, seg_end - seg_beg, q * 4 + kk, r[kk], false));
+        }
+    }
+    __syncthreads();
+    const int n_long = sh_n_long;
+    const int q = threadIdx.x % n_vec, pl = threadIdx.x / n_vec;
+    const int n_pl = kAggThreads / n_vec;                   // part lanes; threads with pl >= n_pl idle
+    for (int i = 0; i < n_long; ++i) {
+        const int j = sh_long[i];
+        const int32_t sg = sh_seg[j];
+        const int64_t win = win0 + j;
+        const int64_t seg_beg = (int64_t)ptr[sg], seg_end = (int64_t)ptr[sg + 1];
+        const int64_t first = (seg_beg / run_len) / runs_per_window;
+        const int64_t n_parts = win - first + 1;
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (pl < n_pl) {
+            for (int64_t p0 = pl; p0 < n_parts; p0 += (int64_t)n_pl * 8) {
+                float4 x[8];
+#pragma unroll
+                for (int t = 0; t < 8; ++t) {
+                    const int64_t p = p0 + (int64_t)t * n_pl;
+                    x[t] = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (p < n_parts)
+                        x[t] = *reinterpret_cast<const float4 *>((p == 0 ? tail2 + first * d : head2 + (first + p) * d) + q * 4);
+                }
+#pragma unroll
+                for (int t = 0; t < 8; ++t) { a.x += x[t].x; a.y += x[t].y; a.z += x[t].z; a.w += x[t].w; }
             }
         }
-        red[warp][lane] = a;
+        red[threadIdx.x] = a;
         __syncthreads();
-        if (warp == 0 && q < n_vec) {
-            float4 t = red[0][lane];
-#pragma unroll
-            for (int w2 = 1; w2 < W; ++w2) {
-                const float4 x = red[w2][lane];
+        if (pl == 0) {
+            float4 t = red[q];
+            for (int w2 = 1; w2 < n_pl; ++w2) {
+                const float4 x = red[w2 * n_vec + q];
                 t.x += x.x; t.y += x.y; t.z += x.z; t.w += x.w;
             }
             const float r[4] = {t.x, t.y, t.z, t.w};
 #pragma unroll
             for (int kk = 0; kk < 4; ++kk)
-                o.out[s * o.ld_out + q * 4 + kk] =
-                    from_float<T>(seg_finish_value(o, s, seg_end - seg_beg, q * 4 + kk, r[kk], false));
+                o.out[(int64_t)sg * o.ld_out + q * 4 + kk] =
+                    from_float<T>(seg_finish_value(o, sg, seg_end - seg_beg, q * 4 + kk, r[kk], false));
         }
         __syncthreads();
     }
@@ -475,27 +535,29 @@ inline void launch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const
                               int64_t n_seg_host, int64_t cap_seg, const float *w, int run_len, int d,
                               const int32_t *seg_of, const SegScratch &sc, const SegOut<T> &o, cudaStream_t st)
 {
+    constexpr size_t smem = seg_run_smem_bytes<LPR, CPL, Chunk<T>::kElems>();
     tap_begin(TAP_SEG_L1, st);
     note_launch();
-    const unsigned grid1 = (unsigned)ceil_div(sc.cap_runs * LPR, kAggThreads);
-    if (o.self || o.mask)
-        seg_run_kernel<T, PtrT, LPR, CPL, kWeight, true><<<grid1, kAggThreads, 0, st>>>(
-            in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head, sc.tail, sc.run_info, sc.cap_runs, seg_of, o);
-    else
-        seg_run_kernel<T, PtrT, LPR, CPL, kWeight, false><<<grid1, kAggThreads, 0, st>>>(
-            in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head, sc.tail, sc.run_info, sc.cap_runs, seg_of, o);
+    const unsigned grid1 = (unsigned)sc.n_windows;
+    if (o.self || o.mask) {
+        auto kern = seg_run_kernel<T, PtrT, LPR, CPL, kWeight, true>;
+        if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        kern<<<grid1, kAggThreads, smem, st>>>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head2, sc.tail2,
+                                               sc.win_info, sc.cap_runs, seg_of, o);
+    } else {
+        auto kern = seg_run_kernel<T, PtrT, LPR, CPL, kWeight, false>;
+        if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        kern<<<grid1, kAggThreads, smem, st>>>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head2, sc.tail2,
+                                               sc.win_info, sc.cap_runs, seg_of, o);
+    }
     tap_end(TAP_SEG_L1, st);
-    tap_begin(TAP_SEG_L2, st);
-    note_launch();
-    seg_window_kernel<T, PtrT><<<(unsigned)ceil_div(sc.n_windows * 32, kAggThreads), kAggThreads, 0, st>>>(
-        ptr, n_seg_dev, n_seg_host, d, sc.head, sc.tail, sc.run_info, sc.head2, sc.tail2, sc.win_info, sc.cap_runs,
-        sc.n_windows, o);
-    tap_end(TAP_SEG_L2, st);
-    const int64_t empty_blocks = std::min<int64_t>(ceil_div((cap_seg > 0 ? cap_seg : 1) * 8, kAggThreads), 148 * 8);
+    const int64_t window_blocks = ceil_div(sc.n_windows, kFinalWindows);
+    const int64_t empty_blocks = std::min<int64_t>(ceil_div(cap_seg > 0 ? cap_seg : 1, kAggThreads), 148 * 8);
     tap_begin(TAP_SEG_L3, st);
     note_launch();
-    seg_final_kernel<T, PtrT><<<(unsigned)(sc.n_windows + empty_blocks), kAggThreads, 0, st>>>(
-        ptr, n_seg_dev, n_seg_host, run_len, d, sc.head2, sc.tail2, sc.win_info, sc.n_windows, o);
+    seg_final_kernel<T, PtrT><<<(unsigned)(window_blocks + empty_blocks), kAggThreads, 0, st>>>(
+        ptr, n_seg_dev, n_seg_host, run_len, sc.runs_per_window, d, sc.head2, sc.tail2, sc.win_info, sc.n_windows,
+        window_blocks, o);
     tap_end(TAP_SEG_L3, st);
 }
 
