@@ -26,7 +26,7 @@ static void dispatch_seg64(const T *in, int64_t ld_in, const int64_t *ptr, const
 {
     const int run_len = full_run_len(n_entries);
     const SegScratch sc = seg_scratch_carve(n_entries, run_len, d, dtype_size(dtype), ws);
-    dispatch_seg_reduce<T, int64_t, kWeight>(in, ld_in, ptr, idx, nullptr, n_seg, n_seg, w, run_len, d, dtype, nullptr, sc, o, st);
+    dispatch_seg_reduce<T, int64_t, kWeight, 2>(in, ld_in, ptr, idx, nullptr, n_seg, n_seg, w, run_len, d, dtype, nullptr, sc, o, st);
 }
 
 static int32_t check_mats(const e2egrec_mat *in, const e2egrec_mat *out, int64_t out_rows)

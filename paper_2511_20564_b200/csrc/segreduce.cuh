@@ -114,15 +114,18 @@ constexpr size_t seg_run_smem_bytes()
 
 // kExtra: the output has a self row and/or a mask row per segment (they are fetched together with the
 // segment's first gathered row); without it those registers and branches disappear.
-template <typename T, typename PtrT, int LPR, int CPL, bool kWeight, bool kExtra>
-__global__ void __launch_bounds__(kAggThreads)
+// kInFlight: gathered rows a lane group requests before it adds any.  Four suit the short streams of a sampled
+// block (few resident warps, latency hidden inside the thread); on streams that fill the machine two are faster,
+// because the smaller register footprint keeps five blocks resident per SM instead of three.
+template <typename T, typename PtrT, int LPR, int CPL, bool kWeight, bool kExtra, int kInFlight>
+__global__ void __launch_bounds__(kAggThreads, (kInFlight <= 2 && !kExtra) ? 5 : 1)
 seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__ ptr, const int32_t *__restrict__ idx,
                const int32_t *n_seg_dev, int64_t n_seg_host, const float *__restrict__ w, int run_len, int d,
                float *__restrict__ head2, float *__restrict__ tail2, int4 *__restrict__ win_info, int64_t cap_runs,
                const int32_t *__restrict__ seg_of, SegOut<T> o)
 {
     constexpr int E = Chunk<T>::kElems;
-    constexpr int U = CPL >= 4 ? 1 : 4 / CPL;
+    constexpr int U = CPL >= kInFlight ? 1 : kInFlight / CPL;
     constexpr int RB = kAggThreads / LPR;          // runs of this block = one window
     constexpr int ROW = LPR * CPL * E;             // floats per shared row (>= d)
     constexpr int kFar = 1 << 30;
@@ -530,7 +533,7 @@ seg_final_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_t
 }
 
 // ------------------------------------------------------------------------------------ host
-template <typename T, typename PtrT, int LPR, int CPL, bool kWeight>
+template <typename T, typename PtrT, int LPR, int CPL, bool kWeight, int kInFlight>
 inline void launch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const int32_t *idx, const int32_t *n_seg_dev,
                               int64_t n_seg_host, int64_t cap_seg, const float *w, int run_len, int d,
                               const int32_t *seg_of, const SegScratch &sc, const SegOut<T> &o, cudaStream_t st)
@@ -540,12 +543,12 @@ inline void launch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const
     note_launch();
     const unsigned grid1 = (unsigned)sc.n_windows;
     if (o.self || o.mask) {
-        auto kern = seg_run_kernel<T, PtrT, LPR, CPL, kWeight, true>;
+        auto kern = seg_run_kernel<T, PtrT, LPR, CPL, kWeight, true, kInFlight>;
         if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         kern<<<grid1, kAggThreads, smem, st>>>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head2, sc.tail2,
                                                sc.win_info, sc.cap_runs, seg_of, o);
     } else {
-        auto kern = seg_run_kernel<T, PtrT, LPR, CPL, kWeight, false>;
+        auto kern = seg_run_kernel<T, PtrT, LPR, CPL, kWeight, false, kInFlight>;
         if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         kern<<<grid1, kAggThreads, smem, st>>>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head2, sc.tail2,
                                                sc.win_info, sc.cap_runs, seg_of, o);
@@ -561,7 +564,7 @@ inline void launch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const
     tap_end(TAP_SEG_L3, st);
 }
 
-template <typename T, typename PtrT, bool kWeight>
+template <typename T, typename PtrT, bool kWeight, int kInFlight = 4>
 inline void dispatch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const int32_t *idx, const int32_t *n_seg_dev,
                                 int64_t n_seg_host, int64_t cap_seg, const float *w, int run_len, int d, int32_t dtype,
                                 const int32_t *seg_of, const SegScratch &sc, const SegOut<T> &o, cudaStream_t st)
@@ -569,7 +572,7 @@ inline void dispatch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, con
     const RowShape rs = row_shape(d, dtype);
 #define E2E_CASE(L, C)                                                                                                \
     if (rs.lpr == L && rs.cpl == C)                                                                                   \
-        return launch_seg_reduce<T, PtrT, L, C, kWeight>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, cap_seg, w, run_len, \
+        return launch_seg_reduce<T, PtrT, L, C, kWeight, kInFlight>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, cap_seg, w, run_len, \
                                                          d, seg_of, sc, o, st);
     E2E_CASE(4, 1) E2E_CASE(8, 1) E2E_CASE(16, 1) E2E_CASE(32, 1) E2E_CASE(32, 2) E2E_CASE(32, 4)
 #undef E2E_CASE
