@@ -305,9 +305,13 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
                         float x[E];
                         Chunk<T>::unpack(v[u][q], x);
 #pragma unroll
-                        for (int e = 0; e < E; ++e) {
-                            if (kWeight) acc[q][e] = fmaf(wt[u], x[e], acc[q][e]);
-                            else acc[q][e] += x[e];
+                        for (int e = 0; e < E; e += 2) {
+                            if (kWeight) {
+                                acc[q][e] = fmaf(wt[u], x[e], acc[q][e]);
+                                acc[q][e + 1] = fmaf(wt[u], x[e + 1], acc[q][e + 1]);
+                            } else {
+                                add2(acc[q][e], acc[q][e + 1], x[e], x[e + 1]);
+                            }
                         }
                     }
                 }
