@@ -128,10 +128,14 @@ def upstream_grad(w, rows):
 
 # ------------------------------------------------------------------------------------------ reference arm
 def oracle_step(w, indptr, indices, X, Ws, seeds, step, dH):
+    """One oracle step.  X is the host feature table, or a callable ids -> rows (table kept elsewhere)."""
     import oracle
     bf16 = w.dtype == "bf16"
     blocks = oracle.sample_khop(indptr, indices, seeds, w.fanouts, w.seed, step)
-    out, ctx = oracle.sage_forward(blocks, X, Ws, bf16=bf16)
+    if callable(X):
+        out, ctx = oracle.sage_forward(blocks, X(blocks[-1]["src_nodes"]), Ws, bf16=bf16, gathered=True)
+    else:
+        out, ctx = oracle.sage_forward(blocks, X, Ws, bf16=bf16)
     oracle.sage_backward(blocks, ctx, Ws, dH[: seeds.size], bf16=bf16)
     return sum(b["n_edges"] for b in blocks)
 
@@ -142,6 +146,13 @@ def run_reference(args, w):
         return
     import oracle
     oracle.build()
+    scale_note = ""
+    if w.n_interactions > 200_000_000:
+        # the full graph is drawn on a GPU; the CPU arm runs the same recipe at 1/100 of the size
+        import dataclasses
+        w = dataclasses.replace(w, n_users=w.n_users // 100, n_items=w.n_items // 100,
+                                n_interactions=w.n_interactions // 100, q=w.q / 100)
+        scale_note = " on a 1/100-scale graph of the same recipe"
     indptr, indices, X, Ws, inter = build_inputs(w)
     sample = args.ref_seeds
     dH = upstream_grad(w, sample).astype(np.float64)
@@ -154,7 +165,7 @@ def run_reference(args, w):
         edges += oracle_step(w, indptr, indices, X, Ws, batches[i], i, dH)
     dt = time.perf_counter() - t0
     val = edges / dt
-    desc = f"first {sample} of the {w.batch} seeds of each step's batch, full sample+forward+backward"
+    desc = f"first {sample} of the {w.batch} seeds of each step's batch, full sample+forward+backward{scale_note}"
     line = dict(impl="reference", metric=METRIC, value=val, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
                 warmup=args.warmup, ms_per_step=dt / args.steps * 1e3, higher_is_better=True, scaling="weak",
                 vs_baseline=None, dtype="f64", data="synthetic",
@@ -183,23 +194,46 @@ def run_ours(args, w):
     E.lib()                                            # fails loudly if the CUDA library is missing
 
     want_cpu = world == 1 and not args.no_cpu_baseline
-    indptr_h, indices_h, X_h, Ws_h, inter = build_inputs(w, host_csr=want_cpu)
     dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    K, Wm = args.steps, args.warmup
+    total = K + Wm
+    first_step = rank * 1_000_000                      # = replicas.first_step_of(rank)
+    on_device = w.n_interactions > 200_000_000         # too large for host-side generation: drawn with torch on the GPU
+    t_setup = time.perf_counter()
+    if on_device:
+        users_d, items_d = S.bipartite_interactions_device(w.n_users, w.n_items, w.n_interactions, w.alpha_user,
+                                                           w.alpha_item, w.seed, w.q, dev)
+        row_d, col_d = torch.cat([users_d, items_d]), torch.cat([items_d, users_d])
+        indptr_h = indices_h = X_h = None
+        Ws_h = S.build_weights(w)
+        inter = None
+    else:
+        indptr_h, indices_h, X_h, Ws_h, inter = build_inputs(w, host_csr=want_cpu)
+        row_d = torch.cat([torch.from_numpy(inter[0]), torch.from_numpy(inter[1])]).to(dev)
+        col_d = torch.cat([torch.from_numpy(inter[1]), torch.from_numpy(inter[0])]).to(dev)
     # graph ingest on the device: both directions of every interaction -> canonical CSR
-    row_d = torch.cat([torch.from_numpy(inter[0]), torch.from_numpy(inter[1])]).to(dev)
-    col_d = torch.cat([torch.from_numpy(inter[1]), torch.from_numpy(inter[0])]).to(dev)
     indptr, indices, ingest_status = E.graph_from_coo(w.n_nodes, row_d, col_d)
     indices = indices.contiguous()
     if int(ingest_status):
         raise RuntimeError("graph ingest: node id out of range")
     del row_d, col_d
-    X = torch.from_numpy(X_h).to(dev, dt)
-    Ws = [torch.from_numpy(W).to(dev, dt) for W in Ws_h]
-    K, Wm = args.steps, args.warmup
-    total = K + Wm
-    first_step = rank * 1_000_000                      # = replicas.first_step_of(rank)
+    torch.cuda.empty_cache()
     # every rank trains on its own batches (data parallel replicas; no exchange on the measured path)
-    seeds_h = make_batches(w, inter, args.seeds, first_step, total)
+    if on_device:
+        if args.seeds == "uniform":
+            seeds_h = np.stack([S.seed_batch(w.n_nodes, w.batch, w.seed, first_step + i) for i in range(total)])
+        else:
+            seeds_h = np.stack([S.seed_batch_from_interactions_device(users_d, items_d, w.batch, w.seed, first_step + i)
+                                for i in range(total)])
+        del users_d, items_d
+        torch.cuda.empty_cache()
+        X = S.normal_features_device(w.n_nodes, w.dim, w.seed, dt, dev)
+    else:
+        seeds_h = make_batches(w, inter, args.seeds, first_step, total)
+        X = torch.from_numpy(X_h).to(dev, dt)
+    Ws = [torch.from_numpy(W).to(dev, dt) for W in Ws_h]
+    torch.cuda.synchronize()
+    setup_s = time.perf_counter() - t_setup
     seeds_pin = torch.from_numpy(seeds_h).pin_memory()
     seeds_dev = seeds_pin.to(dev)
     dH_h = upstream_grad(w, w.batch)
@@ -327,7 +361,7 @@ def run_ours(args, w):
 
     # ---- joint step (sampled encoder + ranking tower + BCE, forward and backward) on the same graph
     joint = None
-    if not args.no_joint:
+    if not args.no_joint and not on_device:
         P, dd = w.batch, 64
         jr = np.random.default_rng(4 + rank)
         picks = jr.integers(0, inter[0].size, (min(K, 200) + Wm, P))
@@ -407,7 +441,8 @@ def run_ours(args, w):
                             parallelism=f"replicas x{world}", launch="one CUDA graph replay per step",
                             l2="inputs larger than L2: feature table + graph = %.0f MB, a new batch every step"
                                % ((X.numel() * es + indices.numel() * 4 + indptr.numel() * 8) / 1e6),
-                            edges_per_step=edges_rank / K),
+                            edges_per_step=edges_rank / K, setup_s=round(setup_s, 1),
+                            generated="on the device (torch)" if on_device else "on the host (numpy)"),
                 clocks=clk,
                 e2e=dict(value=e2e_edges_all / e2e_s, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                          ms_per_step=e2e_s / K * 1e3),
@@ -422,15 +457,31 @@ def run_ours(args, w):
         oracle.build()
         sample = args.ref_seeds
         dH64 = dH_h[:sample].astype(np.float64)
+        note = ""
+        X_src = X_h
+        if on_device:
+            # the oracle samples on a host copy of the device-built CSR and reads the feature rows it needs from the
+            # device table (float64 copies of the whole table would not fit the host)
+            import psutil
+            need = indices.numel() * 4 + indptr.numel() * 8
+            if psutil.virtual_memory().available < need * 1.5:
+                want_cpu = False
+                line["cpu_baseline"] = dict(value=None, unit=UNIT, cores=1, kind="oracle",
+                                            sample=f"skipped: the host copy of the graph ({need / 1e9:.1f} GB) does not fit")
+            else:
+                indptr_h, indices_h = indptr.cpu().numpy(), indices.cpu().numpy()
+                X_src = lambda ids: X[torch.from_numpy(np.ascontiguousarray(ids)).to(dev).long()].float().cpu().numpy()
+                note = "; graph = host copy of the device-built CSR, feature rows fetched from the device table"
+    if want_cpu:
         t0 = time.perf_counter()
         ce, n = 0, 0
         while n < K and time.perf_counter() - t0 < 15.0:
-            ce += oracle_step(w, indptr_h, indices_h, X_h, Ws_h, seeds_h[Wm + n][:sample], Wm + n, dH64)
+            ce += oracle_step(w, indptr_h, indices_h, X_src, Ws_h, seeds_h[Wm + n][:sample], Wm + n, dH64)
             n += 1
         cdt = time.perf_counter() - t0
         line["cpu_baseline"] = dict(value=ce / cdt, unit=UNIT, cores=1, kind="oracle",
                                     sample=f"{n} step(s) on the first {sample} of the {w.batch} seeds of the batch, "
-                                           f"full sample+forward+backward, {cdt:.1f} s")
+                                           f"full sample+forward+backward, {cdt:.1f} s{note}")
     print(json.dumps(line), flush=True)
     if world > 1:
         dist.destroy_process_group()

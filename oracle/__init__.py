@@ -167,16 +167,24 @@ def sage_update(Hself, agg, W, bias, act, bf16=False):
     return Z, Hout
 
 
-def sage_forward(blocks, X, Ws, biases=None, acts=None, bf16=False):
-    """L-layer forward on sampled blocks.  Layer l runs on block L-l; layer 0 reads X rows of F_L."""
+def sage_forward(blocks, X, Ws, biases=None, acts=None, bf16=False, gathered=False):
+    """L-layer forward on sampled blocks.  Layer l runs on block L-l; layer 0 reads X rows of F_L.
+
+    With gathered=True, X already holds those rows (X[i] = features of node F_L[i]); for feature tables
+    whose float64 copy would not fit the host."""
     L = len(Ws)
     acts = [1] * L if acts is None else list(acts)
     biases = [None] * L if biases is None else list(biases)
     X = _f64(X)
     ids = _i32(blocks[L - 1]["src_nodes"])
-    H = np.zeros((ids.size, X.shape[1]), np.float64)
-    lib().oracle_gather_rows(_p(X), C.c_int64(X.shape[1]), _p(ids), C.c_int64(ids.size),
-                             C.c_int32(X.shape[1]), _p(H))
+    if gathered:
+        if X.shape[0] != ids.size:
+            raise ValueError("gathered X must have one row per node of the outermost frontier")
+        H = X.copy()
+    else:
+        H = np.zeros((ids.size, X.shape[1]), np.float64)
+        lib().oracle_gather_rows(_p(X), C.c_int64(X.shape[1]), _p(ids), C.c_int64(ids.size),
+                                 C.c_int32(X.shape[1]), _p(H))
     ctx = dict(H=[H], agg=[], Z=[])
     for l in range(L):
         blk = blocks[L - 1 - l]
@@ -259,12 +267,17 @@ def bce_with_logits(t, y):
 
 # ----------------------------------------------------------------------------- full graph
 
-def full_aggregate_backward(indptr, indices, n_src, G, bf16=False):
+def full_aggregate_backward(indptr, indices, n_src, G, bf16=False, row_len=None):
+    """Adjoint of the whole-graph mean aggregation (Eq. 2 with S(u) = N(u)): dX = A^T D^-1 G.
+
+    row_len: sizes |N(i)| of the whole neighbourhoods when the CSR passed holds only the entries of some
+    columns (to check a few columns of a graph too large to run whole); default: the row lengths."""
     indptr, indices, G = _i64(indptr), _i32(indices), _f64(G)
     n_dst, d = indptr.size - 1, G.shape[1]
     dX = np.zeros((n_src, d), np.float64)
+    rl = None if row_len is None else _i64(row_len)
     lib().oracle_full_aggregate_backward(_p(indptr), _p(indices), C.c_int64(n_dst), C.c_int64(n_src),
-                                         _p(G), C.c_int32(d), _p(dX), C.c_int(int(bf16)))
+                                         _p(G), C.c_int32(d), _p(dX), C.c_int(int(bf16)), _p(rl))
     return dX
 
 

@@ -396,13 +396,15 @@ double oracle_bce_with_logits(const double *t, const double *y, int64_t n, doubl
 /* Full-graph mean aggregation (Sec. 3.1 Eq. 2 with S(u) = N(u)) and adjoint  */
 /* ------------------------------------------------------------------------- */
 
-/* dX[s] = sum over rows i and entries e of row i with indices[e] = s of G[i] / deg(i). */
+/* dX[s] = sum over rows i and entries e of row i with indices[e] = s of G[i] / deg(i).
+ * deg(i) = |N(i)| is the length of row i, unless row_len is given: then the CSR holds only part of the
+ * entries (those whose column is wanted) and row_len[i] is the size of the whole neighbourhood. */
 void oracle_full_aggregate_backward(const int64_t *indptr, const int32_t *indices, int64_t n_dst, int64_t n_src,
-                                    const double *G, int32_t d, double *dX, int round_bf16)
+                                    const double *G, int32_t d, double *dX, int round_bf16, const int64_t *row_len)
 {
     for (int64_t s = 0; s < n_src * d; ++s) dX[s] = 0.0;
     for (int64_t i = 0; i < n_dst; ++i) {
-        int64_t deg = indptr[i + 1] - indptr[i];
+        int64_t deg = row_len ? row_len[i] : indptr[i + 1] - indptr[i];
         for (int64_t e = indptr[i]; e < indptr[i + 1]; ++e)
             for (int32_t k = 0; k < d; ++k) dX[(int64_t)indices[e] * d + k] += G[i * d + k] / (double)deg;
     }

@@ -113,10 +113,90 @@ def seed_batch_from_interactions(users: np.ndarray, items: np.ndarray, batch: in
         cand = np.empty(2 * idx.size, np.int32)
         cand[0::2] = users[idx]
         cand[1::2] = items[idx]
-        cand = np.concatenate([got, cand])
-        _, first = np.unique(cand, return_index=True)
-        got = cand[np.sort(first)]
+        got = first_distinct(np.concatenate([got, cand]), len(got) + cand.size)
     return np.ascontiguousarray(got[:batch])
+
+
+def first_distinct(cand: np.ndarray, batch: int) -> np.ndarray:
+    """The first `batch` distinct values of `cand`, in order of first appearance (fewer if there are not enough)."""
+    _, first = np.unique(cand, return_index=True)
+    return np.ascontiguousarray(cand[np.sort(first)][:batch])
+
+
+# ----------------------------------------------------------------------------- generation on a device
+# The largest workload (10^9 interactions) is drawn with torch on the device that will hold the graph: the host
+# arrays alone would take tens of GB and minutes.  Same law as bipartite_interactions, torch's generator
+# instead of numpy's, so the two are different (equally valid) graphs of the same shape.
+
+def _torch_gen(device, seed: int, stream: int):
+    import torch
+    g = torch.Generator(device=device)
+    g.manual_seed(int(seed) * 1_000_003 + int(stream))
+    return g
+
+
+def zipf_ranks_device(gen, size: int, n: int, alpha: float, q: float, device):
+    """Device version of zipf_ranks: int64 tensor of ranks in [0, n)."""
+    import torch
+    u = torch.rand(size, dtype=torch.float64, device=device, generator=gen)
+    if abs(alpha - 1.0) < 1e-12:
+        lo, hi = np.log(1.0 + q), np.log(n + 1.0 + q)
+        r = torch.exp(lo + u * (hi - lo)) - q
+    else:
+        e = 1.0 - alpha
+        lo, hi = (1.0 + q) ** e, (n + 1.0 + q) ** e
+        r = torch.pow(lo + u * (hi - lo), 1.0 / e) - q
+    return (torch.floor(r).to(torch.int64) - 1).clamp_(0, n - 1)
+
+
+def bipartite_interactions_device(n_users: int, n_items: int, m: int, alpha_user, alpha_item, seed: int,
+                                  q: float, device, chunk: int = 1 << 26):
+    """m (user, item) interactions as int32 tensors on `device`; ids are global as in bipartite_interactions."""
+    import torch
+    perm_u = torch.randperm(n_users, device=device, generator=_torch_gen(device, seed, 1)).to(torch.int32)
+    perm_i = torch.randperm(n_items, device=device, generator=_torch_gen(device, seed, 2)).to(torch.int32)
+    gu, gi = _torch_gen(device, seed, 3), _torch_gen(device, seed, 4)
+    users = torch.empty(m, dtype=torch.int32, device=device)
+    items = torch.empty(m, dtype=torch.int32, device=device)
+    for s in range(0, m, chunk):
+        e = min(m, s + chunk)
+        if alpha_user is None:
+            ku = torch.randint(0, n_users, (e - s,), device=device, generator=gu)
+        else:
+            ku = zipf_ranks_device(gu, e - s, n_users, alpha_user, q, device)
+        if alpha_item is None:
+            ki = torch.randint(0, n_items, (e - s,), device=device, generator=gi)
+        else:
+            ki = zipf_ranks_device(gi, e - s, n_items, alpha_item, q, device)
+        users[s:e] = perm_u[ku]
+        items[s:e] = perm_i[ki] + n_users
+    return users, items
+
+
+def normal_features_device(n: int, d: int, seed: int, dtype, device, stream: int = 10, chunk_rows: int = 1 << 22):
+    """N(0,1) features drawn on the device in `dtype` (chunked, so that no fp32 copy of the table exists)."""
+    import torch
+    g = _torch_gen(device, seed, stream)
+    X = torch.empty(n, d, dtype=dtype, device=device)
+    for s in range(0, n, chunk_rows):
+        e = min(n, s + chunk_rows)
+        X[s:e] = torch.randn(e - s, d, dtype=torch.float32, device=device, generator=g).to(dtype)
+    return X
+
+
+def seed_batch_from_interactions_device(users, items, batch: int, seed: int, step: int) -> np.ndarray:
+    """seed_batch_from_interactions for interaction lists that live on a device (torch tensors)."""
+    import torch
+    rng = _rng(seed, 2000 + step)
+    m = users.numel()
+    got = np.zeros(0, np.int32)
+    while got.size < batch:
+        idx = torch.from_numpy(rng.integers(0, m, 4 * batch)).to(users.device)
+        cand = np.empty(2 * idx.numel(), np.int32)
+        cand[0::2] = users[idx].cpu().numpy()
+        cand[1::2] = items[idx].cpu().numpy()
+        got = first_distinct(np.concatenate([got, cand]), batch)
+    return got
 
 
 def bernoulli_labels(n: int, p: float, seed: int, stream: int = 30) -> np.ndarray:
@@ -171,15 +251,21 @@ def build_graph(w: Workload):
     return indptr, indices, (users, items)
 
 
-def build_model(w: Workload):
-    """Layer weights W_l [hidden x 2*d_in] (Glorot), features X [n x d]; fp32 arrays (bf16 values if w.dtype says so)."""
-    X = normal_features(w.n_nodes, w.dim, w.seed)
+def build_weights(w: Workload):
+    """Layer weights W_l [hidden x 2*d_in] (Glorot); fp32 arrays (bf16 values if w.dtype says so)."""
     Ws = []
     d_in = w.dim
     for l in range(len(w.fanouts)):
         Ws.append(glorot_uniform(w.hidden, 2 * d_in, w.seed, 20 + l))
         d_in = w.hidden
     if w.dtype == "bf16":
-        X = to_bf16_values(X)
         Ws = [to_bf16_values(W) for W in Ws]
-    return X, Ws
+    return Ws
+
+
+def build_model(w: Workload):
+    """Features X [n x d] and the layer weights of build_weights."""
+    X = normal_features(w.n_nodes, w.dim, w.seed)
+    if w.dtype == "bf16":
+        X = to_bf16_values(X)
+    return X, build_weights(w)

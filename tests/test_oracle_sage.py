@@ -187,6 +187,15 @@ def test_full_graph_backward_is_transpose_of_forward():
     deg = A.sum(1, keepdims=True)
     P = np.where(deg > 0, A / np.maximum(deg, 1), 0.0)
     assert np.allclose(AX, P @ X, atol=1e-12) and np.allclose(dX, P.T @ G, atol=1e-12)
+    # a few columns only: the CSR keeps just their entries (renumbered), the neighbourhood sizes are passed
+    cols = np.array([3, 17, 41])
+    keep = np.isin(indices, cols)
+    rows = np.repeat(np.arange(n), np.diff(indptr))[keep]
+    sub_ptr = np.zeros(n + 1, np.int64)
+    np.cumsum(np.bincount(rows, minlength=n), out=sub_ptr[1:])
+    sub_idx = np.searchsorted(cols, indices[keep]).astype(np.int32)
+    part = oracle.full_aggregate_backward(sub_ptr, sub_idx, cols.size, G, row_len=np.diff(indptr))
+    assert np.allclose(part, (P.T @ G)[cols], atol=1e-12)
 
 
 # ----------------------------------------------------------------------------- tower + loss
