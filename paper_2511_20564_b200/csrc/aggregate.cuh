@@ -34,73 +34,98 @@ sage_aggregate_kernel(const T *__restrict__ Hsrc, int64_t ld, const int32_t *__r
     const int32_t n_dst = counts[CNT_DST];
     int64_t pad_end = ((int64_t)n_dst + 127) / 128 * 128;
     if (pad_end > cap_dst) pad_end = cap_dst;
-    const int64_t i = ((int64_t)blockIdx.x * kAggThreads + threadIdx.x) >> 5;
-    if (i >= pad_end) return;
-    T *out = cat + i * 2 * d;
-    if (i >= n_dst) {
-        float z[E];
+    // The grid is sized for the machine, not for the capacity: every warp walks over destinations
+    // i, i + warps, ... and fetches the offsets, the first 32 neighbour ids and the self id of its next
+    // destination before it sums the current one.
+    const int64_t warps = (int64_t)gridDim.x * (kAggThreads / 32);
+    int64_t i = ((int64_t)blockIdx.x * kAggThreads + threadIdx.x) >> 5;
+    int32_t beg = 0, end = 0, mine = 0;
+    int64_t self_row = 0;
+    auto fetch = [&](int64_t ii, int32_t &b, int32_t &e, int32_t &m, int64_t &sr) {
+        b = e = m = 0;
+        sr = ii;
+        if (ii < n_dst) {
+            b = indptr[ii];
+            e = indptr[ii + 1];
+            if (lane < e - b) m = nbr[b + lane];
+            if (self_ids) sr = (int64_t)self_ids[ii];
+        }
+    };
+    fetch(i, beg, end, mine, self_row);
+    while (i < pad_end) {
+        const int64_t i_next = i + warps;
+        int32_t beg_n, end_n, mine_n;
+        int64_t self_n;
+        fetch(i_next, beg_n, end_n, mine_n, self_n);
+        T *out = cat + i * 2 * d;
+        if (i >= n_dst) {
+            float z[E];
 #pragma unroll
-        for (int k = 0; k < E; ++k) z[k] = 0.f;
-        for (int q = lane; q < 2 * n_chunks; q += 32) Chunk<T>::store(out + q * E, z);
-        return;
-    }
-    // self half: plain 16-byte copies
-    const int64_t self_row = self_ids ? (int64_t)self_ids[i] : i;
-    for (int q = lane; q < n_chunks; q += 32)
-        *reinterpret_cast<uint4 *>(out + q * E) = __ldg(reinterpret_cast<const uint4 *>(Hsrc + self_row * ld + q * E));
+            for (int k = 0; k < E; ++k) z[k] = 0.f;
+            for (int q = lane; q < 2 * n_chunks; q += 32) Chunk<T>::store(out + q * E, z);
+        } else {
+            // self half: plain 16-byte copies
+            for (int q = lane; q < n_chunks; q += 32)
+                *reinterpret_cast<uint4 *>(out + q * E) = __ldg(reinterpret_cast<const uint4 *>(Hsrc + self_row * ld + q * E));
 
-    float acc[CPL][E];
+            float acc[CPL][E];
 #pragma unroll
-    for (int q = 0; q < CPL; ++q)
+            for (int q = 0; q < CPL; ++q)
 #pragma unroll
-        for (int k = 0; k < E; ++k) acc[q][k] = 0.f;
+                for (int k = 0; k < E; ++k) acc[q][k] = 0.f;
 
-    const int32_t beg = indptr[i], end = indptr[i + 1];
-    for (int32_t base = beg; base < end; base += 32) {
-        const int m = min(32, end - base);
-        const int32_t mine = lane < m ? nbr[base + lane] : 0;
-        for (int t = 0; t * G < m; t += U) {
-            float v[U][CPL][E];
-            bool ok[U];
+            for (int32_t base = beg; base < end; base += 32) {
+                const int m = min(32, end - base);
+                if (base != beg) mine = lane < m ? nbr[base + lane] : 0;
+                for (int t = 0; t * G < m; t += U) {
+                    float v[U][CPL][E];
+                    bool ok[U];
 #pragma unroll
-            for (int u = 0; u < U; ++u) {
-                const int j = (t + u) * G + g;
-                ok[u] = j < m;
-                const int32_t id = __shfl_sync(0xffffffffu, mine, j & 31);
-                const T *row = Hsrc + (int64_t)id * ld;
+                    for (int u = 0; u < U; ++u) {
+                        const int j = (t + u) * G + g;
+                        ok[u] = j < m;
+                        const int32_t id = __shfl_sync(0xffffffffu, mine, j & 31);
+                        const T *row = Hsrc + (int64_t)id * ld;
 #pragma unroll
-                for (int q = 0; q < CPL; ++q) {
-                    const int ch = c + q * LPR;
-                    if (ok[u] && ch < n_chunks) Chunk<T>::load(row + ch * E, v[u][q]);
+                        for (int q = 0; q < CPL; ++q) {
+                            const int ch = c + q * LPR;
+                            if (ok[u] && ch < n_chunks) Chunk<T>::load(row + ch * E, v[u][q]);
+                        }
+                    }
+#pragma unroll
+                    for (int u = 0; u < U; ++u)
+#pragma unroll
+                        for (int q = 0; q < CPL; ++q)
+                            if (ok[u] && c + q * LPR < n_chunks)
+#pragma unroll
+                                for (int k = 0; k < E; ++k) acc[q][k] += v[u][q][k];
                 }
             }
 #pragma unroll
-            for (int u = 0; u < U; ++u)
+            for (int off = LPR; off < 32; off <<= 1)
 #pragma unroll
                 for (int q = 0; q < CPL; ++q)
-                    if (ok[u] && c + q * LPR < n_chunks)
 #pragma unroll
-                        for (int k = 0; k < E; ++k) acc[q][k] += v[u][q][k];
-        }
-    }
+                    for (int k = 0; k < E; ++k) acc[q][k] += __shfl_xor_sync(0xffffffffu, acc[q][k], off);
+            if (g == 0) {
+                const int32_t cnt = end - beg;
+                const float inv = cnt > 0 ? 1.0f / (float)cnt : 0.0f;
 #pragma unroll
-    for (int off = LPR; off < 32; off <<= 1)
+                for (int q = 0; q < CPL; ++q) {
+                    const int ch = c + q * LPR;
+                    if (ch < n_chunks) {
 #pragma unroll
-        for (int q = 0; q < CPL; ++q)
-#pragma unroll
-            for (int k = 0; k < E; ++k) acc[q][k] += __shfl_xor_sync(0xffffffffu, acc[q][k], off);
-    if (g == 0) {
-        const int32_t cnt = end - beg;
-        const float inv = cnt > 0 ? 1.0f / (float)cnt : 0.0f;
-#pragma unroll
-        for (int q = 0; q < CPL; ++q) {
-            const int ch = c + q * LPR;
-            if (ch < n_chunks) {
-#pragma unroll
-                for (int k = 0; k < E; ++k) acc[q][k] *= inv;
-                Chunk<T>::store(out + d + ch * E, acc[q]);
+                        for (int k = 0; k < E; ++k) acc[q][k] *= inv;
+                        Chunk<T>::store(out + d + ch * E, acc[q]);
+                    }
+                }
             }
         }
+        i = i_next;
+        beg = beg_n;
+        end = end_n;
+        mine = mine_n;
+        self_row = self_n;
     }
 }
 

@@ -2,16 +2,18 @@
 //
 //   D[m, n] = sum_k A[m, k] * B[n, k]        A: [rows x K] row-major, B: [N x K] row-major (both K-major)
 //
-// One CTA computes a 128 x NT tile (NT = the widest multiple of 32, at most 256, that divides N).  A single thread feeds TMA loads of
-// 128 x 64 (A) and NT x 64 (B) bf16 boxes into a ring of 128-byte-swizzled shared-memory stages,
+// Output tiles are 128 x NT (NT = the widest multiple of 32, at most 256, that divides N).  A single thread feeds TMA
+// loads of 128 x 64 (A) and NT x 64 (B) bf16 boxes into a ring of 128-byte-swizzled shared-memory stages,
 // a single thread issues tcgen05.mma (M = 128, N = NT, K = 16 per instruction) into an fp32
-// accumulator in tensor memory, and all four warps read the accumulator back with tcgen05.ld for
+// accumulator in tensor memory, and four warps read the accumulator back with tcgen05.ld for
 // the epilogue (bias / ReLU / per-row scale, bf16 store).  No cluster launch, no multicast.
 // Every mbarrier wait is bounded; on a timeout the CTA raises E2EGREC_DEV_TIMEOUT in the status
 // word, skips its stores, releases its tensor memory and returns.
 #include "gemm_tc.cuh"
 
 #include <cuda.h>
+
+#include <algorithm>
 
 namespace e2egrec {
 
@@ -21,6 +23,8 @@ constexpr int kTileM = 128;
 constexpr int kTileK = 64;                 // 64 bf16 = one 128-byte swizzle row
 constexpr int kUmmaK = 16;
 constexpr int kThreads = 128;
+constexpr int kTnEpilogueWarps = 8;          // tc_gemm_tn_kernel: TMA warp, MMA warp, eight epilogue warps
+constexpr int kTnThreads = (2 + kTnEpilogueWarps) * 32;
 constexpr int kMaxStages = 4;
 constexpr int kMinSplitBlocks = 8;          // k-blocks of 64 rows per split of the weight-gradient product
 constexpr uint32_t kSpinLimit = 4u * 1000u * 1000u;
@@ -160,22 +164,30 @@ struct TcEpilogue {
 };
 
 // ------------------------------------------------------------------------- kernel
-__global__ void __launch_bounds__(kThreads)
+// Persistent: the grid has at most one CTA per SM and every CTA walks over the live output tiles
+// t = blockIdx.x, blockIdx.x + gridDim.x, ... (tile t = row tile t / n_tiles_n, column tile t % n_tiles_n, so
+// that neighbouring CTAs read the same rows of A and find them in L2).  Warp 0 feeds the TMA ring, warp 1
+// issues the MMAs into one of two accumulator buffers in tensor memory, warps 2-9 run the epilogue of the
+// previous tile from the other buffer meanwhile (two warps per group of 32 accumulator lanes, each taking
+// every other block of 32 columns).
+__device__ inline void mbar_arrive(uint64_t *bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__global__ void __launch_bounds__(kTnThreads)
 tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int k_blocks,
-                  int stages, int nt, uint32_t tmem_cols, TcEpilogue ep)
+                  int stages, int nt, int n_tiles_n, uint32_t tmem_cols, TcEpilogue ep)
 {
     extern __shared__ uint8_t smem_raw[];
-    __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], accum_bar;
+    __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_full[2], acc_empty[2];
     __shared__ uint32_t tmem_base_slot;
     __shared__ int abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int64_t m0 = (int64_t)blockIdx.x * kTileM;
-    const int n0 = blockIdx.y * nt;
     const int32_t m_valid = *ep.m_dev;
-    if (m0 >= m_valid) {                       // nothing but padding in this tile: rows stay as they are
-        return;
-    }
+    const int64_t n_work = (((int64_t)m_valid + kTileM - 1) / kTileM) * n_tiles_n;   // tiles wholly beyond *m_dev stay as they are
+    if ((int64_t)blockIdx.x >= n_work) return;
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t a_bytes = kTileM * kTileK * 2, b_bytes = (uint32_t)nt * kTileK * 2;
     uint8_t *a_tiles = tiles;
@@ -186,12 +198,15 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             mbar_init(&full_bar[s], 1);
             mbar_init(&empty_bar[s], 1);
         }
-        mbar_init(&accum_bar, 1);
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_empty[b], kTnEpilogueWarps);
+        }
         abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
-    if (warp == 1) {                            // tensor memory for the accumulator: tmem_cols fp32 columns x 128 lanes
+    if (warp == 1) {                            // tensor memory: two accumulators of tmem_cols / 2 fp32 columns x 128 lanes
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
                      "r"(tmem_cols)
                      : "memory");
@@ -201,99 +216,131 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
+    const uint32_t buf_stride = tmem_cols >> 1;
 
-    int issued = 0;                             // k-blocks whose loads the producer has started
-    if (warp == 0 && lane == 0) {
-        // ---- producer: TMA loads into the stage ring
-        for (int kb = 0; kb < k_blocks; ++kb) {
-            const int s = kb % stages;
-            const uint32_t ph = (uint32_t)(kb / stages) & 1u;
-            if (!mbar_wait(&empty_bar[s], ph ^ 1u, &abort_flag)) break;
-            mbar_expect_tx(&full_bar[s], a_bytes + b_bytes);
-            tma_load_2d(a_tiles + (size_t)s * a_bytes, &map_a, kb * kTileK, (int)m0, &full_bar[s]);
-            tma_load_2d(b_tiles + (size_t)s * b_bytes, &map_b, kb * kTileK, n0, &full_bar[s]);
-            issued = kb + 1;
-        }
-    } else if (warp == 1 && lane == 0) {
-        // ---- MMA issuer
-        const uint32_t idesc = make_idesc(kTileM, nt);
-        bool ok = true;
-        for (int kb = 0; kb < k_blocks && ok; ++kb) {
-            const int s = kb % stages;
-            const uint32_t ph = (uint32_t)(kb / stages) & 1u;
-            ok = mbar_wait(&full_bar[s], ph, &abort_flag);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t a_addr = smem_u32(a_tiles + (size_t)s * a_bytes);
-            const uint32_t b_addr = smem_u32(b_tiles + (size_t)s * b_bytes);
-#pragma unroll
-            for (int k = 0; k < kTileK / kUmmaK; ++k) {
-                const uint64_t ad = make_smem_desc(a_addr + k * kUmmaK * 2);
-                const uint64_t bd = make_smem_desc(b_addr + k * kUmmaK * 2);
-                umma(tmem_base, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---- producer: TMA loads into the stage ring, k-block after k-block across tiles
+            uint32_t g = 0;
+            bool ok = true;
+            for (int64_t t = blockIdx.x; t < n_work && ok; t += gridDim.x) {
+                const int m0 = (int)(t / n_tiles_n) * kTileM, n0 = (int)(t % n_tiles_n) * nt;
+                for (int kb = 0; kb < k_blocks; ++kb, ++g) {
+                    const uint32_t s = g % (uint32_t)stages, ph = (g / (uint32_t)stages) & 1u;
+                    ok = mbar_wait(&empty_bar[s], ph ^ 1u, &abort_flag);
+                    if (!ok) break;
+                    mbar_expect_tx(&full_bar[s], a_bytes + b_bytes);
+                    tma_load_2d(a_tiles + (size_t)s * a_bytes, &map_a, kb * kTileK, m0, &full_bar[s]);
+                    tma_load_2d(b_tiles + (size_t)s * b_bytes, &map_b, kb * kTileK, n0, &full_bar[s]);
+                }
             }
-            umma_commit(&empty_bar[s]);         // the stage is free again once these MMAs have read it
+            if (!ok) {
+                // giving up: let the copies that were started land before the shared memory is released
+                int never = 0;
+                for (uint32_t j = g > (uint32_t)stages ? g - stages : 0; j < g; ++j)
+                    mbar_wait(&full_bar[j % stages], (j / stages) & 1u, &never);
+            }
         }
-        if (ok) umma_commit(&accum_bar);        // accumulator complete
-    }
-    __syncwarp();
-
-    // ---- epilogue: warp w owns accumulator lanes 32w .. 32w+31 = rows m0 + 32w + lane
-    const bool ready = mbar_wait(&accum_bar, 0, &abort_flag);
-    tc_fence_after();
-    if (ready) {
-        const int64_t row = m0 + warp * 32 + lane;
-        const bool live = row < m_valid;
-        const float rs = (ep.row_scale && live) ? ep.row_scale[row] : 1.f;
-        __nv_bfloat16 *orow = ep.out + row * ep.ldo + n0;
-        const __nv_bfloat16 *mrow = ep.mask ? ep.mask + row * ep.ld_mask + n0 : nullptr;
-        for (int c = 0; c < nt; c += 32) {
-            uint32_t r[32];
-            tmem_load32(tmem_base + ((uint32_t)(warp * 32) << 16) + (uint32_t)c, r);
-            uint32_t packed[16];
-            uint32_t mbits = 0xFFFFFFFFu;                 // bit j: output column c + j keeps its value
-            if (mrow && live) {
-                mbits = 0;
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---- MMA issuer
+            const uint32_t idesc = make_idesc(kTileM, nt);
+            uint32_t g = 0, lt = 0;
+            bool ok = true;
+            for (int64_t t = blockIdx.x; t < n_work && ok; t += gridDim.x, ++lt) {
+                const uint32_t buf = lt & 1u;
+                ok = mbar_wait(&acc_empty[buf], ((lt >> 1) & 1u) ^ 1u, &abort_flag);   // the epilogue has drained this buffer
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * buf_stride;
+                for (int kb = 0; kb < k_blocks; ++kb, ++g) {
+                    const uint32_t s = g % (uint32_t)stages, ph = (g / (uint32_t)stages) & 1u;
+                    ok = mbar_wait(&full_bar[s], ph, &abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(a_tiles + (size_t)s * a_bytes);
+                    const uint32_t b_addr = smem_u32(b_tiles + (size_t)s * b_bytes);
 #pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                    const uint4 mv = *reinterpret_cast<const uint4 *>(mrow + c + q * 8);
-                    const uint32_t w[4] = {mv.x, mv.y, mv.z, mv.w};
+                    for (int k = 0; k < kTileK / kUmmaK; ++k) {
+                        const uint64_t ad = make_smem_desc(a_addr + k * kUmmaK * 2);
+                        const uint64_t bd = make_smem_desc(b_addr + k * kUmmaK * 2);
+                        umma(d_tmem, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
+                    }
+                    umma_commit(&empty_bar[s]);     // the stage is free again once these MMAs have read it
+                }
+                if (ok) umma_commit(&acc_full[buf]);   // accumulator complete
+            }
+        }
+    } else {
+        // ---- epilogue: warp w reads accumulator lanes 32 (w % 4) .. + 31 = rows m0 + 32 (w % 4) + lane
+        const int lg = warp & 3;                    // the lane group a warp may read is fixed by its index mod 4
+        const int c_first = warp >= 6 ? 32 : 0;     // warps 2-5 take column blocks 0, 2, 4, ...; warps 6-9 the odd ones
+        int c_last = c_first;                       // this warp's last column block
+        while (c_last + 64 < nt) c_last += 64;
+        uint32_t lt = 0;
+        for (int64_t t = blockIdx.x; t < n_work; t += gridDim.x, ++lt) {
+            const uint32_t buf = lt & 1u;
+            if (!mbar_wait(&acc_full[buf], (lt >> 1) & 1u, &abort_flag)) break;
+            tc_fence_after();
+            const int64_t m0 = (t / n_tiles_n) * kTileM;
+            const int n0 = (int)(t % n_tiles_n) * nt;
+            const int64_t row = m0 + lg * 32 + lane;
+            const bool live = row < m_valid;
+            const float rs = (ep.row_scale && live) ? ep.row_scale[row] : 1.f;
+            __nv_bfloat16 *orow = ep.out + row * ep.ldo + n0;
+            const __nv_bfloat16 *mrow = ep.mask ? ep.mask + row * ep.ld_mask + n0 : nullptr;
+            if (c_first >= nt) {                          // a single column block: nothing for the second set of warps
+                if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                continue;
+            }
+            for (int c = c_first; c < nt; c += 64) {
+                uint32_t r[32];
+                tmem_load32(tmem_base + buf * buf_stride + ((uint32_t)(lg * 32) << 16) + (uint32_t)c, r);
+                if (c == c_last) {                        // this warp's share of the buffer is in registers: hand it back
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                }
+                uint32_t packed[16];
+                uint32_t mbits = 0xFFFFFFFFu;                 // bit j: output column c + j keeps its value
+                if (mrow && live) {
+                    mbits = 0;
 #pragma unroll
-                    for (int t = 0; t < 4; ++t) {
-                        if (__uint_as_float(w[t] << 16) > 0.f) mbits |= 1u << (q * 8 + 2 * t);
-                        if (__uint_as_float(w[t] & 0xFFFF0000u) > 0.f) mbits |= 1u << (q * 8 + 2 * t + 1);
+                    for (int q = 0; q < 4; ++q) {
+                        const uint4 mv = *reinterpret_cast<const uint4 *>(mrow + c + q * 8);
+                        const uint32_t w[4] = {mv.x, mv.y, mv.z, mv.w};
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            if (__uint_as_float(w[u] << 16) > 0.f) mbits |= 1u << (q * 8 + 2 * u);
+                            if (__uint_as_float(w[u] & 0xFFFF0000u) > 0.f) mbits |= 1u << (q * 8 + 2 * u + 1);
+                        }
                     }
                 }
-            }
 #pragma unroll
-            for (int j = 0; j < 32; j += 2) {
-                float v0 = __uint_as_float(r[j]), v1 = __uint_as_float(r[j + 1]);
-                const int col = n0 + c + j;
-                if (ep.bias) { v0 += ep.bias[col]; v1 += ep.bias[col + 1]; }
-                if (ep.relu) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
-                if (ep.row_scale) {
-                    if (col >= ep.scale_from) v0 *= rs;
-                    if (col + 1 >= ep.scale_from) v1 *= rs;
+                for (int j = 0; j < 32; j += 2) {
+                    float v0 = __uint_as_float(r[j]), v1 = __uint_as_float(r[j + 1]);
+                    const int col = n0 + c + j;
+                    if (ep.bias) { v0 += ep.bias[col]; v1 += ep.bias[col + 1]; }
+                    if (ep.relu) { v0 = fmaxf(v0, 0.f); v1 = fmaxf(v1, 0.f); }
+                    if (ep.row_scale) {
+                        if (col >= ep.scale_from) v0 *= rs;
+                        if (col + 1 >= ep.scale_from) v1 *= rs;
+                    }
+                    if (!live || !((mbits >> j) & 1u)) v0 = 0.f;
+                    if (!live || !((mbits >> (j + 1)) & 1u)) v1 = 0.f;
+                    __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
+                    packed[j >> 1] = *reinterpret_cast<uint32_t *>(&h);
                 }
-                if (!live || !((mbits >> j) & 1u)) v0 = 0.f;
-                if (!live || !((mbits >> (j + 1)) & 1u)) v1 = 0.f;
-                __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
-                packed[j >> 1] = *reinterpret_cast<uint32_t *>(&h);
-            }
 #pragma unroll
-            for (int q = 0; q < 4; ++q)
-                *reinterpret_cast<uint4 *>(orow + c + q * 8) =
-                    make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                for (int q = 0; q < 4; ++q)
+                    *reinterpret_cast<uint4 *>(orow + c + q * 8) =
+                        make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+            }
         }
-    } else if (threadIdx.x == 0) {
-        atomicOr(reinterpret_cast<unsigned *>(ep.status), E2EGREC_DEV_TIMEOUT);
-        // giving up: let the copies that were started land before the shared memory is released
-        int never = 0;
-        for (int kb = issued > stages ? issued - stages : 0; kb < issued; ++kb)
-            mbar_wait(&full_bar[kb % stages], (uint32_t)(kb / stages) & 1u, &never);
     }
     tc_fence_before();
     __syncthreads();
+    if (threadIdx.x == 0 && abort_flag) atomicOr(reinterpret_cast<unsigned *>(ep.status), E2EGREC_DEV_TIMEOUT);
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
     }
@@ -315,6 +362,17 @@ EncodeTiledFn encode_fn()
         return reinterpret_cast<EncodeTiledFn>(p);
     }();
     return fn;
+}
+
+int sm_count()
+{
+    static int n = []() {
+        int dev = 0, v = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0)
+            v = 148;
+        return v;
+    }();
+    return n;
 }
 
 // [rows x k] bf16 row-major, box = 64 x box_rows, 128-byte swizzle
@@ -346,8 +404,8 @@ bool launch_tn(const __nv_bfloat16 *A, int64_t rows, int k, int64_t lda, const _
     if (!make_map(&ma, A, rows, k, lda, kTileM) || !make_map(&mb, B, n, k, ldb, nt)) return false;
     const int k_blocks = k / kTileK;
     const int stages = k_blocks < kMaxStages ? k_blocks : kMaxStages;
-    uint32_t tmem_cols = 32;
-    while ((int)tmem_cols < nt) tmem_cols <<= 1;
+    uint32_t tmem_cols = 64;                    // two accumulator buffers, each a power of two of columns >= nt
+    while ((int)tmem_cols < 2 * nt) tmem_cols <<= 1;
     const size_t smem = (size_t)stages * (kTileM * kTileK * 2 + (size_t)nt * kTileK * 2) + 1024;
     static bool attr_set = false;
     if (!attr_set) {
@@ -355,9 +413,11 @@ bool launch_tn(const __nv_bfloat16 *A, int64_t rows, int k, int64_t lda, const _
             return false;
         attr_set = true;
     }
-    dim3 grid((unsigned)(rows / kTileM), (unsigned)(n / nt), 1);
+    const int n_tiles_n = n / nt;
+    const int64_t tiles_cap = (rows / kTileM) * n_tiles_n;
+    const unsigned grid = (unsigned)std::min<int64_t>(tiles_cap, sm_count());
     note_launch();
-    tc_gemm_tn_kernel<<<grid, kThreads, smem, st>>>(ma, mb, k_blocks, stages, nt, tmem_cols, ep);
+    tc_gemm_tn_kernel<<<grid, kTnThreads, smem, st>>>(ma, mb, k_blocks, stages, nt, n_tiles_n, tmem_cols, ep);
     return true;
 }
 

@@ -59,7 +59,8 @@ template <typename T, int LPR, int CPL>
 static void launch_sage_aggregate(const T *Hsrc, int64_t ld, const int32_t *nbr, const int32_t *self_ids,
                                   const e2egrec_block &b, T *cat, int d, int64_t rows, cudaStream_t st)
 {
-    const unsigned grid = (unsigned)std::max<int64_t>(1, ceil_div(rows * 32, kAggThreads));
+    // one warp per destination at a time; at most eight blocks per SM, the warps stride over the destinations
+    const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>(ceil_div(rows * 32, kAggThreads), 148 * 8));
     note_launch();
     sage_aggregate_kernel<T, LPR, CPL><<<grid, kAggThreads, 0, st>>>(Hsrc, ld, nbr, self_ids, b.indptr, b.counts, cat, d,
                                                                       (int32_t)rows);

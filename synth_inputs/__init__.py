@@ -237,6 +237,9 @@ WORKLOADS = {
     "medium": Workload("medium", 200_000, 300_000, 10_000_000, 1.2, 1.2, 1, 128, 128, "bf16", (15, 10), 4096),
     "large": Workload("large", 20_000_000, 30_000_000, 1_000_000_000, 1.05, 1.05, 3, 256, 256, "bf16",
                       (20, 10, 5), 8192, q=80.0),
+    # the model and batch of `large` on the graph of `medium`: same kernel shapes, a few hundred MB on the device
+    "medium_wide": Workload("medium_wide", 200_000, 300_000, 10_000_000, 1.2, 1.2, 1, 256, 256, "bf16",
+                            (20, 10, 5), 8192),
     # shape-preserving reductions used where the full size does not fit the time budget of a test
     "medium_small": Workload("medium_small", 20_000, 30_000, 1_000_000, 1.2, 1.2, 1, 128, 128, "bf16",
                              (15, 10), 1024),
