@@ -427,6 +427,15 @@ def run_ours(args, w):
         peak = peaks["bf16_tflops"] if w.dtype == "bf16" else peaks["bf16_tflops"] / 2.25 * 0.08
         roof = dict(bound="tensor" if w.dtype == "bf16" else "alu", achieved=alg / dom_mean_ms / 1e9, peak=peak,
                     unit="TFLOP/s")
+    # both aggregation kernels of the outermost block, whichever kernel dominates
+    alg_fwd = n_edges * (4 + r) + n_dst * (8 + 4 + r + 2 * r)
+    alg_bwd = n_edges * (4 + r) + n_src * (8 + r) + n_dst * r
+    aggregation = {
+        "outer_block": dict(n_dst=n_dst, n_src=n_src, n_edges=n_edges, row_bytes=r),
+        "forward": dict(kernel="sage_aggregate_kernel", ms=tap_ms[1], algorithmic_bytes=alg_fwd,
+                        gbs=alg_fwd / tap_ms[1] / 1e6, frac_of_hbm=alg_fwd / tap_ms[1] / 1e6 / peaks["hbm_gbs"]),
+        "backward": dict(kernel="seg_run_kernel+seg_final_kernel", ms=tap_ms[2], algorithmic_bytes=alg_bwd,
+                         gbs=alg_bwd / tap_ms[2] / 1e6, frac_of_hbm=alg_bwd / tap_ms[2] / 1e6 / peaks["hbm_gbs"])}
     # DRAM bytes per launch from the ncu launch list of this command (profiles/medium_step_launch_list.md);
     # known only for the aggregation kernels of the outermost block of the `medium` workload
     traffic = {1: 6.30e6}.get(dominant) if w.name == "medium" and args.seeds == "activity" else None
@@ -447,7 +456,7 @@ def run_ours(args, w):
                 e2e=dict(value=e2e_edges_all / e2e_s, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
                          ms_per_step=e2e_s / K * 1e3),
                 gpu_launches=int(launches),
-                roofline=roof,
+                roofline=roof, aggregation=aggregation,
                 kernel_ms={TAP_NAMES[k].split(" (")[0]: v for k, v in tap_ms.items()})
     if joint is not None:
         line["joint"] = joint

@@ -20,7 +20,7 @@ constexpr int kAggThreads = 256;
 // the next multiple of 128 (the dense transform reads whole 128-row tiles).
 // ---------------------------------------------------------------------------------------
 template <typename T, int LPR, int CPL>
-__global__ void __launch_bounds__(kAggThreads)
+__global__ void __launch_bounds__(kAggThreads, CPL == 1 ? 4 : 1)
 sage_aggregate_kernel(const T *__restrict__ Hsrc, int64_t ld, const int32_t *__restrict__ nbr,
                       const int32_t *__restrict__ self_ids, const int32_t *__restrict__ indptr,
                       const int32_t *__restrict__ counts, T *__restrict__ cat, int d, int32_t cap_dst)
@@ -78,27 +78,28 @@ sage_aggregate_kernel(const T *__restrict__ Hsrc, int64_t ld, const int32_t *__r
                 const int m = min(32, end - base);
                 if (base != beg) mine = lane < m ? nbr[base + lane] : 0;
                 for (int t = 0; t * G < m; t += U) {
-                    float v[U][CPL][E];
-                    bool ok[U];
+                    uint4 v[U][CPL];                      // raw 16-byte chunks; unpacked when they are added
 #pragma unroll
                     for (int u = 0; u < U; ++u) {
                         const int j = (t + u) * G + g;
-                        ok[u] = j < m;
                         const int32_t id = __shfl_sync(0xffffffffu, mine, j & 31);
                         const T *row = Hsrc + (int64_t)id * ld;
 #pragma unroll
                         for (int q = 0; q < CPL; ++q) {
                             const int ch = c + q * LPR;
-                            if (ok[u] && ch < n_chunks) Chunk<T>::load(row + ch * E, v[u][q]);
+                            v[u][q] = make_uint4(0, 0, 0, 0);     // zero bits are 0.0 in both types
+                            if (j < m && ch < n_chunks) v[u][q] = Chunk<T>::load_raw(row + ch * E);
                         }
                     }
 #pragma unroll
                     for (int u = 0; u < U; ++u)
 #pragma unroll
-                        for (int q = 0; q < CPL; ++q)
-                            if (ok[u] && c + q * LPR < n_chunks)
+                        for (int q = 0; q < CPL; ++q) {
+                            float x[E];
+                            Chunk<T>::unpack(v[u][q], x);
 #pragma unroll
-                                for (int k = 0; k < E; ++k) acc[q][k] += v[u][q][k];
+                            for (int k = 0; k < E; k += 2) add2(acc[q][k], acc[q][k + 1], x[k], x[k + 1]);
+                        }
                 }
             }
 #pragma unroll
