@@ -196,7 +196,7 @@ def run_ours(args, w):
     want_cpu = world == 1 and not args.no_cpu_baseline
     dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
     K, Wm = args.steps, args.warmup
-    total = K + Wm
+    total = K + Wm + 1                                 # + the batch whose sampling is prefetched during the last step
     first_step = rank * 1_000_000                      # = replicas.first_step_of(rank)
     on_device = w.n_interactions > 200_000_000         # too large for host-side generation: drawn with torch on the GPU
     t_setup = time.perf_counter()
@@ -240,7 +240,9 @@ def run_ours(args, w):
     dH_pin = torch.from_numpy(dH_h).to(dt).pin_memory()
     dH = dH_pin.to(dev)
 
-    blocks = E.Blocks(w.n_nodes, w.batch, w.fanouts, dev)
+    # two sets of block buffers: while the forward/backward of one batch runs, the next batch is sampled beside it
+    blocks2 = [E.Blocks(w.n_nodes, w.batch, w.fanouts, dev) for _ in range(2)]
+    blocks = blocks2[0]
     L = len(Ws)
     ctx = torch.empty(E.binding.sage_forward_ctx_bytes(blocks, X, Ws), dtype=torch.uint8, device=dev)
     H_out = torch.zeros(blocks.caps[0][0], w.hidden, dtype=dt, device=dev)
@@ -248,48 +250,79 @@ def run_ours(args, w):
     dWs = [torch.zeros(W.shape, dtype=torch.float32, device=dev) for W in Ws]
     dX = torch.zeros(blocks.caps[L - 1][1], w.dim, dtype=dt, device=dev)
 
-    seeds_in = torch.empty(w.batch, dtype=torch.int32, device=dev)
+    seeds_in2 = [torch.empty(w.batch, dtype=torch.int32, device=dev) for _ in range(2)]
     dH_in = torch.empty_like(dH)
     count_total = torch.zeros(L, 4, dtype=torch.int64, device=dev)
 
+    def sample_leg(p, defer=False):
+        E.sample_khop(indptr, indices, seeds_in2[p], blocks2[p], w.seed, 0, defer_transpose=defer)   # step = the scratch's offset
+
+    def compute_leg(p):
+        E.sage_forward(blocks2[p], X, Ws, ctx=ctx, H_out=H_out)
+        E.sage_backward(blocks2[p], X, Ws, ctx, dH_in, dWs=dWs, dX_rows=dX, scratch=scratch)
+        count_total.add_(blocks2[p].counts)
+
     def step_body():
-        """Everything of one training step, on fixed buffers (seeds_in, dH_in), so that it can be recorded."""
-        E.sample_khop(indptr, indices, seeds_in, blocks, w.seed, 0, defer_transpose=True)   # step = the scratch's offset
-        E.sage_forward(blocks, X, Ws, ctx=ctx, H_out=H_out)
-        E.sage_backward(blocks, X, Ws, ctx, dH_in, dWs=dWs, dX_rows=dX, scratch=scratch)
-        count_total.add_(blocks.counts)
+        """Everything of one training step back to back on fixed buffers (used for warm-up and per-kernel timing)."""
+        sample_leg(0, defer=True)
+        compute_leg(0)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- record the step once as a CUDA graph (no host work between its kernels) and replay it
-    side = torch.cuda.Stream()
+    # ---- record the step as CUDA graphs (no host work between the kernels) and replay them.  Graph p holds the
+    # forward/backward of the batch in buffer p and, on a second stream, the sampling of the next batch into buffer 1-p.
+    side, side2 = torch.cuda.Stream(), torch.cuda.Stream()
     dH_in.copy_(dH)
     with torch.cuda.stream(side):
         for i in range(Wm):                              # eager warm-up on the capture stream
-            seeds_in.copy_(seeds_dev[i])
+            seeds_in2[0].copy_(seeds_dev[i])
             E.sampler_set_step(blocks.scratch, first_step + i)
             step_body()
+        seeds_in2[1].copy_(seeds_dev[0])
+        E.sampler_set_step(blocks2[1].scratch, first_step)
+        with torch.cuda.stream(side2):                   # the second buffer and the second stream, once, eagerly
+            side2.wait_stream(side)
+            sample_leg(1)
+        side.wait_stream(side2)
+        compute_leg(1)
     side.synchronize()
-    launches_before = E.launch_count()
-    graph = torch.cuda.CUDAGraph()
-    with torch.cuda.graph(graph, stream=side):
-        step_body()
-    kernels_per_step = E.launch_count() - launches_before + 1      # + the counter update (a torch kernel)
+    graphs, kernels_per_step = [], 0
+    for p in range(2):
+        launches_before = E.launch_count()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            side2.wait_stream(side)
+            with torch.cuda.stream(side2):
+                sample_leg(1 - p)
+            compute_leg(p)
+            side.wait_stream(side2)
+        graphs.append(g)
+        kernels_per_step = E.launch_count() - launches_before + 1   # + the counter update (a torch kernel)
 
     ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev_a.record(); ev_b.record()
     torch.cuda.synchronize()
 
-    def run_step(i, g=None):
-        seeds_in.copy_(seeds_dev[i], non_blocking=True)
+    def run_step(i):
+        """One step, eagerly and back to back (sampling, forward, backward of batch i)."""
+        seeds_in2[0].copy_(seeds_dev[i], non_blocking=True)
         E.sampler_set_step(blocks.scratch, first_step + i)
-        if g is None:
-            step_body()
-        else:
-            g.replay()
+        step_body()
+
+    def prime(i, src):
+        """Samples batch i into buffer i & 1 (what the previous replay would have done)."""
+        seeds_in2[i & 1].copy_(src[i], non_blocking=True)
+        E.sampler_set_step(blocks2[i & 1].scratch, first_step + i)
+        sample_leg(i & 1)
+
+    def replay_step(i, src):
+        """Forward/backward of batch i (sampled by the previous replay) beside the sampling of batch i + 1."""
+        seeds_in2[(i + 1) & 1].copy_(src[i + 1], non_blocking=True)
+        E.sampler_set_step(blocks2[(i + 1) & 1].scratch, first_step + i + 1)
+        graphs[i & 1].replay()
 
     def tapped_step(i, which):
         """One eagerly launched step with events around kernel group `which`.  The device is first kept
@@ -306,6 +339,7 @@ def run_ours(args, w):
     dominant = max((k for k in tap_ms if k <= 5), key=lambda k: tap_ms[k])
 
     count_total.zero_()
+    prime(Wm, seeds_dev)
     clocks = ClockSampler(local)
     clocks.start()
     time.sleep(0.6)                                    # let the sampler reach its steady 100 ms period
@@ -314,7 +348,7 @@ def run_ours(args, w):
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     e0.record()
     for i in range(K):
-        run_step(Wm + i, graph)
+        replay_step(Wm + i, seeds_dev)
     e1.record()
     barrier()
     clk = clocks.stop(t_begin, clocks.mark())
@@ -324,7 +358,7 @@ def run_ours(args, w):
     if counts[:, 3].any():
         raise RuntimeError(f"device status bits set during the timed region: {counts[:, 3]}")
     edges_rank = int(counts[:, 2].sum())
-    # the dominant kernel again, timed inside recorded steps over the same batches
+    # the dominant kernel again, timed inside eagerly launched steps over the same batches
     dom_ms = []
     for i in range(min(K, 50)):
         dom_ms.append(tapped_step(Wm + i, dominant))
@@ -338,19 +372,19 @@ def run_ours(args, w):
     d2h = sum(t.numel() * t.element_size() for t in res_pin) + cnt_pin.numel() * 4
 
     def e2e_step(i):
-        seeds_in.copy_(seeds_pin[i], non_blocking=True)
         dH_in.copy_(dH_pin, non_blocking=True)
-        E.sampler_set_step(blocks.scratch, first_step + i)
-        graph.replay()
+        replay_step(i, seeds_pin)                      # copies the seeds of batch i + 1 from pinned host memory
         res_pin[0].copy_(H_out, non_blocking=True)
         for t, s in zip(res_pin[1:], dWs):
             t.copy_(s, non_blocking=True)
-        cnt_pin.copy_(blocks.counts, non_blocking=True)
+        cnt_pin.copy_(blocks2[i & 1].counts, non_blocking=True)
         torch.cuda.current_stream().synchronize()      # the caller reads the results of this step
         return int(cnt_pin[:, 2].sum())
 
+    prime(0, seeds_pin)
     for i in range(min(Wm, 3)):
         e2e_step(i)
+    prime(Wm, seeds_pin)
     barrier()
     t0 = time.perf_counter()
     e2e_edges = 0
@@ -447,7 +481,9 @@ def run_ours(args, w):
                 data="synthetic",
                 config=dict(workload=w.name, nodes=w.n_nodes, csr_entries=int(indices.numel()), dim=w.dim, hidden=w.hidden,
                             layers=L, fanouts=list(w.fanouts), batch=w.batch, seeds=args.seeds,
-                            parallelism=f"replicas x{world}", launch="one CUDA graph replay per step",
+                            parallelism=f"replicas x{world}",
+                            launch="one CUDA graph replay per step: forward/backward of the batch beside the sampling of "
+                                   "the next batch on a second stream (two sets of block buffers)",
                             l2="inputs larger than L2: feature table + graph = %.0f MB, a new batch every step"
                                % ((X.numel() * es + indices.numel() * 4 + indptr.numel() * 8) / 1e6),
                             edges_per_step=edges_rank / K, setup_s=round(setup_s, 1),

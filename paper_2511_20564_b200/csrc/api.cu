@@ -27,24 +27,33 @@ int32_t check_launch(const char *what)
 }
 
 static std::mutex g_side_mutex;
-static SideStream *g_side[64] = {};
+constexpr int kSideSlots = 8;
+static SideStream *g_side[64][kSideSlots] = {};
 
-SideStream *SideStream::get()
+// One helper stream per (device, caller's stream): calls made on different streams (a sampling leg beside a
+// compute leg, say) do not meet on a common helper stream.  With more than kSideSlots caller streams on a
+// device the last slot is shared.
+SideStream *SideStream::get(cudaStream_t caller)
 {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
     std::lock_guard<std::mutex> lock(g_side_mutex);
-    if (!g_side[dev]) {
+    int slot = 0;
+    for (; slot < kSideSlots; ++slot)
+        if (!g_side[dev][slot] || g_side[dev][slot]->owner == caller) break;
+    if (slot == kSideSlots) slot = kSideSlots - 1;
+    if (!g_side[dev][slot]) {
         SideStream *s = new SideStream();
         s->next = 0;
+        s->owner = caller;
         if (cudaStreamCreateWithFlags(&s->stream, cudaStreamNonBlocking) != cudaSuccess) { delete s; cudaGetLastError(); return nullptr; }
         for (int i = 0; i < 32; ++i)
             if (cudaEventCreateWithFlags(&s->ev[i], cudaEventDisableTiming) != cudaSuccess) { delete s; cudaGetLastError(); return nullptr; }
         if (cudaEventCreateWithFlags(&s->pending, cudaEventDisableTiming) != cudaSuccess) { delete s; cudaGetLastError(); return nullptr; }
         s->has_pending = false;
-        g_side[dev] = s;
+        g_side[dev][slot] = s;
     }
-    return g_side[dev];
+    return g_side[dev][slot];
 }
 
 cudaEvent_t SideStream::event() { return ev[(next++) & 31u]; }
@@ -98,7 +107,7 @@ void tap_end(int which, cudaStream_t st)
 
 extern "C" int32_t e2egrec_sample_join(void *stream)
 {
-    e2egrec::SideStream *side = e2egrec::SideStream::get();
+    e2egrec::SideStream *side = e2egrec::SideStream::get(static_cast<cudaStream_t>(stream));
     if (side) side->join_pending(static_cast<cudaStream_t>(stream));
     return e2egrec::check_launch("sample_join");
 }

@@ -24,18 +24,19 @@ inline size_t dtype_size(int32_t dtype) { return dtype == E2EGREC_BF16 ? 2 : 4; 
 // host side: remember the text of a failed launch for e2egrec_last_error()
 void set_last_error(const char *msg);
 int32_t check_launch(const char *what);
-// host side: one helper stream per device for work that may overlap the caller's stream inside one entry
-// point.  fork() makes the helper stream wait for what the caller's stream has enqueued so far; join()
+// host side: one helper stream per device and caller's stream for work that may overlap the caller's stream
+// inside one entry point.  fork() makes the helper stream wait for what the caller's stream has enqueued so far; join()
 // makes the caller's stream wait for the helper stream.  Both are plain event record / wait pairs, so they
 // are legal inside a stream capture.  get() returns nullptr if the stream cannot be created (the caller
 // then stays on its own stream).
 struct SideStream {
     cudaStream_t stream;
+    cudaStream_t owner;           // the caller's stream this helper belongs to
     cudaEvent_t ev[32];
     unsigned next;
     cudaEvent_t pending;          // end of helper-stream work that a later entry point has to wait for
     bool has_pending;
-    static SideStream *get();
+    static SideStream *get(cudaStream_t caller);
     void defer();                 // remember the helper stream's current end as pending
     void join_pending(cudaStream_t into);
     cudaEvent_t event();

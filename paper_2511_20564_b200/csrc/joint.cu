@@ -377,7 +377,7 @@ int32_t run_joint(const JointPlan &jp, const e2egrec_csr *graph, const e2egrec_m
     }
     // the weight gradients feed nothing later in the step: they go to the helper stream (behind the block
     // transposition that the sampler left there); the encoder backward waits for that stream before its first launch
-    SideStream *side = SideStream::get();
+    SideStream *side = SideStream::get(st);
     cudaStream_t ws_st = st;
     if (side) {
         side->fork(st);

@@ -177,7 +177,7 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
             static_cast<const T *>(dH_out->data), dH_out->ld, reinterpret_cast<const T *>(ctx + p.h_off), p.d_out,
             &b.counts[CNT_DST], p.rows, p.d_out, act ? act[n_layers - 1] : 1, dz_buf[(n_layers - 1) & 1]);
     }
-    SideStream *side = SideStream::get();
+    SideStream *side = SideStream::get(st);
     cudaEvent_t dz_free[2] = {nullptr, nullptr};
     for (int l = n_layers - 1; l >= 0; --l) {
         const LayerPlan &p = plan[l];
@@ -341,7 +341,7 @@ extern "C" int32_t e2egrec_sage_backward(const e2egrec_block *blocks, int32_t n_
     const size_t es = dtype_size(X->dtype);
     if ((dX_rows->ld * es) % 16 || reinterpret_cast<uintptr_t>(dX_rows->data) % 16) return E2EGREC_ERR_ALIGN;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (SideStream *side = SideStream::get()) side->join_pending(st);     // a deferred block transposition
+    if (SideStream *side = SideStream::get(st)) side->join_pending(st);     // a deferred block transposition
     if (X->dtype == E2EGREC_BF16)
         return backward_impl<__nv_bfloat16>(blocks, n_layers, X, W, act, plan, static_cast<const char *>(ctx), dH_out, dW,
                                             dbias, dX_rows, static_cast<char *>(scratch), bs, flags, st);

@@ -571,7 +571,7 @@ int32_t e2egrec::sample_khop_impl(const e2egrec_csr *graph, const int32_t *seeds
     }
     // The transposition of a hop (sort + offsets) is only needed by the backward pass, so it runs on the
     // helper stream beside the sampling of the next hop; everything is joined before this call returns.
-    SideStream *side = SideStream::get();
+    SideStream *side = SideStream::get(st);
     if (side) side->join_pending(st);               // a transposition deferred by an earlier call still uses the lanes
     for (int h = 0; h < n_hops; ++h) {
         const e2egrec_block &b = blocks[h];

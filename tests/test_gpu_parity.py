@@ -287,3 +287,50 @@ def test_deferred_transposition_joins_before_use():
     E.sample_join()
     torch.cuda.synchronize()
     assert_blocks_equal(blocks.to_host(), ora["blocks"])
+
+
+def test_sampling_of_the_next_batch_beside_the_current_step():
+    """Two sets of block buffers and two streams, as bench.py runs the step: the forward/backward of batch i beside the
+    sampling of batch i + 1.  Every step's outputs are bit-identical to the same steps run back to back."""
+    import paper_2511_20564_b200 as E
+    w = S.WORKLOADS["medium_small"]
+    indptr_h, indices_h, _ = S.build_graph(w)
+    X_h, Ws_h = S.build_model(w)
+    dev = torch.device("cuda")
+    indptr, indices = torch.from_numpy(indptr_h).to(dev), torch.from_numpy(indices_h).to(dev)
+    X = torch.from_numpy(X_h).to(dev, torch.bfloat16)
+    Ws = [torch.from_numpy(W).to(dev, torch.bfloat16) for W in Ws_h]
+    n_steps = 4
+    seeds = [torch.from_numpy(S.seed_batch(w.n_nodes, w.batch, w.seed, i)).to(dev) for i in range(n_steps + 1)]
+    dH = torch.from_numpy(S.to_bf16_values(np.random.default_rng(5).standard_normal((w.batch, w.hidden)).astype(np.float32)))
+    dH = dH.to(dev, torch.bfloat16)
+    bufs = [E.Blocks(w.n_nodes, w.batch, w.fanouts, dev) for _ in range(2)]
+
+    def compute(b):
+        H, ctx = E.sage_forward(b, X, Ws)
+        g = torch.zeros(H.shape, dtype=torch.bfloat16, device=dev)
+        g[: w.batch] = dH
+        dWs, dX = E.sage_backward(b, X, Ws, ctx, g)
+        return [H.clone()] + [t.clone() for t in dWs] + [dX.clone(), b.counts.clone()]
+
+    want = []
+    for i in range(n_steps):
+        E.sample_khop(indptr, indices, seeds[i], bufs[0], w.seed, i)
+        want.append(compute(bufs[0]))
+    torch.cuda.synchronize()
+
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    got = []
+    with torch.cuda.stream(s1):
+        E.sample_khop(indptr, indices, seeds[0], bufs[0], w.seed, 0)
+        for i in range(n_steps):
+            s2.wait_stream(s1)
+            with torch.cuda.stream(s2):
+                E.sample_khop(indptr, indices, seeds[i + 1], bufs[(i + 1) & 1], w.seed, i + 1)
+            got.append(compute(bufs[i & 1]))
+            s1.wait_stream(s2)
+    torch.cuda.synchronize()
+    for i in range(n_steps):
+        assert int(got[i][-1][:, 3].sum()) == 0
+        for a, b in zip(got[i], want[i]):
+            assert torch.equal(a, b), f"step {i}"
