@@ -427,6 +427,30 @@ seg_final_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_t
                 uint4 *row = reinterpret_cast<uint4 *>(o.out + s * o.ld_out);
                 for (int q = 0; q < n16; ++q) row[q] = make_uint4(0, 0, 0, 0);
             }
+        } else if ((d * (int)sizeof(T)) % 16 == 0 && o.ld_out * (int64_t)sizeof(T) % 16 == 0 &&
+                   reinterpret_cast<uintptr_t>(o.out) % 16 == 0 && o.ld_self * (int64_t)sizeof(T) % 16 == 0 &&
+                   reinterpret_cast<uintptr_t>(o.self) % 16 == 0 &&
+                   (!o.mask || (o.ld_mask * (int64_t)sizeof(T) % 16 == 0 && reinterpret_cast<uintptr_t>(o.mask) % 16 == 0))) {
+            // fin(0) = mask * self: eight lanes per segment, 16-byte chunks
+            constexpr int E = Chunk<T>::kElems;
+            const int n16 = d / E;
+            for (int64_t s = (b * kAggThreads + threadIdx.x) >> 3; s < n_seg; s += n_extra * (kAggThreads / 8)) {
+                if (ptr[s + 1] != ptr[s]) continue;
+                for (int q = threadIdx.x & 7; q < n16; q += 8) {
+                    float v[E];
+#pragma unroll
+                    for (int e = 0; e < E; ++e) v[e] = 0.f;
+                    if (s < n_self) Chunk<T>::load(o.self + s * o.ld_self + q * E, v);
+                    if (o.mask) {
+                        float m[E];
+                        Chunk<T>::load(o.mask + s * o.ld_mask + q * E, m);
+#pragma unroll
+                        for (int e = 0; e < E; ++e)
+                            if (!(m[e] > 0.f)) v[e] = 0.f;
+                    }
+                    Chunk<T>::store(o.out + s * o.ld_out + q * E, v);
+                }
+            }
         } else {
             for (int64_t s = (b * kAggThreads + threadIdx.x) >> 3; s < n_seg; s += n_extra * (kAggThreads / 8)) {
                 if (ptr[s + 1] != ptr[s]) continue;
