@@ -99,14 +99,26 @@ def csr_transpose(n_rows, n_cols, indptr, indices):
 
 # ----------------------------------------------------------------------------- sampling
 
-def sample_khop(indptr, indices, seeds, fanouts, seed, step):
+def edge_cumulate(indptr, q):
+    """Per-row running sums (uint64) of integer edge weights q (uint32), the table of the weighted sampler."""
+    indptr = _i64(indptr)
+    q = np.ascontiguousarray(q, dtype=np.uint32)
+    cum = np.zeros(q.size, np.uint64)
+    lib().oracle_edge_cumulate(C.c_int64(indptr.size - 1), _p(indptr), _p(q), _p(cum))
+    return cum
+
+
+def sample_khop(indptr, indices, seeds, fanouts, seed, step, edge_cum=None):
     """k-hop sampled blocks (Sec. 4.1 subgraph construction; Sec. 3.1 multiset S_l(u)).
 
     Hop h (1-based) samples for every node of D_h = F_{h-1} (F_0 = the seeds) with
     fanouts[h-1]; returns one dict per hop with the block CSR (indptr, col,
     nbr_global), the frontier src_nodes = F_h, the transposed block and 1/|S|.
+    edge_cum (from edge_cumulate) switches the draws to the weighted form p ~ q of Sec. 4.1.
     """
     indptr, indices = _i64(indptr), _i32(indices)
+    if edge_cum is not None:
+        edge_cum = np.ascontiguousarray(edge_cum, dtype=np.uint64)
     n = indptr.size - 1
     dst = _i32(seeds)
     blocks = []
@@ -115,7 +127,7 @@ def sample_khop(indptr, indices, seeds, fanouts, seed, step):
         cap = max(1, n_dst * int(f))
         blk_indptr = np.zeros(n_dst + 1, np.int32)
         nbr = np.zeros(cap, np.int32)
-        ne = lib().oracle_sample_hop(_p(indptr), _p(indices), _p(dst), C.c_int32(n_dst), C.c_int32(int(f)),
+        ne = lib().oracle_sample_hop(_p(indptr), _p(indices), _p(edge_cum), _p(dst), C.c_int32(n_dst), C.c_int32(int(f)),
                                      C.c_uint64(int(seed)), C.c_uint32(int(step)), C.c_int32(h),
                                      _p(blk_indptr), _p(nbr))
         nbr = nbr[:ne].copy()

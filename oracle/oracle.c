@@ -135,6 +135,20 @@ void oracle_csr_transpose(int64_t n_rows, int64_t n_cols, const int64_t *indptr,
 /* number of sampled neighbours bounded by k)                                 */
 /* ------------------------------------------------------------------------- */
 
+/* Running sums of the integer edge weights inside every row: cum[e] = q[row begin] + ... + q[e].
+ * q_e is the caller's quantisation of omega_e^beta (Sec. 4.1); the integers make the weighted draw
+ * exact and identical on every machine. */
+void oracle_edge_cumulate(int64_t n_nodes, const int64_t *indptr, const uint32_t *q, uint64_t *cum)
+{
+    for (int64_t u = 0; u < n_nodes; ++u) {
+        uint64_t run = 0;
+        for (int64_t e = indptr[u]; e < indptr[u + 1]; ++e) {
+            run += q[e];
+            cum[e] = run;
+        }
+    }
+}
+
 /* One hop.  For every destination u = dst_nodes[i]:
  *   deg <= fanout : S(u) = N(u), every stored entry once, in CSR order
  *                   (k is an upper bound; the mean is then exact);
@@ -148,9 +162,14 @@ void oracle_csr_transpose(int64_t n_rows, int64_t n_cols, const int64_t *indptr,
  * number r and picks entry floor(r * deg / 2^64) of the row.  The counter holds
  * the global node id, so S(u) does not depend on which other nodes share the
  * batch or on their order.
+ * With g_cum (the per-row running sums of integer edge weights q_e, see
+ * oracle_edge_cumulate) a draw is weighted instead: p(u -> v) = q_uv / sum_k q_uk,
+ * the sampling probability of Sec. 4.1 with q standing for omega^beta; t =
+ * floor(r * total / 2^64) and the first entry whose running sum exceeds t is
+ * picked.  A row whose weights sum to zero is drawn uniformly.
  * Outputs: blk_indptr[n_dst+1] (prefix sums of |S(u)|), nbr_global[...] (global
  * ids, row after row).  Returns the number of entries written. */
-int64_t oracle_sample_hop(const int64_t *g_indptr, const int32_t *g_indices,
+int64_t oracle_sample_hop(const int64_t *g_indptr, const int32_t *g_indices, const uint64_t *g_cum,
                           const int32_t *dst_nodes, int32_t n_dst, int32_t fanout,
                           uint64_t seed, uint32_t step, int32_t hop,
                           int32_t *blk_indptr, int32_t *nbr_global)
@@ -170,7 +189,17 @@ int64_t oracle_sample_hop(const int64_t *g_indptr, const int32_t *g_indices,
                 oracle_philox4x32_10(ctr, key, out);
                 int half = j & 1;
                 uint64_t r = ((uint64_t)out[2 * half + 1] << 32) | out[2 * half];
-                uint64_t pos = (uint64_t)(((unsigned __int128)r * (unsigned __int128)(uint64_t)deg) >> 64);
+                uint64_t pos;
+                uint64_t total = g_cum ? g_cum[beg + deg - 1] : 0;
+                if (total > 0) {
+                    /* importance sampling (Sec. 4.1): t is uniform over [0, total), the entry whose interval
+                     * [cum[e-1], cum[e]) holds t is drawn, i.e. entry e with probability q_e / total */
+                    uint64_t t = (uint64_t)(((unsigned __int128)r * (unsigned __int128)total) >> 64);
+                    pos = 0;
+                    while (g_cum[beg + (int64_t)pos] <= t) ++pos;
+                } else {
+                    pos = (uint64_t)(((unsigned __int128)r * (unsigned __int128)(uint64_t)deg) >> 64);
+                }
                 nbr_global[w++] = g_indices[beg + (int64_t)pos];
             }
         }

@@ -199,6 +199,21 @@ def seed_batch_from_interactions_device(users, items, batch: int, seed: int, ste
     return got
 
 
+def edge_weight_units(indptr: np.ndarray, seed: int, beta: float, stream: int = 40, bits: int = 16) -> np.ndarray:
+    """Integer sampling weights q_e for every CSR entry: omega_e log-normal (a stand-in for the Swing scores of the
+    paper's item graph), q_e = max(1, round(2^bits * (omega_e / max of its row)^beta)).  beta = 0 gives equal
+    weights.  Drawn and quantised once, here, so that both sides are handed the same integers."""
+    indptr = np.asarray(indptr, np.int64)
+    m = int(indptr[-1])
+    omega = np.exp(_rng(seed, stream).standard_normal(m))
+    deg = np.diff(indptr)
+    nz = deg > 0
+    row_max = np.ones(indptr.size - 1)
+    row_max[nz] = np.maximum.reduceat(omega, indptr[:-1][nz]) if m else 1.0
+    rel = omega / np.repeat(row_max, deg)
+    return np.maximum(1, np.rint((1 << bits) * rel ** beta)).astype(np.uint32)
+
+
 def bernoulli_labels(n: int, p: float, seed: int, stream: int = 30) -> np.ndarray:
     return (_rng(seed, stream).random(n) < p).astype(np.float32)
 
