@@ -472,7 +472,7 @@ def run_ours(args, w):
                          gbs=alg_bwd / tap_ms[2] / 1e6, frac_of_hbm=alg_bwd / tap_ms[2] / 1e6 / peaks["hbm_gbs"])}
     # DRAM bytes per launch from the ncu launch list of this command (profiles/medium_step_launch_list.md);
     # known only for the aggregation kernels of the outermost block of the `medium` workload
-    traffic = {1: 6.30e6}.get(dominant) if w.name == "medium" and args.seeds == "activity" else None
+    traffic = {1: 6.30e6, 2: 5.55e6 + 1.80e6}.get(dominant) if w.name == "medium" and args.seeds == "activity" else None
     roof.update(frac=roof["achieved"] / roof["peak"], traffic=traffic, kernel=TAP_NAMES[dominant],
                 ms_per_launch=dom_mean_ms, algorithmic_units_per_launch=alg, peak_source=peaks["source"])
 
@@ -611,7 +611,10 @@ def run_fullgraph(args):
     roof = dict(bound="hbm", achieved=alg / tk / 1e6, peak=peaks["hbm_gbs"], unit="GB/s", traffic=None,
                 kernel=f"seg_run_kernel+seg_final_kernel ({big})", ms_per_launch=tk,
                 algorithmic_units_per_launch=alg, peak_source=peaks["source"],
-                compulsory_bytes=n * r * 2 + m * 4 + n * 16)
+                compulsory_bytes=n * r * 2 + m * 4 + n * 16,
+                # ncu DRAM bytes (read + write, both kernels) of one launch on the 1/5-scale graph
+                # (profiles/seg_run_kernel_fullgraph.md); not scaled up: the L2 hit rate changes with the table size
+                traffic_at_scale_0_2=dict(fwd=383.0e6, bwd=355.0e6))
     roof["frac"] = roof["achieved"] / roof["peak"]
     line = dict(metric="fullgraph_mean_aggregation_fwd_bwd_edges_per_sec", value=m / ((t_f + t_b) / 1e3), unit="edges/s",
                 n_gpus=1, steps=K, warmup=Wm, ms_per_step=ms / K, higher_is_better=True, scaling="weak", vs_baseline=None,

@@ -69,13 +69,15 @@ extern "C" {
 
 /* Graph G=(V,E) in compressed sparse row form (Sec. 3, Notation): row u lists N(u),
  * parallel edges kept.  indptr: device int64[n_nodes+1]; indices: device int32[n_edges].
- * edge_weight is reserved for the weighted sampler (omega_uv of Sec. 4.1) and must be NULL. */
+ * edge_cum: NULL (uniform sampling) or device uint64[n_edges], the running sums of integer edge
+ * weights inside every row as e2egrec_edge_cumulate writes them; the sampler then draws a neighbour
+ * with probability q_uv / sum_k q_uk (the importance sampling of Sec. 4.1 with q for omega^beta). */
 typedef struct e2egrec_csr {
-    int64_t        n_nodes;
-    int64_t        n_edges;
-    const int64_t *indptr;
-    const int32_t *indices;
-    const float   *edge_weight;
+    int64_t         n_nodes;
+    int64_t         n_edges;
+    const int64_t  *indptr;
+    const int32_t  *indices;
+    const uint64_t *edge_cum;
 } e2egrec_csr;
 
 /* Row-major matrix on the device: `rows` x `dim`, leading dimension `ld` elements. */
@@ -153,6 +155,13 @@ int32_t e2egrec_sample_khop_workspace(int64_t n_nodes, int32_t n_seeds, int32_t 
  * leaves the buffer idle again when it finishes, so one buffer serves every step. */
 int32_t e2egrec_sampler_scratch_init(int64_t n_nodes, void *scratch, size_t scratch_bytes, void *stream);
 
+/* Table of the weighted sampler (Sec. 4.1, sampling probability p(u->v) = omega_uv^beta / sum_k omega_uk^beta).
+ * q: device uint32[n_edges], the caller's integer quantisation of omega^beta per CSR entry (integers make the
+ * draw exact and the sampled lists identical on every machine); cum: device uint64[n_edges], receives
+ * cum[e] = q[first entry of e's row] + ... + q[e].  Set-up work, once per graph (and per beta). */
+int32_t e2egrec_edge_cumulate(int64_t n_nodes, int64_t n_edges, const int64_t *indptr, const uint32_t *q,
+                              uint64_t *cum, void *stream);
+
 /* Sets the step offset kept in the sampler scratch: every later e2egrec_sample_khop that uses this
  * scratch draws with step = its `step` argument + step_offset (mod 2^32).  init sets it to 0.  This is
  * for callers that record the kernels of one training step once (a CUDA graph) and replay them: the
@@ -170,6 +179,9 @@ int32_t e2egrec_sampler_set_step(void *scratch, uint32_t step_offset, void *stre
  *       (j/2, u, (1<<8)|h, step); output words 2(j%2), 2(j%2)+1 form a 64-bit r and the
  *       entry picked is floor(r * deg / 2^64).  The lists are therefore a function of
  *       (seed, step, h, u) only and reproducible bit for bit.
+ *       With graph->edge_cum the draw is weighted (beta > 0): t = floor(r * total / 2^64) with total
+ *       the row's last running sum, and the first entry of the row whose running sum exceeds t is
+ *       picked; a row whose weights sum to zero is drawn uniformly as above.
  *   blocks host array[n_hops] of structs holding device pointers; blocks[h-1] receives hop h
  *       including its transposed form.  F_h = D_h followed by the new nodes in ascending order.
  *   scratch device buffer initialised by e2egrec_sampler_scratch_init for the same n_nodes.

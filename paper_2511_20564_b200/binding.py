@@ -25,7 +25,7 @@ class E2EGrecError(RuntimeError):
 
 class Csr(C.Structure):
     _fields_ = [("n_nodes", C.c_int64), ("n_edges", C.c_int64), ("indptr", C.c_void_p),
-                ("indices", C.c_void_p), ("edge_weight", C.c_void_p)]
+                ("indices", C.c_void_p), ("edge_cum", C.c_void_p)]
 
 
 class Mat(C.Structure):
@@ -68,6 +68,8 @@ def lib():
         L.e2egrec_sample_khop.argtypes = [C.POINTER(Csr), C.c_void_p, C.c_int32, C.c_int32, C.c_void_p,
                                           C.c_uint64, C.c_uint32, C.c_uint32, C.POINTER(Block), C.c_void_p,
                                           C.c_size_t, C.c_void_p]
+        L.e2egrec_edge_cumulate.restype = C.c_int32
+        L.e2egrec_edge_cumulate.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.e2egrec_sage_forward.restype = C.c_int32
         L.e2egrec_sage_forward.argtypes = [C.POINTER(Block), C.c_int32, C.POINTER(Mat), C.POINTER(Mat),
                                            C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_size_t),
@@ -236,11 +238,24 @@ def sample_join(stream=None):
     _check(lib().e2egrec_sample_join(_stream(stream)), "e2egrec_sample_join")
 
 
+def edge_cumulate(indptr: torch.Tensor, q: torch.Tensor, stream=None):
+    """Per-row running sums (uint64, returned as an int64 tensor of the same bits) of the integer edge weights q
+    (uint32 values in an int32 / uint32 tensor); see e2egrec_edge_cumulate."""
+    assert indptr.dtype == torch.int64 and q.element_size() == 4 and q.is_contiguous()
+    cum = torch.empty(max(q.numel(), 1), dtype=torch.int64, device=q.device)
+    _check(lib().e2egrec_edge_cumulate(indptr.numel() - 1, q.numel(), _ptr(indptr), _ptr(q), _ptr(cum), _stream(stream)),
+           "e2egrec_edge_cumulate")
+    return cum[: q.numel()]
+
+
 def sample_khop(indptr: torch.Tensor, indices: torch.Tensor, seeds: torch.Tensor, blocks: Blocks, seed: int,
-                step: int, stream=None, defer_transpose=False):
-    """Enqueues the k-hop sample of `seeds` into `blocks` (see e2egrec_sample_khop)."""
+                step: int, stream=None, defer_transpose=False, edge_cum=None):
+    """Enqueues the k-hop sample of `seeds` into `blocks` (see e2egrec_sample_khop); edge_cum (from edge_cumulate)
+    switches to the weighted draws."""
     assert indptr.dtype == torch.int64 and indices.dtype == torch.int32 and seeds.dtype == torch.int32
-    g = Csr(indptr.numel() - 1, indices.numel(), indptr.data_ptr(), indices.data_ptr(), None)
+    assert edge_cum is None or (edge_cum.element_size() == 8 and edge_cum.numel() == indices.numel())
+    g = Csr(indptr.numel() - 1, indices.numel(), indptr.data_ptr(), indices.data_ptr(),
+            None if edge_cum is None else edge_cum.data_ptr())
     f = _i32_host(blocks.fanouts)
     _check(lib().e2egrec_sample_khop(C.byref(g), _ptr(seeds), seeds.numel(), len(blocks), f,
                                      C.c_uint64(seed), C.c_uint32(step), DEFER_TRANSPOSE if defer_transpose else 0, blocks.c,

@@ -132,10 +132,12 @@ __global__ void seed_init_kernel(const int32_t *__restrict__ seeds, int32_t n_se
 // destination, a chained scan for the block's offset into the entry arrays, then one thread per
 // (destination, slot).  Slot j of node u at hop h draws with the counter (j/2, u, (1<<8)|h, step) and
 // key (seed lo, seed hi); words 2(j%2), 2(j%2)+1 form r and the picked row position is
-// floor(r * deg / 2^64).  deg <= fanout copies the row instead.  Sampled nodes that are not yet in
-// the frontier are marked in the bitmap.
+// floor(r * deg / 2^64); with running sums of integer edge weights (g_cum) it is the first entry of the row
+// whose running sum exceeds floor(r * total / 2^64).  deg <= fanout copies the row instead.  Sampled nodes
+// that are not yet in the frontier are marked in the bitmap.
 __global__ void __launch_bounds__(kDstThreads)
-hop_sample_kernel(const int64_t *__restrict__ g_indptr, const int32_t *__restrict__ g_indices, int64_t n_nodes,
+hop_sample_kernel(const int64_t *__restrict__ g_indptr, const int32_t *__restrict__ g_indices,
+                  const uint64_t *__restrict__ g_cum, int64_t n_nodes,
                   const int32_t *__restrict__ dst_nodes, const int32_t *n_dst_ptr, int32_t cap_dst, int32_t cap_edges,
                   int32_t fanout, int32_t hop, uint32_t seed_lo, uint32_t seed_hi, uint32_t step_arg,
                   const uint32_t *__restrict__ step_offset, int first_hop, int32_t *__restrict__ counts,
@@ -228,7 +230,20 @@ hop_sample_kernel(const int64_t *__restrict__ g_indptr, const int32_t *__restric
                 const uint4 r4 = philox4x32_10(make_uint4((uint32_t)(j >> 1), (uint32_t)node[lo], (1u << 8) | (uint32_t)hop, step),
                                                make_uint2(seed_lo, seed_hi));
                 const uint64_t rnd = (j & 1) ? (((uint64_t)r4.w << 32) | r4.z) : (((uint64_t)r4.y << 32) | r4.x);
-                pos = (int64_t)__umul64hi(rnd, (uint64_t)deg);
+                const uint64_t *cum = g_cum ? g_cum + gbeg_s[lo] : nullptr;
+                const uint64_t total = cum ? cum[deg - 1] : 0;
+                if (total > 0) {
+                    // weighted draw: the first entry of the row whose running sum exceeds t
+                    const uint64_t t = __umul64hi(rnd, total);
+                    int64_t a = 0, b = deg - 1;                 // cum[b] > t always
+                    while (a < b) {
+                        const int64_t mid = (a + b) >> 1;
+                        if (cum[mid] > t) b = mid; else a = mid + 1;
+                    }
+                    pos = a;
+                } else {
+                    pos = (int64_t)__umul64hi(rnd, (uint64_t)deg);
+                }
             }
             src[q] = gbeg_s[lo] + pos;
         }
@@ -499,6 +514,43 @@ extern "C" int32_t e2egrec_sampler_set_step(void *scratch, uint32_t step_offset,
     return check_launch("sampler_set_step");
 }
 
+// Running sums of the integer edge weights of every row, one warp per row at a time: 32 entries per round, a
+// 64-bit warp scan, the carry kept in a register.
+__global__ void __launch_bounds__(256)
+edge_cumulate_kernel(int64_t n_nodes, const int64_t *__restrict__ indptr, const uint32_t *__restrict__ q,
+                     uint64_t *__restrict__ cum)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t warps = (int64_t)gridDim.x * (blockDim.x >> 5);
+    for (int64_t u = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5; u < n_nodes; u += warps) {
+        const int64_t beg = indptr[u], end = indptr[u + 1];
+        uint64_t carry = 0;
+        for (int64_t e0 = beg; e0 < end; e0 += 32) {
+            const int64_t e = e0 + lane;
+            uint64_t v = e < end ? (uint64_t)q[e] : 0;
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) {
+                const uint64_t up = __shfl_up_sync(0xffffffffu, v, off);
+                if (lane >= off) v += up;
+            }
+            if (e < end) cum[e] = carry + v;
+            carry += __shfl_sync(0xffffffffu, v, 31);
+        }
+    }
+}
+
+extern "C" int32_t e2egrec_edge_cumulate(int64_t n_nodes, int64_t n_edges, const int64_t *indptr, const uint32_t *q,
+                                         uint64_t *cum, void *stream)
+{
+    if (n_nodes < 0 || n_edges < 0) return E2EGREC_ERR_ARG;
+    if (!indptr || (n_edges > 0 && (!q || !cum))) return E2EGREC_ERR_NULL;
+    if (n_nodes == 0 || n_edges == 0) return E2EGREC_OK;
+    const unsigned grid = (unsigned)std::min<int64_t>(ceil_div(n_nodes * 32, 256), 148 * 16);
+    note_launch();
+    edge_cumulate_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(n_nodes, indptr, q, cum);
+    return check_launch("edge_cumulate");
+}
+
 extern "C" int32_t e2egrec_sample_khop(const e2egrec_csr *graph, const int32_t *seeds, int32_t n_seeds,
                                        int32_t n_hops, const int32_t *fanouts, uint64_t seed, uint32_t step,
                                        uint32_t flags, const e2egrec_block *blocks,
@@ -515,7 +567,6 @@ int32_t e2egrec::sample_khop_impl(const e2egrec_csr *graph, const int32_t *seeds
 {
     if (!graph || !fanouts || !blocks || !scratch || !graph->indptr) return E2EGREC_ERR_NULL;
     if (graph->n_edges > 0 && !graph->indices) return E2EGREC_ERR_NULL;
-    if (graph->edge_weight) return E2EGREC_ERR_UNSUPPORTED;
     if (reinterpret_cast<uintptr_t>(scratch) % 256) return E2EGREC_ERR_ALIGN;
     int32_t cd[kMaxHops], cs[kMaxHops], ce[kMaxHops];
     int32_t rc = khop_caps(graph->n_nodes, n_seeds, n_hops, fanouts, cd, cs, ce);
@@ -581,7 +632,7 @@ int32_t e2egrec::sample_khop_impl(const e2egrec_csr *graph, const int32_t *seeds
         cudaMemsetAsync(s.arena, 0, s.arena_bytes, st);
         note_launch();
         hop_sample_kernel<<<grid_for(b.cap_dst, kDstTile), kDstThreads, 0, st>>>(
-            graph->indptr, graph->indices, n, dst_nodes, n_dst_ptr, b.cap_dst, b.cap_edges, f, h + 1,
+            graph->indptr, graph->indices, graph->edge_cum, n, dst_nodes, n_dst_ptr, b.cap_dst, b.cap_edges, f, h + 1,
             (uint32_t)(seed & 0xFFFFFFFFu), (uint32_t)(seed >> 32), step, s.step_offset, h == 0, b.counts, b.indptr,
             b.inv_cnt, b.src_nodes, b.nbr_global, l.edge_row, s.local_id, s.bitmap, s.tickets + 0, s.state_dst);
         note_launch();

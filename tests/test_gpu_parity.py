@@ -334,3 +334,35 @@ def test_sampling_of_the_next_batch_beside_the_current_step():
         assert int(got[i][-1][:, 3].sum()) == 0
         for a, b in zip(got[i], want[i]):
             assert torch.equal(a, b), f"step {i}"
+
+
+# ----------------------------------------------------------------------------- weighted sampling
+
+@pytest.mark.parametrize("beta", [0.0, 1.0, 2.5])
+def test_weighted_sampling_is_bit_exact(beta):
+    """Importance sampling p ~ q (Sec. 4.1): running sums built on the device, blocks against the oracle bit for bit;
+    hubs (binary search over tens of thousands of running sums), short rows taken whole, rows of weight zero."""
+    import paper_2511_20564_b200 as E
+    w = S.WORKLOADS["medium_small"]
+    indptr_h, indices_h, _ = S.build_graph(w)
+    q = S.edge_weight_units(indptr_h, w.seed, beta)
+    deg = np.diff(indptr_h)
+    hub = int(np.argmax(deg))
+    zero_row = int(np.flatnonzero(deg > 40)[3])
+    q[indptr_h[zero_row]: indptr_h[zero_row + 1]] = 0           # sums to zero: drawn uniformly
+    q[indptr_h[hub]: indptr_h[hub] + 5] = 0                      # entries that can never be drawn
+    dev = torch.device("cuda")
+    indptr, indices = torch.from_numpy(indptr_h).to(dev), torch.from_numpy(indices_h).to(dev)
+    cum = E.edge_cumulate(indptr, torch.from_numpy(q.view(np.int32)).to(dev))
+    want_cum = oracle.edge_cumulate(indptr_h, q)
+    assert np.array_equal(cum.cpu().numpy().view(np.uint64), want_cum)
+    seeds = np.unique(np.concatenate([S.seed_batch(w.n_nodes, 500, w.seed, 2), [hub, zero_row]])).astype(np.int32)
+    blocks = E.Blocks(w.n_nodes, seeds.size, w.fanouts, dev)
+    for step in (0, 9):
+        E.sample_khop(indptr, indices, torch.from_numpy(seeds).to(dev), blocks, w.seed, step, edge_cum=cum)
+        torch.cuda.synchronize()
+        want = oracle.sample_khop(indptr_h, indices_h, seeds, w.fanouts, w.seed, step, edge_cum=want_cum)
+        assert_blocks_equal(blocks.to_host(), want)
+    if beta > 0:
+        plain = oracle.sample_khop(indptr_h, indices_h, seeds, w.fanouts, w.seed, 9)
+        assert not np.array_equal(plain[0]["nbr_global"], want[0]["nbr_global"])
