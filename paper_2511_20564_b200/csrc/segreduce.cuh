@@ -398,7 +398,7 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
 }
 
 // ------------------------------------------------------------------------------------ across windows
-constexpr int kFinalWindows = 64;       // windows per block of seg_final_kernel
+constexpr int kFinalWindows = 8;        // windows per block and round of seg_final_kernel: one per warp
 constexpr int kFinalWarpParts = 64;     // longest chain of window parts that one warp adds by itself
 template <typename T, typename PtrT>
 __global__ void __launch_bounds__(kAggThreads)
@@ -468,10 +468,10 @@ seg_final_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_t
     }
     if (n_seg == 0) return;
 
-    // kFinalWindows windows per block.  A chain of up to kFinalWarpParts parts is added by one warp (the warps of
+    // kFinalWindows windows per block and round; the window blocks stride over the windows.  A chain of up to kFinalWarpParts parts is added by one warp (the warps of
     // the block work on different windows at the same time); a longer one is left to the whole block.
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t win0 = (int64_t)blockIdx.x * kFinalWindows;
+    for (int64_t win0 = (int64_t)blockIdx.x * kFinalWindows; win0 < n_windows; win0 += n_window_blocks * kFinalWindows) {
     if (threadIdx.x < kFinalWindows) {
         int32_t sg = -1;
         const int64_t wi = win0 + threadIdx.x;
@@ -558,6 +558,8 @@ seg_final_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_t
         }
         __syncthreads();
     }
+    __syncthreads();                               // sh_seg / sh_long are rewritten by the next round
+    }
 }
 
 // ------------------------------------------------------------------------------------ host
@@ -582,7 +584,7 @@ inline void launch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const
                                                sc.win_info, sc.cap_runs, seg_of, o);
     }
     tap_end(TAP_SEG_L1, st);
-    const int64_t window_blocks = ceil_div(sc.n_windows, kFinalWindows);
+    const int64_t window_blocks = std::min<int64_t>(ceil_div(sc.n_windows, kFinalWindows), 148 * 16);
     const int64_t empty_blocks = std::min<int64_t>(ceil_div(cap_seg > 0 ? cap_seg : 1, kAggThreads), 148 * 8);
     tap_begin(TAP_SEG_L3, st);
     note_launch();
