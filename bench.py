@@ -127,11 +127,11 @@ def upstream_grad(w, rows):
 
 
 # ------------------------------------------------------------------------------------------ reference arm
-def oracle_step(w, indptr, indices, X, Ws, seeds, step, dH):
+def oracle_step(w, indptr, indices, X, Ws, seeds, step, dH, edge_cum=None):
     """One oracle step.  X is the host feature table, or a callable ids -> rows (table kept elsewhere)."""
     import oracle
     bf16 = w.dtype == "bf16"
-    blocks = oracle.sample_khop(indptr, indices, seeds, w.fanouts, w.seed, step)
+    blocks = oracle.sample_khop(indptr, indices, seeds, w.fanouts, w.seed, step, edge_cum=edge_cum)
     if callable(X):
         out, ctx = oracle.sage_forward(blocks, X(blocks[-1]["src_nodes"]), Ws, bf16=bf16, gathered=True)
     else:
@@ -154,15 +154,18 @@ def run_reference(args, w):
                                 n_interactions=w.n_interactions // 100, q=w.q / 100)
         scale_note = " on a 1/100-scale graph of the same recipe"
     indptr, indices, X, Ws, inter = build_inputs(w)
+    cum = None
+    if args.beta is not None:
+        cum = oracle.edge_cumulate(indptr, S.edge_weight_units(indptr, w.seed, args.beta))
     sample = args.ref_seeds
     dH = upstream_grad(w, sample).astype(np.float64)
     batches = make_batches(w, inter, args.seeds, 0, args.warmup + args.steps)[:, :sample]
     for i in range(args.warmup):
-        oracle_step(w, indptr, indices, X, Ws, batches[i], i, dH)
+        oracle_step(w, indptr, indices, X, Ws, batches[i], i, dH, cum)
     t0 = time.perf_counter()
     edges = 0
     for i in range(args.warmup, args.warmup + args.steps):
-        edges += oracle_step(w, indptr, indices, X, Ws, batches[i], i, dH)
+        edges += oracle_step(w, indptr, indices, X, Ws, batches[i], i, dH, cum)
     dt = time.perf_counter() - t0
     val = edges / dt
     desc = f"first {sample} of the {w.batch} seeds of each step's batch, full sample+forward+backward{scale_note}"
@@ -218,6 +221,16 @@ def run_ours(args, w):
         raise RuntimeError("graph ingest: node id out of range")
     del row_d, col_d
     torch.cuda.empty_cache()
+    edge_cum = q_h = None
+    if args.beta is not None:
+        if on_device:
+            raise SystemExit("--beta is not wired for workloads drawn on the device")
+        # importance sampling p ~ omega^beta (Sec. 4.1): integer weights drawn from the row lengths alone, running sums on the device
+        deg_h = np.bincount(np.concatenate([inter[0], inter[1]]), minlength=w.n_nodes)
+        ip_h = np.zeros(w.n_nodes + 1, np.int64)
+        np.cumsum(deg_h, out=ip_h[1:])
+        q_h = S.edge_weight_units(ip_h, w.seed, args.beta)
+        edge_cum = E.edge_cumulate(indptr, torch.from_numpy(q_h.view(np.int32)).to(dev))
     # every rank trains on its own batches (data parallel replicas; no exchange on the measured path)
     if on_device:
         if args.seeds == "uniform":
@@ -255,7 +268,8 @@ def run_ours(args, w):
     count_total = torch.zeros(L, 4, dtype=torch.int64, device=dev)
 
     def sample_leg(p, defer=False):
-        E.sample_khop(indptr, indices, seeds_in2[p], blocks2[p], w.seed, 0, defer_transpose=defer)   # step = the scratch's offset
+        E.sample_khop(indptr, indices, seeds_in2[p], blocks2[p], w.seed, 0, defer_transpose=defer,
+                      edge_cum=edge_cum)                 # step = the scratch's offset
 
     def compute_leg(p):
         E.sage_forward(blocks2[p], X, Ws, ctx=ctx, H_out=H_out)
@@ -481,6 +495,7 @@ def run_ours(args, w):
                 data="synthetic",
                 config=dict(workload=w.name, nodes=w.n_nodes, csr_entries=int(indices.numel()), dim=w.dim, hidden=w.hidden,
                             layers=L, fanouts=list(w.fanouts), batch=w.batch, seeds=args.seeds,
+                            sampling="uniform" if args.beta is None else f"weighted, beta={args.beta}",
                             parallelism=f"replicas x{world}",
                             launch="one CUDA graph replay per step: forward/backward of the batch beside the sampling of "
                                    "the next batch on a second stream (two sets of block buffers)",
@@ -518,10 +533,14 @@ def run_ours(args, w):
                 X_src = lambda ids: X[torch.from_numpy(np.ascontiguousarray(ids)).to(dev).long()].float().cpu().numpy()
                 note = "; graph = host copy of the device-built CSR, feature rows fetched from the device table"
     if want_cpu:
+        cum_h = None
+        if q_h is not None:
+            import oracle
+            cum_h = oracle.edge_cumulate(indptr_h, q_h)
         t0 = time.perf_counter()
         ce, n = 0, 0
         while n < K and time.perf_counter() - t0 < 15.0:
-            ce += oracle_step(w, indptr_h, indices_h, X_src, Ws_h, seeds_h[Wm + n][:sample], Wm + n, dH64)
+            ce += oracle_step(w, indptr_h, indices_h, X_src, Ws_h, seeds_h[Wm + n][:sample], Wm + n, dH64, cum_h)
             n += 1
         cdt = time.perf_counter() - t0
         line["cpu_baseline"] = dict(value=ce / cdt, unit=UNIT, cores=1, kind="oracle",
@@ -651,6 +670,8 @@ def main():
     ap.add_argument("--ref-seeds", type=int, default=256, help="seeds per step given to the CPU oracle")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-joint", action="store_true", help="skip the joint-step measurement")
+    ap.add_argument("--beta", type=float, default=None,
+                    help="weighted neighbour sampling p ~ omega^beta with synthetic log-normal omega (default: uniform)")
     ap.add_argument("--seeds", default="activity", choices=["activity", "uniform"],
                     help="how seed batches are drawn (see make_batches)")
     args = ap.parse_args()

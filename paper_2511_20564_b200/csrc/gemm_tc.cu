@@ -105,12 +105,13 @@ __device__ inline uint64_t make_smem_desc_mn(uint32_t smem_addr, uint32_t block_
     return d;
 }
 
-// Instruction descriptor of kind::f16: bf16 x bf16 -> fp32; mn_major = both operands have their M / N
-// index contiguous in memory (a transposed product), else both are K-major.
-__device__ inline uint32_t make_idesc(int m, int n, bool mn_major = false)
+// Instruction descriptor of kind::f16: bf16 x bf16 -> fp32; a_mn_major / b_mn_major = that operand has its M / N
+// index contiguous in memory, else it is K-major.
+__device__ inline uint32_t make_idesc(int m, int n, bool a_mn_major = false, bool b_mn_major = false)
 {
     uint32_t d = 0;
-    if (mn_major) d |= (1u << 15) | (1u << 16);
+    if (a_mn_major) d |= 1u << 15;
+    if (b_mn_major) d |= 1u << 16;
     d |= 1u << 4;                    // accumulator fp32
     d |= 1u << 7;                    // A bf16
     d |= 1u << 10;                   // B bf16
@@ -177,7 +178,7 @@ __device__ inline void mbar_arrive(uint64_t *bar)
 
 __global__ void __launch_bounds__(kTnThreads)
 tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int k_blocks,
-                  int stages, int nt, int n_tiles_n, uint32_t tmem_cols, TcEpilogue ep)
+                  int stages, int nt, int n_tiles_n, uint32_t tmem_cols, int b_mn, TcEpilogue ep)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_full[2], acc_empty[2];
@@ -231,7 +232,13 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     if (!ok) break;
                     mbar_expect_tx(&full_bar[s], a_bytes + b_bytes);
                     tma_load_2d(a_tiles + (size_t)s * a_bytes, &map_a, kb * kTileK, m0, &full_bar[s]);
-                    tma_load_2d(b_tiles + (size_t)s * b_bytes, &map_b, kb * kTileK, n0, &full_bar[s]);
+                    if (b_mn) {                 // B stored [K x N]: one 64-column block of 64 K lines per copy
+                        for (int j = 0; j < nt / 64; ++j)
+                            tma_load_2d(b_tiles + (size_t)s * b_bytes + j * (kTileK * 128), &map_b, n0 + j * 64, kb * kTileK,
+                                        &full_bar[s]);
+                    } else {
+                        tma_load_2d(b_tiles + (size_t)s * b_bytes, &map_b, kb * kTileK, n0, &full_bar[s]);
+                    }
                 }
             }
             if (!ok) {
@@ -244,7 +251,7 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     } else if (warp == 1) {
         if (lane == 0) {
             // ---- MMA issuer
-            const uint32_t idesc = make_idesc(kTileM, nt);
+            const uint32_t idesc = make_idesc(kTileM, nt, false, b_mn != 0);
             uint32_t g = 0, lt = 0;
             bool ok = true;
             for (int64_t t = blockIdx.x; t < n_work && ok; t += gridDim.x, ++lt) {
@@ -263,7 +270,8 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 #pragma unroll
                     for (int k = 0; k < kTileK / kUmmaK; ++k) {
                         const uint64_t ad = make_smem_desc(a_addr + k * kUmmaK * 2);
-                        const uint64_t bd = make_smem_desc(b_addr + k * kUmmaK * 2);
+                        const uint64_t bd = b_mn ? make_smem_desc_mn(b_addr + k * kUmmaK * 128, kTileK * 128)
+                                                 : make_smem_desc(b_addr + k * kUmmaK * 2);
                         umma(d_tmem, ad, bd, idesc, (kb | k) != 0 ? 1u : 0u);
                     }
                     umma_commit(&empty_bar[s]);     // the stage is free again once these MMAs have read it
@@ -389,19 +397,24 @@ bool make_map(CUtensorMap *map, const void *base, int64_t rows, int64_t k, int64
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+bool make_map_mn(CUtensorMap *map, const void *base, int64_t rows, int64_t cols);
+
+// b_mn: B is stored [k x n] row-major (its N index contiguous) instead of [n x k]
 bool launch_tn(const __nv_bfloat16 *A, int64_t rows, int k, int64_t lda, const __nv_bfloat16 *B, int n, int64_t ldb,
-               const TcEpilogue &ep, cudaStream_t st)
+               const TcEpilogue &ep, cudaStream_t st, bool b_mn = false)
 {
     if (rows <= 0 || rows % kTileM || k % kTileK || k < kTileK) return false;
-    int nt = 0;                                 // widest tile <= 256 columns that divides n (a multiple of 32)
-    for (int c = 256; c >= 32; c -= 32)
+    int nt = 0;                                 // widest tile <= 256 columns that divides n (a multiple of 32, or of 64 for b_mn)
+    const int unit = b_mn ? 64 : 32;
+    for (int c = 256; c >= unit; c -= unit)
         if (n % c == 0) { nt = c; break; }
     if (!nt) return false;
     if (reinterpret_cast<uintptr_t>(A) % 16 || reinterpret_cast<uintptr_t>(B) % 16 || (lda * 2) % 16 || (ldb * 2) % 16 ||
         reinterpret_cast<uintptr_t>(ep.out) % 16 || (ep.ldo * 2) % 16)
         return false;
     CUtensorMap ma, mb;
-    if (!make_map(&ma, A, rows, k, lda, kTileM) || !make_map(&mb, B, n, k, ldb, nt)) return false;
+    if (!make_map(&ma, A, rows, k, lda, kTileM)) return false;
+    if (b_mn ? (ldb != n || !make_map_mn(&mb, B, k, n)) : !make_map(&mb, B, n, k, ldb, nt)) return false;
     const int k_blocks = k / kTileK;
     const int stages = k_blocks < kMaxStages ? k_blocks : kMaxStages;
     uint32_t tmem_cols = 64;                    // two accumulator buffers, each a power of two of columns >= nt
@@ -417,7 +430,7 @@ bool launch_tn(const __nv_bfloat16 *A, int64_t rows, int k, int64_t lda, const _
     const int64_t tiles_cap = (rows / kTileM) * n_tiles_n;
     const unsigned grid = (unsigned)std::min<int64_t>(tiles_cap, sm_count());
     note_launch();
-    tc_gemm_tn_kernel<<<grid, kTnThreads, smem, st>>>(ma, mb, k_blocks, stages, nt, n_tiles_n, tmem_cols, ep);
+    tc_gemm_tn_kernel<<<grid, kTnThreads, smem, st>>>(ma, mb, k_blocks, stages, nt, n_tiles_n, tmem_cols, b_mn ? 1 : 0, ep);
     return true;
 }
 
@@ -497,7 +510,7 @@ tc_gemm_rows_kernel(const __grid_constant__ CUtensorMap map_y, const __grid_cons
             issued = kb + 1;
         }
     } else if (warp == 1 && lane == 0) {
-        const uint32_t idesc = make_idesc(kTileM, nt, true);
+        const uint32_t idesc = make_idesc(kTileM, nt, true, true);
         bool ok = true;
         for (int kb = 0; kb < k_blocks && ok; ++kb) {
             const int s = kb % stages;
@@ -577,7 +590,7 @@ bool tc_update_forward(const __nv_bfloat16 *cat, int64_t rows, int k, const __nv
 
 bool tc_linear(const __nv_bfloat16 *A, int64_t rows, int k, const __nv_bfloat16 *B, int n, const float *bias, int relu,
                const __nv_bfloat16 *mask, int64_t ld_mask, __nv_bfloat16 *out, int64_t ldo, const int32_t *m_dev,
-               int32_t *status, cudaStream_t st)
+               int32_t *status, cudaStream_t st, bool b_is_k_by_n)
 {
     TcEpilogue ep{};
     ep.out = out;
@@ -588,10 +601,10 @@ bool tc_linear(const __nv_bfloat16 *A, int64_t rows, int k, const __nv_bfloat16 
     ep.ld_mask = ld_mask;
     ep.m_dev = m_dev;
     ep.status = status;
-    return launch_tn(A, rows, k, k, B, n, k, ep, st);
+    return b_is_k_by_n ? launch_tn(A, rows, k, k, B, n, n, ep, st, true) : launch_tn(A, rows, k, k, B, n, k, ep, st);
 }
 
-bool tc_dcat_backward(const __nv_bfloat16 *dz, int64_t rows, int d_out, const __nv_bfloat16 *Wt, int two_d_in,
+bool tc_dcat_backward(const __nv_bfloat16 *dz, int64_t rows, int d_out, const __nv_bfloat16 *W, int two_d_in,
                       const float *inv_cnt, __nv_bfloat16 *dcat, const int32_t *m_dev, int32_t *status, cudaStream_t st)
 {
     TcEpilogue ep{};
@@ -603,7 +616,7 @@ bool tc_dcat_backward(const __nv_bfloat16 *dz, int64_t rows, int d_out, const __
     ep.scale_from = two_d_in / 2;
     ep.m_dev = m_dev;
     ep.status = status;
-    return launch_tn(dz, rows, d_out, d_out, Wt, two_d_in, d_out, ep, st);
+    return launch_tn(dz, rows, d_out, d_out, W, two_d_in, two_d_in, ep, st, true);
 }
 
 }  // namespace e2egrec

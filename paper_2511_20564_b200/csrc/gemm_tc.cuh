@@ -12,16 +12,18 @@ namespace e2egrec {
 bool tc_update_forward(const __nv_bfloat16 *cat, int64_t rows, int k, const __nv_bfloat16 *W, int n, const float *bias,
                        int relu, __nv_bfloat16 *out, const int32_t *m_dev, int32_t *status, cudaStream_t st);
 
-// dCat = dZ Wt^T with Wt [2 d_in x d_out] (the transposed layer weight); columns >= d_in are scaled by
-// inv_cnt[row].  Same conventions as above.
-bool tc_dcat_backward(const __nv_bfloat16 *dz, int64_t rows, int d_out, const __nv_bfloat16 *Wt, int two_d_in,
+// dCat = dZ W with the layer weight W [d_out x 2 d_in] as stored (the tensor cores read it with its N index
+// contiguous, no transposed copy is made); columns >= d_in are scaled by inv_cnt[row].  2 d_in must be a multiple
+// of 64.  Same conventions as above.
+bool tc_dcat_backward(const __nv_bfloat16 *dz, int64_t rows, int d_out, const __nv_bfloat16 *W, int two_d_in,
                       const float *inv_cnt, __nv_bfloat16 *dcat, const int32_t *m_dev, int32_t *status, cudaStream_t st);
 
 // out = mask * act(A B^T + bias): A [rows x k], B [n x k], out [rows x ldo], optional mask [rows x ld_mask]
-// (outputs zeroed where mask <= 0).  Same conventions as above.
+// (outputs zeroed where mask <= 0).  With b_is_k_by_n, B is given as [k x n] row-major instead (out = A B; n a
+// multiple of 64).  Same conventions as above.
 bool tc_linear(const __nv_bfloat16 *A, int64_t rows, int k, const __nv_bfloat16 *B, int n, const float *bias, int relu,
                const __nv_bfloat16 *mask, int64_t ld_mask, __nv_bfloat16 *out, int64_t ldo, const int32_t *m_dev,
-               int32_t *status, cudaStream_t st);
+               int32_t *status, cudaStream_t st, bool b_is_k_by_n = false);
 
 // part[z] = (rows of split z of dY)^T (same rows of Xin): dY [rows x m], Xin [rows x n] bf16 row-major, part
 // [splits x m x n] fp32.  Rows between *m_dev and the next multiple of 64 must be zero in both matrices.

@@ -176,6 +176,12 @@ void linear_backward_input(const T *dY, int64_t rows, int n_out, const T *W, int
                            const int32_t *m_dev, int32_t *status, cudaStream_t st)
 {
     if (use_tc<T>()) {
+        // W [n_out x n_in] as stored is the [k x n] operand of dY W
+        if (tc_linear(reinterpret_cast<const __nv_bfloat16 *>(dY), rows, n_out, reinterpret_cast<const __nv_bfloat16 *>(W),
+                      n_in, nullptr, 0, reinterpret_cast<const __nv_bfloat16 *>(mask), n_in,
+                      reinterpret_cast<__nv_bfloat16 *>(dX), n_in, m_dev, status, st, true))
+            return;
+        // shapes the tensor-core kernel does not take in that form: through a transposed copy
         note_launch();
         transpose_kernel<T><<<dim3((unsigned)ceil_div(n_in, 32), (unsigned)ceil_div(n_out, 32)), dim3(32, 8), 0, st>>>(
             W, n_out, n_in, wt);

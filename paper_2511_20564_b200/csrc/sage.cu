@@ -227,12 +227,10 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
         if (l == 0) tap_begin(TAP_DCAT_OUTER, st);
         bool dcat_done = false;
         if (X->dtype == E2EGREC_BF16) {
-            __nv_bfloat16 *wt = reinterpret_cast<__nv_bfloat16 *>(scratch + bs.wt_off);
-            note_launch();
-            transpose_kernel<__nv_bfloat16><<<dim3((unsigned)ceil_div(two_d, 32), (unsigned)ceil_div(p.d_out, 32)), dim3(32, 8), 0, st>>>(
-                static_cast<const __nv_bfloat16 *>(W[l].data), p.d_out, two_d, wt);
-            dcat_done = tc_dcat_backward(reinterpret_cast<const __nv_bfloat16 *>(dz), p.rows, p.d_out, wt, two_d, b.inv_cnt,
-                                         reinterpret_cast<__nv_bfloat16 *>(dcat), n_dst, &b.counts[CNT_STATUS], st);
+            if (W[l].ld == two_d)               // W as stored: the product reads it with its N index contiguous
+                dcat_done = tc_dcat_backward(reinterpret_cast<const __nv_bfloat16 *>(dz), p.rows, p.d_out,
+                                             static_cast<const __nv_bfloat16 *>(W[l].data), two_d, b.inv_cnt,
+                                             reinterpret_cast<__nv_bfloat16 *>(dcat), n_dst, &b.counts[CNT_STATUS], st);
         }
         if (!dcat_done) {
             EpiDCat<T> epi{dcat, two_d, p.d_in, b.inv_cnt};

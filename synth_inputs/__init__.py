@@ -252,6 +252,12 @@ WORKLOADS = {
     "medium": Workload("medium", 200_000, 300_000, 10_000_000, 1.2, 1.2, 1, 128, 128, "bf16", (15, 10), 4096),
     "large": Workload("large", 20_000_000, 30_000_000, 1_000_000_000, 1.05, 1.05, 3, 256, 256, "bf16",
                       (20, 10, 5), 8192, q=80.0),
+    # the sampler shapes of the paper's experiments (Sec. 5.1: one hop x 100 neighbours, the default; two hops x 25, 15)
+    # on the graph and features of `medium`; one GNN layer per hop
+    "medium_1hop100": Workload("medium_1hop100", 200_000, 300_000, 10_000_000, 1.2, 1.2, 1, 128, 128, "bf16",
+                               (100,), 4096),
+    "medium_2hop25_15": Workload("medium_2hop25_15", 200_000, 300_000, 10_000_000, 1.2, 1.2, 1, 128, 128, "bf16",
+                                 (25, 15), 4096),
     # the model and batch of `large` on the graph of `medium`: same kernel shapes, a few hundred MB on the device
     "medium_wide": Workload("medium_wide", 200_000, 300_000, 10_000_000, 1.2, 1.2, 1, 256, 256, "bf16",
                             (20, 10, 5), 8192),
