@@ -353,3 +353,60 @@ def lightgcn_forward(indptr, indices, H0, n_layers, bf16=False):
         acc += H
     Y = acc / (n_layers + 1)
     return round_bf16(Y) if bf16 else Y
+
+
+def _lightgcn_block_scales(blk, inv_sqrt_deg):
+    """s_v = 1/sqrt|N(v)| for the sources, t_i = sqrt|N(i)| / |S(i)| = (1/|S(i)|) / s_i for the destinations
+    (0 for a node without neighbours).  inv_sqrt_deg is the caller's float32 table over all nodes."""
+    s = np.asarray(inv_sqrt_deg, np.float32)[blk["src_nodes"]].astype(np.float64)
+    cnt = np.diff(blk["indptr"]).astype(np.float64)
+    sd = s[: blk["n_dst"]]
+    t = np.where((cnt > 0) & (sd > 0), (1.0 / np.maximum(cnt, 1)) / np.where(sd > 0, sd, 1.0), 0.0)
+    return s, t
+
+
+def lightgcn_sampled_forward(blocks, X, inv_sqrt_deg, bf16=False, gathered=False):
+    """LightGCN (Eqs. 4-7) on sampled blocks: layer l runs on block L-l, H^0 = X rows of the outermost frontier, and
+    Y = (1/(L+1)) sum_l H^l on the seed rows (the seeds open every frontier).  Returns (Y [n_seeds x d], ctx)."""
+    L = len(blocks)
+    X = _f64(X)
+    ids = _i32(blocks[L - 1]["src_nodes"])
+    H = X.copy() if gathered else X[ids]
+    n_seeds = blocks[0]["n_dst"]
+    acc = H[:n_seeds].copy()
+    scales = []
+    for l in range(L):
+        blk = blocks[L - 1 - l]
+        s, t = _lightgcn_block_scales(blk, inv_sqrt_deg)
+        scales.append((s, t))
+        out = np.zeros((blk["n_dst"], H.shape[1]), np.float64)
+        lib().oracle_lightgcn_block_forward(_p(_i64(blk["indptr"])), _p(_i32(blk["col"])), C.c_int64(blk["n_dst"]),
+                                            _p(np.ascontiguousarray(H)), _p(s), _p(t), C.c_int32(H.shape[1]), _p(out),
+                                            C.c_int(int(bf16)))
+        H = out
+        acc += H[:n_seeds]
+    Y = acc / (L + 1)
+    return (round_bf16(Y) if bf16 else Y), dict(scales=scales)
+
+
+def lightgcn_sampled_backward(blocks, ctx, dY, bf16=False):
+    """Adjoint of lightgcn_sampled_forward with respect to the rows of the outermost frontier: dX_rows [n_src_L x d].
+    Storage points with bf16: dY/(L+1); every propagated gradient; the seed rows after dY/(L+1) is added to them."""
+    L = len(blocks)
+    dYs = _f64(dY) / (L + 1)
+    if bf16:
+        dYs = round_bf16(dYs)
+    n_seeds = blocks[0]["n_dst"]
+    G = dYs.copy()
+    for l in range(L - 1, -1, -1):
+        blk = blocks[L - 1 - l]
+        s, t = ctx["scales"][l]
+        dH = np.zeros((blk["n_src"], G.shape[1]), np.float64)
+        lib().oracle_lightgcn_block_backward(_p(_i64(blk["indptr"])), _p(_i32(blk["col"])), C.c_int64(blk["n_dst"]),
+                                             C.c_int64(blk["n_src"]), _p(np.ascontiguousarray(G)), _p(s), _p(t),
+                                             C.c_int32(G.shape[1]), _p(dH), C.c_int(int(bf16)))
+        dH[:n_seeds] += dYs
+        if bf16:
+            dH[:n_seeds] = round_bf16(dH[:n_seeds])
+        G = dH
+    return G

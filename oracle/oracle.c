@@ -463,3 +463,36 @@ void oracle_lightgcn_propagate(const int64_t *indptr, const int32_t *indices, in
         }
     }
 }
+
+/* LightGCN on sampled blocks.  One propagation over a block with destinations D and sources F:
+ *   out_i = t_i * sum_{e in S(i)} s_{col e} * H[col e],   s_v = 1/sqrt|N(v)|,   t_i = sqrt|N(i)| / |S(i)|.
+ * This is Eqs. 4-5 with the sum over N(i) estimated from the sampled multiset S(i): the factor |N(i)|/|S(i)|
+ * makes the estimate of the sum unbiased, and with S(i) = N(i) (fanout >= degree) it is A_hat exactly.
+ * s [n_src] and t [n_dst] are passed in.  With round_bf16 the result is stored as bf16. */
+void oracle_lightgcn_block_forward(const int64_t *blk_indptr, const int32_t *col, int64_t n_dst, const double *H,
+                                   const double *s, const double *t, int32_t d, double *out, int round_bf16)
+{
+    for (int64_t i = 0; i < n_dst; ++i)
+        for (int32_t k = 0; k < d; ++k) {
+            double sum = 0.0;
+            for (int64_t e = blk_indptr[i]; e < blk_indptr[i + 1]; ++e) sum += s[col[e]] * H[(int64_t)col[e] * d + k];
+            sum *= t[i];
+            out[i * d + k] = round_bf16 ? oracle_round_bf16(sum) : sum;
+        }
+}
+
+/* Its adjoint: dH_j = s_j * sum over entries (i, j) of t_i * G_i. */
+void oracle_lightgcn_block_backward(const int64_t *blk_indptr, const int32_t *col, int64_t n_dst, int64_t n_src,
+                                    const double *G, const double *s, const double *t, int32_t d, double *dH,
+                                    int round_bf16)
+{
+    for (int64_t j = 0; j < n_src * d; ++j) dH[j] = 0.0;
+    for (int64_t i = 0; i < n_dst; ++i)
+        for (int64_t e = blk_indptr[i]; e < blk_indptr[i + 1]; ++e)
+            for (int32_t k = 0; k < d; ++k) dH[(int64_t)col[e] * d + k] += t[i] * G[i * d + k];
+    for (int64_t j = 0; j < n_src; ++j)
+        for (int32_t k = 0; k < d; ++k) {
+            double v = s[j] * dH[j * d + k];
+            dH[j * d + k] = round_bf16 ? oracle_round_bf16(v) : v;
+        }
+}
