@@ -312,6 +312,24 @@ int32_t e2egrec_lightgcn_backward(int64_t n_nodes, int64_t n_entries, const int6
                                   const e2egrec_mat *dY, const e2egrec_mat *dH0, void *ws, size_t *ws_bytes,
                                   void *stream);
 
+/* LightGCN on sampled blocks (Sec. 3.1, Eqs. 4-7, on the sub-graph of Sec. 4.1; the paper's default backbone).
+ * Layer l = 0 .. L-1 runs on block L-1-l:  H^(l+1)_i = t_i * sum_{e in S(i)} s_{v(e)} H^(l)_{v(e)}  with
+ * s_v = inv_sqrt_deg[v] = 1/sqrt|N(v)| (device float[n_nodes], supplied by the caller, 0 for an isolated node) and
+ * t_i = sqrt|N(i)| / |S(i)|: the sum over N(i) of Eqs. 4-5 estimated from the sampled multiset, equal to the entry of
+ * A_hat when S(i) = N(i).  H^(0) = X rows of the outermost frontier; Y_i = (1/(L+1)) sum_{l=0..L} H^(l)_i on the seed
+ * rows i < n_seeds (Eq. 7), Y: [>= blocks[0].cap_dst x dim].  Every H^(l) is stored in X's dtype, Y is rounded once
+ * from the fp32 sum.  ctx: device buffer (size query with ctx == NULL) that keeps the scales for the backward call.
+ * e2egrec_lightgcn_sampled_backward is the adjoint with respect to those X rows: dX_rows [>= blocks[L-1].cap_src x dim],
+ * aligned with blocks[L-1].src_nodes; dY: [>= blocks[0].cap_dst x dim], rows >= n_seeds ignored.  Storage points:
+ * dY/(L+1), every propagated gradient, and the seed rows after dY/(L+1) has been added to them.  It needs the csc_*
+ * arrays of the blocks (a deferred transposition is joined first).  scratch: size query with scratch == NULL. */
+int32_t e2egrec_lightgcn_sampled_forward(const e2egrec_block *blocks, int32_t n_hops, const e2egrec_mat *X,
+                                         const float *inv_sqrt_deg, void *ctx, size_t *ctx_bytes,
+                                         const e2egrec_mat *Y, void *stream);
+int32_t e2egrec_lightgcn_sampled_backward(const e2egrec_block *blocks, int32_t n_hops, const void *ctx,
+                                          const e2egrec_mat *dY, const e2egrec_mat *dX_rows, void *scratch,
+                                          size_t *scratch_bytes, void *stream);
+
 /* e2egrec_aggregate_forward without a workspace argument (the paper has no counterpart; this is a
  * packaging variant of the call above and computes exactly the same result).
  *

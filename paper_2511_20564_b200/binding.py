@@ -68,6 +68,12 @@ def lib():
         L.e2egrec_sample_khop.argtypes = [C.POINTER(Csr), C.c_void_p, C.c_int32, C.c_int32, C.c_void_p,
                                           C.c_uint64, C.c_uint32, C.c_uint32, C.POINTER(Block), C.c_void_p,
                                           C.c_size_t, C.c_void_p]
+        L.e2egrec_lightgcn_sampled_forward.restype = C.c_int32
+        L.e2egrec_lightgcn_sampled_forward.argtypes = [C.POINTER(Block), C.c_int32, C.POINTER(Mat), C.c_void_p, C.c_void_p,
+                                                       C.POINTER(C.c_size_t), C.POINTER(Mat), C.c_void_p]
+        L.e2egrec_lightgcn_sampled_backward.restype = C.c_int32
+        L.e2egrec_lightgcn_sampled_backward.argtypes = [C.POINTER(Block), C.c_int32, C.c_void_p, C.POINTER(Mat),
+                                                        C.POINTER(Mat), C.c_void_p, C.POINTER(C.c_size_t), C.c_void_p]
         L.e2egrec_edge_cumulate.restype = C.c_int32
         L.e2egrec_edge_cumulate.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.e2egrec_sage_forward.restype = C.c_int32
@@ -513,3 +519,38 @@ def lightgcn_backward(csc_ptr, csc_row, inv_sqrt_deg, n_layers, dY, dH0=None, ws
     """Enqueues the adjoint of lightgcn_forward over the CSC arrays; returns (dH0, ws)."""
     return _lightgcn(lib().e2egrec_lightgcn_backward, "e2egrec_lightgcn_backward", csc_ptr, csc_row, inv_sqrt_deg,
                      n_layers, dY, dH0, ws, stream)
+
+
+def lightgcn_sampled_forward(blocks: Blocks, X: torch.Tensor, inv_sqrt_deg: torch.Tensor, ctx=None, Y=None, stream=None):
+    """Enqueues LightGCN on the sampled blocks (see e2egrec_lightgcn_sampled_forward); returns (Y, ctx)."""
+    assert inv_sqrt_deg.dtype == torch.float32
+    x = _mat(X)
+    n = C.c_size_t(0)
+    _check(lib().e2egrec_lightgcn_sampled_forward(blocks.c, len(blocks), C.byref(x), None, None, C.byref(n), None, None),
+           "e2egrec_lightgcn_sampled_forward(size query)")
+    if ctx is None:
+        ctx = _dev_bytes(n.value, X.device)
+    if Y is None:
+        Y = torch.zeros(blocks.caps[0][0], X.shape[1], dtype=X.dtype, device=X.device)
+    y = _mat(Y)
+    n = C.c_size_t(ctx.numel())
+    _check(lib().e2egrec_lightgcn_sampled_forward(blocks.c, len(blocks), C.byref(x), _ptr(inv_sqrt_deg), _ptr(ctx), C.byref(n),
+                                                  C.byref(y), _stream(stream)), "e2egrec_lightgcn_sampled_forward")
+    return Y, ctx
+
+
+def lightgcn_sampled_backward(blocks: Blocks, ctx: torch.Tensor, dY: torch.Tensor, dX_rows=None, scratch=None, stream=None):
+    """Enqueues the adjoint (see e2egrec_lightgcn_sampled_backward); returns (dX_rows, scratch)."""
+    dy = _mat(dY)
+    n = C.c_size_t(0)
+    _check(lib().e2egrec_lightgcn_sampled_backward(blocks.c, len(blocks), None, C.byref(dy), None, None, C.byref(n), None),
+           "e2egrec_lightgcn_sampled_backward(size query)")
+    if scratch is None:
+        scratch = _dev_bytes(n.value, dY.device)
+    if dX_rows is None:
+        dX_rows = torch.zeros(blocks.caps[-1][1], dY.shape[1], dtype=dY.dtype, device=dY.device)
+    dx = _mat(dX_rows)
+    n = C.c_size_t(scratch.numel())
+    _check(lib().e2egrec_lightgcn_sampled_backward(blocks.c, len(blocks), _ptr(ctx), C.byref(dy), C.byref(dx), _ptr(scratch),
+                                                   C.byref(n), _stream(stream)), "e2egrec_lightgcn_sampled_backward")
+    return dX_rows, scratch

@@ -366,3 +366,53 @@ def test_weighted_sampling_is_bit_exact(beta):
     if beta > 0:
         plain = oracle.sample_khop(indptr_h, indices_h, seeds, w.fanouts, w.seed, 9)
         assert not np.array_equal(plain[0]["nbr_global"], want[0]["nbr_global"])
+
+
+# ----------------------------------------------------------------------------- LightGCN on sampled blocks
+
+@pytest.mark.parametrize("dtype,d,fanouts", [("bf16", 128, (100,)), ("bf16", 64, (15, 10)), ("f32", 32, (10, 5, 3))])
+def test_lightgcn_on_sampled_blocks_forward_and_adjoint(dtype, d, fanouts):
+    """Eqs. 4-7 on the sampled sub-graph (one hop x 100 is the paper's default shape): Y on the seeds and the gradient
+    with respect to the gathered feature rows, hubs and isolated seeds included."""
+    import paper_2511_20564_b200 as E
+    base = S.WORKLOADS["medium_small"]
+    indptr_h, indices_h, _ = S.build_graph(base)
+    n = base.n_nodes
+    deg = np.diff(indptr_h)
+    bf16 = dtype == "bf16"
+    dt = torch.bfloat16 if bf16 else torch.float32
+    X_h = S.normal_features(n, d, 31)
+    if bf16:
+        X_h = S.to_bf16_values(X_h)
+    s_h = np.where(deg > 0, 1.0 / np.sqrt(np.maximum(deg, 1)), 0.0).astype(np.float32)
+    seeds = np.unique(np.concatenate([S.seed_batch(n, 700, base.seed, 4), [int(np.argmax(deg))],
+                                      np.flatnonzero(deg == 0)[:3]])).astype(np.int32)
+    dev = torch.device("cuda")
+    indptr, indices = torch.from_numpy(indptr_h).to(dev), torch.from_numpy(indices_h).to(dev)
+    blocks = E.Blocks(n, seeds.size, fanouts, dev)
+    E.sample_khop(indptr, indices, torch.from_numpy(seeds).to(dev), blocks, base.seed, 3)
+    X = torch.from_numpy(X_h).to(dev, dt)
+    Y, ctx = E.lightgcn_sampled_forward(blocks, X, torch.from_numpy(s_h).to(dev))
+    dY_h = np.random.default_rng(8).standard_normal((seeds.size, d)).astype(np.float32)
+    if bf16:
+        dY_h = S.to_bf16_values(dY_h)
+    dY = torch.zeros(Y.shape, dtype=dt, device=dev)
+    dY[: seeds.size] = torch.from_numpy(dY_h).to(dev, dt)
+    dX, _ = E.lightgcn_sampled_backward(blocks, ctx, dY)
+    torch.cuda.synchronize()
+
+    ora_blocks = oracle.sample_khop(indptr_h, indices_h, seeds, fanouts, base.seed, 3)
+    assert_blocks_equal(blocks.to_host(), ora_blocks)
+    want_Y, octx = oracle.lightgcn_sampled_forward(ora_blocks, X_h, s_h, bf16)
+    want_dX = oracle.lightgcn_sampled_backward(ora_blocks, octx, dY_h, bf16)
+    # scale of the terms behind an element: the same maps applied to the squares, with squared scales
+    s2 = (s_h.astype(np.float64) ** 2).astype(np.float32)
+    rssY = rssX = None
+    if bf16:
+        sq_blocks = ora_blocks
+        Y2, c2 = oracle.lightgcn_sampled_forward(sq_blocks, X_h.astype(np.float64) ** 2, s_h)
+        rssY = np.sqrt(np.abs(Y2)) + np.abs(want_Y)
+        rssX = np.sqrt(np.abs(oracle.lightgcn_sampled_backward(sq_blocks, c2, dY_h.astype(np.float64) ** 2))) + np.abs(want_dX)
+    assert_close("lightgcn sampled forward", Y[: seeds.size].float().cpu().numpy(), want_Y, bf16, rssY)
+    n_src = ora_blocks[-1]["n_src"]
+    assert_close("lightgcn sampled backward", dX[:n_src].float().cpu().numpy(), want_dX, bf16, rssX)
