@@ -551,6 +551,135 @@ def run_ours(args, w):
         dist.destroy_process_group()
 
 
+# ------------------------------------------------------------------------------------------ LightGCN on sampled blocks
+def run_lightgcn(args, w):
+    """Sampling + LightGCN propagation (Eqs. 4-7) on the sampled blocks + its adjoint, per step; same schedule as the
+    GraphSAGE step (the sampling of the next batch beside the propagation of the current one)."""
+    import torch
+    import paper_2511_20564_b200 as E
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    E.lib()
+    dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
+    users, items = S.bipartite_interactions(w.n_users, w.n_items, w.n_interactions, w.alpha_user, w.alpha_item, w.seed, w.q)
+    row_d = torch.cat([torch.from_numpy(users), torch.from_numpy(items)]).to(dev)
+    col_d = torch.cat([torch.from_numpy(items), torch.from_numpy(users)]).to(dev)
+    indptr, indices, st = E.graph_from_coo(w.n_nodes, row_d, col_d)
+    indices = indices.contiguous()
+    if int(st):
+        raise RuntimeError("graph ingest: node id out of range")
+    del row_d, col_d
+    deg_h = np.bincount(np.concatenate([users, items]), minlength=w.n_nodes)
+    s_h = np.where(deg_h > 0, 1.0 / np.sqrt(np.maximum(deg_h, 1)), 0.0).astype(np.float32)
+    s_d = torch.from_numpy(s_h).to(dev)
+    X_h = S.normal_features(w.n_nodes, w.dim, w.seed)
+    if w.dtype == "bf16":
+        X_h = S.to_bf16_values(X_h)
+    X = torch.from_numpy(X_h).to(dev, dt)
+    K, Wm = args.steps, args.warmup
+    seeds_h = make_batches(w, (users, items), args.seeds, 0, K + Wm + 1)
+    seeds_dev = torch.from_numpy(seeds_h).to(dev)
+    dY_h = upstream_grad(w, w.batch)[:, : w.dim] if w.hidden >= w.dim else np.zeros((w.batch, w.dim), np.float32)
+    blocks2 = [E.Blocks(w.n_nodes, w.batch, w.fanouts, dev) for _ in range(2)]
+    seeds_in2 = [torch.empty(w.batch, dtype=torch.int32, device=dev) for _ in range(2)]
+    Y = torch.zeros(blocks2[0].caps[0][0], w.dim, dtype=dt, device=dev)
+    dY = torch.zeros_like(Y)
+    dY[: w.batch] = torch.from_numpy(dY_h).to(dev, dt)
+    dX = torch.zeros(blocks2[0].caps[-1][1], w.dim, dtype=dt, device=dev)
+    _, ctx = E.lightgcn_sampled_forward(blocks2[0], X, s_d, Y=Y)
+    _, scratch = E.lightgcn_sampled_backward(blocks2[0], ctx, dY, dX_rows=dX)
+    count_total = torch.zeros(len(w.fanouts), 4, dtype=torch.int64, device=dev)
+
+    def sample_leg(p):
+        E.sample_khop(indptr, indices, seeds_in2[p], blocks2[p], w.seed, 0)
+
+    def compute_leg(p):
+        E.lightgcn_sampled_forward(blocks2[p], X, s_d, ctx=ctx, Y=Y)
+        E.lightgcn_sampled_backward(blocks2[p], ctx, dY, dX_rows=dX, scratch=scratch)
+        count_total.add_(blocks2[p].counts)
+
+    side, side2 = torch.cuda.Stream(), torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        for i in range(max(Wm, 3)):
+            for p in range(2):
+                seeds_in2[p].copy_(seeds_dev[i])
+                E.sampler_set_step(blocks2[p].scratch, i)
+                with torch.cuda.stream(side2):
+                    side2.wait_stream(side)
+                    sample_leg(p)
+                side.wait_stream(side2)
+                compute_leg(p)
+    side.synchronize()
+    graphs = []
+    l0 = E.launch_count()
+    for p in range(2):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            side2.wait_stream(side)
+            with torch.cuda.stream(side2):
+                sample_leg(1 - p)
+            compute_leg(p)
+            side.wait_stream(side2)
+        graphs.append(g)
+    kernels_per_step = (E.launch_count() - l0) // 2 + 1
+
+    def prime(i):
+        seeds_in2[i & 1].copy_(seeds_dev[i], non_blocking=True)
+        E.sampler_set_step(blocks2[i & 1].scratch, i)
+        sample_leg(i & 1)
+
+    def replay_step(i):
+        seeds_in2[(i + 1) & 1].copy_(seeds_dev[i + 1], non_blocking=True)
+        E.sampler_set_step(blocks2[(i + 1) & 1].scratch, i + 1)
+        graphs[i & 1].replay()
+
+    prime(Wm)
+    count_total.zero_()
+    clocks = ClockSampler(0)
+    clocks.start()
+    time.sleep(0.6)
+    torch.cuda.synchronize()
+    t_begin = clocks.mark()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(K):
+        replay_step(Wm + i)
+    e1.record()
+    torch.cuda.synchronize()
+    clk = clocks.stop(t_begin, clocks.mark())
+    ms = e0.elapsed_time(e1)
+    counts = count_total.cpu().numpy()
+    if counts[:, 3].any():
+        raise RuntimeError(f"device status bits set during the timed region: {counts[:, 3]}")
+    edges = int(counts[:, 2].sum())
+    line = dict(metric="sampled_lightgcn_sample_fwd_bwd_edges_per_sec", value=edges / (ms / 1e3), unit=UNIT, n_gpus=1, steps=K,
+                warmup=Wm, ms_per_step=ms / K, higher_is_better=True, scaling="weak", vs_baseline=None, dtype=w.dtype,
+                data="synthetic",
+                config=dict(workload=w.name, backbone="lightgcn", nodes=w.n_nodes, csr_entries=int(indices.numel()), dim=w.dim,
+                            layers=len(w.fanouts), fanouts=list(w.fanouts), batch=w.batch, seeds=args.seeds,
+                            launch="one CUDA graph replay per step: propagation and adjoint of the batch beside the sampling "
+                                   "of the next batch", edges_per_step=edges / K),
+                clocks=clk, gpu_launches=int(K * (kernels_per_step + 2)))
+    if not args.no_cpu_baseline:
+        import oracle
+        oracle.build()
+        row, col = S.undirected_coo(users, items)
+        indptr_h, indices_h = S.coo_to_csr(w.n_nodes, row, col)
+        sample = args.ref_seeds
+        t0 = time.perf_counter()
+        ce, n = 0, 0
+        while n < K and time.perf_counter() - t0 < 15.0:
+            blocks = oracle.sample_khop(indptr_h, indices_h, seeds_h[Wm + n][:sample], w.fanouts, w.seed, Wm + n)
+            _, octx = oracle.lightgcn_sampled_forward(blocks, X_h, s_h, w.dtype == "bf16")
+            oracle.lightgcn_sampled_backward(blocks, octx, dY_h[:sample], w.dtype == "bf16")
+            ce += sum(b["n_edges"] for b in blocks)
+            n += 1
+        cdt = time.perf_counter() - t0
+        line["cpu_baseline"] = dict(value=ce / cdt, unit=UNIT, cores=1, kind="oracle",
+                                    sample=f"{n} step(s) on the first {sample} of the {w.batch} seeds of the batch, {cdt:.1f} s")
+    print(json.dumps(line), flush=True)
+
+
 # ------------------------------------------------------------------------------------------ whole-graph aggregation
 def run_fullgraph(args):
     """Mean aggregation over the whole graph (no sampling) and its transpose: one forward (CSR gather) and one
@@ -670,6 +799,8 @@ def main():
     ap.add_argument("--ref-seeds", type=int, default=256, help="seeds per step given to the CPU oracle")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-joint", action="store_true", help="skip the joint-step measurement")
+    ap.add_argument("--backbone", default="sage", choices=["sage", "lightgcn"],
+                    help="lightgcn: sampling + LightGCN propagation on the sampled blocks + its adjoint (no weights)")
     ap.add_argument("--beta", type=float, default=None,
                     help="weighted neighbour sampling p ~ omega^beta with synthetic log-normal omega (default: uniform)")
     ap.add_argument("--seeds", default="activity", choices=["activity", "uniform"],
@@ -681,6 +812,10 @@ def main():
             run_fullgraph(args)
         return
     w = S.WORKLOADS[args.workload]
+    if args.backbone == "lightgcn":
+        if args.impl == "ours" and int(os.environ.get("RANK", "0")) == 0:
+            run_lightgcn(args, w)
+        return
     if args.impl == "reference":
         run_reference(args, w)
     else:
