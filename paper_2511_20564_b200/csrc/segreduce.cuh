@@ -112,12 +112,12 @@ constexpr size_t seg_run_smem_bytes()
     return (size_t)2 * (kAggThreads / LPR) * (LPR * CPL * E) * sizeof(float) + (size_t)(kAggThreads / LPR) * sizeof(int4);
 }
 
-// kExtra: the output has a self row and/or a mask row per segment (they are fetched together with the
-// segment's first gathered row); without it those registers and branches disappear.
+// kExtra: 1 = the output has a self row per segment, 2 = a self row and / or a mask row (they are fetched together
+// with the segment's first gathered row); 0 = neither, and those registers and branches disappear.
 // kInFlight: gathered rows a lane group requests before it adds any.  Four suit the short streams of a sampled
 // block (few resident warps, latency hidden inside the thread); on streams that fill the machine two are faster,
 // because the smaller register footprint keeps five blocks resident per SM instead of three.
-template <typename T, typename PtrT, int LPR, int CPL, bool kWeight, bool kExtra, int kInFlight>
+template <typename T, typename PtrT, int LPR, int CPL, bool kWeight, int kExtra, int kInFlight>
 __global__ void __launch_bounds__(kAggThreads, (kInFlight <= 2 && !kExtra) ? 5 : 1)
 seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__ ptr, const int32_t *__restrict__ idx,
                const int32_t *n_seg_dev, int64_t n_seg_host, const float *__restrict__ w, int run_len, int d,
@@ -153,7 +153,7 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
                 float r[E];
 #pragma unroll
                 for (int e = 0; e < E; ++e) r[e] = to_float<T>(from_float<T>(acc[q][e] * inv));   // inv = 1 without mean / scale
-                if (kExtra && o.mask) {
+                if (kExtra == 2 && o.mask) {
                     float m[E];
                     Chunk<T>::unpack(mrow[q], m);
 #pragma unroll
@@ -254,7 +254,7 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
             int32_t seg_c[U];
             bool start_c[U];
             float wt[U];
-            uint4 v[U][CPL], sv[kExtra ? U : 1][CPL], mv[kExtra ? U : 1][CPL];
+            uint4 v[U][CPL], sv[kExtra ? U : 1][CPL], mv[kExtra == 2 ? U : 1][CPL];
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 seg_c[u] = seg_n[u];
@@ -270,12 +270,13 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
                     if (live && ch < n_chunks) v[u][q] = Chunk<T>::load_raw(in + (int64_t)id * ld_in + ch * E);
                     if (kExtra) {
                         sv[u][q] = make_uint4(0, 0, 0, 0);
-                        mv[u][q] = make_uint4(0, 0, 0, 0);
+                        if (kExtra == 2) mv[u][q] = make_uint4(0, 0, 0, 0);
                         if (live && start_c[u] && ch < n_chunks) {
                             const bool begins = r0 + u != 0 || first_begins;
                             if (begins && seg_c[u] < n_self)
                                 sv[u][q] = Chunk<T>::load_raw(o.self + (int64_t)seg_c[u] * o.ld_self + ch * E);
-                            if (o.mask) mv[u][q] = Chunk<T>::load_raw(o.mask + (int64_t)seg_c[u] * o.ld_mask + ch * E);
+                            if (kExtra == 2 && o.mask)
+                                mv[u][q] = Chunk<T>::load_raw(o.mask + (int64_t)seg_c[u] * o.ld_mask + ch * E);
                         }
                     }
                 }
@@ -293,7 +294,7 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
                         for (int q = 0; q < CPL; ++q) {
                             if (kExtra) {
                                 Chunk<T>::unpack(sv[u][q], acc[q]);          // the self row (zeros if there is none)
-                                cur_mask[q] = mv[u][q];
+                                if (kExtra == 2) cur_mask[q] = mv[u][q];
                             } else {
 #pragma unroll
                                 for (int e = 0; e < E; ++e) acc[q][e] = 0.f;
@@ -353,7 +354,7 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
                 float inv = 1.0f;
                 if (o.mean) inv = 1.0f / (float)((int64_t)ptr[sg + 1] - (int64_t)ptr[sg]);
                 else if (o.seg_scale) inv = o.seg_scale[sg];
-                if (kExtra && o.mask) {
+                if (kExtra == 2 && o.mask) {
 #pragma unroll
                     for (int q = 0; q < CPL; ++q) {
                         const int ch = c + q * LPR;
@@ -572,13 +573,18 @@ inline void launch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const
     tap_begin(TAP_SEG_L1, st);
     note_launch();
     const unsigned grid1 = (unsigned)sc.n_windows;
-    if (o.self || o.mask) {
-        auto kern = seg_run_kernel<T, PtrT, LPR, CPL, kWeight, true, kInFlight>;
+    if (o.mask) {
+        auto kern = seg_run_kernel<T, PtrT, LPR, CPL, kWeight, 2, kInFlight>;
+        if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        kern<<<grid1, kAggThreads, smem, st>>>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head2, sc.tail2,
+                                               sc.win_info, sc.cap_runs, seg_of, o);
+    } else if (o.self) {
+        auto kern = seg_run_kernel<T, PtrT, LPR, CPL, kWeight, 1, kInFlight>;
         if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         kern<<<grid1, kAggThreads, smem, st>>>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head2, sc.tail2,
                                                sc.win_info, sc.cap_runs, seg_of, o);
     } else {
-        auto kern = seg_run_kernel<T, PtrT, LPR, CPL, kWeight, false, kInFlight>;
+        auto kern = seg_run_kernel<T, PtrT, LPR, CPL, kWeight, 0, kInFlight>;
         if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         kern<<<grid1, kAggThreads, smem, st>>>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head2, sc.tail2,
                                                sc.win_info, sc.cap_runs, seg_of, o);
