@@ -157,7 +157,7 @@ def _powerlaw_graph(n, m, seed):
     return S.coo_to_csr(n, dst, src)
 
 
-@pytest.mark.parametrize("dtype,d", [("bf16", 64), ("f32", 32), ("bf16", 256)])
+@pytest.mark.parametrize("dtype,d", [("bf16", 64), ("f32", 32), ("bf16", 256), ("f32", 512), ("bf16", 1024)])
 def test_full_graph_aggregation_forward_and_transpose(dtype, d):
     """Rows with tens of thousands of entries (split over many warps), empty rows, and a ragged tail."""
     import paper_2511_20564_b200 as E
@@ -220,6 +220,20 @@ def test_three_hops_wide_rows_bf16():
     w = S.Workload("large_shape", base.n_users, base.n_items, base.n_interactions, 1.05, 1.05, 3, 256, 256, "bf16",
                    (20, 10, 5), 128)
     case = Case(w, step=0)
+    dH = case.upstream_grad(case.seeds.size, w.hidden)
+    ora = case.run_oracle(dH)
+    gpu = case.run_gpu(dH)
+    assert_blocks_equal(gpu["blocks"], ora["blocks"])
+    _check_float(case, gpu, ora)
+
+
+@pytest.mark.parametrize("dtype,d,fanouts", [("bf16", 512, (6, 4)), ("f32", 256, (3, 3, 3, 3))])
+def test_widest_rows_and_four_hops(dtype, d, fanouts):
+    """Rows of 1 024 bytes (several 16-byte chunks per lane, the large shared-memory form of the segment kernel) and the
+    largest number of hops the library takes."""
+    base = S.WORKLOADS["medium_small"]
+    w = S.Workload("wide", base.n_users, base.n_items, base.n_interactions, 1.2, 1.2, 1, d, d, dtype, fanouts, 48)
+    case = Case(w, step=2)
     dH = case.upstream_grad(case.seeds.size, w.hidden)
     ora = case.run_oracle(dH)
     gpu = case.run_gpu(dH)
