@@ -199,7 +199,7 @@ def run_ours(args, w):
     want_cpu = world == 1 and not args.no_cpu_baseline
     dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
     K, Wm = args.steps, args.warmup
-    total = K + Wm + 1                                 # + the batch whose sampling is prefetched during the last step
+    total = K + Wm + 2                                 # + the batches whose sampling / upload is prefetched during the last steps
     first_step = rank * 1_000_000                      # = replicas.first_step_of(rank)
     on_device = w.n_interactions > 200_000_000         # too large for host-side generation: drawn with torch on the GPU
     t_setup = time.perf_counter()
@@ -258,13 +258,18 @@ def run_ours(args, w):
     blocks = blocks2[0]
     L = len(Ws)
     ctx = torch.empty(E.binding.sage_forward_ctx_bytes(blocks, X, Ws), dtype=torch.uint8, device=dev)
-    H_out = torch.zeros(blocks.caps[0][0], w.hidden, dtype=dt, device=dev)
+    # outputs, the upstream gradient and a snapshot of the block counts exist once per buffer set, so that the copies
+    # of one step's results and of the next step's inputs can run beside the step in between
+    H_out2 = [torch.zeros(blocks.caps[0][0], w.hidden, dtype=dt, device=dev) for _ in range(2)]
+    H_out = H_out2[0]
     scratch = torch.empty(E.binding.sage_backward_scratch_bytes(blocks, X, Ws), dtype=torch.uint8, device=dev)
-    dWs = [torch.zeros(W.shape, dtype=torch.float32, device=dev) for W in Ws]
+    dWs2 = [[torch.zeros(W.shape, dtype=torch.float32, device=dev) for W in Ws] for _ in range(2)]
+    dWs = dWs2[0]
     dX = torch.zeros(blocks.caps[L - 1][1], w.dim, dtype=dt, device=dev)
 
     seeds_in2 = [torch.empty(w.batch, dtype=torch.int32, device=dev) for _ in range(2)]
-    dH_in = torch.empty_like(dH)
+    dH_in2 = [torch.empty_like(dH) for _ in range(2)]
+    counts_snap2 = [torch.zeros(L, 4, dtype=torch.int32, device=dev) for _ in range(2)]
     count_total = torch.zeros(L, 4, dtype=torch.int64, device=dev)
 
     def sample_leg(p, defer=False):
@@ -272,9 +277,10 @@ def run_ours(args, w):
                       edge_cum=edge_cum)                 # step = the scratch's offset
 
     def compute_leg(p):
-        E.sage_forward(blocks2[p], X, Ws, ctx=ctx, H_out=H_out)
-        E.sage_backward(blocks2[p], X, Ws, ctx, dH_in, dWs=dWs, dX_rows=dX, scratch=scratch)
+        E.sage_forward(blocks2[p], X, Ws, ctx=ctx, H_out=H_out2[p])
+        E.sage_backward(blocks2[p], X, Ws, ctx, dH_in2[p], dWs=dWs2[p], dX_rows=dX, scratch=scratch)
         count_total.add_(blocks2[p].counts)
+        counts_snap2[p].copy_(blocks2[p].counts)
 
     def step_body():
         """Everything of one training step back to back on fixed buffers (used for warm-up and per-kernel timing)."""
@@ -289,7 +295,8 @@ def run_ours(args, w):
     # ---- record the step as CUDA graphs (no host work between the kernels) and replay them.  Graph p holds the
     # forward/backward of the batch in buffer p and, on a second stream, the sampling of the next batch into buffer 1-p.
     side, side2 = torch.cuda.Stream(), torch.cuda.Stream()
-    dH_in.copy_(dH)
+    for t in dH_in2:
+        t.copy_(dH)
     with torch.cuda.stream(side):
         for i in range(Wm):                              # eager warm-up on the capture stream
             seeds_in2[0].copy_(seeds_dev[i])
@@ -314,7 +321,7 @@ def run_ours(args, w):
             compute_leg(p)
             side.wait_stream(side2)
         graphs.append(g)
-        kernels_per_step = E.launch_count() - launches_before + 1   # + the counter update (a torch kernel)
+        kernels_per_step = E.launch_count() - launches_before + 2   # + the counter update and snapshot (torch kernels)
 
     ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     ev_a.record(); ev_b.record()
@@ -378,32 +385,60 @@ def run_ours(args, w):
         dom_ms.append(tapped_step(Wm + i, dominant))
     outer_counts = count_total.cpu().numpy()[L - 1] / (K + len(dom_ms))
 
-    # ---- end to end: host buffers in, results out, every step
-    res_pin = [torch.empty(H_out.shape, dtype=dt).pin_memory()] + [torch.empty(W.shape, dtype=torch.float32).pin_memory()
-                                                                   for W in Ws]
-    cnt_pin = torch.empty(L, 4, dtype=torch.int32).pin_memory()
+    # ---- end to end: host buffers in, results out, every step.  Three streams: the step itself; the upload of the
+    # next step's inputs (seeds of the batch sampled next, upstream gradient) while the step runs; the download of
+    # the step's results while the next step runs.  The host reads the results of step i while step i + 1 runs.
+    res_pin2 = [[torch.empty(H_out.shape, dtype=dt).pin_memory()] +
+                [torch.empty(W.shape, dtype=torch.float32).pin_memory() for W in Ws] for _ in range(2)]
+    cnt_pin2 = [torch.empty(L, 4, dtype=torch.int32).pin_memory() for _ in range(2)]
     h2d = seeds_pin[0].numel() * 4 + dH_pin.numel() * dH_pin.element_size()
-    d2h = sum(t.numel() * t.element_size() for t in res_pin) + cnt_pin.numel() * 4
+    d2h = sum(t.numel() * t.element_size() for t in res_pin2[0]) + cnt_pin2[0].numel() * 4
+    main_s = torch.cuda.current_stream()
+    up_s, down_s = torch.cuda.Stream(), torch.cuda.Stream()
+    ev = lambda: torch.cuda.Event()
+    done_ev, up_ev, out_ev = [ev(), ev()], [ev(), ev()], [ev(), ev()]
 
-    def e2e_step(i):
-        dH_in.copy_(dH_pin, non_blocking=True)
-        replay_step(i, seeds_pin)                      # copies the seeds of batch i + 1 from pinned host memory
-        res_pin[0].copy_(H_out, non_blocking=True)
-        for t, s in zip(res_pin[1:], dWs):
-            t.copy_(s, non_blocking=True)
-        cnt_pin.copy_(blocks2[i & 1].counts, non_blocking=True)
-        torch.cuda.current_stream().synchronize()      # the caller reads the results of this step
-        return int(cnt_pin[:, 2].sum())
+    def e2e_run(first, count):
+        """Steps first .. first + count - 1; returns the edges their results report."""
+        edges = 0
+        prime(first, seeds_pin)                                     # batch `first` sampled into its buffer
+        with torch.cuda.stream(up_s):
+            up_s.wait_stream(main_s)
+            seeds_in2[(first + 1) & 1].copy_(seeds_pin[first + 1], non_blocking=True)
+            dH_in2[first & 1].copy_(dH_pin, non_blocking=True)
+            up_ev[first & 1].record(up_s)
+        for i in range(first, first + count):
+            p = i & 1
+            main_s.wait_event(up_ev[p])                              # inputs of step i are on the device
+            E.sampler_set_step(blocks2[1 - p].scratch, first_step + i + 1)
+            graphs[p].replay()
+            done_ev[p].record(main_s)
+            with torch.cuda.stream(up_s):                            # inputs of step i + 1, beside step i
+                if i > first:
+                    up_s.wait_event(done_ev[1 - p])                  # step i - 1 no longer reads these buffers
+                seeds_in2[p].copy_(seeds_pin[i + 2], non_blocking=True)
+                dH_in2[1 - p].copy_(dH_pin, non_blocking=True)
+                up_ev[1 - p].record(up_s)
+            with torch.cuda.stream(down_s):                          # results of step i, beside step i + 1
+                down_s.wait_event(done_ev[p])
+                res_pin2[p][0].copy_(H_out2[p], non_blocking=True)
+                for t, src in zip(res_pin2[p][1:], dWs2[p]):
+                    t.copy_(src, non_blocking=True)
+                cnt_pin2[p].copy_(counts_snap2[p], non_blocking=True)
+                out_ev[p].record(down_s)
+            if i > first:                                            # the caller reads the results of step i - 1
+                out_ev[1 - p].synchronize()
+                edges += int(cnt_pin2[1 - p][:, 2].sum())
+        last = (first + count - 1) & 1
+        out_ev[last].synchronize()
+        edges += int(cnt_pin2[last][:, 2].sum())
+        torch.cuda.synchronize()
+        return edges
 
-    prime(0, seeds_pin)
-    for i in range(min(Wm, 3)):
-        e2e_step(i)
-    prime(Wm, seeds_pin)
+    e2e_run(0, min(Wm, 3))
     barrier()
     t0 = time.perf_counter()
-    e2e_edges = 0
-    for i in range(K):
-        e2e_edges += e2e_step(Wm + i)
+    e2e_edges = e2e_run(Wm, K)
     barrier()
     e2e_s = time.perf_counter() - t0
 
