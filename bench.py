@@ -447,7 +447,7 @@ def run_ours(args, w):
     if not args.no_joint and not on_device:
         P, dd = w.batch, 64
         jr = np.random.default_rng(4 + rank)
-        picks = jr.integers(0, inter[0].size, (min(K, 200) + Wm, P))
+        picks = jr.integers(0, inter[0].size, (min(K, 200) + Wm + 1, P))
         pu_all = torch.from_numpy(inter[0][picks].astype(np.int32)).to(dev)
         pi_all = torch.from_numpy(inter[1][picks].astype(np.int32)).to(dev)
         dense = torch.from_numpy(jr.standard_normal((P, dd)).astype(np.float32)).to(dev)
@@ -456,34 +456,64 @@ def run_ours(args, w):
         Wt_h = [S.glorot_uniform(512, zdim, 4, 40), S.glorot_uniform(256, 512, 4, 41), S.glorot_uniform(1, 256, 4, 42)]
         Wt = [torch.from_numpy(a).to(dev, dt) for a in Wt_h]
         bt = [torch.zeros(a.shape[0], dtype=torch.float32, device=dev) for a in Wt_h]
-        js = E.JointStep(indptr, indices, X, P, dd, w.fanouts, Ws, Wt, bt)
-        pu_in, pi_in = torch.empty_like(pu_all[0]), torch.empty_like(pi_all[0])
+        # two workspaces: the pairs of the next step are turned into seeds and sampled (phase 1) on a second stream
+        # while the rest of the current step (phase 2) runs
+        js2 = [E.JointStep(indptr, indices, X, P, dd, w.fanouts, Ws, Wt, bt) for _ in range(2)]
+        pu_in2 = [torch.empty_like(pu_all[0]) for _ in range(2)]
+        pi_in2 = [torch.empty_like(pi_all[0]) for _ in range(2)]
+
+        def j_sample(p):
+            js2[p].run(pu_in2[p], pi_in2[p], dense, labels, 4, 0, phase=1)
+
+        def j_compute(p):
+            js2[p].run(pu_in2[p], pi_in2[p], dense, labels, 4, 0, phase=2)
+
         with torch.cuda.stream(side):
             for i in range(Wm):
-                pu_in.copy_(pu_all[i]); pi_in.copy_(pi_all[i])
-                js.run(pu_in, pi_in, dense, labels, 4, i)
+                for p in range(2):
+                    pu_in2[p].copy_(pu_all[i]); pi_in2[p].copy_(pi_all[i])
+                    E.sampler_set_step(js2[p].ws, first_step + i)
+                    with torch.cuda.stream(side2):
+                        side2.wait_stream(side)
+                        j_sample(p)
+                    side.wait_stream(side2)
+                    j_compute(p)
         side.synchronize()
-        jgraph = torch.cuda.CUDAGraph()
-        with torch.cuda.graph(jgraph, stream=side):
-            js.run(pu_in, pi_in, dense, labels, 4, 0)
-        KJ = picks.shape[0] - Wm
+        jgraphs = []
+        for p in range(2):
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=side):
+                side2.wait_stream(side)
+                with torch.cuda.stream(side2):
+                    j_sample(1 - p)
+                j_compute(p)
+                side.wait_stream(side2)
+            jgraphs.append(g)
+        KJ = picks.shape[0] - Wm - 1
+        # batch Wm sampled ahead, as the previous replay would have done
+        pu_in2[Wm & 1].copy_(pu_all[Wm]); pi_in2[Wm & 1].copy_(pi_all[Wm])
+        E.sampler_set_step(js2[Wm & 1].ws, first_step + Wm)
+        j_sample(Wm & 1)
         barrier()
         j0, j1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         j0.record()
-        for i in range(KJ):
-            pu_in.copy_(pu_all[Wm + i], non_blocking=True)
-            pi_in.copy_(pi_all[Wm + i], non_blocking=True)
-            E.sampler_set_step(js.ws, first_step + i)
-            jgraph.replay()
+        for i in range(Wm, Wm + KJ):
+            q = (i + 1) & 1
+            pu_in2[q].copy_(pu_all[i + 1], non_blocking=True)
+            pi_in2[q].copy_(pi_all[i + 1], non_blocking=True)
+            E.sampler_set_step(js2[q].ws, first_step + i + 1)
+            jgraphs[i & 1].replay()
         j1.record()
         barrier()
         jms = j0.elapsed_time(j1)
+        js = js2[(Wm + KJ - 1) & 1]
         n_rows, jstatus = js.n_rows.tolist()
-        if jstatus:
+        if jstatus or js2[0].n_rows.tolist()[1] or js2[1].n_rows.tolist()[1]:
             raise RuntimeError(f"joint step: device status bits {jstatus}")
         joint = dict(metric="joint_step_samples_per_sec", value=KJ * P * world / (jms / 1e3), unit="pairs/s",
                      ms_per_step=jms / KJ, steps=KJ, pairs_per_step=P, tower="320-512-256-1", dense_dim=dd,
-                     loss=float(js.loss), launch="one CUDA graph replay per step")
+                     loss=float(js.loss),
+                     launch="one CUDA graph replay per step: e2egrec_joint_step_phase COMPUTE of the batch beside SAMPLE of the next")
 
     # ---- reduce over ranks: slowest rank's time, all ranks' edges
     from paper_2511_20564_b200 import replicas

@@ -275,6 +275,24 @@ int32_t e2egrec_joint_step(const e2egrec_csr *graph, const e2egrec_mat *X, const
                            float *const *dW_tower, float *const *db_tower, const e2egrec_mat *dX_rows,
                            int32_t *dX_ids, int32_t *n_dX_rows, void *ws, size_t *ws_bytes, void *stream);
 
+/* The joint step in two phases, for callers that prepare the sub-graph of the next batch (Sec. 4.1: "constructed in
+ * real time") while the current batch trains: phase E2EGREC_JOINT_SAMPLE derives the seeds from the pairs and samples
+ * the blocks into ws (only graph, the pairs, fanouts, seed, step and ws are read; the other arguments fix the layout
+ * of ws and must be the ones of the later call); phase E2EGREC_JOINT_COMPUTE runs everything else of
+ * e2egrec_joint_step on the blocks that a SAMPLE call with the same shapes left in ws (the two calls may be issued
+ * on different streams; the caller orders them).  E2EGREC_JOINT_WHOLE is e2egrec_joint_step. */
+#define E2EGREC_JOINT_WHOLE   0u
+#define E2EGREC_JOINT_SAMPLE  1u
+#define E2EGREC_JOINT_COMPUTE 2u
+int32_t e2egrec_joint_step_phase(const e2egrec_csr *graph, const e2egrec_mat *X, const int32_t *pair_user,
+                                 const int32_t *pair_item, int32_t n_pairs, const float *dense, int32_t dense_dim,
+                                 const float *labels, int32_t n_hops, const int32_t *fanouts,
+                                 const e2egrec_mat *W_gnn, const e2egrec_mat *W_tower, const float *const *b_tower,
+                                 uint64_t seed, uint32_t step, float *loss, float *logits, float *const *dW_gnn,
+                                 float *const *dW_tower, float *const *db_tower, const e2egrec_mat *dX_rows,
+                                 int32_t *dX_ids, int32_t *n_dX_rows, void *ws, size_t *ws_bytes, uint32_t phase,
+                                 void *stream);
+
 /* Whole-graph neighbourhood aggregation without sampling (Sec. 3.1 Eq. 2 with S(u) = N(u); the
  * "complete graph" case of Sec. 4.1):  out[i] = (1/deg i) sum_{e in row i} X[indices[e]]  (0 for an
  * empty row; the plain sum with E2EGREC_AGG_SUM).  indptr: device int64[n_dst+1], indices: device

@@ -106,6 +106,8 @@ def lib():
                                          C.c_void_p, C.c_uint64, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
                                          C.c_void_p, C.c_void_p, C.POINTER(Mat), C.c_void_p, C.c_void_p, C.c_void_p,
                                          C.POINTER(C.c_size_t), C.c_void_p]
+        L.e2egrec_joint_step_phase.restype = C.c_int32
+        L.e2egrec_joint_step_phase.argtypes = L.e2egrec_joint_step.argtypes[:-1] + [C.c_uint32, C.c_void_p]
         L.e2egrec_graph_from_coo.restype = C.c_int32
         L.e2egrec_graph_from_coo.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                              C.c_void_p, C.c_void_p, C.POINTER(C.c_size_t), C.c_void_p]
@@ -442,17 +444,19 @@ class JointStep:
         self.ws = _dev_bytes(n.value, dev)
         sampler_scratch_init(self.n_nodes, self.ws)
 
-    def _call(self, user, item, dense, labels, nbytes, stream, seed, step):
+    def _call(self, user, item, dense, labels, nbytes, stream, seed, step, phase=0):
         L = len(self.fanouts)
-        _check(lib().e2egrec_joint_step(
+        _check(lib().e2egrec_joint_step_phase(
             C.byref(self._g), C.byref(self._x), _ptr(user), _ptr(item), self.n_pairs, _ptr(dense), self.dense_dim,
             _ptr(labels), L, self._f, self._wg, self._wt, _ptr_array(self.b_tower, 3), C.c_uint64(seed),
             C.c_uint32(step), _ptr(self.loss), _ptr(self.logits), _ptr_array(self.dW_gnn, L),
             _ptr_array(self.dW_tower, 3), _ptr_array(self.db_tower, 3), C.byref(self._dx), _ptr(self.dX_ids),
-            _ptr(self.n_rows), None if user is None else _ptr(self.ws), C.byref(nbytes), stream), "e2egrec_joint_step")
+            _ptr(self.n_rows), None if user is None else _ptr(self.ws), C.byref(nbytes), C.c_uint32(phase), stream),
+            "e2egrec_joint_step_phase")
 
-    def run(self, pair_user, pair_item, dense, labels, seed, step, stream=None):
-        self._call(pair_user, pair_item, dense, labels, C.c_size_t(self.ws.numel()), _stream(stream), seed, step)
+    def run(self, pair_user, pair_item, dense, labels, seed, step, stream=None, phase=0):
+        """phase 0: the whole step; 1: seeds + sampling only; 2: everything else, on the blocks phase 1 left in ws."""
+        self._call(pair_user, pair_item, dense, labels, C.c_size_t(self.ws.numel()), _stream(stream), seed, step, phase)
         return self
 
 

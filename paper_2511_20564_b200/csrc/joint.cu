@@ -315,7 +315,7 @@ int32_t run_joint(const JointPlan &jp, const e2egrec_csr *graph, const e2egrec_m
                   const e2egrec_mat *W_gnn, const e2egrec_mat *W_tower, const float *const *b_tower, uint64_t seed,
                   uint32_t step, float *loss, float *logits, float *const *dW_gnn, float *const *dW_tower,
                   float *const *db_tower, const e2egrec_mat *dX_rows, int32_t *dX_ids, int32_t *n_dX_rows, char *ws,
-                  cudaStream_t st)
+                  uint32_t phase, cudaStream_t st)
 {
     e2egrec_block blocks[kMaxHops];
     fill_blocks(jp, ws, blocks);
@@ -339,11 +339,17 @@ int32_t run_joint(const JointPlan &jp, const e2egrec_csr *graph, const e2egrec_m
     pi.pcsc_col = i32(jp.pcsc_col_off);
     pi.units_per_row = jp.zdim / jp.unit;
     pi.item_unit_off = jp.dL / jp.unit;
-    int32_t rc = sample_khop_impl(graph, nullptr, jp.P2, &pi, jp.n_hops, fanouts, seed, step, E2EGREC_SAMPLE_DEFER_TRANSPOSE, blocks, ws,
-                                  jp.sampler_bytes, st);
-    if (rc != E2EGREC_OK) return rc;
-    note_launch();
-    joint_meta_kernel<<<1, 1, 0, st>>>(pmeta, jp.P);
+    int32_t rc = E2EGREC_OK;
+    if (phase != E2EGREC_JOINT_COMPUTE) {
+        // alone, the sampling phase completes the block transposition before it returns (the other phase may run
+        // on another stream); inside a whole step the transposition is joined by the encoder backward
+        rc = sample_khop_impl(graph, nullptr, jp.P2, &pi, jp.n_hops, fanouts, seed, step,
+                              phase == E2EGREC_JOINT_SAMPLE ? 0u : E2EGREC_SAMPLE_DEFER_TRANSPOSE, blocks, ws, jp.sampler_bytes, st);
+        if (rc != E2EGREC_OK) return rc;
+        note_launch();
+        joint_meta_kernel<<<1, 1, 0, st>>>(pmeta, jp.P);
+        if (phase == E2EGREC_JOINT_SAMPLE) return check_launch("joint_step(sample)");
+    }
 
     // 2. encoder forward: embeddings of the seeds
     e2egrec_mat Hs{tp(jp.hseed_off), pad128(jp.cd[0]), jp.dL, jp.dL, X->dtype};
@@ -432,7 +438,22 @@ extern "C" int32_t e2egrec_joint_step(const e2egrec_csr *graph, const e2egrec_ma
                                       float *const *dW_tower, float *const *db_tower, const e2egrec_mat *dX_rows,
                                       int32_t *dX_ids, int32_t *n_dX_rows, void *ws, size_t *ws_bytes, void *stream)
 {
+    return e2egrec_joint_step_phase(graph, X, pair_user, pair_item, n_pairs, dense, dense_dim, labels, n_hops, fanouts, W_gnn,
+                                    W_tower, b_tower, seed, step, loss, logits, dW_gnn, dW_tower, db_tower, dX_rows, dX_ids,
+                                    n_dX_rows, ws, ws_bytes, E2EGREC_JOINT_WHOLE, stream);
+}
+
+extern "C" int32_t e2egrec_joint_step_phase(const e2egrec_csr *graph, const e2egrec_mat *X, const int32_t *pair_user,
+                                            const int32_t *pair_item, int32_t n_pairs, const float *dense,
+                                            int32_t dense_dim, const float *labels, int32_t n_hops,
+                                            const int32_t *fanouts, const e2egrec_mat *W_gnn, const e2egrec_mat *W_tower,
+                                            const float *const *b_tower, uint64_t seed, uint32_t step, float *loss,
+                                            float *logits, float *const *dW_gnn, float *const *dW_tower,
+                                            float *const *db_tower, const e2egrec_mat *dX_rows, int32_t *dX_ids,
+                                            int32_t *n_dX_rows, void *ws, size_t *ws_bytes, uint32_t phase, void *stream)
+{
     if (!ws_bytes) return E2EGREC_ERR_NULL;
+    if (phase > E2EGREC_JOINT_COMPUTE) return E2EGREC_ERR_ARG;
     JointPlan jp{};
     int32_t rc = make_plan(graph, X, n_pairs, dense_dim, n_hops, fanouts, W_gnn, W_tower, jp);
     if (rc != E2EGREC_OK) return rc;
@@ -450,7 +471,7 @@ extern "C" int32_t e2egrec_joint_step(const e2egrec_csr *graph, const e2egrec_ma
     if (X->dtype == E2EGREC_BF16)
         return run_joint<__nv_bfloat16>(jp, graph, X, pair_user, pair_item, dense, labels, fanouts, W_gnn, W_tower, b_tower, seed,
                                         step, loss, logits, dW_gnn, dW_tower, db_tower, dX_rows, dX_ids, n_dX_rows,
-                                        static_cast<char *>(ws), st);
+                                        static_cast<char *>(ws), phase, st);
     return run_joint<float>(jp, graph, X, pair_user, pair_item, dense, labels, fanouts, W_gnn, W_tower, b_tower, seed, step, loss,
-                            logits, dW_gnn, dW_tower, db_tower, dX_rows, dX_ids, n_dX_rows, static_cast<char *>(ws), st);
+                            logits, dW_gnn, dW_tower, db_tower, dX_rows, dX_ids, n_dX_rows, static_cast<char *>(ws), phase, st);
 }

@@ -85,3 +85,32 @@ def _check_grad(name, got, want, bf16):
     tol = 1e-3 + 2e-2 * np.abs(want) + 2e-2 * scale
     frac = np.mean(np.abs(got - want) <= tol)
     assert frac >= 0.99, f"{name}: only {frac:.4f} of the elements within tolerance"
+
+
+def test_joint_step_in_two_phases_equals_the_whole_step():
+    """Sampling of a batch on one stream, the rest of its step on another (as a caller that prepares the next batch
+    during the current one would issue them): bit-identical to the single call."""
+    import paper_2511_20564_b200 as E
+    w = S.WORKLOADS["medium_small"]
+    args = _inputs(w, 512, 64, 512, 256, 11)
+    indptr, indices, X, W_gnn, pu, pi, dense, labels, W_t, b_t = args
+    whole = _run_gpu(w, *args, 5)
+    dt = torch.bfloat16
+    cu = lambda a, t=None: torch.from_numpy(np.ascontiguousarray(a)).cuda().to(t) if t else torch.from_numpy(np.ascontiguousarray(a)).cuda()
+    js = E.JointStep(cu(indptr), cu(indices), cu(X, dt), pu.size, dense.shape[1], w.fanouts, [cu(W, dt) for W in W_gnn],
+                     [cu(W, dt) for W in W_t], [cu(b) for b in b_t])
+    pu_d, pi_d, dense_d, labels_d = cu(pu), cu(pi), cu(dense), cu(labels)
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    with torch.cuda.stream(s2):
+        js.run(pu_d, pi_d, dense_d, labels_d, w.seed, 5, phase=1)
+    s1.wait_stream(s2)
+    with torch.cuda.stream(s1):
+        js.run(pu_d, pi_d, dense_d, labels_d, w.seed, 5, phase=2)
+    torch.cuda.synchronize()
+    assert js.n_rows.tolist() == whole.n_rows.tolist() and js.n_rows.tolist()[1] == 0
+    n_rows = js.n_rows.tolist()[0]
+    assert torch.equal(js.loss, whole.loss) and torch.equal(js.logits, whole.logits)
+    assert torch.equal(js.dX_ids[:n_rows], whole.dX_ids[:n_rows]) and torch.equal(js.dX_rows[:n_rows], whole.dX_rows[:n_rows])
+    for a, b in zip(js.dW_gnn + js.dW_tower + js.db_tower, whole.dW_gnn + whole.dW_tower + whole.db_tower):
+        assert torch.equal(a, b)
