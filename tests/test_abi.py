@@ -39,3 +39,32 @@ def test_status_strings_and_size_queries_work_without_a_gpu():
     assert cd == [4096, 65536] and ce == [61440, 655360] and cs == [65536, 500000] and nbytes > 0
     with pytest.raises(E.E2EGrecError):
         E.sample_khop_workspace(1 << 31, 4, [3])
+
+
+def test_host_side_argument_checks_of_the_newer_entry_points_need_no_gpu():
+    """Every entry point validates on the host before it enqueues anything: bad sizes, missing pointers and size
+    queries answer without touching a device."""
+    import ctypes as C
+    from paper_2511_20564_b200 import binding as B
+    L = B.lib()
+    ERR_NULL, ERR_ARG, ERR_UNSUPPORTED = -1, -2, -6
+    # running sums of the weighted sampler
+    assert L.e2egrec_edge_cumulate(-1, 0, None, None, None, None) == ERR_ARG
+    assert L.e2egrec_edge_cumulate(4, 8, None, None, None, None) == ERR_NULL
+    assert L.e2egrec_edge_cumulate(0, 0, C.c_void_p(256), None, None, None) == 0
+    # LightGCN on sampled blocks: size queries from capacities alone
+    blocks = (B.Block * 2)()
+    blocks[0] = B.Block(64, 704, 640, *([None] * 10))
+    blocks[1] = B.Block(704, 4224, 3520, *([None] * 10))
+    x = B.Mat(None, 5000, 64, 64, B.BF16)
+    n = C.c_size_t(0)
+    assert L.e2egrec_lightgcn_sampled_forward(blocks, 2, C.byref(x), None, None, C.byref(n), None, None) == 0 and n.value > 0
+    m = C.c_size_t(0)
+    assert L.e2egrec_lightgcn_sampled_backward(blocks, 2, None, C.byref(x), None, None, C.byref(m), None) == 0 and m.value > 0
+    assert L.e2egrec_lightgcn_sampled_forward(blocks, 9, C.byref(x), None, None, C.byref(n), None, None) == ERR_UNSUPPORTED
+    assert L.e2egrec_lightgcn_sampled_forward(blocks, 2, C.byref(x), None, None, None, None, None) == ERR_NULL
+    bad = B.Mat(None, 5000, 60, 60, B.BF16)            # rows of 120 bytes: not a multiple of 16
+    assert L.e2egrec_lightgcn_sampled_forward(blocks, 2, C.byref(bad), None, None, C.byref(n), None, None) == -4
+    # the frontier of a hop must fit the destinations of the next one
+    blocks[1] = B.Block(100, 4224, 3520, *([None] * 10))
+    assert L.e2egrec_lightgcn_sampled_forward(blocks, 2, C.byref(x), None, None, C.byref(n), None, None) == ERR_ARG
