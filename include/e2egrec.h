@@ -123,8 +123,9 @@ const char *e2egrec_last_error(void);
  * stop_event just after it, then disarms the tap.  Groups: 1 = mean aggregation of the outermost
  * block (layer 0, gathers from X), 2 = transposed aggregation of the outermost block (writes dX_rows),
  * 3 = dense transform of layer 0, 4 = weight gradient of layer 0, 5 = input gradient (dCat) of layer 0,
- * 6 = the whole of e2egrec_sample_khop, 7 / 8 / 9 = the three levels of the first segment reduction
- * that follows (the innermost layer's transposed aggregation in e2egrec_sage_backward).  which = 0 disarms. */
+ * 6 = the whole of e2egrec_sample_khop, 7 / 9 = the two kernels (runs and their join; chains across windows) of
+ * the first segment reduction that follows (the innermost layer's transposed aggregation in
+ * e2egrec_sage_backward); 8 is unused.  which = 0 disarms. */
 uint64_t e2egrec_launch_count(void);
 int32_t e2egrec_profile_tap(int32_t which, void *start_event, void *stop_event);
 

@@ -48,7 +48,7 @@ void note_launch();
 // host side: timing taps (e2egrec_profile_tap).  tap_begin/tap_end record the armed events around
 // kernel group `which` and disarm the tap.
 enum { TAP_AGG_FWD_OUTER = 1, TAP_AGG_BWD_OUTER = 2, TAP_UPDATE_FWD_OUTER = 3, TAP_DW_OUTER = 4, TAP_DCAT_OUTER = 5,
-       TAP_SAMPLE = 6, TAP_SEG_L1 = 7, TAP_SEG_L2 = 8, TAP_SEG_L3 = 9, TAP_LAST = 9 };
+       TAP_SAMPLE = 6, TAP_SEG_L1 = 7, TAP_SEG_L3 = 9, TAP_LAST = 9 };   // 8 is unused
 void tap_begin(int which, cudaStream_t st);
 void tap_end(int which, cudaStream_t st);
 
