@@ -410,3 +410,39 @@ def lightgcn_sampled_backward(blocks, ctx, dY, bf16=False):
             dH[:n_seeds] = round_bf16(dH[:n_seeds])
         G = dH
     return G
+
+
+# ----------------------------------------------------------------------------- SSL task and GradNorm (Sec. 4.2)
+
+def ssl_loss(H, X_rows, weight=1.0, bf16=False):
+    """Graph feature auto-encoder loss with the identity decoder (Sec. 4.2): L_ssl = ||X - H||_F^2 over the seed
+    rows, and the gradient of weight * L_ssl with respect to H, 2 * weight * (H - X) (stored as bf16 with bf16)."""
+    H, X_rows = _f64(H), _f64(X_rows)
+    diff = H - X_rows
+    dH = 2.0 * float(weight) * diff
+    return float((diff * diff).sum()), (round_bf16(dH) if bf16 else dH)
+
+
+def frobenius_norm(a):
+    """||a||_2 over all elements: the norm of GradNorm's G_i for the gradient rows of the shared input h^(0)."""
+    a = _f64(a)
+    return float(np.sqrt((a * a).sum()))
+
+
+def gradnorm_update(w, L, L0, g, gamma=1.0, lr=0.025, w_min=1e-6):
+    """One GradNorm step for the task weights (Sec. 4.2, "Gradient-Based Task Weighting").
+
+    w: current weights; L, L0: current and initial task losses; g: norms of the *unweighted* task gradients with
+    respect to the shared input, so that G_i = w_i g_i.  With r_i = (L_i/L0_i) / mean_j(L_j/L0_j) and the targets
+    c_i = mean(G) r_i^gamma held constant, L_gn = sum_i |G_i - c_i| has dL_gn/dw_i = sign(G_i - c_i) g_i; the
+    weights take one gradient step of size lr, stay >= w_min and are rescaled to sum to the number of tasks.
+    Returns (w_new, L_gn)."""
+    w, L, L0, g = (_f64(np.atleast_1d(v)) for v in (w, L, L0, g))
+    T = w.size
+    G = w * g
+    ratio = L / L0
+    r = ratio / ratio.mean()
+    c = G.mean() * r ** gamma
+    L_gn = float(np.abs(G - c).sum())
+    w_new = np.maximum(w - lr * np.sign(G - c) * g, w_min)
+    return w_new * (T / w_new.sum()), L_gn
