@@ -349,6 +349,28 @@ int32_t e2egrec_lightgcn_sampled_backward(const e2egrec_block *blocks, int32_t n
                                           const e2egrec_mat *dY, const e2egrec_mat *dX_rows, void *scratch,
                                           size_t *scratch_bytes, void *stream);
 
+/* The self-supervised task of the GNN and the balancing of the two losses (Sec. 4.2).
+ * e2egrec_ssl_loss: graph feature auto-encoder with the identity decoder, L_ssl = || X_seeds - H ||_F^2 over the rows
+ *   i < *n_rows_dev (NULL: all H->rows rows) with X_seeds[i] = X[seed_ids[i]]; loss: device float[1] (unweighted);
+ *   dH [>= H->rows x dim] receives the gradient of weight[0] * L_ssl with respect to H, 2 weight (H - X), in H's
+ *   dtype (weight: device float[1], so that a weight updated on the device feeds the next step without a host round
+ *   trip).  H is the encoder output (e2egrec_sage_forward's H_out), whose width must equal X's.
+ * e2egrec_gradient_norm: || A[:n_rows] ||_2 into norm (device float[1]): GradNorm's gradient norm of one task with
+ *   respect to the shared input rows (the dX_rows of a backward pass run with that task's gradient alone).
+ * e2egrec_gradnorm_update: one GradNorm step for n_tasks <= 8 weights w (device, updated in place) from the current
+ *   and initial losses L, L0 and the norms g of the unweighted task gradients (G_i = w_i g_i): with r_i =
+ *   (L_i/L0_i) / mean_j (L_j/L0_j) and the targets c_i = mean(G) r_i^gamma held constant, w_i takes one step of size
+ *   lr down the gradient sign(G_i - c_i) g_i of sum_i |G_i - c_i|, stays >= 1e-6 and the weights are rescaled to sum
+ *   to n_tasks; L_gn (optional, device float[1]) receives the objective.  The paper fixes gamma = 1 and leaves lr open.
+ * ws: scratch (size query with ws == NULL).  All sums run in a fixed order. */
+int32_t e2egrec_ssl_loss(const e2egrec_mat *H, const e2egrec_mat *X, const int32_t *seed_ids, const int32_t *n_rows_dev,
+                         const float *weight, float *loss, const e2egrec_mat *dH, void *ws, size_t *ws_bytes,
+                         void *stream);
+int32_t e2egrec_gradient_norm(const e2egrec_mat *A, const int32_t *n_rows_dev, float *norm, void *ws, size_t *ws_bytes,
+                              void *stream);
+int32_t e2egrec_gradnorm_update(float *w, const float *L, const float *L0, const float *g, int32_t n_tasks, float gamma,
+                                float lr, float *L_gn, void *stream);
+
 /* e2egrec_aggregate_forward without a workspace argument (the paper has no counterpart; this is a
  * packaging variant of the call above and computes exactly the same result).
  *

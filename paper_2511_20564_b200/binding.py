@@ -74,6 +74,15 @@ def lib():
         L.e2egrec_lightgcn_sampled_backward.restype = C.c_int32
         L.e2egrec_lightgcn_sampled_backward.argtypes = [C.POINTER(Block), C.c_int32, C.c_void_p, C.POINTER(Mat),
                                                         C.POINTER(Mat), C.c_void_p, C.POINTER(C.c_size_t), C.c_void_p]
+        L.e2egrec_ssl_loss.restype = C.c_int32
+        L.e2egrec_ssl_loss.argtypes = [C.POINTER(Mat), C.POINTER(Mat), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
+                                       C.POINTER(Mat), C.c_void_p, C.POINTER(C.c_size_t), C.c_void_p]
+        L.e2egrec_gradient_norm.restype = C.c_int32
+        L.e2egrec_gradient_norm.argtypes = [C.POINTER(Mat), C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_size_t),
+                                            C.c_void_p]
+        L.e2egrec_gradnorm_update.restype = C.c_int32
+        L.e2egrec_gradnorm_update.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_float,
+                                              C.c_float, C.c_void_p, C.c_void_p]
         L.e2egrec_edge_cumulate.restype = C.c_int32
         L.e2egrec_edge_cumulate.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.e2egrec_sage_forward.restype = C.c_int32
@@ -558,3 +567,55 @@ def lightgcn_sampled_backward(blocks: Blocks, ctx: torch.Tensor, dY: torch.Tenso
     _check(lib().e2egrec_lightgcn_sampled_backward(blocks.c, len(blocks), _ptr(ctx), C.byref(dy), C.byref(dx), _ptr(scratch),
                                                    C.byref(n), _stream(stream)), "e2egrec_lightgcn_sampled_backward")
     return dX_rows, scratch
+
+
+# ------------------------------------------------------------------------------------------ SSL task, GradNorm
+
+_SUM_WS = {}
+
+
+def _sum_ws(device):
+    """The 1 KB scratch of the fixed-order sums, one per device."""
+    key = str(device)
+    if key not in _SUM_WS:
+        _SUM_WS[key] = _dev_bytes(1024, device)
+    return _SUM_WS[key]
+
+
+def ssl_loss(H: torch.Tensor, X: torch.Tensor, seed_ids: torch.Tensor, n_rows_dev, weight: torch.Tensor, loss=None,
+             dH=None, stream=None):
+    """Enqueues L_ssl = ||X[seed_ids] - H||_F^2 and dH = 2 weight (H - X[seed_ids]); returns (loss, dH)."""
+    assert weight.dtype == torch.float32 and seed_ids.dtype == torch.int32
+    if loss is None:
+        loss = torch.zeros(1, dtype=torch.float32, device=H.device)
+    if dH is None:
+        dH = torch.zeros_like(H)
+    ws = _sum_ws(H.device)
+    n = C.c_size_t(ws.numel())
+    h, x, g = _mat(H), _mat(X), _mat(dH)
+    _check(lib().e2egrec_ssl_loss(C.byref(h), C.byref(x), _ptr(seed_ids), None if n_rows_dev is None else _ptr(n_rows_dev),
+                                  _ptr(weight), _ptr(loss), C.byref(g), _ptr(ws), C.byref(n), _stream(stream)),
+           "e2egrec_ssl_loss")
+    return loss, dH
+
+
+def gradient_norm(A: torch.Tensor, n_rows_dev=None, out=None, stream=None):
+    """Enqueues ||A[:n_rows]||_2 into a device float; see e2egrec_gradient_norm."""
+    if out is None:
+        out = torch.zeros(1, dtype=torch.float32, device=A.device)
+    ws = _sum_ws(A.device)
+    n = C.c_size_t(ws.numel())
+    a = _mat(A)
+    _check(lib().e2egrec_gradient_norm(C.byref(a), None if n_rows_dev is None else _ptr(n_rows_dev), _ptr(out), _ptr(ws),
+                                       C.byref(n), _stream(stream)), "e2egrec_gradient_norm")
+    return out
+
+
+def gradnorm_update(w: torch.Tensor, L: torch.Tensor, L0: torch.Tensor, g: torch.Tensor, gamma=1.0, lr=0.025, L_gn=None,
+                    stream=None):
+    """Enqueues one GradNorm step on the device-resident task weights w (in place); see e2egrec_gradnorm_update."""
+    for t in (w, L, L0, g):
+        assert t.dtype == torch.float32 and t.numel() == w.numel()
+    _check(lib().e2egrec_gradnorm_update(_ptr(w), _ptr(L), _ptr(L0), _ptr(g), w.numel(), C.c_float(gamma), C.c_float(lr),
+                                         None if L_gn is None else _ptr(L_gn), _stream(stream)), "e2egrec_gradnorm_update")
+    return w
