@@ -276,9 +276,27 @@ def run_ours(args, w):
         E.sample_khop(indptr, indices, seeds_in2[p], blocks2[p], w.seed, 0, defer_transpose=defer,
                       edge_cum=edge_cum)                 # step = the scratch's offset
 
+    if args.multitask:
+        # the two-task step of Sec. 4.2: the recommendation gradient and the gradient of the SSL reconstruction loss go
+        # through the encoder one after the other (weight gradients accumulate), their norms at the shared input feed
+        # one GradNorm step of the task weights
+        if w.hidden != w.dim:
+            raise SystemExit("--multitask needs hidden == dim (the identity decoder compares H with X)")
+        f32 = dict(dtype=torch.float32, device=dev)
+        mt = dict(dX_ssl=torch.zeros_like(dX), dH_ssl=torch.zeros_like(H_out), one=torch.ones(1, **f32),
+                  wts=torch.ones(2, **f32), L=torch.ones(2, **f32), L0=torch.ones(2, **f32), g=torch.zeros(2, **f32))
+
     def compute_leg(p):
         E.sage_forward(blocks2[p], X, Ws, ctx=ctx, H_out=H_out2[p])
         E.sage_backward(blocks2[p], X, Ws, ctx, dH_in2[p], dWs=dWs2[p], dX_rows=dX, scratch=scratch)
+        if args.multitask:
+            n_seeds_dev, n_rows_dev = blocks2[p].counts[0][0:1], blocks2[p].counts[L - 1][1:2]
+            E.ssl_loss(H_out2[p], X, seeds_in2[p], n_seeds_dev, mt["one"], loss=mt["L"][0:1], dH=mt["dH_ssl"])
+            E.gradient_norm(dX, n_rows_dev, out=mt["g"][1:2])
+            E.sage_backward(blocks2[p], X, Ws, ctx, mt["dH_ssl"], dWs=dWs2[p], dX_rows=mt["dX_ssl"], scratch=scratch,
+                            accumulate=True)
+            E.gradient_norm(mt["dX_ssl"], n_rows_dev, out=mt["g"][0:1])
+            E.gradnorm_update(mt["wts"], mt["L"], mt["L0"], mt["g"], 1.0, 0.025)
         count_total.add_(blocks2[p].counts)
         counts_snap2[p].copy_(blocks2[p].counts)
 
@@ -561,6 +579,8 @@ def run_ours(args, w):
                 config=dict(workload=w.name, nodes=w.n_nodes, csr_entries=int(indices.numel()), dim=w.dim, hidden=w.hidden,
                             layers=L, fanouts=list(w.fanouts), batch=w.batch, seeds=args.seeds,
                             sampling="uniform" if args.beta is None else f"weighted, beta={args.beta}",
+                            tasks="recommendation gradient + SSL reconstruction loss, two backward passes, GradNorm step"
+                                  if args.multitask else "recommendation gradient",
                             parallelism=f"replicas x{world}",
                             launch="one CUDA graph replay per step: forward/backward of the batch beside the sampling of "
                                    "the next batch on a second stream (two sets of block buffers)",
@@ -866,6 +886,8 @@ def main():
     ap.add_argument("--no-joint", action="store_true", help="skip the joint-step measurement")
     ap.add_argument("--backbone", default="sage", choices=["sage", "lightgcn"],
                     help="lightgcn: sampling + LightGCN propagation on the sampled blocks + its adjoint (no weights)")
+    ap.add_argument("--multitask", action="store_true",
+                    help="add the SSL reconstruction task: second backward pass, gradient norms, GradNorm weight step")
     ap.add_argument("--beta", type=float, default=None,
                     help="weighted neighbour sampling p ~ omega^beta with synthetic log-normal omega (default: uniform)")
     ap.add_argument("--seeds", default="activity", choices=["activity", "uniform"],
