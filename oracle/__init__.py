@@ -446,3 +446,35 @@ def gradnorm_update(w, L, L0, g, gamma=1.0, lr=0.025, w_min=1e-6):
     L_gn = float(np.abs(G - c).sum())
     w_new = np.maximum(w - lr * np.sign(G - c) * g, w_min)
     return w_new * (T / w_new.sum()), L_gn
+
+
+# ----------------------------------------------------------------------------- gated fusion (Sec. 4.3.1)
+
+def gate_fusion_forward(F, Wg, bg, bf16=False):
+    """Concatenation with gating: g = sigmoid(F Wg^T + bg), F_fused = g * F (element-wise), F = the concatenated
+    feature groups [N x d].  Storage points with bf16: the pre-activation, the gate, the fused features.
+    Returns (fused, gate)."""
+    F, Wg = _f64(F), _f64(Wg)
+    pre = F @ Wg.T + (0.0 if bg is None else _f64(bg))
+    if bf16:
+        pre = round_bf16(pre)
+    g = np.where(pre >= 0, 1.0 / (1.0 + np.exp(-np.abs(pre))), np.exp(-np.abs(pre)) / (1.0 + np.exp(-np.abs(pre))))
+    if bf16:
+        g = round_bf16(g)
+    fused = g * F
+    return (round_bf16(fused) if bf16 else fused), g
+
+
+def gate_fusion_backward(dFused, F, gate, Wg, bf16=False):
+    """Adjoint of gate_fusion_forward: returns (dF, dWg, dbg).  d pre = dFused * F * g (1 - g);
+    dF = dFused * g + d pre Wg; dWg = d pre^T F; dbg = column sums of d pre.  Storage points with bf16: d pre, the
+    product d pre Wg, dF."""
+    dFused, F, g, Wg = _f64(dFused), _f64(F), _f64(gate), _f64(Wg)
+    dpre = dFused * F * g * (1.0 - g)
+    if bf16:
+        dpre = round_bf16(dpre)
+    t = dpre @ Wg
+    if bf16:
+        t = round_bf16(t)
+    dF = t + dFused * g
+    return (round_bf16(dF) if bf16 else dF), dpre.T @ F, dpre.sum(0)
