@@ -371,6 +371,21 @@ int32_t e2egrec_gradient_norm(const e2egrec_mat *A, const int32_t *n_rows_dev, f
 int32_t e2egrec_gradnorm_update(float *w, const float *L, const float *L0, const float *g, int32_t n_tasks, float gamma,
                                 float lr, float *L_gn, void *stream);
 
+/* Feature fusion by concatenation with gating (Sec. 4.3.1):  g = sigmoid(F Wg^T + bg),  F_fused = g * F, for the
+ * n_rows rows of F [rows x d] (the concatenated feature groups, GNN output among them); Wg [d x d] row-major in F's
+ * dtype, bg device float[d] or NULL.  gate and fused: [>= n_rows x d] outputs (the gate is kept for the backward call).
+ * e2egrec_gate_fusion_backward: dF = dFused * g + (dFused * F * g (1 - g)) Wg, dWg = (dFused * F * g (1 - g))^T F
+ * (device float[d x d]), dbg its column sums (device float[d] or NULL).  F must have at least n_rows rounded up to 128
+ * rows allocated, holding finite values (the dense products read whole 128-row tiles); bf16 shapes with d a multiple
+ * of 64 and ld = d run on the tensor cores, others on fp32 FMA.  With bf16 the pre-activation, the gate, the fused
+ * features and the intermediate gradients are stored as bf16.  ws: scratch (size query with ws == NULL). */
+int32_t e2egrec_gate_fusion_forward(const e2egrec_mat *F, int32_t n_rows, const e2egrec_mat *Wg, const float *bg,
+                                    const e2egrec_mat *gate, const e2egrec_mat *fused, void *ws, size_t *ws_bytes,
+                                    void *stream);
+int32_t e2egrec_gate_fusion_backward(const e2egrec_mat *dFused, const e2egrec_mat *F, int32_t n_rows,
+                                     const e2egrec_mat *gate, const e2egrec_mat *Wg, const e2egrec_mat *dF, float *dWg,
+                                     float *dbg, void *ws, size_t *ws_bytes, void *stream);
+
 /* e2egrec_aggregate_forward without a workspace argument (the paper has no counterpart; this is a
  * packaging variant of the call above and computes exactly the same result).
  *

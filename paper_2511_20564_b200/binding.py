@@ -83,6 +83,13 @@ def lib():
         L.e2egrec_gradnorm_update.restype = C.c_int32
         L.e2egrec_gradnorm_update.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_float,
                                               C.c_float, C.c_void_p, C.c_void_p]
+        L.e2egrec_gate_fusion_forward.restype = C.c_int32
+        L.e2egrec_gate_fusion_forward.argtypes = [C.POINTER(Mat), C.c_int32, C.POINTER(Mat), C.c_void_p, C.POINTER(Mat),
+                                                  C.POINTER(Mat), C.c_void_p, C.POINTER(C.c_size_t), C.c_void_p]
+        L.e2egrec_gate_fusion_backward.restype = C.c_int32
+        L.e2egrec_gate_fusion_backward.argtypes = [C.POINTER(Mat), C.POINTER(Mat), C.c_int32, C.POINTER(Mat), C.POINTER(Mat),
+                                                   C.POINTER(Mat), C.c_void_p, C.c_void_p, C.c_void_p,
+                                                   C.POINTER(C.c_size_t), C.c_void_p]
         L.e2egrec_edge_cumulate.restype = C.c_int32
         L.e2egrec_edge_cumulate.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p]
         L.e2egrec_sage_forward.restype = C.c_int32
@@ -619,3 +626,35 @@ def gradnorm_update(w: torch.Tensor, L: torch.Tensor, L0: torch.Tensor, g: torch
     _check(lib().e2egrec_gradnorm_update(_ptr(w), _ptr(L), _ptr(L0), _ptr(g), w.numel(), C.c_float(gamma), C.c_float(lr),
                                          None if L_gn is None else _ptr(L_gn), _stream(stream)), "e2egrec_gradnorm_update")
     return w
+
+
+# ------------------------------------------------------------------------------------------ gated fusion
+
+def gate_fusion_forward(F: torch.Tensor, n_rows: int, Wg: torch.Tensor, bg=None, ws=None, stream=None):
+    """Enqueues g = sigmoid(F Wg^T + bg), fused = g * F on the first n_rows rows; returns (fused, gate, ws)."""
+    f, w = _mat(F), _mat(Wg)
+    gate, fused = torch.zeros_like(F), torch.zeros_like(F)
+    g, o = _mat(gate), _mat(fused)
+    n = C.c_size_t(0)
+    _check(lib().e2egrec_gate_fusion_forward(C.byref(f), n_rows, C.byref(w), None, None, None, None, C.byref(n), None),
+           "e2egrec_gate_fusion_forward(size query)")
+    if ws is None:
+        ws = _dev_bytes(n.value, F.device)
+    n = C.c_size_t(ws.numel())
+    _check(lib().e2egrec_gate_fusion_forward(C.byref(f), n_rows, C.byref(w), _ptr(bg), C.byref(g), C.byref(o), _ptr(ws),
+                                             C.byref(n), _stream(stream)), "e2egrec_gate_fusion_forward")
+    return fused, gate, ws
+
+
+def gate_fusion_backward(dFused: torch.Tensor, F: torch.Tensor, n_rows: int, gate: torch.Tensor, Wg: torch.Tensor, ws,
+                         with_bias=True, stream=None):
+    """Enqueues the adjoint of gate_fusion_forward; returns (dF, dWg, dbg)."""
+    d = F.shape[1]
+    dF = torch.zeros_like(F)
+    dWg = torch.zeros(d, d, dtype=torch.float32, device=F.device)
+    dbg = torch.zeros(d, dtype=torch.float32, device=F.device) if with_bias else None
+    a, f, g, w, o = _mat(dFused), _mat(F), _mat(gate), _mat(Wg), _mat(dF)
+    n = C.c_size_t(ws.numel())
+    _check(lib().e2egrec_gate_fusion_backward(C.byref(a), C.byref(f), n_rows, C.byref(g), C.byref(w), C.byref(o), _ptr(dWg),
+                                              _ptr(dbg), _ptr(ws), C.byref(n), _stream(stream)), "e2egrec_gate_fusion_backward")
+    return dF, dWg, dbg

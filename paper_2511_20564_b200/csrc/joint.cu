@@ -475,3 +475,217 @@ extern "C" int32_t e2egrec_joint_step_phase(const e2egrec_csr *graph, const e2eg
     return run_joint<float>(jp, graph, X, pair_user, pair_item, dense, labels, fanouts, W_gnn, W_tower, b_tower, seed, step, loss,
                             logits, dW_gnn, dW_tower, db_tower, dX_rows, dX_ids, n_dX_rows, static_cast<char *>(ws), phase, st);
 }
+
+// ------------------------------------------------------------------------------------------ gated fusion (Sec. 4.3.1)
+//   g = sigmoid(F Wg^T + bg),  F_fused = g * F.  The product runs on the dense helpers above (tcgen05 for bf16 shapes
+//   they take, fp32 FMA otherwise); the gate itself and its derivative are element-wise kernels.
+namespace e2egrec {
+namespace {
+
+__global__ void gate_meta_kernel(int32_t *meta, int32_t n_rows) { meta[0] = n_rows; }
+
+// gate = sigmoid(pre), fused = gate * F for rows < n_rows; zero rows up to rows_alloc
+template <typename T>
+__global__ void gate_apply_kernel(const T *__restrict__ pre, const T *__restrict__ F, int64_t ldf, int d, int32_t n_rows,
+                                  int64_t rows_alloc, T *__restrict__ gate, int64_t ldg, T *__restrict__ fused, int64_t ldo)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t i = t / d;
+    const int k = (int)(t - i * d);
+    if (i >= rows_alloc) return;
+    float g = 0.f, o = 0.f;
+    if (i < n_rows) {
+        const float p = to_float<T>(pre[i * d + k]);
+        const float e = expf(-fabsf(p));
+        g = to_float<T>(from_float<T>(p >= 0.f ? 1.0f / (1.0f + e) : e / (1.0f + e)));      // the stored gate
+        o = g * to_float<T>(F[i * ldf + k]);
+    }
+    gate[i * ldg + k] = from_float<T>(g);
+    fused[i * ldo + k] = from_float<T>(o);
+}
+
+// dpre = dFused * F * g (1 - g) for rows < n_rows, zero rows up to rows_alloc
+template <typename T>
+__global__ void gate_dpre_kernel(const T *__restrict__ dFused, int64_t ldd, const T *__restrict__ F, int64_t ldf,
+                                 const T *__restrict__ gate, int64_t ldg, int d, int32_t n_rows, int64_t rows_alloc,
+                                 T *__restrict__ dpre)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t i = t / d;
+    const int k = (int)(t - i * d);
+    if (i >= rows_alloc) return;
+    float v = 0.f;
+    if (i < n_rows) {
+        const float g = to_float<T>(gate[i * ldg + k]);
+        v = to_float<T>(dFused[i * ldd + k]) * to_float<T>(F[i * ldf + k]) * g * (1.0f - g);
+    }
+    dpre[i * d + k] = from_float<T>(v);
+}
+
+// dF = t + dFused * g for rows < n_rows
+template <typename T>
+__global__ void gate_dF_kernel(const T *__restrict__ tprod, const T *__restrict__ dFused, int64_t ldd,
+                               const T *__restrict__ gate, int64_t ldg, int d, int32_t n_rows, T *__restrict__ dF, int64_t ldo)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t i = t / d;
+    const int k = (int)(t - i * d);
+    if (i >= n_rows) return;
+    dF[i * ldo + k] = from_float<T>(to_float<T>(tprod[i * d + k]) + to_float<T>(dFused[i * ldd + k]) * to_float<T>(gate[i * ldg + k]));
+}
+
+struct GatePlan {
+    int d;
+    int64_t rows;          // rows of the scratch matrices: n_rows rounded up to 128
+    size_t es, meta_off, a_off, b_off, wt_off, part_off, bytes;
+};
+
+int32_t gate_plan(const e2egrec_mat *F, int32_t n_rows, const e2egrec_mat *Wg, GatePlan &gp)
+{
+    if (!F || !Wg || !F->data || !Wg->data) return E2EGREC_ERR_NULL;
+    if (F->dtype != E2EGREC_F32 && F->dtype != E2EGREC_BF16) return E2EGREC_ERR_DTYPE;
+    if (Wg->dtype != F->dtype) return E2EGREC_ERR_DTYPE;
+    if (n_rows < 0 || F->dim < 1 || F->dim > kMaxDim || F->ld < F->dim) return E2EGREC_ERR_ARG;
+    if (Wg->rows != F->dim || Wg->dim != F->dim || Wg->ld != Wg->dim) return E2EGREC_ERR_ARG;
+    gp.d = F->dim;
+    gp.es = dtype_size(F->dtype);
+    gp.rows = pad128(n_rows > 0 ? n_rows : 1);
+    if (F->rows < gp.rows) return E2EGREC_ERR_ARG;       // the dense products read whole 128-row tiles of F
+    size_t off = 0;
+    auto take = [&](size_t b) { size_t o = off; off += align_up(b, 256); return o; };
+    gp.meta_off = take(256);
+    gp.a_off = take((size_t)gp.rows * gp.d * gp.es);     // pre-activation / d pre
+    gp.b_off = take((size_t)gp.rows * gp.d * gp.es);     // d pre Wg
+    gp.wt_off = take((size_t)gp.d * gp.d * gp.es);
+    gp.part_off = take((size_t)kSplits * gp.d * gp.d * sizeof(float));
+    gp.bytes = off;
+    return E2EGREC_OK;
+}
+
+unsigned cells_grid(int64_t rows, int d) { return (unsigned)std::max<int64_t>(1, ceil_div(rows * d, 256)); }
+
+}  // namespace
+}  // namespace e2egrec
+
+namespace e2egrec {
+namespace {
+
+template <typename T>
+int32_t gate_forward_impl(const GatePlan &gp, const e2egrec_mat *F, int32_t n_rows, const e2egrec_mat *Wg, const float *bg,
+                          const e2egrec_mat *gate, const e2egrec_mat *fused, char *ws, cudaStream_t st)
+{
+    int32_t *meta = reinterpret_cast<int32_t *>(ws + gp.meta_off);      // {rows, status}
+    T *pre = reinterpret_cast<T *>(ws + gp.a_off);
+    note_launch();
+    gate_meta_kernel<<<1, 1, 0, st>>>(meta, n_rows);
+    cudaMemsetAsync(meta + 1, 0, sizeof(int32_t), st);
+    const bool dense_f = F->ld == F->dim;                               // the tensor-core path takes a dense operand
+    if (dense_f) {
+        linear_forward<T>(static_cast<const T *>(F->data), gp.rows, gp.d, static_cast<const T *>(Wg->data), gp.d, bg, 0, pre, meta,
+                          meta + 1, st);
+    } else {
+        EpiUpdate<T> epi{pre, gp.d, bg, 0};
+        dim3 grid((unsigned)ceil_div(gp.rows, kGemmBM), (unsigned)ceil_div(gp.d, kGemmBN), 1);
+        note_launch();
+        gemm_simt_kernel<T, false, false, EpiUpdate<T>><<<grid, kGemmThreads, 0, st>>>(
+            static_cast<const T *>(F->data), F->ld, static_cast<const T *>(Wg->data), gp.d, gp.rows, gp.d, gp.d, meta, nullptr, epi);
+    }
+    note_launch();
+    gate_apply_kernel<T><<<cells_grid(gp.rows, gp.d), 256, 0, st>>>(pre, static_cast<const T *>(F->data), F->ld, gp.d, n_rows,
+                                                                  std::min<int64_t>(gp.rows, std::min(gate->rows, fused->rows)),
+                                                                  static_cast<T *>(gate->data), gate->ld,
+                                                                  static_cast<T *>(fused->data), fused->ld);
+    return check_launch("gate_fusion_forward");
+}
+
+template <typename T>
+int32_t gate_backward_impl(const GatePlan &gp, const e2egrec_mat *dFused, const e2egrec_mat *F, int32_t n_rows,
+                           const e2egrec_mat *gate, const e2egrec_mat *Wg, const e2egrec_mat *dF, float *dWg, float *dbg,
+                           char *ws, cudaStream_t st)
+{
+    int32_t *meta = reinterpret_cast<int32_t *>(ws + gp.meta_off);
+    T *dpre = reinterpret_cast<T *>(ws + gp.a_off), *tprod = reinterpret_cast<T *>(ws + gp.b_off);
+    T *wt = reinterpret_cast<T *>(ws + gp.wt_off);
+    float *part = reinterpret_cast<float *>(ws + gp.part_off);
+    note_launch();
+    gate_meta_kernel<<<1, 1, 0, st>>>(meta, n_rows);
+    cudaMemsetAsync(meta + 1, 0, sizeof(int32_t), st);
+    note_launch();
+    gate_dpre_kernel<T><<<cells_grid(gp.rows, gp.d), 256, 0, st>>>(static_cast<const T *>(dFused->data), dFused->ld,
+                                                                 static_cast<const T *>(F->data), F->ld,
+                                                                 static_cast<const T *>(gate->data), gate->ld, gp.d, n_rows,
+                                                                 gp.rows, dpre);
+    if (F->ld == F->dim) {
+        linear_backward_weight<T>(dpre, gp.rows, gp.d, static_cast<const T *>(F->data), gp.d, meta, part, dWg, dbg, meta + 1, st);
+    } else {                                                             // strided F: fp32-FMA product
+        EpiPartial epi{part, gp.d, (int64_t)gp.d * gp.d};
+        dim3 grid((unsigned)ceil_div(gp.d, kGemmBM), (unsigned)ceil_div(gp.d, kGemmBN), kSplits);
+        note_launch();
+        gemm_simt_kernel<T, true, true, EpiPartial><<<grid, kGemmThreads, 0, st>>>(dpre, gp.d, static_cast<const T *>(F->data),
+                                                                                  F->ld, gp.d, gp.d, gp.rows, nullptr, meta, epi);
+        note_launch();
+        splitk_reduce_kernel<<<(unsigned)ceil_div((int64_t)gp.d * gp.d, 256), 256, 0, st>>>(part, (int64_t)gp.d * gp.d, kSplits, 0,
+                                                                                         dWg, nullptr);
+        if (dbg) {
+            note_launch();
+            colsum_kernel<T><<<(unsigned)ceil_div(gp.d, 32), 256, 0, st>>>(dpre, gp.d, meta, gp.d, 0, dbg);
+        }
+    }
+    linear_backward_input<T>(dpre, gp.rows, gp.d, static_cast<const T *>(Wg->data), gp.d, nullptr, tprod, wt, meta, meta + 1, st);
+    note_launch();
+    gate_dF_kernel<T><<<cells_grid(n_rows > 0 ? n_rows : 1, gp.d), 256, 0, st>>>(tprod, static_cast<const T *>(dFused->data),
+                                                                               dFused->ld, static_cast<const T *>(gate->data),
+                                                                               gate->ld, gp.d, n_rows, static_cast<T *>(dF->data),
+                                                                               dF->ld);
+    return check_launch("gate_fusion_backward");
+}
+
+int32_t gate_check_out(const e2egrec_mat *m, const e2egrec_mat *F, int32_t n_rows)
+{
+    if (!m || !m->data) return E2EGREC_ERR_NULL;
+    if (m->dtype != F->dtype) return E2EGREC_ERR_DTYPE;
+    if (m->dim != F->dim || m->ld < m->dim || m->rows < n_rows) return E2EGREC_ERR_ARG;
+    return E2EGREC_OK;
+}
+
+}  // namespace
+}  // namespace e2egrec
+
+extern "C" int32_t e2egrec_gate_fusion_forward(const e2egrec_mat *F, int32_t n_rows, const e2egrec_mat *Wg, const float *bg,
+                                               const e2egrec_mat *gate, const e2egrec_mat *fused, void *ws, size_t *ws_bytes,
+                                               void *stream)
+{
+    if (!ws_bytes) return E2EGREC_ERR_NULL;
+    GatePlan gp{};
+    int32_t rc = gate_plan(F, n_rows, Wg, gp);
+    if (rc != E2EGREC_OK) return rc;
+    if (!ws) { *ws_bytes = gp.bytes; return E2EGREC_OK; }
+    if (*ws_bytes < gp.bytes) { *ws_bytes = gp.bytes; return E2EGREC_ERR_WORKSPACE; }
+    if (reinterpret_cast<uintptr_t>(ws) % 256) return E2EGREC_ERR_ALIGN;
+    if ((rc = gate_check_out(gate, F, n_rows)) != E2EGREC_OK || (rc = gate_check_out(fused, F, n_rows)) != E2EGREC_OK) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (F->dtype == E2EGREC_BF16)
+        return gate_forward_impl<__nv_bfloat16>(gp, F, n_rows, Wg, bg, gate, fused, static_cast<char *>(ws), st);
+    return gate_forward_impl<float>(gp, F, n_rows, Wg, bg, gate, fused, static_cast<char *>(ws), st);
+}
+
+extern "C" int32_t e2egrec_gate_fusion_backward(const e2egrec_mat *dFused, const e2egrec_mat *F, int32_t n_rows,
+                                                const e2egrec_mat *gate, const e2egrec_mat *Wg, const e2egrec_mat *dF,
+                                                float *dWg, float *dbg, void *ws, size_t *ws_bytes, void *stream)
+{
+    if (!ws_bytes) return E2EGREC_ERR_NULL;
+    GatePlan gp{};
+    int32_t rc = gate_plan(F, n_rows, Wg, gp);
+    if (rc != E2EGREC_OK) return rc;
+    if (!ws) { *ws_bytes = gp.bytes; return E2EGREC_OK; }
+    if (*ws_bytes < gp.bytes) { *ws_bytes = gp.bytes; return E2EGREC_ERR_WORKSPACE; }
+    if (reinterpret_cast<uintptr_t>(ws) % 256) return E2EGREC_ERR_ALIGN;
+    if (!dWg) return E2EGREC_ERR_NULL;
+    if ((rc = gate_check_out(dFused, F, n_rows)) != E2EGREC_OK || (rc = gate_check_out(gate, F, n_rows)) != E2EGREC_OK ||
+        (rc = gate_check_out(dF, F, n_rows)) != E2EGREC_OK)
+        return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (F->dtype == E2EGREC_BF16)
+        return gate_backward_impl<__nv_bfloat16>(gp, dFused, F, n_rows, gate, Wg, dF, dWg, dbg, static_cast<char *>(ws), st);
+    return gate_backward_impl<float>(gp, dFused, F, n_rows, gate, Wg, dF, dWg, dbg, static_cast<char *>(ws), st);
+}
