@@ -77,7 +77,9 @@ static void dispatch_sage_aggregate(const T *Hsrc, int64_t ld, const int32_t *nb
 #undef E2E_CASE
 }
 
-constexpr int kBlockRun = 32;         // transposed-block entries per lane group (level-1 run)
+// transposed-block entries per lane group: short runs (shorter chains of dependent loads, more groups) unless the
+// block can hold millions of entries, where the longer run's lower overhead per entry wins
+static inline int block_run_len(int64_t cap_edges) { return cap_edges >= (1ll << 21) ? 32 : 16; }
 constexpr int kDwSplits = 148;        // split-K factor of the weight-gradient product
 
 // ------------------------------------------------------------------------------ forward
@@ -141,7 +143,7 @@ static BackwardScratch plan_backward(const e2egrec_block *blocks, int32_t n_laye
         dcat = std::max(dcat, (size_t)p.rows * 2 * p.d_in * es);
         part = std::max(part, (size_t)kDwSplits * p.d_out * 2 * p.d_in * sizeof(float));
         wt = std::max(wt, (size_t)p.d_out * 2 * p.d_in * es);
-        ht = std::max(ht, seg_scratch_carve(blocks[p.block].cap_edges, kBlockRun, p.d_in, es, nullptr).bytes);
+        ht = std::max(ht, seg_scratch_carve(blocks[p.block].cap_edges, block_run_len(blocks[p.block].cap_edges), p.d_in, es, nullptr).bytes);
     }
     size_t off = 0;
     auto take = [&](size_t b) { size_t o = off; off += align_up(b, 256); return o; };
@@ -265,9 +267,9 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
             o.mask = nullptr;
         }
         if (l == 0) tap_begin(TAP_AGG_BWD_OUTER, st);
-        const SegScratch sc = seg_scratch_carve(b.cap_edges, kBlockRun, p.d_in, dtype_size(X->dtype), scratch + bs.seg_off);
+        const SegScratch sc = seg_scratch_carve(b.cap_edges, block_run_len(b.cap_edges), p.d_in, dtype_size(X->dtype), scratch + bs.seg_off);
         dispatch_seg_reduce<T, int32_t, false>(dcat + p.d_in, two_d, b.csc_ptr, b.csc_row, &b.counts[CNT_SRC], 0, b.cap_src,
-                                               nullptr, kBlockRun, p.d_in, X->dtype, b.csc_col, sc, o, st);
+                                               nullptr, block_run_len(b.cap_edges), p.d_in, X->dtype, b.csc_col, sc, o, st);
         if (l == 0) tap_end(TAP_AGG_BWD_OUTER, st);
     }
     if (side) side->join(st);

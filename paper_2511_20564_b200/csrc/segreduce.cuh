@@ -142,6 +142,9 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
     const int64_t n_seg = n_seg_dev ? (int64_t)*n_seg_dev : n_seg_host;
     const int64_t total = n_seg > 0 ? (int64_t)ptr[n_seg] : 0;
     const int64_t k0 = run * run_len;
+    // a window that lies wholly beyond the stream (grids are sized for capacities) has nothing to do, not even a
+    // record: seg_final_kernel only looks at the windows that hold entries
+    if ((int64_t)blockIdx.x * RB * run_len >= total) return;
     int32_t head_seg = -1, head_ends = 0, tail_seg = -1;
 
     // finishes segment `seg` whose entries sum to acc: scale, round to the storage type, mask, store
@@ -468,6 +471,11 @@ seg_final_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_t
         return;
     }
     if (n_seg == 0) return;
+    {   // only the windows that hold entries carry a record
+        const int64_t total = (int64_t)ptr[n_seg];
+        const int64_t live = ceil_div(ceil_div(total, (int64_t)run_len), (int64_t)runs_per_window);
+        if (live < n_windows) n_windows = live;
+    }
 
     // kFinalWindows windows per block and round; the window blocks stride over the windows.  A chain of up to kFinalWarpParts parts is added by one warp (the warps of
     // the block work on different windows at the same time); a longer one is left to the whole block.
