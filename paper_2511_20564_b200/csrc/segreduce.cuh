@@ -25,6 +25,8 @@
 
 namespace e2egrec {
 
+constexpr int kSegRing = 8;        // entries requested ahead in the ring form of seg_run_kernel
+
 // runs per window = lane groups per block of seg_run_kernel
 inline int seg_runs_per_window(int d, size_t elem_size) { return kAggThreads / row_shape_bytes((int64_t)d * elem_size).lpr; }
 
@@ -104,6 +106,14 @@ __device__ __noinline__ SegStep seg_advance(const PtrT *__restrict__ ptr, int64_
     return SegStep{s, end};
 }
 
+__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 // Shared memory of seg_run_kernel (dynamic): head and tail rows of the block's runs, fp32, one row of
 // LPR*CPL*E floats per run, then one record per run.
 template <int LPR, int CPL, int E>
@@ -117,7 +127,11 @@ constexpr size_t seg_run_smem_bytes()
 // kInFlight: gathered rows a lane group requests before it adds any.  Four suit the short streams of a sampled
 // block (few resident warps, latency hidden inside the thread); on streams that fill the machine two are faster,
 // because the smaller register footprint keeps five blocks resident per SM instead of three.
-template <typename T, typename PtrT, int LPR, int CPL, bool kWeight, int kExtra, int kInFlight>
+// kRing > 0 (sampled blocks with a self row, 16-byte chunk per lane): the gathered chunk of every entry, and the self
+// chunk where a segment begins, are requested kRing entries ahead with cp.async into a ring in shared memory (each
+// thread reads back only what it requested itself, so the ring needs no barrier); the bytes in flight then no longer
+// occupy registers and do not stop at the four rows of a batch.
+template <typename T, typename PtrT, int LPR, int CPL, bool kWeight, int kExtra, int kInFlight, int kRing = 0>
 __global__ void __launch_bounds__(kAggThreads, (kInFlight <= 2 && !kExtra) ? 5 : 1)
 seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__ ptr, const int32_t *__restrict__ idx,
                const int32_t *n_seg_dev, int64_t n_seg_host, const float *__restrict__ w, int run_len, int d,
@@ -252,12 +266,36 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
             }
         };
 
+        static_assert(kRing == 0 || (CPL == 1 && !kWeight && kExtra == 1 && kRing >= U), "ring form: one chunk per lane, self rows only");
+        constexpr int kSlot = kAggThreads * 16;               // bytes of one ring slot (one 16-byte chunk per thread)
+        uint8_t *ring_g = reinterpret_cast<uint8_t *>(sh_info + RB) + threadIdx.x * 16;     // gathered chunks
+        uint8_t *ring_s = ring_g + (kRing > 0 ? kRing : 1) * kSlot;                            // self chunks
+        // requests entry r (same tests as the sums below make when they read the slot back)
+        auto issue = [&](int r) {
+            if (kRing > 0) {
+                if (r < len && c < n_chunks) {
+                    const int slot = r % (kRing > 0 ? kRing : 1);
+                    cp_async16(ring_g + slot * kSlot, in + (int64_t)idx0[r] * ld_in + c * E);
+                    const int32_t sg = seg0[r];
+                    const bool st = r == 0 || sg != seg0[r - 1];
+                    if (st && (r != 0 || first_begins) && sg < n_self)
+                        cp_async16(ring_s + slot * kSlot, o.self + (int64_t)sg * o.ld_self + c * E);
+                }
+                cp_async_commit();
+            }
+        };
+        if (kRing > 0) {
+#pragma unroll
+            for (int r = 0; r < (kRing > 0 ? kRing : 1); ++r) issue(r);
+        }
+
         classify(0);
         for (int r0 = 0; r0 < len; r0 += U) {
             int32_t seg_c[U];
             bool start_c[U];
             float wt[U];
             uint4 v[U][CPL], sv[kExtra ? U : 1][CPL], mv[kExtra == 2 ? U : 1][CPL];
+            if (kRing > 0) cp_async_wait<(kRing > U ? kRing - U : 0)>();       // the entries of this batch have landed
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 seg_c[u] = seg_n[u];
@@ -266,6 +304,17 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
                 const bool live = r0 + u < len;
                 const int32_t id = id_n[u];
                 if (kWeight && live) wt[u] = w[id];
+                if (kRing > 0) {
+                    const int slot = (r0 + u) % (kRing > 0 ? kRing : 1);
+                    v[u][0] = make_uint4(0, 0, 0, 0);
+                    sv[u][0] = make_uint4(0, 0, 0, 0);
+                    if (live && c < n_chunks) {
+                        v[u][0] = *reinterpret_cast<const uint4 *>(ring_g + slot * kSlot);
+                        if (start_c[u] && (r0 + u != 0 || first_begins) && seg_c[u] < n_self)
+                            sv[u][0] = *reinterpret_cast<const uint4 *>(ring_s + slot * kSlot);
+                    }
+                }
+                if (kRing == 0) {
 #pragma unroll
                 for (int q = 0; q < CPL; ++q) {
                     const int ch = c + q * LPR;
@@ -282,6 +331,7 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
                                 mv[u][q] = Chunk<T>::load_raw(o.mask + (int64_t)seg_c[u] * o.ld_mask + ch * E);
                         }
                     }
+                }
                 }
             }
             if (r0 + U < len) classify(r0 + U);
@@ -320,7 +370,12 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
                     }
                 }
             }
+            if (kRing > 0) {                                  // the slots just read take the entries kRing further on
+#pragma unroll
+                for (int u = 0; u < U; ++u) issue(r0 + (kRing > 0 ? kRing : 1) + u);
+            }
         }
+        if (kRing > 0) cp_async_wait<0>();
         emit(seg0 ? last_ends : rel_end <= len, len);
     }
     if (c == 0) sh_info[rl] = make_int4(head_seg, head_ends, tail_seg, 0);
@@ -586,6 +641,15 @@ inline void launch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const
         if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         kern<<<grid1, kAggThreads, smem, st>>>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head2, sc.tail2,
                                                sc.win_info, sc.cap_runs, seg_of, o);
+    } else if (o.self && kSegRing > 0 && CPL == 1 && !kWeight && sizeof(PtrT) == 4 && LPR >= 16 && kInFlight == 4 && seg_of) {
+        // rows of 256 bytes and more on a sampled block: the ring form
+        if constexpr (CPL == 1 && !kWeight && sizeof(PtrT) == 4 && LPR >= 16 && kInFlight == 4) {
+            constexpr size_t smem_ring = smem + (size_t)2 * kSegRing * kAggThreads * 16;
+            auto kern = seg_run_kernel<T, PtrT, LPR, CPL, kWeight, 1, kInFlight, kSegRing>;
+            cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_ring);
+            kern<<<grid1, kAggThreads, smem_ring, st>>>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head2,
+                                                        sc.tail2, sc.win_info, sc.cap_runs, seg_of, o);
+        }
     } else if (o.self) {
         auto kern = seg_run_kernel<T, PtrT, LPR, CPL, kWeight, 1, kInFlight>;
         if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
