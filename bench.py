@@ -47,12 +47,53 @@ def measured_peaks():
 
 
 class ClockSampler:
-    def __init__(self, gpu_index):
-        self.path = f"/tmp/e2egrec_clocks_{os.getpid()}.csv"
+    """SM clock and clock-event reasons read DURING the timed region.  NVML is polled from a thread every few
+    milliseconds (read-only queries), so even a region of tens of milliseconds holds several samples; without
+    the NVML module the same fields come from an `nvidia-smi -lms` child process."""
+    NAMES = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+
+    def __init__(self, gpu_index, period_s=0.004):
         self.gpu = gpu_index
-        self.p = None
+        self.period = period_s
+        self.rows = []                  # (time.time(), sm MHz, max sm MHz, [reason names])
+        self.thread = self.p = self.nv = None
+        self.stop_flag = False
+        self.path = f"/tmp/e2egrec_clocks_{os.getpid()}.csv"
+
+    def _nvml_handle(self):
+        import pynvml
+        pynvml.nvmlInit()
+        try:
+            uuid = str(torch.cuda.get_device_properties(self.gpu).uuid)
+            return pynvml, pynvml.nvmlDeviceGetHandleByUUID(("GPU-" + uuid).encode())
+        except Exception:
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES", "")
+            ids = [v for v in vis.split(",") if v.strip().isdigit()]
+            return pynvml, pynvml.nvmlDeviceGetHandleByIndex(int(ids[self.gpu]) if self.gpu < len(ids) else self.gpu)
+
+    def _poll(self):
+        nv, h = self.nv
+        bits = [nv.nvmlClocksEventReasonHwSlowdown, nv.nvmlClocksEventReasonHwThermalSlowdown,
+                nv.nvmlClocksEventReasonSwThermalSlowdown, nv.nvmlClocksEventReasonSwPowerCap]
+        smax = float(nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM))
+        while not self.stop_flag:
+            try:
+                mask = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
+                sm = float(nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM))
+                self.rows.append((time.time(), sm, smax, [n for n, b in zip(self.NAMES, bits) if mask & b]))
+            except Exception:
+                pass
+            time.sleep(self.period)
 
     def start(self):
+        try:
+            self.nv = self._nvml_handle()
+            import threading
+            self.thread = threading.Thread(target=self._poll, daemon=True)
+            self.thread.start()
+            return
+        except Exception:
+            self.nv = self.thread = None
         try:
             self.f = open(self.path, "w")
             self.p = subprocess.Popen(["nvidia-smi", "-i", str(self.gpu), f"--query-gpu={CLOCK_QUERY}",
@@ -62,42 +103,46 @@ class ClockSampler:
             self.p = None
 
     def mark(self):
-        """Wall-clock stamp in nvidia-smi's timestamp format resolution (seconds since epoch)."""
         return time.time()
 
-    def stop(self, t_begin=None, t_end=None):
-        if self.p is None:
-            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+    def _smi_rows(self):
+        import datetime
         self.p.terminate()
         try:
             self.p.wait(timeout=5)
         except Exception:
             self.p.kill()
         self.f.close()
-        sm, smax, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for line in open(self.path):
             c = [x.strip() for x in line.split(",")]
             if len(c) < 9:
                 continue
             try:
-                import datetime
                 ts = datetime.datetime.strptime(c[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
-                if t_begin is not None and not (t_begin - 0.05 <= ts <= t_end + 0.05):
-                    continue
-                sm.append(float(c[1]))
-                smax.append(float(c[2]))
+                self.rows.append((ts, float(c[1]), float(c[2]),
+                                  [n for n, v in zip(self.NAMES, c[5:9]) if v.lower().startswith("active")]))
             except ValueError:
                 continue
-            for n, v in zip(names, c[5:9]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
         try:
             os.remove(self.path)
         except OSError:
             pass
+
+    def stop(self, t_begin=None, t_end=None):
+        if self.thread is not None:
+            self.stop_flag = True
+            self.thread.join(timeout=2)
+            source, slack = "nvml", 0.0
+        elif self.p is not None:
+            self._smi_rows()
+            source, slack = "nvidia-smi", 0.05
+        else:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no clock source"], samples=0)
+        rows = [r for r in self.rows if t_begin is None or t_begin - slack <= r[0] <= t_end + slack]
+        sm, smax = [r[1] for r in rows], [r[2] for r in rows]
+        reasons = sorted({n for r in rows for n in r[3]})
         return dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=max(smax) if smax else None,
-                    reasons=sorted(reasons), samples=len(sm))
+                    reasons=reasons, samples=len(sm), source=source)
 
 
 def build_inputs(w: S.Workload, host_csr=True):
@@ -381,7 +426,7 @@ def run_ours(args, w):
     prime(Wm, seeds_dev)
     clocks = ClockSampler(local)
     clocks.start()
-    time.sleep(0.6)                                    # let the sampler reach its steady 100 ms period
+    time.sleep(0.3)                                    # the sampler is polling before the region starts
     barrier()
     t_begin = clocks.mark()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
