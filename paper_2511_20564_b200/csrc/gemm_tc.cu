@@ -161,6 +161,8 @@ struct TcEpilogue {
     const __nv_bfloat16 *mask; // optional [rows x ld_mask]: outputs are zeroed where mask <= 0 (ReLU derivative)
     int64_t ld_mask;
     const int32_t *m_dev;      // rows at and beyond *m_dev are written as zeros
+    __nv_bfloat16 *out2;       // optional second copy of the output: rows below rows2, leading dimension ldo2
+    int64_t ldo2, rows2;
     int32_t *status;           // device status word (E2EGREC_DEV_TIMEOUT)
 };
 
@@ -297,6 +299,7 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             const float rs = (ep.row_scale && live) ? ep.row_scale[row] : 1.f;
             __nv_bfloat16 *orow = ep.out + row * ep.ldo + n0;
             const __nv_bfloat16 *mrow = ep.mask ? ep.mask + row * ep.ld_mask + n0 : nullptr;
+            __nv_bfloat16 *orow2 = (ep.out2 && row < ep.rows2) ? ep.out2 + row * ep.ldo2 + n0 : nullptr;
             if (c_first >= nt) {                          // a single column block: nothing for the second set of warps
                 if (lane == 0) mbar_arrive(&acc_empty[buf]);
                 continue;
@@ -343,6 +346,12 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 for (int q = 0; q < 4; ++q)
                     *reinterpret_cast<uint4 *>(orow + c + q * 8) =
                         make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                if (orow2) {
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        *reinterpret_cast<uint4 *>(orow2 + c + q * 8) =
+                            make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+                }
             }
         }
     }
@@ -574,9 +583,14 @@ bool make_map_mn(CUtensorMap *map, const void *base, int64_t rows, int64_t cols)
 }  // namespace
 
 bool tc_update_forward(const __nv_bfloat16 *cat, int64_t rows, int k, const __nv_bfloat16 *W, int n, const float *bias,
-                       int relu, __nv_bfloat16 *out, const int32_t *m_dev, int32_t *status, cudaStream_t st)
+                       int relu, __nv_bfloat16 *out, const int32_t *m_dev, int32_t *status, cudaStream_t st,
+                       __nv_bfloat16 *out2, int64_t ldo2, int64_t rows2)
 {
+    if (out2 && (reinterpret_cast<uintptr_t>(out2) % 16 || (ldo2 * 2) % 16 || ldo2 < n)) return false;
     TcEpilogue ep{};
+    ep.out2 = out2;
+    ep.ldo2 = ldo2;
+    ep.rows2 = rows2;
     ep.out = out;
     ep.ldo = n;
     ep.bias = bias;

@@ -9,8 +9,10 @@ namespace e2egrec {
 // row-major; rows at and beyond *m_dev inside a partly used 128-row tile are written as zeros, tiles
 // wholly beyond it are left alone.  `status` receives E2EGREC_DEV_TIMEOUT if a bounded wait runs out.
 // Returns false when the shape is outside what the kernel takes, in which case nothing was enqueued.
+// out2 (optional, [rows2 x ldo2]): the rows below rows2 of every written tile are stored there as well.
 bool tc_update_forward(const __nv_bfloat16 *cat, int64_t rows, int k, const __nv_bfloat16 *W, int n, const float *bias,
-                       int relu, __nv_bfloat16 *out, const int32_t *m_dev, int32_t *status, cudaStream_t st);
+                       int relu, __nv_bfloat16 *out, const int32_t *m_dev, int32_t *status, cudaStream_t st,
+                       __nv_bfloat16 *out2 = nullptr, int64_t ldo2 = 0, int64_t rows2 = 0);
 
 // dCat = dZ W with the layer weight W [d_out x 2 d_in] as stored (the tensor cores read it with its N index
 // contiguous, no transposed copy is made); columns >= d_in are scaled by inv_cnt[row].  2 d_in must be a multiple

@@ -35,10 +35,9 @@ IngestScratch carve_ingest(int64_t m, void *base)
     s.rs.tiles = ceil_div((int64_t)mm, kSortTile);
     const size_t arena_begin = off;
     s.arena = base ? static_cast<char *>(base) + off : nullptr;
-    s.rs.tickets = (unsigned *)take(256);
     s.rs.ghist = (unsigned *)take(sizeof(unsigned) * kMaxPasses * kMaxRadix);
-    s.rs.state = (unsigned long long *)take(8 * (size_t)kMaxPasses * kMaxRadix * (size_t)s.rs.tiles);
     s.arena_bytes = off - arena_begin;
+    s.rs.thist = (int32_t *)take(radix_thist_bytes(s.rs.tiles));
     s.bytes = off;
     return s;
 }

@@ -1,6 +1,6 @@
 // Building blocks shared by the sampler and the graph ingest: single-pass prefix sums across thread
-// blocks, and a stable least-significant-digit radix sort of (int32 key, int32 value) pairs with one
-// launch per digit.
+// blocks, and a stable least-significant-digit radix sort of (int32 key, int32 value) pairs (counts per
+// tile, scan over tiles, scatter: three launches per digit).
 #pragma once
 
 #include "common.cuh"
@@ -82,28 +82,79 @@ __device__ inline int chain_ticket(unsigned *ticket, int *bcast)
 
 
 // ---------------------------------------------------------------------------------------
-// Stable LSD radix sort of (key = col, value = block position), one launch per digit.  A block owns
-// a tile of kSortTile consecutive elements, ranks equal digits in element order (per warp by
-// match_any, then across warps), and finds where its elements of each digit start from the digit's
-// global start (digit counts of the whole array, known beforehand) plus a per-digit chained scan
-// over the tiles before it.
+// Stable LSD radix sort of (key = col, value = block position), three launches per digit and no
+// waiting between thread blocks: (1) digit counts of every tile of kSortTile consecutive elements,
+// (2) per digit an exclusive scan of those counts over the tiles, (3) the scatter: a block ranks
+// the equal digits of its tile in element order (per warp by match_any, then across warps) and
+// places them at  start of the digit's bin (digit counts of the whole array, known beforehand)
+// + count of that digit in the tiles before it + rank.
 // ---------------------------------------------------------------------------------------
 template <int BITS>
 __global__ void __launch_bounds__(kSortThreads)
+tile_hist_kernel(const int32_t *__restrict__ keys, const int32_t *__restrict__ counts, int shift,
+                 int32_t *__restrict__ thist)
+{
+    constexpr int R = 1 << BITS;
+    constexpr int W = kSortThreads / 32;
+    __shared__ int32_t h[W][R];                  // one histogram per warp: fewer colliding atomics
+    const int32_t n = counts[CNT_EDGES];
+    const int64_t n_live = ((int64_t)n + kSortTile - 1) / kSortTile;
+    const int warp = threadIdx.x >> 5;
+    for (int64_t tile = blockIdx.x; tile < n_live; tile += gridDim.x) {
+        for (int d = threadIdx.x; d < W * R; d += kSortThreads) (&h[0][0])[d] = 0;
+        __syncthreads();
+        const int64_t base = tile * kSortTile;
+#pragma unroll
+        for (int k = 0; k < kSortItems; ++k) {
+            const int64_t idx = base + k * kSortThreads + threadIdx.x;
+            if (idx < n) atomicAdd(&h[warp][(keys[idx] >> shift) & (R - 1)], 1);
+        }
+        __syncthreads();
+        for (int d = threadIdx.x; d < R; d += kSortThreads) {
+            int32_t c = 0;
+#pragma unroll
+            for (int w = 0; w < W; ++w) c += h[w][d];
+            thist[tile * R + d] = c;
+        }
+        __syncthreads();
+    }
+}
+
+// thist[tile][d] <- sum of thist[tile'][d] over tile' < tile; one block per digit d
+template <int BITS>
+__global__ void __launch_bounds__(kSortThreads)
+tile_scan_kernel(const int32_t *__restrict__ counts, int32_t *__restrict__ thist)
+{
+    constexpr int R = 1 << BITS;
+    __shared__ int32_t scan_sm[kSortThreads / 32 + 1];
+    const int32_t n = counts[CNT_EDGES];
+    const int64_t n_live = ((int64_t)n + kSortTile - 1) / kSortTile;
+    const int d = blockIdx.x;
+    int32_t carry = 0;
+    for (int64_t t0 = 0; t0 < n_live; t0 += kSortThreads) {
+        const int64_t t = t0 + threadIdx.x;
+        const int32_t v = t < n_live ? thist[t * R + d] : 0;
+        int32_t tot;
+        const int32_t ex = block_exclusive_scan<kSortThreads, int32_t>(v, tot, scan_sm);
+        if (t < n_live) thist[t * R + d] = carry + ex;
+        carry += tot;
+    }
+}
+
+template <int BITS>
+__global__ void __launch_bounds__(kSortThreads)
 sort_pass_kernel(const int32_t *__restrict__ keys_in, const int32_t *__restrict__ vals_in,
-                 int32_t *__restrict__ counts, int shift, const unsigned *__restrict__ ghist, int n_tiles,
-                 unsigned long long *__restrict__ state, unsigned *ticket, int32_t *__restrict__ keys_out,
-                 int32_t *__restrict__ vals_out)
+                 const int32_t *__restrict__ counts, int shift, const unsigned *__restrict__ ghist,
+                 const int32_t *__restrict__ thist, int32_t *__restrict__ keys_out, int32_t *__restrict__ vals_out)
 {
     constexpr int R = 1 << BITS;
     constexpr int W = kSortThreads / 32;
     __shared__ int32_t wc[W][R];                 // per-warp digit counts, then start offsets
     __shared__ int32_t bin_base[R];
     __shared__ int32_t scan_sm[kSortThreads / 32 + 1];
-    __shared__ int tile_s;
-    const int tile = chain_ticket(ticket, &tile_s);
+    const int64_t tile = blockIdx.x;
     const int32_t n = counts[CNT_EDGES];
-    if ((int64_t)tile * kSortTile >= n) return;
+    if (tile * kSortTile >= n) return;
     for (int d = threadIdx.x; d < W * R; d += kSortThreads) (&wc[0][0])[d] = 0;
     // start of every digit's bin: exclusive scan of the global digit counts
     {
@@ -119,7 +170,7 @@ sort_pass_kernel(const int32_t *__restrict__ keys_in, const int32_t *__restrict_
     }
     __syncthreads();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t wbase = (int64_t)tile * kSortTile + (int64_t)warp * (32 * kSortItems);
+    const int64_t wbase = tile * kSortTile + (int64_t)warp * (32 * kSortItems);
     int32_t key[kSortItems], val[kSortItems], rank[kSortItems];
 #pragma unroll
     for (int k = 0; k < kSortItems; ++k) {
@@ -140,69 +191,9 @@ sort_pass_kernel(const int32_t *__restrict__ keys_in, const int32_t *__restrict_
         __syncwarp();
     }
     __syncthreads();
-    // per digit: publish this tile's count, then a chained look-back over earlier tiles, then warp start offsets
-    constexpr int DPT = (R + kSortThreads - 1) / kSortThreads;
-    int32_t cnt[DPT];
-#pragma unroll
-    for (int q = 0; q < DPT; ++q) {
-        const int d = threadIdx.x + q * kSortThreads;
-        cnt[q] = 0;
-        if (d < R) {
-#pragma unroll
-            for (int w = 0; w < W; ++w) cnt[q] += wc[w][d];
-            atomicExch(&state[(size_t)d * n_tiles + tile], (tile == 0 ? kChainPrefix : kChainAgg) | (unsigned long long)cnt[q]);
-        }
-    }
-    // look-back for all of this thread's digits together: a batch of earlier tiles per digit is read at
-    // once, then taken in order; an entry that is not published yet is polled (bounded) before going on
-    long long excl[DPT];
-    int next_p[DPT];
-    bool timed_out = false;
-#pragma unroll
-    for (int q = 0; q < DPT; ++q) {
-        excl[q] = 0;
-        next_p[q] = (threadIdx.x + q * kSortThreads < R && tile > 0) ? tile - 1 : -1;
-    }
-    for (;;) {
-        bool any = false;
-#pragma unroll
-        for (int q = 0; q < DPT; ++q) any = any || next_p[q] >= 0;
-        if (!any || timed_out) break;
-        constexpr int kBatch = 8;
-        unsigned long long v[DPT][kBatch];
-#pragma unroll
-        for (int q = 0; q < DPT; ++q) {
-            const unsigned long long *st = state + (size_t)(threadIdx.x + q * kSortThreads) * n_tiles;
-#pragma unroll
-            for (int j = 0; j < kBatch; ++j) v[q][j] = next_p[q] - j >= 0 ? chain_read(&st[next_p[q] - j]) : kChainPrefix;
-        }
-#pragma unroll
-        for (int q = 0; q < DPT; ++q) {
-            if (next_p[q] < 0) continue;
-            const unsigned long long *st = state + (size_t)(threadIdx.x + q * kSortThreads) * n_tiles;
-            bool found = false;
-#pragma unroll
-            for (int j = 0; j < kBatch; ++j) {
-                if (found || timed_out) continue;
-                unsigned long long x = v[q][j];
-                for (int spin = 0; (x >> 62) == 0; ++spin) {
-                    if (spin >= kChainSpinLimit) { timed_out = true; break; }
-                    x = chain_read(&st[next_p[q] - j]);
-                }
-                if (timed_out) continue;
-                excl[q] += (long long)(x & kChainMask);
-                if ((x >> 62) == 2) found = true;
-            }
-            next_p[q] = found ? -1 : next_p[q] - kBatch;
-        }
-    }
-    if (timed_out) atomicOr(reinterpret_cast<unsigned *>(&counts[CNT_STATUS]), E2EGREC_DEV_TIMEOUT);
-#pragma unroll
-    for (int q = 0; q < DPT; ++q) {
-        const int d = threadIdx.x + q * kSortThreads;
-        if (d >= R) continue;
-        if (tile > 0) atomicExch(&state[(size_t)d * n_tiles + tile], kChainPrefix | (unsigned long long)(excl[q] + cnt[q]));
-        int32_t run = bin_base[d] + (int32_t)excl[q];
+    // per digit: where the elements of each warp start
+    for (int d = threadIdx.x; d < R; d += kSortThreads) {
+        int32_t run = bin_base[d] + thist[tile * R + d];
 #pragma unroll
         for (int w = 0; w < W; ++w) {
             const int32_t c2 = wc[w][d];
@@ -259,17 +250,32 @@ key_hist_kernel(const int32_t *__restrict__ keys, const int32_t *__restrict__ co
         if (h[d]) atomicAdd(&ghist[(d / R) * kMaxRadix + (d % R)], h[d]);
 }
 
-// Buffers of one sort: two ping-pong pairs and the zeroed arena (tickets, digit counts, tile states).
+// Buffers of one sort: two ping-pong pairs, the digit counts of the whole array (filled before the sort) and
+// the per-tile digit counts (written before they are read: no zeroing needed).
 struct RadixScratch {
     int32_t *keys[2], *vals[2];        // [n] each
-    unsigned *tickets;                 // [kMaxPasses]
     unsigned *ghist;                   // [kMaxPasses x kMaxRadix]
-    unsigned long long *state;         // [kMaxPasses x kMaxRadix x tiles]
+    int32_t *thist;                    // [tiles x radix], reused by every pass
     int64_t tiles;
 };
 
+constexpr size_t radix_thist_bytes(int64_t tiles) { return sizeof(int32_t) * (size_t)kMaxRadix * (size_t)tiles; }
+
+template <int BITS>
+static inline void radix_pass(const int32_t *kin, const int32_t *vin, int32_t *counts, int n_tiles, int shift,
+                              const unsigned *ghist, int32_t *thist, int32_t *kout, int32_t *vout, cudaStream_t st)
+{
+    const int hist_grid = n_tiles < 8 * 148 ? n_tiles : 8 * 148;
+    note_launch();
+    tile_hist_kernel<BITS><<<hist_grid, kSortThreads, 0, st>>>(kin, counts, shift, thist);
+    note_launch();
+    tile_scan_kernel<BITS><<<1 << BITS, kSortThreads, 0, st>>>(counts, thist);
+    note_launch();
+    sort_pass_kernel<BITS><<<n_tiles, kSortThreads, 0, st>>>(kin, vin, counts, shift, ghist, thist, kout, vout);
+}
+
 // Sorts (keys, vals) by key, stable; vals == nullptr means "value = position".  counts[CNT_EDGES] holds the
-// number of elements (device).  ghist must already hold the digit counts; tickets / state must be zero.
+// number of elements (device).  ghist must already hold the digit counts.
 static inline void radix_sort_pairs(const int32_t *keys, const int32_t *vals, int32_t *counts, int64_t cap,
                                     int32_t *keys_out, int32_t *vals_out, const SortPlan &sp, const RadixScratch &rs,
                                     cudaStream_t st)
@@ -281,14 +287,10 @@ static inline void radix_sort_pairs(const int32_t *keys, const int32_t *vals, in
         const bool last = p == sp.passes - 1;
         int32_t *kout = last ? keys_out : rs.keys[p & 1];
         int32_t *vout = last ? vals_out : rs.vals[p & 1];
-        unsigned long long *state = rs.state + (size_t)p * kMaxRadix * (size_t)rs.tiles;
-        note_launch();
         if (sp.bits == 8)
-            sort_pass_kernel<8><<<n_tiles, kSortThreads, 0, st>>>(kin, vin, counts, p * sp.bits, rs.ghist + p * kMaxRadix, n_tiles,
-                                                                 state, rs.tickets + p, kout, vout);
+            radix_pass<8>(kin, vin, counts, n_tiles, p * sp.bits, rs.ghist + p * kMaxRadix, rs.thist, kout, vout, st);
         else
-            sort_pass_kernel<10><<<n_tiles, kSortThreads, 0, st>>>(kin, vin, counts, p * sp.bits, rs.ghist + p * kMaxRadix, n_tiles,
-                                                                  state, rs.tickets + p, kout, vout);
+            radix_pass<10>(kin, vin, counts, n_tiles, p * sp.bits, rs.ghist + p * kMaxRadix, rs.thist, kout, vout, st);
         kin = kout;
         vin = vout;
     }

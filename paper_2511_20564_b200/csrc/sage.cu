@@ -91,6 +91,8 @@ static int32_t forward_impl(const e2egrec_block *blocks, int32_t n_layers, const
                             const e2egrec_mat *H_out, cudaStream_t st)
 {
     const size_t es = sizeof(T);
+    const int64_t out_rows = blocks[0].cap_dst < H_out->rows ? blocks[0].cap_dst : H_out->rows;
+    bool top_stored = false;
     for (int l = 0; l < n_layers; ++l) {
         const LayerPlan &p = plan[l];
         const e2egrec_block &b = blocks[p.block];
@@ -108,10 +110,15 @@ static int32_t forward_impl(const e2egrec_block *blocks, int32_t n_layers, const
         const int relu = act ? act[l] : 1;
         bool done = false;
         if (l == 0) tap_begin(TAP_UPDATE_FWD_OUTER, st);
-        if (X->dtype == E2EGREC_BF16)
+        if (X->dtype == E2EGREC_BF16) {
+            // the last layer's product stores its rows into H_out as well as into the context
+            const bool top = l == n_layers - 1;
             done = tc_update_forward(reinterpret_cast<const __nv_bfloat16 *>(cat), p.rows, 2 * p.d_in,
                                      static_cast<const __nv_bfloat16 *>(W[l].data), p.d_out, bl, relu,
-                                     reinterpret_cast<__nv_bfloat16 *>(hn), &b.counts[CNT_DST], &b.counts[CNT_STATUS], st);
+                                     reinterpret_cast<__nv_bfloat16 *>(hn), &b.counts[CNT_DST], &b.counts[CNT_STATUS], st,
+                                     top ? static_cast<__nv_bfloat16 *>(H_out->data) : nullptr, H_out->ld, out_rows);
+            top_stored = done && top;
+        }
         if (!done) {
             EpiUpdate<T> epi{hn, p.d_out, bl, relu};
             dim3 grid((unsigned)std::max<int64_t>(1, ceil_div(p.rows, kGemmBM)), (unsigned)ceil_div(p.d_out, kGemmBN), 1);
@@ -123,8 +130,8 @@ static int32_t forward_impl(const e2egrec_block *blocks, int32_t n_layers, const
         if (l == 0) tap_end(TAP_UPDATE_FWD_OUTER, st);
     }
     const LayerPlan &top = plan[n_layers - 1];
-    const int64_t rows = blocks[0].cap_dst < H_out->rows ? blocks[0].cap_dst : H_out->rows;
-    if (rows > 0)
+    const int64_t rows = out_rows;
+    if (rows > 0 && !top_stored)
         cudaMemcpy2DAsync(H_out->data, (size_t)H_out->ld * es, ctx + top.h_off, (size_t)top.d_out * es,
                       (size_t)top.d_out * es, (size_t)rows, cudaMemcpyDeviceToDevice, st);
     return check_launch("sage_forward");

@@ -46,10 +46,7 @@ struct SortLane {
     int32_t  *keys[2];     // [max cap_edges]   radix sort ping-pong
     int32_t  *vals[2];
     unsigned *ghist;                   // [kMaxPasses x kMaxRadix] digit counts of the whole key array (zeroed before relabel)
-    char     *arena;                   // tickets + tile states, zeroed before the sort
-    size_t    arena_bytes;
-    unsigned *tickets;                 // [kMaxPasses]
-    unsigned long long *state;         // [kMaxPasses x kMaxRadix x sort tiles]
+    int32_t  *thist;                   // [sort tiles x kMaxRadix] digit counts per tile of the pass that runs
 };
 
 struct SamplerScratch {
@@ -95,11 +92,7 @@ static SamplerScratch carve(int64_t n_nodes, int64_t max_dst, int64_t max_src, i
         for (int i = 0; i < 2; ++i) l.keys[i] = (int32_t *)take(sizeof(int32_t) * (size_t)(max_edges + 1));
         for (int i = 0; i < 2; ++i) l.vals[i] = (int32_t *)take(sizeof(int32_t) * (size_t)(max_edges + 1));
         l.ghist = (unsigned *)take(sizeof(unsigned) * kMaxPasses * kMaxRadix);
-        begin = off;
-        l.arena = base ? static_cast<char *>(base) + off : nullptr;
-        l.tickets = (unsigned *)take(256);
-        l.state = (unsigned long long *)take(8 * (size_t)kMaxPasses * kMaxRadix * (size_t)s.sort_tiles);
-        l.arena_bytes = off - begin;
+        l.thist = (int32_t *)take(radix_thist_bytes(s.sort_tiles));
     }
     s.bytes = off;
     return s;
@@ -423,9 +416,8 @@ static void sort_by_col(const int32_t *col, int32_t *counts, int32_t cap_edges, 
     RadixScratch rs{};
     rs.keys[0] = l.keys[0]; rs.keys[1] = l.keys[1];
     rs.vals[0] = l.vals[0]; rs.vals[1] = l.vals[1];
-    rs.tickets = l.tickets;
     rs.ghist = l.ghist;
-    rs.state = l.state;
+    rs.thist = l.thist;
     rs.tiles = sort_tiles;
     radix_sort_pairs(col, nullptr, counts, cap_edges, csc_col, csc_eid, sp, rs, st);
 }
@@ -608,7 +600,6 @@ int32_t e2egrec::sample_khop_impl(const e2egrec_csr *graph, const int32_t *seeds
         const SortPlan sp = sort_plan(P2 > 1 ? P2 : 2);
         const SortLane &l = s.lane[0];
         cudaMemsetAsync(l.ghist, 0, sizeof(unsigned) * kMaxPasses * kMaxRadix, st);
-        cudaMemsetAsync(l.arena, 0, l.arena_bytes, st);
         note_launch();
         pair_local_kernel<<<(unsigned)std::min<int64_t>(grid_for(P2, T), 148 * 4), T, 0, st>>>(
             pi.user, pi.item, pi.n_pairs, n, s.local_id, pi.pair_local, pi.entry_unit, pi.units_per_row, pi.item_unit_off,
@@ -648,7 +639,6 @@ int32_t e2egrec::sample_khop_impl(const e2egrec_csr *graph, const int32_t *seeds
             side->fork(st);
             ts = side->stream;
         }
-        cudaMemsetAsync(l.arena, 0, l.arena_bytes, ts);
         sort_by_col(b.col, b.counts, b.cap_edges, b.csc_col, b.csc_eid, sp, l, s.sort_tiles, ts);
         note_launch();
         csc_finalize_kernel<<<grid_for(std::max<int64_t>(b.cap_edges, (int64_t)b.cap_src + 1), T), T, 0, ts>>>(
