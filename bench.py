@@ -244,7 +244,7 @@ def run_ours(args, w):
     want_cpu = world == 1 and not args.no_cpu_baseline
     dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
     K, Wm = args.steps, args.warmup
-    total = K + Wm + 2                                 # + the batches whose sampling / upload is prefetched during the last steps
+    total = K + Wm + 4                                 # + the batches whose sampling / upload is prefetched during the last steps
     first_step = rank * 1_000_000                      # = replicas.first_step_of(rank)
     on_device = w.n_interactions > 200_000_000         # too large for host-side generation: drawn with torch on the GPU
     t_setup = time.perf_counter()
@@ -298,28 +298,33 @@ def run_ours(args, w):
     dH_pin = torch.from_numpy(dH_h).to(dt).pin_memory()
     dH = dH_pin.to(dev)
 
-    # two sets of block buffers: while the forward/backward of one batch runs, the next batch is sampled beside it
-    blocks2 = [E.Blocks(w.n_nodes, w.batch, w.fanouts, dev) for _ in range(2)]
+    # three sets of block buffers, one per stage of the step's pipeline: the hops of batch i + 2 are sampled and the
+    # transposed form of batch i + 1 is built while the forward/backward of batch i runs
+    NB = 3
+    blocks2 = [E.Blocks(w.n_nodes, w.batch, w.fanouts, dev) for _ in range(NB)]
     blocks = blocks2[0]
     L = len(Ws)
     ctx = torch.empty(E.binding.sage_forward_ctx_bytes(blocks, X, Ws), dtype=torch.uint8, device=dev)
     # outputs, the upstream gradient and a snapshot of the block counts exist once per buffer set, so that the copies
     # of one step's results and of the next step's inputs can run beside the step in between
-    H_out2 = [torch.zeros(blocks.caps[0][0], w.hidden, dtype=dt, device=dev) for _ in range(2)]
+    H_out2 = [torch.zeros(blocks.caps[0][0], w.hidden, dtype=dt, device=dev) for _ in range(NB)]
     H_out = H_out2[0]
     scratch = torch.empty(E.binding.sage_backward_scratch_bytes(blocks, X, Ws), dtype=torch.uint8, device=dev)
-    dWs2 = [[torch.zeros(W.shape, dtype=torch.float32, device=dev) for W in Ws] for _ in range(2)]
+    dWs2 = [[torch.zeros(W.shape, dtype=torch.float32, device=dev) for W in Ws] for _ in range(NB)]
     dWs = dWs2[0]
     dX = torch.zeros(blocks.caps[L - 1][1], w.dim, dtype=dt, device=dev)
 
-    seeds_in2 = [torch.empty(w.batch, dtype=torch.int32, device=dev) for _ in range(2)]
-    dH_in2 = [torch.empty_like(dH) for _ in range(2)]
-    counts_snap2 = [torch.zeros(L, 4, dtype=torch.int32, device=dev) for _ in range(2)]
+    seeds_in2 = [torch.empty(w.batch, dtype=torch.int32, device=dev) for _ in range(NB)]
+    dH_in2 = [torch.empty_like(dH) for _ in range(NB)]
+    counts_snap2 = [torch.zeros(L, 4, dtype=torch.int32, device=dev) for _ in range(NB)]
     count_total = torch.zeros(L, 4, dtype=torch.int64, device=dev)
 
-    def sample_leg(p, defer=False):
+    def sample_leg(p, defer=False, transpose=True):
         E.sample_khop(indptr, indices, seeds_in2[p], blocks2[p], w.seed, 0, defer_transpose=defer,
-                      edge_cum=edge_cum)                 # step = the scratch's offset
+                      edge_cum=edge_cum, transpose=transpose)     # step = the scratch's offset
+
+    def transpose_leg(p):
+        E.blocks_transpose(blocks2[p])
 
     if args.multitask:
         # the two-task step of Sec. 4.2: the recommendation gradient and the gradient of the SSL reconstruction loss go
@@ -356,8 +361,9 @@ def run_ours(args, w):
         torch.cuda.synchronize()
 
     # ---- record the step as CUDA graphs (no host work between the kernels) and replay them.  Graph p holds the
-    # forward/backward of the batch in buffer p and, on a second stream, the sampling of the next batch into buffer 1-p.
-    side, side2 = torch.cuda.Stream(), torch.cuda.Stream()
+    # forward/backward of the batch in buffer p and, on two more streams, the transposed form of the batch in buffer
+    # p + 1 and the hops of the batch after that into buffer p + 2 (indices mod 3).
+    side, side2, side3 = torch.cuda.Stream(), torch.cuda.Stream(priority=-1), torch.cuda.Stream(priority=-1)
     for t in dH_in2:
         t.copy_(dH)
     with torch.cuda.stream(side):
@@ -365,24 +371,32 @@ def run_ours(args, w):
             seeds_in2[0].copy_(seeds_dev[i])
             E.sampler_set_step(blocks.scratch, first_step + i)
             step_body()
-        seeds_in2[1].copy_(seeds_dev[0])
-        E.sampler_set_step(blocks2[1].scratch, first_step)
-        with torch.cuda.stream(side2):                   # the second buffer and the second stream, once, eagerly
-            side2.wait_stream(side)
-            sample_leg(1)
-        side.wait_stream(side2)
-        compute_leg(1)
+        for p in range(1, NB):                           # the other buffers and streams, once, eagerly
+            seeds_in2[p].copy_(seeds_dev[0])
+            E.sampler_set_step(blocks2[p].scratch, first_step)
+            with torch.cuda.stream(side2):
+                side2.wait_stream(side)
+                sample_leg(p, transpose=False)
+            with torch.cuda.stream(side3):
+                side3.wait_stream(side2)
+                transpose_leg(p)
+            side.wait_stream(side3)
+            compute_leg(p)
     side.synchronize()
     graphs, kernels_per_step = [], 0
-    for p in range(2):
+    for p in range(NB):
         launches_before = E.launch_count()
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g, stream=side):
             side2.wait_stream(side)
+            side3.wait_stream(side)
             with torch.cuda.stream(side2):
-                sample_leg(1 - p)
+                sample_leg((p + 2) % NB, transpose=False)
+            with torch.cuda.stream(side3):
+                transpose_leg((p + 1) % NB)
             compute_leg(p)
             side.wait_stream(side2)
+            side.wait_stream(side3)
         graphs.append(g)
         kernels_per_step = E.launch_count() - launches_before + 2   # + the counter update and snapshot (torch kernels)
 
@@ -397,16 +411,18 @@ def run_ours(args, w):
         step_body()
 
     def prime(i, src):
-        """Samples batch i into buffer i & 1 (what the previous replay would have done)."""
-        seeds_in2[i & 1].copy_(src[i], non_blocking=True)
-        E.sampler_set_step(blocks2[i & 1].scratch, first_step + i)
-        sample_leg(i & 1)
+        """What the two replays before step i would have done: batch i sampled and transposed into buffer i % 3,
+        the hops of batch i + 1 into the next buffer."""
+        for k, tr in ((i, True), (i + 1, False)):
+            seeds_in2[k % NB].copy_(src[k], non_blocking=True)
+            E.sampler_set_step(blocks2[k % NB].scratch, first_step + k)
+            sample_leg(k % NB, transpose=tr)
 
     def replay_step(i, src):
-        """Forward/backward of batch i (sampled by the previous replay) beside the sampling of batch i + 1."""
-        seeds_in2[(i + 1) & 1].copy_(src[i + 1], non_blocking=True)
-        E.sampler_set_step(blocks2[(i + 1) & 1].scratch, first_step + i + 1)
-        graphs[i & 1].replay()
+        """Forward/backward of batch i beside the transposition of batch i + 1 and the hops of batch i + 2."""
+        seeds_in2[(i + 2) % NB].copy_(src[i + 2], non_blocking=True)
+        E.sampler_set_step(blocks2[(i + 2) % NB].scratch, first_step + i + 2)
+        graphs[i % NB].replay()
 
     def tapped_step(i, which):
         """One eagerly launched step with events around kernel group `which`.  The device is first kept
@@ -452,36 +468,36 @@ def run_ours(args, w):
     # next step's inputs (seeds of the batch sampled next, upstream gradient) while the step runs; the download of
     # the step's results while the next step runs.  The host reads the results of step i while step i + 1 runs.
     res_pin2 = [[torch.empty(H_out.shape, dtype=dt).pin_memory()] +
-                [torch.empty(W.shape, dtype=torch.float32).pin_memory() for W in Ws] for _ in range(2)]
-    cnt_pin2 = [torch.empty(L, 4, dtype=torch.int32).pin_memory() for _ in range(2)]
+                [torch.empty(W.shape, dtype=torch.float32).pin_memory() for W in Ws] for _ in range(NB)]
+    cnt_pin2 = [torch.empty(L, 4, dtype=torch.int32).pin_memory() for _ in range(NB)]
     h2d = seeds_pin[0].numel() * 4 + dH_pin.numel() * dH_pin.element_size()
     d2h = sum(t.numel() * t.element_size() for t in res_pin2[0]) + cnt_pin2[0].numel() * 4
     main_s = torch.cuda.current_stream()
     up_s, down_s = torch.cuda.Stream(), torch.cuda.Stream()
     ev = lambda: torch.cuda.Event()
-    done_ev, up_ev, out_ev = [ev(), ev()], [ev(), ev()], [ev(), ev()]
+    done_ev, up_ev, out_ev = [ev() for _ in range(NB)], [ev() for _ in range(NB)], [ev() for _ in range(NB)]
 
     def e2e_run(first, count):
         """Steps first .. first + count - 1; returns the edges their results report."""
         edges = 0
-        prime(first, seeds_pin)                                     # batch `first` sampled into its buffer
+        prime(first, seeds_pin)                                     # batches `first`, `first + 1` into their buffers
         with torch.cuda.stream(up_s):
             up_s.wait_stream(main_s)
-            seeds_in2[(first + 1) & 1].copy_(seeds_pin[first + 1], non_blocking=True)
-            dH_in2[first & 1].copy_(dH_pin, non_blocking=True)
-            up_ev[first & 1].record(up_s)
+            seeds_in2[(first + 2) % NB].copy_(seeds_pin[first + 2], non_blocking=True)
+            dH_in2[first % NB].copy_(dH_pin, non_blocking=True)
+            up_ev[first % NB].record(up_s)
         for i in range(first, first + count):
-            p = i & 1
+            p, q = i % NB, (i + 1) % NB
             main_s.wait_event(up_ev[p])                              # inputs of step i are on the device
-            E.sampler_set_step(blocks2[1 - p].scratch, first_step + i + 1)
+            E.sampler_set_step(blocks2[(i + 2) % NB].scratch, first_step + i + 2)
             graphs[p].replay()
             done_ev[p].record(main_s)
             with torch.cuda.stream(up_s):                            # inputs of step i + 1, beside step i
                 if i > first:
-                    up_s.wait_event(done_ev[1 - p])                  # step i - 1 no longer reads these buffers
-                seeds_in2[p].copy_(seeds_pin[i + 2], non_blocking=True)
-                dH_in2[1 - p].copy_(dH_pin, non_blocking=True)
-                up_ev[1 - p].record(up_s)
+                    up_s.wait_event(done_ev[(i - 1) % NB])           # step i - 1 no longer reads these buffers
+                seeds_in2[p].copy_(seeds_pin[i + 3], non_blocking=True)    # read by step i + 1 (hops of batch i + 3)
+                dH_in2[q].copy_(dH_pin, non_blocking=True)
+                up_ev[q].record(up_s)
             with torch.cuda.stream(down_s):                          # results of step i, beside step i + 1
                 down_s.wait_event(done_ev[p])
                 res_pin2[p][0].copy_(H_out2[p], non_blocking=True)
@@ -490,9 +506,9 @@ def run_ours(args, w):
                 cnt_pin2[p].copy_(counts_snap2[p], non_blocking=True)
                 out_ev[p].record(down_s)
             if i > first:                                            # the caller reads the results of step i - 1
-                out_ev[1 - p].synchronize()
-                edges += int(cnt_pin2[1 - p][:, 2].sum())
-        last = (first + count - 1) & 1
+                out_ev[(i - 1) % NB].synchronize()
+                edges += int(cnt_pin2[(i - 1) % NB][:, 2].sum())
+        last = (first + count - 1) % NB
         out_ev[last].synchronize()
         edges += int(cnt_pin2[last][:, 2].sum())
         torch.cuda.synchronize()
@@ -627,8 +643,8 @@ def run_ours(args, w):
                             tasks="recommendation gradient + SSL reconstruction loss, two backward passes, GradNorm step"
                                   if args.multitask else "recommendation gradient",
                             parallelism=f"replicas x{world}",
-                            launch="one CUDA graph replay per step: forward/backward of the batch beside the sampling of "
-                                   "the next batch on a second stream (two sets of block buffers)",
+                            launch="one CUDA graph replay per step, three streams: forward/backward of batch i beside the "
+                                   "transposed form of batch i+1 and the hops of batch i+2 (three sets of block buffers)",
                             l2="inputs larger than L2: feature table + graph = %.0f MB, a new batch every step"
                                % ((X.numel() * es + indices.numel() * 4 + indptr.numel() * 8) / 1e6),
                             edges_per_step=edges_rank / K, setup_s=round(setup_s, 1),
@@ -728,7 +744,9 @@ def run_lightgcn(args, w):
         E.lightgcn_sampled_backward(blocks2[p], ctx, dY, dX_rows=dX, scratch=scratch)
         count_total.add_(blocks2[p].counts)
 
-    side, side2 = torch.cuda.Stream(), torch.cuda.Stream()
+    # the sampling leg runs at high priority: its short dependent kernels take the next free slots of an SM
+    # instead of queueing behind the thousands of blocks of a gather or a dense product
+    side, side2 = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
     with torch.cuda.stream(side):
         for i in range(max(Wm, 3)):
             for p in range(2):

@@ -63,6 +63,7 @@ extern "C" {
 
 /* flags of e2egrec_sample_khop */
 #define E2EGREC_SAMPLE_DEFER_TRANSPOSE 1u   /* csc_* arrays become valid only after e2egrec_sage_backward / e2egrec_sample_join */
+#define E2EGREC_SAMPLE_NO_TRANSPOSE 2u      /* csc_* arrays are not built; e2egrec_blocks_transpose builds them later */
 
 /* flags of e2egrec_sage_backward */
 #define E2EGREC_ACCUMULATE_DW 1u     /* add to dW / dbias instead of overwriting them */
@@ -186,7 +187,7 @@ int32_t e2egrec_sampler_set_step(void *scratch, uint32_t step_offset, void *stre
  *   blocks host array[n_hops] of structs holding device pointers; blocks[h-1] receives hop h
  *       including its transposed form.  F_h = D_h followed by the new nodes in ascending order.
  *   scratch device buffer initialised by e2egrec_sampler_scratch_init for the same n_nodes.
- *   flags 0 or E2EGREC_SAMPLE_DEFER_TRANSPOSE.
+ *   flags 0, E2EGREC_SAMPLE_DEFER_TRANSPOSE or E2EGREC_SAMPLE_NO_TRANSPOSE.
  * The transposed form of a hop is built on a helper stream of the library (one per device, created on
  * the first call) beside the sampling of the next hop.  By default the call joins that work back into
  * `stream` before it returns.  With E2EGREC_SAMPLE_DEFER_TRANSPOSE it does not: indptr / col / nbr_global /
@@ -202,6 +203,18 @@ int32_t e2egrec_sample_khop(const e2egrec_csr *graph, const int32_t *seeds, int3
 
 /* Makes `stream` wait for a block transposition that e2egrec_sample_khop deferred (no-op if there is none). */
 int32_t e2egrec_sample_join(void *stream);
+
+/* The transposed form (csc_ptr / csc_row / csc_eid / csc_col: the block's entries ordered by source, then by
+ * position; what the backward aggregation of Sec. 4.1's sampled sub-graph walks) of blocks that
+ * e2egrec_sample_khop filled with E2EGREC_SAMPLE_NO_TRANSPOSE.  A training loop can so build the transposed
+ * form of one batch beside the sampling of the next and the forward/backward of the previous one.
+ *   n_nodes, n_hops, blocks, scratch, scratch_bytes: as given to that e2egrec_sample_khop call; the scratch
+ *       must not have been used by another call in between (it still holds the entries' rows and the digit
+ *       counts of the columns).
+ * Independent blocks run partly on the library's helper stream; all work is joined into `stream` before the
+ * call returns.  Host errors: E2EGREC_ERR_NULL / _ARG / _ALIGN / _WORKSPACE, nothing is enqueued then. */
+int32_t e2egrec_blocks_transpose(int64_t n_nodes, int32_t n_hops, const e2egrec_block *blocks, void *scratch,
+                                 size_t scratch_bytes, void *stream);
 
 /* GraphSAGE forward over sampled blocks (Sec. 3.1): for layer l = 0..n_layers-1, on block
  * h = n_layers - l,

@@ -64,6 +64,8 @@ def lib():
         L.e2egrec_sampler_set_step.argtypes = [C.c_void_p, C.c_uint32, C.c_void_p]
         L.e2egrec_sample_join.restype = C.c_int32
         L.e2egrec_sample_join.argtypes = [C.c_void_p]
+        L.e2egrec_blocks_transpose.restype = C.c_int32
+        L.e2egrec_blocks_transpose.argtypes = [C.c_int64, C.c_int32, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p]
         L.e2egrec_sample_khop.restype = C.c_int32
         L.e2egrec_sample_khop.argtypes = [C.POINTER(Csr), C.c_void_p, C.c_int32, C.c_int32, C.c_void_p,
                                           C.c_uint64, C.c_uint32, C.c_uint32, C.POINTER(Block), C.c_void_p,
@@ -256,6 +258,7 @@ def sampler_set_step(scratch: torch.Tensor, step_offset: int, stream=None):
 
 
 DEFER_TRANSPOSE = 1
+NO_TRANSPOSE = 2
 
 
 def sample_join(stream=None):
@@ -273,18 +276,25 @@ def edge_cumulate(indptr: torch.Tensor, q: torch.Tensor, stream=None):
 
 
 def sample_khop(indptr: torch.Tensor, indices: torch.Tensor, seeds: torch.Tensor, blocks: Blocks, seed: int,
-                step: int, stream=None, defer_transpose=False, edge_cum=None):
+                step: int, stream=None, defer_transpose=False, edge_cum=None, transpose=True):
     """Enqueues the k-hop sample of `seeds` into `blocks` (see e2egrec_sample_khop); edge_cum (from edge_cumulate)
-    switches to the weighted draws."""
+    switches to the weighted draws; transpose=False leaves the transposed form to blocks_transpose."""
     assert indptr.dtype == torch.int64 and indices.dtype == torch.int32 and seeds.dtype == torch.int32
     assert edge_cum is None or (edge_cum.element_size() == 8 and edge_cum.numel() == indices.numel())
     g = Csr(indptr.numel() - 1, indices.numel(), indptr.data_ptr(), indices.data_ptr(),
             None if edge_cum is None else edge_cum.data_ptr())
     f = _i32_host(blocks.fanouts)
     _check(lib().e2egrec_sample_khop(C.byref(g), _ptr(seeds), seeds.numel(), len(blocks), f,
-                                     C.c_uint64(seed), C.c_uint32(step), DEFER_TRANSPOSE if defer_transpose else 0, blocks.c,
+                                     C.c_uint64(seed), C.c_uint32(step),
+                                     (DEFER_TRANSPOSE if defer_transpose else 0) | (0 if transpose else NO_TRANSPOSE), blocks.c,
                                      _ptr(blocks.scratch),
                                      blocks.scratch.numel(), _stream(stream)), "e2egrec_sample_khop")
+
+
+def blocks_transpose(blocks: Blocks, stream=None):
+    """Builds the transposed form of blocks sampled with transpose=False (see e2egrec_blocks_transpose)."""
+    _check(lib().e2egrec_blocks_transpose(C.c_int64(blocks.n_nodes), len(blocks), blocks.c, _ptr(blocks.scratch),
+                                          C.c_size_t(blocks.scratch.numel()), _stream(stream)), "e2egrec_blocks_transpose")
 
 
 # ------------------------------------------------------------------------------------------ GraphSAGE

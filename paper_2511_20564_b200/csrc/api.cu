@@ -46,7 +46,9 @@ SideStream *SideStream::get(cudaStream_t caller)
         SideStream *s = new SideStream();
         s->next = 0;
         s->owner = caller;
-        if (cudaStreamCreateWithFlags(&s->stream, cudaStreamNonBlocking) != cudaSuccess) { delete s; cudaGetLastError(); return nullptr; }
+        int prio = 0;                                // the helper runs at its caller's priority
+        if (cudaStreamGetPriority(caller, &prio) != cudaSuccess) { prio = 0; cudaGetLastError(); }
+        if (cudaStreamCreateWithPriority(&s->stream, cudaStreamNonBlocking, prio) != cudaSuccess) { delete s; cudaGetLastError(); return nullptr; }
         for (int i = 0; i < 32; ++i)
             if (cudaEventCreateWithFlags(&s->ev[i], cudaEventDisableTiming) != cudaSuccess) { delete s; cudaGetLastError(); return nullptr; }
         if (cudaEventCreateWithFlags(&s->pending, cudaEventDisableTiming) != cudaSuccess) { delete s; cudaGetLastError(); return nullptr; }

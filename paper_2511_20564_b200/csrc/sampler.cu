@@ -634,19 +634,21 @@ int32_t e2egrec::sample_khop_impl(const e2egrec_csr *graph, const int32_t *seeds
         note_launch();
         relabel_kernel<<<(unsigned)std::min<int64_t>(grid_for(b.cap_edges, T), 148 * 4), T, 0, st>>>(
             b.nbr_global, s.local_id, b.counts, b.col, sp.bits, sp.passes, l.ghist);
-        cudaStream_t ts = st;                        // stream of the transposition
-        if (side) {
-            side->fork(st);
-            ts = side->stream;
+        if (!(flags & E2EGREC_SAMPLE_NO_TRANSPOSE)) {
+            cudaStream_t ts = st;                    // stream of the transposition
+            if (side) {
+                side->fork(st);
+                ts = side->stream;
+            }
+            sort_by_col(b.col, b.counts, b.cap_edges, b.csc_col, b.csc_eid, sp, l, s.sort_tiles, ts);
+            note_launch();
+            csc_finalize_kernel<<<grid_for(std::max<int64_t>(b.cap_edges, (int64_t)b.cap_src + 1), T), T, 0, ts>>>(
+                b.csc_col, b.csc_eid, l.edge_row, b.counts, b.csc_ptr, b.csc_row);
         }
-        sort_by_col(b.col, b.counts, b.cap_edges, b.csc_col, b.csc_eid, sp, l, s.sort_tiles, ts);
-        note_launch();
-        csc_finalize_kernel<<<grid_for(std::max<int64_t>(b.cap_edges, (int64_t)b.cap_src + 1), T), T, 0, ts>>>(
-            b.csc_col, b.csc_eid, l.edge_row, b.counts, b.csc_ptr, b.csc_row);
         dst_nodes = b.src_nodes;
         n_dst_ptr = &b.counts[CNT_SRC];
     }
-    if (side) {
+    if (side && !(flags & E2EGREC_SAMPLE_NO_TRANSPOSE)) {
         if (flags & E2EGREC_SAMPLE_DEFER_TRANSPOSE) side->defer();
         else side->join(st);
     }
@@ -656,3 +658,45 @@ int32_t e2egrec::sample_khop_impl(const e2egrec_csr *graph, const int32_t *seeds
     tap_end(TAP_SAMPLE, st);
     return check_launch("sample_khop");
 }
+
+// The transposed form of blocks sampled with E2EGREC_SAMPLE_NO_TRANSPOSE: the sort of every block by source and
+// its offsets, from what the sampling left in the blocks and in the scratch (entry rows, digit counts of the
+// columns).  Blocks are independent, so every other one runs on the helper stream.
+extern "C" int32_t e2egrec_blocks_transpose(int64_t n_nodes, int32_t n_hops, const e2egrec_block *blocks, void *scratch,
+                                            size_t scratch_bytes, void *stream)
+{
+    using namespace e2egrec;
+    if (!blocks || !scratch) return E2EGREC_ERR_NULL;
+    if (n_hops < 1 || n_hops > kMaxHops || n_nodes < 1) return E2EGREC_ERR_ARG;
+    if (reinterpret_cast<uintptr_t>(scratch) % 256) return E2EGREC_ERR_ALIGN;
+    int64_t md = 0, ms = 0, me = 0;
+    for (int h = 0; h < n_hops; ++h) {
+        const e2egrec_block &b = blocks[h];
+        if (!b.counts || !b.col || !b.csc_ptr || !b.csc_row || !b.csc_eid || !b.csc_col) return E2EGREC_ERR_NULL;
+        if (b.cap_dst > md) md = b.cap_dst;
+        if (b.cap_src > ms) ms = b.cap_src;
+        if (b.cap_edges > me) me = b.cap_edges;
+    }
+    SamplerScratch s = carve(n_nodes, md, ms, me, scratch);
+    if (scratch_bytes < s.bytes) return E2EGREC_ERR_WORKSPACE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    SideStream *side = SideStream::get(st);
+    if (side) side->join_pending(st);
+    const int T = 256;
+    const bool forked = side && n_hops > 1;
+    if (forked) side->fork(st);
+    for (int h = n_hops - 1; h >= 0; --h) {          // the largest block first, on the caller's stream
+        const e2egrec_block &b = blocks[h];
+        const SortPlan sp = sort_plan(b.cap_src);
+        const SortLane &l = s.lane[h];
+        cudaStream_t ts = st;
+        if (forked && ((n_hops - 1 - h) & 1)) ts = side->stream;
+        sort_by_col(b.col, b.counts, b.cap_edges, b.csc_col, b.csc_eid, sp, l, s.sort_tiles, ts);
+        note_launch();
+        csc_finalize_kernel<<<grid_for(std::max<int64_t>(b.cap_edges, (int64_t)b.cap_src + 1), T), T, 0, ts>>>(
+            b.csc_col, b.csc_eid, l.edge_row, b.counts, b.csc_ptr, b.csc_row);
+    }
+    if (forked) side->join(st);
+    return check_launch("blocks_transpose");
+}
+

@@ -350,6 +350,69 @@ def test_sampling_of_the_next_batch_beside_the_current_step():
             assert torch.equal(a, b), f"step {i}"
 
 
+def test_three_stage_pipeline_sampling_transposition_compute():
+    """Three sets of block buffers and three streams, as bench.py runs the step: the hops of batch i + 2, the transposed
+    form of batch i + 1 (e2egrec_blocks_transpose) and the forward/backward of batch i side by side.  The blocks of
+    the split path equal the oracle's bit for bit; every step's outputs are bit-identical to steps run back to back."""
+    import paper_2511_20564_b200 as E
+    w = S.WORKLOADS["medium_small"]
+    case = Case(w, step=3)
+    ora = case.run_oracle(case.upstream_grad(case.seeds.size, w.hidden))
+    dev = torch.device("cuda")
+    indptr, indices = torch.from_numpy(case.indptr).to(dev), torch.from_numpy(case.indices).to(dev)
+    X = torch.from_numpy(case.X).to(dev, torch.bfloat16)
+    Ws = [torch.from_numpy(W).to(dev, torch.bfloat16) for W in case.Ws]
+    bufs = [E.Blocks(w.n_nodes, w.batch, w.fanouts, dev) for _ in range(3)]
+
+    # the split path alone, against the oracle
+    own = E.Blocks(w.n_nodes, case.seeds.size, w.fanouts, dev)
+    E.sample_khop(indptr, indices, torch.from_numpy(case.seeds).to(dev), own, w.seed, 3, transpose=False)
+    E.blocks_transpose(own)
+    torch.cuda.synchronize()
+    assert_blocks_equal(own.to_host(), ora["blocks"])
+
+    n_steps = 5
+    seeds = [torch.from_numpy(S.seed_batch(w.n_nodes, w.batch, w.seed, i)).to(dev) for i in range(n_steps + 2)]
+    dH = torch.from_numpy(S.to_bf16_values(np.random.default_rng(5).standard_normal((w.batch, w.hidden)).astype(np.float32)))
+    dH = dH.to(dev, torch.bfloat16)
+
+    def compute(b):
+        H, ctx = E.sage_forward(b, X, Ws)
+        g = torch.zeros(H.shape, dtype=torch.bfloat16, device=dev)
+        g[: w.batch] = dH
+        dWs, dX = E.sage_backward(b, X, Ws, ctx, g)
+        n_src, n_edges = int(b.counts[-1][1]), int(b.counts[-1][2])
+        return [H.clone()] + [t.clone() for t in dWs] + [dX[:n_src].clone(), b.counts.clone()] + \
+               [b.t[-1]["csc_row"][:n_edges].clone(), b.t[-1]["csc_ptr"][: n_src + 1].clone()]
+
+    want = []
+    for i in range(n_steps):
+        E.sample_khop(indptr, indices, seeds[i], bufs[0], w.seed, i)
+        want.append(compute(bufs[0]))
+    torch.cuda.synchronize()
+
+    s1, s2, s3 = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    got = []
+    with torch.cuda.stream(s1):
+        E.sample_khop(indptr, indices, seeds[0], bufs[0], w.seed, 0)
+        E.sample_khop(indptr, indices, seeds[1], bufs[1], w.seed, 1, transpose=False)
+        for i in range(n_steps):
+            s2.wait_stream(s1)
+            s3.wait_stream(s1)
+            with torch.cuda.stream(s2):
+                E.sample_khop(indptr, indices, seeds[i + 2], bufs[(i + 2) % 3], w.seed, i + 2, transpose=False)
+            with torch.cuda.stream(s3):
+                E.blocks_transpose(bufs[(i + 1) % 3])
+            got.append(compute(bufs[i % 3]))
+            s1.wait_stream(s2)
+            s1.wait_stream(s3)
+    torch.cuda.synchronize()
+    for i in range(n_steps):
+        assert int(got[i][-3][:, 3].sum()) == 0
+        for a, b in zip(got[i], want[i]):
+            assert torch.equal(a, b), f"step {i}"
+
+
 # ----------------------------------------------------------------------------- weighted sampling
 
 @pytest.mark.parametrize("beta", [0.0, 1.0, 2.5])
