@@ -172,12 +172,18 @@ sort_pass_kernel(const int32_t *__restrict__ keys_in, const int32_t *__restrict_
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t wbase = tile * kSortTile + (int64_t)warp * (32 * kSortItems);
     int32_t key[kSortItems], val[kSortItems], rank[kSortItems];
+    // all loads first: the warp barrier inside the ranking loop would otherwise keep every round's load behind it
 #pragma unroll
     for (int k = 0; k < kSortItems; ++k) {
         const int64_t idx = wbase + k * 32 + lane;
         const bool ok = idx < n;
         key[k] = ok ? keys_in[idx] : 0;
         val[k] = ok ? (vals_in ? vals_in[idx] : (int32_t)idx) : 0;
+    }
+#pragma unroll
+    for (int k = 0; k < kSortItems; ++k) {
+        const int64_t idx = wbase + k * 32 + lane;
+        const bool ok = idx < n;
         const uint32_t digit = ok ? (uint32_t)((key[k] >> shift) & (R - 1)) : 0xFFFFFFFFu;
         const uint32_t peers = __match_any_sync(0xffffffffu, digit);
         const int leader = __ffs(peers) - 1;

@@ -181,7 +181,8 @@ hop_sample_kernel(const int64_t *__restrict__ g_indptr, const int32_t *__restric
     }
     int32_t tile_total;
     const int32_t ex = block_exclusive_scan<kDstThreads, int32_t>(c, tile_total, scan_sm);
-    if (threadIdx.x <= kDstTile) off[threadIdx.x] = ex;          // off[kDstTile] = the tile's total
+    if (threadIdx.x < kDstTile) off[threadIdx.x] = ex;
+    if (threadIdx.x == 0) off[kDstTile] = tile_total;
     const long long base = chain_lookback(state, tile, tile_total, &counts[CNT_STATUS], &bcast);   // syncs the block
     if (threadIdx.x < kDstTile && i < n_dst) blk_indptr[i] = (int32_t)(base + ex);
     const bool last_tile = i0 + kDstTile >= n_dst;
