@@ -81,7 +81,7 @@ static void dispatch_sage_aggregate(const T *Hsrc, int64_t ld, const int32_t *nb
 
 // transposed-block entries per lane group: 32, or 128 where the block can hold millions of entries (the longer run's
 // lower overhead per entry wins there; measured on the 2 * 10^9-entry workload: 0.69 -> 0.63 ms)
-static inline int block_run_len(int64_t cap_edges) { return cap_edges >= (1ll << 21) ? 128 : 32; }
+static inline int block_run_len(int64_t cap_edges) { return cap_edges >= (1ll << 21) ? 128 : 16; }
 constexpr int kDwSplits = 148;        // split-K factor of the weight-gradient product
 
 // ------------------------------------------------------------------------------ forward
