@@ -633,7 +633,7 @@ def run_ours(args, w):
                          gbs=alg_bwd / tap_ms[2] / 1e6, frac_of_hbm=alg_bwd / tap_ms[2] / 1e6 / peaks["hbm_gbs"])}
     # DRAM bytes per launch from the ncu launch list of this command (profiles/medium_step_launch_list.md);
     # known only for the aggregation kernels of the outermost block of the `medium` workload
-    traffic = {1: 6.30e6, 2: 5.55e6 + 1.78e6}.get(dominant) if w.name == "medium" and args.seeds == "activity" else None
+    traffic = {1: 6.30e6, 2: 5.55e6 + 1.91e6}.get(dominant) if w.name == "medium" and args.seeds == "activity" else None
     roof.update(frac=roof["achieved"] / roof["peak"], traffic=traffic, kernel=TAP_NAMES[dominant],
                 ms_per_launch=dom_mean_ms, algorithmic_units_per_launch=alg, peak_source=peaks["source"])
 
