@@ -641,8 +641,10 @@ inline void launch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const
         if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         kern<<<grid1, kAggThreads, smem, st>>>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head2, sc.tail2,
                                                sc.win_info, sc.cap_runs, seg_of, o);
-    } else if (o.self && kSegRing > 0 && CPL == 1 && !kWeight && sizeof(PtrT) == 4 && LPR >= 16 && kInFlight == 4 && seg_of) {
-        // rows of 256 bytes and more on a sampled block: the ring form
+    } else if (o.self && run_len >= 128 && kSegRing > 0 && CPL == 1 && !kWeight && sizeof(PtrT) == 4 && LPR >= 16 && kInFlight == 4 &&
+               seg_of) {
+        // rows of 256 bytes and more on a sampled block that can hold millions of entries (long runs: the rows it gathers do
+        // not fit in L2): the ring form.  On smaller blocks, whose rows come from L2, registers in flight are faster.
         if constexpr (CPL == 1 && !kWeight && sizeof(PtrT) == 4 && LPR >= 16 && kInFlight == 4) {
             constexpr size_t smem_ring = smem + (size_t)2 * kSegRing * kAggThreads * 16;
             auto kern = seg_run_kernel<T, PtrT, LPR, CPL, kWeight, 1, kInFlight, kSegRing>;

@@ -151,7 +151,7 @@ class Case:
         g = np.random.default_rng(1234 + self.step).standard_normal((n_rows, d)).astype(np.float32)
         return S.to_bf16_values(g) if self.bf16 else g
 
-    def run_gpu(self, dH=None):
+    def run_gpu(self, dH=None, cap_seeds=None):
         import paper_2511_20564_b200 as E
         dev = "cuda"
         dt = torch_dtype(self.w.dtype)
@@ -160,7 +160,7 @@ class Case:
         X = torch.from_numpy(self.X).to(dev, dt)
         Ws = [torch.from_numpy(W).to(dev, dt) for W in self.Ws]
         seeds = torch.from_numpy(self.seeds).to(dev)
-        blocks = E.Blocks(self.w.n_nodes, self.seeds.size, self.w.fanouts, dev)
+        blocks = E.Blocks(self.w.n_nodes, cap_seeds or self.seeds.size, self.w.fanouts, dev)   # capacity may exceed the batch
         E.sample_khop(indptr, indices, seeds, blocks, self.w.seed, self.step)
         H, ctx = E.sage_forward(blocks, X, Ws, acts=self.acts)
         res = dict(blocks_obj=blocks, H=H, ctx=ctx)
