@@ -363,7 +363,9 @@ def run_ours(args, w):
     # ---- record the step as CUDA graphs (no host work between the kernels) and replay them.  Graph p holds the
     # forward/backward of the batch in buffer p and, on two more streams, the transposed form of the batch in buffer
     # p + 1 and the hops of the batch after that into buffer p + 2 (indices mod 3).
-    side, side2, side3 = torch.cuda.Stream(), torch.cuda.Stream(priority=-1), torch.cuda.Stream(priority=-1)
+    # The forward/backward leg decides the step time, so its stream (and the library's helper stream, which takes its
+    # caller's priority) runs at high priority: its kernels get SM slots before the short kernels of the other legs.
+    side, side2, side3 = torch.cuda.Stream(priority=-1), torch.cuda.Stream(), torch.cuda.Stream()
     for t in dH_in2:
         t.copy_(dH)
     with torch.cuda.stream(side):
@@ -747,8 +749,8 @@ def run_lightgcn(args, w):
         E.lightgcn_sampled_backward(blocks2[p], ctx, dY, dX_rows=dX, scratch=scratch)
         count_total.add_(blocks2[p].counts)
 
-    # the sampling leg runs at high priority: its short dependent kernels take the next free slots of an SM
-    # instead of queueing behind the thousands of blocks of a gather or a dense product
+    # here the sampling leg is the longer one and runs at high priority: its short dependent kernels take the next
+    # free slots of an SM instead of queueing behind the blocks of the propagation
     side, side2 = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
     with torch.cuda.stream(side):
         for i in range(max(Wm, 3)):
