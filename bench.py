@@ -728,11 +728,12 @@ def run_lightgcn(args, w):
         X_h = S.to_bf16_values(X_h)
     X = torch.from_numpy(X_h).to(dev, dt)
     K, Wm = args.steps, args.warmup
-    seeds_h = make_batches(w, (users, items), args.seeds, 0, K + Wm + 1)
+    seeds_h = make_batches(w, (users, items), args.seeds, 0, K + Wm + 3)
     seeds_dev = torch.from_numpy(seeds_h).to(dev)
     dY_h = upstream_grad(w, w.batch)[:, : w.dim] if w.hidden >= w.dim else np.zeros((w.batch, w.dim), np.float32)
-    blocks2 = [E.Blocks(w.n_nodes, w.batch, w.fanouts, dev) for _ in range(2)]
-    seeds_in2 = [torch.empty(w.batch, dtype=torch.int32, device=dev) for _ in range(2)]
+    NB = 3                                               # hops of batch i+2, transposed form of batch i+1, compute of batch i
+    blocks2 = [E.Blocks(w.n_nodes, w.batch, w.fanouts, dev) for _ in range(NB)]
+    seeds_in2 = [torch.empty(w.batch, dtype=torch.int32, device=dev) for _ in range(NB)]
     Y = torch.zeros(blocks2[0].caps[0][0], w.dim, dtype=dt, device=dev)
     dY = torch.zeros_like(Y)
     dY[: w.batch] = torch.from_numpy(dY_h).to(dev, dt)
@@ -741,50 +742,58 @@ def run_lightgcn(args, w):
     _, scratch = E.lightgcn_sampled_backward(blocks2[0], ctx, dY, dX_rows=dX)
     count_total = torch.zeros(len(w.fanouts), 4, dtype=torch.int64, device=dev)
 
-    def sample_leg(p):
-        E.sample_khop(indptr, indices, seeds_in2[p], blocks2[p], w.seed, 0)
+    def sample_leg(p, transpose=True):
+        E.sample_khop(indptr, indices, seeds_in2[p], blocks2[p], w.seed, 0, transpose=transpose)
 
     def compute_leg(p):
         E.lightgcn_sampled_forward(blocks2[p], X, s_d, ctx=ctx, Y=Y)
         E.lightgcn_sampled_backward(blocks2[p], ctx, dY, dX_rows=dX, scratch=scratch)
         count_total.add_(blocks2[p].counts)
 
-    # here the sampling leg is the longer one and runs at high priority: its short dependent kernels take the next
-    # free slots of an SM instead of queueing behind the blocks of the propagation
-    side, side2 = torch.cuda.Stream(), torch.cuda.Stream(priority=-1)
+    # the same three-stage pipeline as the GraphSAGE step; here the two sampling legs are the longer ones and run at
+    # high priority: their short dependent kernels take the next free slots of an SM
+    side, side2, side3 = torch.cuda.Stream(), torch.cuda.Stream(priority=-1), torch.cuda.Stream(priority=-1)
     with torch.cuda.stream(side):
         for i in range(max(Wm, 3)):
-            for p in range(2):
+            for p in range(NB):
                 seeds_in2[p].copy_(seeds_dev[i])
                 E.sampler_set_step(blocks2[p].scratch, i)
                 with torch.cuda.stream(side2):
                     side2.wait_stream(side)
-                    sample_leg(p)
-                side.wait_stream(side2)
+                    sample_leg(p, transpose=False)
+                with torch.cuda.stream(side3):
+                    side3.wait_stream(side2)
+                    E.blocks_transpose(blocks2[p])
+                side.wait_stream(side3)
                 compute_leg(p)
     side.synchronize()
     graphs = []
     l0 = E.launch_count()
-    for p in range(2):
+    for p in range(NB):
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g, stream=side):
             side2.wait_stream(side)
+            side3.wait_stream(side)
             with torch.cuda.stream(side2):
-                sample_leg(1 - p)
+                sample_leg((p + 2) % NB, transpose=False)
+            with torch.cuda.stream(side3):
+                E.blocks_transpose(blocks2[(p + 1) % NB])
             compute_leg(p)
             side.wait_stream(side2)
+            side.wait_stream(side3)
         graphs.append(g)
-    kernels_per_step = (E.launch_count() - l0) // 2 + 1
+    kernels_per_step = (E.launch_count() - l0) // NB + 1
 
     def prime(i):
-        seeds_in2[i & 1].copy_(seeds_dev[i], non_blocking=True)
-        E.sampler_set_step(blocks2[i & 1].scratch, i)
-        sample_leg(i & 1)
+        for k, tr in ((i, True), (i + 1, False)):
+            seeds_in2[k % NB].copy_(seeds_dev[k], non_blocking=True)
+            E.sampler_set_step(blocks2[k % NB].scratch, k)
+            sample_leg(k % NB, transpose=tr)
 
     def replay_step(i):
-        seeds_in2[(i + 1) & 1].copy_(seeds_dev[i + 1], non_blocking=True)
-        E.sampler_set_step(blocks2[(i + 1) & 1].scratch, i + 1)
-        graphs[i & 1].replay()
+        seeds_in2[(i + 2) % NB].copy_(seeds_dev[i + 2], non_blocking=True)
+        E.sampler_set_step(blocks2[(i + 2) % NB].scratch, i + 2)
+        graphs[i % NB].replay()
 
     prime(Wm)
     count_total.zero_()
@@ -810,8 +819,8 @@ def run_lightgcn(args, w):
                 data="synthetic",
                 config=dict(workload=w.name, backbone="lightgcn", nodes=w.n_nodes, csr_entries=int(indices.numel()), dim=w.dim,
                             layers=len(w.fanouts), fanouts=list(w.fanouts), batch=w.batch, seeds=args.seeds,
-                            launch="one CUDA graph replay per step: propagation and adjoint of the batch beside the sampling "
-                                   "of the next batch", edges_per_step=edges / K),
+                            launch="one CUDA graph replay per step, three streams: propagation and adjoint of batch i beside "
+                                   "the transposed form of batch i+1 and the hops of batch i+2", edges_per_step=edges / K),
                 clocks=clk, gpu_launches=int(K * (kernels_per_step + 2)))
     if not args.no_cpu_baseline:
         import oracle
