@@ -68,3 +68,11 @@ def test_host_side_argument_checks_of_the_newer_entry_points_need_no_gpu():
     # the frontier of a hop must fit the destinations of the next one
     blocks[1] = B.Block(100, 4224, 3520, *([None] * 10))
     assert L.e2egrec_lightgcn_sampled_forward(blocks, 2, C.byref(x), None, None, C.byref(n), None, None) == ERR_ARG
+    # the transposed form as a call of its own
+    blocks[1] = B.Block(704, 4224, 3520, *([None] * 10))
+    assert L.e2egrec_blocks_transpose(5000, 2, None, C.c_void_p(256), 1 << 20, None) == ERR_NULL
+    assert L.e2egrec_blocks_transpose(5000, 2, blocks, None, 1 << 20, None) == ERR_NULL
+    assert L.e2egrec_blocks_transpose(5000, 0, blocks, C.c_void_p(256), 1 << 20, None) == ERR_ARG
+    assert L.e2egrec_blocks_transpose(0, 2, blocks, C.c_void_p(256), 1 << 20, None) == ERR_ARG
+    assert L.e2egrec_blocks_transpose(5000, 2, blocks, C.c_void_p(264), 1 << 20, None) == -4         # scratch not 256-byte aligned
+    assert L.e2egrec_blocks_transpose(5000, 2, blocks, C.c_void_p(256), 1 << 20, None) == ERR_NULL    # blocks without arrays
