@@ -188,20 +188,23 @@ int32_t e2egrec_sampler_set_step(void *scratch, uint32_t step_offset, void *stre
  *       including its transposed form.  F_h = D_h followed by the new nodes in ascending order.
  *   scratch device buffer initialised by e2egrec_sampler_scratch_init for the same n_nodes.
  *   flags 0, E2EGREC_SAMPLE_DEFER_TRANSPOSE or E2EGREC_SAMPLE_NO_TRANSPOSE.
- * The transposed form of a hop is built on a helper stream of the library (one per device, created on
- * the first call) beside the sampling of the next hop.  By default the call joins that work back into
- * `stream` before it returns.  With E2EGREC_SAMPLE_DEFER_TRANSPOSE it does not: indptr / col / nbr_global /
- * src_nodes / inv_cnt / counts are valid in stream order as always, but the csc_* arrays are only complete
- * after the next e2egrec_sage_backward or e2egrec_sample_join issued from the same device on this or any
- * later-ordered stream (e2egrec_sage_forward does not need them, so the forward pass overlaps the
- * transposition).  The next e2egrec_sample_khop joins by itself.  Do not interleave deferred calls from
- * several host threads on one device. */
+ * The transposed form of a hop is built on a helper stream of the library (one per device and caller stream,
+ * created on the first call, at the caller stream's priority, kept until the process ends) beside the sampling of
+ * the next hop.  By default the call joins that work back into `stream` before it returns.  With
+ * E2EGREC_SAMPLE_DEFER_TRANSPOSE it does not: indptr / col / nbr_global / src_nodes / inv_cnt / counts are valid in
+ * stream order as always, but the csc_* arrays are only complete after the next e2egrec_sage_backward,
+ * e2egrec_lightgcn_sampled_backward, e2egrec_sample_khop or e2egrec_sample_join that the host issues on any stream
+ * of the same device: that call makes its stream wait for every transposition deferred on the device so far
+ * (e2egrec_sage_forward does not need the csc_* arrays, so the forward pass overlaps the transposition).  Inside a
+ * stream capture the deferring call and the joining call must belong to the same capture.  Calls that share a
+ * caller stream must not be issued from two host threads at once. */
 int32_t e2egrec_sample_khop(const e2egrec_csr *graph, const int32_t *seeds, int32_t n_seeds,
                             int32_t n_hops, const int32_t *fanouts, uint64_t seed, uint32_t step,
                             uint32_t flags, const e2egrec_block *blocks,
                             void *scratch, size_t scratch_bytes, void *stream);
 
-/* Makes `stream` wait for a block transposition that e2egrec_sample_khop deferred (no-op if there is none). */
+/* Makes `stream` wait for every block transposition that e2egrec_sample_khop calls have deferred on the current device
+ * (on whichever stream; no-op if there is none). */
 int32_t e2egrec_sample_join(void *stream);
 
 /* The transposed form (csc_ptr / csc_row / csc_eid / csc_col: the block's entries ordered by source, then by
@@ -362,7 +365,8 @@ int32_t e2egrec_lightgcn_sampled_backward(const e2egrec_block *blocks, int32_t n
                                           const e2egrec_mat *dY, const e2egrec_mat *dX_rows, void *scratch,
                                           size_t *scratch_bytes, void *stream);
 
-/* The self-supervised task of the GNN and the balancing of the two losses (Sec. 4.2).
+/* The self-supervised task of the GNN and the balancing of the two losses (the SSL task: Sec. 4.2; the
+ * gradient-based task weighting: Sec. 4.3.1).
  * e2egrec_ssl_loss: graph feature auto-encoder with the identity decoder, L_ssl = || X_seeds - H ||_F^2 over the rows
  *   i < *n_rows_dev (NULL: all H->rows rows) with X_seeds[i] = X[seed_ids[i]]; loss: device float[1] (unweighted);
  *   dH [>= H->rows x dim] receives the gradient of weight[0] * L_ssl with respect to H, 2 weight (H - X), in H's
@@ -384,7 +388,7 @@ int32_t e2egrec_gradient_norm(const e2egrec_mat *A, const int32_t *n_rows_dev, f
 int32_t e2egrec_gradnorm_update(float *w, const float *L, const float *L0, const float *g, int32_t n_tasks, float gamma,
                                 float lr, float *L_gn, void *stream);
 
-/* Feature fusion by concatenation with gating (Sec. 4.3.1):  g = sigmoid(F Wg^T + bg),  F_fused = g * F, for the
+/* Feature fusion by concatenation with gating (Sec. 4.3.2):  g = sigmoid(F Wg^T + bg),  F_fused = g * F, for the
  * n_rows rows of F [rows x d] (the concatenated feature groups, GNN output among them); Wg [d x d] row-major in F's
  * dtype, bg device float[d] or NULL.  gate and fused: [>= n_rows x d] outputs (the gate is kept for the backward call).
  * e2egrec_gate_fusion_backward: dF = dFused * g + (dFused * F * g (1 - g)) Wg, dWg = (dFused * F * g (1 - g))^T F
@@ -400,7 +404,8 @@ int32_t e2egrec_gate_fusion_backward(const e2egrec_mat *dFused, const e2egrec_ma
                                      float *dbg, void *ws, size_t *ws_bytes, void *stream);
 
 /* e2egrec_aggregate_forward without a workspace argument (the paper has no counterpart; this is a
- * packaging variant of the call above and computes exactly the same result).
+ * packaging variant of the call above: it enqueues the same kernels with the same launch shapes, so its
+ * output equals that call's bit for bit).
  *
  * Who needs it: code that is not allowed to obtain device memory at the point where it aggregates --
  * a plug-in running inside a host application that owns the whole memory pool, a step executed while
@@ -410,10 +415,11 @@ int32_t e2egrec_gate_fusion_backward(const e2egrec_mat *dFused, const e2egrec_ma
  *
  * Here the partial-sum scratch is an 8 MiB array built into the library (every GPU that loads the
  * library holds it until the process ends; e2egrec_aggregate_forward_static_limit() returns the size).
- * The call allocates and frees nothing.  A problem fits if
- *     2 * round_up_256( ceil(n_entries / 128) * dim * 4 bytes ) <= 8 MiB,
- * e.g. up to about 2.1 M entries at dim 64.  Larger inputs are rejected with E2EGREC_ERR_WORKSPACE and
- * e2egrec_last_error() then says how many bytes were needed; nothing is enqueued in that case.
+ * The call allocates and frees nothing.  A problem fits if the scratch size that
+ * e2egrec_aggregate_forward's size query reports for the same n_entries, dim and dtype is at most
+ * 8 MiB: e.g. about 260 thousand entries of 1024 fp32 values, or about 130 million entries of 64 bf16 values.
+ * Larger inputs are rejected with E2EGREC_ERR_WORKSPACE and e2egrec_last_error() then says how many
+ * bytes were needed; nothing is enqueued in that case.
  *
  * The first call on each device looks up the device address of the built-in array (with that device
  * current).  Make that first call outside any stream capture.  All calls on a device share the one

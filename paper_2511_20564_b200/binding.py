@@ -384,6 +384,15 @@ def sage_backward(blocks: Blocks, X, Ws, ctx, dH_out, acts=None, dWs=None, dbs=N
 
 # ------------------------------------------------------------------------------------------ whole graph
 
+def aggregate_ws_bytes(n_entries, X) -> int:
+    """Scratch bytes e2egrec_aggregate_forward asks for with n_entries entries and rows like X's (size query only)."""
+    x = _mat(X)
+    n = C.c_size_t(0)
+    _check(lib().e2egrec_aggregate_forward(1, int(n_entries), None, None, C.byref(x), C.byref(x), 0, None, C.byref(n), None),
+           "e2egrec_aggregate_forward(size query)")
+    return n.value
+
+
 def aggregate_forward(indptr, indices, X, out=None, ws=None, sum_only=False, stream=None):
     """Enqueues out[i] = mean (or sum) of X[indices[row i]]; returns (out, ws)."""
     n_dst, n_entries = indptr.numel() - 1, indices.numel()

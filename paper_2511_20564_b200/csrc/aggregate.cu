@@ -3,6 +3,7 @@
 // shared by many warps.
 #include <algorithm>
 
+#include "internal.cuh"
 #include "segreduce.cuh"
 
 namespace e2egrec {
@@ -14,22 +15,28 @@ static inline int full_run_len(int64_t n_entries)
     return n_entries >= (1ll << 24) ? 256 : n_entries >= (1ll << 22) ? 128 : n_entries >= (1ll << 20) ? 64 : 32;
 }
 
-static size_t full_ws_bytes(int64_t n_entries, int d, int32_t dtype)
+size_t full_ws_bytes(int64_t n_entries, int d, int32_t dtype)
 {
     return seg_scratch_carve(n_entries, full_run_len(n_entries), d, dtype_size(dtype), nullptr).bytes;
 }
 
 template <typename T, bool kWeight>
-static void dispatch_seg64(const T *in, int64_t ld_in, const int64_t *ptr, const int32_t *idx, int64_t n_seg,
+static bool dispatch_seg64(const T *in, int64_t ld_in, const int64_t *ptr, const int32_t *idx, int64_t n_seg,
                            int64_t n_entries, const float *w, int d, void *ws, const SegOut<T> &o, int32_t dtype,
                            cudaStream_t st)
 {
     const int run_len = full_run_len(n_entries);
     const SegScratch sc = seg_scratch_carve(n_entries, run_len, d, dtype_size(dtype), ws);
-    dispatch_seg_reduce<T, int64_t, kWeight, 2>(in, ld_in, ptr, idx, nullptr, n_seg, n_seg, w, run_len, d, dtype, nullptr, sc, o, st);
+    return dispatch_seg_reduce<T, int64_t, kWeight, 2>(in, ld_in, ptr, idx, nullptr, n_seg, n_seg, w, run_len, d, dtype, nullptr, sc, o, st);
 }
 
-static int32_t check_mats(const e2egrec_mat *in, const e2egrec_mat *out, int64_t out_rows)
+static int32_t unsupported_width(const char *what)
+{
+    set_last_error(what);
+    return E2EGREC_ERR_UNSUPPORTED;
+}
+
+int32_t check_mats(const e2egrec_mat *in, const e2egrec_mat *out, int64_t out_rows)
 {
     if (!in || !out || !in->data || !out->data) return E2EGREC_ERR_NULL;
     if (in->dtype != E2EGREC_F32 && in->dtype != E2EGREC_BF16) return E2EGREC_ERR_DTYPE;
@@ -43,31 +50,33 @@ static int32_t check_mats(const e2egrec_mat *in, const e2egrec_mat *out, int64_t
     return E2EGREC_OK;
 }
 
-// Shared body of the two entry points.
-static int32_t full_aggregate(int64_t n_seg, int64_t n_entries, const int64_t *ptr, const int32_t *idx, const float *w,
+// Shared body of the entry points (e2egrec_aggregate_forward_static calls it with the library's built-in scratch).
+int32_t full_aggregate(int64_t n_seg, int64_t n_entries, const int64_t *ptr, const int32_t *idx, const float *w,
                        const e2egrec_mat *in, const e2egrec_mat *out, int mean, void *ws, cudaStream_t st)
 {
+    bool ok;
     if (in->dtype == E2EGREC_BF16) {
         using T = __nv_bfloat16;
         SegOut<T> o{};
         o.out = static_cast<T *>(out->data);
         o.ld_out = out->ld;
         o.mean = mean;
-        if (w) dispatch_seg64<T, true>(static_cast<const T *>(in->data), in->ld, ptr, idx, n_seg, n_entries, w, in->dim,
-                                       ws, o, in->dtype, st);
-        else dispatch_seg64<T, false>(static_cast<const T *>(in->data), in->ld, ptr, idx, n_seg, n_entries, w, in->dim,
-                                      ws, o, in->dtype, st);
+        ok = w ? dispatch_seg64<T, true>(static_cast<const T *>(in->data), in->ld, ptr, idx, n_seg, n_entries, w, in->dim, ws, o,
+                                         in->dtype, st)
+               : dispatch_seg64<T, false>(static_cast<const T *>(in->data), in->ld, ptr, idx, n_seg, n_entries, w, in->dim, ws, o,
+                                          in->dtype, st);
     } else {
         using T = float;
         SegOut<T> o{};
         o.out = static_cast<T *>(out->data);
         o.ld_out = out->ld;
         o.mean = mean;
-        if (w) dispatch_seg64<T, true>(static_cast<const T *>(in->data), in->ld, ptr, idx, n_seg, n_entries, w, in->dim,
-                                       ws, o, in->dtype, st);
-        else dispatch_seg64<T, false>(static_cast<const T *>(in->data), in->ld, ptr, idx, n_seg, n_entries, w, in->dim,
-                                      ws, o, in->dtype, st);
+        ok = w ? dispatch_seg64<T, true>(static_cast<const T *>(in->data), in->ld, ptr, idx, n_seg, n_entries, w, in->dim, ws, o,
+                                         in->dtype, st)
+               : dispatch_seg64<T, false>(static_cast<const T *>(in->data), in->ld, ptr, idx, n_seg, n_entries, w, in->dim, ws, o,
+                                          in->dtype, st);
     }
+    if (!ok) return unsupported_width("aggregate: no kernel for this row width");
     return check_launch("aggregate");
 }
 
@@ -129,21 +138,23 @@ __global__ void layer_mean_kernel(LayerList list, int n_in, int64_t cells, float
 static int32_t lightgcn_propagate(int64_t n, int64_t m, const int64_t *ptr, const int32_t *idx, const float *s,
                                   const e2egrec_mat *in, void *out_data, void *ws, cudaStream_t st)
 {
+    bool ok;
     if (in->dtype == E2EGREC_BF16) {
         using T = __nv_bfloat16;
         SegOut<T> o{};
         o.out = static_cast<T *>(out_data);
         o.ld_out = in->dim;
         o.seg_scale = s;
-        dispatch_seg64<T, true>(static_cast<const T *>(in->data), in->ld, ptr, idx, n, m, s, in->dim, ws, o, in->dtype, st);
+        ok = dispatch_seg64<T, true>(static_cast<const T *>(in->data), in->ld, ptr, idx, n, m, s, in->dim, ws, o, in->dtype, st);
     } else {
         using T = float;
         SegOut<T> o{};
         o.out = static_cast<T *>(out_data);
         o.ld_out = in->dim;
         o.seg_scale = s;
-        dispatch_seg64<T, true>(static_cast<const T *>(in->data), in->ld, ptr, idx, n, m, s, in->dim, ws, o, in->dtype, st);
+        ok = dispatch_seg64<T, true>(static_cast<const T *>(in->data), in->ld, ptr, idx, n, m, s, in->dim, ws, o, in->dtype, st);
     }
+    if (!ok) return unsupported_width("lightgcn: no kernel for this row width");
     return check_launch("lightgcn_propagate");
 }
 

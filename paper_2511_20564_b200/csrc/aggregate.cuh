@@ -1,6 +1,6 @@
-// Row-gather reductions: the neighbourhood mean (Eq. 2) over a sampled block, and the
-// general "segment s = sum of gathered rows" kernel used by the transposed aggregation
-// (gather over the block's CSC) and by whole-graph aggregation with hub rows.
+// Row-gather reductions: the neighbourhood mean (Eq. 2) over a sampled block, and the types
+// shared with the general "segment s = sum of gathered rows" kernels (segreduce.cuh) used by the
+// transposed aggregation (gather over the block's CSC) and by whole-graph aggregation with hub rows.
 //
 // A row of d values is d*sizeof(T)/16 chunks of 16 bytes.  LPR lanes (a power of two) own
 // one row at a time, lane c of the group holding chunks c, c+LPR, ... (CPL of them), so a
@@ -132,13 +132,7 @@ sage_aggregate_kernel(const T *__restrict__ Hsrc, int64_t ld, const int32_t *__r
 
 // ---------------------------------------------------------------------------------------
 // General segment reduction   out[s] = fin( sum_{k in [ptr[s], ptr[s+1])} w[idx[k]] * in[idx[k]] )
-// with  fin(x) = mask_s * ( x * (mean ? 1/len : 1) + self[s] ).
-//
-// Work is cut into chunks of `chunk_len` consecutive entries, one warp each, so a hub
-// segment with millions of entries is shared by many warps.  A segment that lies inside
-// one chunk is finished there.  Otherwise the chunk in which it starts stores its part in
-// tail[chunk], every later chunk stores its part in head[chunk], and the finishing kernel
-// adds tail[first] + head[first+1] + ... + head[last] in that fixed order.
+// with  fin(x) = mask_s * ( x * (mean ? 1/len : 1) + self[s] ); the kernels are in segreduce.cuh.
 // ---------------------------------------------------------------------------------------
 template <typename T>
 struct SegOut {
@@ -174,174 +168,6 @@ __device__ inline int64_t seg_containing(const PtrT *__restrict__ ptr, int64_t n
         if ((int64_t)ptr[mid] <= k) lo = mid; else hi = mid;
     }
     return lo;
-}
-
-template <typename T, typename PtrT, int LPR, int CPL, bool kWeight>
-__global__ void __launch_bounds__(kAggThreads)
-seg_chunk_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__ ptr,
-                 const int32_t *__restrict__ idx, const int32_t *n_seg_dev, int64_t n_seg_host,
-                 const float *__restrict__ w, int chunk_len, int d, float *__restrict__ head,
-                 float *__restrict__ tail, SegOut<T> o)
-{
-    constexpr int E = Chunk<T>::kElems;
-    constexpr int G = 32 / LPR;
-    constexpr int U = CPL >= 4 ? 1 : 4 / CPL;
-    const int lane = threadIdx.x & 31;
-    const int g = lane / LPR, c = lane % LPR;
-    const int n_chunks = d / E;
-    const int64_t n_seg = n_seg_dev ? (int64_t)*n_seg_dev : n_seg_host;
-    if (n_seg <= 0) return;
-    const int64_t total = (int64_t)ptr[n_seg];
-    const int64_t chunk = ((int64_t)blockIdx.x * kAggThreads + threadIdx.x) >> 5;
-    const int64_t k0 = chunk * chunk_len;
-    if (k0 >= total) return;
-    const int64_t k1 = min(k0 + (int64_t)chunk_len, total);
-    const int64_t n_self = o.self ? (o.n_self ? (int64_t)*o.n_self : n_seg) : 0;
-
-    int64_t s = seg_containing(ptr, n_seg, k0);
-    int64_t k = k0;
-    while (k < k1) {
-        int64_t seg_beg = (int64_t)ptr[s], seg_end = (int64_t)ptr[s + 1];
-        while (seg_end <= k) { ++s; seg_beg = seg_end; seg_end = (int64_t)ptr[s + 1]; }   // empty segments
-        const int64_t e1 = min(seg_end, k1);
-
-        float acc[CPL][E];
-#pragma unroll
-        for (int q = 0; q < CPL; ++q)
-#pragma unroll
-            for (int kk = 0; kk < E; ++kk) acc[q][kk] = 0.f;
-        for (int64_t base = k; base < e1; base += 32) {
-            const int m = (int)min((int64_t)32, e1 - base);
-            const int32_t mine = lane < m ? idx[base + lane] : 0;
-            float wmine = 1.f;
-            if (kWeight) wmine = lane < m ? w[mine] : 0.f;
-            for (int t = 0; t * G < m; t += U) {
-                float v[U][CPL][E];
-                float wt[U];
-                bool ok[U];
-#pragma unroll
-                for (int u = 0; u < U; ++u) {
-                    const int j = (t + u) * G + g;
-                    ok[u] = j < m;
-                    const int32_t id = __shfl_sync(0xffffffffu, mine, j & 31);
-                    wt[u] = kWeight ? __shfl_sync(0xffffffffu, wmine, j & 31) : 1.f;
-                    const T *row = in + (int64_t)id * ld_in;
-#pragma unroll
-                    for (int q = 0; q < CPL; ++q) {
-                        const int ch = c + q * LPR;
-                        if (ok[u] && ch < n_chunks) Chunk<T>::load(row + ch * E, v[u][q]);
-                    }
-                }
-#pragma unroll
-                for (int u = 0; u < U; ++u)
-#pragma unroll
-                    for (int q = 0; q < CPL; ++q)
-                        if (ok[u] && c + q * LPR < n_chunks)
-#pragma unroll
-                            for (int kk = 0; kk < E; ++kk) {
-                                if (kWeight) acc[q][kk] = fmaf(wt[u], v[u][q][kk], acc[q][kk]);
-                                else acc[q][kk] += v[u][q][kk];
-                            }
-            }
-        }
-#pragma unroll
-        for (int off = LPR; off < 32; off <<= 1)
-#pragma unroll
-            for (int q = 0; q < CPL; ++q)
-#pragma unroll
-                for (int kk = 0; kk < E; ++kk) acc[q][kk] += __shfl_xor_sync(0xffffffffu, acc[q][kk], off);
-
-        const bool begins = seg_beg >= k0;
-        const bool ends = seg_end <= k1;
-        if (g == 0) {
-#pragma unroll
-            for (int q = 0; q < CPL; ++q) {
-                const int ch = c + q * LPR;
-                if (ch >= n_chunks) continue;
-                if (begins && ends) {
-                    float r[E];
-#pragma unroll
-                    for (int kk = 0; kk < E; ++kk)
-                        r[kk] = seg_finish_value(o, s, seg_end - seg_beg, ch * E + kk, acc[q][kk], s < n_self);
-                    Chunk<T>::store(o.out + s * o.ld_out + ch * E, r);
-                } else {
-                    float *dst = (begins ? tail : head) + chunk * d + ch * E;
-#pragma unroll
-                    for (int kk = 0; kk < E; kk += 4)
-                        *reinterpret_cast<float4 *>(dst + kk) =
-                            make_float4(acc[q][kk], acc[q][kk + 1], acc[q][kk + 2], acc[q][kk + 3]);
-                }
-            }
-        }
-        k = e1;
-        ++s;
-    }
-}
-
-// Finishing kernel.  Blocks [0, n_chunk_blocks): block b looks at chunk b; if the segment that
-// holds the chunk's first entry started in an earlier chunk and ends in this one, the block adds
-// its partial rows in order and writes the result.  Blocks beyond that: one thread group per
-// segment, writing fin(0) for segments without entries.
-template <typename T, typename PtrT>
-__global__ void __launch_bounds__(kAggThreads)
-seg_finish_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_t n_seg_host, int chunk_len, int d,
-                  const float *__restrict__ head, const float *__restrict__ tail, int64_t n_chunk_blocks,
-                  SegOut<T> o)
-{
-    constexpr int W = kAggThreads / 32;
-    __shared__ float4 red[W][32];
-    const int64_t n_seg = n_seg_dev ? (int64_t)*n_seg_dev : n_seg_host;
-    if (n_seg <= 0) return;
-    const int64_t total = (int64_t)ptr[n_seg];
-    const int64_t n_self = o.self ? (o.n_self ? (int64_t)*o.n_self : n_seg) : 0;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-
-    if ((int64_t)blockIdx.x >= n_chunk_blocks) {
-        // segments without entries: 8 lanes per segment
-        const int64_t s = ((int64_t)(blockIdx.x - n_chunk_blocks) * kAggThreads + threadIdx.x) >> 3;
-        if (s >= n_seg || ptr[s + 1] != ptr[s]) return;
-        for (int k = threadIdx.x & 7; k < d; k += 8)
-            o.out[s * o.ld_out + k] = from_float<T>(seg_finish_value(o, s, 0, k, 0.f, s < n_self));
-        return;
-    }
-
-    const int64_t chunk = blockIdx.x;
-    const int64_t k0 = chunk * chunk_len;
-    if (chunk == 0 || k0 >= total) return;
-    const int64_t k1 = min(k0 + (int64_t)chunk_len, total);
-    const int64_t s = seg_containing(ptr, n_seg, k0);
-    const int64_t seg_beg = (int64_t)ptr[s], seg_end = (int64_t)ptr[s + 1];
-    if (seg_beg >= k0 || seg_end > k1) return;          // not split, or finished by a later chunk
-    const int64_t first = seg_beg / chunk_len;          // its part there is tail[first]
-    const int64_t n_parts = chunk - first + 1;
-    const int n_vec = d / 4;
-    for (int vb = 0; vb < n_vec; vb += 32) {
-        const int q = vb + lane;
-        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (q < n_vec) {
-            for (int64_t p = warp; p < n_parts; p += W) {
-                const float *src = (p == 0 ? tail + first * d : head + (first + p) * d) + q * 4;
-                const float4 x = *reinterpret_cast<const float4 *>(src);
-                a.x += x.x; a.y += x.y; a.z += x.z; a.w += x.w;
-            }
-        }
-        red[warp][lane] = a;
-        __syncthreads();
-        if (warp == 0 && q < n_vec) {
-            float4 t = red[0][lane];
-#pragma unroll
-            for (int w2 = 1; w2 < W; ++w2) {
-                const float4 x = red[w2][lane];
-                t.x += x.x; t.y += x.y; t.z += x.z; t.w += x.w;
-            }
-            const float r[4] = {t.x, t.y, t.z, t.w};
-#pragma unroll
-            for (int kk = 0; kk < 4; ++kk)
-                o.out[s * o.ld_out + q * 4 + kk] =
-                    from_float<T>(seg_finish_value(o, s, seg_end - seg_beg, q * 4 + kk, r[kk], s < n_self));
-        }
-        __syncthreads();
-    }
 }
 
 // Host side --------------------------------------------------------------------------------

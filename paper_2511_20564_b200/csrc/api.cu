@@ -1,6 +1,9 @@
 // Status strings and error bookkeeping of the C ABI.
 #include <atomic>
+#include <functional>
 #include <mutex>
+#include <unordered_map>
+#include <vector>
 #include <stdio.h>
 #include <string.h>
 
@@ -26,36 +29,44 @@ int32_t check_launch(const char *what)
     return E2EGREC_ERR_CUDA;
 }
 
+// Helper streams: one per (device, caller's stream), created on first use and kept until the process ends, so calls
+// made on different streams (a sampling leg beside a compute leg, say) never meet on a common helper stream.
+// Deferred work (a block transposition left running by e2egrec_sample_khop) is tracked per device: whichever stream
+// of that device asks next (e2egrec_sage_backward, e2egrec_sample_join, the next e2egrec_sample_khop) waits for all of
+// it.  The table and the pending lists are guarded by one mutex; the event ring of a helper stream is touched only by
+// calls issued on its caller's stream, which the caller must not issue from two host threads at once.
 static std::mutex g_side_mutex;
-constexpr int kSideSlots = 8;
-static SideStream *g_side[64][kSideSlots] = {};
+struct SideKey {
+    int dev;
+    cudaStream_t stream;
+    bool operator==(const SideKey &o) const { return dev == o.dev && stream == o.stream; }
+};
+struct SideKeyHash {
+    size_t operator()(const SideKey &k) const { return std::hash<const void *>()(k.stream) * 31u + (size_t)k.dev; }
+};
+static std::unordered_map<SideKey, SideStream *, SideKeyHash> g_side;
+static std::vector<SideStream *> g_pending[64];          // per device: helper streams whose `pending` event is unjoined
 
-// One helper stream per (device, caller's stream): calls made on different streams (a sampling leg beside a
-// compute leg, say) do not meet on a common helper stream.  With more than kSideSlots caller streams on a
-// device the last slot is shared.
 SideStream *SideStream::get(cudaStream_t caller)
 {
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
     std::lock_guard<std::mutex> lock(g_side_mutex);
-    int slot = 0;
-    for (; slot < kSideSlots; ++slot)
-        if (!g_side[dev][slot] || g_side[dev][slot]->owner == caller) break;
-    if (slot == kSideSlots) slot = kSideSlots - 1;
-    if (!g_side[dev][slot]) {
-        SideStream *s = new SideStream();
-        s->next = 0;
-        s->owner = caller;
-        int prio = 0;                                // the helper runs at its caller's priority
-        if (cudaStreamGetPriority(caller, &prio) != cudaSuccess) { prio = 0; cudaGetLastError(); }
-        if (cudaStreamCreateWithPriority(&s->stream, cudaStreamNonBlocking, prio) != cudaSuccess) { delete s; cudaGetLastError(); return nullptr; }
-        for (int i = 0; i < 32; ++i)
-            if (cudaEventCreateWithFlags(&s->ev[i], cudaEventDisableTiming) != cudaSuccess) { delete s; cudaGetLastError(); return nullptr; }
-        if (cudaEventCreateWithFlags(&s->pending, cudaEventDisableTiming) != cudaSuccess) { delete s; cudaGetLastError(); return nullptr; }
-        s->has_pending = false;
-        g_side[dev][slot] = s;
-    }
-    return g_side[dev][slot];
+    auto it = g_side.find(SideKey{dev, caller});
+    if (it != g_side.end()) return it->second;
+    SideStream *s = new SideStream();
+    s->next = 0;
+    s->owner = caller;
+    s->device = dev;
+    int prio = 0;                                // the helper runs at its caller's priority
+    if (cudaStreamGetPriority(caller, &prio) != cudaSuccess) { prio = 0; cudaGetLastError(); }
+    if (cudaStreamCreateWithPriority(&s->stream, cudaStreamNonBlocking, prio) != cudaSuccess) { delete s; cudaGetLastError(); return nullptr; }
+    for (int i = 0; i < 32; ++i)
+        if (cudaEventCreateWithFlags(&s->ev[i], cudaEventDisableTiming) != cudaSuccess) { delete s; cudaGetLastError(); return nullptr; }
+    if (cudaEventCreateWithFlags(&s->pending, cudaEventDisableTiming) != cudaSuccess) { delete s; cudaGetLastError(); return nullptr; }
+    s->has_pending = false;
+    g_side.emplace(SideKey{dev, caller}, s);
+    return s;
 }
 
 cudaEvent_t SideStream::event() { return ev[(next++) & 31u]; }
@@ -76,15 +87,20 @@ void SideStream::join(cudaStream_t into)
 
 void SideStream::defer()
 {
+    std::lock_guard<std::mutex> lock(g_side_mutex);
     cudaEventRecord(pending, stream);
+    if (!has_pending) g_pending[device].push_back(this);
     has_pending = true;
 }
 
 void SideStream::join_pending(cudaStream_t into)
 {
-    if (!has_pending) return;
-    cudaStreamWaitEvent(into, pending, 0);
-    has_pending = false;
+    std::lock_guard<std::mutex> lock(g_side_mutex);
+    for (SideStream *s : g_pending[device]) {
+        cudaStreamWaitEvent(into, s->pending, 0);
+        s->has_pending = false;
+    }
+    g_pending[device].clear();
 }
 
 static std::atomic<uint64_t> g_launches{0};

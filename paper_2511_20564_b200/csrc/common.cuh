@@ -28,17 +28,19 @@ int32_t check_launch(const char *what);
 // inside one entry point.  fork() makes the helper stream wait for what the caller's stream has enqueued so far; join()
 // makes the caller's stream wait for the helper stream.  Both are plain event record / wait pairs, so they
 // are legal inside a stream capture.  get() returns nullptr if the stream cannot be created (the caller
-// then stays on its own stream).
+// then stays on its own stream).  defer() leaves the helper stream's work unjoined and notes it for the device;
+// join_pending() makes a stream wait for everything deferred on this helper's device, whichever stream deferred it.
 struct SideStream {
     cudaStream_t stream;
     cudaStream_t owner;           // the caller's stream this helper belongs to
+    int device;
     cudaEvent_t ev[32];
     unsigned next;
     cudaEvent_t pending;          // end of helper-stream work that a later entry point has to wait for
     bool has_pending;
     static SideStream *get(cudaStream_t caller);
-    void defer();                 // remember the helper stream's current end as pending
-    void join_pending(cudaStream_t into);
+    void defer();                 // remember the helper stream's current end as pending work of the device
+    void join_pending(cudaStream_t into);   // `into` waits for all pending work of this helper's device
     cudaEvent_t event();
     void fork(cudaStream_t from);
     void join(cudaStream_t into);

@@ -28,4 +28,12 @@ int32_t sample_khop_impl(const e2egrec_csr *graph, const int32_t *seeds, int32_t
                          int32_t n_hops, const int32_t *fanouts, uint64_t seed, uint32_t step, uint32_t flags,
                          const e2egrec_block *blocks, void *scratch, size_t scratch_bytes, cudaStream_t st);
 
+// aggregate.cu ----------------------------------------------------------------------------
+// Whole-graph segment reduction shared by e2egrec_aggregate_forward / _backward and the workspace-free entry point:
+// argument checks, the scratch size for n_entries entries of d values, and the launch itself on scratch `ws`.
+int32_t check_mats(const e2egrec_mat *in, const e2egrec_mat *out, int64_t out_rows);
+size_t full_ws_bytes(int64_t n_entries, int d, int32_t dtype);
+int32_t full_aggregate(int64_t n_seg, int64_t n_entries, const int64_t *ptr, const int32_t *idx, const float *w,
+                       const e2egrec_mat *in, const e2egrec_mat *out, int mean, void *ws, cudaStream_t st);
+
 }  // namespace e2egrec

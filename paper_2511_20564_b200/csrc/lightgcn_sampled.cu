@@ -134,15 +134,20 @@ int32_t forward_impl(const e2egrec_block *blocks, const LgPlan &p, const e2egrec
         o.ld_out = p.d;
         o.seg_scale = reinterpret_cast<const float *>(ctx + p.t_off[L - 1 - l]);
         const SegScratch sc = seg_scratch_carve(b.cap_edges, kLgRun, p.d, p.es, ctx + p.seg_off);
+        bool ok;
         if (l == 0)     // H^(0) rows are read straight from the feature table through the global ids
-            dispatch_seg_reduce<T, int32_t, true>(static_cast<const T *>(X->data), X->ld, b.indptr, b.nbr_global,
+            ok = dispatch_seg_reduce<T, int32_t, true>(static_cast<const T *>(X->data), X->ld, b.indptr, b.nbr_global,
                                                   &b.counts[CNT_DST], 0, b.cap_dst, inv_sqrt_deg, kLgRun, p.d, X->dtype, nullptr,
                                                   sc, o, st);
         else
-            dispatch_seg_reduce<T, int32_t, true>(reinterpret_cast<const T *>(ctx + p.h_off[l - 1]), p.d, b.indptr, b.col,
+            ok = dispatch_seg_reduce<T, int32_t, true>(reinterpret_cast<const T *>(ctx + p.h_off[l - 1]), p.d, b.indptr, b.col,
                                                   &b.counts[CNT_DST], 0, b.cap_dst,
                                                   reinterpret_cast<const float *>(ctx + p.s_off[L - 1 - l]), kLgRun, p.d,
                                                   X->dtype, nullptr, sc, o, st);
+        if (!ok) {
+            set_last_error("lightgcn_sampled_forward: no kernel for this row width");
+            return E2EGREC_ERR_UNSUPPORTED;
+        }
         layers.h[l] = out;
     }
     note_launch();
@@ -173,9 +178,12 @@ int32_t backward_impl(const e2egrec_block *blocks, const LgPlan &fp, const LgPla
         o.ld_out = ld_out;
         o.seg_scale = reinterpret_cast<const float *>(ctx + fp.s_off[L - 1 - l]);
         const SegScratch sc = seg_scratch_carve(b.cap_edges, kLgRun, d, fp.es, scratch + bp.seg_off);
-        dispatch_seg_reduce<T, int32_t, true>(g_in, d, b.csc_ptr, b.csc_row, &b.counts[CNT_SRC], 0, b.cap_src,
-                                              reinterpret_cast<const float *>(ctx + fp.t_off[L - 1 - l]), kLgRun, d, dtype,
-                                              b.csc_col, sc, o, st);
+        if (!dispatch_seg_reduce<T, int32_t, true>(g_in, d, b.csc_ptr, b.csc_row, &b.counts[CNT_SRC], 0, b.cap_src,
+                                                   reinterpret_cast<const float *>(ctx + fp.t_off[L - 1 - l]), kLgRun, d, dtype,
+                                                   b.csc_col, sc, o, st)) {
+            set_last_error("lightgcn_sampled_backward: no kernel for this row width");
+            return E2EGREC_ERR_UNSUPPORTED;
+        }
         note_launch();
         lightgcn_add_rows_kernel<T><<<lg_grid((int64_t)blocks[0].cap_dst * d), 256, 0, st>>>(out, ld_out, dys, counts0, d);
         g_in = out;

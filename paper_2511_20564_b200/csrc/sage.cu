@@ -69,14 +69,21 @@ static void launch_sage_aggregate(const T *Hsrc, int64_t ld, const int32_t *nbr,
 }
 
 template <typename T>
-static void dispatch_sage_aggregate(const T *Hsrc, int64_t ld, const int32_t *nbr, const int32_t *self_ids,
+static bool dispatch_sage_aggregate(const T *Hsrc, int64_t ld, const int32_t *nbr, const int32_t *self_ids,
                                     const e2egrec_block &b, T *cat, int d, int64_t rows, int32_t dtype, cudaStream_t st)
 {
     const RowShape rs = row_shape(d, dtype);
-#define E2E_CASE(L, C) \
-    if (rs.lpr == L && rs.cpl == C) return launch_sage_aggregate<T, L, C>(Hsrc, ld, nbr, self_ids, b, cat, d, rows, st);
+#define E2E_CASE(L, C)                                                                           \
+    if (rs.lpr == L && rs.cpl == C) {                                                            \
+        launch_sage_aggregate<T, L, C>(Hsrc, ld, nbr, self_ids, b, cat, d, rows, st);            \
+        return true;                                                                             \
+    }
     E2E_CASE(4, 1) E2E_CASE(8, 1) E2E_CASE(16, 1) E2E_CASE(32, 1) E2E_CASE(32, 2) E2E_CASE(32, 4)
+    if constexpr (sizeof(T) == 4) {      // rows of 2049 .. 4096 bytes exist only for fp32 (dim <= kMaxDim)
+        E2E_CASE(32, 8)
+    }
 #undef E2E_CASE
+    return false;
 }
 
 // transposed-block entries per lane group: 32, or 128 where the block can hold millions of entries (the longer run's
@@ -98,14 +105,19 @@ static int32_t forward_impl(const e2egrec_block *blocks, int32_t n_layers, const
         const e2egrec_block &b = blocks[p.block];
         T *cat = reinterpret_cast<T *>(ctx + p.cat_off);
         T *hn = reinterpret_cast<T *>(ctx + p.h_off);
+        bool agg_ok;
         if (l == 0) {  // h^(0) rows are read straight from the feature table through the global ids
             tap_begin(TAP_AGG_FWD_OUTER, st);
-            dispatch_sage_aggregate<T>(static_cast<const T *>(X->data), X->ld, b.nbr_global, b.src_nodes, b, cat, p.d_in,
-                                       p.rows, X->dtype, st);
+            agg_ok = dispatch_sage_aggregate<T>(static_cast<const T *>(X->data), X->ld, b.nbr_global, b.src_nodes, b, cat,
+                                                p.d_in, p.rows, X->dtype, st);
             tap_end(TAP_AGG_FWD_OUTER, st);
         } else
-            dispatch_sage_aggregate<T>(reinterpret_cast<const T *>(ctx + plan[l - 1].h_off), p.d_in, b.col, nullptr, b, cat,
-                                       p.d_in, p.rows, X->dtype, st);
+            agg_ok = dispatch_sage_aggregate<T>(reinterpret_cast<const T *>(ctx + plan[l - 1].h_off), p.d_in, b.col, nullptr, b,
+                                                cat, p.d_in, p.rows, X->dtype, st);
+        if (!agg_ok) {
+            set_last_error("sage_forward: no aggregation kernel for this row width");
+            return E2EGREC_ERR_UNSUPPORTED;
+        }
         const float *bl = bias ? bias[l] : nullptr;
         const int relu = act ? act[l] : 1;
         bool done = false;
@@ -277,9 +289,15 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
         }
         if (l == 0) tap_begin(TAP_AGG_BWD_OUTER, st);
         const SegScratch sc = seg_scratch_carve(b.cap_edges, block_run_len(b.cap_edges), p.d_in, dtype_size(X->dtype), scratch + bs.seg_off);
-        dispatch_seg_reduce<T, int32_t, false>(dcat + p.d_in, two_d, b.csc_ptr, b.csc_row, &b.counts[CNT_SRC], 0, b.cap_src,
-                                               nullptr, block_run_len(b.cap_edges), p.d_in, X->dtype, b.csc_col, sc, o, st);
+        const bool seg_ok = dispatch_seg_reduce<T, int32_t, false>(dcat + p.d_in, two_d, b.csc_ptr, b.csc_row, &b.counts[CNT_SRC], 0,
+                                                                   b.cap_src, nullptr, block_run_len(b.cap_edges), p.d_in, X->dtype,
+                                                                   b.csc_col, sc, o, st);
         if (l == 0) tap_end(TAP_AGG_BWD_OUTER, st);
+        if (!seg_ok) {
+            if (side) side->join(st);
+            set_last_error("sage_backward: no aggregation kernel for this row width");
+            return E2EGREC_ERR_UNSUPPORTED;
+        }
     }
     if (side) side->join(st);
     return check_launch("sage_backward");

@@ -674,18 +674,26 @@ inline void launch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const
     tap_end(TAP_SEG_L3, st);
 }
 
+// Returns false (nothing enqueued) when no kernel is built for the row width; rows of up to 4096 bytes (kMaxDim fp32
+// values) are covered, so callers that checked dim <= kMaxDim never see it.
 template <typename T, typename PtrT, bool kWeight, int kInFlight = 4>
-inline void dispatch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const int32_t *idx, const int32_t *n_seg_dev,
+inline bool dispatch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const int32_t *idx, const int32_t *n_seg_dev,
                                 int64_t n_seg_host, int64_t cap_seg, const float *w, int run_len, int d, int32_t dtype,
                                 const int32_t *seg_of, const SegScratch &sc, const SegOut<T> &o, cudaStream_t st)
 {
     const RowShape rs = row_shape(d, dtype);
 #define E2E_CASE(L, C)                                                                                                \
-    if (rs.lpr == L && rs.cpl == C)                                                                                   \
-        return launch_seg_reduce<T, PtrT, L, C, kWeight, kInFlight>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, cap_seg, w, run_len, \
-                                                         d, seg_of, sc, o, st);
+    if (rs.lpr == L && rs.cpl == C) {                                                                                 \
+        launch_seg_reduce<T, PtrT, L, C, kWeight, kInFlight>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, cap_seg, w, run_len, \
+                                                         d, seg_of, sc, o, st);                                       \
+        return true;                                                                                                  \
+    }
     E2E_CASE(4, 1) E2E_CASE(8, 1) E2E_CASE(16, 1) E2E_CASE(32, 1) E2E_CASE(32, 2) E2E_CASE(32, 4)
+    if constexpr (sizeof(T) == 4) {      // rows of 2049 .. 4096 bytes exist only for fp32 (dim <= kMaxDim)
+        E2E_CASE(32, 8)
+    }
 #undef E2E_CASE
+    return false;
 }
 
 }  // namespace e2egrec

@@ -172,9 +172,11 @@ def _powerlaw_graph(n, m, seed):
     return S.coo_to_csr(n, dst, src)
 
 
-@pytest.mark.parametrize("dtype,d", [("bf16", 64), ("f32", 32), ("bf16", 256), ("f32", 512), ("bf16", 1024)])
+@pytest.mark.parametrize("dtype,d", [("bf16", 64), ("f32", 32), ("bf16", 256), ("f32", 512), ("bf16", 1024),
+                                     ("f32", 768), ("f32", 1024)])
 def test_full_graph_aggregation_forward_and_transpose(dtype, d):
-    """Rows with tens of thousands of entries (split over many warps), empty rows, and a ragged tail."""
+    """Rows with tens of thousands of entries (split over many warps), empty rows, and a ragged tail; row widths up to
+    the documented limit of 1024 values in either dtype (4096-byte rows in fp32)."""
     import paper_2511_20564_b200 as E
     n, m = 20_011, 600_000
     indptr, indices = _powerlaw_graph(n, m, 2)
@@ -242,10 +244,11 @@ def test_three_hops_wide_rows_bf16():
     _check_float(case, gpu, ora)
 
 
-@pytest.mark.parametrize("dtype,d,fanouts", [("bf16", 512, (6, 4)), ("f32", 256, (3, 3, 3, 3))])
+@pytest.mark.parametrize("dtype,d,fanouts", [("bf16", 512, (6, 4)), ("f32", 256, (3, 3, 3, 3)), ("f32", 768, (4, 3)),
+                                             ("f32", 1024, (5,)), ("bf16", 1024, (4, 2))])
 def test_widest_rows_and_four_hops(dtype, d, fanouts):
-    """Rows of 1 024 bytes (several 16-byte chunks per lane, the large shared-memory form of the segment kernel) and the
-    largest number of hops the library takes."""
+    """Rows of 1 024 to 4 096 bytes (several 16-byte chunks per lane, the large shared-memory form of the segment kernel;
+    1024 values per row is the documented limit for both dtypes) and the largest number of hops the library takes."""
     base = S.WORKLOADS["medium_small"]
     w = S.Workload("wide", base.n_users, base.n_items, base.n_interactions, 1.2, 1.2, 1, d, d, dtype, fanouts, 48)
     case = Case(w, step=2)
@@ -316,6 +319,34 @@ def test_deferred_transposition_joins_before_use():
     E.sample_join()
     torch.cuda.synchronize()
     assert_blocks_equal(blocks.to_host(), ora["blocks"])
+
+
+def test_deferred_transposition_is_joined_from_another_stream():
+    """A transposition deferred on one stream is complete for a later-ordered stream once that stream has called
+    e2egrec_sample_join (or the backward pass): the join covers everything deferred on the device."""
+    import paper_2511_20564_b200 as E
+    w = S.WORKLOADS["medium_small"]
+    case = Case(w, step=7)
+    ora = case.run_oracle()
+    ip, ix = torch.from_numpy(case.indptr).cuda(), torch.from_numpy(case.indices).cuda()
+    seeds = torch.from_numpy(case.seeds).cuda()
+    blocks = E.Blocks(w.n_nodes, case.seeds.size, w.fanouts)
+    sa, sb = torch.cuda.Stream(), torch.cuda.Stream()
+    torch.cuda.synchronize()
+    for _ in range(3):
+        with torch.cuda.stream(sa):
+            E.sample_khop(ip, ix, seeds, blocks, w.seed, 7, defer_transpose=True)
+        sb.wait_stream(sa)
+        with torch.cuda.stream(sb):
+            E.sample_join()
+            snap = [{k: blocks.t[h][k].clone() for k in ("csc_ptr", "csc_row", "csc_eid", "csc_col")}
+                    for h in range(len(w.fanouts))]
+        sb.synchronize()
+        for h, (got, o) in enumerate(zip(snap, ora["blocks"])):
+            assert np.array_equal(got["csc_ptr"].cpu().numpy()[: o["n_src"] + 1], o["csc_ptr"])
+            for k in ("csc_row", "csc_eid", "csc_col"):
+                assert np.array_equal(got[k].cpu().numpy()[: o["n_edges"]], o[k]), f"hop {h}: {k}"
+        sa.wait_stream(sb)
 
 
 def test_sampling_of_the_next_batch_beside_the_current_step():

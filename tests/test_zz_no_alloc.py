@@ -10,6 +10,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 import synth_inputs as S
 from helpers import assert_close
 
@@ -33,21 +34,54 @@ def test_static_scratch_variant_matches_the_workspace_variant_twice_in_a_row():
         out = torch.full((n, d), float("nan"), dtype=dtype, device="cuda")
         E.aggregate_forward_static(ip, ix, X, out)
         torch.cuda.synchronize()
-        assert_close("static vs workspace", out.float().cpu().numpy(), want.float().cpu().numpy()[:n],
-                     dtype == torch.bfloat16)
+        bf16 = dtype == torch.bfloat16
+        # against the other entry point: the same launches on another scratch buffer, so within the tests' tolerance
+        # and in fact bit for bit
+        assert_close("static vs workspace", out.float().cpu().numpy(), want.float().cpu().numpy()[:n], bf16)
+        assert torch.equal(out, want[:n])
+        # and against the CPU oracle's mean aggregation (Eq. 2 over whole rows), like every other parity test
+        X_h = X.float().cpu().numpy()
+        deg = np.maximum(np.diff(indptr), 1).astype(np.float64)[:, None]
+        rss = np.sqrt(oracle.mean_aggregate(indptr, indices, X_h.astype(np.float64) ** 2) / deg)
+        assert_close("static vs oracle", out.float().cpu().numpy(), oracle.mean_aggregate(indptr, indices, X_h, bf16), bf16, rss)
 
 
-def test_static_scratch_variant_rejects_what_does_not_fit():
+def _largest_fitting_entries(E, d, dtype, limit):
+    """Largest entry count whose scratch (the size e2egrec_aggregate_forward asks for) still fits the built-in buffer."""
+    X = torch.zeros(1, d, dtype=dtype, device="cuda")
+    need = lambda m: E.binding.aggregate_ws_bytes(m, X)
+    lo, hi = 1, 1 << 31
+    while hi - lo > 1:
+        mid = (lo + hi) // 2
+        lo, hi = (mid, hi) if need(mid) <= limit else (lo, mid)
+    return lo
+
+
+def test_static_scratch_variant_at_its_limit_and_beyond():
+    """The largest input that fits is computed (and matches the workspace variant bit for bit); one entry more is
+    refused with the sizes in the message and nothing is written."""
     import paper_2511_20564_b200 as E
     limit = E.aggregate_forward_static_limit()
     assert limit == 8 << 20
-    d = 256
-    m = (limit // (2 * d * 4) + 2) * 128             # one chunk of 128 entries too many
-    n = 10
-    indptr = torch.zeros(n + 1, dtype=torch.int64, device="cuda")
-    indptr[1:] = m
-    indices = torch.zeros(m, dtype=torch.int32, device="cuda")
-    X = torch.zeros(n, d, dtype=torch.bfloat16, device="cuda")
-    out = torch.zeros(n, d, dtype=torch.bfloat16, device="cuda")
+    d, dtype = 1024, torch.float32                      # the widest rows: the limit is reached with few entries
+    m = _largest_fitting_entries(E, d, dtype, limit)
+    assert m < 2_000_000
+    n = 64
+    rng = np.random.default_rng(0)
+    cuts = np.sort(rng.integers(0, m + 1, n - 1))
+    indptr_h = np.concatenate([[0], cuts, [m]]).astype(np.int64)
+    indices_h = rng.integers(0, n, m + 1).astype(np.int32)
+    X = torch.from_numpy(S.normal_features(n, d, 1)).cuda()
+    ip, ix = torch.from_numpy(indptr_h).cuda(), torch.from_numpy(indices_h).cuda()
+    out = torch.full((n, d), float("nan"), dtype=dtype, device="cuda")
+    E.aggregate_forward_static(ip, ix[:m], X, out)
+    want, _ = E.aggregate_forward(ip, ix[:m], X)
+    torch.cuda.synchronize()
+    assert torch.equal(out, want[:n])
+    ip2 = ip.clone()
+    ip2[-1] = m + 1
+    out.fill_(7.0)
     with pytest.raises(E.E2EGrecError, match="built-in buffer"):
-        E.aggregate_forward_static(indptr, indices, X, out)
+        E.aggregate_forward_static(ip2, ix, X, out)
+    torch.cuda.synchronize()
+    assert bool((out == 7.0).all())
