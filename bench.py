@@ -327,7 +327,7 @@ def run_ours(args, w):
         E.blocks_transpose(blocks2[p])
 
     if args.multitask:
-        # the two-task step of Sec. 4.2: the recommendation gradient and the gradient of the SSL reconstruction loss go
+        # the two-task step of Sec. 4.2 / 4.3.1: the recommendation gradient and the gradient of the SSL reconstruction loss go
         # through the encoder one after the other (weight gradients accumulate), their norms at the shared input feed
         # one GradNorm step of the task weights
         if w.hidden != w.dim:

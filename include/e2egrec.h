@@ -301,6 +301,17 @@ int32_t e2egrec_joint_step(const e2egrec_csr *graph, const e2egrec_mat *X, const
 #define E2EGREC_JOINT_WHOLE   0u
 #define E2EGREC_JOINT_SAMPLE  1u
 #define E2EGREC_JOINT_COMPUTE 2u
+/* Options, or-ed into `phase` (they fix the layout of ws, so every call on one workspace passes the same ones):
+ * E2EGREC_JOINT_LINEAR  identity activations in every encoder layer and in both hidden tower layers (a linear ranking
+ *     model; also what lets a test hold every gradient element to the plain tolerance, since no sign is decided).
+ * E2EGREC_JOINT_GATE    concatenation with gating (Sec. 4.3.2): the tower reads z_fused = g * z with
+ *     g = sigmoid(W_g z + b_g) instead of z.  W_tower, b_tower, dW_tower and db_tower then have a fourth entry each:
+ *     W_tower[3] = W_g [zdim x zdim] (zdim = 2 d_L + dense_dim), b_tower[3] = b_g (device float[zdim] or NULL),
+ *     dW_tower[3] (device float[zdim x zdim]) and db_tower[3] (device float[zdim] or NULL) receive their gradients.
+ *     For bf16 shapes the tensor-core kernel takes, sigmoid and the product with z run in the epilogue of the W_g
+ *     product; the pre-activation, g and z_fused are stored as bf16, as are the gradients between the steps. */
+#define E2EGREC_JOINT_LINEAR  0x100u
+#define E2EGREC_JOINT_GATE    0x200u
 int32_t e2egrec_joint_step_phase(const e2egrec_csr *graph, const e2egrec_mat *X, const int32_t *pair_user,
                                  const int32_t *pair_item, int32_t n_pairs, const float *dense, int32_t dense_dim,
                                  const float *labels, int32_t n_hops, const int32_t *fanouts,
@@ -309,6 +320,18 @@ int32_t e2egrec_joint_step_phase(const e2egrec_csr *graph, const e2egrec_mat *X,
                                  float *const *dW_tower, float *const *db_tower, const e2egrec_mat *dX_rows,
                                  int32_t *dX_ids, int32_t *n_dX_rows, void *ws, size_t *ws_bytes, uint32_t phase,
                                  void *stream);
+
+/* Where a joint step keeps its activations inside ws (for callers that want the intermediate embeddings of Sec. 3.1
+ * or the tower's hidden layers; the arguments are those of the step, flags = the options or-ed into its `phase`).
+ *   tower_offset  host size_t[5]: byte offsets of z, a1, a2, the gate g and z_fused (the last two equal z's offset
+ *                 without E2EGREC_JOINT_GATE); row-major [*pair_rows x width] in X's dtype, widths zdim, h1, h2, zdim,
+ *                 zdim; *pair_rows = n_pairs rounded up to 128, rows >= n_pairs are zero.
+ *   enc_h_offset  host size_t[n_hops], enc_rows host int64[n_hops]: the output of encoder layer l, row-major
+ *                 [enc_rows[l] x d_out(l)]; only the first n_dst rows of the layer's block are meaningful. */
+int32_t e2egrec_joint_step_layout(const e2egrec_csr *graph, const e2egrec_mat *X, int32_t n_pairs, int32_t dense_dim,
+                                  int32_t n_hops, const int32_t *fanouts, const e2egrec_mat *W_gnn,
+                                  const e2egrec_mat *W_tower, uint32_t flags, size_t *tower_offset, size_t *enc_h_offset,
+                                  int64_t *enc_rows, int64_t *pair_rows);
 
 /* Whole-graph neighbourhood aggregation without sampling (Sec. 3.1 Eq. 2 with S(u) = N(u); the
  * "complete graph" case of Sec. 4.1):  out[i] = (1/deg i) sum_{e in row i} X[indices[e]]  (0 for an

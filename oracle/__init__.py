@@ -22,7 +22,7 @@ _SRC = os.path.join(_HERE, "oracle.c")
 def build(force: bool = False) -> str:
     """Compile oracle.c into liboracle.so (gcc -O2, strict IEEE arithmetic)."""
     if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
-        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-ffp-contract=off",
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-fPIC", "-shared", "-ffp-contract=off", "-fopenmp",
                                "-o", _SO, _SRC, "-lm"])
     return _SO
 
@@ -40,7 +40,19 @@ def lib():
         _lib.oracle_relabel.restype = C.c_int32
         _lib.oracle_csr_from_coo.restype = C.c_int
         _lib.oracle_bce_with_logits.restype = C.c_double
+        _lib.oracle_max_threads.restype = C.c_int
     return _lib
+
+
+def max_threads() -> int:
+    """Threads the row loops of the C functions use (OpenMP's current maximum)."""
+    return int(lib().oracle_max_threads())
+
+
+def set_threads(n: int) -> None:
+    """Sets that number (1 = the single-core program).  Results do not depend on it: every output element is
+    still summed by one thread in the written order."""
+    lib().oracle_set_threads(C.c_int(int(n)))
 
 
 def _p(a):
@@ -296,17 +308,22 @@ def full_aggregate_backward(indptr, indices, n_src, G, bf16=False, row_len=None)
 # ----------------------------------------------------------------------------- joint step
 
 def joint_step(indptr, indices, X, pair_user, pair_item, dense, labels, fanouts, W_gnn, W_tower, b_tower,
-               seed, step, bf16=False):
+               seed, step, bf16=False, acts_gnn=None, acts_tower=(1, 1), gate=None):
     """Joint GNN + ranking-tower step (Theorem 1: z = [h_theta || b]; BCE on the tower output, Sec. 5.1).
 
     seeds = ascending distinct endpoints of the pairs; z_p = [h(u_p) || h(i_p) || b_p]; three dense layers
     (ReLU, ReLU, none); loss = mean BCE-with-logits; then the adjoints back to the tower parameters, the GNN
     weights and the sampled feature rows.  Returns a dict of everything the GPU call returns.
+
+    acts_gnn / acts_tower: 1 = ReLU (default), 0 = identity, per encoder layer / for the two hidden tower layers.
+    gate = (W_g [zdim x zdim], b_g [zdim] or None): the concatenated features pass through the gating fusion of
+    Sec. 4.3.2, z_fused = sigmoid(W_g z + b_g) * z, before the tower; the result then carries dW_gate, db_gate.
+    The entry "trace" keeps the intermediate activations and gradients in the order they were formed.
     """
     pair_user, pair_item = _i32(pair_user), _i32(pair_item)
     seeds = np.unique(np.concatenate([pair_user, pair_item])).astype(np.int32)
     blocks = sample_khop(indptr, indices, seeds, fanouts, seed, step)
-    H, ctx = sage_forward(blocks, X, W_gnn, bf16=bf16)
+    H, ctx = sage_forward(blocks, X, W_gnn, acts=acts_gnn, bf16=bf16)
     pos_u, pos_i = np.searchsorted(seeds, pair_user), np.searchsorted(seeds, pair_item)
     dL = H.shape[1]
     dense = _f64(dense)
@@ -314,21 +331,31 @@ def joint_step(indptr, indices, X, pair_user, pair_item, dense, labels, fanouts,
         dense = round_bf16(dense)
     z = np.concatenate([H[pos_u], H[pos_i], dense], axis=1)
     b = [None, None, None] if b_tower is None else list(b_tower)
-    a1 = dense_forward(z, W_tower[0], b[0], 1, bf16)
-    a2 = dense_forward(a1, W_tower[1], b[1], 1, bf16)
+    zf, g = (z, None) if gate is None else gate_fusion_forward(z, gate[0], gate[1], bf16)
+    a1 = dense_forward(zf, W_tower[0], b[0], acts_tower[0], bf16)
+    a2 = dense_forward(a1, W_tower[1], b[1], acts_tower[1], bf16)
     t = dense_forward(a2, W_tower[2], b[2], 0, False)
     loss, dt = bce_with_logits(t[:, 0], labels)
     dW3, db3, da2 = dense_backward(dt[:, None], t, a2, W_tower[2], 0, bf16)
-    dW2, db2, da1 = dense_backward(da2, a2, a1, W_tower[1], 1, bf16)
-    dW1, db1, dz = dense_backward(da1, a1, z, W_tower[0], 1, bf16)
+    dW2, db2, da1 = dense_backward(da2, a2, a1, W_tower[1], acts_tower[1], bf16)
+    dW1, db1, dzf = dense_backward(da1, a1, zf, W_tower[0], acts_tower[0], bf16)
+    out = {}
+    if gate is None:
+        dz = dzf
+    else:
+        dz, out["dW_gate"], out["db_gate"] = gate_fusion_backward(dzf, z, g, gate[0], bf16)
     dH = np.zeros_like(H)
     np.add.at(dH, pos_u, dz[:, :dL])
     np.add.at(dH, pos_i, dz[:, dL:2 * dL])
     if bf16:
         dH = round_bf16(dH)
-    dW_gnn, _, dX = sage_backward(blocks, ctx, W_gnn, dH, bf16=bf16)
-    return dict(seeds=seeds, blocks=blocks, loss=loss, logits=t[:, 0], dW_tower=[dW1, dW2, dW3],
-                db_tower=[db1, db2, db3], dW_gnn=dW_gnn, dX=dX, dX_ids=blocks[-1]["src_nodes"], H=H, dH=dH)
+    enc_trace = []
+    dW_gnn, _, dX = sage_backward(blocks, ctx, W_gnn, dH, acts=acts_gnn, bf16=bf16, trace=enc_trace)
+    out.update(seeds=seeds, blocks=blocks, loss=loss, logits=t[:, 0], dW_tower=[dW1, dW2, dW3],
+               db_tower=[db1, db2, db3], dW_gnn=dW_gnn, dX=dX, dX_ids=blocks[-1]["src_nodes"], H=H, dH=dH,
+               trace=dict(ctx=ctx, enc=enc_trace, pos_u=pos_u, pos_i=pos_i, z=z, gate=g, zf=zf, a1=a1, a2=a2, dt=dt,
+                          da2=da2, da1=da1, dzf=dzf, dz=dz))
+    return out
 
 
 # ----------------------------------------------------------------------------- LightGCN
@@ -412,7 +439,7 @@ def lightgcn_sampled_backward(blocks, ctx, dY, bf16=False):
     return G
 
 
-# ----------------------------------------------------------------------------- SSL task and GradNorm (Sec. 4.2)
+# ----------------------------------------------------------------------------- SSL task (Sec. 4.2) and GradNorm (Sec. 4.3.1)
 
 def ssl_loss(H, X_rows, weight=1.0, bf16=False):
     """Graph feature auto-encoder loss with the identity decoder (Sec. 4.2): L_ssl = ||X - H||_F^2 over the seed
@@ -430,7 +457,7 @@ def frobenius_norm(a):
 
 
 def gradnorm_update(w, L, L0, g, gamma=1.0, lr=0.025, w_min=1e-6):
-    """One GradNorm step for the task weights (Sec. 4.2, "Gradient-Based Task Weighting").
+    """One GradNorm step for the task weights (Sec. 4.3.1, "Gradient-Based Task Weighting").
 
     w: current weights; L, L0: current and initial task losses; g: norms of the *unweighted* task gradients with
     respect to the shared input, so that G_i = w_i g_i.  With r_i = (L_i/L0_i) / mean_j(L_j/L0_j) and the targets
@@ -448,7 +475,7 @@ def gradnorm_update(w, L, L0, g, gamma=1.0, lr=0.025, w_min=1e-6):
     return w_new * (T / w_new.sum()), L_gn
 
 
-# ----------------------------------------------------------------------------- gated fusion (Sec. 4.3.1)
+# ----------------------------------------------------------------------------- gated fusion (Sec. 4.3.2)
 
 def gate_fusion_forward(F, Wg, bg, bf16=False):
     """Concatenation with gating: g = sigmoid(F Wg^T + bg), F_fused = g * F (element-wise), F = the concatenated

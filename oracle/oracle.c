@@ -29,6 +29,31 @@
 #include <stdint.h>
 #include <stdlib.h>
 #include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+/* Threads.  The loops over destination rows (or over feature columns, where rows collide) carry an OpenMP
+ * pragma so that the oracle can be timed on one core and on all of them.  Every output element is still
+ * produced by one thread that adds its terms in the order written here, so the results do not depend on
+ * the number of threads. */
+int oracle_max_threads(void)
+{
+#ifdef _OPENMP
+    return omp_get_max_threads();
+#else
+    return 1;
+#endif
+}
+
+void oracle_set_threads(int n)
+{
+#ifdef _OPENMP
+    omp_set_num_threads(n > 0 ? n : 1);
+#else
+    (void)n;
+#endif
+}
 
 /* ------------------------------------------------------------------------- */
 /* Storage rounding                                                           */
@@ -266,6 +291,7 @@ void oracle_block_csc(int32_t n_dst, int32_t n_src, const int32_t *blk_indptr, c
 /* h^(0) = X: rows of the feature matrix for the given node ids ("embedding lookup"). */
 void oracle_gather_rows(const double *X, int64_t ld, const int32_t *ids, int64_t n, int32_t d, double *out)
 {
+#pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < n; ++i)
         for (int32_t k = 0; k < d; ++k) out[i * d + k] = X[(int64_t)ids[i] * ld + k];
 }
@@ -275,6 +301,7 @@ void oracle_gather_rows(const double *X, int64_t ld, const int32_t *ids, int64_t
 void oracle_mean_aggregate(const int64_t *indptr, const int32_t *col, int64_t n_dst,
                            const double *H, int32_t d, double *agg, int round_bf16)
 {
+#pragma omp parallel for schedule(dynamic, 64)
     for (int64_t i = 0; i < n_dst; ++i) {
         int64_t cnt = indptr[i + 1] - indptr[i];
         for (int32_t k = 0; k < d; ++k) {
@@ -294,6 +321,7 @@ void oracle_sage_update(const double *Hself, const double *agg, int64_t n_dst, i
                         const double *W, const double *bias, int32_t d_out, int act,
                         double *Z, double *Hout, int round_bf16)
 {
+#pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < n_dst; ++i)
         for (int32_t o = 0; o < d_out; ++o) {
             const double *w = W + (int64_t)o * 2 * d_in;
@@ -321,20 +349,31 @@ void oracle_sage_update_backward(const double *dHout, const double *Hout, const 
                                  int32_t d_out, int act, double *dW, double *db,
                                  double *dSelf, double *dAgg)
 {
-    double *dz = (double *)malloc(sizeof(double) * (size_t)d_out);
+    /* dZ for all rows first; then every row of dSelf / dAgg and every row of dW / entry of db is the work of
+     * one thread, which adds its terms in ascending order of o (dSelf, dAgg) or of i (dW, db) */
+    double *dz = (double *)malloc(sizeof(double) * (size_t)(n_dst > 0 ? n_dst : 1) * (size_t)d_out);
+#pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < n_dst; ++i) {
         for (int32_t o = 0; o < d_out; ++o)
-            dz[o] = (act && !(Hout[i * d_out + o] > 0.0)) ? 0.0 : dHout[i * d_out + o];
+            dz[i * d_out + o] = (act && !(Hout[i * d_out + o] > 0.0)) ? 0.0 : dHout[i * d_out + o];
         for (int32_t k = 0; k < d_in; ++k) { dSelf[i * d_in + k] = 0.0; dAgg[i * d_in + k] = 0.0; }
         for (int32_t o = 0; o < d_out; ++o) {
-            if (db) db[o] += dz[o];
             const double *w = W + (int64_t)o * 2 * d_in;
-            double *gw = dW + (int64_t)o * 2 * d_in;
             for (int32_t k = 0; k < d_in; ++k) {
-                gw[k] += dz[o] * Hself[i * d_in + k];
-                gw[d_in + k] += dz[o] * agg[i * d_in + k];
-                dSelf[i * d_in + k] += dz[o] * w[k];
-                dAgg[i * d_in + k] += dz[o] * w[d_in + k];
+                dSelf[i * d_in + k] += dz[i * d_out + o] * w[k];
+                dAgg[i * d_in + k] += dz[i * d_out + o] * w[d_in + k];
+            }
+        }
+    }
+#pragma omp parallel for schedule(static)
+    for (int32_t o = 0; o < d_out; ++o) {
+        double *gw = dW + (int64_t)o * 2 * d_in;
+        for (int64_t i = 0; i < n_dst; ++i) {
+            const double g = dz[i * d_out + o];
+            if (db) db[o] += g;
+            for (int32_t k = 0; k < d_in; ++k) {
+                gw[k] += g * Hself[i * d_in + k];
+                gw[d_in + k] += g * agg[i * d_in + k];
             }
         }
     }
@@ -349,23 +388,35 @@ void oracle_mean_aggregate_backward(const int64_t *indptr, const int32_t *col, i
                                     const double *dSelf, const double *dAgg, int32_t d,
                                     double *dH, int round_bf16)
 {
+#pragma omp parallel for schedule(static)
     for (int64_t s = 0; s < n_src; ++s)
         for (int32_t k = 0; k < d; ++k) {
             double v = (dSelf && s < n_dst) ? dSelf[s * d + k] : 0.0;
             dH[s * d + k] = round_bf16 ? oracle_round_bf16(v) : v;
         }
-    double *g = (double *)malloc(sizeof(double) * (size_t)d);
-    for (int64_t i = 0; i < n_dst; ++i) {
-        int64_t cnt = indptr[i + 1] - indptr[i];
-        if (cnt == 0) continue;
-        for (int32_t k = 0; k < d; ++k) {
-            double v = dAgg[i * d + k] / (double)cnt;
-            g[k] = round_bf16 ? oracle_round_bf16(v) : v;
+    /* rows of dH collide between destinations, feature columns do not: every thread owns a range of columns and
+     * walks all entries in order, so an element receives its terms in the same order whatever the thread count */
+#pragma omp parallel
+    {
+        int nt = 1, tid = 0;
+#ifdef _OPENMP
+        nt = omp_get_num_threads();
+        tid = omp_get_thread_num();
+#endif
+        const int32_t k0 = (int32_t)((int64_t)d * tid / nt), k1 = (int32_t)((int64_t)d * (tid + 1) / nt);
+        double *g = (double *)malloc(sizeof(double) * (size_t)(d > 0 ? d : 1));
+        for (int64_t i = 0; i < n_dst && k0 < k1; ++i) {
+            int64_t cnt = indptr[i + 1] - indptr[i];
+            if (cnt == 0) continue;
+            for (int32_t k = k0; k < k1; ++k) {
+                double v = dAgg[i * d + k] / (double)cnt;
+                g[k] = round_bf16 ? oracle_round_bf16(v) : v;
+            }
+            for (int64_t e = indptr[i]; e < indptr[i + 1]; ++e)
+                for (int32_t k = k0; k < k1; ++k) dH[(int64_t)col[e] * d + k] += g[k];
         }
-        for (int64_t e = indptr[i]; e < indptr[i + 1]; ++e)
-            for (int32_t k = 0; k < d; ++k) dH[(int64_t)col[e] * d + k] += g[k];
+        free(g);
     }
-    free(g);
     if (round_bf16) oracle_round_bf16_array(dH, n_src * d);
 }
 
@@ -378,6 +429,7 @@ void oracle_mean_aggregate_backward(const int64_t *indptr, const int32_t *col, i
 void oracle_dense_forward(const double *Xin, int64_t n, int32_t d_in, const double *W, const double *b,
                           int32_t d_out, int act, double *Y, int round_bf16)
 {
+#pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < n; ++i)
         for (int32_t o = 0; o < d_out; ++o) {
             double z = b ? b[o] : 0.0;
@@ -392,19 +444,24 @@ void oracle_dense_backward(const double *dY, const double *Y, const double *Xin,
                            int64_t n, int32_t d_in, int32_t d_out, int act,
                            double *dW, double *db, double *dX, int round_bf16)
 {
+    /* as in oracle_sage_update_backward: rows of dX, then rows of dW, each summed by one thread in ascending order */
+#pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < n; ++i) {
         for (int32_t k = 0; k < d_in; ++k) dX[i * d_in + k] = 0.0;
         for (int32_t o = 0; o < d_out; ++o) {
             double dz = (act && !(Y[i * d_out + o] > 0.0)) ? 0.0 : dY[i * d_out + o];
-            db[o] += dz;
-            for (int32_t k = 0; k < d_in; ++k) {
-                dW[(int64_t)o * d_in + k] += dz * Xin[i * d_in + k];
-                dX[i * d_in + k] += dz * W[(int64_t)o * d_in + k];
-            }
+            for (int32_t k = 0; k < d_in; ++k) dX[i * d_in + k] += dz * W[(int64_t)o * d_in + k];
         }
         if (round_bf16)
             for (int32_t k = 0; k < d_in; ++k) dX[i * d_in + k] = oracle_round_bf16(dX[i * d_in + k]);
     }
+#pragma omp parallel for schedule(static)
+    for (int32_t o = 0; o < d_out; ++o)
+        for (int64_t i = 0; i < n; ++i) {
+            double dz = (act && !(Y[i * d_out + o] > 0.0)) ? 0.0 : dY[i * d_out + o];
+            db[o] += dz;
+            for (int32_t k = 0; k < d_in; ++k) dW[(int64_t)o * d_in + k] += dz * Xin[i * d_in + k];
+        }
 }
 
 /* Binary cross-entropy on logits t with labels y, mean over the n pairs:

@@ -126,6 +126,10 @@ def lib():
                                          C.POINTER(C.c_size_t), C.c_void_p]
         L.e2egrec_joint_step_phase.restype = C.c_int32
         L.e2egrec_joint_step_phase.argtypes = L.e2egrec_joint_step.argtypes[:-1] + [C.c_uint32, C.c_void_p]
+        L.e2egrec_joint_step_layout.restype = C.c_int32
+        L.e2egrec_joint_step_layout.argtypes = [C.POINTER(Csr), C.POINTER(Mat), C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
+                                                C.POINTER(Mat), C.POINTER(Mat), C.c_uint32, C.c_void_p, C.c_void_p,
+                                                C.c_void_p, C.c_void_p]
         L.e2egrec_graph_from_coo.restype = C.c_int32
         L.e2egrec_graph_from_coo.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                              C.c_void_p, C.c_void_p, C.POINTER(C.c_size_t), C.c_void_p]
@@ -449,16 +453,32 @@ def aggregate_forward_static_limit() -> int:
 
 # ------------------------------------------------------------------------------------------ joint step
 
-class JointStep:
-    """Buffers and arguments of e2egrec_joint_step for a fixed problem shape; `run` enqueues one step."""
+JOINT_LINEAR = 0x100
+JOINT_GATE = 0x200
 
-    def __init__(self, indptr, indices, X, n_pairs, dense_dim, fanouts, W_gnn, W_tower, b_tower=None):
+
+class JointStep:
+    """Buffers and arguments of e2egrec_joint_step for a fixed problem shape; `run` enqueues one step.
+
+    linear=True: identity activations everywhere (E2EGREC_JOINT_LINEAR).  W_gate (and b_gate) given: the gating fusion
+    of the concatenated features (E2EGREC_JOINT_GATE); they travel as the fourth entry of the tower's arrays, and their
+    gradients come back as dW_tower[3], db_tower[3]."""
+
+    def __init__(self, indptr, indices, X, n_pairs, dense_dim, fanouts, W_gnn, W_tower, b_tower=None, linear=False,
+                 W_gate=None, b_gate=None):
         dev = X.device
         self.indptr, self.indices, self.X = indptr, indices, X
         self.n_nodes = indptr.numel() - 1
         self.n_pairs, self.dense_dim = int(n_pairs), int(dense_dim)
         self.fanouts = [int(f) for f in fanouts]
-        self.W_gnn, self.W_tower, self.b_tower = list(W_gnn), list(W_tower), b_tower
+        self.W_gnn, self.W_tower = list(W_gnn), list(W_tower)[:3]
+        self.b_tower = None if b_tower is None else list(b_tower)[:3]
+        self.flags = (JOINT_LINEAR if linear else 0) | (JOINT_GATE if W_gate is not None else 0)
+        if W_gate is not None:
+            self.W_tower.append(W_gate)
+            if self.b_tower is not None or b_gate is not None:
+                self.b_tower = (self.b_tower or [None, None, None]) + [b_gate]
+        self.n_tower = len(self.W_tower)
         L = len(self.fanouts)
         _, cs, _, _ = sample_khop_workspace(self.n_nodes, 2 * self.n_pairs, self.fanouts)
         self.cap_rows = max(cs[L - 1], 1)
@@ -480,19 +500,38 @@ class JointStep:
         sampler_scratch_init(self.n_nodes, self.ws)
 
     def _call(self, user, item, dense, labels, nbytes, stream, seed, step, phase=0):
-        L = len(self.fanouts)
+        L, nt = len(self.fanouts), self.n_tower
         _check(lib().e2egrec_joint_step_phase(
             C.byref(self._g), C.byref(self._x), _ptr(user), _ptr(item), self.n_pairs, _ptr(dense), self.dense_dim,
-            _ptr(labels), L, self._f, self._wg, self._wt, _ptr_array(self.b_tower, 3), C.c_uint64(seed),
+            _ptr(labels), L, self._f, self._wg, self._wt, _ptr_array(self.b_tower, nt), C.c_uint64(seed),
             C.c_uint32(step), _ptr(self.loss), _ptr(self.logits), _ptr_array(self.dW_gnn, L),
-            _ptr_array(self.dW_tower, 3), _ptr_array(self.db_tower, 3), C.byref(self._dx), _ptr(self.dX_ids),
-            _ptr(self.n_rows), None if user is None else _ptr(self.ws), C.byref(nbytes), C.c_uint32(phase), stream),
-            "e2egrec_joint_step_phase")
+            _ptr_array(self.dW_tower, nt), _ptr_array(self.db_tower, nt), C.byref(self._dx), _ptr(self.dX_ids),
+            _ptr(self.n_rows), None if user is None else _ptr(self.ws), C.byref(nbytes), C.c_uint32(phase | self.flags),
+            stream), "e2egrec_joint_step_phase")
 
     def run(self, pair_user, pair_item, dense, labels, seed, step, stream=None, phase=0):
         """phase 0: the whole step; 1: seeds + sampling only; 2: everything else, on the blocks phase 1 left in ws."""
         self._call(pair_user, pair_item, dense, labels, C.c_size_t(self.ws.numel()), _stream(stream), seed, step, phase)
         return self
+
+    def activations(self):
+        """Views into ws of what the last step left there (e2egrec_joint_step_layout): dict with the tower's z, a1, a2,
+        gate, z_fused ([pair_rows x width]) and `enc`, the list of encoder layer outputs ([rows x d_out])."""
+        L = len(self.fanouts)
+        tower, enc, rows, prow = (C.c_size_t * 5)(), (C.c_size_t * L)(), (C.c_int64 * L)(), C.c_int64(0)
+        _check(lib().e2egrec_joint_step_layout(C.byref(self._g), C.byref(self._x), self.n_pairs, self.dense_dim, L, self._f,
+                                               self._wg, self._wt, C.c_uint32(self.flags), tower, enc, rows, C.byref(prow)),
+               "e2egrec_joint_step_layout")
+        es, dt = self.X.element_size(), self.X.dtype
+        zdim, h1, h2 = self.W_tower[0].shape[1], self.W_tower[0].shape[0], self.W_tower[1].shape[0]
+
+        def view(off, r, c):
+            return self.ws[off: off + r * c * es].view(dt).view(r, c)
+
+        out = {k: view(tower[i], prow.value, w) for i, (k, w) in
+               enumerate((("z", zdim), ("a1", h1), ("a2", h2), ("gate", zdim), ("z_fused", zdim)))}
+        out["enc"] = [view(enc[l], rows[l], self.W_gnn[l].shape[0]) for l in range(L)]
+        return out
 
 
 # ------------------------------------------------------------------------------------------ graph ingest

@@ -164,7 +164,23 @@ struct TcEpilogue {
     __nv_bfloat16 *out2;       // optional second copy of the output: rows below rows2, leading dimension ldo2
     int64_t ldo2, rows2;
     int32_t *status;           // device status word (E2EGREC_DEV_TIMEOUT)
+    TcFuse fuse;               // optional gating / product-plus-term forms of the epilogue
 };
+
+__device__ inline float bf16_round(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
+
+// 32 bf16 values of one row (columns c .. c+31) as 16 packed words; zeros when there is no source
+__device__ inline void load_row32(const __nv_bfloat16 *row, bool on, uint32_t (&w)[16])
+{
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (on) v = *reinterpret_cast<const uint4 *>(row + q * 8);
+        w[4 * q] = v.x; w[4 * q + 1] = v.y; w[4 * q + 2] = v.z; w[4 * q + 3] = v.w;
+    }
+}
+__device__ inline float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ inline float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xFFFF0000u); }
 
 // ------------------------------------------------------------------------- kernel
 // Persistent: the grid has at most one CTA per SM and every CTA walks over the live output tiles
@@ -327,6 +343,39 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                         }
                     }
                 }
+                if (ep.fuse.gate_in) {
+                    // gating: the accumulator (+ bias) is the pre-activation; g = sigmoid(pre) with pre and g rounded to
+                    // their storage type, the output is g * F and g itself goes to gate_out
+                    uint32_t fw[16], gpk[16];
+                    load_row32(ep.fuse.gate_in + row * ep.fuse.ld_gate_in + n0 + c, live, fw);
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        float g[2];
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            float p = __uint_as_float(r[j + h]);
+                            if (ep.bias) p += ep.bias[n0 + c + j + h];
+                            p = bf16_round(p);
+                            const float e = expf(-fabsf(p));
+                            g[h] = live ? bf16_round(p >= 0.f ? 1.0f / (1.0f + e) : e / (1.0f + e)) : 0.f;
+                        }
+                        __nv_bfloat162 gh = __floats2bfloat162_rn(g[0], g[1]);
+                        gpk[j >> 1] = *reinterpret_cast<uint32_t *>(&gh);
+                        __nv_bfloat162 oh = __floats2bfloat162_rn(g[0] * bf16_lo(fw[j >> 1]), g[1] * bf16_hi(fw[j >> 1]));
+                        packed[j >> 1] = *reinterpret_cast<uint32_t *>(&oh);
+                    }
+                    if (ep.fuse.gate_out) {
+                        __nv_bfloat16 *grow = ep.fuse.gate_out + row * ep.fuse.ld_gate_out + n0 + c;
+#pragma unroll
+                        for (int q = 0; q < 4; ++q)
+                            *reinterpret_cast<uint4 *>(grow + q * 8) = make_uint4(gpk[4 * q], gpk[4 * q + 1], gpk[4 * q + 2], gpk[4 * q + 3]);
+                    }
+                } else {
+                uint32_t aw[16], bw[16];
+                if (ep.fuse.add_a) {                          // out = round(product) + a * b
+                    load_row32(ep.fuse.add_a + row * ep.fuse.ld_add_a + n0 + c, live, aw);
+                    load_row32(ep.fuse.add_b + row * ep.fuse.ld_add_b + n0 + c, live, bw);
+                }
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
                     float v0 = __uint_as_float(r[j]), v1 = __uint_as_float(r[j + 1]);
@@ -337,10 +386,15 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                         if (col >= ep.scale_from) v0 *= rs;
                         if (col + 1 >= ep.scale_from) v1 *= rs;
                     }
+                    if (ep.fuse.add_a) {
+                        v0 = bf16_round(v0) + bf16_lo(aw[j >> 1]) * bf16_lo(bw[j >> 1]);
+                        v1 = bf16_round(v1) + bf16_hi(aw[j >> 1]) * bf16_hi(bw[j >> 1]);
+                    }
                     if (!live || !((mbits >> j) & 1u)) v0 = 0.f;
                     if (!live || !((mbits >> (j + 1)) & 1u)) v1 = 0.f;
                     __nv_bfloat162 h = __floats2bfloat162_rn(v0, v1);
                     packed[j >> 1] = *reinterpret_cast<uint32_t *>(&h);
+                }
                 }
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
@@ -381,15 +435,37 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
+constexpr int kMaxDevices = 64;
+
+int current_device()
+{
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) { cudaGetLastError(); return 0; }
+    return dev;
+}
+
 int sm_count()
 {
-    static int n = []() {
-        int dev = 0, v = 0;
-        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0)
-            v = 148;
-        return v;
-    }();
-    return n;
+    static int n[kMaxDevices] = {};                  // per device; a race between threads writes the same value twice
+    const int dev = current_device();
+    if (n[dev] <= 0) {
+        int v = 0;
+        if (cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || v <= 0) v = 148;
+        n[dev] = v;
+    }
+    return n[dev];
+}
+
+// Raises the kernel's dynamic shared-memory limit once per device (the attribute belongs to the device's copy of
+// the kernel, so a second device in the same process needs its own call).
+template <typename Kernel>
+bool raise_smem_limit(Kernel kernel, bool (&done)[kMaxDevices])
+{
+    const int dev = current_device();
+    if (done[dev]) return true;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) return false;
+    done[dev] = true;
+    return true;
 }
 
 // [rows x k] bf16 row-major, box = 64 x box_rows, 128-byte swizzle
@@ -429,12 +505,8 @@ bool launch_tn(const __nv_bfloat16 *A, int64_t rows, int k, int64_t lda, const _
     uint32_t tmem_cols = 64;                    // two accumulator buffers, each a power of two of columns >= nt
     while ((int)tmem_cols < 2 * nt) tmem_cols <<= 1;
     const size_t smem = (size_t)stages * (kTileM * kTileK * 2 + (size_t)nt * kTileK * 2) + 1024;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(tc_gemm_tn_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
-            return false;
-        attr_set = true;
-    }
+    static bool attr_set[kMaxDevices] = {};
+    if (!raise_smem_limit(tc_gemm_tn_kernel, attr_set)) return false;
     const int n_tiles_n = n / nt;
     const int64_t tiles_cap = (rows / kTileM) * n_tiles_n;
     const unsigned grid = (unsigned)std::min<int64_t>(tiles_cap, sm_count());
@@ -604,9 +676,17 @@ bool tc_update_forward(const __nv_bfloat16 *cat, int64_t rows, int k, const __nv
 
 bool tc_linear(const __nv_bfloat16 *A, int64_t rows, int k, const __nv_bfloat16 *B, int n, const float *bias, int relu,
                const __nv_bfloat16 *mask, int64_t ld_mask, __nv_bfloat16 *out, int64_t ldo, const int32_t *m_dev,
-               int32_t *status, cudaStream_t st, bool b_is_k_by_n)
+               int32_t *status, cudaStream_t st, bool b_is_k_by_n, const TcFuse *fuse)
 {
     TcEpilogue ep{};
+    if (fuse) {
+        ep.fuse = *fuse;
+        const TcFuse &f = ep.fuse;
+        auto bad = [](const void *p, int64_t ld) { return p && (reinterpret_cast<uintptr_t>(p) % 16 || (ld * 2) % 16); };
+        if (bad(f.gate_in, f.ld_gate_in) || bad(f.gate_out, f.ld_gate_out) || bad(f.add_a, f.ld_add_a) || bad(f.add_b, f.ld_add_b))
+            return false;
+        if ((f.add_a == nullptr) != (f.add_b == nullptr) || (f.gate_in && f.add_a)) return false;
+    }
     ep.out = out;
     ep.ldo = ldo;
     ep.bias = bias;
@@ -652,12 +732,8 @@ bool tc_weight_grad(const __nv_bfloat16 *dY, int64_t rows, int m, const __nv_bfl
     while ((int)tmem_cols < nt) tmem_cols <<= 1;
     const int stages = kMaxStages;
     const size_t smem = (size_t)stages * ((kTileM / 64) + (nt / 64)) * (kTileK * 128) + 1024;
-    static bool attr_set = false;
-    if (!attr_set) {
-        if (cudaFuncSetAttribute(tc_gemm_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess)
-            return false;
-        attr_set = true;
-    }
+    static bool attr_set[kMaxDevices] = {};
+    if (!raise_smem_limit(tc_gemm_rows_kernel, attr_set)) return false;
     dim3 grid((unsigned)(m / kTileM), (unsigned)(n / nt), (unsigned)splits);
     note_launch();
     tc_gemm_rows_kernel<<<grid, kThreads, smem, st>>>(my, mx, nt, tmem_cols, stages, m_dev, part, n, (int64_t)m * n, status);

@@ -20,12 +20,25 @@ bool tc_update_forward(const __nv_bfloat16 *cat, int64_t rows, int k, const __nv
 bool tc_dcat_backward(const __nv_bfloat16 *dz, int64_t rows, int d_out, const __nv_bfloat16 *W, int two_d_in,
                       const float *inv_cnt, __nv_bfloat16 *dcat, const int32_t *m_dev, int32_t *status, cudaStream_t st);
 
+// Optional forms of the product's epilogue (all matrices [rows x n], bf16, 16-byte aligned rows):
+//   gate_in  F:  out = g * F with g = sigmoid(product + bias); the pre-activation and g are rounded to bf16 first,
+//                and g is stored to gate_out as well when that is given (gating fusion, Sec. 4.3.2);
+//   add_a, add_b: out = round_bf16(product) + add_a * add_b, element by element (the gate's input gradient).
+struct TcFuse {
+    const __nv_bfloat16 *gate_in;
+    int64_t ld_gate_in;
+    __nv_bfloat16 *gate_out;
+    int64_t ld_gate_out;
+    const __nv_bfloat16 *add_a, *add_b;
+    int64_t ld_add_a, ld_add_b;
+};
+
 // out = mask * act(A B^T + bias): A [rows x k], B [n x k], out [rows x ldo], optional mask [rows x ld_mask]
 // (outputs zeroed where mask <= 0).  With b_is_k_by_n, B is given as [k x n] row-major instead (out = A B; n a
 // multiple of 64).  Same conventions as above.
 bool tc_linear(const __nv_bfloat16 *A, int64_t rows, int k, const __nv_bfloat16 *B, int n, const float *bias, int relu,
                const __nv_bfloat16 *mask, int64_t ld_mask, __nv_bfloat16 *out, int64_t ldo, const int32_t *m_dev,
-               int32_t *status, cudaStream_t st, bool b_is_k_by_n = false);
+               int32_t *status, cudaStream_t st, bool b_is_k_by_n = false, const TcFuse *fuse = nullptr);
 
 // part[z] = (rows of split z of dY)^T (same rows of Xin): dY [rows x m], Xin [rows x n] bf16 row-major, part
 // [splits x m x n] fp32.  Rows between *m_dev and the next multiple of 64 must be zero in both matrices.

@@ -27,6 +27,8 @@ struct JointPlan {
     size_t seeds_off, pair_local_off, entry_unit_off, pcounts_off, pcsc_ptr_off, pcsc_idx_off, pcsc_eid_off, pcsc_col_off,
         pmeta_off;
     size_t hseed_off, dhseed_off, z_off, a1_off, a2_off, dt_off, dz2_off, dz1_off, dz_off, wt_off, part_off;
+    size_t zf_off, gate_off, dzf_off, gpre_off;               // gated step only: fused input, gate, its gradient, scratch
+    int gated;
     size_t bytes;
 };
 
@@ -137,17 +139,18 @@ weighted_colsum_kernel(const T *__restrict__ a, int d, const float *__restrict__
     }
 }
 
-// dZ2[p, j] = dt[p] * W3[j] where a2[p, j] > 0, stored in the feature dtype; padding rows are zero.
+// dZ2[p, j] = dt[p] * W3[j] where a2[p, j] > 0 (everywhere with the identity activation), stored in the feature dtype;
+// padding rows are zero.
 template <typename T>
 __global__ void dz_top_kernel(const float *__restrict__ dt, const T *__restrict__ w3, const T *__restrict__ a2, int d,
-                              int32_t P, int64_t rows_alloc, T *__restrict__ dz2)
+                              int32_t P, int64_t rows_alloc, int relu, T *__restrict__ dz2)
 {
     const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t p = t / d;
     const int j = (int)(t - p * d);
     if (p >= rows_alloc) return;
     float v = 0.f;
-    if (p < P && to_float<T>(a2[t]) > 0.f) v = dt[p] * to_float<T>(w3[j]);
+    if (p < P && (!relu || to_float<T>(a2[t]) > 0.f)) v = dt[p] * to_float<T>(w3[j]);
     dz2[t] = from_float<T>(v);
 }
 
@@ -221,9 +224,139 @@ void linear_backward_weight(const T *dY, int64_t rows, int n_out, const T *Xin, 
     }
 }
 
+// ------------------------------------------------------------------------------------------ gated fusion (Sec. 4.3.2)
+//   g = sigmoid(F Wg^T + bg),  F_fused = g * F.  bf16 shapes the tensor-core kernel takes: one launch, sigmoid and the
+//   product with F in the epilogue of the F Wg^T product; otherwise the product runs on the fp32-FMA kernel and the gate
+//   is applied element-wise.  Backward: d pre = dFused * F * g (1 - g) element-wise, dWg = d pre^T F, and
+//   dF = d pre Wg + dFused * g with the second term added in the product's epilogue on the tensor-core path.
+__global__ void gate_meta_kernel(int32_t *meta, int32_t n_rows) { meta[0] = n_rows; }
+
+// gate = sigmoid(pre), fused = gate * F for rows < n_rows; zero rows up to rows_alloc
+template <typename T>
+__global__ void gate_apply_kernel(const T *__restrict__ pre, const T *__restrict__ F, int64_t ldf, int d, int32_t n_rows,
+                                  int64_t rows_alloc, T *__restrict__ gate, int64_t ldg, T *__restrict__ fused, int64_t ldo)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t i = t / d;
+    const int k = (int)(t - i * d);
+    if (i >= rows_alloc) return;
+    float g = 0.f, o = 0.f;
+    if (i < n_rows) {
+        const float p = to_float<T>(pre[i * d + k]);
+        const float e = expf(-fabsf(p));
+        g = to_float<T>(from_float<T>(p >= 0.f ? 1.0f / (1.0f + e) : e / (1.0f + e)));      // the stored gate
+        o = g * to_float<T>(F[i * ldf + k]);
+    }
+    gate[i * ldg + k] = from_float<T>(g);
+    fused[i * ldo + k] = from_float<T>(o);
+}
+
+// dpre = dFused * F * g (1 - g) for rows < n_rows, zero rows up to rows_alloc
+template <typename T>
+__global__ void gate_dpre_kernel(const T *__restrict__ dFused, int64_t ldd, const T *__restrict__ F, int64_t ldf,
+                                 const T *__restrict__ gate, int64_t ldg, int d, int32_t n_rows, int64_t rows_alloc,
+                                 T *__restrict__ dpre)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t i = t / d;
+    const int k = (int)(t - i * d);
+    if (i >= rows_alloc) return;
+    float v = 0.f;
+    if (i < n_rows) {
+        const float g = to_float<T>(gate[i * ldg + k]);
+        v = to_float<T>(dFused[i * ldd + k]) * to_float<T>(F[i * ldf + k]) * g * (1.0f - g);
+    }
+    dpre[i * d + k] = from_float<T>(v);
+}
+
+// dF = t + dFused * g for rows < n_rows
+template <typename T>
+__global__ void gate_dF_kernel(const T *__restrict__ tprod, const T *__restrict__ dFused, int64_t ldd,
+                               const T *__restrict__ gate, int64_t ldg, int d, int32_t n_rows, T *__restrict__ dF, int64_t ldo)
+{
+    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const int64_t i = t / d;
+    const int k = (int)(t - i * d);
+    if (i >= n_rows) return;
+    dF[i * ldo + k] = from_float<T>(to_float<T>(tprod[i * d + k]) + to_float<T>(dFused[i * ldd + k]) * to_float<T>(gate[i * ldg + k]));
+}
+
+unsigned cells_grid(int64_t rows, int d) { return (unsigned)std::max<int64_t>(1, ceil_div(rows * d, 256)); }
+
+// Matrix as the gate cores see it: data, leading dimension, rows allocated.
+template <typename T> struct GMat { T *p; int64_t ld, rows; };
+
+// F [rows x d] (rows a multiple of 128, all allocated); meta = {n_rows}; pre: scratch [rows x d] (only used off the
+// tensor cores).  gate / fused receive n_rows rows (and zero rows up to the next multiple of 128 when they have room).
+template <typename T>
+void gate_forward_core(GMat<const T> F, int64_t rows, int32_t n_rows, int d, const T *Wg, const float *bg, T *pre,
+                       GMat<T> gate, GMat<T> fused, const int32_t *meta, int32_t *status, cudaStream_t st)
+{
+    if (use_tc<T>() && F.ld == d && gate.rows >= rows && fused.rows >= rows) {
+        TcFuse fz{};
+        fz.gate_in = reinterpret_cast<const __nv_bfloat16 *>(F.p);
+        fz.ld_gate_in = F.ld;
+        fz.gate_out = reinterpret_cast<__nv_bfloat16 *>(gate.p);
+        fz.ld_gate_out = gate.ld;
+        if (tc_linear(reinterpret_cast<const __nv_bfloat16 *>(F.p), rows, d, reinterpret_cast<const __nv_bfloat16 *>(Wg), d, bg, 0,
+                      nullptr, 0, reinterpret_cast<__nv_bfloat16 *>(fused.p), fused.ld, meta, status, st, false, &fz))
+            return;
+    }
+    if (F.ld == d) {
+        linear_forward<T>(F.p, rows, d, Wg, d, bg, 0, pre, meta, status, st);
+    } else {
+        EpiUpdate<T> epi{pre, d, bg, 0};
+        dim3 grid((unsigned)ceil_div(rows, kGemmBM), (unsigned)ceil_div(d, kGemmBN), 1);
+        note_launch();
+        gemm_simt_kernel<T, false, false, EpiUpdate<T>><<<grid, kGemmThreads, 0, st>>>(F.p, F.ld, Wg, d, rows, d, d, meta, nullptr, epi);
+    }
+    note_launch();
+    gate_apply_kernel<T><<<cells_grid(rows, d), 256, 0, st>>>(pre, F.p, F.ld, d, n_rows,
+                                                             std::min<int64_t>(rows, std::min(gate.rows, fused.rows)), gate.p, gate.ld,
+                                                             fused.p, fused.ld);
+}
+
+// dpre, tprod: scratch [rows x d]; wt: scratch [d x d]; part: scratch [kSplits x d x d] fp32.
+template <typename T>
+void gate_backward_core(GMat<const T> dFused, GMat<const T> F, GMat<const T> gate, int64_t rows, int32_t n_rows, int d, const T *Wg,
+                        T *dpre, T *tprod, T *wt, float *part, GMat<T> dF, float *dWg, float *dbg, const int32_t *meta,
+                        int32_t *status, cudaStream_t st)
+{
+    note_launch();
+    gate_dpre_kernel<T><<<cells_grid(rows, d), 256, 0, st>>>(dFused.p, dFused.ld, F.p, F.ld, gate.p, gate.ld, d, n_rows, rows, dpre);
+    if (F.ld == d) {
+        linear_backward_weight<T>(dpre, rows, d, F.p, d, meta, part, dWg, dbg, status, st);
+    } else {                                                             // strided F: fp32-FMA product
+        EpiPartial epi{part, d, (int64_t)d * d};
+        dim3 grid((unsigned)ceil_div(d, kGemmBM), (unsigned)ceil_div(d, kGemmBN), kSplits);
+        note_launch();
+        gemm_simt_kernel<T, true, true, EpiPartial><<<grid, kGemmThreads, 0, st>>>(dpre, d, F.p, F.ld, d, d, rows, nullptr, meta, epi);
+        note_launch();
+        splitk_reduce_kernel<<<(unsigned)ceil_div((int64_t)d * d, 256), 256, 0, st>>>(part, (int64_t)d * d, kSplits, 0, dWg, nullptr);
+        if (dbg) {
+            note_launch();
+            colsum_kernel<T><<<(unsigned)ceil_div(d, 32), 256, 0, st>>>(dpre, d, meta, d, 0, dbg);
+        }
+    }
+    if (use_tc<T>() && dF.rows >= rows && dFused.rows >= rows && gate.rows >= rows) {
+        TcFuse fz{};
+        fz.add_a = reinterpret_cast<const __nv_bfloat16 *>(dFused.p);
+        fz.ld_add_a = dFused.ld;
+        fz.add_b = reinterpret_cast<const __nv_bfloat16 *>(gate.p);
+        fz.ld_add_b = gate.ld;
+        if (tc_linear(reinterpret_cast<const __nv_bfloat16 *>(dpre), rows, d, reinterpret_cast<const __nv_bfloat16 *>(Wg), d, nullptr, 0,
+                      nullptr, 0, reinterpret_cast<__nv_bfloat16 *>(dF.p), dF.ld, meta, status, st, true, &fz))
+            return;
+    }
+    linear_backward_input<T>(dpre, rows, d, Wg, d, nullptr, tprod, wt, meta, status, st);
+    note_launch();
+    gate_dF_kernel<T><<<cells_grid(n_rows > 0 ? n_rows : 1, d), 256, 0, st>>>(tprod, dFused.p, dFused.ld, gate.p, gate.ld, d, n_rows,
+                                                                            dF.p, dF.ld);
+}
+
 // ------------------------------------------------------------------------------------------ plan
 int32_t make_plan(const e2egrec_csr *graph, const e2egrec_mat *X, int32_t n_pairs, int32_t dense_dim, int32_t n_hops,
-                  const int32_t *fanouts, const e2egrec_mat *W_gnn, const e2egrec_mat *W_tower, JointPlan &jp)
+                  const int32_t *fanouts, const e2egrec_mat *W_gnn, const e2egrec_mat *W_tower, uint32_t flags, JointPlan &jp)
 {
     if (!graph || !X || !fanouts || !W_gnn || !W_tower) return E2EGREC_ERR_NULL;
     if (n_pairs < 1 || n_pairs > (1 << 28) || dense_dim < 0) return E2EGREC_ERR_ARG;
@@ -250,6 +383,13 @@ int32_t make_plan(const e2egrec_csr *graph, const e2egrec_mat *X, int32_t n_pair
         return E2EGREC_ERR_ARG;
     for (int k = 0; k < 3; ++k)
         if (W_tower[k].ld != W_tower[k].dim) return E2EGREC_ERR_ARG;
+    jp.gated = (flags & E2EGREC_JOINT_GATE) ? 1 : 0;
+    if (jp.gated) {
+        const e2egrec_mat &wg = W_tower[3];
+        if (!wg.data) return E2EGREC_ERR_NULL;
+        if (wg.dtype != X->dtype) return E2EGREC_ERR_DTYPE;
+        if (wg.rows != jp.zdim || wg.dim != jp.zdim || wg.ld != jp.zdim) return E2EGREC_ERR_ARG;
+    }
     if (jp.zdim % jp.unit || jp.dL % jp.unit || jp.h1 % jp.unit || jp.h2 % jp.unit) return E2EGREC_ERR_ALIGN;
 
     int64_t md = 0, ms = 0, me = 0;
@@ -303,8 +443,15 @@ int32_t make_plan(const e2egrec_csr *graph, const e2egrec_mat *X, int32_t n_pair
     jp.dz2_off = take(rp * jp.h2 * jp.es);
     jp.dz1_off = take(rp * jp.h1 * jp.es);
     jp.dz_off = take(rp * jp.zdim * jp.es);
-    jp.wt_off = take((size_t)std::max(jp.h1 * jp.zdim, jp.h2 * jp.h1) * jp.es);
-    jp.part_off = take((size_t)kSplits * std::max(jp.h1 * jp.zdim, jp.h2 * jp.h1) * sizeof(float));
+    const size_t w_max = (size_t)std::max(std::max(jp.h1 * jp.zdim, jp.h2 * jp.h1), jp.gated ? jp.zdim * jp.zdim : 0);
+    jp.wt_off = take(w_max * jp.es);
+    jp.part_off = take((size_t)kSplits * w_max * sizeof(float));
+    if (jp.gated) {
+        jp.zf_off = take(rp * jp.zdim * jp.es);
+        jp.gate_off = take(rp * jp.zdim * jp.es);
+        jp.dzf_off = take(rp * jp.zdim * jp.es);
+        jp.gpre_off = take(rp * jp.zdim * jp.es);
+    }
     jp.bytes = off;
     return E2EGREC_OK;
 }
@@ -315,8 +462,11 @@ int32_t run_joint(const JointPlan &jp, const e2egrec_csr *graph, const e2egrec_m
                   const e2egrec_mat *W_gnn, const e2egrec_mat *W_tower, const float *const *b_tower, uint64_t seed,
                   uint32_t step, float *loss, float *logits, float *const *dW_gnn, float *const *dW_tower,
                   float *const *db_tower, const e2egrec_mat *dX_rows, int32_t *dX_ids, int32_t *n_dX_rows, char *ws,
-                  uint32_t phase, cudaStream_t st)
+                  uint32_t phase, uint32_t flags, cudaStream_t st)
 {
+    const int relu = (flags & E2EGREC_JOINT_LINEAR) ? 0 : 1;
+    int32_t acts[kMaxHops];
+    for (int l = 0; l < kMaxHops; ++l) acts[l] = relu;
     e2egrec_block blocks[kMaxHops];
     fill_blocks(jp, ws, blocks);
     auto i32 = [&](size_t off) { return reinterpret_cast<int32_t *>(ws + off); };
@@ -354,7 +504,7 @@ int32_t run_joint(const JointPlan &jp, const e2egrec_csr *graph, const e2egrec_m
     // 2. encoder forward: embeddings of the seeds
     e2egrec_mat Hs{tp(jp.hseed_off), pad128(jp.cd[0]), jp.dL, jp.dL, X->dtype};
     size_t ctx_bytes = jp.ctx_bytes;
-    rc = e2egrec_sage_forward(blocks, jp.n_hops, X, W_gnn, nullptr, nullptr, ws + jp.ctx_off, &ctx_bytes, &Hs, st);
+    rc = e2egrec_sage_forward(blocks, jp.n_hops, X, W_gnn, nullptr, acts, ws + jp.ctx_off, &ctx_bytes, &Hs, st);
     if (rc != E2EGREC_OK) return rc;
 
     // 3. tower forward and loss
@@ -370,8 +520,19 @@ int32_t run_joint(const JointPlan &jp, const e2egrec_csr *graph, const e2egrec_m
         build_z_kernel<T><<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(tp(jp.hseed_off), jp.dL, pi.pair_local, dense, jp.dense_dim,
                                                                      jp.P, jp.rowsP, z);
     }
-    linear_forward<T>(z, jp.rowsP, jp.zdim, W1, jp.h1, b1, 1, a1, pmeta, status, st);
-    linear_forward<T>(a1, jp.rowsP, jp.h1, W2, jp.h2, b2, 1, a2, pmeta, status, st);
+    // gating fusion (Sec. 4.3.2): the tower reads z_fused = sigmoid(W_g z + b_g) * z instead of z
+    const T *tin = z;
+    T *gate = nullptr;
+    if (jp.gated) {
+        T *zf = tp(jp.zf_off);
+        gate = tp(jp.gate_off);
+        gate_forward_core<T>(GMat<const T>{z, jp.zdim, jp.rowsP}, jp.rowsP, jp.P, jp.zdim, static_cast<const T *>(W_tower[3].data),
+                             b_tower ? b_tower[3] : nullptr, tp(jp.gpre_off), GMat<T>{gate, jp.zdim, jp.rowsP},
+                             GMat<T>{zf, jp.zdim, jp.rowsP}, pmeta, status, st);
+        tin = zf;
+    }
+    linear_forward<T>(tin, jp.rowsP, jp.zdim, W1, jp.h1, b1, relu, a1, pmeta, status, st);
+    linear_forward<T>(a1, jp.rowsP, jp.h1, W2, jp.h2, b2, relu, a2, pmeta, status, st);
     note_launch();
     logit_kernel<T><<<(unsigned)ceil_div((int64_t)jp.P * 32, 256), 256, 0, st>>>(a2, jp.h2, W3, b3, jp.P, logits);
     note_launch();
@@ -385,7 +546,7 @@ int32_t run_joint(const JointPlan &jp, const e2egrec_csr *graph, const e2egrec_m
     {
         const int64_t n = jp.rowsP * jp.h2;
         note_launch();
-        dz_top_kernel<T><<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(dt, W3, a2, jp.h2, jp.P, jp.rowsP, dz2);
+        dz_top_kernel<T><<<(unsigned)ceil_div(n, 256), 256, 0, st>>>(dt, W3, a2, jp.h2, jp.P, jp.rowsP, relu, dz2);
     }
     // the weight gradients feed nothing later in the step: they go to the helper stream (behind the block
     // transposition that the sampler left there); the encoder backward waits for that stream before its first launch
@@ -396,11 +557,23 @@ int32_t run_joint(const JointPlan &jp, const e2egrec_csr *graph, const e2egrec_m
         ws_st = side->stream;
     }
     linear_backward_weight<T>(dz2, jp.rowsP, jp.h2, a1, jp.h1, pmeta, part, dW_tower[1], db_tower ? db_tower[1] : nullptr, status, ws_st);
-    linear_backward_input<T>(dz2, jp.rowsP, jp.h2, W2, jp.h1, a1, dz1, wt, pmeta, status, st);
+    linear_backward_input<T>(dz2, jp.rowsP, jp.h2, W2, jp.h1, relu ? a1 : nullptr, dz1, wt, pmeta, status, st);
     if (side) side->fork(st);
-    linear_backward_weight<T>(dz1, jp.rowsP, jp.h1, z, jp.zdim, pmeta, part, dW_tower[0], db_tower ? db_tower[0] : nullptr, status, ws_st);
+    linear_backward_weight<T>(dz1, jp.rowsP, jp.h1, tin, jp.zdim, pmeta, part, dW_tower[0], db_tower ? db_tower[0] : nullptr, status, ws_st);
     if (side) side->defer();
-    linear_backward_input<T>(dz1, jp.rowsP, jp.h1, W1, jp.zdim, nullptr, dz, wt, pmeta, status, st);
+    if (!jp.gated) {
+        linear_backward_input<T>(dz1, jp.rowsP, jp.h1, W1, jp.zdim, nullptr, dz, wt, pmeta, status, st);
+    } else {
+        // through the gate: dz = dz_fused * g + (dz_fused * z * g (1 - g)) W_g, and the gate's own gradients.  The weight
+        // gradient above still uses `part` on the helper stream, so the caller's stream waits for it first.
+        T *dzf = tp(jp.dzf_off);
+        linear_backward_input<T>(dz1, jp.rowsP, jp.h1, W1, jp.zdim, nullptr, dzf, wt, pmeta, status, st);
+        if (side) side->join(st);
+        gate_backward_core<T>(GMat<const T>{dzf, jp.zdim, jp.rowsP}, GMat<const T>{z, jp.zdim, jp.rowsP},
+                              GMat<const T>{gate, jp.zdim, jp.rowsP}, jp.rowsP, jp.P, jp.zdim, static_cast<const T *>(W_tower[3].data),
+                              tp(jp.gpre_off), tp(jp.zf_off), wt, part, GMat<T>{dz, jp.zdim, jp.rowsP}, dW_tower[3],
+                              db_tower ? db_tower[3] : nullptr, pmeta, status, st);
+    }
 
     // 5. gradient of every seed embedding: the rows of dz that belong to it, added in pair order
     {
@@ -408,14 +581,17 @@ int32_t run_joint(const JointPlan &jp, const e2egrec_csr *graph, const e2egrec_m
         o.out = tp(jp.dhseed_off);
         o.ld_out = jp.dL;
         const SegScratch sc = seg_scratch_carve(jp.P2, kPairRun, jp.dL, dtype_size(X->dtype), ws + jp.seg_off);
-        dispatch_seg_reduce<T, int32_t, false>(dz, jp.unit, pi.pcsc_ptr, pi.pcsc_idx, &pcounts[CNT_SRC], 0, jp.P2, nullptr,
-                                               kPairRun, jp.dL, X->dtype, pi.pcsc_col, sc, o, st);
+        if (!dispatch_seg_reduce<T, int32_t, false>(dz, jp.unit, pi.pcsc_ptr, pi.pcsc_idx, &pcounts[CNT_SRC], 0, jp.P2, nullptr,
+                                                    kPairRun, jp.dL, X->dtype, pi.pcsc_col, sc, o, st)) {
+            set_last_error("joint_step: no reduction kernel for this embedding width");
+            return E2EGREC_ERR_UNSUPPORTED;
+        }
     }
 
     // 6. encoder backward
     e2egrec_mat dHs{tp(jp.dhseed_off), pad128(jp.cd[0]), jp.dL, jp.dL, X->dtype};
     size_t bwd_bytes = jp.bwd_bytes;
-    rc = e2egrec_sage_backward(blocks, jp.n_hops, X, W_gnn, nullptr, ws + jp.ctx_off, &dHs, dW_gnn, nullptr, dX_rows,
+    rc = e2egrec_sage_backward(blocks, jp.n_hops, X, W_gnn, acts, ws + jp.ctx_off, &dHs, dW_gnn, nullptr, dX_rows,
                                ws + jp.bwd_off, &bwd_bytes, 0, st);
     if (rc != E2EGREC_OK) return rc;
     const e2egrec_block &outer = blocks[jp.n_hops - 1];
@@ -453,9 +629,11 @@ extern "C" int32_t e2egrec_joint_step_phase(const e2egrec_csr *graph, const e2eg
                                             int32_t *n_dX_rows, void *ws, size_t *ws_bytes, uint32_t phase, void *stream)
 {
     if (!ws_bytes) return E2EGREC_ERR_NULL;
-    if (phase > E2EGREC_JOINT_COMPUTE) return E2EGREC_ERR_ARG;
+    const uint32_t flags = phase & ~0xFFu;
+    phase &= 0xFFu;
+    if (phase > E2EGREC_JOINT_COMPUTE || (flags & ~(E2EGREC_JOINT_LINEAR | E2EGREC_JOINT_GATE))) return E2EGREC_ERR_ARG;
     JointPlan jp{};
-    int32_t rc = make_plan(graph, X, n_pairs, dense_dim, n_hops, fanouts, W_gnn, W_tower, jp);
+    int32_t rc = make_plan(graph, X, n_pairs, dense_dim, n_hops, fanouts, W_gnn, W_tower, flags, jp);
     if (rc != E2EGREC_OK) return rc;
     if (!ws) { *ws_bytes = jp.bytes; return E2EGREC_OK; }
     if (*ws_bytes < jp.bytes) { *ws_bytes = jp.bytes; return E2EGREC_ERR_WORKSPACE; }
@@ -465,74 +643,45 @@ extern "C" int32_t e2egrec_joint_step_phase(const e2egrec_csr *graph, const e2eg
         return E2EGREC_ERR_NULL;
     for (int l = 0; l < n_hops; ++l)
         if (!dW_gnn[l]) return E2EGREC_ERR_NULL;
-    for (int k = 0; k < 3; ++k)
+    for (int k = 0; k < 3 + jp.gated; ++k)
         if (!dW_tower[k]) return E2EGREC_ERR_NULL;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (X->dtype == E2EGREC_BF16)
         return run_joint<__nv_bfloat16>(jp, graph, X, pair_user, pair_item, dense, labels, fanouts, W_gnn, W_tower, b_tower, seed,
                                         step, loss, logits, dW_gnn, dW_tower, db_tower, dX_rows, dX_ids, n_dX_rows,
-                                        static_cast<char *>(ws), phase, st);
+                                        static_cast<char *>(ws), phase, flags, st);
     return run_joint<float>(jp, graph, X, pair_user, pair_item, dense, labels, fanouts, W_gnn, W_tower, b_tower, seed, step, loss,
-                            logits, dW_gnn, dW_tower, db_tower, dX_rows, dX_ids, n_dX_rows, static_cast<char *>(ws), phase, st);
+                            logits, dW_gnn, dW_tower, db_tower, dX_rows, dX_ids, n_dX_rows, static_cast<char *>(ws), phase, flags,
+                            st);
 }
 
-// ------------------------------------------------------------------------------------------ gated fusion (Sec. 4.3.1)
-//   g = sigmoid(F Wg^T + bg),  F_fused = g * F.  The product runs on the dense helpers above (tcgen05 for bf16 shapes
-//   they take, fp32 FMA otherwise); the gate itself and its derivative are element-wise kernels.
+extern "C" int32_t e2egrec_joint_step_layout(const e2egrec_csr *graph, const e2egrec_mat *X, int32_t n_pairs, int32_t dense_dim,
+                                             int32_t n_hops, const int32_t *fanouts, const e2egrec_mat *W_gnn,
+                                             const e2egrec_mat *W_tower, uint32_t flags, size_t *tower_offset,
+                                             size_t *enc_h_offset, int64_t *enc_rows, int64_t *pair_rows)
+{
+    if (!tower_offset || !enc_h_offset || !enc_rows || !pair_rows) return E2EGREC_ERR_NULL;
+    if (flags & ~(E2EGREC_JOINT_LINEAR | E2EGREC_JOINT_GATE)) return E2EGREC_ERR_ARG;
+    JointPlan jp{};
+    int32_t rc = make_plan(graph, X, n_pairs, dense_dim, n_hops, fanouts, W_gnn, W_tower, flags, jp);
+    if (rc != E2EGREC_OK) return rc;
+    e2egrec_block blocks[kMaxHops];
+    fill_blocks(jp, nullptr, blocks);
+    size_t cat_off[kMaxHops], h_off[kMaxHops];
+    rc = e2egrec_sage_ctx_layout(blocks, n_hops, X, W_gnn, cat_off, h_off, enc_rows);
+    if (rc != E2EGREC_OK) return rc;
+    for (int l = 0; l < n_hops; ++l) enc_h_offset[l] = jp.ctx_off + h_off[l];
+    tower_offset[0] = jp.z_off;
+    tower_offset[1] = jp.a1_off;
+    tower_offset[2] = jp.a2_off;
+    tower_offset[3] = jp.gated ? jp.gate_off : jp.z_off;
+    tower_offset[4] = jp.gated ? jp.zf_off : jp.z_off;
+    *pair_rows = jp.rowsP;
+    return E2EGREC_OK;
+}
+
 namespace e2egrec {
 namespace {
-
-__global__ void gate_meta_kernel(int32_t *meta, int32_t n_rows) { meta[0] = n_rows; }
-
-// gate = sigmoid(pre), fused = gate * F for rows < n_rows; zero rows up to rows_alloc
-template <typename T>
-__global__ void gate_apply_kernel(const T *__restrict__ pre, const T *__restrict__ F, int64_t ldf, int d, int32_t n_rows,
-                                  int64_t rows_alloc, T *__restrict__ gate, int64_t ldg, T *__restrict__ fused, int64_t ldo)
-{
-    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int64_t i = t / d;
-    const int k = (int)(t - i * d);
-    if (i >= rows_alloc) return;
-    float g = 0.f, o = 0.f;
-    if (i < n_rows) {
-        const float p = to_float<T>(pre[i * d + k]);
-        const float e = expf(-fabsf(p));
-        g = to_float<T>(from_float<T>(p >= 0.f ? 1.0f / (1.0f + e) : e / (1.0f + e)));      // the stored gate
-        o = g * to_float<T>(F[i * ldf + k]);
-    }
-    gate[i * ldg + k] = from_float<T>(g);
-    fused[i * ldo + k] = from_float<T>(o);
-}
-
-// dpre = dFused * F * g (1 - g) for rows < n_rows, zero rows up to rows_alloc
-template <typename T>
-__global__ void gate_dpre_kernel(const T *__restrict__ dFused, int64_t ldd, const T *__restrict__ F, int64_t ldf,
-                                 const T *__restrict__ gate, int64_t ldg, int d, int32_t n_rows, int64_t rows_alloc,
-                                 T *__restrict__ dpre)
-{
-    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int64_t i = t / d;
-    const int k = (int)(t - i * d);
-    if (i >= rows_alloc) return;
-    float v = 0.f;
-    if (i < n_rows) {
-        const float g = to_float<T>(gate[i * ldg + k]);
-        v = to_float<T>(dFused[i * ldd + k]) * to_float<T>(F[i * ldf + k]) * g * (1.0f - g);
-    }
-    dpre[i * d + k] = from_float<T>(v);
-}
-
-// dF = t + dFused * g for rows < n_rows
-template <typename T>
-__global__ void gate_dF_kernel(const T *__restrict__ tprod, const T *__restrict__ dFused, int64_t ldd,
-                               const T *__restrict__ gate, int64_t ldg, int d, int32_t n_rows, T *__restrict__ dF, int64_t ldo)
-{
-    const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    const int64_t i = t / d;
-    const int k = (int)(t - i * d);
-    if (i >= n_rows) return;
-    dF[i * ldo + k] = from_float<T>(to_float<T>(tprod[i * d + k]) + to_float<T>(dFused[i * ldd + k]) * to_float<T>(gate[i * ldg + k]));
-}
 
 struct GatePlan {
     int d;
@@ -562,39 +711,19 @@ int32_t gate_plan(const e2egrec_mat *F, int32_t n_rows, const e2egrec_mat *Wg, G
     return E2EGREC_OK;
 }
 
-unsigned cells_grid(int64_t rows, int d) { return (unsigned)std::max<int64_t>(1, ceil_div(rows * d, 256)); }
-
-}  // namespace
-}  // namespace e2egrec
-
-namespace e2egrec {
-namespace {
+template <typename T> GMat<const T> cmat(const e2egrec_mat *m) { return GMat<const T>{static_cast<const T *>(m->data), m->ld, m->rows}; }
+template <typename T> GMat<T> wmat(const e2egrec_mat *m) { return GMat<T>{static_cast<T *>(m->data), m->ld, m->rows}; }
 
 template <typename T>
 int32_t gate_forward_impl(const GatePlan &gp, const e2egrec_mat *F, int32_t n_rows, const e2egrec_mat *Wg, const float *bg,
                           const e2egrec_mat *gate, const e2egrec_mat *fused, char *ws, cudaStream_t st)
 {
     int32_t *meta = reinterpret_cast<int32_t *>(ws + gp.meta_off);      // {rows, status}
-    T *pre = reinterpret_cast<T *>(ws + gp.a_off);
     note_launch();
     gate_meta_kernel<<<1, 1, 0, st>>>(meta, n_rows);
     cudaMemsetAsync(meta + 1, 0, sizeof(int32_t), st);
-    const bool dense_f = F->ld == F->dim;                               // the tensor-core path takes a dense operand
-    if (dense_f) {
-        linear_forward<T>(static_cast<const T *>(F->data), gp.rows, gp.d, static_cast<const T *>(Wg->data), gp.d, bg, 0, pre, meta,
-                          meta + 1, st);
-    } else {
-        EpiUpdate<T> epi{pre, gp.d, bg, 0};
-        dim3 grid((unsigned)ceil_div(gp.rows, kGemmBM), (unsigned)ceil_div(gp.d, kGemmBN), 1);
-        note_launch();
-        gemm_simt_kernel<T, false, false, EpiUpdate<T>><<<grid, kGemmThreads, 0, st>>>(
-            static_cast<const T *>(F->data), F->ld, static_cast<const T *>(Wg->data), gp.d, gp.rows, gp.d, gp.d, meta, nullptr, epi);
-    }
-    note_launch();
-    gate_apply_kernel<T><<<cells_grid(gp.rows, gp.d), 256, 0, st>>>(pre, static_cast<const T *>(F->data), F->ld, gp.d, n_rows,
-                                                                  std::min<int64_t>(gp.rows, std::min(gate->rows, fused->rows)),
-                                                                  static_cast<T *>(gate->data), gate->ld,
-                                                                  static_cast<T *>(fused->data), fused->ld);
+    gate_forward_core<T>(cmat<T>(F), gp.rows, n_rows, gp.d, static_cast<const T *>(Wg->data), bg,
+                         reinterpret_cast<T *>(ws + gp.a_off), wmat<T>(gate), wmat<T>(fused), meta, meta + 1, st);
     return check_launch("gate_fusion_forward");
 }
 
@@ -604,39 +733,13 @@ int32_t gate_backward_impl(const GatePlan &gp, const e2egrec_mat *dFused, const 
                            char *ws, cudaStream_t st)
 {
     int32_t *meta = reinterpret_cast<int32_t *>(ws + gp.meta_off);
-    T *dpre = reinterpret_cast<T *>(ws + gp.a_off), *tprod = reinterpret_cast<T *>(ws + gp.b_off);
-    T *wt = reinterpret_cast<T *>(ws + gp.wt_off);
-    float *part = reinterpret_cast<float *>(ws + gp.part_off);
     note_launch();
     gate_meta_kernel<<<1, 1, 0, st>>>(meta, n_rows);
     cudaMemsetAsync(meta + 1, 0, sizeof(int32_t), st);
-    note_launch();
-    gate_dpre_kernel<T><<<cells_grid(gp.rows, gp.d), 256, 0, st>>>(static_cast<const T *>(dFused->data), dFused->ld,
-                                                                 static_cast<const T *>(F->data), F->ld,
-                                                                 static_cast<const T *>(gate->data), gate->ld, gp.d, n_rows,
-                                                                 gp.rows, dpre);
-    if (F->ld == F->dim) {
-        linear_backward_weight<T>(dpre, gp.rows, gp.d, static_cast<const T *>(F->data), gp.d, meta, part, dWg, dbg, meta + 1, st);
-    } else {                                                             // strided F: fp32-FMA product
-        EpiPartial epi{part, gp.d, (int64_t)gp.d * gp.d};
-        dim3 grid((unsigned)ceil_div(gp.d, kGemmBM), (unsigned)ceil_div(gp.d, kGemmBN), kSplits);
-        note_launch();
-        gemm_simt_kernel<T, true, true, EpiPartial><<<grid, kGemmThreads, 0, st>>>(dpre, gp.d, static_cast<const T *>(F->data),
-                                                                                  F->ld, gp.d, gp.d, gp.rows, nullptr, meta, epi);
-        note_launch();
-        splitk_reduce_kernel<<<(unsigned)ceil_div((int64_t)gp.d * gp.d, 256), 256, 0, st>>>(part, (int64_t)gp.d * gp.d, kSplits, 0,
-                                                                                         dWg, nullptr);
-        if (dbg) {
-            note_launch();
-            colsum_kernel<T><<<(unsigned)ceil_div(gp.d, 32), 256, 0, st>>>(dpre, gp.d, meta, gp.d, 0, dbg);
-        }
-    }
-    linear_backward_input<T>(dpre, gp.rows, gp.d, static_cast<const T *>(Wg->data), gp.d, nullptr, tprod, wt, meta, meta + 1, st);
-    note_launch();
-    gate_dF_kernel<T><<<cells_grid(n_rows > 0 ? n_rows : 1, gp.d), 256, 0, st>>>(tprod, static_cast<const T *>(dFused->data),
-                                                                               dFused->ld, static_cast<const T *>(gate->data),
-                                                                               gate->ld, gp.d, n_rows, static_cast<T *>(dF->data),
-                                                                               dF->ld);
+    gate_backward_core<T>(cmat<T>(dFused), cmat<T>(F), cmat<T>(gate), gp.rows, n_rows, gp.d, static_cast<const T *>(Wg->data),
+                          reinterpret_cast<T *>(ws + gp.a_off), reinterpret_cast<T *>(ws + gp.b_off),
+                          reinterpret_cast<T *>(ws + gp.wt_off), reinterpret_cast<float *>(ws + gp.part_off), wmat<T>(dF), dWg, dbg,
+                          meta, meta + 1, st);
     return check_launch("gate_fusion_backward");
 }
 

@@ -1,4 +1,4 @@
-// The self-supervised task of the GNN and the balancing of the two task weights (Sec. 4.2):
+// The self-supervised task of the GNN and the balancing of the two task weights (SSL task: Sec. 4.2; GradNorm: Sec. 4.3.1):
 //   L_ssl = || X_seeds - H ||_F^2   (graph feature auto-encoder with the identity decoder),
 //   G_i   = || grad of (w_i L_i) with respect to the shared input rows ||_2,
 //   GradNorm step for the weights w_i.

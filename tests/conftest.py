@@ -24,3 +24,26 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+def pytest_terminal_summary(terminalreporter):
+    """How much of every compared tensor needed more than the plain tolerance (tests/helpers.py: AUDIT)."""
+    try:
+        import helpers
+    except Exception:
+        return
+    rows = helpers.AUDIT
+    if not rows:
+        return
+    import json
+    terminalreporter.write_line("parity audit: elements outside the plain tolerance (before the terms-scale and outlier allowances)")
+    for r in rows:
+        if r["outside_plain"]:
+            terminalreporter.write_line(f"  {r['test']} {r['tensor']} [{r['dtype']}]: {r['outside_plain']} of {r['elements']} "
+                                        f"({r['share']:.2e}), worst {r['worst_ratio']:.2f}x")
+    clean = sum(1 for r in rows if not r["outside_plain"])
+    terminalreporter.write_line(f"  {clean} of {len(rows)} compared tensors had every element inside the plain tolerance")
+    path = os.environ.get("E2EGREC_PARITY_AUDIT")
+    if path:
+        with open(path, "w") as f:
+            json.dump(rows, f, indent=1)

@@ -48,22 +48,22 @@ def tolerance(want, bf16, terms_rss=None):
     return tol
 
 
-def reduction_rss(case, ora):
-    """Root-sum-square of the terms of the last reduction behind every compared output, from oracle tensors:
-    forward output, dW per layer, dX rows."""
-    Ws, blocks, ctx, L = case.Ws, ora["blocks"], ora["ctx"], len(case.Ws)
-    acts = [1] * L if case.acts is None else case.acts
+def encoder_rss(Ws, acts, blocks, ctx, trace=None):
+    """Root-sum-square of the terms of the last reduction behind every compared output of the encoder, from oracle
+    tensors: forward output, and (given the trace of gradients that arrived at each layer) dW per layer, dX rows."""
+    L = len(Ws)
+    acts = [1] * L if acts is None else acts
     out = {}
     n0 = blocks[0]["n_dst"]
     cat_top = np.concatenate([ctx["H"][L - 1][:n0], ctx["agg"][L - 1]], axis=1)
     out["forward"] = np.sqrt((cat_top ** 2) @ (np.asarray(Ws[L - 1], np.float64) ** 2).T)
-    if "trace" not in ora:
+    if trace is None:
         return out
     out["dW"] = []
     for l in range(L):
         blk = blocks[L - 1 - l]
         n_dst = blk["n_dst"]
-        dZ = ora["trace"][l] * ((ctx["H"][l + 1] > 0) if acts[l] else 1.0)
+        dZ = trace[l] * ((ctx["H"][l + 1] > 0) if acts[l] else 1.0)
         cat = np.concatenate([ctx["H"][l][:n_dst], ctx["agg"][l]], axis=1)
         out["dW"].append(np.sqrt((dZ ** 2).T @ (cat ** 2)))
         if l == 0:
@@ -82,12 +82,51 @@ def reduction_rss(case, ora):
     return out
 
 
-def assert_close(name, got, want, bf16, terms_rss=None, budget=None):
+def reduction_rss(case, ora):
+    """encoder_rss for a Case and its oracle run."""
+    return encoder_rss(case.Ws, case.acts, ora["blocks"], ora["ctx"], ora.get("trace"))
+
+
+def plain_tolerance(want, bf16):
+    """The tolerance as first stated for the two paths, before any allowance: fp32 |a-b| <= 1e-5 max(|b|, rms(b));
+    bf16 storage |a-b| <= 1e-3 + 2e-2 |b|."""
+    want = np.asarray(want, np.float64)
+    if bf16:
+        return 1e-3 + 2e-2 * np.abs(want)
+    return 1e-5 * np.maximum(np.abs(want), np.sqrt(np.mean(want ** 2)) if want.size else 0.0)
+
+
+# One record per compared tensor: how many elements needed more than the plain tolerance (with the ReLU-flip budget
+# where the test has one, but without the terms-scale or the outlier allowance) and by how much.  conftest.py prints
+# the table at the end of the session and writes it to $E2EGREC_PARITY_AUDIT.
+AUDIT = []
+# ceilings on what may need the allowances at all: share of a tensor's elements (index: bf16?), and the worst ratio
+# error / plain tolerance.  Measured on B200: bf16 weight gradients (sums over thousands of rows whose operands the two
+# sides stored one bf16 step apart here and there) reach 1.1e-3 of their elements and 12x; everything fp32 stays below
+# 5e-6 of the elements and 5x.
+AUDIT_MAX_SHARE = {True: 2e-3, False: 1e-4}
+AUDIT_MAX_RATIO = {True: 16.0, False: 8.0}
+
+
+def _audit(name, err, plain, bf16, budget):
+    import os
+    over = err > plain
+    share = float(over.mean())
+    ratio = float((err[over] / plain[over]).max()) if over.any() else 0.0
+    AUDIT.append(dict(test=os.environ.get("PYTEST_CURRENT_TEST", "").split(" ")[0], tensor=name, dtype="bf16" if bf16 else "f32",
+                      elements=int(err.size), outside_plain=int(over.sum()), share=share, worst_ratio=ratio,
+                      flip_budget=budget is not None))
+    return share, ratio
+
+
+def assert_close(name, got, want, bf16, terms_rss=None, budget=None, audit_share=None):
     """Element-wise tolerance check with a report of the worst element.
 
     Every element within tolerance(); on the bf16 path at most 1e-4 of the elements may miss it by up
     to 4x (a stored operand one bf16 step apart two layers up, which the last reduction's terms do
-    not see).
+    not see).  Before either allowance is applied the elements outside plain_tolerance() are counted,
+    recorded (AUDIT) and held to a ceiling: a small share of the tensor, each within a fixed multiple
+    of the plain tolerance, so a widened tolerance cannot hide a wrong row or a mis-scaled column.
     """
     want = np.asarray(want, np.float64)
     got = np.asarray(got, np.float64)
@@ -96,15 +135,21 @@ def assert_close(name, got, want, bf16, terms_rss=None, budget=None):
         return
     assert np.isfinite(got).all(), f"{name}: non-finite values"
     tol = tolerance(want, bf16, terms_rss)
+    plain = plain_tolerance(want, bf16)
     if budget is not None:
         tol = tol + 1.05 * budget
+        plain = plain + 1.05 * budget
     err = np.abs(got - want)
+    share, ratio = _audit(name, err, plain, bf16, budget)
+    note = f"{name}: {share:.2e} of {err.size} elements outside the plain tolerance, worst {ratio:.2f}x"
+    assert share <= (audit_share or AUDIT_MAX_SHARE[bf16]) or (err > plain).sum() <= 2, note
+    assert ratio <= AUDIT_MAX_RATIO[bf16], note
     bad = err > tol
     if not bad.any():
         return
     i = np.unravel_index(np.argmax(err / np.maximum(tol, 1e-300)), err.shape)
     msg = (f"{name}: {bad.sum()} of {bad.size} outside tolerance; worst at {i}: got {got[i]!r} want {want[i]!r} "
-           f"err {err[i]:.3e} tol {tol[i]:.3e}")
+           f"err {err[i]:.3e} tol {tol[i]:.3e}; {note}")
     if bf16 and bad.sum() <= max(1, int(1e-4 * bad.size)) and (err <= 4 * tol).all():
         return
     raise AssertionError(msg)
@@ -177,8 +222,8 @@ class Case:
         return res
 
 
-def relu_flip_budgets(case, ora, gpu, tau):
-    """Upper bounds on how far the gradients may differ because the two sides took a ReLU decision
+def encoder_flip_budgets(Ws, acts, blocks, ctx, trace, gpu_layer_out, tau, B_dH0=None):
+    """Upper bounds on how far the encoder's gradients may differ because the two sides took a ReLU decision
     differently.
 
     The derivative of ReLU is decided by the sign of a sum that the GPU forms in fp32 and the oracle in
@@ -187,22 +232,22 @@ def relu_flip_budgets(case, ora, gpu, tau):
     (i, o) of layer l changes dZ_l[i, o] by at most |dH[i, o]|; that bound is pushed through the same
     linear adjoint with absolute-valued operands.  Flips are only accepted where the oracle's
     pre-activation is within tau of the kink; everything a flip cannot reach keeps the strict tolerance.
+    B_dH0: bound on the difference of the gradient that arrives at the encoder output (zero by default).
     Returns (budget_dW list, budget_dX).
     """
-    Ws, blocks, ctx = case.Ws, ora["blocks"], ora["ctx"]
     L = len(Ws)
-    acts = [1] * L if case.acts is None else case.acts
-    B_dH = np.zeros_like(ora["trace"][L - 1])
+    acts = [1] * L if acts is None else acts
+    B_dH = np.zeros_like(trace[L - 1]) if B_dH0 is None else np.asarray(B_dH0, np.float64)
     B_dW = [None] * L
     for l in range(L - 1, -1, -1):
         blk = blocks[L - 1 - l]
         n_dst, n_src = blk["n_dst"], blk["n_src"]
         flips = np.zeros(ctx["Z"][l].shape, bool)
         if acts[l]:
-            flips = (ctx["H"][l + 1] > 0) != (gpu["layer_out"][l][:n_dst] > 0)
+            flips = (ctx["H"][l + 1] > 0) != (gpu_layer_out[l][:n_dst] > 0)
             assert (np.abs(ctx["Z"][l][flips]) <= tau).all(), \
                 f"layer {l}: ReLU decision differs where the pre-activation is not near zero"
-        B_dZ = B_dH + np.abs(ora["trace"][l]) * flips
+        B_dZ = B_dH[:n_dst] + np.abs(trace[l]) * flips
         W = np.abs(np.asarray(Ws[l], np.float64))
         d_in = W.shape[1] // 2
         cat = np.abs(np.concatenate([ctx["H"][l][:n_dst], ctx["agg"][l]], axis=1))
@@ -216,6 +261,62 @@ def relu_flip_budgets(case, ora, gpu, tau):
             oracle._p(ip), oracle._p(blk["col"]), oracle.C.c_int64(n_dst), oracle.C.c_int64(n_src),
             oracle._p(B_dSelf), oracle._p(B_dAgg), oracle.C.c_int32(d_in), oracle._p(B_dH), oracle.C.c_int(0))
     return B_dW, B_dH
+
+
+def relu_flip_budgets(case, ora, gpu, tau):
+    """encoder_flip_budgets for a Case, its oracle run and the GPU's stored layer outputs."""
+    return encoder_flip_budgets(case.Ws, case.acts, ora["blocks"], ora["ctx"], ora["trace"], gpu["layer_out"], tau)
+
+
+def joint_rss_and_budgets(ora, W_gnn, W_tower, b_tower, gpu_act, tau, acts=1, gate=None):
+    """For a joint step (oracle result `ora` with its trace; gpu_act = the GPU's stored activations a1, a2 and encoder
+    layer outputs): per compared tensor the root-sum-square of the terms of its last reduction and the ReLU-flip
+    budget, pushed from the tower's two hidden layers through the pair -> seed sum into the encoder.
+    Returns (rss, budget): dicts with logits, dW_t, db_t (lists), dW_g (list), dX, and dW_gate / db_gate with a gate."""
+    tr = ora["trace"]
+    W1, W2, W3 = (np.asarray(W, np.float64) for W in W_tower[:3])
+    b1, b2 = (np.zeros(W.shape[0]) if b is None else np.asarray(b, np.float64) for W, b in zip((W1, W2), b_tower[:2]))
+    zf, a1, a2, z = tr["zf"], tr["a1"], tr["a2"], tr["z"]
+    P = zf.shape[0]
+    m2 = (a2 > 0) if acts else np.ones_like(a2, bool)
+    m1 = (a1 > 0) if acts else np.ones_like(a1, bool)
+    dz2, dz1 = tr["da2"] * m2, tr["da1"] * m1
+    # a logit sums 'a2 * W3' terms; a2 itself already carries the one-step deviations of a1 through its own sum, so the
+    # scale of a logit's terms takes the terms of a2's reduction along (where a2 is active)
+    rss_a2 = np.sqrt((a1 ** 2) @ (W2 ** 2).T) * m2
+    rss = dict(logits=np.sqrt((a2 ** 2 + rss_a2 ** 2) @ (W3 ** 2).T)[:, 0],
+               dW_t=[np.sqrt((dz1 ** 2).T @ (zf ** 2)), np.sqrt((dz2 ** 2).T @ (a1 ** 2)), np.sqrt((tr["dt"] ** 2)[None, :] @ (a2 ** 2))],
+               db_t=[np.sqrt((dz1 ** 2).sum(0)), np.sqrt((dz2 ** 2).sum(0)), np.sqrt((tr["dt"] ** 2).sum(keepdims=True))])
+    f2 = np.zeros_like(m2)
+    f1 = np.zeros_like(m1)
+    if acts:
+        f2 = m2 != (gpu_act["a2"][:P] > 0)
+        f1 = m1 != (gpu_act["a1"][:P] > 0)
+        assert (np.abs(a1 @ W2.T + b2)[f2] <= tau).all(), "tower layer 2: ReLU decision differs away from the kink"
+        assert (np.abs(zf @ W1.T + b1)[f1] <= tau).all(), "tower layer 1: ReLU decision differs away from the kink"
+    B_dz2 = np.abs(tr["da2"]) * f2
+    B_dz1 = B_dz2 @ np.abs(W2) + np.abs(tr["da1"]) * f1
+    B_dzf = B_dz1 @ np.abs(W1)
+    bud = dict(logits=None, dW_t=[B_dz1.T @ np.abs(zf), B_dz2.T @ np.abs(a1), np.zeros_like(W3)],
+               db_t=[B_dz1.sum(0), B_dz2.sum(0), np.zeros(1)])
+    B_dz = B_dzf
+    if gate is not None:
+        Wg = np.asarray(gate[0], np.float64)
+        g = tr["gate"]
+        dpre = tr["dzf"] * z * g * (1.0 - g)
+        rss["dW_gate"], rss["db_gate"] = np.sqrt((dpre ** 2).T @ (z ** 2)), np.sqrt((dpre ** 2).sum(0))
+        B_dpre = B_dzf * np.abs(z) * g * (1.0 - g)
+        bud["dW_gate"], bud["db_gate"] = B_dpre.T @ np.abs(z), B_dpre.sum(0)
+        B_dz = B_dzf * g + B_dpre @ np.abs(Wg)
+    dL = ora["H"].shape[1]
+    B_dH = np.zeros_like(ora["H"])
+    np.add.at(B_dH, tr["pos_u"], B_dz[:, :dL])
+    np.add.at(B_dH, tr["pos_i"], B_dz[:, dL:2 * dL])
+    enc_acts = [acts] * len(W_gnn)
+    enc = encoder_rss(W_gnn, enc_acts, ora["blocks"], tr["ctx"], tr["enc"])
+    rss["dW_g"], rss["dX"] = enc["dW"], enc["dX"]
+    bud["dW_g"], bud["dX"] = encoder_flip_budgets(W_gnn, enc_acts, ora["blocks"], tr["ctx"], tr["enc"], gpu_act["enc"], tau, B_dH)
+    return rss, bud
 
 
 def assert_close_budget(name, got, want, budget, bf16, terms_rss=None):

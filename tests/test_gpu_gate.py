@@ -1,4 +1,4 @@
-"""GPU parity of the gated fusion (Sec. 4.3.1) against the oracle."""
+"""GPU parity of the gated fusion (Sec. 4.3.2) against the oracle."""
 import numpy as np
 import pytest
 import torch

@@ -5,7 +5,7 @@ import torch
 
 import oracle
 import synth_inputs as S
-from helpers import assert_blocks_equal, assert_close, tolerance
+from helpers import assert_close, joint_rss_and_budgets
 
 pytestmark = pytest.mark.gpu
 
@@ -27,64 +27,99 @@ def _inputs(w, n_pairs, dense_dim, h1, h2, seed):
     return indptr, indices, X, W_gnn, pu, pi, dense, labels, W_t, b_t
 
 
-def _run_gpu(w, indptr, indices, X, W_gnn, pu, pi, dense, labels, W_t, b_t, step):
+def _gate(w, dense_dim, seed):
+    zdim = 2 * w.hidden + dense_dim
+    Wg = S.glorot_uniform(zdim, zdim, seed, 43)
+    bg = 0.1 * np.random.default_rng(seed + 1).standard_normal(zdim).astype(np.float32)
+    return (S.to_bf16_values(Wg) if w.dtype == "bf16" else Wg), bg
+
+
+def _run_gpu(w, indptr, indices, X, W_gnn, pu, pi, dense, labels, W_t, b_t, step, linear=False, gate=None):
     import paper_2511_20564_b200 as E
     dt = torch.bfloat16 if w.dtype == "bf16" else torch.float32
     cu = lambda a, t=None: torch.from_numpy(np.ascontiguousarray(a)).cuda().to(t) if t else torch.from_numpy(np.ascontiguousarray(a)).cuda()
     js = E.JointStep(cu(indptr), cu(indices), cu(X, dt), pu.size, dense.shape[1], w.fanouts, [cu(W, dt) for W in W_gnn],
-                     [cu(W, dt) for W in W_t], [cu(b) for b in b_t])
+                     [cu(W, dt) for W in W_t], [cu(b) for b in b_t], linear=linear,
+                     W_gate=None if gate is None else cu(gate[0], dt), b_gate=None if gate is None else cu(gate[1]))
     js.run(cu(pu), cu(pi), cu(dense), cu(labels), w.seed, step)
     torch.cuda.synchronize()
     return js
 
 
-@pytest.mark.parametrize("name,n_pairs,dense_dim,h1,h2", [("tiny", 96, 8, 48, 24), ("medium_small", 512, 64, 512, 256)])
-def test_joint_step_matches_oracle(name, n_pairs, dense_dim, h1, h2):
-    w = S.WORKLOADS[name]
+def _compare(w, args, step, linear=False, gate=None):
+    """One joint step on both sides; every output compared element by element.  Gradients carry the tolerance of their
+    last reduction (helpers.tolerance) and, with ReLU on, the budget of the sign decisions that the two sides took
+    differently (helpers.joint_rss_and_budgets); with identity activations there is no budget at all."""
     bf16 = w.dtype == "bf16"
-    args = _inputs(w, n_pairs, dense_dim, h1, h2, 7)
     indptr, indices, X, W_gnn, pu, pi, dense, labels, W_t, b_t = args
-    step = 3
-    ora = oracle.joint_step(indptr, indices, X, pu, pi, dense, labels, w.fanouts, W_gnn, W_t, b_t, w.seed, step, bf16=bf16)
-    js = _run_gpu(w, *args, step)
+    acts = 0 if linear else 1
+    L = len(W_gnn)
+    ora = oracle.joint_step(indptr, indices, X, pu, pi, dense, labels, w.fanouts, W_gnn, W_t, b_t, w.seed, step, bf16=bf16,
+                            acts_gnn=[acts] * L, acts_tower=(acts, acts), gate=gate)
+    js = _run_gpu(w, *args, step, linear=linear, gate=gate)
     n_rows, status = js.n_rows.tolist()
     assert status == 0
     # integer side: the sampled sub-graph of the distinct endpoints
     assert n_rows == ora["dX_ids"].size and np.array_equal(js.dX_ids[:n_rows].cpu().numpy(), ora["dX_ids"])
+    act = js.activations()
+    gpu_act = dict(a1=act["a1"].float().cpu().numpy(), a2=act["a2"].float().cpu().numpy(),
+                   enc=[h.float().cpu().numpy() for h in act["enc"]])
+    rss, bud = joint_rss_and_budgets(ora, W_gnn, W_t, b_t, gpu_act, 2e-2 if bf16 else 1e-5, acts=acts, gate=gate)
     # forward
-    logits = js.logits.cpu().numpy().astype(np.float64)
-    assert_close("logits", logits, ora["logits"], bf16, np.full(n_pairs, np.linalg.norm(W_t[2])) if bf16 else None)
+    # a logit is a 256-term sum over a2, whose elements the two sides store one bf16 step apart in a few percent of the
+    # cases (fp32 against float64 sums before the rounding): up to 3.4e-2 of the logits were measured outside the plain
+    # tolerance, none by more than 5x, all inside the tolerance scaled by the terms
+    assert_close("logits", js.logits.cpu().numpy(), ora["logits"], bf16, rss["logits"], audit_share=6e-2 if bf16 else None)
     assert abs(float(js.loss) - ora["loss"]) <= (2e-2 * abs(ora["loss"]) + 1e-3 if bf16 else 1e-5 * abs(ora["loss"]))
     # gradients
-    got = dict(dW_t=[g.cpu().numpy() for g in js.dW_tower], db_t=[g.cpu().numpy() for g in js.db_tower],
-               dW_g=[g.cpu().numpy() for g in js.dW_gnn], dX=js.dX_rows[:n_rows].float().cpu().numpy())
-    want = dict(dW_t=ora["dW_tower"], db_t=ora["db_tower"], dW_g=ora["dW_gnn"], dX=ora["dX"])
-    for key in ("dW_t", "db_t", "dW_g"):
-        for k, (g, o) in enumerate(zip(got[key], want[key])):
-            _check_grad(f"{key}[{k}]", g, o, bf16)
-    _check_grad("dX", got["dX"], want["dX"], bf16)
+    nt = 3
+    for k in range(nt):
+        assert_close(f"dW_tower[{k}]", js.dW_tower[k].cpu().numpy(), ora["dW_tower"][k], bf16, rss["dW_t"][k], bud["dW_t"][k])
+        assert_close(f"db_tower[{k}]", js.db_tower[k].cpu().numpy(), ora["db_tower"][k], bf16, rss["db_t"][k], bud["db_t"][k])
+    if gate is not None:
+        assert_close("dW_gate", js.dW_tower[3].cpu().numpy(), ora["dW_gate"], bf16, rss["dW_gate"], bud["dW_gate"])
+        assert_close("db_gate", js.db_tower[3].cpu().numpy(), ora["db_gate"], bf16, rss["db_gate"], bud["db_gate"])
+    for l in range(L):
+        assert_close(f"dW_gnn[{l}]", js.dW_gnn[l].cpu().numpy(), ora["dW_gnn"][l], bf16, rss["dW_g"][l], bud["dW_g"][l])
+    dX = js.dX_rows[:n_rows].float().cpu().numpy()
+    assert_close("dX", dX, ora["dX"], bf16, rss["dX"], bud["dX"])
+    if linear:                                              # no sign decisions: no allowance for them
+        assert all(float(np.max(b)) == 0.0 for b in bud["dW_t"] + bud["db_t"] + bud["dW_g"] + [bud["dX"]])
     # Theorem 1: the ranking loss reaches the encoder
-    assert all(np.abs(g).max() > 0 for g in got["dW_g"]) and np.abs(got["dX"]).max() > 0
+    assert all(np.abs(g.cpu().numpy()).max() > 0 for g in js.dW_gnn) and np.abs(dX).max() > 0
+    return ora, js
 
 
-def _check_grad(name, got, want, bf16):
-    """fp32: element-wise at 1e-5 (relative to the tensor's scale).  bf16: the masks of five ReLU layers are
-    decided from fp32 sums on one side and float64 sums on the other, and where they differ both gradients
-    are valid; the comparison is therefore norm-wise (3e-2) with 99% of the elements inside the element-wise
-    tolerance.  The same kernels are held to the element-wise tolerance by the linear-activation and budgeted
-    encoder tests."""
-    got, want = np.asarray(got, np.float64).reshape(np.shape(want)), np.asarray(want, np.float64)
-    assert np.isfinite(got).all(), name
-    scale = np.sqrt(np.mean(want ** 2))
-    if not bf16:
-        bad = np.abs(got - want) > 2e-5 * np.maximum(np.abs(want), scale)
-        assert not bad.any(), f"{name}: {bad.sum()} of {bad.size} outside 2e-5"
-        return
-    rel = np.linalg.norm(got - want) / max(np.linalg.norm(want), 1e-30)
-    assert rel <= 3e-2, f"{name}: relative Frobenius error {rel:.3e}"
-    tol = 1e-3 + 2e-2 * np.abs(want) + 2e-2 * scale
-    frac = np.mean(np.abs(got - want) <= tol)
-    assert frac >= 0.99, f"{name}: only {frac:.4f} of the elements within tolerance"
+@pytest.mark.parametrize("name,n_pairs,dense_dim,h1,h2", [("tiny", 96, 8, 48, 24), ("medium_small", 512, 64, 512, 256)])
+def test_joint_step_matches_oracle(name, n_pairs, dense_dim, h1, h2):
+    w = S.WORKLOADS[name]
+    _compare(w, _inputs(w, n_pairs, dense_dim, h1, h2, 7), step=3)
+
+
+@pytest.mark.parametrize("name,n_pairs,dense_dim,h1,h2", [("tiny", 96, 8, 48, 24), ("medium_small", 512, 64, 512, 256)])
+def test_joint_step_with_identity_activations_is_strict(name, n_pairs, dense_dim, h1, h2):
+    """E2EGREC_JOINT_LINEAR: no ReLU anywhere, so no gradient element gets a sign-decision allowance; the bf16 case
+    runs the same tensor-core products, segment reductions and pair -> seed sum as the default step."""
+    w = S.WORKLOADS[name]
+    _compare(w, _inputs(w, n_pairs, dense_dim, h1, h2, 8), step=1, linear=True)
+
+
+@pytest.mark.parametrize("name,n_pairs,dense_dim,h1,h2,linear", [("tiny", 96, 8, 48, 24, False),
+                                                                 ("medium_small", 512, 64, 512, 256, False),
+                                                                 ("medium_small", 384, 64, 256, 128, True)])
+def test_gated_joint_step_matches_oracle(name, n_pairs, dense_dim, h1, h2, linear):
+    """E2EGREC_JOINT_GATE (Sec. 4.3.2): z_fused = sigmoid(W_g z + b_g) * z feeds the tower; the gate's own gradients and
+    everything upstream of it are compared like the rest.  bf16: the gate runs in the epilogue of the W_g product."""
+    w = S.WORKLOADS[name]
+    _compare(w, _inputs(w, n_pairs, dense_dim, h1, h2, 9), step=2, linear=linear, gate=_gate(w, dense_dim, 9))
+
+
+def test_joint_step_at_benchmark_size():
+    """The joint step of the benchmark in full: 4 096 pairs on the 500 k-node / 20 M-entry graph, d = 128 bf16, fanout
+    (15, 10), tower 320-512-256-1, Bernoulli(0.1) labels; every output against the oracle."""
+    w = S.WORKLOADS["medium"]
+    ora, js = _compare(w, _inputs(w, 4096, 64, 512, 256, 4), step=0)
+    assert ora["blocks"][-1]["n_edges"] > 50_000 and ora["seeds"].size > 1_000
 
 
 def test_joint_step_in_two_phases_equals_the_whole_step():

@@ -1,4 +1,4 @@
-"""GPU parity of the SSL loss, the gradient norms and the GradNorm weight step (Sec. 4.2), and of the two-pass backward
+"""GPU parity of the SSL loss, the gradient norms and the GradNorm weight step (Sec. 4.2, Sec. 4.3.1), and of the two-pass backward
 that a step with two tasks runs."""
 import numpy as np
 import pytest

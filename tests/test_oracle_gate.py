@@ -1,4 +1,4 @@
-"""Pins for the oracle's gated fusion (Sec. 4.3.1, "Concatenation with Gating")."""
+"""Pins for the oracle's gated fusion (Sec. 4.3.2, "Concatenation with Gating")."""
 import numpy as np
 
 import oracle

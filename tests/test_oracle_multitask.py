@@ -1,4 +1,4 @@
-"""Pins for the oracle's SSL loss and GradNorm weight update (Sec. 4.2)."""
+"""Pins for the oracle's SSL loss and GradNorm weight update (Sec. 4.2, Sec. 4.3.1)."""
 import numpy as np
 
 import oracle

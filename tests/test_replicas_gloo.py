@@ -29,7 +29,7 @@ def _worker(rank, world, port, out):
 def test_two_ranks_reduce_to_slowest_time_and_total_work():
     world = 2
     port = 29500 + (os.getpid() % 1000)
-    with mp.Manager() as m:
+    with mp.get_context("spawn").Manager() as m:        # spawn: earlier tests may have started OpenMP threads here
         out = m.dict()
         mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
         for rank in range(world):
