@@ -3,12 +3,20 @@
 
 One step = k-hop sampling of one seed batch, the GraphSAGE forward over the sampled blocks and the
 full backward (weight gradients and feature-row gradients), through the library's C ABI.  Prints one
-JSON line (rank 0).  `--impl reference` times the CPU oracle instead (a deliberately plain program).
+JSON line (rank 0).
+
+Without --workload the line is the `large` workload (the largest configuration that fits one GPU) and
+carries, as sub-records, the `medium` workload, the joint step (encoder + ranking tower) on the medium
+graph and the whole-graph aggregation, each with its own roofline block.  With --workload only that
+workload runs.  `--impl reference` times the CPU oracle instead (a deliberately plain program).
 """
 from __future__ import annotations
 
 import argparse
+import gc
+import hashlib
 import json
+import math
 import os
 import statistics
 import subprocess
@@ -24,6 +32,8 @@ import synth_inputs as S  # noqa: E402
 
 METRIC = "sampled_gnn_sample_fwd_bwd_edges_per_sec"
 UNIT = "edges/s"
+NOMINAL_HBM_GBS = 8000.0            # the ~8 TB/s figure of the hardware's data sheet; fractions are given against it and the measured copy peak
+MIN_TIMED_S = 0.5                   # the K-step loop is repeated until the timed region is at least this long
 CLOCK_QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
                "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
                "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
@@ -35,6 +45,8 @@ TAP_NAMES = {1: "sage_aggregate_kernel (layer-0 mean aggregation, gathers X rows
              6: "e2egrec_sample_khop (all sampling kernels)",
              7: "seg_run_kernel (first transposed aggregation of the backward pass)",
              9: "seg_final_kernel (same)"}
+# source files whose kernels a recorded DRAM-traffic figure belongs to (the figure is dropped when they change)
+TRAFFIC_SOURCES = ("aggregate.cuh", "segreduce.cuh", "common.cuh")
 
 
 def measured_peaks():
@@ -42,8 +54,34 @@ def measured_peaks():
     if os.path.exists(p):
         d = json.load(open(p))
         return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d["bf16_tflops"]),
-                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])), source="measured")
-    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+                    bf16_tflops_sustained=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                    sm_max_mhz=float(d.get("sm_max_mhz", 1965.0)), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, sm_max_mhz=1965.0, source="fallback")
+
+
+def fp32_alu_peak_tflops(peaks):
+    """Plain fp32 FMA peak: 148 SMs x 128 fp32 lanes x 2 flop per FMA x the maximum SM clock (74.4 TFLOP/s at 1965 MHz)."""
+    return 148 * 128 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12
+
+
+def source_digest():
+    h = hashlib.sha256()
+    for name in TRAFFIC_SOURCES:
+        with open(os.path.join(ROOT, "paper_2511_20564_b200", "csrc", name), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic(key):
+    """DRAM bytes (read + write) per unit of work of one ncu capture, recorded in profiles/traffic.json beside the
+    summary it came from; None when there is no record or the kernel sources have changed since the capture."""
+    p = os.path.join(ROOT, "profiles", "traffic.json")
+    if not os.path.exists(p):
+        return None
+    rec = json.load(open(p)).get(key)
+    if not rec or rec.get("source_sha") != source_digest():
+        return None
+    return rec
 
 
 class ClockSampler:
@@ -62,6 +100,7 @@ class ClockSampler:
 
     def _nvml_handle(self):
         import pynvml
+        import torch
         pynvml.nvmlInit()
         try:
             uuid = str(torch.cuda.get_device_properties(self.gpu).uuid)
@@ -145,6 +184,10 @@ class ClockSampler:
                     reasons=reasons, samples=len(sm), source=source)
 
 
+def hbm_fractions(gbs, peaks):
+    return dict(gbs=gbs, frac_of_measured_copy=gbs / peaks["hbm_gbs"], frac_of_nominal_8tbs=gbs / NOMINAL_HBM_GBS)
+
+
 def build_inputs(w: S.Workload, host_csr=True):
     """Interactions, features and weights; the host CSR (numpy) is only built for the CPU oracle."""
     users, items = S.bipartite_interactions(w.n_users, w.n_items, w.n_interactions, w.alpha_user, w.alpha_item,
@@ -171,7 +214,13 @@ def upstream_grad(w, rows):
     return S.to_bf16_values(g) if w.dtype == "bf16" else g
 
 
-# ------------------------------------------------------------------------------------------ reference arm
+def on_device_workload(w):
+    """Graphs of 10^8 interactions and more are drawn with torch on the GPU that will hold them (the host arrays
+    alone would take minutes and tens of GB)."""
+    return w.n_interactions >= 100_000_000
+
+
+# ------------------------------------------------------------------------------------------ the CPU oracle, timed
 def oracle_step(w, indptr, indices, X, Ws, seeds, step, dH, edge_cum=None):
     """One oracle step.  X is the host feature table, or a callable ids -> rows (table kept elsewhere)."""
     import oracle
@@ -185,19 +234,46 @@ def oracle_step(w, indptr, indices, X, Ws, seeds, step, dH, edge_cum=None):
     return sum(b["n_edges"] for b in blocks)
 
 
+def time_oracle(step_fn, budget_s, max_steps, unit, describe):
+    """The oracle as it stands on all host cores (its row loops carry OpenMP pragmas) and on one: `step_fn(i)` runs
+    step i and returns the units of work it did.  Returns the cpu_baseline record (value = the all-core figure)."""
+    import oracle
+    out = {}
+    all_cores = oracle.max_threads()
+    for label, threads in (("all", all_cores), ("one", 1)):
+        oracle.set_threads(threads)
+        t0 = time.perf_counter()
+        work, n = 0, 0
+        while n < max_steps and (n == 0 or time.perf_counter() - t0 < budget_s):
+            work += step_fn(n)
+            n += 1
+        dt = time.perf_counter() - t0
+        out[label] = dict(value=work / dt, steps=n, seconds=dt)
+    oracle.set_threads(all_cores)
+    return dict(value=out["all"]["value"], unit=unit, cores=all_cores, kind="oracle",
+                sample=describe(out["all"]["steps"], out["all"]["seconds"]),
+                single_core=dict(value=out["one"]["value"], unit=unit, cores=1,
+                                 sample=describe(out["one"]["steps"], out["one"]["seconds"])),
+                host_cores=os.cpu_count())
+
+
+def reference_workload(w):
+    """The CPU arm runs the device-drawn workloads on a 1/100-scale graph of the same recipe."""
+    if not on_device_workload(w):
+        return w, ""
+    import dataclasses
+    small = dataclasses.replace(w, n_users=w.n_users // 100, n_items=w.n_items // 100,
+                                n_interactions=w.n_interactions // 100, q=w.q / 100)
+    return small, " on a 1/100-scale graph of the same recipe"
+
+
 def run_reference(args, w):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
-        return
+        return None
     import oracle
     oracle.build()
-    scale_note = ""
-    if w.n_interactions > 200_000_000:
-        # the full graph is drawn on a GPU; the CPU arm runs the same recipe at 1/100 of the size
-        import dataclasses
-        w = dataclasses.replace(w, n_users=w.n_users // 100, n_items=w.n_items // 100,
-                                n_interactions=w.n_interactions // 100, q=w.q / 100)
-        scale_note = " on a 1/100-scale graph of the same recipe"
+    w, scale_note = reference_workload(w)
     indptr, indices, X, Ws, inter = build_inputs(w)
     cum = None
     if args.beta is not None:
@@ -205,6 +281,7 @@ def run_reference(args, w):
     sample = args.ref_seeds
     dH = upstream_grad(w, sample).astype(np.float64)
     batches = make_batches(w, inter, args.seeds, 0, args.warmup + args.steps)[:, :sample]
+    cores = oracle.max_threads()
     for i in range(args.warmup):
         oracle_step(w, indptr, indices, X, Ws, batches[i], i, dH, cum)
     t0 = time.perf_counter()
@@ -214,20 +291,19 @@ def run_reference(args, w):
     dt = time.perf_counter() - t0
     val = edges / dt
     desc = f"first {sample} of the {w.batch} seeds of each step's batch, full sample+forward+backward{scale_note}"
-    line = dict(impl="reference", metric=METRIC, value=val, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
+    return dict(impl="reference", metric=METRIC, value=val, unit=UNIT, n_gpus=args.gpus, steps=args.steps,
                 warmup=args.warmup, ms_per_step=dt / args.steps * 1e3, higher_is_better=True, scaling="weak",
                 vs_baseline=None, dtype="f64", data="synthetic",
                 config=dict(workload=w.name, nodes=w.n_nodes, csr_entries=int(indptr[-1]), dim=w.dim, hidden=w.hidden,
                             layers=len(w.fanouts), fanouts=list(w.fanouts), batch=w.batch, seeds=args.seeds,
                             sample=desc),
-                cpu_baseline=dict(value=val, unit=UNIT, cores=1, kind="oracle", sample=desc),
+                cpu_baseline=dict(value=val, unit=UNIT, cores=cores, kind="oracle", sample=desc),
                 e2e=dict(value=val, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0),
                 gpu_launches=0)
-    print(json.dumps(line), flush=True)
 
 
 # ------------------------------------------------------------------------------------------ our arm
-def run_ours(args, w):
+def run_ours(args, w, with_joint):
     import torch
     import torch.distributed as dist
     import paper_2511_20564_b200 as E
@@ -237,8 +313,6 @@ def run_ours(args, w):
     local = int(os.environ.get("LOCAL_RANK", "0"))
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
-        dist.init_process_group("nccl", device_id=dev)
     E.lib()                                            # fails loudly if the CUDA library is missing
 
     want_cpu = world == 1 and not args.no_cpu_baseline
@@ -246,7 +320,7 @@ def run_ours(args, w):
     K, Wm = args.steps, args.warmup
     total = K + Wm + 4                                 # + the batches whose sampling / upload is prefetched during the last steps
     first_step = rank * 1_000_000                      # = replicas.first_step_of(rank)
-    on_device = w.n_interactions > 200_000_000         # too large for host-side generation: drawn with torch on the GPU
+    on_device = on_device_workload(w)
     t_setup = time.perf_counter()
     if on_device:
         users_d, items_d = S.bipartite_interactions_device(w.n_users, w.n_items, w.n_interactions, w.alpha_user,
@@ -311,8 +385,7 @@ def run_ours(args, w):
     H_out = H_out2[0]
     scratch = torch.empty(E.binding.sage_backward_scratch_bytes(blocks, X, Ws), dtype=torch.uint8, device=dev)
     dWs2 = [[torch.zeros(W.shape, dtype=torch.float32, device=dev) for W in Ws] for _ in range(NB)]
-    dWs = dWs2[0]
-    dX = torch.zeros(blocks.caps[L - 1][1], w.dim, dtype=dt, device=dev)
+    dX2 = [torch.zeros(blocks.caps[L - 1][1], w.dim, dtype=dt, device=dev) for _ in range(NB)]
 
     seeds_in2 = [torch.empty(w.batch, dtype=torch.int32, device=dev) for _ in range(NB)]
     dH_in2 = [torch.empty_like(dH) for _ in range(NB)]
@@ -327,22 +400,22 @@ def run_ours(args, w):
         E.blocks_transpose(blocks2[p])
 
     if args.multitask:
-        # the two-task step of Sec. 4.2 / 4.3.1: the recommendation gradient and the gradient of the SSL reconstruction loss go
-        # through the encoder one after the other (weight gradients accumulate), their norms at the shared input feed
-        # one GradNorm step of the task weights
+        # the two-task step of Sec. 4.2 / 4.3.1: the recommendation gradient and the gradient of the SSL reconstruction
+        # loss go through the encoder one after the other (weight gradients accumulate), their norms at the shared
+        # input feed one GradNorm step of the task weights
         if w.hidden != w.dim:
             raise SystemExit("--multitask needs hidden == dim (the identity decoder compares H with X)")
         f32 = dict(dtype=torch.float32, device=dev)
-        mt = dict(dX_ssl=torch.zeros_like(dX), dH_ssl=torch.zeros_like(H_out), one=torch.ones(1, **f32),
+        mt = dict(dX_ssl=torch.zeros_like(dX2[0]), dH_ssl=torch.zeros_like(H_out), one=torch.ones(1, **f32),
                   wts=torch.ones(2, **f32), L=torch.ones(2, **f32), L0=torch.ones(2, **f32), g=torch.zeros(2, **f32))
 
     def compute_leg(p):
         E.sage_forward(blocks2[p], X, Ws, ctx=ctx, H_out=H_out2[p])
-        E.sage_backward(blocks2[p], X, Ws, ctx, dH_in2[p], dWs=dWs2[p], dX_rows=dX, scratch=scratch)
+        E.sage_backward(blocks2[p], X, Ws, ctx, dH_in2[p], dWs=dWs2[p], dX_rows=dX2[p], scratch=scratch)
         if args.multitask:
             n_seeds_dev, n_rows_dev = blocks2[p].counts[0][0:1], blocks2[p].counts[L - 1][1:2]
             E.ssl_loss(H_out2[p], X, seeds_in2[p], n_seeds_dev, mt["one"], loss=mt["L"][0:1], dH=mt["dH_ssl"])
-            E.gradient_norm(dX, n_rows_dev, out=mt["g"][1:2])
+            E.gradient_norm(dX2[p], n_rows_dev, out=mt["g"][1:2])
             E.sage_backward(blocks2[p], X, Ws, ctx, mt["dH_ssl"], dWs=dWs2[p], dX_rows=mt["dX_ssl"], scratch=scratch,
                             accumulate=True)
             E.gradient_norm(mt["dX_ssl"], n_rows_dev, out=mt["g"][0:1])
@@ -443,57 +516,92 @@ def run_ours(args, w):
     # waits for SMs that those kernels hold
     dominant = max((k for k in tap_ms if k <= 5 and k != 4), key=lambda k: tap_ms[k])
 
-    count_total.zero_()
-    prime(Wm, seeds_dev)
+    # ---- the timed region: the K-step replay loop, repeated until the region is at least MIN_TIMED_S long.  Every
+    # repetition is bracketed by a barrier and a device synchronisation and timed with CUDA events; the reported step
+    # time is the median over the repetitions.
+    def timed_loop():
+        count_total.zero_()
+        prime(Wm, seeds_dev)
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(K):
+            replay_step(Wm + i, seeds_dev)
+        e1.record()
+        barrier()
+        c = count_total.cpu().numpy()
+        if c[:, 3].any():
+            raise RuntimeError(f"device status bits set during the timed region: {c[:, 3]}")
+        return e0.elapsed_time(e1), c
+
+    probe_ms, _ = timed_loop()                          # untimed repetition: sizes the number of repetitions
+    repeats = max(1, min(2000, math.ceil(MIN_TIMED_S * 1e3 / max(probe_ms, 1e-3))))
     clocks = ClockSampler(local)
     clocks.start()
     time.sleep(0.3)                                    # the sampler is polling before the region starts
     barrier()
     t_begin = clocks.mark()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(K):
-        replay_step(Wm + i, seeds_dev)
-    e1.record()
-    barrier()
+    reps = [timed_loop() for _ in range(repeats)]
     clk = clocks.stop(t_begin, clocks.mark())
-    ms = e0.elapsed_time(e1)
-    launches = K * (kernels_per_step + 2)               # + seed copy and step-offset kernel per step
-    counts = count_total.cpu().numpy()                  # [L, 4] summed over the K steps
-    if counts[:, 3].any():
-        raise RuntimeError(f"device status bits set during the timed region: {counts[:, 3]}")
+    rep_ms = [r[0] for r in reps]
+    ms = float(statistics.median(rep_ms))              # one repetition of K steps
+    counts = reps[0][1]                                 # [L, 4] summed over the K steps (the same batches in every repetition)
     edges_rank = int(counts[:, 2].sum())
+    launches = K * (kernels_per_step + 2)               # + seed copy and step-offset kernel per step
     # the dominant kernel again, timed inside eagerly launched steps over the same batches
-    dom_ms = []
-    for i in range(min(K, 50)):
-        dom_ms.append(tapped_step(Wm + i, dominant))
-    outer_counts = count_total.cpu().numpy()[L - 1] / (K + len(dom_ms))
+    count_total.zero_()
+    dom_ms = [tapped_step(Wm + i, dominant) for i in range(min(K, 50))]
+    outer_counts = count_total.cpu().numpy()[L - 1] / len(dom_ms)
+    max_rows = int(np.ceil(1.3 * outer_counts[1])) + 1024
 
     # ---- end to end: host buffers in, results out, every step.  Three streams: the step itself; the upload of the
     # next step's inputs (seeds of the batch sampled next, upstream gradient) while the step runs; the download of
-    # the step's results while the next step runs.  The host reads the results of step i while step i + 1 runs.
+    # the step's results while the next step runs: the embeddings, the weight gradients, the counts and -- with_dx --
+    # the gradient rows of the input features with their node ids (true count, read from the counts first).
     res_pin2 = [[torch.empty(H_out.shape, dtype=dt).pin_memory()] +
                 [torch.empty(W.shape, dtype=torch.float32).pin_memory() for W in Ws] for _ in range(NB)]
     cnt_pin2 = [torch.empty(L, 4, dtype=torch.int32).pin_memory() for _ in range(NB)]
+    pin_rows = min(blocks.caps[L - 1][1], max_rows)
+    dx_pin2 = [torch.empty(pin_rows, w.dim, dtype=dt).pin_memory() for _ in range(NB)]
+    id_pin2 = [torch.empty(pin_rows, dtype=torch.int32).pin_memory() for _ in range(NB)]
     h2d = seeds_pin[0].numel() * 4 + dH_pin.numel() * dH_pin.element_size()
-    d2h = sum(t.numel() * t.element_size() for t in res_pin2[0]) + cnt_pin2[0].numel() * 4
+    d2h_fixed = sum(t.numel() * t.element_size() for t in res_pin2[0]) + cnt_pin2[0].numel() * 4
     main_s = torch.cuda.current_stream()
     up_s, down_s = torch.cuda.Stream(), torch.cuda.Stream()
     ev = lambda: torch.cuda.Event()
-    done_ev, up_ev, out_ev = [ev() for _ in range(NB)], [ev() for _ in range(NB)], [ev() for _ in range(NB)]
+    done_ev, up_ev, out_ev, cnt_ev = ([ev() for _ in range(NB)] for _ in range(4))
 
-    def e2e_run(first, count):
-        """Steps first .. first + count - 1; returns the edges their results report."""
-        edges = 0
+    def e2e_run(first, count, with_dx):
+        """Steps first .. first + count - 1; returns (edges their results report, dX bytes downloaded, rows cut off)."""
+        edges, dx_bytes, cut = 0, 0, 0
         prime(first, seeds_pin)                                     # batches `first`, `first + 1` into their buffers
         with torch.cuda.stream(up_s):
             up_s.wait_stream(main_s)
             seeds_in2[(first + 2) % NB].copy_(seeds_pin[first + 2], non_blocking=True)
             dH_in2[first % NB].copy_(dH_pin, non_blocking=True)
             up_ev[first % NB].record(up_s)
+
+        def collect(j):
+            """Downloads of step j (its counts are already on their way) and the host's read of them."""
+            nonlocal edges, dx_bytes, cut
+            p = j % NB
+            cnt_ev[p].synchronize()
+            edges += int(cnt_pin2[p][:, 2].sum())
+            if with_dx:
+                n_src = int(cnt_pin2[p][L - 1, 1])
+                rows = min(n_src, pin_rows)
+                cut += n_src - rows
+                with torch.cuda.stream(down_s):
+                    dx_pin2[p][:rows].copy_(dX2[p][:rows], non_blocking=True)
+                    id_pin2[p][:rows].copy_(blocks2[p].t[L - 1]["src_nodes"][:rows], non_blocking=True)
+                    out_ev[p].record(down_s)
+                dx_bytes += rows * (w.dim * dx_pin2[p].element_size() + 4)
+
         for i in range(first, first + count):
             p, q = i % NB, (i + 1) % NB
             main_s.wait_event(up_ev[p])                              # inputs of step i are on the device
+            if i >= first + NB:
+                main_s.wait_event(out_ev[p])                         # the results of step i - 3 have left these buffers
             E.sampler_set_step(blocks2[(i + 2) % NB].scratch, first_step + i + 2)
             graphs[p].replay()
             done_ev[p].record(main_s)
@@ -505,107 +613,41 @@ def run_ours(args, w):
                 up_ev[q].record(up_s)
             with torch.cuda.stream(down_s):                          # results of step i, beside step i + 1
                 down_s.wait_event(done_ev[p])
+                cnt_pin2[p].copy_(counts_snap2[p], non_blocking=True)
+                cnt_ev[p].record(down_s)
                 res_pin2[p][0].copy_(H_out2[p], non_blocking=True)
                 for t, src in zip(res_pin2[p][1:], dWs2[p]):
                     t.copy_(src, non_blocking=True)
-                cnt_pin2[p].copy_(counts_snap2[p], non_blocking=True)
                 out_ev[p].record(down_s)
             if i > first:                                            # the caller reads the results of step i - 1
-                out_ev[(i - 1) % NB].synchronize()
-                edges += int(cnt_pin2[(i - 1) % NB][:, 2].sum())
-        last = (first + count - 1) % NB
-        out_ev[last].synchronize()
-        edges += int(cnt_pin2[last][:, 2].sum())
+                collect(i - 1)
+        collect(first + count - 1)
         torch.cuda.synchronize()
-        return edges
+        return edges, dx_bytes, cut
 
-    e2e_run(0, min(Wm, 3))
-    barrier()
-    t0 = time.perf_counter()
-    e2e_edges = e2e_run(Wm, K)
-    barrier()
-    e2e_s = time.perf_counter() - t0
+    def e2e_timed(with_dx):
+        e2e_run(0, min(Wm, 3), with_dx)
+        barrier()
+        t0 = time.perf_counter()
+        edges, dx_bytes, cut = e2e_run(Wm, K, with_dx)
+        barrier()
+        return time.perf_counter() - t0, edges, dx_bytes, cut
+
+    e2e_s, e2e_edges, dx_bytes, dx_cut = e2e_timed(True)
+    e2e_dev_s, e2e_dev_edges, _, _ = e2e_timed(False)
 
     # ---- joint step (sampled encoder + ranking tower + BCE, forward and backward) on the same graph
     joint = None
-    if not args.no_joint and not on_device:
-        P, dd = w.batch, 64
-        jr = np.random.default_rng(4 + rank)
-        picks = jr.integers(0, inter[0].size, (min(K, 200) + Wm + 1, P))
-        pu_all = torch.from_numpy(inter[0][picks].astype(np.int32)).to(dev)
-        pi_all = torch.from_numpy(inter[1][picks].astype(np.int32)).to(dev)
-        dense = torch.from_numpy(jr.standard_normal((P, dd)).astype(np.float32)).to(dev)
-        labels = torch.from_numpy(S.bernoulli_labels(P, 0.1, 4)).to(dev)
-        zdim = 2 * w.hidden + dd
-        Wt_h = [S.glorot_uniform(512, zdim, 4, 40), S.glorot_uniform(256, 512, 4, 41), S.glorot_uniform(1, 256, 4, 42)]
-        Wt = [torch.from_numpy(a).to(dev, dt) for a in Wt_h]
-        bt = [torch.zeros(a.shape[0], dtype=torch.float32, device=dev) for a in Wt_h]
-        # two workspaces: the pairs of the next step are turned into seeds and sampled (phase 1) on a second stream
-        # while the rest of the current step (phase 2) runs
-        js2 = [E.JointStep(indptr, indices, X, P, dd, w.fanouts, Ws, Wt, bt) for _ in range(2)]
-        pu_in2 = [torch.empty_like(pu_all[0]) for _ in range(2)]
-        pi_in2 = [torch.empty_like(pi_all[0]) for _ in range(2)]
-
-        def j_sample(p):
-            js2[p].run(pu_in2[p], pi_in2[p], dense, labels, 4, 0, phase=1)
-
-        def j_compute(p):
-            js2[p].run(pu_in2[p], pi_in2[p], dense, labels, 4, 0, phase=2)
-
-        with torch.cuda.stream(side):
-            for i in range(Wm):
-                for p in range(2):
-                    pu_in2[p].copy_(pu_all[i]); pi_in2[p].copy_(pi_all[i])
-                    E.sampler_set_step(js2[p].ws, first_step + i)
-                    with torch.cuda.stream(side2):
-                        side2.wait_stream(side)
-                        j_sample(p)
-                    side.wait_stream(side2)
-                    j_compute(p)
-        side.synchronize()
-        jgraphs = []
-        for p in range(2):
-            g = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(g, stream=side):
-                side2.wait_stream(side)
-                with torch.cuda.stream(side2):
-                    j_sample(1 - p)
-                j_compute(p)
-                side.wait_stream(side2)
-            jgraphs.append(g)
-        KJ = picks.shape[0] - Wm - 1
-        # batch Wm sampled ahead, as the previous replay would have done
-        pu_in2[Wm & 1].copy_(pu_all[Wm]); pi_in2[Wm & 1].copy_(pi_all[Wm])
-        E.sampler_set_step(js2[Wm & 1].ws, first_step + Wm)
-        j_sample(Wm & 1)
-        barrier()
-        j0, j1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        j0.record()
-        for i in range(Wm, Wm + KJ):
-            q = (i + 1) & 1
-            pu_in2[q].copy_(pu_all[i + 1], non_blocking=True)
-            pi_in2[q].copy_(pi_all[i + 1], non_blocking=True)
-            E.sampler_set_step(js2[q].ws, first_step + i + 1)
-            jgraphs[i & 1].replay()
-        j1.record()
-        barrier()
-        jms = j0.elapsed_time(j1)
-        js = js2[(Wm + KJ - 1) & 1]
-        n_rows, jstatus = js.n_rows.tolist()
-        if jstatus or js2[0].n_rows.tolist()[1] or js2[1].n_rows.tolist()[1]:
-            raise RuntimeError(f"joint step: device status bits {jstatus}")
-        joint = dict(metric="joint_step_samples_per_sec", value=KJ * P * world / (jms / 1e3), unit="pairs/s",
-                     ms_per_step=jms / KJ, steps=KJ, pairs_per_step=P, tower="320-512-256-1", dense_dim=dd,
-                     loss=float(js.loss),
-                     launch="one CUDA graph replay per step: e2egrec_joint_step_phase COMPUTE of the batch beside SAMPLE of the next")
+    if with_joint and not on_device:
+        joint = run_joint(args, w, E, dev, dt, world, rank, first_step, indptr, indices, X, Ws, inter, indptr_h, indices_h,
+                          X_h, Ws_h, (side, side2), barrier, want_cpu)
 
     # ---- reduce over ranks: slowest rank's time, all ranks' edges
     from paper_2511_20564_b200 import replicas
-    (ms, e2e_s), (edges_all, e2e_edges_all) = replicas.reduce_measurements([ms, e2e_s], [edges_rank, e2e_edges], dev)
+    (ms, e2e_s, e2e_dev_s), (edges_all, e2e_edges_all, e2e_dev_edges_all) = replicas.reduce_measurements(
+        [ms, e2e_s, e2e_dev_s], [edges_rank, e2e_edges, e2e_dev_edges], dev)
     if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return
+        return None
 
     # ---- roofline of the dominant kernel (algorithmic bytes or flops per launch / mean launch time)
     peaks = measured_peaks()
@@ -613,35 +655,43 @@ def run_ours(args, w):
     r = w.dim * es
     n_dst, n_src, n_edges = float(outer_counts[0]), float(outer_counts[1]), float(outer_counts[2])
     dom_mean_ms = float(np.mean(dom_ms))
-    if dominant == 1:      # per entry: id + gathered row; per destination: offsets, self id, self row, [self|mean] row out
-        alg = n_edges * (4 + r) + n_dst * (8 + 4 + r + 2 * r)
-        roof = dict(bound="hbm", achieved=alg / dom_mean_ms / 1e6, peak=peaks["hbm_gbs"], unit="GB/s")
-    elif dominant == 2:    # per entry: row id + gathered row; per source: offsets + row out; per destination: self row
-        alg = n_edges * (4 + r) + n_src * (8 + r) + n_dst * r
-        roof = dict(bound="hbm", achieved=alg / dom_mean_ms / 1e6, peak=peaks["hbm_gbs"], unit="GB/s")
-    else:                  # dense products of layer 0: 2 * rows * (2 d) * hidden flop each
-        alg = 2.0 * n_dst * 2 * w.dim * w.hidden
-        peak = peaks["bf16_tflops"] if w.dtype == "bf16" else peaks["bf16_tflops"] / 2.25 * 0.08
-        roof = dict(bound="tensor" if w.dtype == "bf16" else "alu", achieved=alg / dom_mean_ms / 1e9, peak=peak,
-                    unit="TFLOP/s")
-    # both aggregation kernels of the outermost block, whichever kernel dominates
+    # both aggregation kernels of the outermost block, whichever kernel dominates.  forward, per entry: id + gathered
+    # row; per destination: offsets, self id, self row, [self|mean] row out.  backward, per entry: row id + gathered
+    # row; per source: offsets + row out; per destination: self row
     alg_fwd = n_edges * (4 + r) + n_dst * (8 + 4 + r + 2 * r)
     alg_bwd = n_edges * (4 + r) + n_src * (8 + r) + n_dst * r
+    if dominant in (1, 2):
+        alg = alg_fwd if dominant == 1 else alg_bwd
+        roof = dict(bound="hbm", achieved=alg / dom_mean_ms / 1e6, peak=peaks["hbm_gbs"], unit="GB/s")
+        roof["frac_of_nominal_8tbs"] = roof["achieved"] / NOMINAL_HBM_GBS
+    else:                  # dense products of layer 0: 2 * rows * (2 d) * hidden flop each
+        alg = 2.0 * n_dst * 2 * w.dim * w.hidden
+        peak = peaks["bf16_tflops"] if w.dtype == "bf16" else fp32_alu_peak_tflops(peaks)
+        roof = dict(bound="tensor" if w.dtype == "bf16" else "alu", achieved=alg / dom_mean_ms / 1e9, peak=peak,
+                    unit="TFLOP/s")
     aggregation = {
         "outer_block": dict(n_dst=n_dst, n_src=n_src, n_edges=n_edges, row_bytes=r),
         "forward": dict(kernel="sage_aggregate_kernel", ms=tap_ms[1], algorithmic_bytes=alg_fwd,
-                        gbs=alg_fwd / tap_ms[1] / 1e6, frac_of_hbm=alg_fwd / tap_ms[1] / 1e6 / peaks["hbm_gbs"]),
+                        **hbm_fractions(alg_fwd / tap_ms[1] / 1e6, peaks)),
         "backward": dict(kernel="seg_run_kernel+seg_final_kernel", ms=tap_ms[2], algorithmic_bytes=alg_bwd,
-                         gbs=alg_bwd / tap_ms[2] / 1e6, frac_of_hbm=alg_bwd / tap_ms[2] / 1e6 / peaks["hbm_gbs"])}
-    # DRAM bytes per launch from the ncu launch list of this command (profiles/medium_step_launch_list.md);
-    # known only for the aggregation kernels of the outermost block of the `medium` workload
-    traffic = {1: 6.30e6, 2: 5.55e6 + 1.91e6}.get(dominant) if w.name == "medium" and args.seeds == "activity" else None
-    roof.update(frac=roof["achieved"] / roof["peak"], traffic=traffic, kernel=TAP_NAMES[dominant],
+                         **hbm_fractions(alg_bwd / tap_ms[2] / 1e6, peaks))}
+    # DRAM bytes per launch: a recorded ncu capture of the same kernel (bytes per entry of the outermost block, taken on
+    # this workload or on its reduced-size stand-in) times the entries of one launch here; null without a fresh record
+    traffic, traffic_from = None, None
+    if dominant in (1, 2) and args.seeds == "activity" and args.beta is None:
+        rec = recorded_traffic(f"{w.name}:{'forward' if dominant == 1 else 'backward'}")
+        if rec:
+            traffic = rec["dram_bytes_per_entry"] * n_edges
+            traffic_from = rec.get("captured_on")
+    roof.update(frac=roof["achieved"] / roof["peak"], traffic=traffic, traffic_from=traffic_from, kernel=TAP_NAMES[dominant],
                 ms_per_launch=dom_mean_ms, algorithmic_units_per_launch=alg, peak_source=peaks["source"])
 
+    d2h_dx = dx_bytes / K
     line = dict(metric=METRIC, value=edges_all / (ms / 1e3), unit=UNIT, n_gpus=world, steps=K, warmup=Wm,
                 ms_per_step=ms / K, higher_is_better=True, scaling="weak", vs_baseline=None, dtype=w.dtype,
                 data="synthetic",
+                timing=dict(repeats=repeats, timed_region_s=sum(rep_ms) / 1e3, ms_per_step_min=min(rep_ms) / K,
+                            ms_per_step_max=max(rep_ms) / K, statistic="median over the repetitions of the K-step loop"),
                 config=dict(workload=w.name, nodes=w.n_nodes, csr_entries=int(indices.numel()), dim=w.dim, hidden=w.hidden,
                             layers=L, fanouts=list(w.fanouts), batch=w.batch, seeds=args.seeds,
                             sampling="uniform" if args.beta is None else f"weighted, beta={args.beta}",
@@ -655,9 +705,16 @@ def run_ours(args, w):
                             edges_per_step=edges_rank / K, setup_s=round(setup_s, 1),
                             generated="on the device (torch)" if on_device else "on the host (numpy)"),
                 clocks=clk,
-                e2e=dict(value=e2e_edges_all / e2e_s, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h,
-                         ms_per_step=e2e_s / K * 1e3),
-                gpu_launches=int(launches),
+                e2e=dict(value=e2e_edges_all / e2e_s, unit=UNIT, h2d_bytes_per_step=h2d, d2h_bytes_per_step=d2h_fixed + d2h_dx,
+                         ms_per_step=e2e_s / K * 1e3,
+                         results="embeddings, weight gradients, counts, and the feature-gradient rows with their node ids "
+                                 "(true count per step)", dx_rows_not_copied=int(dx_cut)),
+                e2e_dx_on_device=dict(value=e2e_dev_edges_all / e2e_dev_s, unit=UNIT, h2d_bytes_per_step=h2d,
+                                      d2h_bytes_per_step=d2h_fixed, ms_per_step=e2e_dev_s / K * 1e3,
+                                      dx_left_on_device_bytes=d2h_dx,
+                                      note="same steps with the feature-gradient rows left on the device, where the feature "
+                                           "table lives and a sparse update would consume them"),
+                gpu_launches=int(launches * repeats),
                 roofline=roof, aggregation=aggregation,
                 kernel_ms={TAP_NAMES[k].split(" (")[0]: v for k, v in tap_ms.items()})
     if joint is not None:
@@ -677,7 +734,7 @@ def run_ours(args, w):
             need = indices.numel() * 4 + indptr.numel() * 8
             if psutil.virtual_memory().available < need * 1.5:
                 want_cpu = False
-                line["cpu_baseline"] = dict(value=None, unit=UNIT, cores=1, kind="oracle",
+                line["cpu_baseline"] = dict(value=None, unit=UNIT, cores=0, kind="oracle",
                                             sample=f"skipped: the host copy of the graph ({need / 1e9:.1f} GB) does not fit")
             else:
                 indptr_h, indices_h = indptr.cpu().numpy(), indices.cpu().numpy()
@@ -688,18 +745,153 @@ def run_ours(args, w):
         if q_h is not None:
             import oracle
             cum_h = oracle.edge_cumulate(indptr_h, q_h)
-        t0 = time.perf_counter()
-        ce, n = 0, 0
-        while n < K and time.perf_counter() - t0 < 15.0:
-            ce += oracle_step(w, indptr_h, indices_h, X_src, Ws_h, seeds_h[Wm + n][:sample], Wm + n, dH64, cum_h)
-            n += 1
-        cdt = time.perf_counter() - t0
-        line["cpu_baseline"] = dict(value=ce / cdt, unit=UNIT, cores=1, kind="oracle",
-                                    sample=f"{n} step(s) on the first {sample} of the {w.batch} seeds of the batch, "
-                                           f"full sample+forward+backward, {cdt:.1f} s{note}")
-    print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+        line["cpu_baseline"] = time_oracle(
+            lambda n: oracle_step(w, indptr_h, indices_h, X_src, Ws_h, seeds_h[Wm + n][:sample], Wm + n, dH64, cum_h),
+            args.cpu_seconds, K, UNIT,
+            lambda n, s: f"{n} step(s) on the first {sample} of the {w.batch} seeds of the batch, full "
+                         f"sample+forward+backward, {s:.1f} s{note}")
+    return line
+
+
+# ------------------------------------------------------------------------------------------ joint step
+def run_joint(args, w, E, dev, dt, world, rank, first_step, indptr, indices, X, Ws, inter, indptr_h, indices_h, X_h, Ws_h,
+              streams, barrier, want_cpu):
+    """Joint step (sampled encoder + ranking tower + BCE, forward and full backward) on the graph of workload w:
+    4 096 training pairs drawn from the interaction list, 64 dense features per pair, tower 512-256-1."""
+    import torch
+    side, side2 = streams
+    K, Wm = args.steps, args.warmup
+    P, dd = w.batch, 64
+    n_j = min(K, 200)
+    jr = np.random.default_rng(4 + rank)
+    picks = jr.integers(0, inter[0].size, (n_j + Wm + 1, P))
+    pu_h, pi_h = inter[0][picks].astype(np.int32), inter[1][picks].astype(np.int32)
+    pu_all, pi_all = torch.from_numpy(pu_h).to(dev), torch.from_numpy(pi_h).to(dev)
+    dense_h = jr.standard_normal((P, dd)).astype(np.float32)
+    labels_h = S.bernoulli_labels(P, 0.1, 4)
+    dense, labels = torch.from_numpy(dense_h).to(dev), torch.from_numpy(labels_h).to(dev)
+    zdim = 2 * w.hidden + dd
+    Wt_h = [S.glorot_uniform(512, zdim, 4, 40), S.glorot_uniform(256, 512, 4, 41), S.glorot_uniform(1, 256, 4, 42)]
+    if w.dtype == "bf16":
+        Wt_h = [S.to_bf16_values(a) for a in Wt_h]
+    Wt = [torch.from_numpy(a).to(dev, dt) for a in Wt_h]
+    bt = [torch.zeros(a.shape[0], dtype=torch.float32, device=dev) for a in Wt_h]
+    gate_kw = {}
+    if args.gate:
+        Wg_h = S.glorot_uniform(zdim, zdim, 4, 43)
+        gate_kw = dict(W_gate=torch.from_numpy(Wg_h).to(dev, dt), b_gate=torch.zeros(zdim, dtype=torch.float32, device=dev))
+    # two workspaces: the pairs of the next step are turned into seeds and sampled (phase 1) on a second stream
+    # while the rest of the current step (phase 2) runs
+    js2 = [E.JointStep(indptr, indices, X, P, dd, w.fanouts, Ws, Wt, bt, **gate_kw) for _ in range(2)]
+    pu_in2 = [torch.empty_like(pu_all[0]) for _ in range(2)]
+    pi_in2 = [torch.empty_like(pi_all[0]) for _ in range(2)]
+
+    def j_sample(p):
+        js2[p].run(pu_in2[p], pi_in2[p], dense, labels, 4, 0, phase=1)
+
+    def j_compute(p):
+        js2[p].run(pu_in2[p], pi_in2[p], dense, labels, 4, 0, phase=2)
+
+    with torch.cuda.stream(side):
+        for i in range(Wm):
+            for p in range(2):
+                pu_in2[p].copy_(pu_all[i]); pi_in2[p].copy_(pi_all[i])
+                E.sampler_set_step(js2[p].ws, first_step + i)
+                with torch.cuda.stream(side2):
+                    side2.wait_stream(side)
+                    j_sample(p)
+                side.wait_stream(side2)
+                j_compute(p)
+    side.synchronize()
+    jgraphs, per_step = [], 0
+    for p in range(2):
+        l0 = E.launch_count()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            side2.wait_stream(side)
+            with torch.cuda.stream(side2):
+                j_sample(1 - p)
+            j_compute(p)
+            side.wait_stream(side2)
+        jgraphs.append(g)
+        per_step = E.launch_count() - l0
+
+    def joint_loop():
+        # batch Wm sampled ahead, as the previous replay would have done
+        pu_in2[Wm & 1].copy_(pu_all[Wm]); pi_in2[Wm & 1].copy_(pi_all[Wm])
+        E.sampler_set_step(js2[Wm & 1].ws, first_step + Wm)
+        j_sample(Wm & 1)
+        barrier()
+        j0, j1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        j0.record()
+        for i in range(Wm, Wm + n_j):
+            q = (i + 1) & 1
+            pu_in2[q].copy_(pu_all[i + 1], non_blocking=True)
+            pi_in2[q].copy_(pi_all[i + 1], non_blocking=True)
+            E.sampler_set_step(js2[q].ws, first_step + i + 1)
+            jgraphs[i & 1].replay()
+        j1.record()
+        barrier()
+        for js in js2:
+            if js.n_rows.tolist()[1]:
+                raise RuntimeError(f"joint step: device status bits {js.n_rows.tolist()[1]}")
+        return j0.elapsed_time(j1)
+
+    probe = joint_loop()
+    repeats = max(1, min(2000, math.ceil(MIN_TIMED_S * 1e3 / max(probe, 1e-3))))
+    clocks = ClockSampler(dev.index or 0)
+    clocks.start()
+    time.sleep(0.3)
+    t_begin = clocks.mark()
+    rep_ms = [joint_loop() for _ in range(repeats)]
+    clk = clocks.stop(t_begin, clocks.mark())
+    jms = float(statistics.median(rep_ms))
+    js = js2[(Wm + n_j - 1) & 1]
+
+    # roofline of the step's widest aggregation kernel group: the transposed aggregation of the outermost block, timed
+    # with events around it inside eagerly launched whole steps
+    ev_a, ev_b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev_a.record(); ev_b.record()                        # the tap wants events whose CUDA handles exist
+    torch.cuda.synchronize()
+    tap, cnts = [], []
+    for i in range(min(n_j, 20)):
+        pu_in2[0].copy_(pu_all[Wm + i]); pi_in2[0].copy_(pi_all[Wm + i])
+        E.sampler_set_step(js2[0].ws, first_step + Wm + i)
+        torch.cuda._sleep(2_000_000)
+        E.profile_tap(2, ev_a, ev_b)
+        js2[0].run(pu_in2[0], pi_in2[0], dense, labels, 4, 0)
+        torch.cuda.synchronize()
+        tap.append(ev_a.elapsed_time(ev_b))
+        cnts.append(js2[0].activations()["counts"][len(w.fanouts) - 1].tolist())
+    peaks = measured_peaks()
+    r = w.dim * (2 if w.dtype == "bf16" else 4)
+    n_dst, n_src, n_edges = (float(np.mean([c[k] for c in cnts])) for k in range(3))
+    alg_bwd = n_edges * (4 + r) + n_src * (8 + r) + n_dst * r
+    tms = float(np.mean(tap))
+    roof = dict(bound="hbm", achieved=alg_bwd / tms / 1e6, peak=peaks["hbm_gbs"], unit="GB/s", traffic=None,
+                kernel=TAP_NAMES[2], ms_per_launch=tms, algorithmic_units_per_launch=alg_bwd, peak_source=peaks["source"],
+                outer_block=dict(n_dst=n_dst, n_src=n_src, n_edges=n_edges, row_bytes=r))
+    roof["frac"] = roof["achieved"] / roof["peak"]
+    roof["frac_of_nominal_8tbs"] = roof["achieved"] / NOMINAL_HBM_GBS
+    joint = dict(metric="joint_step_samples_per_sec", value=n_j * P * world / (jms / 1e3), unit="pairs/s",
+                 ms_per_step=jms / n_j, steps=n_j, pairs_per_step=P, tower="320-512-256-1", dense_dim=dd,
+                 gate_fusion=bool(args.gate), loss=float(js.loss), clocks=clk,
+                 timing=dict(repeats=repeats, timed_region_s=sum(rep_ms) / 1e3, ms_per_step_min=min(rep_ms) / n_j,
+                             ms_per_step_max=max(rep_ms) / n_j, statistic="median over the repetitions of the loop"),
+                 gpu_launches=int(per_step * n_j * repeats), roofline=roof,
+                 launch="one CUDA graph replay per step: e2egrec_joint_step_phase COMPUTE of the batch beside SAMPLE of the next")
+    if want_cpu and indptr_h is not None and not args.gate:
+        import oracle
+        oracle.build()
+        sample = max(32, args.ref_seeds // 2)             # pairs per oracle step (two endpoints each)
+        bf16 = w.dtype == "bf16"
+        joint["cpu_baseline"] = time_oracle(
+            lambda n: (oracle.joint_step(indptr_h, indices_h, X_h, pu_h[Wm + n][:sample], pi_h[Wm + n][:sample],
+                                         dense_h[:sample], labels_h[:sample], w.fanouts, Ws_h, Wt_h, None, 4, Wm + n,
+                                         bf16=bf16) and sample),
+            args.cpu_seconds, n_j, "pairs/s",
+            lambda n, s: f"{n} step(s) on the first {sample} of the {P} pairs of the batch, whole joint step, {s:.1f} s")
+    return joint
 
 
 # ------------------------------------------------------------------------------------------ LightGCN on sampled blocks
@@ -795,21 +987,27 @@ def run_lightgcn(args, w):
         E.sampler_set_step(blocks2[(i + 2) % NB].scratch, i + 2)
         graphs[i % NB].replay()
 
-    prime(Wm)
-    count_total.zero_()
+    def timed_loop():
+        prime(Wm)
+        count_total.zero_()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(K):
+            replay_step(Wm + i)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    probe = timed_loop()
+    repeats = max(1, min(2000, math.ceil(MIN_TIMED_S * 1e3 / max(probe, 1e-3))))
     clocks = ClockSampler(0)
     clocks.start()
-    time.sleep(0.6)
-    torch.cuda.synchronize()
+    time.sleep(0.3)
     t_begin = clocks.mark()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for i in range(K):
-        replay_step(Wm + i)
-    e1.record()
-    torch.cuda.synchronize()
+    rep_ms = [timed_loop() for _ in range(repeats)]
     clk = clocks.stop(t_begin, clocks.mark())
-    ms = e0.elapsed_time(e1)
+    ms = float(statistics.median(rep_ms))
     counts = count_total.cpu().numpy()
     if counts[:, 3].any():
         raise RuntimeError(f"device status bits set during the timed region: {counts[:, 3]}")
@@ -817,29 +1015,28 @@ def run_lightgcn(args, w):
     line = dict(metric="sampled_lightgcn_sample_fwd_bwd_edges_per_sec", value=edges / (ms / 1e3), unit=UNIT, n_gpus=1, steps=K,
                 warmup=Wm, ms_per_step=ms / K, higher_is_better=True, scaling="weak", vs_baseline=None, dtype=w.dtype,
                 data="synthetic",
+                timing=dict(repeats=repeats, timed_region_s=sum(rep_ms) / 1e3, statistic="median over the repetitions"),
                 config=dict(workload=w.name, backbone="lightgcn", nodes=w.n_nodes, csr_entries=int(indices.numel()), dim=w.dim,
                             layers=len(w.fanouts), fanouts=list(w.fanouts), batch=w.batch, seeds=args.seeds,
                             launch="one CUDA graph replay per step, three streams: propagation and adjoint of batch i beside "
                                    "the transposed form of batch i+1 and the hops of batch i+2", edges_per_step=edges / K),
-                clocks=clk, gpu_launches=int(K * (kernels_per_step + 2)))
+                clocks=clk, gpu_launches=int(K * (kernels_per_step + 2) * repeats))
     if not args.no_cpu_baseline:
         import oracle
         oracle.build()
         row, col = S.undirected_coo(users, items)
         indptr_h, indices_h = S.coo_to_csr(w.n_nodes, row, col)
         sample = args.ref_seeds
-        t0 = time.perf_counter()
-        ce, n = 0, 0
-        while n < K and time.perf_counter() - t0 < 15.0:
+
+        def ostep(n):
             blocks = oracle.sample_khop(indptr_h, indices_h, seeds_h[Wm + n][:sample], w.fanouts, w.seed, Wm + n)
             _, octx = oracle.lightgcn_sampled_forward(blocks, X_h, s_h, w.dtype == "bf16")
             oracle.lightgcn_sampled_backward(blocks, octx, dY_h[:sample], w.dtype == "bf16")
-            ce += sum(b["n_edges"] for b in blocks)
-            n += 1
-        cdt = time.perf_counter() - t0
-        line["cpu_baseline"] = dict(value=ce / cdt, unit=UNIT, cores=1, kind="oracle",
-                                    sample=f"{n} step(s) on the first {sample} of the {w.batch} seeds of the batch, {cdt:.1f} s")
-    print(json.dumps(line), flush=True)
+            return sum(b["n_edges"] for b in blocks)
+
+        line["cpu_baseline"] = time_oracle(ostep, args.cpu_seconds, K, UNIT,
+                                           lambda n, s: f"{n} step(s) on the first {sample} of the {w.batch} seeds of the batch, {s:.1f} s")
+    return line
 
 
 # ------------------------------------------------------------------------------------------ whole-graph aggregation
@@ -874,7 +1071,7 @@ def run_fullgraph(args):
     dX = torch.empty(n, d, dtype=torch.bfloat16, device=dev)
     _, ws_f = E.aggregate_forward(indptr, indices, X, out)
     _, ws_b = E.aggregate_backward(csc_ptr, csc_row, inv_deg, G, dX)
-    K, Wm = args.steps, max(args.warmup, 3)
+    Wm = max(args.warmup, 3)
 
     def fwd():
         E.aggregate_forward(indptr, indices, X, out, ws_f)
@@ -885,9 +1082,14 @@ def run_fullgraph(args):
     for _ in range(Wm):
         fwd(); bwd()
     torch.cuda.synchronize()
+    pa, pb, pc = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+    pa.record(); fwd(); pb.record(); bwd(); pc.record()
+    torch.cuda.synchronize()
+    # as many steps as the caller asked for, and at least enough for a timed region of MIN_TIMED_S
+    K = max(args.steps, math.ceil(MIN_TIMED_S * 1e3 / max(pa.elapsed_time(pc), 1e-3)))
     clocks = ClockSampler(0)
     clocks.start()
-    time.sleep(0.6)
+    time.sleep(0.3)
     t_begin = clocks.mark()
     l0 = E.launch_count()
     ef = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
@@ -897,8 +1099,8 @@ def run_fullgraph(args):
     torch.cuda.synchronize()
     clk = clocks.stop(t_begin, clocks.mark())
     launches = E.launch_count() - l0
-    t_f = float(np.mean([a.elapsed_time(b) for a, b, _ in ef]))
-    t_b = float(np.mean([b.elapsed_time(c) for _, b, c in ef]))
+    t_f = float(statistics.median([a.elapsed_time(b) for a, b, _ in ef]))
+    t_b = float(statistics.median([b.elapsed_time(c) for _, b, c in ef]))
     ms = ef[0][0].elapsed_time(ef[-1][2])
     # end to end: features from pinned host memory in, aggregated rows out, every step
     X_pin, G_pin = X.cpu().pin_memory(), G.cpu().pin_memory()
@@ -914,26 +1116,43 @@ def run_fullgraph(args):
     e2e_s = (time.perf_counter() - t0) / ke
     peaks = measured_peaks()
     r = d * 2
-    alg_f = m * (4 + r) + n * (16 + r)          # per entry: id + gathered row; per row: two offsets + the output row
-    alg_b = m * (4 + 4 + r) + n * (16 + r)      # + the per-entry weight 1/deg
-    big = "fwd" if t_f >= t_b else "bwd"
-    alg, tk = (alg_f, t_f) if big == "fwd" else (alg_b, t_b)
-    roof = dict(bound="hbm", achieved=alg / tk / 1e6, peak=peaks["hbm_gbs"], unit="GB/s", traffic=None,
-                kernel=f"seg_run_kernel+seg_final_kernel ({big})", ms_per_launch=tk,
-                algorithmic_units_per_launch=alg, peak_source=peaks["source"],
-                compulsory_bytes=n * r * 2 + m * 4 + n * 16,
-                # ncu DRAM bytes (read + write, both kernels) of one launch on the 1/5-scale graph
-                # (profiles/seg_run_kernel_fullgraph.md); not scaled up: the L2 hit rate changes with the table size
-                traffic_at_scale_0_2=dict(fwd=383.0e6, bwd=355.0e6))
+    # (no-reuse) per entry: id + gathered row; per row: two offsets + the output row; backward + the per-entry weight 1/deg
+    alg_f = m * (4 + r) + n * (16 + r)
+    alg_b = m * (4 + 4 + r) + n * (16 + r)
+    # (compulsory) every distinct byte once: the table in, the table out, the ids, the offsets (+ the weights)
+    comp_f = n * r * 2 + m * 4 + n * 16
+    comp_b = comp_f + n * 4
+
+    def direction(name, t_ms, alg, comp):
+        rec = recorded_traffic(f"fullgraph:{name}")
+        out_d = dict(ms=t_ms, edges_per_s=m / (t_ms / 1e3),
+                     no_reuse=dict(bytes=alg, **hbm_fractions(alg / t_ms / 1e6, peaks)),
+                     compulsory=dict(bytes=comp, **hbm_fractions(comp / t_ms / 1e6, peaks)),
+                     dram_counter=None)
+        if rec:   # bytes per entry measured by ncu on the reduced graph named in the record, times this graph's entries
+            tr = rec["dram_bytes_per_entry"] * m
+            out_d["dram_counter"] = dict(bytes=tr, captured_on=rec.get("captured_on"), **hbm_fractions(tr / t_ms / 1e6, peaks))
+        return out_d
+
+    fwd_d, bwd_d = direction("forward", t_f, alg_f, comp_f), direction("backward", t_b, alg_b, comp_b)
+    big, big_d = ("fwd", fwd_d) if t_f >= t_b else ("bwd", bwd_d)
+    roof = dict(bound="hbm", achieved=big_d["no_reuse"]["gbs"], peak=peaks["hbm_gbs"], unit="GB/s",
+                traffic=big_d["dram_counter"]["bytes"] if big_d["dram_counter"] else None,
+                kernel=f"seg_run_kernel+seg_final_kernel ({big})", ms_per_launch=big_d["ms"],
+                algorithmic_units_per_launch=big_d["no_reuse"]["bytes"], peak_source=peaks["source"],
+                frac_of_nominal_8tbs=big_d["no_reuse"]["frac_of_nominal_8tbs"],
+                compulsory_frac=big_d["compulsory"]["frac_of_measured_copy"],
+                dram_counter_frac=big_d["dram_counter"]["frac_of_measured_copy"] if big_d["dram_counter"] else None,
+                note="achieved = algorithmic no-reuse bytes / time; the compulsory-bytes and DRAM-counter fractions beside it")
     roof["frac"] = roof["achieved"] / roof["peak"]
     line = dict(metric="fullgraph_mean_aggregation_fwd_bwd_edges_per_sec", value=m / ((t_f + t_b) / 1e3), unit="edges/s",
-                n_gpus=1, steps=K, warmup=Wm, ms_per_step=ms / K, higher_is_better=True, scaling="weak", vs_baseline=None,
+                n_gpus=1, steps=K, warmup=Wm, ms_per_step=t_f + t_b, higher_is_better=True, scaling="weak", vs_baseline=None,
                 dtype="bf16", data="synthetic",
+                timing=dict(timed_region_s=ms / 1e3, statistic="median over the steps, forward and backward timed apart"),
                 config=dict(workload="fullgraph", nodes=n, csr_entries=m, dim=d, alpha=1.1, max_degree=max_degree,
                             l2="inputs larger than L2 (features %.0f MB, indices %.0f MB)" % (n * r / 1e6, m * 4 / 1e6),
                             ingest_s=round(setup_s, 1)),
-                fwd_ms=t_f, bwd_ms=t_b, fwd_edges_per_s=m / (t_f / 1e3), bwd_edges_per_s=m / (t_b / 1e3),
-                fwd_gbs=alg_f / t_f / 1e6, bwd_gbs=alg_b / t_b / 1e6, clocks=clk,
+                forward=fwd_d, backward=bwd_d, clocks=clk,
                 e2e=dict(value=m / e2e_s, unit="edges/s", h2d_bytes_per_step=2 * n * r, d2h_bytes_per_step=2 * n * r,
                          ms_per_step=e2e_s * 1e3),
                 gpu_launches=int(launches), roofline=roof)
@@ -941,26 +1160,36 @@ def run_fullgraph(args):
         import oracle
         oracle.build()
         rows = min(n, 200_000)
-        indptr_h, indices_h = S.coo_to_csr(n, dst, src)           # host CSR for the oracle only
-        t0 = time.perf_counter()
-        oracle.mean_aggregate(indptr_h[: rows + 1], indices_h[: int(indptr_h[rows])], X_h, True)
-        cdt = time.perf_counter() - t0
-        line["cpu_baseline"] = dict(value=int(indptr_h[rows]) / cdt, unit="edges/s", cores=1, kind="oracle",
-                                    sample=f"forward mean aggregation of the first {rows} rows ({int(indptr_h[rows])} entries), {cdt:.1f} s")
-    print(json.dumps(line), flush=True)
+        keep = dst < rows                                           # host CSR of the first rows only, for the oracle
+        indptr_h, indices_h = S.coo_to_csr(rows, dst[keep], src[keep])
+        line["cpu_baseline"] = time_oracle(
+            lambda k: (oracle.mean_aggregate(indptr_h, indices_h, X_h, True) is not None) * int(indptr_h[rows]),
+            args.cpu_seconds, 3, "edges/s",
+            lambda k, s: f"{k} forward mean aggregation(s) of the first {rows} rows ({int(indptr_h[rows])} entries), {s:.1f} s")
+    return line
+
+
+def free_device_memory():
+    import torch
+    gc.collect()
+    torch.cuda.empty_cache()
 
 
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="medium", choices=sorted(S.WORKLOADS) + ["fullgraph"])
+    ap.add_argument("--workload", default=None, choices=sorted(S.WORKLOADS) + ["fullgraph"],
+                    help="default: `large` with `medium`, the joint step and `fullgraph` as sub-records")
     ap.add_argument("--scale", type=float, default=1.0, help="fullgraph only: fraction of the 5 M node / 100 M entry graph")
     ap.add_argument("--ref-seeds", type=int, default=256, help="seeds per step given to the CPU oracle")
+    ap.add_argument("--cpu-seconds", type=float, default=8.0, help="time budget of each CPU-oracle timing (all cores, one core)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-joint", action="store_true", help="skip the joint-step measurement")
+    ap.add_argument("--no-sub", action="store_true", help="default run: skip the sub-records")
+    ap.add_argument("--gate", action="store_true", help="joint step with the gating fusion of the tower's input (Sec. 4.3.2)")
     ap.add_argument("--backbone", default="sage", choices=["sage", "lightgcn"],
                     help="lightgcn: sampling + LightGCN propagation on the sampled blocks + its adjoint (no weights)")
     ap.add_argument("--multitask", action="store_true",
@@ -971,19 +1200,47 @@ def main():
                     help="how seed batches are drawn (see make_batches)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
-    if args.workload == "fullgraph":
-        if args.impl == "ours" and int(os.environ.get("RANK", "0")) == 0:
-            run_fullgraph(args)
-        return
-    w = S.WORKLOADS[args.workload]
-    if args.backbone == "lightgcn":
-        if args.impl == "ours" and int(os.environ.get("RANK", "0")) == 0:
-            run_lightgcn(args, w)
-        return
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    suite = args.workload is None
+    name = "large" if suite else args.workload
+
     if args.impl == "reference":
-        run_reference(args, w)
-    else:
-        run_ours(args, w)
+        if name == "fullgraph":
+            raise SystemExit("--impl reference runs the sampled workloads")
+        line = run_reference(args, S.WORKLOADS[name])
+        if line is not None:
+            print(json.dumps(line), flush=True)
+        return
+    if name == "fullgraph":
+        if rank == 0:
+            print(json.dumps(run_fullgraph(args)), flush=True)
+        return
+    if args.backbone == "lightgcn":
+        if rank == 0:
+            print(json.dumps(run_lightgcn(args, S.WORKLOADS[name])), flush=True)
+        return
+
+    import torch
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(int(os.environ.get("LOCAL_RANK", "0")))
+        dist.init_process_group("nccl", device_id=torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0"))))
+    line = run_ours(args, S.WORKLOADS[name], with_joint=not suite and not args.no_joint)
+    if suite and not args.no_sub and world == 1:
+        # the other configurations, each with its own roofline, clocks and CPU baseline
+        free_device_memory()
+        medium = run_ours(args, S.WORKLOADS["medium"], with_joint=not args.no_joint)
+        free_device_memory()
+        sub = dict(medium=medium)
+        if medium is not None and "joint" in medium:
+            sub["joint"] = medium.pop("joint")
+        sub["fullgraph"] = run_fullgraph(args)
+        line["sub"] = sub
+    if line is not None:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        import torch.distributed as dist
+        dist.destroy_process_group()
 
 
 if __name__ == "__main__":

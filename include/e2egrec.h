@@ -327,11 +327,12 @@ int32_t e2egrec_joint_step_phase(const e2egrec_csr *graph, const e2egrec_mat *X,
  *                 without E2EGREC_JOINT_GATE); row-major [*pair_rows x width] in X's dtype, widths zdim, h1, h2, zdim,
  *                 zdim; *pair_rows = n_pairs rounded up to 128, rows >= n_pairs are zero.
  *   enc_h_offset  host size_t[n_hops], enc_rows host int64[n_hops]: the output of encoder layer l, row-major
- *                 [enc_rows[l] x d_out(l)]; only the first n_dst rows of the layer's block are meaningful. */
+ *                 [enc_rows[l] x d_out(l)]; only the first n_dst rows of the layer's block are meaningful.
+ *   counts_offset host size_t[n_hops]: the int32[4] counts {n_dst, n_src, n_edges, status} of the block of hop h+1. */
 int32_t e2egrec_joint_step_layout(const e2egrec_csr *graph, const e2egrec_mat *X, int32_t n_pairs, int32_t dense_dim,
                                   int32_t n_hops, const int32_t *fanouts, const e2egrec_mat *W_gnn,
                                   const e2egrec_mat *W_tower, uint32_t flags, size_t *tower_offset, size_t *enc_h_offset,
-                                  int64_t *enc_rows, int64_t *pair_rows);
+                                  int64_t *enc_rows, int64_t *pair_rows, size_t *counts_offset);
 
 /* Whole-graph neighbourhood aggregation without sampling (Sec. 3.1 Eq. 2 with S(u) = N(u); the
  * "complete graph" case of Sec. 4.1):  out[i] = (1/deg i) sum_{e in row i} X[indices[e]]  (0 for an

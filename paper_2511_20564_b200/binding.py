@@ -129,7 +129,7 @@ def lib():
         L.e2egrec_joint_step_layout.restype = C.c_int32
         L.e2egrec_joint_step_layout.argtypes = [C.POINTER(Csr), C.POINTER(Mat), C.c_int32, C.c_int32, C.c_int32, C.c_void_p,
                                                 C.POINTER(Mat), C.POINTER(Mat), C.c_uint32, C.c_void_p, C.c_void_p,
-                                                C.c_void_p, C.c_void_p]
+                                                C.c_void_p, C.c_void_p, C.c_void_p]
         L.e2egrec_graph_from_coo.restype = C.c_int32
         L.e2egrec_graph_from_coo.argtypes = [C.c_int64, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p,
                                              C.c_void_p, C.c_void_p, C.POINTER(C.c_size_t), C.c_void_p]
@@ -516,11 +516,13 @@ class JointStep:
 
     def activations(self):
         """Views into ws of what the last step left there (e2egrec_joint_step_layout): dict with the tower's z, a1, a2,
-        gate, z_fused ([pair_rows x width]) and `enc`, the list of encoder layer outputs ([rows x d_out])."""
+        gate, z_fused ([pair_rows x width]), `enc`, the list of encoder layer outputs ([rows x d_out]), and `counts`,
+        the int32[4] counts of every hop's block."""
         L = len(self.fanouts)
         tower, enc, rows, prow = (C.c_size_t * 5)(), (C.c_size_t * L)(), (C.c_int64 * L)(), C.c_int64(0)
+        cnt = (C.c_size_t * L)()
         _check(lib().e2egrec_joint_step_layout(C.byref(self._g), C.byref(self._x), self.n_pairs, self.dense_dim, L, self._f,
-                                               self._wg, self._wt, C.c_uint32(self.flags), tower, enc, rows, C.byref(prow)),
+                                               self._wg, self._wt, C.c_uint32(self.flags), tower, enc, rows, C.byref(prow), cnt),
                "e2egrec_joint_step_layout")
         es, dt = self.X.element_size(), self.X.dtype
         zdim, h1, h2 = self.W_tower[0].shape[1], self.W_tower[0].shape[0], self.W_tower[1].shape[0]
@@ -531,6 +533,7 @@ class JointStep:
         out = {k: view(tower[i], prow.value, w) for i, (k, w) in
                enumerate((("z", zdim), ("a1", h1), ("a2", h2), ("gate", zdim), ("z_fused", zdim)))}
         out["enc"] = [view(enc[l], rows[l], self.W_gnn[l].shape[0]) for l in range(L)]
+        out["counts"] = [self.ws[cnt[h]: cnt[h] + 16].view(torch.int32) for h in range(L)]   # {n_dst, n_src, n_edges, status}
         return out
 
 

@@ -194,6 +194,9 @@ __device__ inline void mbar_arrive(uint64_t *bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
+// kFuse: the gating / product-plus-term forms of the epilogue (TcFuse); the plain instantiation carries none of their
+// registers or branches.
+template <bool kFuse>
 __global__ void __launch_bounds__(kTnThreads)
 tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int k_blocks,
                   int stages, int nt, int n_tiles_n, uint32_t tmem_cols, int b_mn, TcEpilogue ep)
@@ -343,7 +346,7 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                         }
                     }
                 }
-                if (ep.fuse.gate_in) {
+                if (kFuse && ep.fuse.gate_in) {
                     // gating: the accumulator (+ bias) is the pre-activation; g = sigmoid(pre) with pre and g rounded to
                     // their storage type, the output is g * F and g itself goes to gate_out
                     uint32_t fw[16], gpk[16];
@@ -371,10 +374,12 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                             *reinterpret_cast<uint4 *>(grow + q * 8) = make_uint4(gpk[4 * q], gpk[4 * q + 1], gpk[4 * q + 2], gpk[4 * q + 3]);
                     }
                 } else {
-                uint32_t aw[16], bw[16];
-                if (ep.fuse.add_a) {                          // out = round(product) + a * b
-                    load_row32(ep.fuse.add_a + row * ep.fuse.ld_add_a + n0 + c, live, aw);
-                    load_row32(ep.fuse.add_b + row * ep.fuse.ld_add_b + n0 + c, live, bw);
+                uint32_t aw[16], bw[16];                      // dead (and removed) in the plain instantiation
+                if constexpr (kFuse) {
+                    if (ep.fuse.add_a) {                      // out = round(product) + a * b
+                        load_row32(ep.fuse.add_a + row * ep.fuse.ld_add_a + n0 + c, live, aw);
+                        load_row32(ep.fuse.add_b + row * ep.fuse.ld_add_b + n0 + c, live, bw);
+                    }
                 }
 #pragma unroll
                 for (int j = 0; j < 32; j += 2) {
@@ -386,9 +391,11 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                         if (col >= ep.scale_from) v0 *= rs;
                         if (col + 1 >= ep.scale_from) v1 *= rs;
                     }
-                    if (ep.fuse.add_a) {
-                        v0 = bf16_round(v0) + bf16_lo(aw[j >> 1]) * bf16_lo(bw[j >> 1]);
-                        v1 = bf16_round(v1) + bf16_hi(aw[j >> 1]) * bf16_hi(bw[j >> 1]);
+                    if constexpr (kFuse) {
+                        if (ep.fuse.add_a) {
+                            v0 = bf16_round(v0) + bf16_lo(aw[j >> 1]) * bf16_lo(bw[j >> 1]);
+                            v1 = bf16_round(v1) + bf16_hi(aw[j >> 1]) * bf16_hi(bw[j >> 1]);
+                        }
                     }
                     if (!live || !((mbits >> j) & 1u)) v0 = 0.f;
                     if (!live || !((mbits >> (j + 1)) & 1u)) v1 = 0.f;
@@ -505,13 +512,18 @@ bool launch_tn(const __nv_bfloat16 *A, int64_t rows, int k, int64_t lda, const _
     uint32_t tmem_cols = 64;                    // two accumulator buffers, each a power of two of columns >= nt
     while ((int)tmem_cols < 2 * nt) tmem_cols <<= 1;
     const size_t smem = (size_t)stages * (kTileM * kTileK * 2 + (size_t)nt * kTileK * 2) + 1024;
-    static bool attr_set[kMaxDevices] = {};
-    if (!raise_smem_limit(tc_gemm_tn_kernel, attr_set)) return false;
+    const bool fused = ep.fuse.gate_in || ep.fuse.add_a;
+    static bool attr_set[2][kMaxDevices] = {};
+    if (!(fused ? raise_smem_limit(tc_gemm_tn_kernel<true>, attr_set[1]) : raise_smem_limit(tc_gemm_tn_kernel<false>, attr_set[0])))
+        return false;
     const int n_tiles_n = n / nt;
     const int64_t tiles_cap = (rows / kTileM) * n_tiles_n;
     const unsigned grid = (unsigned)std::min<int64_t>(tiles_cap, sm_count());
     note_launch();
-    tc_gemm_tn_kernel<<<grid, kTnThreads, smem, st>>>(ma, mb, k_blocks, stages, nt, n_tiles_n, tmem_cols, b_mn ? 1 : 0, ep);
+    if (fused)
+        tc_gemm_tn_kernel<true><<<grid, kTnThreads, smem, st>>>(ma, mb, k_blocks, stages, nt, n_tiles_n, tmem_cols, b_mn ? 1 : 0, ep);
+    else
+        tc_gemm_tn_kernel<false><<<grid, kTnThreads, smem, st>>>(ma, mb, k_blocks, stages, nt, n_tiles_n, tmem_cols, b_mn ? 1 : 0, ep);
     return true;
 }
 

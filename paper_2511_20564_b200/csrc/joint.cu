@@ -658,9 +658,10 @@ extern "C" int32_t e2egrec_joint_step_phase(const e2egrec_csr *graph, const e2eg
 extern "C" int32_t e2egrec_joint_step_layout(const e2egrec_csr *graph, const e2egrec_mat *X, int32_t n_pairs, int32_t dense_dim,
                                              int32_t n_hops, const int32_t *fanouts, const e2egrec_mat *W_gnn,
                                              const e2egrec_mat *W_tower, uint32_t flags, size_t *tower_offset,
-                                             size_t *enc_h_offset, int64_t *enc_rows, int64_t *pair_rows)
+                                             size_t *enc_h_offset, int64_t *enc_rows, int64_t *pair_rows,
+                                             size_t *counts_offset)
 {
-    if (!tower_offset || !enc_h_offset || !enc_rows || !pair_rows) return E2EGREC_ERR_NULL;
+    if (!tower_offset || !enc_h_offset || !enc_rows || !pair_rows || !counts_offset) return E2EGREC_ERR_NULL;
     if (flags & ~(E2EGREC_JOINT_LINEAR | E2EGREC_JOINT_GATE)) return E2EGREC_ERR_ARG;
     JointPlan jp{};
     int32_t rc = make_plan(graph, X, n_pairs, dense_dim, n_hops, fanouts, W_gnn, W_tower, flags, jp);
@@ -671,6 +672,7 @@ extern "C" int32_t e2egrec_joint_step_layout(const e2egrec_csr *graph, const e2e
     rc = e2egrec_sage_ctx_layout(blocks, n_hops, X, W_gnn, cat_off, h_off, enc_rows);
     if (rc != E2EGREC_OK) return rc;
     for (int l = 0; l < n_hops; ++l) enc_h_offset[l] = jp.ctx_off + h_off[l];
+    for (int h = 0; h < n_hops; ++h) counts_offset[h] = jp.blk_off[h][0];
     tower_offset[0] = jp.z_off;
     tower_offset[1] = jp.a1_off;
     tower_offset[2] = jp.a2_off;

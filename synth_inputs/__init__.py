@@ -252,6 +252,10 @@ WORKLOADS = {
     "medium": Workload("medium", 200_000, 300_000, 10_000_000, 1.2, 1.2, 1, 128, 128, "bf16", (15, 10), 4096),
     "large": Workload("large", 20_000_000, 30_000_000, 1_000_000_000, 1.05, 1.05, 3, 256, 256, "bf16",
                       (20, 10, 5), 8192, q=80.0),
+    # `large` at one eighth of its graph (same law, model, batch and fanouts): the feature table (3.2 GB) is still far
+    # larger than L2, the whole workload holds under 5 GB on the device; used for counter captures and tests
+    "large_eighth": Workload("large_eighth", 2_500_000, 3_750_000, 125_000_000, 1.05, 1.05, 3, 256, 256, "bf16",
+                             (20, 10, 5), 8192, q=10.0),
     # the sampler shapes of the paper's experiments (Sec. 5.1: one hop x 100 neighbours, the default; two hops x 25, 15)
     # on the graph and features of `medium`; one GNN layer per hop
     "medium_1hop100": Workload("medium_1hop100", 200_000, 300_000, 10_000_000, 1.2, 1.2, 1, 128, 128, "bf16",
