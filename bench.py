@@ -479,6 +479,31 @@ def run_ours(args, w, with_joint):
     ev_a.record(); ev_b.record()
     torch.cuda.synchronize()
 
+    def leg_alone_ms(body, n):
+        """One leg of the step in a CUDA graph of its own, replayed n times back to back with nothing beside it."""
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=side):
+            body()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g.replay()
+        torch.cuda.synchronize()
+        a.record()
+        for _ in range(n):
+            g.replay()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / n
+
+    def hops_then_transposition():
+        sample_leg(1, transpose=False)
+        transpose_leg(1)
+
+    seeds_in2[1].copy_(seeds_dev[Wm])
+    n_leg = max(20, min(K, 200))
+    legs_ms = dict(forward_backward=leg_alone_ms(lambda: compute_leg(0), n_leg),
+                   hops=leg_alone_ms(lambda: sample_leg(1, transpose=False), n_leg),
+                   hops_and_transposition=leg_alone_ms(hops_then_transposition, n_leg))
+
     def run_step(i):
         """One step, eagerly and back to back (sampling, forward, backward of batch i)."""
         seeds_in2[0].copy_(seeds_dev[i], non_blocking=True)
@@ -716,7 +741,9 @@ def run_ours(args, w, with_joint):
                                            "table lives and a sparse update would consume them"),
                 gpu_launches=int(launches * repeats),
                 roofline=roof, aggregation=aggregation,
-                kernel_ms={TAP_NAMES[k].split(" (")[0]: v for k, v in tap_ms.items()})
+                kernel_ms={TAP_NAMES[k].split(" (")[0]: v for k, v in tap_ms.items()},
+                legs_alone_ms=dict(legs_ms, note="each leg of the step replayed alone in a CUDA graph of its own (one batch, "
+                                                 "nothing beside it); in the step the three legs run side by side"))
     if joint is not None:
         line["joint"] = joint
 

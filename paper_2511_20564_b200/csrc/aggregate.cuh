@@ -31,6 +31,8 @@ sage_aggregate_kernel(const T *__restrict__ Hsrc, int64_t ld, const int32_t *__r
     const int lane = threadIdx.x & 31;
     const int g = lane / LPR, c = lane % LPR;
     const int n_chunks = d / E;
+    pdl_launch_dependents();
+    pdl_wait();                                    // the kernel before this one in the stream has completed
     const int32_t n_dst = counts[CNT_DST];
     int64_t pad_end = ((int64_t)n_dst + 127) / 128 * 128;
     if (pad_end > cap_dst) pad_end = cap_dst;

@@ -5,6 +5,7 @@
 #include <unordered_map>
 #include <vector>
 #include <stdio.h>
+#include <stdlib.h>
 #include <string.h>
 
 #include "common.cuh"
@@ -29,6 +30,24 @@ int32_t check_launch(const char *what)
     return E2EGREC_ERR_CUDA;
 }
 
+bool pdl_enabled()
+{
+    static const bool on = []() {
+        const char *v = getenv("E2EGREC_PDL");
+        return v && *v && strcmp(v, "0") != 0;
+    }();
+    return on;
+}
+
+static bool helper_streams_enabled()
+{
+    static const bool on = []() {
+        const char *v = getenv("E2EGREC_NO_HELPER_STREAM");
+        return !(v && *v && strcmp(v, "0") != 0);
+    }();
+    return on;
+}
+
 // Helper streams: one per (device, caller's stream), created on first use and kept until the process ends, so calls
 // made on different streams (a sampling leg beside a compute leg, say) never meet on a common helper stream.
 // Deferred work (a block transposition left running by e2egrec_sample_khop) is tracked per device: whichever stream
@@ -49,6 +68,7 @@ static std::vector<SideStream *> g_pending[64];          // per device: helper s
 
 SideStream *SideStream::get(cudaStream_t caller)
 {
+    if (!helper_streams_enabled()) return nullptr;     // every entry point then stays on its caller's stream
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
     std::lock_guard<std::mutex> lock(g_side_mutex);

@@ -110,6 +110,8 @@ struct EpiPartial {
 static __global__ void splitk_reduce_kernel(const float *__restrict__ partial, int64_t n, int splits, int accumulate,
                                             float *__restrict__ out, const int32_t *rows_dev)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     int active = splits;
@@ -129,6 +131,8 @@ template <typename T>
 __global__ void relu_mask_kernel(const T *__restrict__ dH, int64_t ld_dh, const T *__restrict__ H, int64_t ld_h,
                                  const int32_t *n_dev, int64_t rows_alloc, int d, int relu, T *__restrict__ dZ)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t r = i / d;
     const int k = (int)(i - r * d);

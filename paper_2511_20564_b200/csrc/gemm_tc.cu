@@ -207,9 +207,7 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     __shared__ int abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int32_t m_valid = *ep.m_dev;
-    const int64_t n_work = (((int64_t)m_valid + kTileM - 1) / kTileM) * n_tiles_n;   // tiles wholly beyond *m_dev stay as they are
-    if ((int64_t)blockIdx.x >= n_work) return;
+    pdl_launch_dependents();                    // (with programmatic launches) the next kernel may set itself up beside this one
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
     const uint32_t a_bytes = kTileM * kTileK * 2, b_bytes = (uint32_t)nt * kTileK * 2;
     uint8_t *a_tiles = tiles;
@@ -239,8 +237,14 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_slot;
     const uint32_t buf_stride = tmem_cols >> 1;
+    // barriers and tensor memory are set up; global memory is touched only once the preceding kernel has completed
+    pdl_wait();
+    const int32_t m_valid = *ep.m_dev;
+    const int64_t n_work = (((int64_t)m_valid + kTileM - 1) / kTileM) * n_tiles_n;   // tiles wholly beyond *m_dev stay as they are
 
-    if (warp == 0) {
+    if ((int64_t)blockIdx.x >= n_work) {
+        // nothing for this CTA: straight to the release of its tensor memory
+    } else if (warp == 0) {
         if (lane == 0) {
             // ---- producer: TMA loads into the stage ring, k-block after k-block across tiles
             uint32_t g = 0;
@@ -521,9 +525,11 @@ bool launch_tn(const __nv_bfloat16 *A, int64_t rows, int k, int64_t lda, const _
     const unsigned grid = (unsigned)std::min<int64_t>(tiles_cap, sm_count());
     note_launch();
     if (fused)
-        tc_gemm_tn_kernel<true><<<grid, kTnThreads, smem, st>>>(ma, mb, k_blocks, stages, nt, n_tiles_n, tmem_cols, b_mn ? 1 : 0, ep);
+        launch_pdl(tc_gemm_tn_kernel<true>, dim3(grid), dim3(kTnThreads), smem, st, ma, mb, k_blocks, stages, nt, n_tiles_n, tmem_cols,
+                   b_mn ? 1 : 0, ep);
     else
-        tc_gemm_tn_kernel<false><<<grid, kTnThreads, smem, st>>>(ma, mb, k_blocks, stages, nt, n_tiles_n, tmem_cols, b_mn ? 1 : 0, ep);
+        launch_pdl(tc_gemm_tn_kernel<false>, dim3(grid), dim3(kTnThreads), smem, st, ma, mb, k_blocks, stages, nt, n_tiles_n, tmem_cols,
+                   b_mn ? 1 : 0, ep);
     return true;
 }
 
@@ -546,6 +552,8 @@ tc_gemm_rows_kernel(const __grid_constant__ CUtensorMap map_y, const __grid_cons
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int m0 = blockIdx.x * kTileM, n0 = blockIdx.y * nt;
+    pdl_launch_dependents();
+    pdl_wait();                                 // the preceding kernel of the stream has completed
     const int64_t m_valid = *m_dev;
     const int64_t total_blocks = (m_valid + kTileK - 1) / kTileK;
     // at least kMinSplitBlocks k-blocks per split: only the first ceil(total / per) splits do work and
@@ -748,7 +756,8 @@ bool tc_weight_grad(const __nv_bfloat16 *dY, int64_t rows, int m, const __nv_bfl
     if (!raise_smem_limit(tc_gemm_rows_kernel, attr_set)) return false;
     dim3 grid((unsigned)(m / kTileM), (unsigned)(n / nt), (unsigned)splits);
     note_launch();
-    tc_gemm_rows_kernel<<<grid, kThreads, smem, st>>>(my, mx, nt, tmem_cols, stages, m_dev, part, n, (int64_t)m * n, status);
+    launch_pdl(tc_gemm_rows_kernel, grid, dim3(kThreads), smem, st, my, mx, nt, tmem_cols, stages, m_dev, part, (int64_t)n,
+               (int64_t)m * n, status);
     return true;
 }
 

@@ -1,5 +1,6 @@
 // GraphSAGE forward / backward over sampled blocks: host orchestration and kernel dispatch.
 #include <algorithm>
+#include <stdlib.h>
 
 #include "aggregate.cuh"
 #include "common.cuh"
@@ -64,8 +65,8 @@ static void launch_sage_aggregate(const T *Hsrc, int64_t ld, const int32_t *nbr,
     const int64_t per_sm = rows >= (1ll << 20) ? 32 : 8;
     const unsigned grid = (unsigned)std::max<int64_t>(1, std::min<int64_t>(ceil_div(rows * 32, kAggThreads), 148 * per_sm));
     note_launch();
-    sage_aggregate_kernel<T, LPR, CPL><<<grid, kAggThreads, 0, st>>>(Hsrc, ld, nbr, self_ids, b.indptr, b.counts, cat, d,
-                                                                      (int32_t)rows);
+    launch_pdl(sage_aggregate_kernel<T, LPR, CPL>, dim3(grid), dim3(kAggThreads), 0, st, Hsrc, ld, nbr, self_ids, b.indptr,
+               b.counts, cat, d, (int32_t)rows);
 }
 
 template <typename T>
@@ -90,6 +91,21 @@ static bool dispatch_sage_aggregate(const T *Hsrc, int64_t ld, const int32_t *nb
 // lower overhead per entry wins there; measured on the 2 * 10^9-entry workload: 0.69 -> 0.63 ms)
 static inline int block_run_len(int64_t cap_edges) { return cap_edges >= (1ll << 21) ? 128 : 16; }
 constexpr int kDwSplits = 148;        // split-K factor of the weight-gradient product
+
+// A layer whose weight-gradient product may move this many bytes or more (by the capacity of its block) keeps that
+// product on the caller's stream.  Beside the input-gradient product and the transposed aggregation of such a layer it
+// only competes with them for the same HBM bandwidth and SM slots (measured on the 2 * 10^9-entry workload: the three
+// kernels take 0.18 + 0.25 + 0.47 ms one after the other and 1.0 ms overlapped); small layers, whose kernels are
+// bound by latency, gain from the overlap.  E2EGREC_DW_SERIAL_MB overrides the threshold (in MB).
+static size_t dw_serial_bytes()
+{
+    static const size_t v = []() {
+        const char *e = getenv("E2EGREC_DW_SERIAL_MB");
+        const long mb = (e && *e) ? atol(e) : 256;
+        return (size_t)(mb < 0 ? 0 : mb) << 20;
+    }();
+    return v;
+}
 
 // ------------------------------------------------------------------------------ forward
 template <typename T>
@@ -151,13 +167,13 @@ static int32_t forward_impl(const e2egrec_block *blocks, int32_t n_layers, const
 
 // ------------------------------------------------------------------------------ backward
 struct BackwardScratch {
-    size_t dz_off[2], dcat_off, seg_off, seg_bytes, part_off, wt_off, bytes;
+    size_t dz_off[2], dcat_off, seg_off, seg_bytes, chain_off, chain_bytes, part_off, wt_off, bytes;
 };
 
 static BackwardScratch plan_backward(const e2egrec_block *blocks, int32_t n_layers, const LayerPlan *plan, size_t es)
 {
     BackwardScratch s{};
-    size_t dz = 0, dcat = 0, part = 0, ht = 0, wt = 0;
+    size_t dz = 0, dcat = 0, part = 0, ht = 0, wt = 0, chain = 0;
     for (int l = 0; l < n_layers; ++l) {
         const LayerPlan &p = plan[l];
         dz = std::max(dz, (size_t)p.rows * p.d_out * es);
@@ -165,6 +181,7 @@ static BackwardScratch plan_backward(const e2egrec_block *blocks, int32_t n_laye
         part = std::max(part, (size_t)kDwSplits * p.d_out * 2 * p.d_in * sizeof(float));
         wt = std::max(wt, (size_t)p.d_out * 2 * p.d_in * es);
         ht = std::max(ht, seg_scratch_carve(blocks[p.block].cap_edges, block_run_len(blocks[p.block].cap_edges), p.d_in, es, nullptr).bytes);
+        chain = std::max(chain, seg_chain_bytes(blocks[p.block].cap_edges, block_run_len(blocks[p.block].cap_edges), p.d_in, es));
     }
     size_t off = 0;
     auto take = [&](size_t b) { size_t o = off; off += align_up(b, 256); return o; };
@@ -173,6 +190,8 @@ static BackwardScratch plan_backward(const e2egrec_block *blocks, int32_t n_laye
     s.dcat_off = take(dcat);
     s.seg_off = take(ht);
     s.seg_bytes = ht;
+    s.chain_off = take(chain);
+    s.chain_bytes = chain;
     s.part_off = take(part);
     s.wt_off = take(wt);
     s.bytes = off;
@@ -190,15 +209,17 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
     T *dcat = reinterpret_cast<T *>(scratch + bs.dcat_off);
     float *part = reinterpret_cast<float *>(scratch + bs.part_off);
 
+    // counters of the transposed aggregation (one per window of a block's entry stream); every launch leaves them zero
+    cudaMemsetAsync(scratch + bs.chain_off, 0, bs.chain_bytes, st);
     // gradient entering the top layer, masked by its activation
     {
         const LayerPlan &p = plan[n_layers - 1];
         const e2egrec_block &b = blocks[p.block];
         const int64_t total = p.rows * p.d_out;
         note_launch();
-        relu_mask_kernel<T><<<(unsigned)std::max<int64_t>(1, ceil_div(total, 256)), 256, 0, st>>>(
-            static_cast<const T *>(dH_out->data), dH_out->ld, reinterpret_cast<const T *>(ctx + p.h_off), p.d_out,
-            &b.counts[CNT_DST], p.rows, p.d_out, act ? act[n_layers - 1] : 1, dz_buf[(n_layers - 1) & 1]);
+        launch_pdl(relu_mask_kernel<T>, dim3((unsigned)std::max<int64_t>(1, ceil_div(total, 256))), dim3(256), 0, st,
+                   static_cast<const T *>(dH_out->data), dH_out->ld, reinterpret_cast<const T *>(ctx + p.h_off), (int64_t)p.d_out,
+                   &b.counts[CNT_DST], p.rows, p.d_out, act ? act[n_layers - 1] : 1, dz_buf[(n_layers - 1) & 1]);
     }
     SideStream *side = SideStream::get(st);
     cudaEvent_t dz_free[2] = {nullptr, nullptr};
@@ -213,7 +234,8 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
         // this call reads dW, so it runs on the helper stream beside the dCat product and the transposed
         // aggregation; `dz_free` holds the event after which the helper stream no longer reads a dZ buffer.
         cudaStream_t ws = st;
-        if (side) {
+        const bool dw_beside = side && (size_t)p.rows * (p.d_out + two_d) * sizeof(T) < dw_serial_bytes();
+        if (dw_beside) {
             side->fork(st);
             ws = side->stream;
         }
@@ -233,8 +255,8 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
         {
             const int64_t n = (int64_t)p.d_out * two_d;
             note_launch();
-            splitk_reduce_kernel<<<(unsigned)ceil_div(n, 256), 256, 0, ws>>>(part, n, kDwSplits, accumulate, dW[l],
-                                                                             dw_done ? n_dst : nullptr);
+            launch_pdl(splitk_reduce_kernel, dim3((unsigned)ceil_div(n, 256)), dim3(256), 0, ws, part, n, kDwSplits, accumulate,
+                       dW[l], dw_done ? n_dst : nullptr);
         }
         if (l == 0) tap_end(TAP_DW_OUTER, ws);
         if (dbias && dbias[l]) {
@@ -242,7 +264,7 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
             colsum_kernel<T><<<(unsigned)ceil_div(p.d_out, 32), 256, 0, ws>>>(dz, p.d_out, n_dst, p.d_out, accumulate,
                                                                              dbias[l]);
         }
-        if (side) {
+        if (dw_beside) {
             dz_free[l & 1] = side->event();
             cudaEventRecord(dz_free[l & 1], side->stream);
         }
@@ -288,7 +310,8 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
             o.mask = nullptr;
         }
         if (l == 0) tap_begin(TAP_AGG_BWD_OUTER, st);
-        const SegScratch sc = seg_scratch_carve(b.cap_edges, block_run_len(b.cap_edges), p.d_in, dtype_size(X->dtype), scratch + bs.seg_off);
+        SegScratch sc = seg_scratch_carve(b.cap_edges, block_run_len(b.cap_edges), p.d_in, dtype_size(X->dtype), scratch + bs.seg_off);
+        sc.chain_cnt = reinterpret_cast<int32_t *>(scratch + bs.chain_off);
         const bool seg_ok = dispatch_seg_reduce<T, int32_t, false>(dcat + p.d_in, two_d, b.csc_ptr, b.csc_row, &b.counts[CNT_SRC], 0,
                                                                    b.cap_src, nullptr, block_run_len(b.cap_edges), p.d_in, X->dtype,
                                                                    b.csc_col, sc, o, st);

@@ -19,13 +19,14 @@
 //   (all threads of a block share one such sum), and extra blocks write fin(0) for segments without entries.
 #pragma once
 
+#include <stdlib.h>
+
 #include <algorithm>
 
 #include "aggregate.cuh"
 
 namespace e2egrec {
 
-constexpr int kSegRing = 8;        // entries requested ahead in the ring form of seg_run_kernel
 
 // runs per window = lane groups per block of seg_run_kernel
 inline int seg_runs_per_window(int d, size_t elem_size) { return kAggThreads / row_shape_bytes((int64_t)d * elem_size).lpr; }
@@ -37,7 +38,17 @@ struct SegScratch {
     int64_t cap_runs, n_windows;
     int runs_per_window;
     size_t bytes;
+    // One counter per window, for callers of the sampled-block form: nullptr (the default) keeps the two-kernel form.
+    // The caller sets it to n_windows zeroed int32 (seg_chain_bytes) before the first launch that uses them; every
+    // launch leaves them zero again.
+    int32_t *chain_cnt;
 };
+
+inline size_t seg_chain_bytes(int64_t cap_entries, int run_len, int d, size_t elem_size)
+{
+    const int64_t runs = ceil_div(cap_entries > 0 ? cap_entries : 1, run_len);
+    return align_up((size_t)ceil_div(runs, seg_runs_per_window(d, elem_size)) * sizeof(int32_t), 256);
+}
 
 inline SegScratch seg_scratch_carve(int64_t cap_entries, int run_len, int d, size_t elem_size, void *base)
 {
@@ -106,13 +117,186 @@ __device__ __noinline__ SegStep seg_advance(const PtrT *__restrict__ ptr, int64_
     return SegStep{s, end};
 }
 
-__device__ __forceinline__ void cp_async16(void *smem_dst, const void *gmem_src)
+// Finishes segment `seg` whose entries (and self row) sum to acc: scale, round to the storage type, mask, store.
+template <typename T, int LPR, int CPL, int kExtra>
+__device__ __forceinline__ void seg_store_row(const SegOut<T> &o, int32_t seg, float inv, const float (&acc)[CPL][Chunk<T>::kElems],
+                                              const uint4 (&mrow)[CPL], int c, int n_chunks)
 {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gmem_src)
-                 : "memory");
+    constexpr int E = Chunk<T>::kElems;
+#pragma unroll
+    for (int q = 0; q < CPL; ++q) {
+        const int ch = c + q * LPR;
+        if (ch < n_chunks) {
+            float r[E];
+#pragma unroll
+            for (int e = 0; e < E; ++e) r[e] = to_float<T>(from_float<T>(acc[q][e] * inv));   // inv = 1 without mean / scale
+            if (kExtra == 2 && o.mask) {
+                float m[E];
+                Chunk<T>::unpack(mrow[q], m);
+#pragma unroll
+                for (int e = 0; e < E; ++e)
+                    if (!(m[e] > 0.f)) r[e] = 0.f;
+            }
+            Chunk<T>::store(o.out + (int64_t)seg * o.ld_out + ch * E, r);
+        }
+    }
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
+// A lane group has just written its window's part (a row of head2 or tail2) of segment sg, which is cut by window
+// boundaries.  The parts of a segment are counted in chain_cnt[its first window]; the group that brings the count to
+// the number of windows the segment spans adds the parts in window order -- tail2[first], head2[first + 1], ... -- and
+// stores the finished row, so the sum does not depend on which group closes it.  No group waits for another.
+template <typename T, int LPR, int kExtra>
+__device__ __forceinline__ void seg_chain_arrive(int32_t sg, const int32_t *__restrict__ ptr, int run_len, int d, int c, int n_chunks,
+                                                 const float *head2, const float *tail2, int32_t *chain_cnt, const SegOut<T> &o)
+{
+    constexpr int E = Chunk<T>::kElems;
+    constexpr int RB = kAggThreads / LPR;
+    const int32_t beg = ptr[sg], end = ptr[sg + 1];
+    const int32_t first = (beg / run_len) / RB, last = ((end - 1) / run_len) / RB;
+    const int group_lane0 = (threadIdx.x & 31) / LPR * LPR;
+    const unsigned gmask = LPR >= 32 ? 0xffffffffu : (((1u << (LPR & 31)) - 1u) << group_lane0);
+    __threadfence();                               // this lane's share of the part is visible before the count moves
+    __syncwarp(gmask);
+    int32_t old = 0;
+    if (c == 0) old = atomicAdd(&chain_cnt[first], 1);
+    old = __shfl_sync(gmask, old, group_lane0);
+    if (old != last - first) return;               // other windows' parts are still to come: their group will close it
+    if (c == 0) chain_cnt[first] = 0;              // idle again for the next launch
+    __threadfence();
+    float acc[1][E];
+    uint4 mrow[1] = {make_uint4(0, 0, 0, 0)};
+#pragma unroll
+    for (int e = 0; e < E; ++e) acc[0][e] = 0.f;
+    if (c < n_chunks) {
+        const float *t = tail2 + (int64_t)first * d + c * E;
+#pragma unroll
+        for (int e = 0; e < E; e += 4) {
+            const float4 x = __ldcg(reinterpret_cast<const float4 *>(t + e));
+            acc[0][e] = x.x; acc[0][e + 1] = x.y; acc[0][e + 2] = x.z; acc[0][e + 3] = x.w;
+        }
+        for (int32_t p0 = first + 1; p0 <= last; p0 += 4) {
+            float4 x[4][E / 4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int e = 0; e < E / 4; ++e)
+                    x[u][e] = p0 + u <= last ? __ldcg(reinterpret_cast<const float4 *>(head2 + (int64_t)(p0 + u) * d + c * E + 4 * e))
+                                             : make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+#pragma unroll
+                for (int e = 0; e < E / 4; ++e) {
+                    acc[0][4 * e] += x[u][e].x; acc[0][4 * e + 1] += x[u][e].y;
+                    acc[0][4 * e + 2] += x[u][e].z; acc[0][4 * e + 3] += x[u][e].w;
+                }
+        }
+        if (kExtra == 2 && o.mask) mrow[0] = Chunk<T>::load_raw(o.mask + (int64_t)sg * o.ld_mask + c * E);
+    }
+    seg_store_row<T, LPR, 1, kExtra>(o, sg, 1.0f, acc, mrow, c, n_chunks);
+}
+
+// Second half of a run kernel: every lane group has left the parts of the segments that its run cuts in sh_head /
+// sh_tail (head_seg / head_ends / tail_seg say which); after a block barrier the runs of the block (its window) are
+// joined.  The group of run rl acts where a chain of parts of one cut segment ends: at the run that holds the
+// segment's end, or at the window's last run.  It walks back to the run in which the segment began (if that run is in
+// the window) and adds the parts forward, in run order.  A segment that also leaves the window leaves one row in
+// head2[window] or tail2[window] and a record in win_info[window].  Called by all threads of the block.
+// With chain_cnt (sampled-block form, CPL = 1, no mean / scale) nothing is left for a second kernel: a group that has
+// written a window's part of a cut segment counts it in chain_cnt[first window of the segment]; the group whose part
+// completes the count adds all parts of the segment in window order and stores the row (seg_chain_arrive).
+template <typename T, typename PtrT, int LPR, int CPL, int kExtra>
+__device__ __forceinline__ void seg_join_window(float *sh_head, float *sh_tail, int4 *sh_info, int32_t *sh_win, int rl, int c,
+                                                int n_chunks, int d, int32_t head_seg, int32_t head_ends, int32_t tail_seg,
+                                                const PtrT *__restrict__ ptr, float *__restrict__ head2, float *__restrict__ tail2,
+                                                int4 *__restrict__ win_info, const SegOut<T> &o, int32_t *chain_cnt = nullptr,
+                                                int run_len = 0)
+{
+    constexpr int E = Chunk<T>::kElems;
+    constexpr int RB = kAggThreads / LPR;
+    constexpr int ROW = LPR * CPL * E;
+    if (c == 0) sh_info[rl] = make_int4(head_seg, head_ends, tail_seg, 0);
+    if (threadIdx.x < 4) sh_win[threadIdx.x] = threadIdx.x == 1 || threadIdx.x == 3 ? 0 : -1;
+    __syncthreads();
+
+    // ---- join the runs of the window.  The group of run rl acts where a chain of parts of one cut segment
+    // ends: at the run that holds the segment's end, or at the window's last run.  It walks back to the run in
+    // which the segment began (if that run is in the window) and adds the parts forward, in run order.
+    {
+        const bool last_run = rl == RB - 1;
+        if (head_seg >= 0 && (head_ends || last_run)) {
+            int first = rl - 1;                    // the run whose tail begins the chain, or -1: began before the window
+            while (first >= 0 && sh_info[first].z != head_seg) --first;
+            float acc[CPL][E];
+            uint4 mrow[CPL];
+#pragma unroll
+            for (int q = 0; q < CPL; ++q) {
+                const int ch = c + q * LPR;
+                mrow[q] = make_uint4(0, 0, 0, 0);
+#pragma unroll
+                for (int e = 0; e < E; ++e) acc[q][e] = 0.f;
+                if (first >= 0) {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) acc[q][e] = sh_tail[first * ROW + ch * E + e];
+                }
+                for (int j = first + 1; j <= rl; ++j) {
+#pragma unroll
+                    for (int e = 0; e < E; ++e) acc[q][e] += sh_head[j * ROW + ch * E + e];
+                }
+            }
+            if (first >= 0 && head_ends) {
+                const int64_t sg = head_seg;
+                float inv = 1.0f;
+                if (o.mean) inv = 1.0f / (float)((int64_t)ptr[sg + 1] - (int64_t)ptr[sg]);
+                else if (o.seg_scale) inv = o.seg_scale[sg];
+                if (kExtra == 2 && o.mask) {
+#pragma unroll
+                    for (int q = 0; q < CPL; ++q) {
+                        const int ch = c + q * LPR;
+                        if (ch < n_chunks) mrow[q] = Chunk<T>::load_raw(o.mask + sg * o.ld_mask + ch * E);
+                    }
+                }
+                seg_store_row<T, LPR, CPL, kExtra>(o, head_seg, inv, acc, mrow, c, n_chunks);
+            } else {
+                // leaves the window: towards earlier windows (head2) or, begun here and still open, later ones (tail2)
+                float *dst = (first >= 0 ? tail2 : head2) + (int64_t)blockIdx.x * d;
+#pragma unroll
+                for (int q = 0; q < CPL; ++q) {
+                    const int ch = c + q * LPR;
+                    if (ch < n_chunks) {
+#pragma unroll
+                        for (int e = 0; e < E; e += 4)
+                            *reinterpret_cast<float4 *>(dst + ch * E + e) = make_float4(acc[q][e], acc[q][e + 1], acc[q][e + 2], acc[q][e + 3]);
+                    }
+                }
+                if (c == 0) {
+                    if (first >= 0) sh_win[2] = head_seg;
+                    else { sh_win[0] = head_seg; sh_win[1] = head_ends; }
+                }
+                if constexpr (CPL == 1 && sizeof(PtrT) == 4)
+                    if (chain_cnt) seg_chain_arrive<T, LPR, kExtra>(head_seg, ptr, run_len, d, c, n_chunks, head2, tail2, chain_cnt, o);
+            }
+        }
+        if (last_run && tail_seg >= 0) {           // a segment that begins in the window's last run and continues
+            float *dst = tail2 + (int64_t)blockIdx.x * d;
+#pragma unroll
+            for (int q = 0; q < CPL; ++q) {
+                const int ch = c + q * LPR;
+                if (ch < n_chunks) {
+#pragma unroll
+                    for (int e = 0; e < E; e += 4)
+                        *reinterpret_cast<float4 *>(dst + ch * E + e) = *reinterpret_cast<const float4 *>(sh_tail + rl * ROW + ch * E + e);
+                }
+            }
+            if (c == 0) sh_win[2] = tail_seg;
+            if constexpr (CPL == 1 && sizeof(PtrT) == 4)
+                if (chain_cnt) seg_chain_arrive<T, LPR, kExtra>(tail_seg, ptr, run_len, d, c, n_chunks, head2, tail2, chain_cnt, o);
+        }
+    }
+    if (chain_cnt) return;                        // no record: nobody reads it
+    __syncthreads();
+    if (threadIdx.x == 0) win_info[blockIdx.x] = make_int4(sh_win[0], sh_win[1], sh_win[2], 0);
+}
 
 // Shared memory of seg_run_kernel (dynamic): head and tail rows of the block's runs, fp32, one row of
 // LPR*CPL*E floats per run, then one record per run.
@@ -127,11 +311,7 @@ constexpr size_t seg_run_smem_bytes()
 // kInFlight: gathered rows a lane group requests before it adds any.  Four suit the short streams of a sampled
 // block (few resident warps, latency hidden inside the thread); on streams that fill the machine two are faster,
 // because the smaller register footprint keeps five blocks resident per SM instead of three.
-// kRing > 0 (sampled blocks with a self row, 16-byte chunk per lane): the gathered chunk of every entry, and the self
-// chunk where a segment begins, are requested kRing entries ahead with cp.async into a ring in shared memory (each
-// thread reads back only what it requested itself, so the ring needs no barrier); the bytes in flight then no longer
-// occupy registers and do not stop at the four rows of a batch.
-template <typename T, typename PtrT, int LPR, int CPL, bool kWeight, int kExtra, int kInFlight, int kRing = 0>
+template <typename T, typename PtrT, int LPR, int CPL, bool kWeight, int kExtra, int kInFlight>
 __global__ void __launch_bounds__(kAggThreads, (kInFlight <= 2 && !kExtra) ? 5 : 1)
 seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__ ptr, const int32_t *__restrict__ idx,
                const int32_t *n_seg_dev, int64_t n_seg_host, const float *__restrict__ w, int run_len, int d,
@@ -153,6 +333,8 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
     const int rl = threadIdx.x / LPR;              // run within the block
     const int n_chunks = d / E;
     const int64_t run = (int64_t)blockIdx.x * RB + rl;
+    pdl_launch_dependents();
+    pdl_wait();                                    // the kernel before this one in the stream has completed
     const int64_t n_seg = n_seg_dev ? (int64_t)*n_seg_dev : n_seg_host;
     const int64_t total = n_seg > 0 ? (int64_t)ptr[n_seg] : 0;
     const int64_t k0 = run * run_len;
@@ -266,36 +448,12 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
             }
         };
 
-        static_assert(kRing == 0 || (CPL == 1 && !kWeight && kExtra == 1 && kRing >= U), "ring form: one chunk per lane, self rows only");
-        constexpr int kSlot = kAggThreads * 16;               // bytes of one ring slot (one 16-byte chunk per thread)
-        uint8_t *ring_g = reinterpret_cast<uint8_t *>(sh_info + RB) + threadIdx.x * 16;     // gathered chunks
-        uint8_t *ring_s = ring_g + (kRing > 0 ? kRing : 1) * kSlot;                            // self chunks
-        // requests entry r (same tests as the sums below make when they read the slot back)
-        auto issue = [&](int r) {
-            if (kRing > 0) {
-                if (r < len && c < n_chunks) {
-                    const int slot = r % (kRing > 0 ? kRing : 1);
-                    cp_async16(ring_g + slot * kSlot, in + (int64_t)idx0[r] * ld_in + c * E);
-                    const int32_t sg = seg0[r];
-                    const bool st = r == 0 || sg != seg0[r - 1];
-                    if (st && (r != 0 || first_begins) && sg < n_self)
-                        cp_async16(ring_s + slot * kSlot, o.self + (int64_t)sg * o.ld_self + c * E);
-                }
-                cp_async_commit();
-            }
-        };
-        if (kRing > 0) {
-#pragma unroll
-            for (int r = 0; r < (kRing > 0 ? kRing : 1); ++r) issue(r);
-        }
-
         classify(0);
         for (int r0 = 0; r0 < len; r0 += U) {
             int32_t seg_c[U];
             bool start_c[U];
             float wt[U];
             uint4 v[U][CPL], sv[kExtra ? U : 1][CPL], mv[kExtra == 2 ? U : 1][CPL];
-            if (kRing > 0) cp_async_wait<(kRing > U ? kRing - U : 0)>();       // the entries of this batch have landed
 #pragma unroll
             for (int u = 0; u < U; ++u) {
                 seg_c[u] = seg_n[u];
@@ -304,17 +462,6 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
                 const bool live = r0 + u < len;
                 const int32_t id = id_n[u];
                 if (kWeight && live) wt[u] = w[id];
-                if (kRing > 0) {
-                    const int slot = (r0 + u) % (kRing > 0 ? kRing : 1);
-                    v[u][0] = make_uint4(0, 0, 0, 0);
-                    sv[u][0] = make_uint4(0, 0, 0, 0);
-                    if (live && c < n_chunks) {
-                        v[u][0] = *reinterpret_cast<const uint4 *>(ring_g + slot * kSlot);
-                        if (start_c[u] && (r0 + u != 0 || first_begins) && seg_c[u] < n_self)
-                            sv[u][0] = *reinterpret_cast<const uint4 *>(ring_s + slot * kSlot);
-                    }
-                }
-                if (kRing == 0) {
 #pragma unroll
                 for (int q = 0; q < CPL; ++q) {
                     const int ch = c + q * LPR;
@@ -331,7 +478,6 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
                                 mv[u][q] = Chunk<T>::load_raw(o.mask + (int64_t)seg_c[u] * o.ld_mask + ch * E);
                         }
                     }
-                }
                 }
             }
             if (r0 + U < len) classify(r0 + U);
@@ -370,90 +516,170 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
                     }
                 }
             }
-            if (kRing > 0) {                                  // the slots just read take the entries kRing further on
-#pragma unroll
-                for (int u = 0; u < U; ++u) issue(r0 + (kRing > 0 ? kRing : 1) + u);
-            }
         }
-        if (kRing > 0) cp_async_wait<0>();
         emit(seg0 ? last_ends : rel_end <= len, len);
     }
-    if (c == 0) sh_info[rl] = make_int4(head_seg, head_ends, tail_seg, 0);
-    if (threadIdx.x < 4) sh_win[threadIdx.x] = threadIdx.x == 1 || threadIdx.x == 3 ? 0 : -1;
-    __syncthreads();
+    seg_join_window<T, PtrT, LPR, CPL, kExtra>(sh_head, sh_tail, sh_info, sh_win, rl, c, n_chunks, d, head_seg, head_ends, tail_seg, ptr,
+                                               head2, tail2, win_info, o);
+}
 
-    // ---- join the runs of the window.  The group of run rl acts where a chain of parts of one cut segment
-    // ends: at the run that holds the segment's end, or at the window's last run.  It walks back to the run in
-    // which the segment began (if that run is in the window) and adds the parts forward, in run order.
-    {
-        const bool last_run = rl == RB - 1;
-        if (head_seg >= 0 && (head_ends || last_run)) {
-            int first = rl - 1;                    // the run whose tail begins the chain, or -1: began before the window
-            while (first >= 0 && sh_info[first].z != head_seg) --first;
-            float acc[CPL][E];
-            uint4 mrow[CPL];
+// ------------------------------------------------------------------------------------ the sampled-block form
+// seg_run_kernel for the transposed aggregation of a sampled block, where the entry -> segment array exists, offsets
+// are 32-bit, a row is one 16-byte chunk per lane, entries carry no weight and the output is the plain sum plus the
+// self row (kMask: zeroed where the mask row is not positive).  Same runs, same order of additions, same records for
+// the join and for seg_final_kernel, hence the same bits as the general kernel; but the walk over the run is written
+// for this case alone (entry ids and segment ids fetched four at a time, 32-bit arithmetic, no scale, no walk of the
+// offsets), which takes the instructions per entry from ~110 to ~35: with two entries per segment on average the
+// general kernel was bound by instruction issue, not by memory.
+template <typename T, int LPR, bool kMask, int U = 4, int kMinBlocks = (kMask ? 3 : 4)>
+__global__ void __launch_bounds__(kAggThreads, kMinBlocks)
+seg_run_block_kernel(const T *__restrict__ in, int64_t ld_in, const int32_t *__restrict__ ptr, const int32_t *__restrict__ idx,
+                     const int32_t *__restrict__ seg_of, const int32_t *__restrict__ n_seg_dev, int run_len, int d,
+                     float *__restrict__ head2, float *__restrict__ tail2, int4 *__restrict__ win_info, int64_t cap_runs,
+                     int32_t *__restrict__ chain_cnt, SegOut<T> o)
+{
+    constexpr int E = Chunk<T>::kElems;
+    constexpr int RB = kAggThreads / LPR;
+    constexpr int ROW = LPR * E;
+    constexpr int kExtra = kMask ? 2 : 1;
+    extern __shared__ float4 seg_smem[];
+    float *sh_head = reinterpret_cast<float *>(seg_smem);
+    float *sh_tail = sh_head + RB * ROW;
+    int4 *sh_info = reinterpret_cast<int4 *>(sh_tail + RB * ROW);
+    __shared__ int32_t sh_win[4];
+
+    const int c = threadIdx.x % LPR;
+    const int rl = threadIdx.x / LPR;
+    const int n_chunks = d / E;
+    const int64_t run = (int64_t)blockIdx.x * RB + rl;
+    pdl_launch_dependents();
+    pdl_wait();                                    // the kernel before this one in the stream has completed
+    const int32_t n_seg = *n_seg_dev;
+    const int32_t total = n_seg > 0 ? ptr[n_seg] : 0;
+    const int64_t k0 = run * run_len;
+    int32_t head_seg = -1, head_ends = 0, tail_seg = -1;
+    // a window that lies wholly beyond the stream (grids are sized for capacities) has no run work and no join, but
+    // still takes its share of the segments without entries below
+    const bool live_window = (int64_t)blockIdx.x * RB * run_len < total;
+
+    if (run < cap_runs && k0 < total) {
+        const int len = (int)min((int64_t)run_len, (int64_t)total - k0);
+        const int32_t *__restrict__ idx0 = idx + k0;
+        const int32_t *__restrict__ seg0 = seg_of + k0;
+        const int32_t n_self = o.n_self ? *o.n_self : n_seg;
+        const bool lane_on = c < n_chunks;
+        const T *__restrict__ in_c = in + c * E;
+        const T *__restrict__ self_c = o.self + c * E;
+        const T *__restrict__ mask_c = kMask ? o.mask + c * E : nullptr;
+        const bool vec_ok = ((reinterpret_cast<uintptr_t>(idx0) | reinterpret_cast<uintptr_t>(seg0)) & 15u) == 0;
+        const bool first_begins = k0 == 0 || seg0[-1] != seg0[0];
+        const bool last_ends = k0 + len == total || seg0[len] != seg0[len - 1];
+
+        int32_t cur_seg = -1, last_sg = -1;
+        bool cur_begins = false;
+        float acc[1][E];
+        uint4 cur_mask[1] = {make_uint4(0, 0, 0, 0)};
 #pragma unroll
-            for (int q = 0; q < CPL; ++q) {
-                const int ch = c + q * LPR;
-                mrow[q] = make_uint4(0, 0, 0, 0);
+        for (int e = 0; e < E; ++e) acc[0][e] = 0.f;
+
+        // closes the current segment: a whole segment goes to the output, a part of one to the block's shared rows
+        auto emit = [&](bool ended) {
+            if (cur_begins && ended) {
+                seg_store_row<T, LPR, 1, kExtra>(o, cur_seg, 1.0f, acc, cur_mask, c, n_chunks);
+            } else {
+                float *dst = (cur_begins ? sh_tail : sh_head) + rl * ROW + c * E;
 #pragma unroll
-                for (int e = 0; e < E; ++e) acc[q][e] = 0.f;
-                if (first >= 0) {
+                for (int e = 0; e < E; e += 4) *reinterpret_cast<float4 *>(dst + e) = make_float4(acc[0][e], acc[0][e + 1], acc[0][e + 2], acc[0][e + 3]);
+                if (cur_begins) tail_seg = cur_seg;
+                else { head_seg = cur_seg; head_ends = ended ? 1 : 0; }
+            }
+        };
+
+        for (int r0 = 0; r0 < len; r0 += U) {
+            int32_t id[U], sg[U];
+            if (vec_ok && r0 + U <= len) {
 #pragma unroll
-                    for (int e = 0; e < E; ++e) acc[q][e] = sh_tail[first * ROW + ch * E + e];
+                for (int q = 0; q < U / 4; ++q) {
+                    const int4 a = __ldg(reinterpret_cast<const int4 *>(idx0 + r0) + q);
+                    const int4 b = __ldg(reinterpret_cast<const int4 *>(seg0 + r0) + q);
+                    id[4 * q] = a.x; id[4 * q + 1] = a.y; id[4 * q + 2] = a.z; id[4 * q + 3] = a.w;
+                    sg[4 * q] = b.x; sg[4 * q + 1] = b.y; sg[4 * q + 2] = b.z; sg[4 * q + 3] = b.w;
                 }
-                for (int j = first + 1; j <= rl; ++j) {
+            } else {
 #pragma unroll
-                    for (int e = 0; e < E; ++e) acc[q][e] += sh_head[j * ROW + ch * E + e];
+                for (int u = 0; u < U; ++u) {
+                    const bool live = r0 + u < len;
+                    id[u] = live ? __ldg(idx0 + r0 + u) : 0;
+                    sg[u] = live ? __ldg(seg0 + r0 + u) : -1;
                 }
             }
-            if (first >= 0 && head_ends) {
-                const int64_t sg = head_seg;
-                float inv = 1.0f;
-                if (o.mean) inv = 1.0f / (float)((int64_t)ptr[sg + 1] - (int64_t)ptr[sg]);
-                else if (o.seg_scale) inv = o.seg_scale[sg];
-                if (kExtra == 2 && o.mask) {
+            uint4 v[U], sv[U], mv[kMask ? U : 1];
+            bool start[U];
 #pragma unroll
-                    for (int q = 0; q < CPL; ++q) {
-                        const int ch = c + q * LPR;
-                        if (ch < n_chunks) mrow[q] = Chunk<T>::load_raw(o.mask + sg * o.ld_mask + ch * E);
+            for (int u = 0; u < U; ++u) {
+                const bool live = r0 + u < len;
+                start[u] = live && sg[u] != (u == 0 ? last_sg : sg[u - 1]);      // entry 0 always starts (last_sg = -1)
+                v[u] = make_uint4(0, 0, 0, 0);
+                sv[u] = make_uint4(0, 0, 0, 0);
+                if (kMask) mv[u] = make_uint4(0, 0, 0, 0);
+                if (live && lane_on) {
+                    v[u] = Chunk<T>::load_raw(in_c + (int64_t)id[u] * ld_in);
+                    if (start[u]) {
+                        if ((r0 + u != 0 || first_begins) && sg[u] < n_self) sv[u] = Chunk<T>::load_raw(self_c + (int64_t)sg[u] * o.ld_self);
+                        if (kMask) mv[u] = Chunk<T>::load_raw(mask_c + (int64_t)sg[u] * o.ld_mask);
                     }
                 }
-                finish(head_seg, inv, acc, mrow);
-            } else {
-                // leaves the window: towards earlier windows (head2) or, begun here and still open, later ones (tail2)
-                float *dst = (first >= 0 ? tail2 : head2) + (int64_t)blockIdx.x * d;
+            }
+            last_sg = sg[U - 1];
 #pragma unroll
-                for (int q = 0; q < CPL; ++q) {
-                    const int ch = c + q * LPR;
-                    if (ch < n_chunks) {
-#pragma unroll
-                        for (int e = 0; e < E; e += 4)
-                            *reinterpret_cast<float4 *>(dst + ch * E + e) = make_float4(acc[q][e], acc[q][e + 1], acc[q][e + 2], acc[q][e + 3]);
+            for (int u = 0; u < U; ++u) {
+                if (r0 + u < len) {
+                    if (start[u]) {
+                        if (cur_seg >= 0) emit(true);
+                        cur_seg = sg[u];
+                        cur_begins = r0 + u != 0 || first_begins;
+                        Chunk<T>::unpack(sv[u], acc[0]);                 // the self row (zeros if there is none)
+                        if (kMask) cur_mask[0] = mv[u];
                     }
-                }
-                if (c == 0) {
-                    if (first >= 0) sh_win[2] = head_seg;
-                    else { sh_win[0] = head_seg; sh_win[1] = head_ends; }
+                    float x[E];
+                    Chunk<T>::unpack(v[u], x);
+#pragma unroll
+                    for (int e = 0; e < E; e += 2) add2(acc[0][e], acc[0][e + 1], x[e], x[e + 1]);
                 }
             }
         }
-        if (last_run && tail_seg >= 0) {           // a segment that begins in the window's last run and continues
-            float *dst = tail2 + (int64_t)blockIdx.x * d;
-#pragma unroll
-            for (int q = 0; q < CPL; ++q) {
-                const int ch = c + q * LPR;
-                if (ch < n_chunks) {
-#pragma unroll
-                    for (int e = 0; e < E; e += 4)
-                        *reinterpret_cast<float4 *>(dst + ch * E + e) = *reinterpret_cast<const float4 *>(sh_tail + rl * ROW + ch * E + e);
-                }
+        emit(last_ends);
+    }
+    if (live_window)
+        seg_join_window<T, int32_t, LPR, 1, kExtra>(sh_head, sh_tail, sh_info, sh_win, rl, c, n_chunks, d, head_seg, head_ends,
+                                                    tail_seg, ptr, head2, tail2, win_info, o, chain_cnt, run_len);
+    if (!chain_cnt) return;                        // the two-kernel form: seg_final_kernel writes the rest
+
+    // ---- segments without entries (their row is the self row, masked, or zero) and the zero rows up to the next
+    // multiple of 128: every block of the grid takes a slice, one lane group per segment
+    {
+        const int32_t n_self = o.n_self ? *o.n_self : n_seg;
+        const int32_t per = (n_seg + (int32_t)gridDim.x - 1) / (int32_t)gridDim.x;
+        const int32_t s1 = min(n_seg, ((int32_t)blockIdx.x + 1) * per);
+        for (int32_t sg = (int32_t)blockIdx.x * per + rl; sg < s1; sg += RB) {
+            if (ptr[sg + 1] != ptr[sg]) continue;
+            float acc[1][E];
+            uint4 mrow[1] = {make_uint4(0, 0, 0, 0)};
+            uint4 raw = make_uint4(0, 0, 0, 0);
+            if (c < n_chunks) {
+                if (sg < n_self) raw = Chunk<T>::load_raw(o.self + (int64_t)sg * o.ld_self + c * E);
+                if (kMask) mrow[0] = Chunk<T>::load_raw(o.mask + (int64_t)sg * o.ld_mask + c * E);
             }
-            if (c == 0) sh_win[2] = tail_seg;
+            Chunk<T>::unpack(raw, acc[0]);
+            seg_store_row<T, LPR, 1, kExtra>(o, sg, 1.0f, acc, mrow, c, n_chunks);
+        }
+        if (o.pad_rows > 0) {
+            const int64_t pad_end = min(((int64_t)n_seg + 127) / 128 * 128, o.pad_rows);
+            const int64_t cells = (pad_end - n_seg) * d;
+            for (int64_t t = (int64_t)blockIdx.x * kAggThreads + threadIdx.x; t < cells; t += (int64_t)gridDim.x * kAggThreads)
+                o.out[(n_seg + t / d) * o.ld_out + t % d] = from_float<T>(0.f);
         }
     }
-    __syncthreads();
-    if (threadIdx.x == 0) win_info[blockIdx.x] = make_int4(sh_win[0], sh_win[1], sh_win[2], 0);
 }
 
 // ------------------------------------------------------------------------------------ across windows
@@ -469,6 +695,8 @@ seg_final_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_t
     __shared__ int32_t sh_seg[kFinalWindows];
     __shared__ int sh_long[kFinalWindows];
     __shared__ int sh_n_long;
+    pdl_launch_dependents();
+    pdl_wait();
     const int64_t n_seg = n_seg_dev ? (int64_t)*n_seg_dev : n_seg_host;
     if (n_seg < 0) return;
     const int64_t n_self = o.self ? (o.n_self ? (int64_t)*o.n_self : n_seg) : 0;
@@ -627,6 +855,16 @@ seg_final_kernel(const PtrT *__restrict__ ptr, const int32_t *n_seg_dev, int64_t
 }
 
 // ------------------------------------------------------------------------------------ host
+// E2EGREC_SEG_GENERAL=1 keeps sampled blocks on the general kernel (to compare the two forms; same results).
+inline bool seg_general_only()
+{
+    static const bool v = []() {
+        const char *e = getenv("E2EGREC_SEG_GENERAL");
+        return e && *e && e[0] != '0';
+    }();
+    return v;
+}
+
 template <typename T, typename PtrT, int LPR, int CPL, bool kWeight, int kInFlight>
 inline void launch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const int32_t *idx, const int32_t *n_seg_dev,
                               int64_t n_seg_host, int64_t cap_seg, const float *w, int run_len, int d,
@@ -636,41 +874,50 @@ inline void launch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const
     tap_begin(TAP_SEG_L1, st);
     note_launch();
     const unsigned grid1 = (unsigned)sc.n_windows;
-    if (o.mask) {
+    bool block_form = false;
+    if constexpr (CPL == 1 && !kWeight && sizeof(PtrT) == 4) {
+        // the transposed aggregation of a sampled block: the kernel written for that case
+        if (seg_of && n_seg_dev && o.self && !o.mean && !o.seg_scale && !seg_general_only()) {
+            block_form = true;
+            if (o.mask)
+                launch_pdl(seg_run_block_kernel<T, LPR, true>, dim3(grid1), dim3(kAggThreads), smem, st, in, ld_in, ptr, idx, seg_of,
+                           n_seg_dev, run_len, d, sc.head2, sc.tail2, sc.win_info, sc.cap_runs, sc.chain_cnt, o);
+            else
+                launch_pdl(seg_run_block_kernel<T, LPR, false>, dim3(grid1), dim3(kAggThreads), smem, st, in, ld_in, ptr, idx, seg_of,
+                           n_seg_dev, run_len, d, sc.head2, sc.tail2, sc.win_info, sc.cap_runs, sc.chain_cnt, o);
+            if (sc.chain_cnt) {                   // chains, empty segments and padding were all done in that launch
+                tap_end(TAP_SEG_L1, st);
+                tap_begin(TAP_SEG_L3, st);        // (an armed tap of the second kernel reads zero)
+                tap_end(TAP_SEG_L3, st);
+                return;
+            }
+        }
+    }
+    if (block_form) {
+    } else if (o.mask) {
         auto kern = seg_run_kernel<T, PtrT, LPR, CPL, kWeight, 2, kInFlight>;
         if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        kern<<<grid1, kAggThreads, smem, st>>>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head2, sc.tail2,
-                                               sc.win_info, sc.cap_runs, seg_of, o);
-    } else if (o.self && run_len >= 128 && kSegRing > 0 && CPL == 1 && !kWeight && sizeof(PtrT) == 4 && LPR >= 16 && kInFlight == 4 &&
-               seg_of) {
-        // rows of 256 bytes and more on a sampled block that can hold millions of entries (long runs: the rows it gathers do
-        // not fit in L2): the ring form.  On smaller blocks, whose rows come from L2, registers in flight are faster.
-        if constexpr (CPL == 1 && !kWeight && sizeof(PtrT) == 4 && LPR >= 16 && kInFlight == 4) {
-            constexpr size_t smem_ring = smem + (size_t)2 * kSegRing * kAggThreads * 16;
-            auto kern = seg_run_kernel<T, PtrT, LPR, CPL, kWeight, 1, kInFlight, kSegRing>;
-            cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_ring);
-            kern<<<grid1, kAggThreads, smem_ring, st>>>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head2,
-                                                        sc.tail2, sc.win_info, sc.cap_runs, seg_of, o);
-        }
+        launch_pdl(kern, dim3(grid1), dim3(kAggThreads), smem, st, in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head2,
+                   sc.tail2, sc.win_info, sc.cap_runs, seg_of, o);
     } else if (o.self) {
         auto kern = seg_run_kernel<T, PtrT, LPR, CPL, kWeight, 1, kInFlight>;
         if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        kern<<<grid1, kAggThreads, smem, st>>>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head2, sc.tail2,
-                                               sc.win_info, sc.cap_runs, seg_of, o);
+        launch_pdl(kern, dim3(grid1), dim3(kAggThreads), smem, st, in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head2,
+                   sc.tail2, sc.win_info, sc.cap_runs, seg_of, o);
     } else {
         auto kern = seg_run_kernel<T, PtrT, LPR, CPL, kWeight, 0, kInFlight>;
         if (smem > 48 * 1024) cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        kern<<<grid1, kAggThreads, smem, st>>>(in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head2, sc.tail2,
-                                               sc.win_info, sc.cap_runs, seg_of, o);
+        launch_pdl(kern, dim3(grid1), dim3(kAggThreads), smem, st, in, ld_in, ptr, idx, n_seg_dev, n_seg_host, w, run_len, d, sc.head2,
+                   sc.tail2, sc.win_info, sc.cap_runs, seg_of, o);
     }
     tap_end(TAP_SEG_L1, st);
     const int64_t window_blocks = std::min<int64_t>(ceil_div(sc.n_windows, kFinalWindows), 148 * 16);
     const int64_t empty_blocks = std::min<int64_t>(ceil_div(cap_seg > 0 ? cap_seg : 1, kAggThreads), 148 * 8);
     tap_begin(TAP_SEG_L3, st);
     note_launch();
-    seg_final_kernel<T, PtrT><<<(unsigned)(window_blocks + empty_blocks), kAggThreads, 0, st>>>(
-        ptr, n_seg_dev, n_seg_host, run_len, sc.runs_per_window, d, sc.head2, sc.tail2, sc.win_info, sc.n_windows,
-        window_blocks, o);
+    launch_pdl(seg_final_kernel<T, PtrT>, dim3((unsigned)(window_blocks + empty_blocks)), dim3(kAggThreads), 0, st, ptr, n_seg_dev,
+               n_seg_host, run_len, sc.runs_per_window, d, (const float *)sc.head2, (const float *)sc.tail2, (const int4 *)sc.win_info,
+               sc.n_windows, window_blocks, o);
     tap_end(TAP_SEG_L3, st);
 }
 
