@@ -401,24 +401,26 @@ def run_ours(args, w, with_joint):
 
     if args.multitask:
         # the two-task step of Sec. 4.2 / 4.3.1: the recommendation gradient and the gradient of the SSL reconstruction
-        # loss go through the encoder one after the other (weight gradients accumulate), their norms at the shared
-        # input feed one GradNorm step of the task weights
+        # loss go through the encoder together (two right-hand sides of one backward pass, weight gradients summed),
+        # their norms at the shared input feed one GradNorm step of the task weights
         if w.hidden != w.dim:
             raise SystemExit("--multitask needs hidden == dim (the identity decoder compares H with X)")
         f32 = dict(dtype=torch.float32, device=dev)
         mt = dict(dX_ssl=torch.zeros_like(dX2[0]), dH_ssl=torch.zeros_like(H_out), one=torch.ones(1, **f32),
-                  wts=torch.ones(2, **f32), L=torch.ones(2, **f32), L0=torch.ones(2, **f32), g=torch.zeros(2, **f32))
+                  wts=torch.ones(2, **f32), L=torch.ones(2, **f32), L0=torch.ones(2, **f32), g=torch.zeros(2, **f32),
+                  scratch=torch.empty(E.binding.sage_backward_multi_scratch_bytes(blocks, X, Ws, 2), dtype=torch.uint8, device=dev))
 
     def compute_leg(p):
         E.sage_forward(blocks2[p], X, Ws, ctx=ctx, H_out=H_out2[p])
-        E.sage_backward(blocks2[p], X, Ws, ctx, dH_in2[p], dWs=dWs2[p], dX_rows=dX2[p], scratch=scratch)
-        if args.multitask:
+        if not args.multitask:
+            E.sage_backward(blocks2[p], X, Ws, ctx, dH_in2[p], dWs=dWs2[p], dX_rows=dX2[p], scratch=scratch)
+        else:
             n_seeds_dev, n_rows_dev = blocks2[p].counts[0][0:1], blocks2[p].counts[L - 1][1:2]
             E.ssl_loss(H_out2[p], X, seeds_in2[p], n_seeds_dev, mt["one"], loss=mt["L"][0:1], dH=mt["dH_ssl"])
-            E.gradient_norm(dX2[p], n_rows_dev, out=mt["g"][1:2])
-            E.sage_backward(blocks2[p], X, Ws, ctx, mt["dH_ssl"], dWs=dWs2[p], dX_rows=mt["dX_ssl"], scratch=scratch,
-                            accumulate=True)
-            E.gradient_norm(mt["dX_ssl"], n_rows_dev, out=mt["g"][0:1])
+            # both task gradients through the encoder in one pass: two input gradients, summed weight gradients
+            E.sage_backward_multi(blocks2[p], X, Ws, ctx, [dH_in2[p], mt["dH_ssl"]], dWs=dWs2[p], dX_rows=[dX2[p], mt["dX_ssl"]],
+                                  scratch=mt["scratch"])
+            E.gradient_norms([mt["dX_ssl"], dX2[p]], n_rows_dev, out=mt["g"])      # g[0]: SSL task, g[1]: recommendation task
             E.gradnorm_update(mt["wts"], mt["L"], mt["L0"], mt["g"], 1.0, 0.025)
         count_total.add_(blocks2[p].counts)
         counts_snap2[p].copy_(blocks2[p].counts)
@@ -720,7 +722,8 @@ def run_ours(args, w, with_joint):
                 config=dict(workload=w.name, nodes=w.n_nodes, csr_entries=int(indices.numel()), dim=w.dim, hidden=w.hidden,
                             layers=L, fanouts=list(w.fanouts), batch=w.batch, seeds=args.seeds,
                             sampling="uniform" if args.beta is None else f"weighted, beta={args.beta}",
-                            tasks="recommendation gradient + SSL reconstruction loss, two backward passes, GradNorm step"
+                            tasks="recommendation gradient + SSL reconstruction loss as two right-hand sides of one backward pass, "
+                                  "gradient norms, GradNorm step"
                                   if args.multitask else "recommendation gradient",
                             parallelism=f"replicas x{world}",
                             launch="one CUDA graph replay per step, three streams: forward/backward of batch i beside the "

@@ -261,6 +261,22 @@ int32_t e2egrec_sage_backward(const e2egrec_block *blocks, int32_t n_layers, con
                               const e2egrec_mat *dX_rows, void *scratch, size_t *scratch_bytes,
                               uint32_t flags, void *stream);
 
+/* e2egrec_sage_backward for several gradients in one pass (Sec. 4.3.1, gradient-based task weighting: G_i(t), the norm
+ * of each task's gradient with respect to the shared input h^(0), needs the input gradient of every task at every step;
+ * Sec. 4.3.2, the GNN receives w_SSL grad L_SSL + w_r J^T dL_reward/dF_gnn + ...).  dH_out and dX_rows are host arrays of
+ * n_rhs (1 or 2) matrices: gradient r arrives as dH_out[r] and its input-feature gradient leaves as dX_rows[r] (all of one
+ * shape, dtype and leading dimension; see e2egrec_sage_backward).  dW and dbias receive the sum over the gradients, so a
+ * caller folds the task weights into dH_out.  Every layer runs each of its kernels once for all gradients: their rows are
+ * stacked in the dense products (the weight gradient contracts over both stacks at once), and the transposed aggregation
+ * walks the block's csc arrays for both in one launch.  Each dX_rows[r] equals what e2egrec_sage_backward returns for
+ * dH_out[r] alone, bit for bit; dW equals the sum of the separate calls up to the order of the fp32 additions.
+ * scratch: size query with scratch == NULL (it depends on n_rhs). */
+int32_t e2egrec_sage_backward_multi(const e2egrec_block *blocks, int32_t n_layers, const e2egrec_mat *X,
+                                    const e2egrec_mat *W, const int32_t *act, const void *ctx,
+                                    const e2egrec_mat *dH_out, int32_t n_rhs, float *const *dW, float *const *dbias,
+                                    const e2egrec_mat *dX_rows, void *scratch, size_t *scratch_bytes,
+                                    uint32_t flags, void *stream);
+
 /* One joint training step of the GNN and the ranking model (Theorem 1: z_i = [h_theta(x_i) || b_i] is the
  * scorer's input, so the ranking loss reaches the GNN; Sec. 4.2 chain rule; binary cross-entropy as
  * in Sec. 5.1).  For n_pairs training pairs (user u_p, item i_p, dense features b_p, label y_p):
@@ -398,6 +414,8 @@ int32_t e2egrec_lightgcn_sampled_backward(const e2egrec_block *blocks, int32_t n
  *   trip).  H is the encoder output (e2egrec_sage_forward's H_out), whose width must equal X's.
  * e2egrec_gradient_norm: || A[:n_rows] ||_2 into norm (device float[1]): GradNorm's gradient norm of one task with
  *   respect to the shared input rows (the dX_rows of a backward pass run with that task's gradient alone).
+ *   e2egrec_gradient_norms does the same for n <= 4 matrices of one shape and dtype in one pass (A: host array[n],
+ *   norms: device float[n]): the norms of all tasks of a step, e.g. of the results of e2egrec_sage_backward_multi.
  * e2egrec_gradnorm_update: one GradNorm step for n_tasks <= 8 weights w (device, updated in place) from the current
  *   and initial losses L, L0 and the norms g of the unweighted task gradients (G_i = w_i g_i): with r_i =
  *   (L_i/L0_i) / mean_j (L_j/L0_j) and the targets c_i = mean(G) r_i^gamma held constant, w_i takes one step of size
@@ -409,6 +427,8 @@ int32_t e2egrec_ssl_loss(const e2egrec_mat *H, const e2egrec_mat *X, const int32
                          void *stream);
 int32_t e2egrec_gradient_norm(const e2egrec_mat *A, const int32_t *n_rows_dev, float *norm, void *ws, size_t *ws_bytes,
                               void *stream);
+int32_t e2egrec_gradient_norms(const e2egrec_mat *A, int32_t n, const int32_t *n_rows_dev, float *norms, void *ws,
+                               size_t *ws_bytes, void *stream);
 int32_t e2egrec_gradnorm_update(float *w, const float *L, const float *L0, const float *g, int32_t n_tasks, float gamma,
                                 float lr, float *L_gn, void *stream);
 

@@ -82,6 +82,9 @@ def lib():
         L.e2egrec_gradient_norm.restype = C.c_int32
         L.e2egrec_gradient_norm.argtypes = [C.POINTER(Mat), C.c_void_p, C.c_void_p, C.c_void_p, C.POINTER(C.c_size_t),
                                             C.c_void_p]
+        L.e2egrec_gradient_norms.restype = C.c_int32
+        L.e2egrec_gradient_norms.argtypes = [C.POINTER(Mat), C.c_int32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                             C.POINTER(C.c_size_t), C.c_void_p]
         L.e2egrec_gradnorm_update.restype = C.c_int32
         L.e2egrec_gradnorm_update.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int32, C.c_float,
                                               C.c_float, C.c_void_p, C.c_void_p]
@@ -103,6 +106,11 @@ def lib():
                                             C.c_void_p, C.c_void_p, C.POINTER(Mat), C.c_void_p, C.c_void_p,
                                             C.POINTER(Mat), C.c_void_p, C.POINTER(C.c_size_t), C.c_uint32,
                                             C.c_void_p]
+        L.e2egrec_sage_backward_multi.restype = C.c_int32
+        L.e2egrec_sage_backward_multi.argtypes = [C.POINTER(Block), C.c_int32, C.POINTER(Mat), C.POINTER(Mat),
+                                                  C.c_void_p, C.c_void_p, C.POINTER(Mat), C.c_int32, C.c_void_p, C.c_void_p,
+                                                  C.POINTER(Mat), C.c_void_p, C.POINTER(C.c_size_t), C.c_uint32,
+                                                  C.c_void_p]
         L.e2egrec_sage_ctx_layout.restype = C.c_int32
         L.e2egrec_sage_ctx_layout.argtypes = [C.POINTER(Block), C.c_int32, C.POINTER(Mat), C.POINTER(Mat),
                                               C.c_void_p, C.c_void_p, C.c_void_p]
@@ -386,6 +394,36 @@ def sage_backward(blocks: Blocks, X, Ws, ctx, dH_out, acts=None, dWs=None, dbs=N
     return dWs, dX_rows
 
 
+def sage_backward_multi_scratch_bytes(blocks: Blocks, X, Ws, n_rhs: int) -> int:
+    n = C.c_size_t(0)
+    x, w = _mat(X), _mats(Ws)
+    _check(lib().e2egrec_sage_backward_multi(blocks.c, len(Ws), C.byref(x), w, None, None, None, n_rhs, None, None, None, None,
+                                             C.byref(n), 0, None), "e2egrec_sage_backward_multi(size query)")
+    return n.value
+
+
+def sage_backward_multi(blocks: Blocks, X, Ws, ctx, dH_outs, acts=None, dWs=None, dbs=None, dX_rows=None, scratch=None,
+                        accumulate=False, stream=None):
+    """Enqueues one backward pass for the gradients in the list dH_outs (one or two); returns (dWs, list of dX_rows):
+    dWs is the sum over the gradients, dX_rows[r] belongs to dH_outs[r].  Buffers are allocated when not given."""
+    L, R = len(Ws), len(dH_outs)
+    dev = X.device
+    if scratch is None:
+        scratch = _dev_bytes(sage_backward_multi_scratch_bytes(blocks, X, Ws, R), dev)
+    if dWs is None:
+        dWs = [torch.zeros(W.shape, dtype=torch.float32, device=dev) for W in Ws]
+    if dX_rows is None:
+        dX_rows = [torch.zeros(max(blocks.caps[L - 1][1], 1), X.shape[1], dtype=X.dtype, device=dev) for _ in range(R)]
+    x, w = _mat(X), _mats(Ws)
+    dh, dx = _mats(dH_outs), _mats(dX_rows)
+    n = C.c_size_t(scratch.numel())
+    a = None if acts is None else _i32_host(acts)
+    _check(lib().e2egrec_sage_backward_multi(blocks.c, L, C.byref(x), w, a, _ptr(ctx), dh, R, _ptr_array(dWs, L),
+                                             _ptr_array(dbs, L), dx, _ptr(scratch), C.byref(n),
+                                             ACCUMULATE_DW if accumulate else 0, _stream(stream)), "e2egrec_sage_backward_multi")
+    return dWs, dX_rows
+
+
 # ------------------------------------------------------------------------------------------ whole graph
 
 def aggregate_ws_bytes(n_entries, X) -> int:
@@ -643,10 +681,12 @@ _SUM_WS = {}
 
 
 def _sum_ws(device):
-    """The 1 KB scratch of the fixed-order sums, one per device."""
+    """The scratch of the fixed-order sums (size from the library's query), one per device."""
     key = str(device)
     if key not in _SUM_WS:
-        _SUM_WS[key] = _dev_bytes(1024, device)
+        n = C.c_size_t(0)
+        _check(lib().e2egrec_gradient_norms(None, 1, None, None, None, C.byref(n), None), "e2egrec_gradient_norms(size query)")
+        _SUM_WS[key] = _dev_bytes(n.value, device)
     return _SUM_WS[key]
 
 
@@ -676,6 +716,17 @@ def gradient_norm(A: torch.Tensor, n_rows_dev=None, out=None, stream=None):
     a = _mat(A)
     _check(lib().e2egrec_gradient_norm(C.byref(a), None if n_rows_dev is None else _ptr(n_rows_dev), _ptr(out), _ptr(ws),
                                        C.byref(n), _stream(stream)), "e2egrec_gradient_norm")
+    return out
+
+
+def gradient_norms(As, n_rows_dev=None, out=None, stream=None):
+    """Enqueues the norms ||A[:n_rows]||_2 of up to four matrices of one shape into out[len(As)]; see e2egrec_gradient_norms."""
+    if out is None:
+        out = torch.zeros(len(As), dtype=torch.float32, device=As[0].device)
+    ws = _sum_ws(As[0].device)
+    n = C.c_size_t(ws.numel())
+    _check(lib().e2egrec_gradient_norms(_mats(As), len(As), None if n_rows_dev is None else _ptr(n_rows_dev), _ptr(out), _ptr(ws),
+                                        C.byref(n), _stream(stream)), "e2egrec_gradient_norms")
     return out
 
 

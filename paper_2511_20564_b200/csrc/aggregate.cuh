@@ -148,6 +148,10 @@ struct SegOut {
     int mean;               // divide the sum by the segment length
     const float *seg_scale; // optional: multiply the sum of segment s by seg_scale[s] (not together with mean)
     int64_t pad_rows;       // if > 0: rows n_seg .. min(next multiple of 128, pad_rows) - 1 of out are zeroed
+    // Several right-hand sides in one call (same segments and indices, different rows): right-hand side r reads
+    // in + r * rhs_in and self + r * rhs_self and writes out + r * rhs_out (element strides); the mask is shared.
+    int n_rhs;              // 0 or 1: one
+    int64_t rhs_in, rhs_self, rhs_out;
 };
 
 template <typename T>

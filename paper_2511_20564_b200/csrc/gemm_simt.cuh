@@ -108,7 +108,7 @@ struct EpiPartial {
 // tensor-core weight-gradient kernel, which only fills the first ceil(total / per) splits
 // (total = ceil(rows / 64) k-blocks, per = max(8, ceil(total / splits))); without it all splits are added.
 static __global__ void splitk_reduce_kernel(const float *__restrict__ partial, int64_t n, int splits, int accumulate,
-                                            float *__restrict__ out, const int32_t *rows_dev)
+                                            float *__restrict__ out, const int32_t *rows_dev, int n_rhs = 1)
 {
     pdl_launch_dependents();
     pdl_wait();
@@ -116,7 +116,7 @@ static __global__ void splitk_reduce_kernel(const float *__restrict__ partial, i
     if (i >= n) return;
     int active = splits;
     if (rows_dev) {
-        const int64_t total = ((int64_t)*rows_dev + 63) / 64;
+        const int64_t total = (((int64_t)*rows_dev + 63) / 64) * n_rhs;
         const int64_t per = max((int64_t)8, (total + splits - 1) / splits);
         active = (int)max((int64_t)1, (total + per - 1) / per);
     }
@@ -126,13 +126,20 @@ static __global__ void splitk_reduce_kernel(const float *__restrict__ partial, i
 }
 
 // dZ = dH where the stored output is positive (or everywhere for the identity activation);
-// rows in [n, rows_alloc) are set to zero.
+// rows in [n, rows_alloc) are set to zero.  gridDim.y = 2: a second gradient dH1 goes to the block of rows_alloc
+// rows behind the first in dZ (two right-hand sides sent through the backward pass together).
 template <typename T>
 __global__ void relu_mask_kernel(const T *__restrict__ dH, int64_t ld_dh, const T *__restrict__ H, int64_t ld_h,
-                                 const int32_t *n_dev, int64_t rows_alloc, int d, int relu, T *__restrict__ dZ)
+                                 const int32_t *n_dev, int64_t rows_alloc, int d, int relu, T *__restrict__ dZ,
+                                 const T *__restrict__ dH1 = nullptr, int64_t ld_dh1 = 0)
 {
     pdl_launch_dependents();
     pdl_wait();
+    if (blockIdx.y == 1) {
+        dH = dH1;
+        ld_dh = ld_dh1;
+        dZ += rows_alloc * d;
+    }
     const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const int64_t r = i / d;
     const int k = (int)(i - r * d);

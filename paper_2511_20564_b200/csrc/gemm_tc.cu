@@ -165,6 +165,11 @@ struct TcEpilogue {
     int64_t ldo2, rows2;
     int32_t *status;           // device status word (E2EGREC_DEV_TIMEOUT)
     TcFuse fuse;               // optional gating / product-plus-term forms of the epilogue
+    // Several right-hand sides stacked along the rows: A and the output hold n_rhs blocks of rhs_rows rows each (a
+    // multiple of 128); in every block the first *m_dev rows are live.  Row scale and mask are shared by the blocks and
+    // indexed by the row inside its block.  n_rhs = 1: one block, rhs_rows unused.
+    int n_rhs;
+    int64_t rhs_rows;
 };
 
 __device__ inline float bf16_round(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
@@ -240,7 +245,15 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     // barriers and tensor memory are set up; global memory is touched only once the preceding kernel has completed
     pdl_wait();
     const int32_t m_valid = *ep.m_dev;
-    const int64_t n_work = (((int64_t)m_valid + kTileM - 1) / kTileM) * n_tiles_n;   // tiles wholly beyond *m_dev stay as they are
+    const int64_t live_tiles = ((int64_t)m_valid + kTileM - 1) / kTileM;    // per block of rows; tiles wholly beyond *m_dev stay as they are
+    const int64_t n_work = live_tiles * n_tiles_n * ep.n_rhs;
+    // tile t of the list: column tile t % n_tiles_n of live row tile (t / n_tiles_n) % live_tiles of block (t / n_tiles_n) / live_tiles
+    auto tile_rows = [&](int64_t t, int64_t &m0, int64_t &m0_local) {
+        const int64_t rt = t / n_tiles_n;
+        const int64_t rhs = ep.n_rhs > 1 ? rt / live_tiles : 0;
+        m0_local = (rt - rhs * live_tiles) * kTileM;
+        m0 = rhs * ep.rhs_rows + m0_local;
+    };
 
     if ((int64_t)blockIdx.x >= n_work) {
         // nothing for this CTA: straight to the release of its tensor memory
@@ -250,7 +263,9 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             uint32_t g = 0;
             bool ok = true;
             for (int64_t t = blockIdx.x; t < n_work && ok; t += gridDim.x) {
-                const int m0 = (int)(t / n_tiles_n) * kTileM, n0 = (int)(t % n_tiles_n) * nt;
+                int64_t m0_64, m0_local;
+                tile_rows(t, m0_64, m0_local);
+                const int m0 = (int)m0_64, n0 = (int)(t % n_tiles_n) * nt;
                 for (int kb = 0; kb < k_blocks; ++kb, ++g) {
                     const uint32_t s = g % (uint32_t)stages, ph = (g / (uint32_t)stages) & 1u;
                     ok = mbar_wait(&empty_bar[s], ph ^ 1u, &abort_flag);
@@ -315,13 +330,15 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             const uint32_t buf = lt & 1u;
             if (!mbar_wait(&acc_full[buf], (lt >> 1) & 1u, &abort_flag)) break;
             tc_fence_after();
-            const int64_t m0 = (t / n_tiles_n) * kTileM;
+            int64_t m0, m0_local;
+            tile_rows(t, m0, m0_local);
             const int n0 = (int)(t % n_tiles_n) * nt;
             const int64_t row = m0 + lg * 32 + lane;
-            const bool live = row < m_valid;
-            const float rs = (ep.row_scale && live) ? ep.row_scale[row] : 1.f;
+            const int64_t row_local = m0_local + lg * 32 + lane;        // the row inside its block of rows
+            const bool live = row_local < m_valid;
+            const float rs = (ep.row_scale && live) ? ep.row_scale[row_local] : 1.f;
             __nv_bfloat16 *orow = ep.out + row * ep.ldo + n0;
-            const __nv_bfloat16 *mrow = ep.mask ? ep.mask + row * ep.ld_mask + n0 : nullptr;
+            const __nv_bfloat16 *mrow = ep.mask ? ep.mask + row_local * ep.ld_mask + n0 : nullptr;
             __nv_bfloat16 *orow2 = (ep.out2 && row < ep.rows2) ? ep.out2 + row * ep.ldo2 + n0 : nullptr;
             if (c_first >= nt) {                          // a single column block: nothing for the second set of warps
                 if (lane == 0) mbar_arrive(&acc_empty[buf]);
@@ -497,9 +514,12 @@ bool make_map_mn(CUtensorMap *map, const void *base, int64_t rows, int64_t cols)
 
 // b_mn: B is stored [k x n] row-major (its N index contiguous) instead of [n x k]
 bool launch_tn(const __nv_bfloat16 *A, int64_t rows, int k, int64_t lda, const __nv_bfloat16 *B, int n, int64_t ldb,
-               const TcEpilogue &ep, cudaStream_t st, bool b_mn = false)
+               const TcEpilogue &ep_in, cudaStream_t st, bool b_mn = false, int n_rhs = 1)
 {
-    if (rows <= 0 || rows % kTileM || k % kTileK || k < kTileK) return false;
+    if (rows <= 0 || rows % kTileM || k % kTileK || k < kTileK || n_rhs < 1) return false;
+    TcEpilogue ep = ep_in;
+    ep.n_rhs = n_rhs;
+    ep.rhs_rows = rows;
     int nt = 0;                                 // widest tile <= 256 columns that divides n (a multiple of 32, or of 64 for b_mn)
     const int unit = b_mn ? 64 : 32;
     for (int c = 256; c >= unit; c -= unit)
@@ -509,7 +529,7 @@ bool launch_tn(const __nv_bfloat16 *A, int64_t rows, int k, int64_t lda, const _
         reinterpret_cast<uintptr_t>(ep.out) % 16 || (ep.ldo * 2) % 16)
         return false;
     CUtensorMap ma, mb;
-    if (!make_map(&ma, A, rows, k, lda, kTileM)) return false;
+    if (!make_map(&ma, A, rows * n_rhs, k, lda, kTileM)) return false;
     if (b_mn ? (ldb != n || !make_map_mn(&mb, B, k, n)) : !make_map(&mb, B, n, k, ldb, nt)) return false;
     const int k_blocks = k / kTileK;
     const int stages = k_blocks < kMaxStages ? k_blocks : kMaxStages;
@@ -521,7 +541,7 @@ bool launch_tn(const __nv_bfloat16 *A, int64_t rows, int k, int64_t lda, const _
     if (!(fused ? raise_smem_limit(tc_gemm_tn_kernel<true>, attr_set[1]) : raise_smem_limit(tc_gemm_tn_kernel<false>, attr_set[0])))
         return false;
     const int n_tiles_n = n / nt;
-    const int64_t tiles_cap = (rows / kTileM) * n_tiles_n;
+    const int64_t tiles_cap = (rows / kTileM) * n_tiles_n * n_rhs;
     const unsigned grid = (unsigned)std::min<int64_t>(tiles_cap, sm_count());
     note_launch();
     if (fused)
@@ -543,7 +563,7 @@ bool launch_tn(const __nv_bfloat16 *A, int64_t rows, int k, int64_t lda, const _
 __global__ void __launch_bounds__(kThreads)
 tc_gemm_rows_kernel(const __grid_constant__ CUtensorMap map_y, const __grid_constant__ CUtensorMap map_x, int nt,
                     uint32_t tmem_cols, int stages, const int32_t *m_dev, float *__restrict__ part, int64_t ldp,
-                    int64_t split_stride, int32_t *status)
+                    int64_t split_stride, int32_t *status, int n_rhs, int64_t rhs_rows)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], accum_bar;
@@ -555,7 +575,10 @@ tc_gemm_rows_kernel(const __grid_constant__ CUtensorMap map_y, const __grid_cons
     pdl_launch_dependents();
     pdl_wait();                                 // the preceding kernel of the stream has completed
     const int64_t m_valid = *m_dev;
-    const int64_t total_blocks = (m_valid + kTileK - 1) / kTileK;
+    // Y may hold n_rhs blocks of rhs_rows rows (the first *m_dev of each live) that all meet the same rows of X: the
+    // k-blocks of the blocks of rows form one list, and the sum runs over all of them
+    const int64_t blocks_per_rhs = (m_valid + kTileK - 1) / kTileK;
+    const int64_t total_blocks = blocks_per_rhs * n_rhs;
     // at least kMinSplitBlocks k-blocks per split: only the first ceil(total / per) splits do work and
     // write a partial (split 0 writes zeros when there are no rows); splitk_reduce_kernel uses the same rule
     const int64_t per = max((int64_t)kMinSplitBlocks, (total_blocks + gridDim.z - 1) / gridDim.z);
@@ -603,11 +626,14 @@ tc_gemm_rows_kernel(const __grid_constant__ CUtensorMap map_y, const __grid_cons
             const uint32_t ph = (uint32_t)(kb / stages) & 1u;
             if (!mbar_wait(&empty_bar[s], ph ^ 1u, &abort_flag)) break;
             mbar_expect_tx(&full_bar[s], a_bytes + b_bytes);
-            const int row = (int)((kb0 + kb) * kTileK);
+            const int64_t jb = kb0 + kb;
+            const int64_t rhs = n_rhs > 1 ? jb / blocks_per_rhs : 0;
+            const int row_x = (int)((jb - rhs * blocks_per_rhs) * kTileK);
+            const int row_y = (int)(rhs * rhs_rows) + row_x;
             for (int j = 0; j < kTileM / 64; ++j)
-                tma_load_2d(a_tiles + (size_t)s * a_bytes + j * blk_bytes, &map_y, m0 + j * 64, row, &full_bar[s]);
+                tma_load_2d(a_tiles + (size_t)s * a_bytes + j * blk_bytes, &map_y, m0 + j * 64, row_y, &full_bar[s]);
             for (int j = 0; j < nt / 64; ++j)
-                tma_load_2d(b_tiles + (size_t)s * b_bytes + j * blk_bytes, &map_x, n0 + j * 64, row, &full_bar[s]);
+                tma_load_2d(b_tiles + (size_t)s * b_bytes + j * blk_bytes, &map_x, n0 + j * 64, row_x, &full_bar[s]);
             issued = kb + 1;
         }
     } else if (warp == 1 && lane == 0) {
@@ -719,7 +745,8 @@ bool tc_linear(const __nv_bfloat16 *A, int64_t rows, int k, const __nv_bfloat16 
 }
 
 bool tc_dcat_backward(const __nv_bfloat16 *dz, int64_t rows, int d_out, const __nv_bfloat16 *W, int two_d_in,
-                      const float *inv_cnt, __nv_bfloat16 *dcat, const int32_t *m_dev, int32_t *status, cudaStream_t st)
+                      const float *inv_cnt, __nv_bfloat16 *dcat, const int32_t *m_dev, int32_t *status, cudaStream_t st,
+                      int n_rhs)
 {
     TcEpilogue ep{};
     ep.out = dcat;
@@ -730,7 +757,7 @@ bool tc_dcat_backward(const __nv_bfloat16 *dz, int64_t rows, int d_out, const __
     ep.scale_from = two_d_in / 2;
     ep.m_dev = m_dev;
     ep.status = status;
-    return launch_tn(dz, rows, d_out, d_out, W, two_d_in, two_d_in, ep, st, true);
+    return launch_tn(dz, rows, d_out, d_out, W, two_d_in, two_d_in, ep, st, true, n_rhs);
 }
 
 }  // namespace e2egrec
@@ -738,16 +765,16 @@ bool tc_dcat_backward(const __nv_bfloat16 *dz, int64_t rows, int d_out, const __
 namespace e2egrec {
 
 bool tc_weight_grad(const __nv_bfloat16 *dY, int64_t rows, int m, const __nv_bfloat16 *Xin, int n, const int32_t *m_dev,
-                    float *part, int splits, int32_t *status, cudaStream_t st)
+                    float *part, int splits, int32_t *status, cudaStream_t st, int n_rhs)
 {
-    if (rows <= 0 || rows % kTileK || m % kTileM || n % 64) return false;
+    if (rows <= 0 || rows % kTileK || m % kTileM || n % 64 || n_rhs < 1) return false;
     int nt = 0;
     for (int c = 256; c >= 64; c -= 64)
         if (n % c == 0) { nt = c; break; }
     if (!nt) return false;
     if (reinterpret_cast<uintptr_t>(dY) % 16 || reinterpret_cast<uintptr_t>(Xin) % 16) return false;
     CUtensorMap my, mx;
-    if (!make_map_mn(&my, dY, rows, m) || !make_map_mn(&mx, Xin, rows, n)) return false;
+    if (!make_map_mn(&my, dY, rows * n_rhs, m) || !make_map_mn(&mx, Xin, rows, n)) return false;
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < nt) tmem_cols <<= 1;
     const int stages = kMaxStages;
@@ -757,7 +784,7 @@ bool tc_weight_grad(const __nv_bfloat16 *dY, int64_t rows, int m, const __nv_bfl
     dim3 grid((unsigned)(m / kTileM), (unsigned)(n / nt), (unsigned)splits);
     note_launch();
     launch_pdl(tc_gemm_rows_kernel, grid, dim3(kThreads), smem, st, my, mx, nt, tmem_cols, stages, m_dev, part, (int64_t)n,
-               (int64_t)m * n, status);
+               (int64_t)m * n, status, n_rhs, rows);
     return true;
 }
 

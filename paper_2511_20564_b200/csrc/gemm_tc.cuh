@@ -17,8 +17,11 @@ bool tc_update_forward(const __nv_bfloat16 *cat, int64_t rows, int k, const __nv
 // dCat = dZ W with the layer weight W [d_out x 2 d_in] as stored (the tensor cores read it with its N index
 // contiguous, no transposed copy is made); columns >= d_in are scaled by inv_cnt[row].  2 d_in must be a multiple
 // of 64.  Same conventions as above.
+// n_rhs > 1: dz and dcat hold n_rhs blocks of `rows` rows each (several gradients sent through the layer in one pass), the
+// first *m_dev rows of every block live; inv_cnt is indexed by the row inside its block.
 bool tc_dcat_backward(const __nv_bfloat16 *dz, int64_t rows, int d_out, const __nv_bfloat16 *W, int two_d_in,
-                      const float *inv_cnt, __nv_bfloat16 *dcat, const int32_t *m_dev, int32_t *status, cudaStream_t st);
+                      const float *inv_cnt, __nv_bfloat16 *dcat, const int32_t *m_dev, int32_t *status, cudaStream_t st,
+                      int n_rhs = 1);
 
 // Optional forms of the product's epilogue (all matrices [rows x n], bf16, 16-byte aligned rows):
 //   gate_in  F:  out = g * F with g = sigmoid(product + bias); the pre-activation and g are rounded to bf16 first,
@@ -42,7 +45,8 @@ bool tc_linear(const __nv_bfloat16 *A, int64_t rows, int k, const __nv_bfloat16 
 
 // part[z] = (rows of split z of dY)^T (same rows of Xin): dY [rows x m], Xin [rows x n] bf16 row-major, part
 // [splits x m x n] fp32.  Rows between *m_dev and the next multiple of 64 must be zero in both matrices.
+// n_rhs > 1: dY holds n_rhs blocks of `rows` rows that all meet the same `rows` rows of Xin; the result is the sum over them.
 bool tc_weight_grad(const __nv_bfloat16 *dY, int64_t rows, int m, const __nv_bfloat16 *Xin, int n, const int32_t *m_dev,
-                    float *part, int splits, int32_t *status, cudaStream_t st);
+                    float *part, int splits, int32_t *status, cudaStream_t st, int n_rhs = 1);
 
 }  // namespace e2egrec

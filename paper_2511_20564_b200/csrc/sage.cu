@@ -170,18 +170,18 @@ struct BackwardScratch {
     size_t dz_off[2], dcat_off, seg_off, seg_bytes, chain_off, chain_bytes, part_off, wt_off, bytes;
 };
 
-static BackwardScratch plan_backward(const e2egrec_block *blocks, int32_t n_layers, const LayerPlan *plan, size_t es)
+static BackwardScratch plan_backward(const e2egrec_block *blocks, int32_t n_layers, const LayerPlan *plan, size_t es, int n_rhs)
 {
     BackwardScratch s{};
     size_t dz = 0, dcat = 0, part = 0, ht = 0, wt = 0, chain = 0;
     for (int l = 0; l < n_layers; ++l) {
         const LayerPlan &p = plan[l];
-        dz = std::max(dz, (size_t)p.rows * p.d_out * es);
-        dcat = std::max(dcat, (size_t)p.rows * 2 * p.d_in * es);
+        dz = std::max(dz, (size_t)n_rhs * p.rows * p.d_out * es);
+        dcat = std::max(dcat, (size_t)n_rhs * p.rows * 2 * p.d_in * es);
         part = std::max(part, (size_t)kDwSplits * p.d_out * 2 * p.d_in * sizeof(float));
         wt = std::max(wt, (size_t)p.d_out * 2 * p.d_in * es);
-        ht = std::max(ht, seg_scratch_carve(blocks[p.block].cap_edges, block_run_len(blocks[p.block].cap_edges), p.d_in, es, nullptr).bytes);
-        chain = std::max(chain, seg_chain_bytes(blocks[p.block].cap_edges, block_run_len(blocks[p.block].cap_edges), p.d_in, es));
+        ht = std::max(ht, seg_scratch_carve(blocks[p.block].cap_edges, block_run_len(blocks[p.block].cap_edges), p.d_in, es, nullptr, n_rhs).bytes);
+        chain = std::max(chain, seg_chain_bytes(blocks[p.block].cap_edges, block_run_len(blocks[p.block].cap_edges), p.d_in, es, n_rhs));
     }
     size_t off = 0;
     auto take = [&](size_t b) { size_t o = off; off += align_up(b, 256); return o; };
@@ -199,8 +199,10 @@ static BackwardScratch plan_backward(const e2egrec_block *blocks, int32_t n_laye
 }
 
 template <typename T>
+// n_rhs gradients (dH_out[r] -> dX_rows[r]) go through the layers together: their rows are stacked in blocks of p.rows rows
+// in dZ and dCat, every kernel of a layer is launched once for all of them, and dW / dbias receive the sum over them.
 static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, const e2egrec_mat *X, const e2egrec_mat *W,
-                             const int32_t *act, const LayerPlan *plan, const char *ctx, const e2egrec_mat *dH_out,
+                             const int32_t *act, const LayerPlan *plan, const char *ctx, const e2egrec_mat *dH_out, int n_rhs,
                              float *const *dW, float *const *dbias, const e2egrec_mat *dX_rows, char *scratch,
                              const BackwardScratch &bs, uint32_t flags, cudaStream_t st)
 {
@@ -217,9 +219,10 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
         const e2egrec_block &b = blocks[p.block];
         const int64_t total = p.rows * p.d_out;
         note_launch();
-        launch_pdl(relu_mask_kernel<T>, dim3((unsigned)std::max<int64_t>(1, ceil_div(total, 256))), dim3(256), 0, st,
-                   static_cast<const T *>(dH_out->data), dH_out->ld, reinterpret_cast<const T *>(ctx + p.h_off), (int64_t)p.d_out,
-                   &b.counts[CNT_DST], p.rows, p.d_out, act ? act[n_layers - 1] : 1, dz_buf[(n_layers - 1) & 1]);
+        launch_pdl(relu_mask_kernel<T>, dim3((unsigned)std::max<int64_t>(1, ceil_div(total, 256)), (unsigned)n_rhs), dim3(256), 0, st,
+                   static_cast<const T *>(dH_out[0].data), dH_out[0].ld, reinterpret_cast<const T *>(ctx + p.h_off), (int64_t)p.d_out,
+                   &b.counts[CNT_DST], p.rows, p.d_out, act ? act[n_layers - 1] : 1, dz_buf[(n_layers - 1) & 1],
+                   static_cast<const T *>(dH_out[n_rhs - 1].data), dH_out[n_rhs - 1].ld);
     }
     SideStream *side = SideStream::get(st);
     cudaEvent_t dz_free[2] = {nullptr, nullptr};
@@ -234,7 +237,7 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
         // this call reads dW, so it runs on the helper stream beside the dCat product and the transposed
         // aggregation; `dz_free` holds the event after which the helper stream no longer reads a dZ buffer.
         cudaStream_t ws = st;
-        const bool dw_beside = side && (size_t)p.rows * (p.d_out + two_d) * sizeof(T) < dw_serial_bytes();
+        const bool dw_beside = side && (size_t)p.rows * (n_rhs * p.d_out + two_d) * sizeof(T) < dw_serial_bytes();
         if (dw_beside) {
             side->fork(st);
             ws = side->stream;
@@ -244,25 +247,31 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
         if (X->dtype == E2EGREC_BF16)
             dw_done = tc_weight_grad(reinterpret_cast<const __nv_bfloat16 *>(dz), p.rows, p.d_out,
                                      reinterpret_cast<const __nv_bfloat16 *>(cat), two_d, n_dst, part, kDwSplits,
-                                     &b.counts[CNT_STATUS], ws);
-        if (!dw_done) {
-            EpiPartial epi{part, two_d, (int64_t)p.d_out * two_d};
-            dim3 grid((unsigned)ceil_div(p.d_out, kGemmBM), (unsigned)ceil_div(two_d, kGemmBN), kDwSplits);
+                                     &b.counts[CNT_STATUS], ws, n_rhs);
+        const int64_t n_w = (int64_t)p.d_out * two_d;
+        if (dw_done) {
             note_launch();
-            gemm_simt_kernel<T, true, true, EpiPartial><<<grid, kGemmThreads, 0, ws>>>(
-                dz, p.d_out, cat, two_d, p.d_out, two_d, p.rows, nullptr, n_dst, epi);
-        }
-        {
-            const int64_t n = (int64_t)p.d_out * two_d;
-            note_launch();
-            launch_pdl(splitk_reduce_kernel, dim3((unsigned)ceil_div(n, 256)), dim3(256), 0, ws, part, n, kDwSplits, accumulate,
-                       dW[l], dw_done ? n_dst : nullptr);
+            launch_pdl(splitk_reduce_kernel, dim3((unsigned)ceil_div(n_w, 256)), dim3(256), 0, ws, part, n_w, kDwSplits, accumulate,
+                       dW[l], n_dst, n_rhs);
+        } else {
+            for (int r = 0; r < n_rhs; ++r) {             // fp32-FMA product: one right-hand side per pass, added up
+                EpiPartial epi{part, two_d, n_w};
+                dim3 grid((unsigned)ceil_div(p.d_out, kGemmBM), (unsigned)ceil_div(two_d, kGemmBN), kDwSplits);
+                note_launch();
+                gemm_simt_kernel<T, true, true, EpiPartial><<<grid, kGemmThreads, 0, ws>>>(
+                    dz + (int64_t)r * p.rows * p.d_out, p.d_out, cat, two_d, p.d_out, two_d, p.rows, nullptr, n_dst, epi);
+                note_launch();
+                launch_pdl(splitk_reduce_kernel, dim3((unsigned)ceil_div(n_w, 256)), dim3(256), 0, ws, part, n_w, kDwSplits,
+                           (accumulate || r > 0) ? 1 : 0, dW[l], (const int32_t *)nullptr, 1);
+            }
         }
         if (l == 0) tap_end(TAP_DW_OUTER, ws);
         if (dbias && dbias[l]) {
-            note_launch();
-            colsum_kernel<T><<<(unsigned)ceil_div(p.d_out, 32), 256, 0, ws>>>(dz, p.d_out, n_dst, p.d_out, accumulate,
-                                                                             dbias[l]);
+            for (int r = 0; r < n_rhs; ++r) {
+                note_launch();
+                colsum_kernel<T><<<(unsigned)ceil_div(p.d_out, 32), 256, 0, ws>>>(dz + (int64_t)r * p.rows * p.d_out, p.d_out, n_dst,
+                                                                                 p.d_out, (accumulate || r > 0) ? 1 : 0, dbias[l]);
+            }
         }
         if (dw_beside) {
             dz_free[l & 1] = side->event();
@@ -275,14 +284,17 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
             if (W[l].ld == two_d)               // W as stored: the product reads it with its N index contiguous
                 dcat_done = tc_dcat_backward(reinterpret_cast<const __nv_bfloat16 *>(dz), p.rows, p.d_out,
                                              static_cast<const __nv_bfloat16 *>(W[l].data), two_d, b.inv_cnt,
-                                             reinterpret_cast<__nv_bfloat16 *>(dcat), n_dst, &b.counts[CNT_STATUS], st);
+                                             reinterpret_cast<__nv_bfloat16 *>(dcat), n_dst, &b.counts[CNT_STATUS], st, n_rhs);
         }
         if (!dcat_done) {
-            EpiDCat<T> epi{dcat, two_d, p.d_in, b.inv_cnt};
-            dim3 grid((unsigned)std::max<int64_t>(1, ceil_div(p.rows, kGemmBM)), (unsigned)ceil_div(two_d, kGemmBN), 1);
-            note_launch();
-            gemm_simt_kernel<T, false, true, EpiDCat<T>><<<grid, kGemmThreads, 0, st>>>(
-                dz, p.d_out, static_cast<const T *>(W[l].data), two_d, p.rows, two_d, p.d_out, n_dst, nullptr, epi);
+            for (int r = 0; r < n_rhs; ++r) {
+                EpiDCat<T> epi{dcat + (int64_t)r * p.rows * two_d, two_d, p.d_in, b.inv_cnt};
+                dim3 grid((unsigned)std::max<int64_t>(1, ceil_div(p.rows, kGemmBM)), (unsigned)ceil_div(two_d, kGemmBN), 1);
+                note_launch();
+                gemm_simt_kernel<T, false, true, EpiDCat<T>><<<grid, kGemmThreads, 0, st>>>(
+                    dz + (int64_t)r * p.rows * p.d_out, p.d_out, static_cast<const T *>(W[l].data), two_d, p.rows, two_d, p.d_out,
+                    n_dst, nullptr, epi);
+            }
         }
         if (l == 0) tap_end(TAP_DCAT_OUTER, st);
         // transposed aggregation: gather over the block's CSC, plus the self rows, masked by the
@@ -292,6 +304,8 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
         o.ld_self = two_d;
         o.n_self = n_dst;
         o.mean = 0;
+        o.n_rhs = n_rhs;
+        o.rhs_in = o.rhs_self = (int64_t)p.rows * two_d;
         if (l > 0) {
             // the buffer that receives dZ of the layer below may still be read by the helper stream (layer l+1)
             if (side && dz_free[(l - 1) & 1]) {
@@ -301,16 +315,18 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
             o.out = dz_buf[(l - 1) & 1];
             o.ld_out = p.d_in;
             o.pad_rows = plan[l - 1].rows;
+            o.rhs_out = plan[l - 1].rows * p.d_in;
             const int relu_below = act ? act[l - 1] : 1;
             o.mask = relu_below ? reinterpret_cast<const T *>(ctx + plan[l - 1].h_off) : nullptr;
             o.ld_mask = p.d_in;
         } else {
-            o.out = static_cast<T *>(dX_rows->data);
-            o.ld_out = dX_rows->ld;
+            o.out = static_cast<T *>(dX_rows[0].data);
+            o.ld_out = dX_rows[0].ld;
             o.mask = nullptr;
+            o.rhs_out = static_cast<T *>(dX_rows[n_rhs - 1].data) - static_cast<T *>(dX_rows[0].data);
         }
         if (l == 0) tap_begin(TAP_AGG_BWD_OUTER, st);
-        SegScratch sc = seg_scratch_carve(b.cap_edges, block_run_len(b.cap_edges), p.d_in, dtype_size(X->dtype), scratch + bs.seg_off);
+        SegScratch sc = seg_scratch_carve(b.cap_edges, block_run_len(b.cap_edges), p.d_in, dtype_size(X->dtype), scratch + bs.seg_off, n_rhs);
         sc.chain_cnt = reinterpret_cast<int32_t *>(scratch + bs.chain_off);
         const bool seg_ok = dispatch_seg_reduce<T, int32_t, false>(dcat + p.d_in, two_d, b.csc_ptr, b.csc_row, &b.counts[CNT_SRC], 0,
                                                                    b.cap_src, nullptr, block_run_len(b.cap_edges), p.d_in, X->dtype,
@@ -367,34 +383,57 @@ extern "C" int32_t e2egrec_sage_ctx_layout(const e2egrec_block *blocks, int32_t 
     return E2EGREC_OK;
 }
 
+static int32_t sage_backward_entry(const e2egrec_block *blocks, int32_t n_layers, const e2egrec_mat *X, const e2egrec_mat *W,
+                                   const int32_t *act, const void *ctx, const e2egrec_mat *dH_out, int32_t n_rhs,
+                                   float *const *dW, float *const *dbias, const e2egrec_mat *dX_rows, void *scratch,
+                                   size_t *scratch_bytes, uint32_t flags, void *stream)
+{
+    if (!scratch_bytes) return E2EGREC_ERR_NULL;
+    if (n_rhs < 1 || n_rhs > 2) return E2EGREC_ERR_ARG;
+    LayerPlan plan[kMaxHops];
+    size_t ctx_need = 0;
+    int32_t rc = plan_layers(blocks, n_layers, X, W, plan, &ctx_need);
+    if (rc != E2EGREC_OK) return rc;
+    const BackwardScratch bs = plan_backward(blocks, n_layers, plan, dtype_size(X->dtype), n_rhs);
+    if (!scratch) { *scratch_bytes = bs.bytes; return E2EGREC_OK; }
+    if (*scratch_bytes < bs.bytes) { *scratch_bytes = bs.bytes; return E2EGREC_ERR_WORKSPACE; }
+    if (reinterpret_cast<uintptr_t>(scratch) % 256 || reinterpret_cast<uintptr_t>(ctx) % 256) return E2EGREC_ERR_ALIGN;
+    if (!ctx || !dH_out || !dW || !dX_rows) return E2EGREC_ERR_NULL;
+    for (int l = 0; l < n_layers; ++l)
+        if (!dW[l]) return E2EGREC_ERR_NULL;
+    const size_t es = dtype_size(X->dtype);
+    for (int r = 0; r < n_rhs; ++r) {
+        if (!dH_out[r].data || !dX_rows[r].data) return E2EGREC_ERR_NULL;
+        if (dH_out[r].dtype != X->dtype || dX_rows[r].dtype != X->dtype) return E2EGREC_ERR_DTYPE;
+        if (dH_out[r].dim != plan[n_layers - 1].d_out || dX_rows[r].dim != X->dim) return E2EGREC_ERR_ARG;
+        if (dX_rows[r].rows < blocks[n_layers - 1].cap_src || dH_out[r].rows < blocks[0].cap_dst) return E2EGREC_ERR_ARG;
+        if ((dX_rows[r].ld * es) % 16 || reinterpret_cast<uintptr_t>(dX_rows[r].data) % 16) return E2EGREC_ERR_ALIGN;
+        if (dX_rows[r].ld != dX_rows[0].ld) return E2EGREC_ERR_ARG;       // the results share one leading dimension
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (SideStream *side = SideStream::get(st)) side->join_pending(st);     // a deferred block transposition
+    if (X->dtype == E2EGREC_BF16)
+        return backward_impl<__nv_bfloat16>(blocks, n_layers, X, W, act, plan, static_cast<const char *>(ctx), dH_out, n_rhs, dW,
+                                            dbias, dX_rows, static_cast<char *>(scratch), bs, flags, st);
+    return backward_impl<float>(blocks, n_layers, X, W, act, plan, static_cast<const char *>(ctx), dH_out, n_rhs, dW, dbias,
+                                dX_rows, static_cast<char *>(scratch), bs, flags, st);
+}
+
 extern "C" int32_t e2egrec_sage_backward(const e2egrec_block *blocks, int32_t n_layers, const e2egrec_mat *X,
                                          const e2egrec_mat *W, const int32_t *act, const void *ctx,
                                          const e2egrec_mat *dH_out, float *const *dW, float *const *dbias,
                                          const e2egrec_mat *dX_rows, void *scratch, size_t *scratch_bytes,
                                          uint32_t flags, void *stream)
 {
-    if (!scratch_bytes) return E2EGREC_ERR_NULL;
-    LayerPlan plan[kMaxHops];
-    size_t ctx_need = 0;
-    int32_t rc = plan_layers(blocks, n_layers, X, W, plan, &ctx_need);
-    if (rc != E2EGREC_OK) return rc;
-    const BackwardScratch bs = plan_backward(blocks, n_layers, plan, dtype_size(X->dtype));
-    if (!scratch) { *scratch_bytes = bs.bytes; return E2EGREC_OK; }
-    if (*scratch_bytes < bs.bytes) { *scratch_bytes = bs.bytes; return E2EGREC_ERR_WORKSPACE; }
-    if (reinterpret_cast<uintptr_t>(scratch) % 256 || reinterpret_cast<uintptr_t>(ctx) % 256) return E2EGREC_ERR_ALIGN;
-    if (!ctx || !dH_out || !dH_out->data || !dW || !dX_rows || !dX_rows->data) return E2EGREC_ERR_NULL;
-    for (int l = 0; l < n_layers; ++l)
-        if (!dW[l]) return E2EGREC_ERR_NULL;
-    if (dH_out->dtype != X->dtype || dX_rows->dtype != X->dtype) return E2EGREC_ERR_DTYPE;
-    if (dH_out->dim != plan[n_layers - 1].d_out || dX_rows->dim != X->dim) return E2EGREC_ERR_ARG;
-    if (dX_rows->rows < blocks[n_layers - 1].cap_src || dH_out->rows < blocks[0].cap_dst) return E2EGREC_ERR_ARG;
-    const size_t es = dtype_size(X->dtype);
-    if ((dX_rows->ld * es) % 16 || reinterpret_cast<uintptr_t>(dX_rows->data) % 16) return E2EGREC_ERR_ALIGN;
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (SideStream *side = SideStream::get(st)) side->join_pending(st);     // a deferred block transposition
-    if (X->dtype == E2EGREC_BF16)
-        return backward_impl<__nv_bfloat16>(blocks, n_layers, X, W, act, plan, static_cast<const char *>(ctx), dH_out, dW,
-                                            dbias, dX_rows, static_cast<char *>(scratch), bs, flags, st);
-    return backward_impl<float>(blocks, n_layers, X, W, act, plan, static_cast<const char *>(ctx), dH_out, dW, dbias,
-                                dX_rows, static_cast<char *>(scratch), bs, flags, st);
+    return sage_backward_entry(blocks, n_layers, X, W, act, ctx, dH_out, 1, dW, dbias, dX_rows, scratch, scratch_bytes, flags, stream);
+}
+
+extern "C" int32_t e2egrec_sage_backward_multi(const e2egrec_block *blocks, int32_t n_layers, const e2egrec_mat *X,
+                                               const e2egrec_mat *W, const int32_t *act, const void *ctx,
+                                               const e2egrec_mat *dH_out, int32_t n_rhs, float *const *dW, float *const *dbias,
+                                               const e2egrec_mat *dX_rows, void *scratch, size_t *scratch_bytes,
+                                               uint32_t flags, void *stream)
+{
+    return sage_backward_entry(blocks, n_layers, X, W, act, ctx, dH_out, n_rhs, dW, dbias, dX_rows, scratch, scratch_bytes, flags,
+                               stream);
 }

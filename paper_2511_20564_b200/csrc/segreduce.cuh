@@ -44,13 +44,15 @@ struct SegScratch {
     int32_t *chain_cnt;
 };
 
-inline size_t seg_chain_bytes(int64_t cap_entries, int run_len, int d, size_t elem_size)
+inline size_t seg_chain_bytes(int64_t cap_entries, int run_len, int d, size_t elem_size, int n_rhs = 1)
 {
     const int64_t runs = ceil_div(cap_entries > 0 ? cap_entries : 1, run_len);
-    return align_up((size_t)ceil_div(runs, seg_runs_per_window(d, elem_size)) * sizeof(int32_t), 256);
+    return align_up((size_t)n_rhs * ceil_div(runs, seg_runs_per_window(d, elem_size)) * sizeof(int32_t), 256);
 }
 
-inline SegScratch seg_scratch_carve(int64_t cap_entries, int run_len, int d, size_t elem_size, void *base)
+// n_rhs right-hand sides (SegOut::n_rhs) keep their partial rows side by side: every array holds n_rhs blocks of
+// n_windows entries.
+inline SegScratch seg_scratch_carve(int64_t cap_entries, int run_len, int d, size_t elem_size, void *base, int n_rhs = 1)
 {
     SegScratch s{};
     s.runs_per_window = seg_runs_per_window(d, elem_size);
@@ -62,9 +64,9 @@ inline SegScratch seg_scratch_carve(int64_t cap_entries, int run_len, int d, siz
         off += align_up(bytes, 256);
         return p;
     };
-    s.head2 = (float *)take((size_t)s.n_windows * d * sizeof(float));
-    s.tail2 = (float *)take((size_t)s.n_windows * d * sizeof(float));
-    s.win_info = (int4 *)take((size_t)s.n_windows * sizeof(int4));
+    s.head2 = (float *)take((size_t)n_rhs * s.n_windows * d * sizeof(float));
+    s.tail2 = (float *)take((size_t)n_rhs * s.n_windows * d * sizeof(float));
+    s.win_info = (int4 *)take((size_t)n_rhs * s.n_windows * sizeof(int4));
     s.bytes = off;
     return s;
 }
@@ -554,6 +556,15 @@ seg_run_block_kernel(const T *__restrict__ in, int64_t ld_in, const int32_t *__r
     const int64_t run = (int64_t)blockIdx.x * RB + rl;
     pdl_launch_dependents();
     pdl_wait();                                    // the kernel before this one in the stream has completed
+    if (blockIdx.y) {                              // the second right-hand side: other rows, same segments
+        const int64_t r = blockIdx.y, nw = gridDim.x;
+        in += r * o.rhs_in;
+        o.self += r * o.rhs_self;
+        o.out += r * o.rhs_out;
+        head2 += r * nw * d;
+        tail2 += r * nw * d;
+        if (chain_cnt) chain_cnt += r * nw;
+    }
     const int32_t n_seg = *n_seg_dev;
     const int32_t total = n_seg > 0 ? ptr[n_seg] : 0;
     const int64_t k0 = run * run_len;
@@ -871,19 +882,39 @@ inline void launch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const
                               const int32_t *seg_of, const SegScratch &sc, const SegOut<T> &o, cudaStream_t st)
 {
     constexpr size_t smem = seg_run_smem_bytes<LPR, CPL, Chunk<T>::kElems>();
+    bool block_form = false;
+    if constexpr (CPL == 1 && !kWeight && sizeof(PtrT) == 4)
+        block_form = seg_of && n_seg_dev && o.self && !o.mean && !o.seg_scale && !seg_general_only();
+    if (o.n_rhs > 1 && !(block_form && sc.chain_cnt)) {
+        // the general kernels take one right-hand side per pass
+        for (int r = 0; r < o.n_rhs; ++r) {
+            SegOut<T> o1 = o;
+            o1.n_rhs = 1;
+            o1.out = o.out + r * o.rhs_out;
+            if (o.self) o1.self = o.self + r * o.rhs_self;
+            SegScratch s1 = sc;
+            s1.head2 = sc.head2 + (size_t)r * sc.n_windows * d;
+            s1.tail2 = sc.tail2 + (size_t)r * sc.n_windows * d;
+            s1.win_info = sc.win_info + (size_t)r * sc.n_windows;
+            s1.chain_cnt = nullptr;
+            launch_seg_reduce<T, PtrT, LPR, CPL, kWeight, kInFlight>(in + r * o.rhs_in, ld_in, ptr, idx, n_seg_dev, n_seg_host, cap_seg, w,
+                                                                     run_len, d, seg_of, s1, o1, st);
+        }
+        return;
+    }
     tap_begin(TAP_SEG_L1, st);
     note_launch();
     const unsigned grid1 = (unsigned)sc.n_windows;
-    bool block_form = false;
     if constexpr (CPL == 1 && !kWeight && sizeof(PtrT) == 4) {
         // the transposed aggregation of a sampled block: the kernel written for that case
-        if (seg_of && n_seg_dev && o.self && !o.mean && !o.seg_scale && !seg_general_only()) {
+        if (block_form) {
             block_form = true;
+            const dim3 grid_b(grid1, (unsigned)(o.n_rhs > 1 && sc.chain_cnt ? o.n_rhs : 1));
             if (o.mask)
-                launch_pdl(seg_run_block_kernel<T, LPR, true>, dim3(grid1), dim3(kAggThreads), smem, st, in, ld_in, ptr, idx, seg_of,
+                launch_pdl(seg_run_block_kernel<T, LPR, true>, grid_b, dim3(kAggThreads), smem, st, in, ld_in, ptr, idx, seg_of,
                            n_seg_dev, run_len, d, sc.head2, sc.tail2, sc.win_info, sc.cap_runs, sc.chain_cnt, o);
             else
-                launch_pdl(seg_run_block_kernel<T, LPR, false>, dim3(grid1), dim3(kAggThreads), smem, st, in, ld_in, ptr, idx, seg_of,
+                launch_pdl(seg_run_block_kernel<T, LPR, false>, grid_b, dim3(kAggThreads), smem, st, in, ld_in, ptr, idx, seg_of,
                            n_seg_dev, run_len, d, sc.head2, sc.tail2, sc.win_info, sc.cap_runs, sc.chain_cnt, o);
             if (sc.chain_cnt) {                   // chains, empty segments and padding were all done in that launch
                 tap_end(TAP_SEG_L1, st);
