@@ -135,11 +135,13 @@ template <> struct Chunk<__nv_bfloat16> {
 };
 
 // Two fp32 adds in one instruction (packed f32x2 of sm_100): the same round-to-nearest result per element as
-// two scalar adds, at half the issue slots.
+// two scalar adds, at half the issue slots.  Through the compiler's builtin, so that it can keep the operands in
+// aligned register pairs instead of packing and unpacking them around the instruction.
 __device__ __forceinline__ void add2(float &a0, float &a1, float b0, float b1)
 {
-    asm("{ .reg .b64 ra, rb;\n mov.b64 ra, {%0, %1};\n mov.b64 rb, {%2, %3};\n add.rn.f32x2 ra, ra, rb;\n mov.b64 {%0, %1}, ra; }"
-        : "+f"(a0), "+f"(a1) : "f"(b0), "f"(b1));
+    const float2 r = __fadd2_rn(make_float2(a0, a1), make_float2(b0, b1));
+    a0 = r.x;
+    a1 = r.y;
 }
 template <typename T> __device__ inline float to_float(T v);
 template <> __device__ inline float to_float<float>(float v) { return v; }

@@ -3,12 +3,14 @@
 //   D[m, n] = sum_k A[m, k] * B[n, k]        A: [rows x K] row-major, B: [N x K] row-major (both K-major)
 //
 // Output tiles are 128 x NT (NT = the widest multiple of 32, at most 256, that divides N).  A single thread feeds TMA
-// loads of 128 x 64 (A) and NT x 64 (B) bf16 boxes into a ring of 128-byte-swizzled shared-memory stages,
-// a single thread issues tcgen05.mma (M = 128, N = NT, K = 16 per instruction) into an fp32
-// accumulator in tensor memory, and four warps read the accumulator back with tcgen05.ld for
-// the epilogue (bias / ReLU / per-row scale, bf16 store).  No cluster launch, no multicast.
-// Every mbarrier wait is bounded; on a timeout the CTA raises E2EGREC_DEV_TIMEOUT in the status
-// word, skips its stores, releases its tensor memory and returns.
+// loads of 128 x 64 (A) and NT x 64 (B) bf16 boxes into a ring of 128-byte-swizzled shared-memory stages that runs on
+// across tiles, a single thread issues tcgen05.mma (M = 128, N = NT, K = 16 per instruction) into one of two fp32
+// accumulators in tensor memory, and eight warps read the other accumulator back with tcgen05.ld for the epilogue
+// (bias / ReLU / per-row scale / mask, rounding to bf16).  Where NT is a multiple of 64 the plain epilogue stages boxes of
+// 128 rows x 64 columns in shared memory and sends them off with bulk tensor stores (whole 128-byte lines; a lane's own
+// 16-byte stores fill only half a sector each); otherwise, and in the fused forms, each lane stores its row's columns.
+// No cluster launch, no multicast.  Every mbarrier wait is bounded; on a timeout the CTA raises E2EGREC_DEV_TIMEOUT in
+// the status word, skips its remaining tiles, releases its tensor memory and returns.
 #include "gemm_tc.cuh"
 
 #include <cuda.h>
@@ -71,6 +73,27 @@ __device__ inline void tma_load_2d(void *smem_dst, const CUtensorMap *map, int x
         "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(smem_u32(bar))
         : "memory");
+}
+
+// Bulk tensor store shared -> global of one box, and the bookkeeping of such stores (issued and awaited by one thread).
+__device__ inline void tma_store_2d(const CUtensorMap *map, const void *smem_src, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];" ::"l"(reinterpret_cast<uint64_t>(map)),
+                 "r"(x), "r"(y), "r"(smem_u32(smem_src))
+                 : "memory");
+}
+__device__ inline void tma_store_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N> __device__ inline void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+__device__ inline void named_barrier(int id, int threads) { asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory"); }
+// barrier over `threads` threads that also tells every one of them whether all arrived with ok set
+__device__ inline bool named_barrier_all(int id, int threads, bool ok)
+{
+    uint32_t r;
+    asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.and.pred p, %2, %3, q;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(r)
+                 : "r"((uint32_t)ok), "r"(id), "r"(threads)
+                 : "memory");
+    return r != 0;
 }
 
 __device__ inline void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -170,7 +193,51 @@ struct TcEpilogue {
     // indexed by the row inside its block.  n_rhs = 1: one block, rhs_rows unused.
     int n_rhs;
     int64_t rhs_rows;
+    int tma_out;               // the output leaves through bulk tensor stores of 128 x 64 boxes staged in shared memory (map_out)
+    int mode;                  // which steps the plain epilogue has (epi_mode), fixed on the host
 };
+
+// Steps of the plain epilogue as bits: bias, ReLU, mask, and the row scale either for whole blocks of 32 columns
+// (scale_from a multiple of 32) or decided column by column.
+constexpr int kEpiBias = 1, kEpiRelu = 2, kEpiMask = 4, kEpiScaleBlock = 8, kEpiScaleColumn = 16;
+
+// One block of 32 accumulator columns of one row -> 16 packed bf16 pairs:  v = max((acc + bias) * scale, floor), zero where the
+// row is dead or the mask says so.  Bias, ReLU and a scale that holds for the whole block are plain arithmetic with neutral
+// operands when absent (bias 0, floor -inf, scale 1); the mask and a scale that starts inside a block are compiled in.
+// keep: bit j set = column j keeps its value (mask and liveness folded together).
+template <bool kMask, bool kScaleColumn>
+__device__ inline void epi_block(const uint32_t (&r)[32], uint32_t (&packed)[16], const float *__restrict__ bias_c, bool bias_vec,
+                                 float floor_v, float s_block, float rs, int col0, int scale_from, uint32_t keep, bool live)
+{
+#pragma unroll
+    for (int q = 0; q < 8; ++q) {
+        float b[4] = {0.f, 0.f, 0.f, 0.f};
+        if (bias_c) {
+            if (bias_vec) {
+                const float4 v = __ldg(reinterpret_cast<const float4 *>(bias_c) + q);
+                b[0] = v.x; b[1] = v.y; b[2] = v.z; b[3] = v.w;
+            } else {
+#pragma unroll
+                for (int h = 0; h < 4; ++h) b[h] = bias_c[4 * q + h];
+            }
+        }
+        float v[4];
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+            const int j = 4 * q + h;
+            v[h] = fmaxf((__uint_as_float(r[j]) + b[h]) * s_block, floor_v);
+            if constexpr (kScaleColumn) { if (col0 + j >= scale_from) v[h] *= rs; }
+            if constexpr (kMask) { if (!((keep >> j) & 1u)) v[h] = 0.f; }
+        }
+        __nv_bfloat162 p0 = __floats2bfloat162_rn(v[0], v[1]), p1 = __floats2bfloat162_rn(v[2], v[3]);
+        packed[2 * q] = *reinterpret_cast<uint32_t *>(&p0);
+        packed[2 * q + 1] = *reinterpret_cast<uint32_t *>(&p1);
+    }
+    if constexpr (!kMask) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) packed[i] = live ? packed[i] : 0u;
+    }
+}
 
 __device__ inline float bf16_round(float v) { return __bfloat162float(__float2bfloat16_rn(v)); }
 
@@ -199,12 +266,98 @@ __device__ inline void mbar_arrive(uint64_t *bar)
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
+// What the plain epilogue knows about its row of the current tile.
+struct EpiRow {
+    const TcEpilogue *ep;
+    const CUtensorMap *map_out;
+    __nv_bfloat16 *orow, *orow2;         // the row's slice of the output tile (and of the second copy, or null)
+    const __nv_bfloat16 *mrow;           // the row's slice of the mask, or null
+    uint8_t *out_stage;                  // the two staging boxes of the bulk stores
+    float rs, floor_v;
+    int n0, m0, rt;                      // first column / row of the tile, the row inside the tile
+    bool live, bias_vec, store_lead;
+};
+
+// One block of 32 columns of one row, from accumulator registers to memory.
+template <bool kMask, bool kScaleColumn>
+__device__ inline void epi_finish_block(const EpiRow &e, const uint32_t (&r)[32], int c, uint32_t &n_box)
+{
+    const TcEpilogue &ep = *e.ep;
+    uint32_t keep = e.live ? 0xFFFFFFFFu : 0u;
+    if (kMask && e.live) {
+        keep = 0;
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const uint4 mv = *reinterpret_cast<const uint4 *>(e.mrow + c + q * 8);
+            const uint32_t w[4] = {mv.x, mv.y, mv.z, mv.w};
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (__uint_as_float(w[u] << 16) > 0.f) keep |= 1u << (q * 8 + 2 * u);
+                if (__uint_as_float(w[u] & 0xFFFF0000u) > 0.f) keep |= 1u << (q * 8 + 2 * u + 1);
+            }
+        }
+    }
+    uint32_t packed[16];
+    const float s_block = ((ep.mode & kEpiScaleBlock) && e.n0 + c >= ep.scale_from) ? e.rs : 1.f;
+    epi_block<kMask, kScaleColumn>(r, packed, ep.bias ? ep.bias + e.n0 + c : nullptr, e.bias_vec, e.floor_v, s_block, e.rs, e.n0 + c,
+                                   ep.scale_from, keep, e.live);
+    if (ep.tma_out) {
+        // The eight warps fill one box of 128 rows x 64 columns (warps 2-5 its left half, 6-9 its right half) in the
+        // 128-byte swizzle of the output map, and one thread sends it off as whole lines; two boxes alternate, so a box
+        // is refilled only after the store issued two boxes earlier has read it.
+        uint8_t *box = e.out_stage + (size_t)(n_box & 1u) * (kTileM * 128);
+        ++n_box;
+        if (e.store_lead) tma_store_wait_read<1>();
+        named_barrier(1, kTnEpilogueWarps * 32);
+        const int chunk0 = ((c >> 5) & 1) * 4;
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            *reinterpret_cast<uint4 *>(box + e.rt * 128 + (((chunk0 + q) ^ (e.rt & 7)) << 4)) =
+                make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        named_barrier(1, kTnEpilogueWarps * 32);
+        if (e.store_lead) {
+            tma_store_2d(e.map_out, box, e.n0 + (c & ~63), e.m0);
+            tma_store_commit();
+        }
+    } else {
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            *reinterpret_cast<uint4 *>(e.orow + c + q * 8) =
+                make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+    }
+    if (e.orow2) {
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+            *reinterpret_cast<uint4 *>(e.orow2 + c + q * 8) =
+                make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
+    }
+}
+
+// The blocks of 32 columns (c_first, c_first + 64, ...) that one warp takes from a finished accumulator; the accumulator
+// buffer goes back to the MMA warp as soon as the warp's last block is in registers.
+template <bool kMask, bool kScaleColumn>
+__device__ inline void epi_tile_plain(const EpiRow &e, uint32_t taddr, int c_first, int nt, uint64_t *acc_empty, int lane, uint32_t &n_box)
+{
+    for (int c = c_first; c < nt; c += 64) {
+        uint32_t r[32];
+        tmem_load32(taddr + (uint32_t)c, r);
+        if (c + 64 >= nt) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty);
+        }
+        epi_finish_block<kMask, kScaleColumn>(e, r, c, n_box);
+    }
+}
+
 // kFuse: the gating / product-plus-term forms of the epilogue (TcFuse); the plain instantiation carries none of their
 // registers or branches.
 template <bool kFuse>
 __global__ void __launch_bounds__(kTnThreads)
-tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, int k_blocks,
-                  int stages, int nt, int n_tiles_n, uint32_t tmem_cols, int b_mn, TcEpilogue ep)
+tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                  const __grid_constant__ CUtensorMap map_out, int k_blocks, int stages, int nt, int n_tiles_n, uint32_t tmem_cols,
+                  int b_mn, TcEpilogue ep)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ uint64_t full_bar[kMaxStages], empty_bar[kMaxStages], acc_full[2], acc_empty[2];
@@ -217,6 +370,7 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const uint32_t a_bytes = kTileM * kTileK * 2, b_bytes = (uint32_t)nt * kTileK * 2;
     uint8_t *a_tiles = tiles;
     uint8_t *b_tiles = tiles + (size_t)stages * a_bytes;
+    uint8_t *out_stage = b_tiles + (size_t)stages * b_bytes;      // two boxes of 128 rows x 128 bytes (ep.tma_out)
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < stages; ++s) {
@@ -325,10 +479,14 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const int c_first = warp >= 6 ? 32 : 0;     // warps 2-5 take column blocks 0, 2, 4, ...; warps 6-9 the odd ones
         int c_last = c_first;                       // this warp's last column block
         while (c_last + 64 < nt) c_last += 64;
-        uint32_t lt = 0;
+        uint32_t lt = 0, n_box = 0;                 // n_box: boxes of 64 columns handed to the bulk stores so far
+        const bool store_lead = warp == 2 && lane == 0;
         for (int64_t t = blockIdx.x; t < n_work; t += gridDim.x, ++lt) {
             const uint32_t buf = lt & 1u;
-            if (!mbar_wait(&acc_full[buf], (lt >> 1) & 1u, &abort_flag)) break;
+            bool ready = mbar_wait(&acc_full[buf], (lt >> 1) & 1u, &abort_flag);
+            // with staged stores the warps meet at barriers inside the tile: all of them take it, or none does
+            if (!kFuse && ep.tma_out) ready = named_barrier_all(2, kTnEpilogueWarps * 32, ready);
+            if (!ready) break;
             tc_fence_after();
             int64_t m0, m0_local;
             tile_rows(t, m0, m0_local);
@@ -344,6 +502,31 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 if (lane == 0) mbar_arrive(&acc_empty[buf]);
                 continue;
             }
+            if constexpr (!kFuse) {
+                EpiRow e;
+                e.ep = &ep;
+                e.map_out = &map_out;
+                e.orow = orow;
+                e.orow2 = orow2;
+                e.mrow = mrow;
+                e.out_stage = out_stage;
+                e.rs = rs;
+                e.n0 = n0;
+                e.m0 = (int)m0;
+                e.rt = lg * 32 + lane;
+                e.live = live;
+                e.bias_vec = (reinterpret_cast<uintptr_t>(ep.bias) & 15) == 0;
+                e.store_lead = store_lead;
+                const uint32_t taddr = tmem_base + buf * buf_stride + ((uint32_t)(lg * 32) << 16);
+                e.floor_v = ep.relu ? 0.f : -INFINITY;
+                if (ep.mode & kEpiMask) {
+                    if (ep.mode & kEpiScaleColumn) epi_tile_plain<true, true>(e, taddr, c_first, nt, &acc_empty[buf], lane, n_box);
+                    else epi_tile_plain<true, false>(e, taddr, c_first, nt, &acc_empty[buf], lane, n_box);
+                } else {
+                    if (ep.mode & kEpiScaleColumn) epi_tile_plain<false, true>(e, taddr, c_first, nt, &acc_empty[buf], lane, n_box);
+                    else epi_tile_plain<false, false>(e, taddr, c_first, nt, &acc_empty[buf], lane, n_box);
+                }
+            } else {
             for (int c = c_first; c < nt; c += 64) {
                 uint32_t r[32];
                 tmem_load32(tmem_base + buf * buf_stride + ((uint32_t)(lg * 32) << 16) + (uint32_t)c, r);
@@ -435,7 +618,9 @@ tc_gemm_tn_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                             make_uint4(packed[4 * q], packed[4 * q + 1], packed[4 * q + 2], packed[4 * q + 3]);
                 }
             }
+            }
         }
+        if (store_lead) tma_store_wait_read<0>();   // the staging boxes have been read; the kernel's end publishes the stores
     }
     tc_fence_before();
     __syncthreads();
@@ -464,6 +649,7 @@ EncodeTiledFn encode_fn()
 }
 
 constexpr int kMaxDevices = 64;
+constexpr int kMaxDynSmem = 226 * 1024;             // of the 227 KB a block may have; the kernels' static part is below 1 KB
 
 int current_device()
 {
@@ -491,7 +677,7 @@ bool raise_smem_limit(Kernel kernel, bool (&done)[kMaxDevices])
 {
     const int dev = current_device();
     if (done[dev]) return true;
-    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024) != cudaSuccess) return false;
+    if (cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMaxDynSmem) != cudaSuccess) return false;
     done[dev] = true;
     return true;
 }
@@ -528,15 +714,32 @@ bool launch_tn(const __nv_bfloat16 *A, int64_t rows, int k, int64_t lda, const _
     if (reinterpret_cast<uintptr_t>(A) % 16 || reinterpret_cast<uintptr_t>(B) % 16 || (lda * 2) % 16 || (ldb * 2) % 16 ||
         reinterpret_cast<uintptr_t>(ep.out) % 16 || (ep.ldo * 2) % 16)
         return false;
-    CUtensorMap ma, mb;
-    if (!make_map(&ma, A, rows * n_rhs, k, lda, kTileM)) return false;
-    if (b_mn ? (ldb != n || !make_map_mn(&mb, B, k, n)) : !make_map(&mb, B, n, k, ldb, nt)) return false;
+    const bool fused = ep.fuse.gate_in || ep.fuse.add_a;
     const int k_blocks = k / kTileK;
-    const int stages = k_blocks < kMaxStages ? k_blocks : kMaxStages;
+    // the stage ring runs on across tiles, so a short K still keeps kMaxStages loads in flight (the next tiles' operands)
+    // Two to kMaxStages stages inside a budget that leaves a quarter of the SM's shared memory to the blocks of other
+    // streams' kernels: the stage ring runs on across tiles, and a third or fourth stage buys this kernel less than the
+    // co-resident blocks of the sampling kernels lose when they find no room (E2EGREC_GEMM_SMEM_KB overrides the budget).
+    static const bool direct_only = []() { const char *e = getenv("E2EGREC_GEMM_DIRECT_STORE"); return e && *e && e[0] != '0'; }();
+    static const size_t budget = []() {
+        const char *e = getenv("E2EGREC_GEMM_SMEM_KB");
+        const long kb = e && *e ? atol(e) : 178;
+        return (size_t)std::min<long>(std::max<long>(kb, 64), kMaxDynSmem / 1024) * 1024;
+    }();
+    const size_t stage_bytes = kTileM * kTileK * 2 + (size_t)nt * kTileK * 2;
+    ep.tma_out = !fused && !direct_only && nt % 64 == 0;
+    const size_t fixed_bytes = 1024 + (ep.tma_out ? 2 * kTileM * 128 : 0);
+    const int stages = (int)std::max<size_t>(2, std::min<size_t>(kMaxStages, (budget - fixed_bytes) / stage_bytes));
+    const size_t smem = (size_t)stages * stage_bytes + fixed_bytes;
+    ep.mode = (ep.bias ? kEpiBias : 0) | (ep.relu ? kEpiRelu : 0) | (ep.mask ? kEpiMask : 0) |
+              (ep.row_scale ? (ep.scale_from % 32 == 0 ? kEpiScaleBlock : kEpiScaleColumn) : 0);
+    CUtensorMap ma, mb, mo;
+    if (!make_map(&ma, A, rows * n_rhs, k, lda, kTileM)) return false;
+    if (ep.tma_out ? !make_map(&mo, ep.out, rows * n_rhs, n, ep.ldo, kTileM) : false) return false;
+    if (!ep.tma_out) mo = ma;
+    if (b_mn ? (ldb != n || !make_map_mn(&mb, B, k, n)) : !make_map(&mb, B, n, k, ldb, nt)) return false;
     uint32_t tmem_cols = 64;                    // two accumulator buffers, each a power of two of columns >= nt
     while ((int)tmem_cols < 2 * nt) tmem_cols <<= 1;
-    const size_t smem = (size_t)stages * (kTileM * kTileK * 2 + (size_t)nt * kTileK * 2) + 1024;
-    const bool fused = ep.fuse.gate_in || ep.fuse.add_a;
     static bool attr_set[2][kMaxDevices] = {};
     if (!(fused ? raise_smem_limit(tc_gemm_tn_kernel<true>, attr_set[1]) : raise_smem_limit(tc_gemm_tn_kernel<false>, attr_set[0])))
         return false;
@@ -545,10 +748,10 @@ bool launch_tn(const __nv_bfloat16 *A, int64_t rows, int k, int64_t lda, const _
     const unsigned grid = (unsigned)std::min<int64_t>(tiles_cap, sm_count());
     note_launch();
     if (fused)
-        launch_pdl(tc_gemm_tn_kernel<true>, dim3(grid), dim3(kTnThreads), smem, st, ma, mb, k_blocks, stages, nt, n_tiles_n, tmem_cols,
+        launch_pdl(tc_gemm_tn_kernel<true>, dim3(grid), dim3(kTnThreads), smem, st, ma, mb, mo, k_blocks, stages, nt, n_tiles_n, tmem_cols,
                    b_mn ? 1 : 0, ep);
     else
-        launch_pdl(tc_gemm_tn_kernel<false>, dim3(grid), dim3(kTnThreads), smem, st, ma, mb, k_blocks, stages, nt, n_tiles_n, tmem_cols,
+        launch_pdl(tc_gemm_tn_kernel<false>, dim3(grid), dim3(kTnThreads), smem, st, ma, mb, mo, k_blocks, stages, nt, n_tiles_n, tmem_cols,
                    b_mn ? 1 : 0, ep);
     return true;
 }
@@ -777,7 +980,7 @@ bool tc_weight_grad(const __nv_bfloat16 *dY, int64_t rows, int m, const __nv_bfl
     if (!make_map_mn(&my, dY, rows * n_rhs, m) || !make_map_mn(&mx, Xin, rows, n)) return false;
     uint32_t tmem_cols = 32;
     while ((int)tmem_cols < nt) tmem_cols <<= 1;
-    const int stages = kMaxStages;
+    const int stages = 4;
     const size_t smem = (size_t)stages * ((kTileM / 64) + (nt / 64)) * (kTileK * 128) + 1024;
     static bool attr_set[kMaxDevices] = {};
     if (!raise_smem_limit(tc_gemm_rows_kernel, attr_set)) return false;
