@@ -901,6 +901,285 @@ bool make_map_mn(CUtensorMap *map, const void *base, int64_t rows, int64_t cols)
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+
+// ------------------------------------------------------------------------- aggregation fused into the A operand
+// Eq. 2 and Eq. 3 of one layer in one kernel:  h' = act([h_self | mean of the sampled neighbours] W^T + b).  Gather warps
+// build the 128 x 2d rows of a tile of Cat in shared memory, in the 128-byte-swizzled k-block layout the tensor cores read
+// (the layout a TMA load of the stored Cat would leave there), and store the same rows once to global memory for the
+// backward pass; the dense transform never reads Cat back.  W streams through a TMA ring as in tc_gemm_tn_kernel, four
+// warps run the epilogue from two accumulators in tensor memory.  Rows are summed in the order of sage_aggregate_kernel
+// and rounded to bf16 at the same points, so Cat and h' have the bits of the two-kernel path.
+// LPR: lanes per gathered row = 2 d / 16 (d = 64, 128 or 256 values).
+constexpr int kFusedGatherWarps = 20;
+constexpr int kFusedEpiWarps = 4;
+constexpr int kFusedThreads = (2 + kFusedEpiWarps + kFusedGatherWarps) * 32;
+
+template <int LPR>
+__global__ void __launch_bounds__(kFusedThreads)
+tc_sage_fused_kernel(const __grid_constant__ CUtensorMap map_b, const __nv_bfloat16 *__restrict__ Hsrc, int64_t ld,
+                     const int32_t *__restrict__ nbr, const int32_t *__restrict__ self_ids, const int32_t *__restrict__ indptr,
+                     __nv_bfloat16 *__restrict__ cat, int nt, int stages, int a_bufs, uint32_t tmem_cols, TcEpilogue ep)
+{
+    constexpr int kKbHalf = LPR / 8;                 // k-blocks of 64 columns per half of Cat
+    constexpr int kKb = 2 * kKbHalf;
+    constexpr uint32_t kKbBytes = kTileM * 128;      // one k-block of the A tile: 128 rows x 128 bytes
+    constexpr int d = LPR * 8;
+    constexpr int G = 32 / LPR;
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ uint64_t b_full[kMaxStages], b_empty[kMaxStages], a_full[2], a_empty[2], acc_full[2], acc_empty[2];
+    __shared__ uint32_t tmem_base_slot;
+    __shared__ int abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+    uint8_t *a_tiles = tiles;
+    const uint32_t b_bytes = (uint32_t)nt * kTileK * 2;
+    uint8_t *b_tiles = tiles + (size_t)a_bufs * kKb * kKbBytes;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(&b_full[s], 1);
+            mbar_init(&b_empty[s], 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(&a_full[b], kFusedGatherWarps);
+            mbar_init(&a_empty[b], 1);
+            mbar_init(&acc_full[b], 1);
+            mbar_init(&acc_empty[b], kFusedEpiWarps);
+        }
+        abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_slot)),
+                     "r"(tmem_cols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = tmem_base_slot;
+    const uint32_t buf_stride = tmem_cols >> 1;
+    const int32_t n_dst = *ep.m_dev;
+    const int64_t live_tiles = ((int64_t)n_dst + kTileM - 1) / kTileM;
+
+    if ((int64_t)blockIdx.x >= live_tiles) {
+        // nothing for this CTA
+    } else if (warp == 0) {
+        if (lane == 0) {
+            // ---- W through the stage ring, k-block after k-block across tiles
+            uint32_t g = 0;
+            bool ok = true;
+            for (int64_t t = blockIdx.x; t < live_tiles && ok; t += gridDim.x) {
+                for (int kb = 0; kb < kKb; ++kb, ++g) {
+                    const uint32_t s = g % (uint32_t)stages, ph = (g / (uint32_t)stages) & 1u;
+                    ok = mbar_wait(&b_empty[s], ph ^ 1u, &abort_flag);
+                    if (!ok) break;
+                    mbar_expect_tx(&b_full[s], b_bytes);
+                    tma_load_2d(b_tiles + (size_t)s * b_bytes, &map_b, kb * kTileK, 0, &b_full[s]);
+                }
+            }
+            if (!ok) {
+                int never = 0;
+                for (uint32_t j = g > (uint32_t)stages ? g - stages : 0; j < g; ++j)
+                    mbar_wait(&b_full[j % stages], (j / stages) & 1u, &never);
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---- MMA issuer
+            const uint32_t idesc = make_idesc(kTileM, nt);
+            uint32_t g = 0, lt = 0;
+            bool ok = true;
+            for (int64_t t = blockIdx.x; t < live_tiles && ok; t += gridDim.x, ++lt) {
+                const uint32_t buf = lt & 1u;
+                const uint32_t ab = a_bufs == 2 ? (lt & 1u) : 0u, use = a_bufs == 2 ? (lt >> 1) : lt;
+                ok = mbar_wait(&acc_empty[buf], ((lt >> 1) & 1u) ^ 1u, &abort_flag) && mbar_wait(&a_full[ab], use & 1u, &abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + buf * buf_stride;
+                const uint32_t a_base = smem_u32(a_tiles + (size_t)ab * kKb * kKbBytes);
+                for (int kb = 0; kb < kKb; ++kb, ++g) {
+                    const uint32_t s = g % (uint32_t)stages, ph = (g / (uint32_t)stages) & 1u;
+                    ok = mbar_wait(&b_full[s], ph, &abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint32_t a_addr = a_base + kb * kKbBytes;
+                    const uint32_t b_addr = smem_u32(b_tiles + (size_t)s * b_bytes);
+#pragma unroll
+                    for (int k = 0; k < kTileK / kUmmaK; ++k)
+                        umma(d_tmem, make_smem_desc(a_addr + k * kUmmaK * 2), make_smem_desc(b_addr + k * kUmmaK * 2), idesc,
+                             (kb | k) != 0 ? 1u : 0u);
+                    umma_commit(&b_empty[s]);
+                }
+                if (ok) {
+                    umma_commit(&a_empty[ab]);      // the tile of Cat has been read: the gather warps may refill it
+                    umma_commit(&acc_full[buf]);
+                }
+            }
+        }
+    } else if (warp < 2 + kFusedEpiWarps) {
+        // ---- epilogue: warp w reads accumulator lanes 32 (w % 4) .. + 31, all column blocks
+        const int lg = warp & 3;
+        uint32_t lt = 0, n_box = 0;
+        for (int64_t t = blockIdx.x; t < live_tiles; t += gridDim.x, ++lt) {
+            const uint32_t buf = lt & 1u;
+            if (!mbar_wait(&acc_full[buf], (lt >> 1) & 1u, &abort_flag)) break;
+            tc_fence_after();
+            const int64_t row = t * kTileM + lg * 32 + lane;
+            EpiRow e;
+            e.ep = &ep;
+            e.map_out = nullptr;
+            e.orow = ep.out + row * ep.ldo;
+            e.orow2 = (ep.out2 && row < ep.rows2) ? ep.out2 + row * ep.ldo2 : nullptr;
+            e.mrow = nullptr;
+            e.out_stage = nullptr;
+            e.rs = 1.f;
+            e.floor_v = ep.relu ? 0.f : -INFINITY;
+            e.n0 = 0;
+            e.m0 = (int)(t * kTileM);
+            e.rt = lg * 32 + lane;
+            e.live = row < n_dst;
+            e.bias_vec = (reinterpret_cast<uintptr_t>(ep.bias) & 15) == 0;
+            e.store_lead = false;
+            const uint32_t taddr = tmem_base + buf * buf_stride + ((uint32_t)(lg * 32) << 16);
+            for (int c = 0; c < nt; c += 32) {
+                uint32_t r[32];
+                tmem_load32(taddr + (uint32_t)c, r);
+                if (c + 32 >= nt) {
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&acc_empty[buf]);
+                }
+                epi_finish_block<false, false>(e, r, c, n_box);
+            }
+        }
+    } else {
+        // ---- gather: warp gw builds rows gw, gw + kFusedGatherWarps, ... of every tile
+        const int gw = warp - (2 + kFusedEpiWarps);
+        const int g = lane / LPR, c = lane % LPR;
+        uint32_t lt = 0;
+        for (int64_t t = blockIdx.x; t < live_tiles; t += gridDim.x, ++lt) {
+            const uint32_t ab = a_bufs == 2 ? (lt & 1u) : 0u, use = a_bufs == 2 ? (lt >> 1) : lt;
+            if (!mbar_wait(&a_empty[ab], (use & 1u) ^ 1u, &abort_flag)) break;
+            uint8_t *A = a_tiles + (size_t)ab * kKb * kKbBytes;
+            // swizzled place of 16-byte chunk q (0 .. 2 LPR - 1) of row r of the tile
+            auto a_slot = [&](int r, int q) { return A + (q >> 3) * kKbBytes + r * 128 + (((q & 7) ^ (r & 7)) << 4); };
+            int32_t beg = 0, end = 0, mine = 0;
+            int64_t self_row = 0;
+            auto fetch = [&](int64_t ii, int32_t &b, int32_t &e, int32_t &m, int64_t &sr) {
+                b = e = m = 0;
+                sr = ii;
+                if (ii < n_dst) {
+                    b = indptr[ii];
+                    e = indptr[ii + 1];
+                    if (lane < e - b) m = nbr[b + lane];
+                    if (self_ids) sr = (int64_t)self_ids[ii];
+                }
+            };
+            fetch(t * kTileM + gw, beg, end, mine, self_row);
+            for (int r = gw; r < kTileM; r += kFusedGatherWarps) {
+                const int64_t i = t * kTileM + r;
+                int32_t beg_n = 0, end_n = 0, mine_n = 0;
+                int64_t self_n = 0;
+                if (r + kFusedGatherWarps < kTileM) fetch(i + kFusedGatherWarps, beg_n, end_n, mine_n, self_n);
+                __nv_bfloat16 *out = cat + i * 2 * d;
+                if (i >= n_dst) {
+                    // rows beyond the last destination: zeros (the weight gradient reads whole k-blocks of 64 rows of Cat)
+                    for (int q = lane; q < 2 * LPR; q += 32) {
+                        *reinterpret_cast<uint4 *>(out + q * 8) = make_uint4(0, 0, 0, 0);
+                        *reinterpret_cast<uint4 *>(a_slot(r, q)) = make_uint4(0, 0, 0, 0);
+                    }
+                } else {
+                    if (lane < LPR) {           // self half
+                        const uint4 v = __ldg(reinterpret_cast<const uint4 *>(Hsrc + self_row * ld + lane * 8));
+                        *reinterpret_cast<uint4 *>(out + lane * 8) = v;
+                        *reinterpret_cast<uint4 *>(a_slot(r, lane)) = v;
+                    }
+                    float acc[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) acc[k] = 0.f;
+                    for (int32_t base = beg; base < end; base += 32) {
+                        const int m = min(32, end - base);
+                        if (base != beg) mine = lane < m ? nbr[base + lane] : 0;
+                        for (int tt = 0; tt * G < m; tt += 4) {
+                            uint4 v[4];
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                const int j = (tt + u) * G + g;
+                                const int32_t id = __shfl_sync(0xffffffffu, mine, j & 31);
+                                v[u] = make_uint4(0, 0, 0, 0);
+                                if (j < m) v[u] = __ldg(reinterpret_cast<const uint4 *>(Hsrc + (int64_t)id * ld + c * 8));
+                            }
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                float x[8];
+                                Chunk<__nv_bfloat16>::unpack(v[u], x);
+#pragma unroll
+                                for (int k = 0; k < 8; k += 2) add2(acc[k], acc[k + 1], x[k], x[k + 1]);
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int off = LPR; off < 32; off <<= 1)
+#pragma unroll
+                        for (int k = 0; k < 8; ++k) acc[k] += __shfl_xor_sync(0xffffffffu, acc[k], off);
+                    if (g == 0) {
+                        const int32_t cnt = end - beg;
+                        const float inv = cnt > 0 ? 1.0f / (float)cnt : 0.0f;
+                        uint32_t w[4];
+#pragma unroll
+                        for (int k = 0; k < 4; ++k) {
+                            __nv_bfloat162 h = __floats2bfloat162_rn(acc[2 * k] * inv, acc[2 * k + 1] * inv);
+                            w[k] = *reinterpret_cast<uint32_t *>(&h);
+                        }
+                        const uint4 v = make_uint4(w[0], w[1], w[2], w[3]);
+                        *reinterpret_cast<uint4 *>(out + d + c * 8) = v;
+                        *reinterpret_cast<uint4 *>(a_slot(r, LPR + c)) = v;
+                    }
+                }
+                beg = beg_n;
+                end = end_n;
+                mine = mine_n;
+                self_row = self_n;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // the tensor cores read what this warp wrote
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&a_full[ab]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && abort_flag) atomicOr(reinterpret_cast<unsigned *>(ep.status), E2EGREC_DEV_TIMEOUT);
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+    }
+}
+
+template <int LPR>
+bool launch_fused(const CUtensorMap &mb, const __nv_bfloat16 *Hsrc, int64_t ld, const int32_t *nbr, const int32_t *self_ids,
+                  const int32_t *indptr, __nv_bfloat16 *cat, int64_t rows, int n, const TcEpilogue &ep, cudaStream_t st)
+{
+    constexpr int kKb = 2 * (LPR / 8);
+    const size_t a_bytes = (size_t)kKb * kTileM * 128, b_bytes = (size_t)n * kTileK * 2;
+    // two tiles of Cat where they fit beside at least two stages of W, else one
+    const int a_bufs = 2 * a_bytes + 2 * b_bytes + 1024 <= (size_t)kMaxDynSmem ? 2 : 1;
+    if (a_bufs * a_bytes + 2 * b_bytes + 1024 > (size_t)kMaxDynSmem) return false;
+    const int stages = (int)std::min<size_t>(kMaxStages, ((size_t)kMaxDynSmem - 1024 - a_bufs * a_bytes) / b_bytes);
+    const size_t smem = a_bufs * a_bytes + (size_t)stages * b_bytes + 1024;
+    static bool attr_set[kMaxDevices] = {};
+    if (!raise_smem_limit(tc_sage_fused_kernel<LPR>, attr_set)) return false;
+    uint32_t tmem_cols = 64;
+    while ((int)tmem_cols < 2 * n) tmem_cols <<= 1;
+    const unsigned grid = (unsigned)std::min<int64_t>(rows / kTileM, sm_count());
+    note_launch();
+    tc_sage_fused_kernel<LPR><<<grid, kFusedThreads, smem, st>>>(mb, Hsrc, ld, nbr, self_ids, indptr, cat, n, stages, a_bufs,
+                                                                 tmem_cols, ep);
+    return true;
+}
+
 }  // namespace
 
 bool tc_update_forward(const __nv_bfloat16 *cat, int64_t rows, int k, const __nv_bfloat16 *W, int n, const float *bias,
@@ -990,5 +1269,39 @@ bool tc_weight_grad(const __nv_bfloat16 *dY, int64_t rows, int m, const __nv_bfl
                (int64_t)m * n, status, n_rhs, rows);
     return true;
 }
+
+bool tc_sage_fused_forward(const __nv_bfloat16 *Hsrc, int64_t ld, const int32_t *nbr, const int32_t *self_ids,
+                           const int32_t *indptr, int d_in, __nv_bfloat16 *cat, int64_t rows, const __nv_bfloat16 *W, int n,
+                           const float *bias, int relu, __nv_bfloat16 *out, const int32_t *m_dev, int32_t *status,
+                           cudaStream_t st, __nv_bfloat16 *out2, int64_t ldo2, int64_t rows2)
+{
+    if (rows <= 0 || rows % kTileM || n < 32 || n > 256 || n % 32) return false;
+    if (d_in != 64 && d_in != 128 && d_in != 256) return false;
+    if (reinterpret_cast<uintptr_t>(Hsrc) % 16 || (ld * 2) % 16 || reinterpret_cast<uintptr_t>(cat) % 16 ||
+        reinterpret_cast<uintptr_t>(W) % 16 || reinterpret_cast<uintptr_t>(out) % 16)
+        return false;
+    if (out2 && (reinterpret_cast<uintptr_t>(out2) % 16 || (ldo2 * 2) % 16 || ldo2 < n)) return false;
+    TcEpilogue ep{};
+    ep.out = out;
+    ep.ldo = n;
+    ep.out2 = out2;
+    ep.ldo2 = ldo2;
+    ep.rows2 = rows2;
+    ep.bias = bias;
+    ep.relu = relu;
+    ep.m_dev = m_dev;
+    ep.status = status;
+    ep.n_rhs = 1;
+    ep.rhs_rows = rows;
+    ep.mode = (bias ? kEpiBias : 0) | (relu ? kEpiRelu : 0);
+    CUtensorMap mb;
+    if (!make_map(&mb, W, n, 2 * d_in, 2 * d_in, n)) return false;
+    switch (d_in) {
+    case 64: return launch_fused<8>(mb, Hsrc, ld, nbr, self_ids, indptr, cat, rows, n, ep, st);
+    case 128: return launch_fused<16>(mb, Hsrc, ld, nbr, self_ids, indptr, cat, rows, n, ep, st);
+    default: return launch_fused<32>(mb, Hsrc, ld, nbr, self_ids, indptr, cat, rows, n, ep, st);
+    }
+}
+
 
 }  // namespace e2egrec

@@ -14,6 +14,16 @@ bool tc_update_forward(const __nv_bfloat16 *cat, int64_t rows, int k, const __nv
                        int relu, __nv_bfloat16 *out, const int32_t *m_dev, int32_t *status, cudaStream_t st,
                        __nv_bfloat16 *out2 = nullptr, int64_t ldo2 = 0, int64_t rows2 = 0);
 
+// Eq. 2 and Eq. 3 of one layer in one launch (bf16, d_in of 64, 128 or 256 values, n <= 256 a multiple of 32):
+//   cat[i] = [ Hsrc[self_ids ? self_ids[i] : i] | mean over k in [indptr[i], indptr[i+1]) of Hsrc[nbr[k]] ]   (stored for the
+//   backward pass, zero rows from *m_dev up to the next multiple of 128),   out = act(cat W^T + bias)
+// with the rows of cat built in shared memory as the A operand, never read back from global memory.  Same conventions and
+// the same bits as sage_aggregate_kernel followed by tc_update_forward.
+bool tc_sage_fused_forward(const __nv_bfloat16 *Hsrc, int64_t ld, const int32_t *nbr, const int32_t *self_ids,
+                           const int32_t *indptr, int d_in, __nv_bfloat16 *cat, int64_t rows, const __nv_bfloat16 *W, int n,
+                           const float *bias, int relu, __nv_bfloat16 *out, const int32_t *m_dev, int32_t *status,
+                           cudaStream_t st, __nv_bfloat16 *out2 = nullptr, int64_t ldo2 = 0, int64_t rows2 = 0);
+
 // dCat = dZ W with the layer weight W [d_out x 2 d_in] as stored (the tensor cores read it with its N index
 // contiguous, no transposed copy is made); columns >= d_in are scaled by inv_cnt[row].  2 d_in must be a multiple
 // of 64.  Same conventions as above.

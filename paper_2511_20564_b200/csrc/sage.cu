@@ -107,6 +107,15 @@ static size_t dw_serial_bytes()
     return v;
 }
 
+// E2EGREC_FUSED_FORWARD=1: bf16 layers whose shapes allow it run Eq. 2 and Eq. 3 as one kernel (the aggregated rows are
+// built in shared memory as the A operand of the dense transform).  Off by default: measured slower than the two
+// kernels on every workload of the benchmark.
+static bool fused_forward_enabled()
+{
+    static const bool on = []() { const char *e = getenv("E2EGREC_FUSED_FORWARD"); return e && *e && e[0] != '0'; }();
+    return on;
+}
+
 // ------------------------------------------------------------------------------ forward
 template <typename T>
 static int32_t forward_impl(const e2egrec_block *blocks, int32_t n_layers, const e2egrec_mat *X, const e2egrec_mat *W,
@@ -121,6 +130,23 @@ static int32_t forward_impl(const e2egrec_block *blocks, int32_t n_layers, const
         const e2egrec_block &b = blocks[p.block];
         T *cat = reinterpret_cast<T *>(ctx + p.cat_off);
         T *hn = reinterpret_cast<T *>(ctx + p.h_off);
+        if (X->dtype == E2EGREC_BF16 && fused_forward_enabled()) {
+            const bool top = l == n_layers - 1;
+            const __nv_bfloat16 *src = l == 0 ? static_cast<const __nv_bfloat16 *>(X->data)
+                                              : reinterpret_cast<const __nv_bfloat16 *>(ctx + plan[l - 1].h_off);
+            if (l == 0) tap_begin(TAP_AGG_FWD_OUTER, st);
+            const bool fused = tc_sage_fused_forward(
+                src, l == 0 ? X->ld : p.d_in, l == 0 ? b.nbr_global : b.col, l == 0 ? b.src_nodes : nullptr, b.indptr, p.d_in,
+                reinterpret_cast<__nv_bfloat16 *>(cat), p.rows, static_cast<const __nv_bfloat16 *>(W[l].data), p.d_out,
+                bias ? bias[l] : nullptr, act ? act[l] : 1, reinterpret_cast<__nv_bfloat16 *>(hn), &b.counts[CNT_DST],
+                &b.counts[CNT_STATUS], st, top ? static_cast<__nv_bfloat16 *>(H_out->data) : nullptr, H_out->ld, out_rows);
+            if (l == 0) tap_end(TAP_AGG_FWD_OUTER, st);
+            if (fused) {
+                if (l == 0) { tap_begin(TAP_UPDATE_FWD_OUTER, st); tap_end(TAP_UPDATE_FWD_OUTER, st); }
+                top_stored = top_stored || top;
+                continue;
+            }
+        }
         bool agg_ok;
         if (l == 0) {  // h^(0) rows are read straight from the feature table through the global ids
             tap_begin(TAP_AGG_FWD_OUTER, st);
