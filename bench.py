@@ -38,13 +38,13 @@ CLOCK_QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reason
                "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
                "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 TAP_NAMES = {1: "sage_aggregate_kernel (layer-0 mean aggregation, gathers X rows)",
-             2: "seg_run_kernel+seg_final_kernel (layer-0 transposed aggregation -> dX rows)",
+             2: "seg_run_block_kernel (layer-0 transposed aggregation -> dX rows)",
              3: "layer-0 dense transform W[h|agg]",
              4: "layer-0 weight gradient dZ^T[h|agg]",
              5: "layer-0 input gradient dZ W",
              6: "e2egrec_sample_khop (all sampling kernels)",
-             7: "seg_run_kernel (first transposed aggregation of the backward pass)",
-             9: "seg_final_kernel (same)"}
+             7: "seg_run_block_kernel, top layer (first transposed aggregation of the backward pass)",
+             9: "seg_final_kernel (same; empty interval where the one-launch form runs)"}
 # source files whose kernels a recorded DRAM-traffic figure belongs to (the figure is dropped when they change)
 TRAFFIC_SOURCES = ("aggregate.cuh", "segreduce.cuh", "common.cuh")
 
@@ -700,7 +700,7 @@ def run_ours(args, w, with_joint):
         "outer_block": dict(n_dst=n_dst, n_src=n_src, n_edges=n_edges, row_bytes=r),
         "forward": dict(kernel="sage_aggregate_kernel", ms=tap_ms[1], algorithmic_bytes=alg_fwd,
                         **hbm_fractions(alg_fwd / tap_ms[1] / 1e6, peaks)),
-        "backward": dict(kernel="seg_run_kernel+seg_final_kernel", ms=tap_ms[2], algorithmic_bytes=alg_bwd,
+        "backward": dict(kernel="seg_run_block_kernel", ms=tap_ms[2], algorithmic_bytes=alg_bwd,
                          **hbm_fractions(alg_bwd / tap_ms[2] / 1e6, peaks))}
     # DRAM bytes per launch: a recorded ncu capture of the same kernel (bytes per entry of the outermost block, taken on
     # this workload or on its reduced-size stand-in) times the entries of one launch here; null without a fresh record
