@@ -1246,13 +1246,25 @@ bool tc_dcat_backward(const __nv_bfloat16 *dz, int64_t rows, int d_out, const __
 
 namespace e2egrec {
 
+// widest tile of 64 .. 256 columns that divides n (0: none)
+static int weight_grad_nt(int n)
+{
+    for (int c = 256; c >= 64; c -= 64)
+        if (n % c == 0) return c;
+    return 0;
+}
+
+int tc_weight_grad_tiles(int m, int n)
+{
+    const int nt = weight_grad_nt(n);
+    return nt && m >= kTileM ? (m / kTileM) * (n / nt) : 1;
+}
+
 bool tc_weight_grad(const __nv_bfloat16 *dY, int64_t rows, int m, const __nv_bfloat16 *Xin, int n, const int32_t *m_dev,
                     float *part, int splits, int32_t *status, cudaStream_t st, int n_rhs)
 {
-    if (rows <= 0 || rows % kTileK || m % kTileM || n % 64 || n_rhs < 1) return false;
-    int nt = 0;
-    for (int c = 256; c >= 64; c -= 64)
-        if (n % c == 0) { nt = c; break; }
+    if (rows <= 0 || rows % kTileK || m % kTileM || n % 64 || n_rhs < 1 || splits < 1) return false;
+    const int nt = weight_grad_nt(n);
     if (!nt) return false;
     if (reinterpret_cast<uintptr_t>(dY) % 16 || reinterpret_cast<uintptr_t>(Xin) % 16) return false;
     CUtensorMap my, mx;

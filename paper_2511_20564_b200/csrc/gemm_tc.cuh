@@ -58,5 +58,7 @@ bool tc_linear(const __nv_bfloat16 *A, int64_t rows, int k, const __nv_bfloat16 
 // n_rhs > 1: dY holds n_rhs blocks of `rows` rows that all meet the same `rows` rows of Xin; the result is the sum over them.
 bool tc_weight_grad(const __nv_bfloat16 *dY, int64_t rows, int m, const __nv_bfloat16 *Xin, int n, const int32_t *m_dev,
                     float *part, int splits, int32_t *status, cudaStream_t st, int n_rhs = 1);
+// Output tiles (128 x up to 256) of tc_weight_grad for an m x n result: gridDim.x * gridDim.y of its launch.
+int tc_weight_grad_tiles(int m, int n);
 
 }  // namespace e2egrec
