@@ -37,7 +37,7 @@ MIN_TIMED_S = 0.5                   # the K-step loop is repeated until the time
 CLOCK_QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
                "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
                "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
-TAP_NAMES = {1: "sage_aggregate_kernel (layer-0 mean aggregation, gathers X rows)",
+TAP_NAMES = {1: "layer-0 mean aggregation (sage_aggregate_kernel; sage_aggregate_stream_kernel where the block holds 2^21 entries or more)",
              2: "seg_run_block_kernel (layer-0 transposed aggregation -> dX rows)",
              3: "layer-0 dense transform W[h|agg]",
              4: "layer-0 weight gradient dZ^T[h|agg]",
@@ -46,7 +46,7 @@ TAP_NAMES = {1: "sage_aggregate_kernel (layer-0 mean aggregation, gathers X rows
              7: "seg_run_block_kernel, top layer (first transposed aggregation of the backward pass)",
              9: "seg_final_kernel (same; empty interval where the one-launch form runs)"}
 # source files whose kernels a recorded DRAM-traffic figure belongs to (the figure is dropped when they change)
-TRAFFIC_SOURCES = ("aggregate.cuh", "segreduce.cuh", "common.cuh")
+TRAFFIC_SOURCES = ("aggregate.cuh", "segreduce.cuh", "common.cuh", "gather_stream.cu")
 
 
 def measured_peaks():
@@ -681,6 +681,7 @@ def run_ours(args, w, with_joint):
     es = 2 if w.dtype == "bf16" else 4
     r = w.dim * es
     n_dst, n_src, n_edges = float(outer_counts[0]), float(outer_counts[1]), float(outer_counts[2])
+    outer_cap_edges = int(blocks.caps[L - 1][2])
     dom_mean_ms = float(np.mean(dom_ms))
     # both aggregation kernels of the outermost block, whichever kernel dominates.  forward, per entry: id + gathered
     # row; per destination: offsets, self id, self row, [self|mean] row out.  backward, per entry: row id + gathered
@@ -698,7 +699,8 @@ def run_ours(args, w, with_joint):
                     unit="TFLOP/s")
     aggregation = {
         "outer_block": dict(n_dst=n_dst, n_src=n_src, n_edges=n_edges, row_bytes=r),
-        "forward": dict(kernel="sage_aggregate_kernel", ms=tap_ms[1], algorithmic_bytes=alg_fwd,
+        "forward": dict(kernel="sage_aggregate_stream_kernel" if w.dim == 256 and w.dtype == "bf16" and outer_cap_edges >= (1 << 21)
+                        else "sage_aggregate_kernel", ms=tap_ms[1], algorithmic_bytes=alg_fwd,
                         **hbm_fractions(alg_fwd / tap_ms[1] / 1e6, peaks)),
         "backward": dict(kernel="seg_run_block_kernel", ms=tap_ms[2], algorithmic_bytes=alg_bwd,
                          **hbm_fractions(alg_bwd / tap_ms[2] / 1e6, peaks))}

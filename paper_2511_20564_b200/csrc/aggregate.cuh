@@ -152,6 +152,11 @@ struct SegOut {
     // in + r * rhs_in and self + r * rhs_self and writes out + r * rhs_out (element strides); the mask is shared.
     int n_rhs;              // 0 or 1: one
     int64_t rhs_in, rhs_self, rhs_out;
+    // For the form that streams the gathered rows through shared memory (seg_run_block_kernel<..., kStream>): the rows
+    // that `in` holds over all right-hand sides (0: unknown, the form is not used) and the device status word that
+    // receives E2EGREC_DEV_TIMEOUT when a bounded wait for the rows runs out.
+    int64_t in_rows;
+    int32_t *status;
 };
 
 template <typename T>

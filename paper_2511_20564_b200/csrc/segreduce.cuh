@@ -23,7 +23,10 @@
 
 #include <algorithm>
 
+#include <type_traits>
+
 #include "aggregate.cuh"
+#include "tensor_map.cuh"
 
 namespace e2egrec {
 
@@ -533,9 +536,18 @@ seg_run_kernel(const T *__restrict__ in, int64_t ld_in, const PtrT *__restrict__
 // for this case alone (entry ids and segment ids fetched four at a time, 32-bit arithmetic, no scale, no walk of the
 // offsets), which takes the instructions per entry from ~110 to ~35: with two entries per segment on average the
 // general kernel was bound by instruction issue, not by memory.
-template <typename T, int LPR, bool kMask, int U = 4, int kMinBlocks = (kMask ? 3 : 4)>
+//
+// kStream (bf16 rows of 512 bytes, one warp per run): the gathered rows do not pass through registers on their way in.
+// Every warp hands the entry ids of its run, four at a time, to the TMA unit (tile::gather4 on `in_map`, the table `in`
+// as a 2-D tensor), which lands the rows in the warp's own ring of kStreamSlots slots in shared memory; the warp adds
+// them up from there in the same order.  Twice the rows in flight per warp at the same register count; the self and
+// mask rows of beginning segments are still loaded directly.
+constexpr int kStreamSlots = 2;
+constexpr uint32_t kStreamRowBytes = 512;
+
+template <typename T, int LPR, bool kMask, int U = 4, int kMinBlocks = (kMask ? 3 : 4), bool kStream = false>
 __global__ void __launch_bounds__(kAggThreads, kMinBlocks)
-seg_run_block_kernel(const T *__restrict__ in, int64_t ld_in, const int32_t *__restrict__ ptr, const int32_t *__restrict__ idx,
+seg_run_block_kernel(const __grid_constant__ CUtensorMap in_map, const T *__restrict__ in, int64_t ld_in, const int32_t *__restrict__ ptr, const int32_t *__restrict__ idx,
                      const int32_t *__restrict__ seg_of, const int32_t *__restrict__ n_seg_dev, int run_len, int d,
                      float *__restrict__ head2, float *__restrict__ tail2, int4 *__restrict__ win_info, int64_t cap_runs,
                      int32_t *__restrict__ chain_cnt, SegOut<T> o)
@@ -549,15 +561,30 @@ seg_run_block_kernel(const T *__restrict__ in, int64_t ld_in, const int32_t *__r
     float *sh_tail = sh_head + RB * ROW;
     int4 *sh_info = reinterpret_cast<int4 *>(sh_tail + RB * ROW);
     __shared__ int32_t sh_win[4];
+    __shared__ uint64_t sh_bar[kStream ? RB : 1][kStreamSlots];
 
     const int c = threadIdx.x % LPR;
     const int rl = threadIdx.x / LPR;
     const int n_chunks = d / E;
     const int64_t run = (int64_t)blockIdx.x * RB + rl;
+    // kStream: the warp's ring behind the join's rows and records, its barriers, the row offset of its right-hand side
+    uint8_t *ring_w = nullptr;
+    int32_t row_off = 0;
+    if constexpr (kStream) {
+        ring_w = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(sh_info + RB) + 127) & ~uintptr_t(127)) +
+                 (size_t)rl * kStreamSlots * 4 * kStreamRowBytes;
+        if (c == 0) {
+            for (int s = 0; s < kStreamSlots; ++s) tm_mbar_init(&sh_bar[rl][s], 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+        __syncwarp();
+    }
     pdl_launch_dependents();
     pdl_wait();                                    // the kernel before this one in the stream has completed
     if (blockIdx.y) {                              // the second right-hand side: other rows, same segments
         const int64_t r = blockIdx.y, nw = gridDim.x;
+        if constexpr (kStream) row_off = (int32_t)(r * (o.rhs_in / ld_in));
         in += r * o.rhs_in;
         o.self += r * o.rhs_self;
         o.out += r * o.rhs_out;
@@ -606,6 +633,99 @@ seg_run_block_kernel(const T *__restrict__ in, int64_t ld_in, const int32_t *__r
             }
         };
 
+        // kStream: the ids of group g (entries 4g .. 4g + 3 of the run; beyond the run's end the first id again), and the
+        // hand-over of a group to the TMA unit by the warp's first lane
+        bool stream_ok = true;
+        auto group_ids = [&](int g) -> int4 {
+            const int r = 4 * g;
+            if (vec_ok && r + 4 <= len) return __ldg(reinterpret_cast<const int4 *>(idx0 + r));
+            const int32_t first = __ldg(idx0 + (r < len ? r : 0));
+            return make_int4(first, r + 1 < len ? __ldg(idx0 + r + 1) : first, r + 2 < len ? __ldg(idx0 + r + 2) : first,
+                             r + 3 < len ? __ldg(idx0 + r + 3) : first);
+        };
+        auto issue_group = [&](int g, const int4 &ids) {
+            if (c == 0)
+                tm_gather4(ring_w + (size_t)(g % kStreamSlots) * 4 * kStreamRowBytes, &in_map, ids.x + row_off, ids.y + row_off,
+                           ids.z + row_off, ids.w + row_off, &sh_bar[rl][g % kStreamSlots], kStreamRowBytes);
+        };
+        int n_issued = 0;
+        if constexpr (kStream) {
+            // Three things are in flight per warp: the rows of the next kStreamSlots groups (ring), the self / mask rows of
+            // the next group's beginning segments (registers, fetched one group ahead), the segment ids two groups ahead.
+            static_assert(!kStream || U == 4, "a group of the ring is four entries");
+            const int n_g = (len + 3) >> 2;
+            auto load_sg = [&](int g) -> int4 {
+                const int r = 4 * g;
+                if (vec_ok && r + 4 <= len) return __ldg(reinterpret_cast<const int4 *>(seg0 + r));
+                return make_int4(r < len ? __ldg(seg0 + r) : -1, r + 1 < len ? __ldg(seg0 + r + 1) : -1,
+                                 r + 2 < len ? __ldg(seg0 + r + 2) : -1, r + 3 < len ? __ldg(seg0 + r + 3) : -1);
+            };
+            // the entries of group g that begin a segment (bit u) and the self / mask rows of those segments
+            auto load_starts = [&](int g, const int4 &sgv, int32_t prev_last, uint4 (&svv)[4], uint4 (&mvv)[kMask ? 4 : 1]) -> unsigned {
+                const int32_t sgs[4] = {sgv.x, sgv.y, sgv.z, sgv.w};
+                unsigned starts = 0;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int r = 4 * g + u;
+                    const bool st = r < len && sgs[u] != (u == 0 ? prev_last : sgs[u - 1]);
+                    svv[u] = make_uint4(0, 0, 0, 0);
+                    if (kMask) mvv[u] = make_uint4(0, 0, 0, 0);
+                    if (st) {
+                        starts |= 1u << u;
+                        if (lane_on) {
+                            if ((r != 0 || first_begins) && sgs[u] < n_self) svv[u] = Chunk<T>::load_raw(self_c + (int64_t)sgs[u] * o.ld_self);
+                            if (kMask) mvv[u] = Chunk<T>::load_raw(mask_c + (int64_t)sgs[u] * o.ld_mask);
+                        }
+                    }
+                }
+                return starts;
+            };
+            for (int g = 0; g < kStreamSlots && g < n_g; ++g, ++n_issued) issue_group(g, group_ids(g));
+            int4 ids_ahead = kStreamSlots < n_g ? group_ids(kStreamSlots) : make_int4(0, 0, 0, 0);
+            int4 sg_cur = load_sg(0);
+            int4 sg_next = n_g > 1 ? load_sg(1) : make_int4(-1, -1, -1, -1);
+            uint4 sv_cur[4], sv_next[4], mv_cur[kMask ? 4 : 1], mv_next[kMask ? 4 : 1];
+            unsigned starts_cur = load_starts(0, sg_cur, -1, sv_cur, mv_cur), starts_next = 0;
+            for (int g = 0; g < n_g; ++g) {
+                if (g + 1 < n_g) starts_next = load_starts(g + 1, sg_next, sg_cur.w, sv_next, mv_next);
+                const int4 sg_after = g + 2 < n_g ? load_sg(g + 2) : make_int4(-1, -1, -1, -1);
+                const int slot = g % kStreamSlots;
+                stream_ok = stream_ok && __all_sync(0xffffffffu, tm_mbar_wait(&sh_bar[rl][slot], (uint32_t)(g / kStreamSlots) & 1u));
+                const uint8_t *rows = ring_w + (size_t)slot * 4 * kStreamRowBytes + c * 16;
+                const int32_t sgs[4] = {sg_cur.x, sg_cur.y, sg_cur.z, sg_cur.w};
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int r = 4 * g + u;
+                    if (r < len) {
+                        if ((starts_cur >> u) & 1u) {
+                            if (cur_seg >= 0) emit(true);
+                            cur_seg = sgs[u];
+                            cur_begins = r != 0 || first_begins;
+                            Chunk<T>::unpack(sv_cur[u], acc[0]);             // the self row (zeros if there is none)
+                            if (kMask) cur_mask[0] = mv_cur[u];
+                        }
+                        float x[E];
+                        Chunk<T>::unpack(stream_ok ? *reinterpret_cast<const uint4 *>(rows + u * kStreamRowBytes) : make_uint4(0, 0, 0, 0), x);
+#pragma unroll
+                        for (int e = 0; e < E; e += 2) add2(acc[0][e], acc[0][e + 1], x[e], x[e + 1]);
+                    }
+                }
+                __syncwarp();                                   // every lane has read the slot
+                if (stream_ok && g + kStreamSlots < n_g) {
+                    issue_group(g + kStreamSlots, ids_ahead);
+                    n_issued = g + kStreamSlots + 1;
+                    if (g + kStreamSlots + 1 < n_g) ids_ahead = group_ids(g + kStreamSlots + 1);
+                }
+                sg_cur = sg_next;
+                sg_next = sg_after;
+                starts_cur = starts_next;
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    sv_cur[u] = sv_next[u];
+                    if (kMask) mv_cur[u] = mv_next[u];
+                }
+            }
+        } else
         for (int r0 = 0; r0 < len; r0 += U) {
             int32_t id[U], sg[U];
             if (vec_ok && r0 + U <= len) {
@@ -660,6 +780,14 @@ seg_run_block_kernel(const T *__restrict__ in, int64_t ld_in, const int32_t *__r
             }
         }
         emit(last_ends);
+        if constexpr (kStream) {
+            if (!stream_ok) {
+                // a wait for rows ran out: report it and let the copies that were started land before the block leaves
+                if (c == 0 && o.status) atomicOr(reinterpret_cast<unsigned *>(o.status), E2EGREC_DEV_TIMEOUT);
+                for (int g = max(0, n_issued - kStreamSlots); g < n_issued; ++g)
+                    tm_mbar_wait(&sh_bar[rl][g % kStreamSlots], (uint32_t)(g / kStreamSlots) & 1u);
+            }
+        }
     }
     if (live_window)
         seg_join_window<T, int32_t, LPR, 1, kExtra>(sh_head, sh_tail, sh_info, sh_win, rl, c, n_chunks, d, head_seg, head_ends,
@@ -876,6 +1004,16 @@ inline bool seg_general_only()
     return v;
 }
 
+// E2EGREC_NO_STREAM_GATHER=1: no kernel streams its gathered rows through shared memory.
+inline bool seg_stream_off()
+{
+    static const bool v = []() {
+        const char *e = getenv("E2EGREC_NO_STREAM_GATHER");
+        return e && *e && e[0] != '0';
+    }();
+    return v;
+}
+
 template <typename T, typename PtrT, int LPR, int CPL, bool kWeight, int kInFlight>
 inline void launch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const int32_t *idx, const int32_t *n_seg_dev,
                               int64_t n_seg_host, int64_t cap_seg, const float *w, int run_len, int d,
@@ -910,11 +1048,39 @@ inline void launch_seg_reduce(const T *in, int64_t ld_in, const PtrT *ptr, const
         if (block_form) {
             block_form = true;
             const dim3 grid_b(grid1, (unsigned)(o.n_rhs > 1 && sc.chain_cnt ? o.n_rhs : 1));
-            if (o.mask)
-                launch_pdl(seg_run_block_kernel<T, LPR, true>, grid_b, dim3(kAggThreads), smem, st, in, ld_in, ptr, idx, seg_of,
+            CUtensorMap in_map{};
+            bool streamed = false;
+            if constexpr (std::is_same<T, __nv_bfloat16>::value && LPR == 32) {
+                // 512-byte rows in long runs: the rows come in through the TMA unit and a ring in shared memory
+                if (d == 256 && run_len >= 64 && o.in_rows > 0 && !seg_stream_off() && make_row_gather_map(&in_map, in, o.in_rows, d, ld_in)) {
+                    constexpr size_t smem_s = smem + 128 + (size_t)(kAggThreads / LPR) * kStreamSlots * 4 * kStreamRowBytes;
+                    static bool attr_set[2][64] = {};
+                    int dev = 0;
+                    cudaGetDevice(&dev);
+                    const int mk = o.mask ? 1 : 0;
+                    if (dev >= 0 && dev < 64 && !attr_set[mk][dev]) {
+                        const cudaError_t e =
+                            mk ? cudaFuncSetAttribute(seg_run_block_kernel<T, LPR, true, 4, 3, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_s)
+                               : cudaFuncSetAttribute(seg_run_block_kernel<T, LPR, false, 4, 4, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_s);
+                        attr_set[mk][dev] = e == cudaSuccess;
+                    }
+                    if (dev >= 0 && dev < 64 && attr_set[mk][dev]) {
+                        streamed = true;
+                        if (o.mask)
+                            launch_pdl(seg_run_block_kernel<T, LPR, true, 4, 3, true>, grid_b, dim3(kAggThreads), smem_s, st, in_map, in, ld_in, ptr,
+                                       idx, seg_of, n_seg_dev, run_len, d, sc.head2, sc.tail2, sc.win_info, sc.cap_runs, sc.chain_cnt, o);
+                        else
+                            launch_pdl(seg_run_block_kernel<T, LPR, false, 4, 4, true>, grid_b, dim3(kAggThreads), smem_s, st, in_map, in, ld_in, ptr,
+                                       idx, seg_of, n_seg_dev, run_len, d, sc.head2, sc.tail2, sc.win_info, sc.cap_runs, sc.chain_cnt, o);
+                    }
+                }
+            }
+            if (streamed) {
+            } else if (o.mask)
+                launch_pdl(seg_run_block_kernel<T, LPR, true>, grid_b, dim3(kAggThreads), smem, st, in_map, in, ld_in, ptr, idx, seg_of,
                            n_seg_dev, run_len, d, sc.head2, sc.tail2, sc.win_info, sc.cap_runs, sc.chain_cnt, o);
             else
-                launch_pdl(seg_run_block_kernel<T, LPR, false>, grid_b, dim3(kAggThreads), smem, st, in, ld_in, ptr, idx, seg_of,
+                launch_pdl(seg_run_block_kernel<T, LPR, false>, grid_b, dim3(kAggThreads), smem, st, in_map, in, ld_in, ptr, idx, seg_of,
                            n_seg_dev, run_len, d, sc.head2, sc.tail2, sc.win_info, sc.cap_runs, sc.chain_cnt, o);
             if (sc.chain_cnt) {                   // chains, empty segments and padding were all done in that launch
                 tap_end(TAP_SEG_L1, st);

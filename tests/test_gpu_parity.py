@@ -59,6 +59,21 @@ def test_blocks_with_capacity_for_millions_of_entries():
     _check_float(case, gpu, ora)
 
 
+def test_wide_rows_with_capacity_for_millions_of_entries():
+    """256-value bf16 rows in block buffers sized for 40 000 seeds on the 500 k-node graph (outer block: 5 M entries of
+    capacity): the launch
+    shapes of the largest workload, where the aggregation streams its rows through shared memory with the TMA unit."""
+    import dataclasses
+    w = dataclasses.replace(S.WORKLOADS["medium"], dim=256, hidden=256, batch=512)
+    case = Case(w, step=2)
+    dH = case.upstream_grad(case.seeds.size, w.hidden)
+    ora = case.run_oracle(dH)
+    gpu = case.run_gpu(dH, cap_seeds=40000)
+    assert gpu["blocks_obj"].caps[-1][2] >= 1 << 21
+    assert_blocks_equal(gpu["blocks"], ora["blocks"])
+    _check_float(case, gpu, ora)
+
+
 def test_medium_small_bf16_linear_backward_is_strict():
     """Identity activations: no sign decisions, so every gradient element is held to the plain tolerance."""
     case = Case(S.WORKLOADS["medium_small"], step=5, acts=[0, 0])
