@@ -37,7 +37,7 @@ MIN_TIMED_S = 0.5                   # the K-step loop is repeated until the time
 CLOCK_QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
                "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
                "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
-TAP_NAMES = {1: "layer-0 mean aggregation (sage_aggregate_kernel; sage_aggregate_stream_kernel where the block holds 2^21 entries or more)",
+TAP_NAMES = {1: "layer-0 mean aggregation (sage_aggregate_kernel; sage_aggregate_stream_kernel where the block can hold 2^20 entries or more)",
              2: "seg_run_block_kernel (layer-0 transposed aggregation -> dX rows)",
              3: "layer-0 dense transform W[h|agg]",
              4: "layer-0 weight gradient dZ^T[h|agg]",
@@ -699,7 +699,7 @@ def run_ours(args, w, with_joint):
                     unit="TFLOP/s")
     aggregation = {
         "outer_block": dict(n_dst=n_dst, n_src=n_src, n_edges=n_edges, row_bytes=r),
-        "forward": dict(kernel="sage_aggregate_stream_kernel" if w.dim == 256 and w.dtype == "bf16" and outer_cap_edges >= (1 << 21)
+        "forward": dict(kernel="sage_aggregate_stream_kernel" if w.dim == 256 and w.dtype == "bf16" and outer_cap_edges >= (1 << 20)
                         else "sage_aggregate_kernel", ms=tap_ms[1], algorithmic_bytes=alg_fwd,
                         **hbm_fractions(alg_fwd / tap_ms[1] / 1e6, peaks)),
         "backward": dict(kernel="seg_run_block_kernel", ms=tap_ms[2], algorithmic_bytes=alg_bwd,

@@ -88,9 +88,17 @@ static bool dispatch_sage_aggregate(const T *Hsrc, int64_t ld, const int32_t *nb
     return false;
 }
 
-// transposed-block entries per lane group: 32, or 128 where the block can hold millions of entries (the longer run's
+// transposed-block entries per lane group: 16, or 128 where the block can hold a million entries or more (the longer run's
 // lower overhead per entry wins there; measured on the 2 * 10^9-entry workload: 0.69 -> 0.63 ms)
-static inline int block_run_len(int64_t cap_edges) { return cap_edges >= (1ll << 21) ? 128 : 16; }
+// (longer runs were measured with the streamed rows as well: 256 entries 0.422 ms, 512 0.461, 1024 0.777 against 0.421)
+// A block that can hold two million entries gets runs of 128 entries.  Where the rows can be streamed through shared
+// memory (512-byte bf16 rows) the long runs and the streaming start at a million (2 * 10^9-entry workload: the outer
+// block alone 2.207 ms per step, the middle block as well 2.168; with 2^17 the top block joins and its 0.065 ms become
+// 0.127).  Capacities, not sizes, are what the host knows: a small batch in large buffers pays for the long runs (a
+// 71 k-entry block in a 1.2 M-entry buffer: 0.327 -> 0.362 ms per joint step), hence no lower than this.
+static inline bool streamable_rows(int d, size_t es) { return es == 2 && d == 256; }
+static inline int64_t big_block_edges(int d, size_t es) { return streamable_rows(d, es) ? (1ll << 20) : (1ll << 21); }
+static inline int block_run_len(int64_t cap_edges, int d, size_t es) { return cap_edges >= big_block_edges(d, es) ? 128 : 16; }
 constexpr int kDwSplits = 148;        // split-K factor of the weight-gradient product
 
 // A layer whose weight-gradient product may move this many bytes or more (by the capacity of its block) keeps that
@@ -117,7 +125,7 @@ static bool fused_forward_enabled()
     return on;
 }
 
-// bf16 layers with 256-value rows whose block can hold two million entries or more aggregate with the rows streamed
+// bf16 layers with 256-value rows whose block can hold a million entries or more aggregate with the rows streamed
 // through shared memory by the TMA unit (gather_stream.cu) instead of register-staged loads: 0.347 -> 0.240 ms on the
 // outer block of the 2 * 10^9-entry workload, same bits.  Smaller blocks are bound by launch and latency, where the
 // one-warp-per-destination kernel is faster.  E2EGREC_NO_STREAM_GATHER=1 switches it off.
@@ -160,7 +168,7 @@ static int32_t forward_impl(const e2egrec_block *blocks, int32_t n_layers, const
         }
         bool agg_ok = false;
         if (l == 0) tap_begin(TAP_AGG_FWD_OUTER, st);
-        if (X->dtype == E2EGREC_BF16 && p.d_in == 256 && b.cap_edges >= (1ll << 21) && stream_gather_enabled())
+        if (X->dtype == E2EGREC_BF16 && streamable_rows(p.d_in, sizeof(T)) && b.cap_edges >= big_block_edges(p.d_in, sizeof(T)) && stream_gather_enabled())
             agg_ok = stream_sage_aggregate(l == 0 ? static_cast<const __nv_bfloat16 *>(X->data)
                                                   : reinterpret_cast<const __nv_bfloat16 *>(ctx + plan[l - 1].h_off),
                                            l == 0 ? X->rows : plan[l - 1].rows, l == 0 ? X->ld : p.d_in,
@@ -225,8 +233,8 @@ static BackwardScratch plan_backward(const e2egrec_block *blocks, int32_t n_laye
         dcat = std::max(dcat, (size_t)n_rhs * p.rows * 2 * p.d_in * es);
         part = std::max(part, (size_t)kDwSplits * p.d_out * 2 * p.d_in * sizeof(float));
         wt = std::max(wt, (size_t)p.d_out * 2 * p.d_in * es);
-        ht = std::max(ht, seg_scratch_carve(blocks[p.block].cap_edges, block_run_len(blocks[p.block].cap_edges), p.d_in, es, nullptr, n_rhs).bytes);
-        chain = std::max(chain, seg_chain_bytes(blocks[p.block].cap_edges, block_run_len(blocks[p.block].cap_edges), p.d_in, es, n_rhs));
+        ht = std::max(ht, seg_scratch_carve(blocks[p.block].cap_edges, block_run_len(blocks[p.block].cap_edges, p.d_in, es), p.d_in, es, nullptr, n_rhs).bytes);
+        chain = std::max(chain, seg_chain_bytes(blocks[p.block].cap_edges, block_run_len(blocks[p.block].cap_edges, p.d_in, es), p.d_in, es, n_rhs));
     }
     size_t off = 0;
     auto take = [&](size_t b) { size_t o = off; off += align_up(b, 256); return o; };
@@ -378,10 +386,10 @@ static int32_t backward_impl(const e2egrec_block *blocks, int32_t n_layers, cons
             o.rhs_out = static_cast<T *>(dX_rows[n_rhs - 1].data) - static_cast<T *>(dX_rows[0].data);
         }
         if (l == 0) tap_begin(TAP_AGG_BWD_OUTER, st);
-        SegScratch sc = seg_scratch_carve(b.cap_edges, block_run_len(b.cap_edges), p.d_in, dtype_size(X->dtype), scratch + bs.seg_off, n_rhs);
+        SegScratch sc = seg_scratch_carve(b.cap_edges, block_run_len(b.cap_edges, p.d_in, dtype_size(X->dtype)), p.d_in, dtype_size(X->dtype), scratch + bs.seg_off, n_rhs);
         sc.chain_cnt = reinterpret_cast<int32_t *>(scratch + bs.chain_off);
         const bool seg_ok = dispatch_seg_reduce<T, int32_t, false>(dcat + p.d_in, two_d, b.csc_ptr, b.csc_row, &b.counts[CNT_SRC], 0,
-                                                                   b.cap_src, nullptr, block_run_len(b.cap_edges), p.d_in, X->dtype,
+                                                                   b.cap_src, nullptr, block_run_len(b.cap_edges, p.d_in, dtype_size(X->dtype)), p.d_in, X->dtype,
                                                                    b.csc_col, sc, o, st);
         if (l == 0) tap_end(TAP_AGG_BWD_OUTER, st);
         if (!seg_ok) {

@@ -45,7 +45,10 @@ inline bool make_row_gather_map(CUtensorMap *map, const void *base, int64_t rows
 #ifdef __CUDACC__
 __device__ inline uint32_t tm_smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-// Bounded wait for the phase with the given parity of an mbarrier that only the calling warp uses.
+// Bounded wait for the phase with the given parity of an mbarrier that only the calling warp uses.  Each try may
+// suspend the thread for up to kTmWaitHintNs inside the hardware, so a warp that waits for its rows leaves the issue
+// slots to the others instead of polling.
+constexpr uint32_t kTmWaitHintNs = 2000;
 __device__ inline bool tm_mbar_wait(uint64_t *bar, uint32_t parity)
 {
     const uint32_t addr = tm_smem_u32(bar);
@@ -54,11 +57,11 @@ __device__ inline bool tm_mbar_wait(uint64_t *bar, uint32_t parity)
         asm volatile(
             "{\n"
             ".reg .pred p;\n"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n"
             "selp.u32 %0, 1, 0, p;\n"
             "}\n"
             : "=r"(done)
-            : "r"(addr), "r"(parity)
+            : "r"(addr), "r"(parity), "r"(kTmWaitHintNs)
             : "memory");
         if (done) return true;
     }
