@@ -1008,8 +1008,8 @@ inline bool seg_general_only()
 inline bool seg_stream_off()
 {
     static const bool v = []() {
-        const char *e = getenv("E2EGREC_NO_STREAM_GATHER");
-        return e && *e && e[0] != '0';
+        const char *e = getenv("E2EGREC_NO_STREAM_GATHER"), *t = getenv("E2EGREC_NO_STREAM_TRANSPOSED");
+        return (e && *e && e[0] != '0') || (t && *t && t[0] != '0');
     }();
     return v;
 }
