@@ -61,8 +61,8 @@ def test_blocks_with_capacity_for_millions_of_entries():
 
 def test_wide_rows_with_capacity_for_millions_of_entries():
     """256-value bf16 rows in block buffers sized for 40 000 seeds on the 500 k-node graph (outer block: 5 M entries of
-    capacity): the launch
-    shapes of the largest workload, where the aggregation streams its rows through shared memory with the TMA unit."""
+    capacity): the launch shapes of the largest workload, where the aggregation kernels stream their rows through shared
+    memory with the TMA unit."""
     import dataclasses
     w = dataclasses.replace(S.WORKLOADS["medium"], dim=256, hidden=256, batch=512)
     case = Case(w, step=2)
@@ -156,6 +156,27 @@ def test_empty_batch():
     gpu = case.run_gpu()
     for b in gpu["blocks"]:
         assert b["n_dst"] == 0 and b["n_src"] == 0 and b["n_edges"] == 0 and b["status"] == 0
+
+
+def test_empty_and_tiny_batches_in_buffers_for_millions_of_entries():
+    """No seed at all, and three seeds, with 256-value bf16 rows in buffers sized for 40 000 seeds: the kernels that stream
+    their rows through shared memory see warps without any destination, and a stream of a handful of entries."""
+    import dataclasses
+    w = dataclasses.replace(S.WORKLOADS["medium"], dim=256, hidden=256, batch=3)
+    graph = S.build_graph(w)[:2]
+    empty = Case(w, step=0, seeds=np.zeros(0, np.int32), graph=graph)
+    dH0 = empty.upstream_grad(0, w.hidden)
+    gpu = empty.run_gpu(dH0, cap_seeds=40000)
+    assert gpu["blocks_obj"].caps[-1][2] >= 1 << 20
+    for b in gpu["blocks"]:
+        assert b["n_dst"] == 0 and b["n_src"] == 0 and b["n_edges"] == 0 and b["status"] == 0
+    assert all(float(np.abs(g).max()) == 0.0 for g in gpu["dWs"])
+    case = Case(w, step=5, graph=graph)
+    dH = case.upstream_grad(case.seeds.size, w.hidden)
+    ora = case.run_oracle(dH)
+    gpu = case.run_gpu(dH, cap_seeds=40000)
+    assert_blocks_equal(gpu["blocks"], ora["blocks"])
+    _check_float(case, gpu, ora)
 
 
 def test_out_of_range_seed_sets_status_and_does_not_fault():
