@@ -132,9 +132,10 @@ __device__ __forceinline__ void seg_store_row(const SegOut<T> &o, int32_t seg, f
     for (int q = 0; q < CPL; ++q) {
         const int ch = c + q * LPR;
         if (ch < n_chunks) {
+            // the store rounds to the storage type, once; a masked element is zero before and after that rounding alike
             float r[E];
 #pragma unroll
-            for (int e = 0; e < E; ++e) r[e] = to_float<T>(from_float<T>(acc[q][e] * inv));   // inv = 1 without mean / scale
+            for (int e = 0; e < E; ++e) r[e] = acc[q][e] * inv;                                 // inv = 1 without mean / scale
             if (kExtra == 2 && o.mask) {
                 float m[E];
                 Chunk<T>::unpack(mrow[q], m);
@@ -705,7 +706,8 @@ seg_run_block_kernel(const __grid_constant__ CUtensorMap in_map, const T *__rest
                             if (kMask) cur_mask[0] = mv_cur[u];
                         }
                         float x[E];
-                        Chunk<T>::unpack(stream_ok ? *reinterpret_cast<const uint4 *>(rows + u * kStreamRowBytes) : make_uint4(0, 0, 0, 0), x);
+                        // (after a wait that ran out the slot holds stale rows: the launch is reported as failed)
+                        Chunk<T>::unpack(*reinterpret_cast<const uint4 *>(rows + u * kStreamRowBytes), x);
 #pragma unroll
                         for (int e = 0; e < E; e += 2) add2(acc[0][e], acc[0][e + 1], x[e], x[e + 1]);
                     }
