@@ -130,7 +130,8 @@ sage_aggregate_stream_kernel(const __grid_constant__ CUtensorMap map, const int3
         }
         ++i;
         beg_i = end_i;
-        if (i < j1) {
+        end_i = 0x7fffffff;                         // beyond the last destination, or after a wait that ran out: no entry closes anything
+        if (i < j1 && ok) {
             const int32_t o2 = (int32_t)(i - j0);
             if ((o2 >> 5) > dst_win) {
                 ++dst_win;
@@ -154,16 +155,19 @@ sage_aggregate_stream_kernel(const __grid_constant__ CUtensorMap map, const int3
         ok = __all_sync(full, tm_mbar_wait(&bar_n[warp][slot], (uint32_t)(q / kNbrSlots) & 1u));
         if (!ok) break;
         const uint8_t *rows = ring_n + (size_t)slot * kSlotBytes + lane * 16;
+        const int32_t k0 = b_w + 4 * q;
+        auto add_row = [&](int r) {
+            while (k0 + r >= end_i) finalize();     // the entry belongs to a later destination: close the ones before it
+            float x[8];
+            Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4 *>(rows + r * kRowBytes), x);
 #pragma unroll
-        for (int r = 0; r < 4; ++r) {
-            const int32_t k = b_w + 4 * q + r;
-            if (k < e_w) {
-                while (k >= end_i && i < j1 && ok) finalize();
-                float x[8];
-                Chunk<__nv_bfloat16>::unpack(*reinterpret_cast<const uint4 *>(rows + r * kRowBytes), x);
+            for (int kk = 0; kk < 8; kk += 2) add2(acc[kk], acc[kk + 1], x[kk], x[kk + 1]);
+        };
+        if (k0 + 4 <= e_w) {
 #pragma unroll
-                for (int kk = 0; kk < 8; kk += 2) add2(acc[kk], acc[kk + 1], x[kk], x[kk + 1]);
-            }
+            for (int r = 0; r < 4; ++r) add_row(r);
+        } else {                                    // the stream's last group: rows beyond its end repeat the last id
+            for (int r = 0; k0 + r < e_w; ++r) add_row(r);
         }
         __syncwarp();                               // every lane has read the slot
         if (q + kNbrSlots < n_groups) issue_nbr(q + kNbrSlots);
