@@ -46,8 +46,8 @@ def test_medium_small_bf16_sample_forward_backward():
 
 def test_blocks_with_capacity_for_millions_of_entries():
     """Block buffers sized for 40 000 seeds on the 500 k-node graph (outer block: 5 M entries of capacity) while the batch
-    has 512: the library then cuts the transposed aggregation into runs of 128 entries and stages the outer block's
-    rows through its shared-memory ring, the launch shapes of the largest workload."""
+    has 512: the library then cuts the transposed aggregation into runs of 128 entries, the run length of the largest
+    workload (256-byte rows: no streaming through shared memory, which the next test covers)."""
     import dataclasses
     w = dataclasses.replace(S.WORKLOADS["medium"], batch=512)
     case = Case(w, step=2)
